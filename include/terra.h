@@ -1,0 +1,121 @@
+/*
+ * terra.h -- C ABI of the B200 (sm_100a) shifted-window attention block.
+ *
+ * The block is the Swin-style window attention of the TERRA forecaster (paper Section IV-A:
+ * W-MSA / SW-MSA inside each Transformer block), fed from the spatially contiguous lat-lon token
+ * grid that the convolutional sampling modules produce and returned to it (Section IV-D: the token
+ * route converts between the contiguous layout and the window-major layout using the global token
+ * coordinate (u, v), window (floor(u/w), floor(v/w)) and offset (u mod w, v mod w); the shift route
+ * changes the token coordinate, and the backward pass applies the inverse mapping).
+ *
+ * Conventions fixed by this library where the paper is silent:
+ *   - the shift is a cyclic roll by -shift: token (u, v) sits at u' = (u - shift_h) mod H,
+ *     v' = (v - shift_w) mod W, and windows tile the (u', v') frame, row-major (Section V-A);
+ *   - the last window row / column is truncated when w does not divide H / W (no padding tokens);
+ *   - on a non-periodic axis tokens that wrapped across the edge (u < shift_h, v < shift_w) only
+ *     attend to each other (shift mask); a periodic axis has no mask;
+ *   - scores are scale * <q, k> + T[(a_q - a_k + w - 1) * (2w - 1) + (b_q - b_k + w - 1), head]
+ *     with (a, b) the in-window offsets; masked pairs get probability exactly zero.
+ *
+ * All pointers are DEVICE pointers unless stated otherwise, 16-byte aligned, owned by the caller.
+ * Calls enqueue work on `stream` (a cudaStream_t passed as void*; NULL = the legacy default stream)
+ * and return without synchronising.  No call allocates device memory; scratch comes from the
+ * caller's workspace.  Every function returns a terra_status; nothing throws, nothing falls back to
+ * the CPU.  Outputs must not alias inputs.
+ */
+#ifndef TERRA_H_
+#define TERRA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    TERRA_OK = 0,
+    TERRA_ERR_INVALID_ARG = 1,   /* null pointer, non-positive size, element count out of range   */
+    TERRA_ERR_UNSUPPORTED = 2,   /* head_dim not in {32, 64}, window too large, not an sm_100 GPU */
+    TERRA_ERR_ALIGNMENT = 3,     /* a pointer is not 16-byte aligned                              */
+    TERRA_ERR_WORKSPACE = 4,     /* workspace NULL or smaller than terra_swin_workspace_bytes     */
+    TERRA_ERR_CUDA = 5           /* a CUDA call failed; text via terra_last_cuda_error            */
+} terra_status;
+
+/* Problem statement: token grid, window, heads (paper Table I symbols; H, W here are H_T, W_T). */
+typedef struct {
+    int32_t B;                      /* batch (samples / rollout steps), >= 1                      */
+    int32_t H, W;                   /* token grid: latitude rows x longitude columns              */
+    int32_t heads, head_dim;        /* attention heads; per-head width, 32 or 64                  */
+    int32_t window;                 /* w: square window side, 1 <= w <= 32                        */
+    int32_t shift_h, shift_w;       /* >= 0, taken mod H and mod W                                */
+    int32_t periodic_h, periodic_w; /* 0 / 1; the paper's grids: latitude 0, longitude 1          */
+    float scale;                    /* score scale; <= 0 selects 1/sqrt(head_dim)                 */
+} terra_swin_desc;
+
+/*
+ * Sizes of the route arrays (Section IV-D window grid: M_h = ceil(H/w), M_w = ceil(W/w)).
+ * Host-only.  Any output may be NULL.
+ *   n_tokens = H * W, n_windows = M_h * M_w, max_window_tokens = min(w, H) * min(w, W).
+ */
+int terra_route_sizes(const terra_swin_desc* desc, int64_t* n_tokens, int32_t* n_windows,
+                      int32_t* max_window_tokens);
+
+/*
+ * Token route (Section IV-D, with the shift route folded in): the integer map between the
+ * contiguous grid and the window-major layout, for one sample (all samples share it).
+ *   win_offsets [n_windows + 1]  first slot of window g = wr * M_w + wc; last entry = H * W
+ *   perm        [H * W]          perm[slot] = u * W + v, the grid token stored in that slot; slots
+ *                                inside a window run row-major over the window's true extent
+ *   inv_perm    [H * W]          inv_perm[u * W + v] = slot
+ *   pos         [H * W]          pos[slot] = a * w + b, the in-window offset
+ *   label       [H * W]          label[slot] = 2 * [lat non-periodic and u < shift_h]
+ *                                              + [lon non-periodic and v < shift_w]
+ * int32 device arrays; any may be NULL to skip it.  Exact integer work.
+ */
+int terra_window_route(const terra_swin_desc* desc, int32_t* perm, int32_t* inv_perm,
+                       int32_t* win_offsets, int32_t* pos, int32_t* label, void* stream);
+
+/* Scratch bytes the forward (backward = 0) or backward (backward = 1) call needs.  Host-only. */
+int terra_swin_workspace_bytes(const terra_swin_desc* desc, int backward, size_t* bytes);
+
+/*
+ * Forward shifted-window attention (Section IV-A W-MSA / SW-MSA; route + attention + inverse route
+ * in one pass).
+ *   q, k, v      bf16 [B, H, W, heads, head_dim], innermost contiguous (the contiguous grid layout)
+ *   bias_table   fp32 [(2w-1)^2, heads]
+ *   o            bf16 [B, H, W, heads, head_dim]   attention output at the token's grid position
+ *   lse          fp32 [B, H, W, heads]             natural-log sum-exp of each score row (for bwd)
+ *   workspace    >= terra_swin_workspace_bytes(desc, 0) bytes (may be NULL when that is 0)
+ */
+int terra_swin_attn_fwd(const terra_swin_desc* desc, const void* q, const void* k, const void* v,
+                        const float* bias_table, void* o, float* lse,
+                        void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Backward of terra_swin_attn_fwd (Section IV-D: gradients return through the inverse routes).
+ *   q, k, v, o, lse   as given to / produced by the forward call
+ *   d_o               bf16 [B, H, W, heads, head_dim]   upstream gradient
+ *   dq, dk, dv        bf16 [B, H, W, heads, head_dim]   overwritten
+ *   dbias             fp32 [(2w-1)^2, heads]            overwritten (summed over batch and windows;
+ *                                                       the summation order is not fixed)
+ *   workspace         >= terra_swin_workspace_bytes(desc, 1) bytes
+ */
+int terra_swin_attn_bwd(const terra_swin_desc* desc, const void* q, const void* k, const void* v,
+                        const float* bias_table, const void* o, const float* lse, const void* d_o,
+                        void* dq, void* dk, void* dv, float* dbias,
+                        void* workspace, size_t workspace_bytes, void* stream);
+
+/* Static text for a terra_status.  Host-only. */
+const char* terra_strerror(int status);
+
+/* Text of the last CUDA error this library saw on the calling thread ("" if none).  Host-only. */
+const char* terra_last_cuda_error(void);
+
+/* Number of kernels the library has launched in this process (monotonic).  Host-only. */
+int64_t terra_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TERRA_H_ */

@@ -1,0 +1,10 @@
+"""B200 (sm_100a) shifted-window attention block of the TERRA forecaster.
+
+The product is the C-ABI CUDA library (include/terra.h, csrc/); this package builds it
+in-tree and exposes a thin ctypes binding with the same names.  Importing the package
+does not load the library; the first call does, and raises if it is missing.
+"""
+from .binding import (TerraError, launch_count, load_library, make_desc, terra_route_sizes,  # noqa: F401
+                      terra_swin_attn_bwd, terra_swin_attn_fwd, terra_swin_desc, terra_swin_workspace_bytes,
+                      terra_window_route)
+from .workloads import CONFIGS, SwinConfig, make_inputs  # noqa: F401

@@ -1,0 +1,165 @@
+"""Thin Python binding of the C ABI declared in include/terra.h.
+
+Argument marshalling only: tensors must already live on the GPU; every step of the path
+(route, gather, attention, scatter) runs in the library's kernels.  There is no CPU
+fallback: if the shared library is missing or no CUDA device is present, calls raise.
+PyTorch is used for device memory and streams.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+from .build import LIB_PATH
+
+TERRA_OK = 0
+EXPORTS = ("terra_route_sizes", "terra_window_route", "terra_swin_workspace_bytes", "terra_swin_attn_fwd",
+           "terra_swin_attn_bwd", "terra_strerror", "terra_last_cuda_error", "terra_launch_count")
+
+
+class TerraError(RuntimeError):
+    def __init__(self, status: int, text: str):
+        super().__init__(f"terra status {status}: {text}")
+        self.status = status
+
+
+class terra_swin_desc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("B", "H", "W", "heads", "head_dim", "window", "shift_h", "shift_w", "periodic_h", "periodic_w")] + \
+               [("scale", ctypes.c_float)]
+
+
+_lib = None
+
+
+def load_library(path: str | None = None) -> ctypes.CDLL:
+    """dlopen the CUDA library.  Raises if it has not been built: there is no other path."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = path or LIB_PATH
+    if not os.path.exists(p):
+        raise FileNotFoundError(f"{p} not found: build it with `python -m paper_2608_15211_b200.build` "
+                                "(the library has no CPU fallback)")
+    lib = ctypes.CDLL(p)
+    vp, i32p, i64p = ctypes.c_void_p, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int64)
+    dp = ctypes.POINTER(terra_swin_desc)
+    lib.terra_route_sizes.argtypes = [dp, i64p, i32p, i32p]
+    lib.terra_window_route.argtypes = [dp, vp, vp, vp, vp, vp, vp]
+    lib.terra_swin_workspace_bytes.argtypes = [dp, ctypes.c_int, ctypes.POINTER(ctypes.c_size_t)]
+    lib.terra_swin_attn_fwd.argtypes = [dp] + [vp] * 6 + [vp, ctypes.c_size_t, vp]
+    lib.terra_swin_attn_bwd.argtypes = [dp] + [vp] * 11 + [vp, ctypes.c_size_t, vp]
+    for n in ("terra_route_sizes", "terra_window_route", "terra_swin_workspace_bytes", "terra_swin_attn_fwd",
+              "terra_swin_attn_bwd"):
+        getattr(lib, n).restype = ctypes.c_int
+    lib.terra_strerror.argtypes = [ctypes.c_int]
+    lib.terra_strerror.restype = ctypes.c_char_p
+    lib.terra_last_cuda_error.restype = ctypes.c_char_p
+    lib.terra_launch_count.restype = ctypes.c_int64
+    if path is None:
+        _lib = lib
+    return lib
+
+
+def make_desc(cfg, scale: float = 0.0) -> terra_swin_desc:
+    """Descriptor from any object with B, H, W, heads, head_dim, window, shift_*, periodic_* fields."""
+    return terra_swin_desc(cfg.B, cfg.H, cfg.W, cfg.heads, cfg.head_dim, cfg.window, cfg.shift_h, cfg.shift_w,
+                           cfg.periodic_h, cfg.periodic_w, float(scale))
+
+
+def _check(status: int) -> None:
+    if status != TERRA_OK:
+        lib = load_library()
+        text = lib.terra_strerror(status).decode()
+        extra = lib.terra_last_cuda_error().decode()
+        raise TerraError(status, text + (f" [{extra}]" if extra and status == 5 else ""))
+
+
+def _ptr(t) -> ctypes.c_void_p:
+    if t is None:
+        return ctypes.c_void_p(0)
+    if not t.is_cuda:
+        raise ValueError("terra: tensors must be CUDA tensors (the library has no CPU path)")
+    if not t.is_contiguous():
+        raise ValueError("terra: tensors must be contiguous")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream() -> ctypes.c_void_p:
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def launch_count() -> int:
+    return int(load_library().terra_launch_count())
+
+
+def terra_route_sizes(desc: terra_swin_desc):
+    nt, nw, mx = ctypes.c_int64(), ctypes.c_int32(), ctypes.c_int32()
+    _check(load_library().terra_route_sizes(ctypes.byref(desc), ctypes.byref(nt), ctypes.byref(nw), ctypes.byref(mx)))
+    return nt.value, nw.value, mx.value
+
+
+def terra_window_route(desc: terra_swin_desc, device="cuda") -> dict:
+    """Allocates the five int32 route arrays on `device` and fills them."""
+    nt, nw, _ = terra_route_sizes(desc)
+    out = {k: torch.empty(nt, dtype=torch.int32, device=device) for k in ("perm", "inv_perm", "pos", "label")}
+    out["win_offsets"] = torch.empty(nw + 1, dtype=torch.int32, device=device)
+    _check(load_library().terra_window_route(ctypes.byref(desc), _ptr(out["perm"]), _ptr(out["inv_perm"]),
+                                             _ptr(out["win_offsets"]), _ptr(out["pos"]), _ptr(out["label"]), _stream()))
+    return out
+
+
+def terra_swin_workspace_bytes(desc: terra_swin_desc, backward: bool) -> int:
+    n = ctypes.c_size_t()
+    _check(load_library().terra_swin_workspace_bytes(ctypes.byref(desc), int(backward), ctypes.byref(n)))
+    return int(n.value)
+
+
+def _expect(t, dtype, numel, name):
+    if t.dtype != dtype or t.numel() != numel:
+        raise ValueError(f"terra: {name} must be {dtype} with {numel} elements, got {t.dtype} x {t.numel()}")
+
+
+def terra_swin_attn_fwd(desc, q, k, v, bias_table, o=None, lse=None, workspace=None):
+    """Forward.  q, k, v bf16 [B, H, W, heads, head_dim]; bias_table fp32 [(2w-1)^2, heads].
+    Returns (o bf16 like q, lse fp32 [B, H, W, heads]); pass o / lse / workspace to reuse buffers."""
+    n = desc.B * desc.H * desc.W * desc.heads
+    for name, t in (("q", q), ("k", k), ("v", v)):
+        _expect(t, torch.bfloat16, n * desc.head_dim, name)
+    _expect(bias_table, torch.float32, (2 * desc.window - 1) ** 2 * desc.heads, "bias_table")
+    if o is None:
+        o = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty((desc.B, desc.H, desc.W, desc.heads), dtype=torch.float32, device=q.device)
+    _expect(o, torch.bfloat16, n * desc.head_dim, "o")
+    _expect(lse, torch.float32, n, "lse")
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(load_library().terra_swin_attn_fwd(ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(v), _ptr(bias_table),
+                                              _ptr(o), _ptr(lse), _ptr(workspace), ws_bytes, _stream()))
+    return o, lse
+
+
+def terra_swin_attn_bwd(desc, q, k, v, bias_table, o, lse, d_o, dq=None, dk=None, dv=None, dbias=None,
+                        workspace=None):
+    """Backward.  Returns (dq, dk, dv bf16 like q, dbias fp32 like bias_table)."""
+    n = desc.B * desc.H * desc.W * desc.heads
+    for name, t in (("q", q), ("k", k), ("v", v), ("o", o), ("d_o", d_o)):
+        _expect(t, torch.bfloat16, n * desc.head_dim, name)
+    _expect(lse, torch.float32, n, "lse")
+    _expect(bias_table, torch.float32, (2 * desc.window - 1) ** 2 * desc.heads, "bias_table")
+    dq = torch.empty_like(q) if dq is None else dq
+    dk = torch.empty_like(q) if dk is None else dk
+    dv = torch.empty_like(q) if dv is None else dv
+    dbias = torch.empty_like(bias_table) if dbias is None else dbias
+    for name, t in (("dq", dq), ("dk", dk), ("dv", dv)):
+        _expect(t, torch.bfloat16, n * desc.head_dim, name)
+    _expect(dbias, torch.float32, bias_table.numel(), "dbias")
+    if workspace is None:
+        workspace = torch.empty(terra_swin_workspace_bytes(desc, True), dtype=torch.uint8, device=q.device)
+    ws_bytes = workspace.numel() * workspace.element_size()
+    _check(load_library().terra_swin_attn_bwd(ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(v), _ptr(bias_table),
+                                              _ptr(o), _ptr(lse), _ptr(d_o), _ptr(dq), _ptr(dk), _ptr(dv),
+                                              _ptr(dbias), _ptr(workspace), ws_bytes, _stream()))
+    return dq, dk, dv, dbias

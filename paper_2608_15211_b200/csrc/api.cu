@@ -1,0 +1,168 @@
+// C ABI of the shifted-window attention library: argument checks, geometry, launches.
+#include <atomic>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+
+#include "../../include/terra.h"
+#include "swin_kernels.h"
+
+namespace terra {
+
+static std::atomic<long long> g_launches{0};
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+
+static thread_local char g_cuda_error[256] = "";
+
+static int cuda_fail(cudaError_t e, const char* where) {
+    std::snprintf(g_cuda_error, sizeof g_cuda_error, "%s: %s", where, cudaGetErrorString(e));
+    return TERRA_ERR_CUDA;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Checks the descriptor and resolves the window geometry.  Host arithmetic only.
+static int make_geo(const terra_swin_desc* d, bool for_attention, Geo* out) {
+    if (!d) return TERRA_ERR_INVALID_ARG;
+    if (d->B <= 0 || d->H <= 0 || d->W <= 0 || d->heads <= 0 || d->head_dim <= 0 || d->window <= 0 ||
+        d->shift_h < 0 || d->shift_w < 0)
+        return TERRA_ERR_INVALID_ARG;
+    if ((long long)d->H * d->W > 0x7fffffffLL) return TERRA_ERR_INVALID_ARG;             // token index is int32
+    if ((long long)d->B * d->H * d->W * d->heads > (1LL << 40)) return TERRA_ERR_INVALID_ARG;
+    if (for_attention) {
+        if (d->head_dim != 32 && d->head_dim != 64) return TERRA_ERR_UNSUPPORTED;
+        if (d->window > 32) return TERRA_ERR_UNSUPPORTED;
+        if (!(d->scale == d->scale) || std::isinf(d->scale)) return TERRA_ERR_INVALID_ARG;
+    }
+    Geo g;
+    g.B = d->B; g.H = d->H; g.W = d->W;
+    g.heads = d->heads; g.d = d->head_dim; g.w = d->window;
+    g.sh = d->shift_h % d->H; g.sw = d->shift_w % d->W;
+    g.ph = d->periodic_h != 0; g.pw = d->periodic_w != 0;
+    g.Mh = (d->H + d->window - 1) / d->window;
+    g.Mw = (d->W + d->window - 1) / d->window;
+    g.nmax = (d->window < d->H ? d->window : d->H) * (d->window < d->W ? d->window : d->W);
+    const float scale = d->scale > 0.f ? d->scale : 1.0f / std::sqrt((float)d->head_dim);
+    g.scale_log2e = scale * kLog2e;
+    *out = g;
+    return TERRA_OK;
+}
+
+static int device_props(int* sm_count) {
+    static thread_local int cached_dev = -1, cached_sms = 0, cached_major = 0;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    if (dev != cached_dev) {
+        int sms = 0, major = 0;
+        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
+        e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
+        cached_dev = dev; cached_sms = sms; cached_major = major;
+    }
+    if (cached_major != 10) return TERRA_ERR_UNSUPPORTED;
+    *sm_count = cached_sms;
+    return TERRA_OK;
+}
+
+static size_t delta_bytes(const Geo& g) {
+    return align_up(sizeof(float) * (size_t)g.B * g.H * g.W * g.heads, 256);
+}
+
+}  // namespace terra
+
+using namespace terra;
+
+extern "C" {
+
+int terra_route_sizes(const terra_swin_desc* desc, int64_t* n_tokens, int32_t* n_windows,
+                      int32_t* max_window_tokens) {
+    Geo g;
+    int rc = make_geo(desc, false, &g);
+    if (rc) return rc;
+    if (n_tokens) *n_tokens = (int64_t)g.H * g.W;
+    if (n_windows) *n_windows = g.Mh * g.Mw;
+    if (max_window_tokens) *max_window_tokens = g.nmax;
+    return TERRA_OK;
+}
+
+int terra_window_route(const terra_swin_desc* desc, int32_t* perm, int32_t* inv_perm,
+                       int32_t* win_offsets, int32_t* pos, int32_t* label, void* stream) {
+    Geo g;
+    int rc = make_geo(desc, false, &g);
+    if (rc) return rc;
+    cudaError_t e = launch_route(g, perm, inv_perm, win_offsets, pos, label, (cudaStream_t)stream);
+    return e == cudaSuccess ? TERRA_OK : cuda_fail(e, "terra_window_route");
+}
+
+int terra_swin_workspace_bytes(const terra_swin_desc* desc, int backward, size_t* bytes) {
+    Geo g;
+    int rc = make_geo(desc, true, &g);
+    if (rc) return rc;
+    if (!bytes) return TERRA_ERR_INVALID_ARG;
+    *bytes = backward ? delta_bytes(g) : 0;
+    return TERRA_OK;
+}
+
+int terra_swin_attn_fwd(const terra_swin_desc* desc, const void* q, const void* k, const void* v,
+                        const float* bias_table, void* o, float* lse,
+                        void* workspace, size_t workspace_bytes, void* stream) {
+    (void)workspace; (void)workspace_bytes;
+    Geo g;
+    int rc = make_geo(desc, true, &g);
+    if (rc) return rc;
+    if (!q || !k || !v || !bias_table || !o || !lse) return TERRA_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(bias_table) || !aligned16(lse))
+        return TERRA_ERR_ALIGNMENT;
+    int sms = 0;
+    rc = device_props(&sms);
+    if (rc) return rc;
+    cudaError_t e = launch_fwd_mma(g, q, k, v, bias_table, o, lse, (cudaStream_t)stream);
+    return e == cudaSuccess ? TERRA_OK : cuda_fail(e, "terra_swin_attn_fwd");
+}
+
+int terra_swin_attn_bwd(const terra_swin_desc* desc, const void* q, const void* k, const void* v,
+                        const float* bias_table, const void* o, const float* lse, const void* d_o,
+                        void* dq, void* dk, void* dv, float* dbias,
+                        void* workspace, size_t workspace_bytes, void* stream) {
+    Geo g;
+    int rc = make_geo(desc, true, &g);
+    if (rc) return rc;
+    if (!q || !k || !v || !bias_table || !o || !lse || !d_o || !dq || !dk || !dv || !dbias)
+        return TERRA_ERR_INVALID_ARG;
+    const void* ptrs[] = {q, k, v, bias_table, o, lse, d_o, dq, dk, dv, dbias};
+    for (const void* p : ptrs)
+        if (!aligned16(p)) return TERRA_ERR_ALIGNMENT;
+    if (!workspace || workspace_bytes < delta_bytes(g)) return TERRA_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return TERRA_ERR_ALIGNMENT;
+    int sms = 0;
+    rc = device_props(&sms);
+    if (rc) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    float* delta = reinterpret_cast<float*>(workspace);
+    cudaError_t e = launch_bwd_delta(g, o, d_o, delta, st);
+    if (e != cudaSuccess) return cuda_fail(e, "terra_swin_attn_bwd (delta)");
+    e = launch_bwd_mma(g, q, k, v, bias_table, lse, delta, d_o, dq, dk, dv, dbias, sms, st);
+    return e == cudaSuccess ? TERRA_OK : cuda_fail(e, "terra_swin_attn_bwd");
+}
+
+const char* terra_strerror(int status) {
+    switch (status) {
+        case TERRA_OK: return "ok";
+        case TERRA_ERR_INVALID_ARG: return "invalid argument (null pointer, non-positive size, or size out of range)";
+        case TERRA_ERR_UNSUPPORTED: return "unsupported configuration (head_dim must be 32 or 64, window <= 32, GPU must be sm_100)";
+        case TERRA_ERR_ALIGNMENT: return "pointer is not 16-byte aligned";
+        case TERRA_ERR_WORKSPACE: return "workspace missing or too small (see terra_swin_workspace_bytes)";
+        case TERRA_ERR_CUDA: return "CUDA error (see terra_last_cuda_error)";
+        default: return "unknown status";
+    }
+}
+
+const char* terra_last_cuda_error(void) { return g_cuda_error; }
+
+int64_t terra_launch_count(void) { return (int64_t)g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

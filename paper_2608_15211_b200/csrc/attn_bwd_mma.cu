@@ -1,0 +1,361 @@
+// Backward shifted-window attention, register-tile path (warp-level mma.sync).
+//
+// Three launches: (1) delta = rowsum(dO * O); (2) key-tile CTAs produce dK and dV; (3) query-tile
+// CTAs produce dQ and the relative-position-bias gradient.  (2) and (3) are one kernel template: a
+// CTA owns 64 rows of one side of the window (keys or queries), streams the other side through
+// shared memory in 64-row blocks, recomputes P from the saved log-sum-exp and forms
+// dS = P * (dP - delta).  No atomics touch dQ / dK / dV, so those are reproducible run to run; the
+// bias gradient is summed per CTA in shared memory (CTAs are persistent and bound to one head) and
+// flushed once with global atomics.
+#include "swin_common.cuh"
+#include "swin_kernels.h"
+
+namespace terra {
+
+namespace {
+
+constexpr int BM = 64;
+constexpr int BN = 64;
+constexpr int NTHREADS = 128;
+
+template <int D>
+__device__ __forceinline__ void load_rows(unsigned char* s_tile, const __nv_bfloat16* base, const int* s_tok,
+                                          int slot0, size_t sample_off, int heads, int head, int tid) {
+    constexpr int CPR = D / 8;
+    for (int idx = tid; idx < BN * CPR; idx += NTHREADS) {
+        int row = idx / CPR, chunk = idx - row * CPR;
+        int tok = s_tok[slot0 + row];
+        const __nv_bfloat16* src = base;
+        int bytes = 0;
+        if (tok >= 0) {
+            src = base + ((sample_off + (size_t)tok) * heads + head) * D + chunk * 8;
+            bytes = 16;
+        }
+        cp_async16(smem_u32(s_tile + tile_off<D>(row, chunk)), src, bytes);
+    }
+}
+
+// acc (16 x 64 per warp) = own rows (fragments in registers) x streamed block^T
+template <int D>
+__device__ __forceinline__ void rows_times_block_t(float (&acc)[BN / 8][4], const uint32_t (&af)[D / 16][4],
+                                                   const unsigned char* blk, int lane) {
+#pragma unroll
+    for (int i = 0; i < BN / 8; ++i)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) acc[i][e] = 0.f;
+#pragma unroll
+    for (int ks = 0; ks < D / 16; ++ks) {
+#pragma unroll
+        for (int np = 0; np < BN / 16; ++np) {
+            uint32_t bf[4];
+            int r = np * 16 + (lane & 7) + (lane >> 4) * 8;
+            ldmatrix_x4(bf, smem_u32(blk + tile_off<D>(r, 2 * ks + ((lane >> 3) & 1))));
+            mma_bf16(acc[2 * np], af[ks], bf[0], bf[1]);
+            mma_bf16(acc[2 * np + 1], af[ks], bf[2], bf[3]);
+        }
+    }
+}
+
+// out (16 x D per warp) += coef (16 x 64, fp32 fragments, rounded to bf16) x streamed block (64 x D)
+template <int D>
+__device__ __forceinline__ void coef_times_block(float (&out)[D / 8][4], const float (&coef)[BN / 8][4],
+                                                 const unsigned char* blk, int lane) {
+#pragma unroll
+    for (int ks = 0; ks < BN / 16; ++ks) {
+        uint32_t pf[4];
+        pf[0] = pack_bf16(coef[2 * ks][0], coef[2 * ks][1]);
+        pf[1] = pack_bf16(coef[2 * ks][2], coef[2 * ks][3]);
+        pf[2] = pack_bf16(coef[2 * ks + 1][0], coef[2 * ks + 1][1]);
+        pf[3] = pack_bf16(coef[2 * ks + 1][2], coef[2 * ks + 1][3]);
+#pragma unroll
+        for (int dp = 0; dp < D / 16; ++dp) {
+            uint32_t bf[4];
+            int r = ks * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+            ldmatrix_x4_trans(bf, smem_u32(blk + tile_off<D>(r, 2 * dp + (lane >> 4))));
+            mma_bf16(out[2 * dp], pf, bf[0], bf[1]);
+            mma_bf16(out[2 * dp + 1], pf, bf[2], bf[3]);
+        }
+    }
+}
+
+template <int D>
+__device__ __forceinline__ void stage_rows(unsigned char* tile, const float (&acc)[D / 8][4], float mul,
+                                           int warp, int gq, int tq) {
+#pragma unroll
+    for (int i = 0; i < D / 8; ++i) {
+        int lr = warp * 16 + gq;
+        *reinterpret_cast<uint32_t*>(tile + tile_off<D>(lr, i) + tq * 4) = pack_bf16(acc[i][0] * mul, acc[i][1] * mul);
+        *reinterpret_cast<uint32_t*>(tile + tile_off<D>(lr + 8, i) + tq * 4) = pack_bf16(acc[i][2] * mul, acc[i][3] * mul);
+    }
+}
+
+template <int D>
+__device__ __forceinline__ void scatter_rows(const unsigned char* tile, __nv_bfloat16* dst, const int* s_tok, int slot0,
+                                             int n, size_t sample_off, int heads, int head, int tid) {
+    constexpr int CPR = D / 8;
+    for (int idx = tid; idx < BM * CPR; idx += NTHREADS) {
+        int row = idx / CPR, chunk = idx - row * CPR;
+        int slot = slot0 + row;
+        if (slot < n) {
+            uint4 val = *reinterpret_cast<const uint4*>(tile + tile_off<D>(row, chunk));
+            *reinterpret_cast<uint4*>(dst + ((sample_off + (size_t)s_tok[slot]) * heads + head) * D + chunk * 8) = val;
+        }
+    }
+}
+
+// KV = true : CTA owns 64 keys   (own tiles K, V;  streams Q, dO) -> dK, dV
+// KV = false: CTA owns 64 queries (own tiles Q, dO; streams K, V) -> dQ, dBias
+template <int D, bool KV>
+__global__ void __launch_bounds__(NTHREADS)
+swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
+                    const __nv_bfloat16* __restrict__ v, const __nv_bfloat16* __restrict__ d_o,
+                    const float* __restrict__ bias, const float* __restrict__ lse, const float* __restrict__ delta,
+                    __nv_bfloat16* __restrict__ out1, __nv_bfloat16* __restrict__ out2, float* __restrict__ dbias,
+                    int tiles, int ctas_per_head) {
+    constexpr int KS = D / 16;
+    constexpr int DT = D / 8;
+    constexpr int TILE_BYTES = BN * D * 2;
+    extern __shared__ __align__(128) unsigned char smem[];
+
+    const int nbias = (2 * g.w - 1) * (2 * g.w - 1);
+    const int npad_max = ((g.nmax + BN - 1) / BN) * BN;
+    int* s_tok = reinterpret_cast<int*>(smem);
+    int* s_meta = s_tok + npad_max;
+    float* s_lse = reinterpret_cast<float*>(s_meta + npad_max);
+    float* s_delta = s_lse + npad_max;
+    float* s_bias = s_delta + npad_max;
+    float* s_dbias = s_bias + nbias;
+    unsigned char* s_r1 = smem + (((size_t)npad_max * 16 + (size_t)nbias * 8 + 127) / 128) * 128;
+    unsigned char* s_r2 = s_r1 + TILE_BYTES;
+    unsigned char* s_c1 = s_r2 + TILE_BYTES;          // two stages
+    unsigned char* s_c2 = s_c1 + 2 * TILE_BYTES;      // two stages
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int gq = lane >> 2, tq = lane & 3;
+    const int head = blockIdx.x % g.heads;
+    const int M = g.Mh * g.Mw;
+    const int c0 = (g.w - 1) * 2 * g.w;
+    const long long n_items = (long long)g.B * M * tiles;
+
+    const __nv_bfloat16* own1 = KV ? k : q;
+    const __nv_bfloat16* own2 = KV ? v : d_o;
+    const __nv_bfloat16* str1 = KV ? q : k;
+    const __nv_bfloat16* str2 = KV ? d_o : v;
+
+    for (int i = tid; i < nbias; i += NTHREADS) {
+        s_bias[i] = bias[(size_t)i * g.heads + head] * kLog2e;
+        s_dbias[i] = 0.f;
+    }
+
+    for (long long item = blockIdx.x / g.heads; item < n_items; item += ctas_per_head) {
+        const int tile = (int)(item % tiles);
+        const int win = (int)((item / tiles) % M);
+        const int b = (int)(item / ((long long)tiles * M));
+        const WindowRef r = window_ref(g, win);
+        const int r0 = tile * BM;
+        if (r0 >= r.n) continue;
+        const int nblk = (r.n + BN - 1) / BN;
+        const int npad = nblk * BN;
+        const size_t sample_off = (size_t)b * g.H * g.W;
+
+        __syncthreads();   // previous item's readers of the slot tables and tiles are done
+        for (int s = tid; s < npad; s += NTHREADS) {
+            int meta = 0xff << 16, tok = -1;
+            float l2 = INFINITY, dl = 0.f;      // padded queries: P = exp2(x - inf) = 0
+            if (s < r.n) {
+                tok = slot_token(g, r, s, meta);
+                size_t li = (sample_off + (size_t)tok) * g.heads + head;
+                l2 = lse[li] * kLog2e;
+                dl = delta[li];
+            }
+            s_tok[s] = tok;
+            s_meta[s] = meta;
+            s_lse[s] = l2;
+            s_delta[s] = dl;
+        }
+        __syncthreads();
+
+        load_rows<D>(s_r1, own1, s_tok, r0, sample_off, g.heads, head, tid);
+        load_rows<D>(s_r2, own2, s_tok, r0, sample_off, g.heads, head, tid);
+        load_rows<D>(s_c1, str1, s_tok, 0, sample_off, g.heads, head, tid);
+        load_rows<D>(s_c2, str2, s_tok, 0, sample_off, g.heads, head, tid);
+        cp_async_commit();
+
+        uint32_t f1[KS][4], f2[KS][4];
+        float acc1[DT][4], acc2[KV ? DT : 1][4];
+#pragma unroll
+        for (int i = 0; i < DT; ++i)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc1[i][e] = 0.f;
+#pragma unroll
+        for (int i = 0; i < (KV ? DT : 1); ++i)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc2[i][e] = 0.f;
+
+        const int row_slot[2] = {r0 + warp * 16 + gq, r0 + warp * 16 + gq + 8};
+        const int meta_r[2] = {s_meta[row_slot[0]], s_meta[row_slot[1]]};
+        const float lse_r[2] = {s_lse[row_slot[0]], s_lse[row_slot[1]]};
+        const float del_r[2] = {s_delta[row_slot[0]], s_delta[row_slot[1]]};
+
+        for (int blk = 0; blk < nblk; ++blk) {
+            const int stage = blk & 1;
+            if (blk + 1 < nblk) {
+                load_rows<D>(s_c1 + (stage ^ 1) * TILE_BYTES, str1, s_tok, (blk + 1) * BN, sample_off, g.heads, head, tid);
+                load_rows<D>(s_c2 + (stage ^ 1) * TILE_BYTES, str2, s_tok, (blk + 1) * BN, sample_off, g.heads, head, tid);
+                cp_async_commit();
+                cp_async_wait<1>();
+            } else {
+                cp_async_wait<0>();
+            }
+            __syncthreads();
+            if (blk == 0) {
+#pragma unroll
+                for (int ks = 0; ks < KS; ++ks) {
+                    int row = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+                    ldmatrix_x4(f1[ks], smem_u32(s_r1 + tile_off<D>(row, 2 * ks + (lane >> 4))));
+                    ldmatrix_x4(f2[ks], smem_u32(s_r2 + tile_off<D>(row, 2 * ks + (lane >> 4))));
+                }
+            }
+            const unsigned char* c1 = s_c1 + stage * TILE_BYTES;
+            const unsigned char* c2 = s_c2 + stage * TILE_BYTES;
+
+            float acc_s[BN / 8][4], acc_dp[BN / 8][4];
+            rows_times_block_t<D>(acc_s, f1, c1, lane);     // S (or S^T) before scale and bias
+            rows_times_block_t<D>(acc_dp, f2, c2, lane);    // dP (or dP^T)
+
+            // P = exp2(S * scale * log2e + bias * log2e - lse * log2e);  dS = P * (dP - delta)
+#pragma unroll
+            for (int nt = 0; nt < BN / 8; ++nt) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int col = blk * BN + nt * 8 + 2 * tq + (e & 1);
+                    const int mc = s_meta[col];
+                    const int mr = meta_r[e >> 1];
+                    const bool ok = meta_label(mr) == meta_label(mc);
+                    // bias row uses query offset minus key offset
+                    const int bidx = KV ? (meta_code(mc) - meta_code(mr) + c0) : (meta_code(mr) - meta_code(mc) + c0);
+                    const float l2 = KV ? s_lse[col] : lse_r[e >> 1];
+                    const float dl = KV ? s_delta[col] : del_r[e >> 1];
+                    float p = fast_exp2(acc_s[nt][e] * g.scale_log2e + s_bias[bidx] - l2);
+                    p = ok ? p : 0.f;
+                    const float ds = p * (acc_dp[nt][e] - dl);
+                    acc_s[nt][e] = p;
+                    acc_dp[nt][e] = ds;
+                    if (!KV && ok && p != 0.f) atomicAdd(&s_dbias[bidx], ds);
+                }
+            }
+            if constexpr (KV) {
+                coef_times_block<D>(acc1, acc_dp, c1, lane);    // dK += dS^T Q
+                coef_times_block<D>(acc2, acc_s, c2, lane);     // dV += P^T dO
+            } else {
+                coef_times_block<D>(acc1, acc_dp, c1, lane);    // dQ += dS K
+            }
+            __syncthreads();
+        }
+
+        // stage in the own-tile slots (their fragments live in registers), then scatter to the grid
+        const float scale = g.scale_log2e * kLn2;
+        stage_rows<D>(s_r1, acc1, scale, warp, gq, tq);
+        if constexpr (KV) stage_rows<D>(s_r2, acc2, 1.f, warp, gq, tq);
+        __syncthreads();
+        scatter_rows<D>(s_r1, out1, s_tok, r0, r.n, sample_off, g.heads, head, tid);
+        if constexpr (KV) scatter_rows<D>(s_r2, out2, s_tok, r0, r.n, sample_off, g.heads, head, tid);
+    }
+
+    if (!KV) {
+        __syncthreads();
+        for (int i = tid; i < nbias; i += NTHREADS) {
+            float val = s_dbias[i];
+            if (val != 0.f) atomicAdd(&dbias[(size_t)i * g.heads + head], val);
+        }
+    }
+}
+
+// delta[b, token, head] = sum_c dO[b, token, head, c] * O[b, token, head, c]
+template <int D>
+__global__ void __launch_bounds__(256)
+swin_bwd_delta_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloat16* __restrict__ d_o,
+                      float* __restrict__ delta, long long rows) {
+    constexpr int LPR = D / 8;   // lanes per row, each lane takes one 16-byte chunk
+    long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    long long row = gid / LPR;
+    int chunk = (int)(gid % LPR);
+    float acc = 0.f;
+    if (row < rows) {
+        uint4 a = *reinterpret_cast<const uint4*>(o + row * D + chunk * 8);
+        uint4 b = *reinterpret_cast<const uint4*>(d_o + row * D + chunk * 8);
+        const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&a);
+        const __nv_bfloat162* pb = reinterpret_cast<const __nv_bfloat162*>(&b);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float2 x = __bfloat1622float2(pa[i]), y = __bfloat1622float2(pb[i]);
+            acc += x.x * y.x + x.y * y.y;
+        }
+    }
+#pragma unroll
+    for (int off = LPR / 2; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+    if (row < rows && chunk == 0) delta[row] = acc;
+}
+
+size_t bwd_smem_bytes(const Geo& g) {
+    int npad_max = ((g.nmax + BN - 1) / BN) * BN;
+    int nbias = (2 * g.w - 1) * (2 * g.w - 1);
+    size_t head = (((size_t)npad_max * 16 + (size_t)nbias * 8 + 127) / 128) * 128;
+    return head + 6 * (size_t)BN * g.d * 2;
+}
+
+template <int D, bool KV>
+cudaError_t launch_one(const Geo& g, const void* q, const void* k, const void* v, const void* d_o, const float* bias,
+                       const float* lse, const float* delta, void* out1, void* out2, float* dbias, int sm_count,
+                       cudaStream_t stream) {
+    auto kern = swin_bwd_mma_kernel<D, KV>;
+    const size_t smem = bwd_smem_bytes(g);
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    int occ = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, NTHREADS, smem);
+    if (e != cudaSuccess) return e;
+    if (occ < 1) occ = 1;
+    const int tiles = (g.nmax + BM - 1) / BM;
+    const long long items = (long long)g.B * g.Mh * g.Mw * tiles;
+    long long cph = ((long long)sm_count * occ) / g.heads;     // persistent CTAs bound to each head
+    if (cph < 1) cph = 1;
+    if (cph > items) cph = items;
+    kern<<<(unsigned)(cph * g.heads), NTHREADS, smem, stream>>>(
+        g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)d_o, bias,
+        lse, delta, (__nv_bfloat16*)out1, (__nv_bfloat16*)out2, dbias, tiles, (int)cph);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_bwd_delta(const Geo& g, const void* o, const void* d_o, float* delta, cudaStream_t stream) {
+    const long long rows = (long long)g.B * g.H * g.W * g.heads;
+    const int lpr = g.d / 8;
+    const long long threads = rows * lpr;
+    const unsigned blocks = (unsigned)((threads + 255) / 256);
+    if (g.d == 32)
+        swin_bwd_delta_kernel<32><<<blocks, 256, 0, stream>>>((const __nv_bfloat16*)o, (const __nv_bfloat16*)d_o, delta, rows);
+    else
+        swin_bwd_delta_kernel<64><<<blocks, 256, 0, stream>>>((const __nv_bfloat16*)o, (const __nv_bfloat16*)d_o, delta, rows);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_bwd_mma(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
+                           const float* lse, const float* delta, const void* d_o,
+                           void* dq, void* dk, void* dv, float* dbias, int sm_count, cudaStream_t stream) {
+    cudaError_t e = cudaMemsetAsync(dbias, 0, sizeof(float) * (size_t)(2 * g.w - 1) * (2 * g.w - 1) * g.heads, stream);
+    if (e != cudaSuccess) return e;
+    if (g.d == 32) {
+        e = launch_one<32, true>(g, q, k, v, d_o, bias, lse, delta, dk, dv, nullptr, sm_count, stream);
+        if (e != cudaSuccess) return e;
+        return launch_one<32, false>(g, q, k, v, d_o, bias, lse, delta, dq, nullptr, dbias, sm_count, stream);
+    }
+    e = launch_one<64, true>(g, q, k, v, d_o, bias, lse, delta, dk, dv, nullptr, sm_count, stream);
+    if (e != cudaSuccess) return e;
+    return launch_one<64, false>(g, q, k, v, d_o, bias, lse, delta, dq, nullptr, dbias, sm_count, stream);
+}
+
+}  // namespace terra

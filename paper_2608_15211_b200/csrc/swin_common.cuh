@@ -1,0 +1,103 @@
+// Shared device-side definitions of the shifted-window attention kernels (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace terra {
+
+// Window geometry of one call, resolved on the host (paper Section IV-D symbols).
+struct Geo {
+    int B, H, W;          // batch, token grid (H_T x W_T)
+    int heads, d;         // heads, head dim
+    int w;                // window side
+    int sh, sw;           // shifts, already reduced mod H / mod W
+    int ph, pw;           // periodic flags
+    int Mh, Mw;           // window grid: ceil(H / w) x ceil(W / w)
+    int nmax;             // tokens in a full window: min(w, H) * min(w, W)
+    float scale_log2e;    // score scale * log2(e)
+};
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+// Per-slot metadata packed in one int: bias code a * (2w - 1) + b in the low 16 bits, the shift-mask
+// label in bits 16..17.  bias row of (query i, key j) = code_i - code_j + (w - 1) * 2w.
+__device__ __forceinline__ int meta_code(int m) { return m & 0xffff; }
+__device__ __forceinline__ int meta_label(int m) { return m >> 16; }
+
+struct WindowRef {
+    int wr, wc;   // window row / column
+    int eh, ew;   // true extent (truncated at the last row / column)
+    int n;        // eh * ew
+};
+
+__device__ __forceinline__ WindowRef window_ref(const Geo& g, int win) {
+    WindowRef r;
+    r.wr = win / g.Mw;
+    r.wc = win - r.wr * g.Mw;
+    r.eh = min(g.w, g.H - r.wr * g.w);
+    r.ew = min(g.w, g.W - r.wc * g.w);
+    r.n = r.eh * r.ew;
+    return r;
+}
+
+// Slot of a window -> grid token u * W + v (undoing the roll) and packed metadata.
+__device__ __forceinline__ int slot_token(const Geo& g, const WindowRef& r, int slot, int& meta) {
+    int a = slot / r.ew;
+    int b = slot - a * r.ew;
+    int u = r.wr * g.w + a + g.sh;
+    if (u >= g.H) u -= g.H;
+    int v = r.wc * g.w + b + g.sw;
+    if (v >= g.W) v -= g.W;
+    int label = ((!g.ph && u < g.sh) ? 2 : 0) + ((!g.pw && v < g.sw) ? 1 : 0);
+    meta = (a * (2 * g.w - 1) + b) | (label << 16);
+    return u * g.W + v;
+}
+
+// ---- small PTX wrappers -----------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+// 16-byte async copy; src_bytes = 0 writes zeros (used for rows past the window's end).
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N)); }
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+// D (16x8, fp32) += A (16x16, bf16, row) * B (16x8, bf16, col)
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Shared-memory tile of bf16 rows, D elements each, 16-byte chunks XOR-swizzled so that ldmatrix
+// over 8 consecutive rows touches every bank once.  Returns the byte offset of (row, chunk).
+template <int D>
+__device__ __forceinline__ uint32_t tile_off(int row, int chunk) {
+    constexpr int CPR = D / 8;                       // 16-byte chunks per row: 4 (d=32) or 8 (d=64)
+    int sw = (CPR == 4) ? ((row >> 1) & 3) : (row & 7);
+    return static_cast<uint32_t>(row * (D * 2) + ((chunk ^ sw) << 4));
+}
+
+}  // namespace terra

@@ -1,0 +1,27 @@
+// Host-side launch interface between the C ABI (api.cu) and the kernel files.
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "swin_common.cuh"
+
+namespace terra {
+
+void count_launch();   // bumps the process-wide kernel launch counter
+
+cudaError_t launch_route(const Geo& g, int32_t* perm, int32_t* inv_perm, int32_t* win_offsets,
+                         int32_t* pos, int32_t* label, cudaStream_t stream);
+
+cudaError_t launch_fwd_mma(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
+                           void* o, float* lse, cudaStream_t stream);
+
+// delta[b, token, head] = sum_c dO * O   (fp32, same indexing as lse)
+cudaError_t launch_bwd_delta(const Geo& g, const void* o, const void* d_o, float* delta, cudaStream_t stream);
+
+// dK, dV (key-tile CTAs) and dQ, dBias (query-tile CTAs)
+cudaError_t launch_bwd_mma(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
+                           const float* lse, const float* delta, const void* d_o,
+                           void* dq, void* dk, void* dv, float* dbias, int sm_count, cudaStream_t stream);
+
+}  // namespace terra

@@ -1,0 +1,193 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2608_15211_b200 as terra
+from paper_2608_15211_b200.workloads import CONFIGS, make_inputs, small_config
+from tests._parity import gate, gpu_rows, sample_windows
+
+pytestmark = pytest.mark.gpu
+
+EDGE = [
+    # name,            B, H,  W,  heads, d,  w,  sh, sw, ph, pw
+    ("tiny_nonperiodic", 2, 8, 8, 2, 32, 4, 2, 2, 0, 0),
+    ("tiny_periodic", 1, 8, 12, 1, 32, 4, 1, 3, 1, 1),
+    ("ragged_small_rem", 1, 9, 7, 2, 32, 4, 3, 3, 0, 1),       # 0 < H mod w < shift
+    ("window_gt_grid", 1, 3, 5, 2, 32, 8, 1, 2, 0, 1),
+    ("single_row", 1, 1, 70, 1, 32, 6, 0, 5, 0, 1),
+    ("no_shift", 3, 10, 12, 2, 64, 4, 0, 0, 0, 1),
+    ("odd_window", 1, 23, 31, 3, 32, 5, 2, 3, 0, 1),
+    ("w1", 1, 4, 6, 1, 32, 1, 0, 0, 0, 1),
+    ("w32_d32", 1, 40, 70, 1, 32, 32, 16, 16, 0, 1),
+    ("w20_d64", 2, 45, 50, 2, 64, 20, 10, 10, 0, 1),
+    ("shift_ge_grid", 1, 12, 16, 2, 32, 4, 12 + 2, 16 * 3 + 1, 0, 1),
+]
+
+
+def _to_gpu(x):
+    return {k: v.cuda() for k, v in x.items()}
+
+
+def _run_fwd(cfg, xg, scale=0.0):
+    d = terra.make_desc(cfg, scale)
+    o, lse = terra.terra_swin_attn_fwd(d, xg["q"], xg["k"], xg["v"], xg["bias"])
+    torch.cuda.synchronize()
+    return d, o, lse
+
+
+def _run_bwd(cfg, d, xg, o, lse):
+    out = terra.terra_swin_attn_bwd(d, xg["q"], xg["k"], xg["v"], xg["bias"], o, lse, xg["do"])
+    torch.cuda.synchronize()
+    return out
+
+
+def _check_forward(cfg, x, o, lse, sel, scale=0.0):
+    ro, rl = oracle.attn_fwd(cfg, x["q"], x["k"], x["v"], x["bias"].double().numpy(), sel=sel, scale=scale)
+    tok = oracle.selection_tokens(cfg, sel)
+    gate("o", gpu_rows(o, cfg, tok), ro)
+    gate("lse", gpu_rows(lse, cfg, tok), rl)
+
+
+def _check_backward(cfg, x, grads, sel, dbias_ref_is_total, scale=0.0):
+    dq, dk, dv, dbias = grads
+    rq, rk, rv, rb = oracle.attn_bwd(cfg, x["q"], x["k"], x["v"], x["do"], x["bias"].double().numpy(), sel=sel, scale=scale)
+    tok = oracle.selection_tokens(cfg, sel)
+    gate("dq", gpu_rows(dq, cfg, tok), rq)
+    gate("dk", gpu_rows(dk, cfg, tok), rk)
+    gate("dv", gpu_rows(dv, cfg, tok), rv)
+    if dbias_ref_is_total:
+        gate("dbias", dbias.cpu().double().numpy(), rb)
+
+
+@pytest.mark.parametrize("name", ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
+def test_route_bit_exact(name):
+    cfg = CONFIGS[name]
+    got = terra.terra_window_route(terra.make_desc(cfg))
+    torch.cuda.synchronize()
+    ref = oracle.window_route(cfg)
+    for key, val in ref.items():
+        assert np.array_equal(got[key].cpu().numpy(), val), key
+
+
+@pytest.mark.parametrize("case", EDGE, ids=[c[0] for c in EDGE])
+def test_route_bit_exact_edge_cases(case):
+    cfg = small_config(*case)
+    got = terra.terra_window_route(terra.make_desc(cfg))
+    torch.cuda.synchronize()
+    ref = oracle.window_route(cfg)
+    for key, val in ref.items():
+        assert np.array_equal(got[key].cpu().numpy(), val), key
+
+
+def test_route_null_outputs_are_skipped():
+    import ctypes
+    cfg = CONFIGS["cfg1"]
+    d = terra.make_desc(cfg)
+    perm = torch.full((cfg.H * cfg.W,), -1, dtype=torch.int32, device="cuda")
+    null = ctypes.c_void_p(0)
+    lib = terra.load_library()
+    assert lib.terra_window_route(ctypes.byref(d), ctypes.c_void_p(perm.data_ptr()), null, null, null, null, null) == 0
+    torch.cuda.synchronize()
+    assert np.array_equal(perm.cpu().numpy(), oracle.window_route(cfg)["perm"])
+
+
+@pytest.mark.parametrize("case", EDGE, ids=[c[0] for c in EDGE])
+def test_edge_cases_forward_backward(case):
+    cfg = small_config(*case)
+    x = make_inputs(cfg)
+    x["bias"] = x["bias"] * 25.0          # make the bias matter (std 0.5)
+    xg = _to_gpu(x)
+    d, o, lse = _run_fwd(cfg, xg)
+    _check_forward(cfg, x, o, lse, None)
+    grads = _run_bwd(cfg, d, xg, o, lse)
+    _check_backward(cfg, x, grads, None, True)
+
+
+def test_explicit_scale_is_used():
+    cfg = small_config("scale", 1, 12, 16, 2, 32, 4, 2, 2, 0, 1)
+    x = make_inputs(cfg)
+    xg = _to_gpu(x)
+    d, o, lse = _run_fwd(cfg, xg, scale=0.05)
+    _check_forward(cfg, x, o, lse, None, scale=0.05)
+    grads = _run_bwd(cfg, d, xg, o, lse)
+    _check_backward(cfg, x, grads, None, True, scale=0.05)
+
+
+def test_cfg1_forward_full():
+    cfg = CONFIGS["cfg1"]
+    x = make_inputs(cfg)
+    d, o, lse = _run_fwd(cfg, _to_gpu(x))
+    _check_forward(cfg, x, o, lse, None)
+
+
+@pytest.mark.parametrize("name", ["cfg2", "cfg3"])
+def test_full_tensors_forward_backward(name):
+    cfg = CONFIGS[name]
+    x = make_inputs(cfg)
+    xg = _to_gpu(x)
+    d, o, lse = _run_fwd(cfg, xg)
+    _check_forward(cfg, x, o, lse, None)
+    grads = _run_bwd(cfg, d, xg, o, lse)
+    _check_backward(cfg, x, grads, None, True)
+
+
+@pytest.mark.parametrize("name,count", [("cfg4", 8), ("cfg5", 48)])
+def test_full_size_sampled_windows(name, count):
+    """Full-size launch; the oracle recomputes a sample of windows (every edge class included).
+    dBias sums over all windows, so it is checked on a second backward launch whose upstream gradient
+    is zero outside the sampled windows: there the full sum equals the oracle's sum over the sample."""
+    cfg = CONFIGS[name]
+    x = make_inputs(cfg)
+    xg = _to_gpu(x)
+    sel = sample_windows(cfg, count)
+    d, o, lse = _run_fwd(cfg, xg)
+    _check_forward(cfg, x, o, lse, sel)
+    grads = _run_bwd(cfg, d, xg, o, lse)
+    _check_backward(cfg, x, grads, sel, False)
+    # property that holds at any size: every softmax row's dS sums to zero, hence so does dT per head
+    dbias = grads[3].double()
+    assert torch.all(dbias.sum(0).abs() <= 2e-2 * dbias.abs().max())
+    del grads
+    tok = torch.from_numpy(oracle.selection_tokens(cfg, sel)).cuda()
+    do_sparse = torch.zeros_like(xg["do"])
+    flat_src = xg["do"].reshape(cfg.tokens, cfg.heads, cfg.head_dim)
+    do_sparse.reshape(cfg.tokens, cfg.heads, cfg.head_dim)[tok] = flat_src[tok]
+    xs = dict(xg, do=do_sparse)
+    grads = _run_bwd(cfg, d, xs, o, lse)
+    x2 = dict(x, do=do_sparse.cpu())
+    _check_backward(cfg, x2, grads, sel, True)
+
+
+def test_outputs_are_reproducible_and_inputs_untouched():
+    cfg = CONFIGS["cfg2"]
+    x = make_inputs(cfg)
+    xg = _to_gpu(x)
+    keep = {k: v.clone() for k, v in xg.items()}
+    d, o1, l1 = _run_fwd(cfg, xg)
+    g1 = _run_bwd(cfg, d, xg, o1, l1)
+    d, o2, l2 = _run_fwd(cfg, xg)
+    g2 = _run_bwd(cfg, d, xg, o2, l2)
+    assert torch.equal(o1, o2) and torch.equal(l1, l2)
+    for a, b in zip(g1[:3], g2[:3]):
+        assert torch.equal(a, b)
+    for k in xg:
+        assert torch.equal(xg[k], keep[k])
+
+
+def test_alignment_and_workspace_errors():
+    cfg = CONFIGS["cfg1"]
+    x = _to_gpu(make_inputs(small_config("e", 1, 32, 64, 3, 32, 8, 4, 4)))
+    d = terra.make_desc(cfg)
+    n = cfg.tokens * cfg.heads * cfg.head_dim
+    buf = torch.zeros(n + 8, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(terra.TerraError) as e:
+        terra.terra_swin_attn_fwd(d, buf[1:n + 1], x["k"], x["v"], x["bias"])
+    assert e.value.status == 3
+    o, lse = terra.terra_swin_attn_fwd(d, x["q"], x["k"], x["v"], x["bias"])
+    with pytest.raises(terra.TerraError) as e:
+        terra.terra_swin_attn_bwd(d, x["q"], x["k"], x["v"], x["bias"], o, lse, x["do"],
+                                  workspace=torch.empty(16, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == 4
+    torch.cuda.synchronize()
