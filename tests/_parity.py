@@ -17,7 +17,9 @@ def gate(name, got, ref, strict=True):
     ref = np.asarray(ref, dtype=np.float64)
     assert got.shape == ref.shape, (name, got.shape, ref.shape)
     assert np.all(np.isfinite(got)), f"{name}: non-finite values in the GPU result"
-    scale = np.abs(ref).max()
+    # inputs are N(0, 1): a reference that is identically zero (single-token windows give dQ = dK = 0)
+    # is compared on the scale of fp32 rounding of O(1) terms instead of on a zero scale
+    scale = max(np.abs(ref).max(), 1e-3)
     err = np.abs(got - ref)
     assert err.max() <= G1_ABS * scale, f"{name}: G1 max|err| {err.max():.3e} > {G1_ABS * scale:.3e}"
     assert np.all(err <= G1_ABS * scale + G2_REL * np.abs(ref)), f"{name}: G2 failed"

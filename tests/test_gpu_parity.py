@@ -147,8 +147,9 @@ def test_full_size_sampled_windows(name, count):
     grads = _run_bwd(cfg, d, xg, o, lse)
     _check_backward(cfg, x, grads, sel, False)
     # property that holds at any size: every softmax row's dS sums to zero, hence so does dT per head
+    # (up to the rounding of the saved bf16 O that enters delta: a random walk over all query rows)
     dbias = grads[3].double()
-    assert torch.all(dbias.sum(0).abs() <= 2e-2 * dbias.abs().max())
+    assert torch.all(dbias.sum(0).abs() <= 2e-3 * dbias.abs().sum(0))
     del grads
     tok = torch.from_numpy(oracle.selection_tokens(cfg, sel)).cuda()
     do_sparse = torch.zeros_like(xg["do"])
