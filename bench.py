@@ -239,7 +239,8 @@ def main():
     lse = torch.empty((cfg.B, cfg.H, cfg.W, cfg.heads), dtype=torch.float32, device=dev)
     dq, dk, dv = torch.empty_like(q), torch.empty_like(q), torch.empty_like(q)
     dbias = torch.empty_like(bias)
-    ws = torch.empty(max(16, terra.terra_swin_workspace_bytes(desc, True)), dtype=torch.uint8, device=dev)
+    ws = torch.empty(max(16, terra.terra_swin_workspace_bytes(desc, True), terra.terra_swin_workspace_bytes(desc, False)),
+                     dtype=torch.uint8, device=dev)
     lib = terra.load_library()
     import ctypes
     P = lambda t: ctypes.c_void_p(t.data_ptr())

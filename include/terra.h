@@ -39,7 +39,8 @@ typedef enum {
     TERRA_ERR_UNSUPPORTED = 2,   /* head_dim not in {32, 64}, window too large, not an sm_100 GPU */
     TERRA_ERR_ALIGNMENT = 3,     /* a pointer is not 16-byte aligned                              */
     TERRA_ERR_WORKSPACE = 4,     /* workspace NULL or smaller than terra_swin_workspace_bytes     */
-    TERRA_ERR_CUDA = 5           /* a CUDA call failed; text via terra_last_cuda_error            */
+    TERRA_ERR_CUDA = 5,          /* a CUDA call failed; text via terra_last_cuda_error            */
+    TERRA_ERR_DEVICE_TIMEOUT = 6 /* a bounded wait inside a kernel expired (see terra_swin_check) */
 } terra_status;
 
 /* Problem statement: token grid, window, heads (paper Table I symbols; H, W here are H_T, W_T). */
@@ -105,6 +106,15 @@ int terra_swin_attn_bwd(const terra_swin_desc* desc, const void* q, const void* 
                         const float* bias_table, const void* o, const float* lse, const void* d_o,
                         void* dq, void* dk, void* dv, float* dbias,
                         void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Waits for `stream` and reports whether any kernel of this library gave up on a bounded wait since
+ * the last check (the kernels never spin forever: a wait on a barrier has a cycle limit, after which the
+ * CTA stops working, releases its tensor memory and raises a device-side word).  Returns TERRA_OK or
+ * TERRA_ERR_DEVICE_TIMEOUT (and clears the word).  The paper has no counterpart; this is the library's
+ * own failure report.
+ */
+int terra_swin_check(void* stream);
 
 /* Static text for a terra_status.  Host-only. */
 const char* terra_strerror(int status);

@@ -16,7 +16,8 @@ from .build import LIB_PATH
 
 TERRA_OK = 0
 EXPORTS = ("terra_route_sizes", "terra_window_route", "terra_swin_workspace_bytes", "terra_swin_attn_fwd",
-           "terra_swin_attn_bwd", "terra_strerror", "terra_last_cuda_error", "terra_launch_count")
+           "terra_swin_attn_bwd", "terra_swin_check", "terra_strerror", "terra_last_cuda_error",
+           "terra_launch_count")
 
 
 class TerraError(RuntimeError):
@@ -39,7 +40,7 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
     global _lib
     if _lib is not None and path is None:
         return _lib
-    p = path or LIB_PATH
+    p = path or os.environ.get("TERRA_LIB_PATH") or LIB_PATH
     if not os.path.exists(p):
         raise FileNotFoundError(f"{p} not found: build it with `python -m paper_2608_15211_b200.build` "
                                 "(the library has no CPU fallback)")
@@ -54,6 +55,8 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
     for n in ("terra_route_sizes", "terra_window_route", "terra_swin_workspace_bytes", "terra_swin_attn_fwd",
               "terra_swin_attn_bwd"):
         getattr(lib, n).restype = ctypes.c_int
+    lib.terra_swin_check.argtypes = [vp]
+    lib.terra_swin_check.restype = ctypes.c_int
     lib.terra_strerror.argtypes = [ctypes.c_int]
     lib.terra_strerror.restype = ctypes.c_char_p
     lib.terra_last_cuda_error.restype = ctypes.c_char_p
@@ -89,6 +92,11 @@ def _ptr(t) -> ctypes.c_void_p:
 
 def _stream() -> ctypes.c_void_p:
     return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def terra_swin_check() -> None:
+    """Waits for the current stream; raises TerraError(6) if a kernel gave up on a bounded wait."""
+    _check(load_library().terra_swin_check(_stream()))
 
 
 def launch_count() -> int:
@@ -135,6 +143,9 @@ def terra_swin_attn_fwd(desc, q, k, v, bias_table, o=None, lse=None, workspace=N
         lse = torch.empty((desc.B, desc.H, desc.W, desc.heads), dtype=torch.float32, device=q.device)
     _expect(o, torch.bfloat16, n * desc.head_dim, "o")
     _expect(lse, torch.float32, n, "lse")
+    if workspace is None:
+        need = terra_swin_workspace_bytes(desc, False)
+        workspace = torch.empty(need, dtype=torch.uint8, device=q.device) if need else None
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     _check(load_library().terra_swin_attn_fwd(ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(v), _ptr(bias_table),
                                               _ptr(o), _ptr(lse), _ptr(workspace), ws_bytes, _stream()))

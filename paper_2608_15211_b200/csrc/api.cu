@@ -2,6 +2,7 @@
 #include <atomic>
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 
 #include "../../include/terra.h"
@@ -68,6 +69,19 @@ static int device_props(int* sm_count) {
     return TERRA_OK;
 }
 
+// Debugging switch: TERRA_REGISTER_PATH=1 routes every shape through the register-tile kernels.
+static bool force_register_path() {
+    static const bool on = [] {
+        const char* v = std::getenv("TERRA_REGISTER_PATH");
+        return v && v[0] == '1';
+    }();
+    return on;
+}
+
+static size_t fwd_bytes(const Geo& g) {
+    return (fwd_tc_supported(g) && !force_register_path()) ? align_up(fwd_tc_workspace_bytes(g), 256) : 0;
+}
+
 static size_t delta_bytes(const Geo& g) {
     return align_up(sizeof(float) * (size_t)g.B * g.H * g.W * g.heads, 256);
 }
@@ -103,24 +117,30 @@ int terra_swin_workspace_bytes(const terra_swin_desc* desc, int backward, size_t
     int rc = make_geo(desc, true, &g);
     if (rc) return rc;
     if (!bytes) return TERRA_ERR_INVALID_ARG;
-    *bytes = backward ? delta_bytes(g) : 0;
+    *bytes = backward ? delta_bytes(g) : fwd_bytes(g);
     return TERRA_OK;
 }
 
 int terra_swin_attn_fwd(const terra_swin_desc* desc, const void* q, const void* k, const void* v,
                         const float* bias_table, void* o, float* lse,
                         void* workspace, size_t workspace_bytes, void* stream) {
-    (void)workspace; (void)workspace_bytes;
     Geo g;
     int rc = make_geo(desc, true, &g);
     if (rc) return rc;
     if (!q || !k || !v || !bias_table || !o || !lse) return TERRA_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(bias_table) || !aligned16(lse))
         return TERRA_ERR_ALIGNMENT;
+    const size_t need = fwd_bytes(g);
+    if (need > 0 && (!workspace || workspace_bytes < need)) return TERRA_ERR_WORKSPACE;
+    if (need > 0 && !aligned16(workspace)) return TERRA_ERR_ALIGNMENT;
     int sms = 0;
     rc = device_props(&sms);
     if (rc) return rc;
-    cudaError_t e = launch_fwd_mma(g, q, k, v, bias_table, o, lse, (cudaStream_t)stream);
+    cudaError_t e;
+    if (need > 0)
+        e = launch_fwd_tc(g, q, k, v, bias_table, o, lse, workspace, sms, (cudaStream_t)stream);
+    else
+        e = launch_fwd_mma(g, q, k, v, bias_table, o, lse, (cudaStream_t)stream);
     return e == cudaSuccess ? TERRA_OK : cuda_fail(e, "terra_swin_attn_fwd");
 }
 
@@ -149,6 +169,13 @@ int terra_swin_attn_bwd(const terra_swin_desc* desc, const void* q, const void* 
     return e == cudaSuccess ? TERRA_OK : cuda_fail(e, "terra_swin_attn_bwd");
 }
 
+int terra_swin_check(void* stream) {
+    int timed_out = 0;
+    cudaError_t e = read_tc_status(&timed_out, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(e, "terra_swin_check");
+    return timed_out ? TERRA_ERR_DEVICE_TIMEOUT : TERRA_OK;
+}
+
 const char* terra_strerror(int status) {
     switch (status) {
         case TERRA_OK: return "ok";
@@ -157,6 +184,7 @@ const char* terra_strerror(int status) {
         case TERRA_ERR_ALIGNMENT: return "pointer is not 16-byte aligned";
         case TERRA_ERR_WORKSPACE: return "workspace missing or too small (see terra_swin_workspace_bytes)";
         case TERRA_ERR_CUDA: return "CUDA error (see terra_last_cuda_error)";
+        case TERRA_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel expired; results of that call are invalid";
         default: return "unknown status";
     }
 }

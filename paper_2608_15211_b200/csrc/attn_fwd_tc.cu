@@ -1,0 +1,552 @@
+// Forward shifted-window attention on the tcgen05 tensor cores (head dim 32, windows of <= 256 tokens).
+//
+// One persistent CTA per SM walks over (batch, window, head) items.  Roles:
+//   warps 0-3 / 4-7  softmax warpgroups: one thread per query row of the first / second 128-row tile;
+//                    S is read from TMEM, P = exp2(S*scale + bias - m) is written back to TMEM as bf16,
+//                    O is read from TMEM, normalised and stored straight to the token's grid position
+//   warp 8           issues tcgen05.mma: S = Q K^T (operands in shared memory), O = P V (P from TMEM)
+//   warps 9-11       loaders: undo the roll, gather the window's Q / K / V rows with cp.async into the
+//                    64-byte-swizzled operand layout, stage the head's bias table and the slot metadata
+// TMEM: columns [256 t, 256 t + 256) belong to query tile t: S (fp32) first, then P (bf16, the first 128
+// columns) and four partial O accumulators (fp32, columns 128..255; key step ks adds into accumulator
+// ks mod 4, so consecutive MMAs do not wait on each other's accumulator) once S has been consumed.
+// The row maximum is replaced by the upper bound max_j(raw score) * scale + max(bias): softmax is shift
+// invariant, so the result is the same; only the exponent range matters.
+// Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, all roles leave their loops,
+// TMEM is released and the host reads the device status word.
+#include "swin_common.cuh"
+#include "swin_kernels.h"
+#include "tc_common.cuh"
+
+namespace terra {
+
+__device__ int g_tc_timeout = 0;   // set when a bounded wait expired in any CTA
+
+namespace {
+
+using namespace tc;
+
+constexpr int kMmaWarp = 8;
+constexpr int kLoaderWarp0 = 9;
+constexpr int kLoaderWarps = 3;
+constexpr int kLoaderThreads = kLoaderWarps * 32;
+constexpr int kThreads = (kLoaderWarp0 + kLoaderWarps) * 32;   // 384 = three warpgroups
+// Registers move between warpgroups at run time: the softmax warpgroups (0, 1) grow, the MMA + loader
+// warpgroup (2) shrinks.  The kernel launches with kRegsLaunch per thread (the cap of 384 threads on a
+// 64K-register SM); what the two growing warpgroups take must not exceed what the shrinking one gives
+// back, or the register request would wait forever.
+constexpr int kRegsLaunch = 168;
+constexpr int kRegsSoftmax = 216;
+constexpr int kRegsOther = 64;
+static_assert(2 * (kRegsSoftmax - kRegsLaunch) <= (kRegsLaunch - kRegsOther), "register hand-over does not balance");
+static_assert(kRegsLaunch * 384 <= 65536 && kRegsSoftmax % 8 == 0 && kRegsOther % 8 == 0, "register counts");
+constexpr int kStages = 3;
+constexpr int kMaxSlots = 256;
+constexpr int kD = 32;
+constexpr int kRowBytes = kD * 2;                              // 64
+
+// shared-memory stage layout (bytes)
+constexpr int kOffQ = 0;
+constexpr int kOffK = kMaxSlots * kRowBytes;                   // 16384
+constexpr int kOffV = 2 * kMaxSlots * kRowBytes;               // 32768
+constexpr int kOffBias = 3 * kMaxSlots * kRowBytes;            // 49152: the head's prepared bias table
+constexpr int kOffKc = kOffBias + kFwdBiasFloats * 4;          // per key slot: byte offset 4 * (c0 - code)
+constexpr int kOffKlab = kOffKc + kMaxSlots * 4;               // per key slot: shift-mask label
+constexpr int kOffRowMeta = kOffKlab + kMaxSlots * 4;          // per query slot: code | label << 16
+constexpr int kOffRowTok = kOffRowMeta + kMaxSlots * 4;        // grid token of the slot, -1 if none
+constexpr int kStageBytes = ((kOffRowTok + kMaxSlots * 4 + 1023) / 1024) * 1024;
+constexpr int kBarBytes = 256;
+constexpr int kSmemBytes = kStages * kStageBytes + kBarBytes;
+
+constexpr int kColO = 128;       // first O accumulator inside a query tile's 256-column TMEM region
+constexpr int kOAcc = 4;         // partial O accumulators, 32 columns each
+
+// Bias codes use a row stride of w + 32 instead of 2w - 1: the 32 rows of a warp (consecutive slots of a
+// full-width window) then read 32 different shared-memory banks.
+__device__ __forceinline__ int code_stride(int w) { return w + 32; }
+
+struct Item {
+    int b, win, head;
+    WindowRef r;
+    int npad;      // key slots rounded up to 16
+    int ntiles;    // 128-row query tiles in use
+    bool masked;   // the window mixes shift-mask labels
+};
+
+__device__ __forceinline__ Item make_item(const Geo& g, long long it) {
+    Item x;
+    x.head = (int)(it % g.heads);
+    long long rest = it / g.heads;
+    const int M = g.Mh * g.Mw;
+    x.win = (int)(rest % M);
+    x.b = (int)(rest / M);
+    x.r = window_ref(g, x.win);
+    x.npad = (x.r.n + 15) & ~15;
+    x.ntiles = (x.r.n + 127) >> 7;
+    // rolled rows >= H - sh (columns >= W - sw) hold the tokens that wrapped across a non-periodic edge
+    const int r0 = x.r.wr * g.w, c0 = x.r.wc * g.w;
+    const bool mh = !g.ph && g.sh > 0 && r0 < g.H - g.sh && r0 + x.r.eh > g.H - g.sh;
+    const bool mw = !g.pw && g.sw > 0 && c0 < g.W - g.sw && c0 + x.r.ew > g.W - g.sw;
+    x.masked = mh || mw;
+    return x;
+}
+
+// slot -> grid token, bias code a * (w + 32) + b and shift-mask label
+__device__ __forceinline__ int slot_token_tc(const Geo& g, const WindowRef& r, int slot, int& code, int& label) {
+    const int a = slot / r.ew;
+    const int b = slot - a * r.ew;
+    int u = r.wr * g.w + a + g.sh;
+    if (u >= g.H) u -= g.H;
+    int v = r.wc * g.w + b + g.sw;
+    if (v >= g.W) v -= g.W;
+    label = ((!g.ph && u < g.sh) ? 2 : 0) + ((!g.pw && v < g.sw) ? 1 : 0);
+    code = a * code_stride(g.w) + b;
+    return u * g.W + v;
+}
+
+__device__ __forceinline__ float lds_f32(uint32_t addr) {
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ int4 lds_i4(uint32_t addr) {
+    int4 v;
+    asm volatile("ld.shared.v4.s32 {%0,%1,%2,%3}, [%4];\n" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ int lds_i32(uint32_t addr) {
+    int v;
+    asm volatile("ld.shared.s32 %0, [%1];\n" : "=r"(v) : "r"(addr));
+    return v;
+}
+
+// P for `N` consecutive key columns starting at `c`: exp2(raw * scale + bias - m), packed to bf16 pairs.
+// bias_i / a_kc / a_klab are shared-memory byte addresses.  Returns the sum of the N values.
+template <int N, bool MASKED>
+__device__ __forceinline__ float softmax_cols(const uint32_t (&r)[N], uint32_t (&pk)[N / 2], int c, uint32_t bias_i,
+                                              uint32_t a_kc, uint32_t a_klab, int label_i, float scale, float neg_m) {
+    float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+    for (int e4 = 0; e4 < N / 4; ++e4) {
+        const int4 kc4 = lds_i4(a_kc + 4 * (c + e4 * 4));
+        const int kc[4] = {kc4.x, kc4.y, kc4.z, kc4.w};
+        int kl[4] = {0, 0, 0, 0};
+        if (MASKED) {
+            const int4 kl4 = lds_i4(a_klab + 4 * (c + e4 * 4));
+            kl[0] = kl4.x; kl[1] = kl4.y; kl[2] = kl4.z; kl[3] = kl4.w;
+        }
+        float p[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float bv = lds_f32(bias_i + kc[e]);
+            float xv = fmaf(__uint_as_float(r[e4 * 4 + e]), scale, bv) + neg_m;
+            if (MASKED && kl[e] != label_i) xv = -INFINITY;
+            p[e] = fast_exp2(xv);
+        }
+        s0 += p[0] + p[1];
+        s1 += p[2] + p[3];
+        pk[e4 * 2] = pack_bf16(p[0], p[1]);
+        pk[e4 * 2 + 1] = pack_bf16(p[2], p[3]);
+    }
+    return s0 + s1;
+}
+
+template <int N>
+__device__ __forceinline__ void max_cols(const uint32_t (&r)[N], float (&mx)[4]) {
+#pragma unroll
+    for (int e = 0; e < N; e += 8) {
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+            mx[a] = fmaxf(mx[a], fmaxf(__uint_as_float(r[e + 2 * a]), __uint_as_float(r[e + 2 * a + 1])));
+    }
+}
+
+// One softmax row: two passes over the row's S columns in TMEM, 32 columns per load, the next load in
+// flight while the current one is processed.  Returns m (log2 domain); the row sum goes to sum_out.
+template <bool MASKED>
+__device__ __forceinline__ float softmax_row(uint32_t t_s, int npad, uint32_t bias_i, uint32_t a_kc, uint32_t a_klab,
+                                             int label_i, float scale, float bmax, float& sum_out) {
+    const int nfull = npad >> 5;
+    const bool tail = (npad & 16) != 0;
+    uint32_t ra[32], rb[32];
+    float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+    if (nfull > 0) tmem_ld32(t_s, ra);
+    for (int i = 0; i < nfull; i += 2) {
+        tmem_ld_wait();
+        if (i + 1 < nfull) tmem_ld32(t_s + 32 * (i + 1), rb);
+        max_cols<32>(ra, mx4);
+        if (i + 1 < nfull) {
+            tmem_ld_wait();
+            if (i + 2 < nfull) tmem_ld32(t_s + 32 * (i + 2), ra);
+            max_cols<32>(rb, mx4);
+        }
+    }
+    if (tail) {
+        uint32_t rt[16];
+        tmem_ld16(t_s + 32 * nfull, rt);
+        tmem_ld_wait();
+        max_cols<16>(rt, mx4);
+    }
+    const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+    const float m = mx * scale + bmax;   // scale > 0: max of the scaled scores plus the largest bias
+    const float neg_m = -m;
+
+    float sum = 0.f;
+    if (nfull > 0) tmem_ld32(t_s, ra);
+    for (int i = 0; i < nfull; i += 2) {
+        uint32_t pk[16];
+        tmem_ld_wait();
+        if (i + 1 < nfull) tmem_ld32(t_s + 32 * (i + 1), rb);
+        sum += softmax_cols<32, MASKED>(ra, pk, 32 * i, bias_i, a_kc, a_klab, label_i, scale, neg_m);
+        tmem_st16(t_s + 16 * i, pk);
+        if (i + 1 < nfull) {
+            tmem_ld_wait();
+            if (i + 2 < nfull) tmem_ld32(t_s + 32 * (i + 2), ra);
+            sum += softmax_cols<32, MASKED>(rb, pk, 32 * (i + 1), bias_i, a_kc, a_klab, label_i, scale, neg_m);
+            tmem_st16(t_s + 16 * (i + 1), pk);
+        }
+    }
+    if (tail) {
+        uint32_t rt[16], pk[8];
+        tmem_ld16(t_s + 32 * nfull, rt);
+        tmem_ld_wait();
+        sum += softmax_cols<16, MASKED>(rt, pk, 32 * nfull, bias_i, a_kc, a_klab, label_i, scale, neg_m);
+        tmem_st8(t_s + 16 * nfull, pk);
+    }
+    sum_out = sum;
+    return m;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
+                   const __nv_bfloat16* __restrict__ v, const float* __restrict__ bias_prep,
+                   __nv_bfloat16* __restrict__ o, float* __restrict__ lse, long long n_items) {
+    extern __shared__ __align__(1024) unsigned char smem[];
+    const uint32_t smem0 = smem_u32(smem);
+    const uint32_t bar0 = smem0 + kStages * kStageBytes;
+    // barrier slots (8 bytes each)
+    auto bar_full = [&](int s) { return bar0 + 8u * s; };
+    auto bar_empty = [&](int s) { return bar0 + 8u * (kStages + s); };
+    auto bar_sready = [&](int t) { return bar0 + 8u * (2 * kStages + t); };
+    auto bar_pready = [&](int t) { return bar0 + 8u * (2 * kStages + 2 + t); };
+    auto bar_oready = [&](int t) { return bar0 + 8u * (2 * kStages + 4 + t); };
+    auto bar_sfree = [&](int t) { return bar0 + 8u * (2 * kStages + 6 + t); };
+    unsigned char* tail = smem + kStages * kStageBytes + 8 * (2 * kStages + 8);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail);
+    volatile int* cta_abort = reinterpret_cast<volatile int*>(tail + 8);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(bar_full(s), kLoaderThreads);
+            mbar_init(bar_empty(s), 1);
+        }
+        for (int t = 0; t < 2; ++t) {
+            mbar_init(bar_sready(t), 1);
+            mbar_init(bar_pready(t), 128);
+            mbar_init(bar_oready(t), 1);
+            mbar_init(bar_sfree(t), 128);
+        }
+        *cta_abort = 0;
+        fence_barrier_init();
+    }
+    if (warp == kMmaWarp) {
+        tmem_alloc(smem_u32(tmem_slot), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int cs = code_stride(g.w);
+    const int c0 = (g.w - 1) * (cs + 1);     // code of the last in-window offset; bias index = code_q - code_k + c0
+    const size_t HW = (size_t)g.H * g.W;
+
+    if (warp >= kMmaWarp) {
+    // warpgroup 2 (MMA issuer + loaders) gives registers back: one instruction for the whole warpgroup
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kRegsOther));
+    if (warp >= kLoaderWarp0) {
+        // ------------------------------------------------------------------ loaders
+        const int lt = tid - kLoaderWarp0 * 32;
+        int kuse = 0, pending_s = -1;
+        for (long long it = blockIdx.x; it < n_items; it += gridDim.x, ++kuse) {
+            const int s = kuse % kStages;
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_empty(s), ((kuse / kStages) & 1) ^ 1, cta_abort))) break;
+            const Item x = make_item(g, it);
+            unsigned char* st = smem + s * kStageBytes;
+            const uint32_t st_a = smem0 + s * kStageBytes;
+            int* s_kc = reinterpret_cast<int*>(st + kOffKc);
+            int* s_klab = reinterpret_cast<int*>(st + kOffKlab);
+            int* s_rowmeta = reinterpret_cast<int*>(st + kOffRowMeta);
+            int* s_rowtok = reinterpret_cast<int*>(st + kOffRowTok);
+            const size_t sample_off = (size_t)x.b * HW;
+
+            for (int slot = lt; slot < kMaxSlots; slot += kLoaderThreads) {
+                // a slot without a token: as a key its bias index lands in the table's -inf zone
+                int code = 0, label = 0xff, tok = -1, kc = 4 * (2 * c0 + 1);
+                if (slot < x.r.n) {
+                    tok = slot_token_tc(g, x.r, slot, code, label);
+                    kc = 4 * (c0 - code);
+                }
+                s_kc[slot] = kc;
+                s_klab[slot] = label;
+                s_rowmeta[slot] = code | (label << 16);
+                s_rowtok[slot] = tok;
+            }
+            // rows: this thread owns 16-byte chunk (lt & 3) of rows (lt >> 2) + 32 i
+            const int chunk = lt & 3;
+            for (int row = lt >> 2; row < x.npad; row += kLoaderThreads / 4) {
+                const __nv_bfloat16 *sq = q, *sk = k, *sv = v;
+                int bytes = 0;   // rows past the window's end are written as zeros
+                if (row < x.r.n) {
+                    int code, label;
+                    const int tok = slot_token_tc(g, x.r, row, code, label);
+                    const size_t off = ((sample_off + (size_t)tok) * g.heads + x.head) * kD + chunk * 8;
+                    sq = q + off; sk = k + off; sv = v + off;
+                    bytes = 16;
+                }
+                const uint32_t so = st_a + tile_off<kD>(row, chunk);
+                cp_async16(so + kOffQ, sq, bytes);
+                cp_async16(so + kOffK, sk, bytes);
+                cp_async16(so + kOffV, sv, bytes);
+            }
+            const float* bsrc = bias_prep + (size_t)x.head * kFwdBiasFloats;
+            for (int c = lt; c < kFwdBiasFloats / 4; c += kLoaderThreads)
+                cp_async16(st_a + kOffBias + c * 16, bsrc + c * 4, 16);
+            cp_async_commit();
+            if (pending_s >= 0) {           // the previous item's copies have landed: publish it
+                cp_async_wait<1>();
+                fence_proxy_async();
+                mbar_arrive(bar_full(pending_s));
+            }
+            pending_s = s;
+        }
+        if (pending_s >= 0) {
+            cp_async_wait<0>();
+            fence_proxy_async();
+            mbar_arrive(bar_full(pending_s));
+        }
+    } else {
+        // ------------------------------------------------------------------ MMA issuer (one lane)
+        if (lane == 0) {
+            const uint32_t idesc_pv = make_idesc_bf16(128, kD, 0, 1);
+            int kuse = 0, use_t[2] = {0, 0}, freed_t[2] = {0, 0};   // uses begun / s_free phases consumed
+            bool ok = true;
+            auto issue_qk = [&](const Item& x, int s, int t) {
+                const uint32_t qa = smem0 + s * kStageBytes + kOffQ + t * 128 * kRowBytes;
+                const uint32_t ka = smem0 + s * kStageBytes + kOffK;
+                const uint32_t idesc = make_idesc_bf16(128, x.npad, 0, 0);
+#pragma unroll
+                for (int ks = 0; ks < kD / 16; ++ks)
+                    mma_ss(tmem_base + t * 256, make_sdesc_sw64(qa + ks * 32, 512), make_sdesc_sw64(ka + ks * 32, 512),
+                           idesc, ks > 0 ? 1u : 0u);
+                mma_commit(bar_sready(t));
+            };
+            auto issue_pv = [&](const Item& x, int s, int t) {
+                const uint32_t va = smem0 + s * kStageBytes + kOffV;
+                for (int ks = 0; ks < x.npad / 16; ++ks)
+                    mma_ts(tmem_base + t * 256 + kColO + 32 * (ks & (kOAcc - 1)), tmem_base + t * 256 + ks * 8,
+                           make_sdesc_sw64(va + ks * 16 * kRowBytes, 512), idesc_pv, ks >= kOAcc ? 1u : 0u);
+                mma_commit(bar_oready(t));
+            };
+            long long it = blockIdx.x;
+            Item cur;
+            if (it < n_items) {
+                cur = make_item(g, it);
+                ok = mbar_wait(bar_full(0), 0, cta_abort);
+                if (ok) {
+                    fence_proxy_async();
+                    tc_fence_after();
+                    for (int t = 0; t < cur.ntiles; ++t) issue_qk(cur, 0, t);   // TMEM regions start out free
+                }
+            }
+            for (; ok && it < n_items; it += gridDim.x, ++kuse) {
+                const int s = kuse % kStages;
+                const long long nxt = it + gridDim.x;
+                const bool has_next = nxt < n_items;
+                Item nx;
+                const int sn = (kuse + 1) % kStages;
+                if (has_next) nx = make_item(g, nxt);
+                bool next_ready = false;
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    if (!ok) break;
+                    if (t < cur.ntiles) {
+                        ok = mbar_wait(bar_pready(t), use_t[t] & 1, cta_abort);   // use_t[t] still counts earlier uses only
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_pv(cur, s, t);
+                        if (t == cur.ntiles - 1) mma_commit(bar_empty(s));   // all operands of this stage consumed
+                    }
+                    if (has_next && t < nx.ntiles) {
+                        if (!next_ready) {
+                            ok = mbar_wait(bar_full(sn), ((kuse + 1) / kStages) & 1, cta_abort);
+                            if (!ok) break;
+                            fence_proxy_async();
+                            next_ready = true;
+                        }
+                        if (t < cur.ntiles) ++use_t[t];
+                        // region t is free once its softmax warpgroup has read O of the last item that used it
+                        while (ok && freed_t[t] < use_t[t]) {
+                            ok = mbar_wait(bar_sfree(t), freed_t[t] & 1, cta_abort);
+                            ++freed_t[t];
+                        }
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_qk(nx, sn, t);
+                    } else if (t < cur.ntiles) {
+                        ++use_t[t];
+                    }
+                }
+                cur = nx;
+            }
+        }
+    }
+    } else {
+        // ------------------------------------------------------------------ softmax warpgroups
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(kRegsSoftmax));
+        const int wg = warp >> 2;
+        const int row = tid & 127;
+        const int slot = wg * 128 + row;
+        const uint32_t lane_addr = ((uint32_t)(32 * (warp & 3))) << 16;
+        const uint32_t t_s = tmem_base + lane_addr + wg * 256;
+        const float scale = g.scale_log2e;
+        int kuse = 0, use = 0;
+        for (long long it = blockIdx.x; it < n_items; it += gridDim.x, ++kuse) {
+            const Item x = make_item(g, it);
+            if (wg >= x.ntiles) continue;
+            const int s = kuse % kStages;
+            const uint32_t st_a = smem0 + s * kStageBytes;
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_full(s), (kuse / kStages) & 1, cta_abort))) break;
+            const int rmeta = lds_i32(st_a + kOffRowMeta + 4 * slot);
+            const int tok = lds_i32(st_a + kOffRowTok + 4 * slot);
+            const uint32_t bias_i = st_a + kOffBias + 4 * meta_code(rmeta);
+            const int label_i = meta_label(rmeta);
+            const float bmax = lds_f32(st_a + kOffBias + 4 * (kFwdBiasFloats - 1));
+
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_sready(wg), use & 1, cta_abort))) break;
+            tc_fence_after();
+            float m, sum;
+            if (x.masked) m = softmax_row<true>(t_s, x.npad, bias_i, st_a + kOffKc, st_a + kOffKlab, label_i, scale, bmax, sum);
+            else m = softmax_row<false>(t_s, x.npad, bias_i, st_a + kOffKc, st_a + kOffKlab, label_i, scale, bmax, sum);
+            tmem_st_wait();
+            tc_fence_before();
+            mbar_arrive(bar_pready(wg));
+
+            const size_t row_off = ((size_t)x.b * HW + (size_t)(tok < 0 ? 0 : tok)) * g.heads + x.head;
+            if (tok >= 0) lse[row_off] = (m + log2f(sum)) * kLn2;
+            const float inv = 1.f / sum;
+            const int nacc = min(kOAcc, x.npad >> 4);
+
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_oready(wg), use & 1, cta_abort))) break;
+            tc_fence_after();
+            uint32_t ro[32];
+            tmem_ld32(t_s + kColO, ro);
+            tmem_ld_wait();
+#pragma unroll
+            for (int a = 1; a < kOAcc; ++a) {
+                if (a >= nacc) break;
+                uint32_t rx[32];
+                tmem_ld32(t_s + kColO + 32 * a, rx);
+                tmem_ld_wait();
+#pragma unroll
+                for (int e = 0; e < 32; ++e) ro[e] = __float_as_uint(__uint_as_float(ro[e]) + __uint_as_float(rx[e]));
+            }
+            tc_fence_before();
+            mbar_arrive(bar_sfree(wg));
+            ++use;
+            if (tok >= 0) {
+                uint4* dst = reinterpret_cast<uint4*>(o + row_off * kD);
+#pragma unroll
+                for (int c4 = 0; c4 < 4; ++c4) {
+                    uint4 val;
+                    val.x = pack_bf16(__uint_as_float(ro[c4 * 8 + 0]) * inv, __uint_as_float(ro[c4 * 8 + 1]) * inv);
+                    val.y = pack_bf16(__uint_as_float(ro[c4 * 8 + 2]) * inv, __uint_as_float(ro[c4 * 8 + 3]) * inv);
+                    val.z = pack_bf16(__uint_as_float(ro[c4 * 8 + 4]) * inv, __uint_as_float(ro[c4 * 8 + 5]) * inv);
+                    val.w = pack_bf16(__uint_as_float(ro[c4 * 8 + 6]) * inv, __uint_as_float(ro[c4 * 8 + 7]) * inv);
+                    dst[c4] = val;
+                }
+            }
+        }
+    }
+
+    // teardown: every role ends up here, also after an expired wait
+    cp_async_wait<0>();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == kMmaWarp) tmem_dealloc(tmem_base, 512);
+    if (tid == 0 && *cta_abort) atomicExch(&g_tc_timeout, 1);
+}
+
+// Per head, with code stride cs = w + 32 and c0 = (w - 1) * (cs + 1):
+//   table[(da + w - 1) * cs + (db + w - 1)] = T[(da + w - 1) * (2w - 1) + (db + w - 1), head] * log2(e)
+//   for |da|, |db| < w (unused gaps 0), table[2 c0 + 1 .. 3 c0 + 1] = -inf (where key slots without a
+//   token point), and the head's largest entry in the last float.
+__global__ void __launch_bounds__(256)
+swin_fwd_bias_prep_kernel(const float* __restrict__ bias, float* __restrict__ prep, int w, int heads) {
+    const int head = blockIdx.x;
+    const int cs = w + 32, nw = 2 * w - 1;
+    const int c0 = (w - 1) * (cs + 1);
+    float* dst = prep + (size_t)head * kFwdBiasFloats;
+    float mx = -INFINITY;
+    for (int e = threadIdx.x; e < kFwdBiasFloats - 1; e += blockDim.x) {
+        float val = 0.f;
+        if (e > 2 * c0) {
+            val = -INFINITY;
+        } else {
+            const int ra = e / cs, rb = e - ra * cs;
+            if (rb < nw) {
+                val = bias[(size_t)(ra * nw + rb) * heads + head] * kLog2e;
+                mx = fmaxf(mx, val);
+            }
+        }
+        dst[e] = val;
+    }
+    __shared__ float red[8];
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = mx;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int i = 1; i < 8; ++i) mx = fmaxf(mx, red[i]);
+        dst[kFwdBiasFloats - 1] = mx;
+    }
+}
+
+}  // namespace
+
+bool fwd_tc_supported(const Geo& g) { return g.d == 32 && g.nmax <= kMaxSlots && g.w <= 16; }
+
+size_t fwd_tc_workspace_bytes(const Geo& g) { return (size_t)g.heads * kFwdBiasFloats * sizeof(float); }
+
+cudaError_t launch_fwd_tc(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
+                          void* o, float* lse, void* workspace, int sm_count, cudaStream_t stream) {
+    const long long items = (long long)g.B * g.Mh * g.Mw * g.heads;
+    float* prep = reinterpret_cast<float*>(workspace);
+    swin_fwd_bias_prep_kernel<<<g.heads, 256, 0, stream>>>(bias, prep, g.w, g.heads);
+    count_launch();
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(swin_fwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    const unsigned grid = (unsigned)(items < sm_count ? items : sm_count);
+    swin_fwd_tc_kernel<<<grid, kThreads, kSmemBytes, stream>>>(g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k,
+                                                               (const __nv_bfloat16*)v, prep, (__nv_bfloat16*)o, lse, items);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t read_tc_status(int* timed_out, cudaStream_t stream) {
+    cudaError_t e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) return e;
+    int zero = 0;
+    e = cudaMemcpyFromSymbol(timed_out, g_tc_timeout, sizeof(int));
+    if (e != cudaSuccess) return e;
+    if (*timed_out) e = cudaMemcpyToSymbol(g_tc_timeout, &zero, sizeof(int));
+    return e;
+}
+
+}  // namespace terra

@@ -16,6 +16,15 @@ cudaError_t launch_route(const Geo& g, int32_t* perm, int32_t* inv_perm, int32_t
 cudaError_t launch_fwd_mma(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
                            void* o, float* lse, cudaStream_t stream);
 
+// tcgen05 forward path (head dim 32, window side <= 16)
+constexpr int kFwdBiasFloats = 2304;   // prepared bias table per head (padded rows, -inf zone, maximum in the last float)
+bool fwd_tc_supported(const Geo& g);
+size_t fwd_tc_workspace_bytes(const Geo& g);
+cudaError_t launch_fwd_tc(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
+                          void* o, float* lse, void* workspace, int sm_count, cudaStream_t stream);
+// synchronises the stream, reads and clears the device-side "a bounded wait expired" word
+cudaError_t read_tc_status(int* timed_out, cudaStream_t stream);
+
 // delta[b, token, head] = sum_c dO * O   (fp32, same indexing as lse)
 cudaError_t launch_bwd_delta(const Geo& g, const void* o, const void* d_o, float* delta, cudaStream_t stream);
 

@@ -17,10 +17,13 @@ def gate(name, got, ref, strict=True):
     ref = np.asarray(ref, dtype=np.float64)
     assert got.shape == ref.shape, (name, got.shape, ref.shape)
     assert np.all(np.isfinite(got)), f"{name}: non-finite values in the GPU result"
-    # inputs are N(0, 1): a reference that is identically zero (single-token windows give dQ = dK = 0)
-    # is compared on the scale of fp32 rounding of O(1) terms instead of on a zero scale
-    scale = max(np.abs(ref).max(), 1e-3)
     err = np.abs(got - ref)
+    if np.abs(ref).max() < 1e-9:
+        # structurally zero reference (single-token windows: dQ = dK = 0).  The GPU value is the rounding
+        # residue of dP - delta, where delta uses the saved bf16 O: |dO| |O| 2^-9 |k| scale ~ 1e-2 for N(0, 1) inputs
+        assert err.max() <= 2e-2, f"{name}: zero reference, |got| up to {err.max():.3e}"
+        return float(err.max())
+    scale = np.abs(ref).max()
     assert err.max() <= G1_ABS * scale, f"{name}: G1 max|err| {err.max():.3e} > {G1_ABS * scale:.3e}"
     assert np.all(err <= G1_ABS * scale + G2_REL * np.abs(ref)), f"{name}: G2 failed"
     if strict:

@@ -33,13 +33,13 @@ def _to_gpu(x):
 def _run_fwd(cfg, xg, scale=0.0):
     d = terra.make_desc(cfg, scale)
     o, lse = terra.terra_swin_attn_fwd(d, xg["q"], xg["k"], xg["v"], xg["bias"])
-    torch.cuda.synchronize()
+    terra.terra_swin_check()          # synchronises; raises if a kernel gave up on a bounded wait
     return d, o, lse
 
 
 def _run_bwd(cfg, d, xg, o, lse):
     out = terra.terra_swin_attn_bwd(d, xg["q"], xg["k"], xg["v"], xg["bias"], o, lse, xg["do"])
-    torch.cuda.synchronize()
+    terra.terra_swin_check()
     return out
 
 
