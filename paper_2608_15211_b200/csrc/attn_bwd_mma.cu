@@ -4,9 +4,13 @@
 // CTAs produce dQ and the relative-position-bias gradient.  (2) and (3) are one kernel template: a
 // CTA owns 64 rows of one side of the window (keys or queries), streams the other side through
 // shared memory in 64-row blocks, recomputes P from the saved log-sum-exp and forms
-// dS = P * (dP - delta).  No atomics touch dQ / dK / dV, so those are reproducible run to run; the
-// bias gradient is summed per CTA in shared memory (CTAs are persistent and bound to one head) and
-// flushed once with global atomics.
+// dS = P * (dP - delta).  No atomics touch dQ / dK / dV, so those are reproducible run to run.
+// Bias gradient: a query-tile CTA is persistent and bound to one (head, query tile).  For full-width
+// windows the position of a (query, key) pair inside the tile decides its table row, whatever the
+// window, so the CTA first adds dS element by element into a 64 x n shared-memory image that it owns
+// (no atomics, no conflicts) over all its windows, and bins that image into the (2w-1)^2 table once at
+// the end.  Narrow edge windows, and windows too large for the image, add straight into the table with
+// shared-memory atomics.  Each CTA then flushes its table with global atomics.
 #include "swin_common.cuh"
 #include "swin_kernels.h"
 
@@ -111,7 +115,7 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
                     const __nv_bfloat16* __restrict__ v, const __nv_bfloat16* __restrict__ d_o,
                     const float* __restrict__ bias, const float* __restrict__ lse, const float* __restrict__ delta,
                     __nv_bfloat16* __restrict__ out1, __nv_bfloat16* __restrict__ out2, float* __restrict__ dbias,
-                    int tiles, int ctas_per_head) {
+                    int tiles, int ctas_per_group, int acc_stride) {
     constexpr int KS = D / 16;
     constexpr int DT = D / 8;
     constexpr int TILE_BYTES = BN * D * 2;
@@ -129,13 +133,20 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
     unsigned char* s_r2 = s_r1 + TILE_BYTES;
     unsigned char* s_c1 = s_r2 + TILE_BYTES;          // two stages
     unsigned char* s_c2 = s_c1 + 2 * TILE_BYTES;      // two stages
+    float* s_acc = reinterpret_cast<float*>(s_c2 + 2 * TILE_BYTES);   // 64 x acc_stride image of summed dS (query tiles only)
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int gq = lane >> 2, tq = lane & 3;
-    const int head = blockIdx.x % g.heads;
+    // KV: group = head, the CTA walks (batch, window, tile).  Query side: group = (head, tile), the CTA
+    // walks (batch, window), so one CTA always sees the same rows of a window.
+    const int groups = KV ? g.heads : g.heads * tiles;
+    const int group = blockIdx.x % groups;
+    const int head = KV ? group : group / tiles;
+    const int fixed_tile = KV ? 0 : group % tiles;
     const int M = g.Mh * g.Mw;
     const int c0 = (g.w - 1) * 2 * g.w;
-    const long long n_items = (long long)g.B * M * tiles;
+    const long long n_items = KV ? (long long)g.B * M * tiles : (long long)g.B * M;
+    const bool use_acc = !KV && acc_stride > 0;
 
     const __nv_bfloat16* own1 = KV ? k : q;
     const __nv_bfloat16* own2 = KV ? v : d_o;
@@ -146,11 +157,13 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
         s_bias[i] = bias[(size_t)i * g.heads + head] * kLog2e;
         s_dbias[i] = 0.f;
     }
+    if (use_acc)
+        for (int i = tid; i < BM * acc_stride; i += NTHREADS) s_acc[i] = 0.f;
 
-    for (long long item = blockIdx.x / g.heads; item < n_items; item += ctas_per_head) {
-        const int tile = (int)(item % tiles);
-        const int win = (int)((item / tiles) % M);
-        const int b = (int)(item / ((long long)tiles * M));
+    for (long long item = blockIdx.x / groups; item < n_items; item += ctas_per_group) {
+        const int tile = KV ? (int)(item % tiles) : fixed_tile;
+        const int win = KV ? (int)((item / tiles) % M) : (int)(item % M);
+        const int b = KV ? (int)(item / ((long long)tiles * M)) : (int)(item / M);
         const WindowRef r = window_ref(g, win);
         const int r0 = tile * BM;
         if (r0 >= r.n) continue;
@@ -241,7 +254,21 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
                     const float ds = p * (acc_dp[nt][e] - dl);
                     acc_s[nt][e] = p;
                     acc_dp[nt][e] = ds;
-                    if (!KV && ok && p != 0.f) atomicAdd(&s_dbias[bidx], ds);
+                    if (!KV && !(use_acc && r.ew == g.w) && ok && p != 0.f) atomicAdd(&s_dbias[bidx], ds);
+                }
+            }
+            if (!KV && use_acc && r.ew == g.w) {
+                // this thread owns these image cells: plain read-modify-write, 8-byte accesses
+#pragma unroll
+                for (int nt = 0; nt < BN / 8; ++nt) {
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        float2* cell = reinterpret_cast<float2*>(s_acc + (warp * 16 + gq + 8 * h) * acc_stride + blk * BN + nt * 8 + 2 * tq);
+                        float2 cur = *cell;
+                        cur.x += acc_dp[nt][2 * h];
+                        cur.y += acc_dp[nt][2 * h + 1];
+                        *cell = cur;
+                    }
                 }
             }
             if constexpr (KV) {
@@ -264,6 +291,21 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
 
     if (!KV) {
         __syncthreads();
+        if (use_acc) {
+            // bin the image: cell (row, col) of a full-width window belongs to table row code(row) - code(col) + c0
+            const int n_full = g.nmax;
+            for (int cell = tid; cell < BM * n_full; cell += NTHREADS) {
+                const int row = cell / n_full, col = cell - row * n_full;
+                const int slot = fixed_tile * BM + row;
+                if (slot >= n_full) continue;
+                const float val = s_acc[row * acc_stride + col];
+                if (val == 0.f) continue;
+                const int code_r = (slot / g.w) * (2 * g.w - 1) + slot % g.w;
+                const int code_c = (col / g.w) * (2 * g.w - 1) + col % g.w;
+                atomicAdd(&s_dbias[code_r - code_c + c0], val);
+            }
+            __syncthreads();
+        }
         for (int i = tid; i < nbias; i += NTHREADS) {
             float val = s_dbias[i];
             if (val != 0.f) atomicAdd(&dbias[(size_t)i * g.heads + head], val);
@@ -297,11 +339,19 @@ swin_bwd_delta_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloat16* 
     if (row < rows && chunk == 0) delta[row] = acc;
 }
 
-size_t bwd_smem_bytes(const Geo& g) {
+// Row stride (floats) of the summed-dS image, or 0 when the window is too large for it.  The stride is
+// 8 mod 32 so that the 16 lanes of one 8-byte access wave hit 32 different banks.
+int acc_stride_for(const Geo& g) {
+    int npad_max = ((g.nmax + BN - 1) / BN) * BN;
+    return npad_max <= 256 ? npad_max + 8 : 0;
+}
+
+size_t bwd_smem_bytes(const Geo& g, bool query_side) {
     int npad_max = ((g.nmax + BN - 1) / BN) * BN;
     int nbias = (2 * g.w - 1) * (2 * g.w - 1);
     size_t head = (((size_t)npad_max * 16 + (size_t)nbias * 8 + 127) / 128) * 128;
-    return head + 6 * (size_t)BN * g.d * 2;
+    size_t acc = query_side ? (size_t)BM * acc_stride_for(g) * sizeof(float) : 0;
+    return head + 6 * (size_t)BN * g.d * 2 + acc;
 }
 
 template <int D, bool KV>
@@ -309,7 +359,7 @@ cudaError_t launch_one(const Geo& g, const void* q, const void* k, const void* v
                        const float* lse, const float* delta, void* out1, void* out2, float* dbias, int sm_count,
                        cudaStream_t stream) {
     auto kern = swin_bwd_mma_kernel<D, KV>;
-    const size_t smem = bwd_smem_bytes(g);
+    const size_t smem = bwd_smem_bytes(g, !KV);
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     int occ = 0;
@@ -317,13 +367,14 @@ cudaError_t launch_one(const Geo& g, const void* q, const void* k, const void* v
     if (e != cudaSuccess) return e;
     if (occ < 1) occ = 1;
     const int tiles = (g.nmax + BM - 1) / BM;
-    const long long items = (long long)g.B * g.Mh * g.Mw * tiles;
-    long long cph = ((long long)sm_count * occ) / g.heads;     // persistent CTAs bound to each head
-    if (cph < 1) cph = 1;
-    if (cph > items) cph = items;
-    kern<<<(unsigned)(cph * g.heads), NTHREADS, smem, stream>>>(
+    const int groups = KV ? g.heads : g.heads * tiles;          // what a persistent CTA is bound to
+    const long long items = KV ? (long long)g.B * g.Mh * g.Mw * tiles : (long long)g.B * g.Mh * g.Mw;
+    long long cpg = ((long long)sm_count * occ) / groups;
+    if (cpg < 1) cpg = 1;
+    if (cpg > items) cpg = items;
+    kern<<<(unsigned)(cpg * groups), NTHREADS, smem, stream>>>(
         g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)d_o, bias,
-        lse, delta, (__nv_bfloat16*)out1, (__nv_bfloat16*)out2, dbias, tiles, (int)cph);
+        lse, delta, (__nv_bfloat16*)out1, (__nv_bfloat16*)out2, dbias, tiles, (int)cpg, KV ? 0 : acc_stride_for(g));
     count_launch();
     return cudaGetLastError();
 }
