@@ -254,20 +254,38 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
                     const float ds = p * (acc_dp[nt][e] - dl);
                     acc_s[nt][e] = p;
                     acc_dp[nt][e] = ds;
-                    if (!KV && !(use_acc && r.ew == g.w) && ok && p != 0.f) atomicAdd(&s_dbias[bidx], ds);
                 }
             }
-            if (!KV && use_acc && r.ew == g.w) {
-                // this thread owns these image cells: plain read-modify-write, 8-byte accesses
+            if (!KV) {
+                if (use_acc && r.ew == g.w) {
+                    // this thread owns these image cells: plain read-modify-write with 8-byte accesses,
+                    // all loads first so that they overlap
+                    float2* cell0 = reinterpret_cast<float2*>(s_acc + (warp * 16 + gq) * acc_stride + blk * BN + 2 * tq);
+                    float2 cur[BN / 8][2];
 #pragma unroll
-                for (int nt = 0; nt < BN / 8; ++nt) {
+                    for (int nt = 0; nt < BN / 8; ++nt) {
+                        cur[nt][0] = cell0[nt * 4];
+                        cur[nt][1] = cell0[nt * 4 + 4 * acc_stride];
+                    }
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        float2* cell = reinterpret_cast<float2*>(s_acc + (warp * 16 + gq + 8 * h) * acc_stride + blk * BN + nt * 8 + 2 * tq);
-                        float2 cur = *cell;
-                        cur.x += acc_dp[nt][2 * h];
-                        cur.y += acc_dp[nt][2 * h + 1];
-                        *cell = cur;
+                    for (int nt = 0; nt < BN / 8; ++nt) {
+                        cur[nt][0].x += acc_dp[nt][0]; cur[nt][0].y += acc_dp[nt][1];
+                        cur[nt][1].x += acc_dp[nt][2]; cur[nt][1].y += acc_dp[nt][3];
+                    }
+#pragma unroll
+                    for (int nt = 0; nt < BN / 8; ++nt) {
+                        cell0[nt * 4] = cur[nt][0];
+                        cell0[nt * 4 + 4 * acc_stride] = cur[nt][1];
+                    }
+                } else {
+#pragma unroll
+                    for (int nt = 0; nt < BN / 8; ++nt) {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int mc = s_meta[blk * BN + nt * 8 + 2 * tq + (e & 1)];
+                            const int mr = meta_r[e >> 1];
+                            if (acc_dp[nt][e] != 0.f) atomicAdd(&s_dbias[meta_code(mr) - meta_code(mc) + c0], acc_dp[nt][e]);
+                        }
                     }
                 }
             }
