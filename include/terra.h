@@ -40,8 +40,12 @@ typedef enum {
     TERRA_ERR_ALIGNMENT = 3,     /* a pointer is not 16-byte aligned                              */
     TERRA_ERR_WORKSPACE = 4,     /* workspace NULL or smaller than terra_swin_workspace_bytes     */
     TERRA_ERR_CUDA = 5,          /* a CUDA call failed; text via terra_last_cuda_error            */
-    TERRA_ERR_DEVICE_TIMEOUT = 6 /* a bounded wait inside a kernel expired (see terra_swin_check) */
+    TERRA_ERR_DEVICE_TIMEOUT = 6,/* a bounded wait inside a kernel expired (see terra_swin_check) */
+    TERRA_ERR_NOALLOC_LIMIT = 7  /* terra_swin_attn_fwd_noalloc: more heads than its fixed scratch holds */
 } terra_status;
+
+/* Largest `heads` terra_swin_attn_fwd_noalloc accepts on the shapes that need scratch. */
+#define TERRA_NOALLOC_MAX_HEADS 64
 
 /* Problem statement: token grid, window, heads (paper Table I symbols; H, W here are H_T, W_T). */
 typedef struct {
@@ -106,6 +110,31 @@ int terra_swin_attn_bwd(const terra_swin_desc* desc, const void* q, const void* 
                         const float* bias_table, const void* o, const float* lse, const void* d_o,
                         void* dq, void* dk, void* dv, float* dbias,
                         void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Forward pass without a workspace argument.  (The paper has no counterpart: this exists for the way the
+ * library is embedded, not for the method.)
+ *
+ * Who needs it: code that runs where device memory may not be requested -- a plug-in inside a serving
+ * process whose memory is owned by a pool it cannot reach, a real-time loop that was handed all of its
+ * buffers up front, a callback from which cudaMalloc is off limits.  Such a caller still brings the inputs
+ * and outputs, but has nowhere to get the forward kernel's scratch (one prepared bias table per head) from.
+ * Here that scratch is a fixed array compiled into the library: TERRA_NOALLOC_MAX_HEADS * 9216 bytes
+ * (576 KiB) on every GPU that loads the library, held until the process exits.  The call allocates nothing:
+ * no cudaMalloc / cudaFree, no allocating library routine.
+ *
+ * Arguments, layouts, results and error codes are those of terra_swin_attn_fwd; the output is the same.
+ * Extra rules:
+ *   - heads > TERRA_NOALLOC_MAX_HEADS is refused with TERRA_ERR_NOALLOC_LIMIT when the shape uses the
+ *     scratch (head_dim 32, window <= 16); other shapes need no scratch and are not limited;
+ *   - the first call on each device looks the array's device address up (the device must be current);
+ *     make that first call before any stream capture begins;
+ *   - all calls on a device share the one array and every call rewrites the part it uses, so nothing has to
+ *     be cleared in between; but two calls that overlap on the GPU (different streams) race on it and give
+ *     wrong results -- keep calls to this entry point ordered on one stream per device.
+ */
+int terra_swin_attn_fwd_noalloc(const terra_swin_desc* desc, const void* q, const void* k, const void* v,
+                                const float* bias_table, void* o, float* lse, void* stream);
 
 /*
  * Waits for `stream` and reports whether any kernel of this library gave up on a bounded wait since

@@ -16,7 +16,7 @@ from .build import LIB_PATH
 
 TERRA_OK = 0
 EXPORTS = ("terra_route_sizes", "terra_window_route", "terra_swin_workspace_bytes", "terra_swin_attn_fwd",
-           "terra_swin_attn_bwd", "terra_swin_check", "terra_strerror", "terra_last_cuda_error",
+           "terra_swin_attn_fwd_noalloc", "terra_swin_attn_bwd", "terra_swin_check", "terra_strerror", "terra_last_cuda_error",
            "terra_launch_count")
 
 
@@ -52,8 +52,9 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
     lib.terra_swin_workspace_bytes.argtypes = [dp, ctypes.c_int, ctypes.POINTER(ctypes.c_size_t)]
     lib.terra_swin_attn_fwd.argtypes = [dp] + [vp] * 6 + [vp, ctypes.c_size_t, vp]
     lib.terra_swin_attn_bwd.argtypes = [dp] + [vp] * 11 + [vp, ctypes.c_size_t, vp]
+    lib.terra_swin_attn_fwd_noalloc.argtypes = [dp] + [vp] * 6 + [vp]
     for n in ("terra_route_sizes", "terra_window_route", "terra_swin_workspace_bytes", "terra_swin_attn_fwd",
-              "terra_swin_attn_bwd"):
+              "terra_swin_attn_fwd_noalloc", "terra_swin_attn_bwd"):
         getattr(lib, n).restype = ctypes.c_int
     lib.terra_swin_check.argtypes = [vp]
     lib.terra_swin_check.restype = ctypes.c_int
@@ -149,6 +150,20 @@ def terra_swin_attn_fwd(desc, q, k, v, bias_table, o=None, lse=None, workspace=N
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     _check(load_library().terra_swin_attn_fwd(ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(v), _ptr(bias_table),
                                               _ptr(o), _ptr(lse), _ptr(workspace), ws_bytes, _stream()))
+    return o, lse
+
+
+def terra_swin_attn_fwd_noalloc(desc, q, k, v, bias_table, o, lse):
+    """Forward into caller-provided o / lse with no workspace: the library's built-in scratch is used and
+    nothing is allocated, by this binding or by the library (see include/terra.h for who needs this and
+    for its limits: at most TERRA_NOALLOC_MAX_HEADS heads, calls on one device must not overlap)."""
+    n = desc.B * desc.H * desc.W * desc.heads
+    for name, t in (("q", q), ("k", k), ("v", v), ("o", o)):
+        _expect(t, torch.bfloat16, n * desc.head_dim, name)
+    _expect(bias_table, torch.float32, (2 * desc.window - 1) ** 2 * desc.heads, "bias_table")
+    _expect(lse, torch.float32, n, "lse")
+    _check(load_library().terra_swin_attn_fwd_noalloc(ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(v), _ptr(bias_table),
+                                                      _ptr(o), _ptr(lse), _stream()))
     return o, lse
 
 

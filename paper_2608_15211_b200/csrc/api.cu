@@ -86,6 +86,12 @@ static size_t delta_bytes(const Geo& g) {
     return align_up(sizeof(float) * (size_t)g.B * g.H * g.W * g.heads, 256);
 }
 
+// Descriptor check + geometry, and the SM count of the current device, for entry points that live in
+// other files of the library.
+int resolve_attention_geo(const terra_swin_desc* d, Geo* out) { return make_geo(d, true, out); }
+int current_device_sm_count(int* sm_count) { return device_props(sm_count); }
+int report_cuda_failure(cudaError_t e, const char* where) { return cuda_fail(e, where); }
+
 }  // namespace terra
 
 using namespace terra;
@@ -185,6 +191,7 @@ const char* terra_strerror(int status) {
         case TERRA_ERR_WORKSPACE: return "workspace missing or too small (see terra_swin_workspace_bytes)";
         case TERRA_ERR_CUDA: return "CUDA error (see terra_last_cuda_error)";
         case TERRA_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel expired; results of that call are invalid";
+        case TERRA_ERR_NOALLOC_LIMIT: return "terra_swin_attn_fwd_noalloc: heads exceeds TERRA_NOALLOC_MAX_HEADS, the size of its fixed scratch";
         default: return "unknown status";
     }
 }
