@@ -82,7 +82,10 @@ static size_t fwd_bytes(const Geo& g) {
     return (fwd_tc_supported(g) && !force_register_path()) ? align_up(fwd_tc_workspace_bytes(g), 256) : 0;
 }
 
+static bool use_bwd_tc(const Geo& g) { return bwd_tc_supported(g) && !force_register_path(); }
+
 static size_t delta_bytes(const Geo& g) {
+    if (use_bwd_tc(g)) return align_up(bwd_tc_workspace_bytes(g), 256);
     return align_up(sizeof(float) * (size_t)g.B * g.H * g.W * g.heads, 256);
 }
 
@@ -168,6 +171,10 @@ int terra_swin_attn_bwd(const terra_swin_desc* desc, const void* q, const void* 
     rc = device_props(&sms);
     if (rc) return rc;
     cudaStream_t st = (cudaStream_t)stream;
+    if (use_bwd_tc(g)) {
+        cudaError_t et = launch_bwd_tc(g, q, k, v, bias_table, o, lse, d_o, dq, dk, dv, dbias, workspace, sms, st);
+        return et == cudaSuccess ? TERRA_OK : cuda_fail(et, "terra_swin_attn_bwd");
+    }
     float* delta = reinterpret_cast<float*>(workspace);
     cudaError_t e = launch_bwd_delta(g, o, d_o, delta, st);
     if (e != cudaSuccess) return cuda_fail(e, "terra_swin_attn_bwd (delta)");
@@ -179,7 +186,10 @@ int terra_swin_check(void* stream) {
     int timed_out = 0;
     cudaError_t e = read_tc_status(&timed_out, (cudaStream_t)stream);
     if (e != cudaSuccess) return cuda_fail(e, "terra_swin_check");
-    return timed_out ? TERRA_ERR_DEVICE_TIMEOUT : TERRA_OK;
+    int timed_out_bwd = 0;
+    e = read_bwd_tc_status(&timed_out_bwd);
+    if (e != cudaSuccess) return cuda_fail(e, "terra_swin_check");
+    return (timed_out || timed_out_bwd) ? TERRA_ERR_DEVICE_TIMEOUT : TERRA_OK;
 }
 
 const char* terra_strerror(int status) {

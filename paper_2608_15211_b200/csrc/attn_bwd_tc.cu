@@ -1,0 +1,622 @@
+// Backward shifted-window attention on the tcgen05 tensor cores (head dim 32, windows of <= 256 tokens).
+//
+// One kernel template, launched twice per call:
+//   query side (KV = false): rows = queries.  S = Q K^T and dP = dO V^T per key block, dS = P (dP - delta)
+//                            written to TMEM as bf16, dQ += dS K (dS read from TMEM); the bias gradient is
+//                            summed in a per-CTA shared-memory table and flushed once with global atomics.
+//   key side   (KV = true):  rows = keys.  S^T = K Q^T and dP^T = V dO^T per query block, P^T and dS^T
+//                            written to TMEM as bf16, dV += P^T dO and dK += dS^T Q.
+// P is recomputed from the saved log-sum-exp, so the column blocks of a row are independent (no running
+// maximum).  Structure as in the forward kernel: persistent CTAs, two 128-row tiles (one per elementwise
+// warpgroup, one thread per row), one MMA-issuing lane, three loader warps gathering the window's rows with
+// cp.async into the 64-byte-swizzled operand layout.  CTAs are bound to one head (grid = heads x CTAs per
+// head), so the head's bias table is staged once per CTA and the bias-gradient table belongs to one head.
+// TMEM, per 128-row tile (256 columns):  query side [S 112 | dP 112 | dQ 32], key side
+// [S^T 96 | dP^T 96 | dV 32 | dK 32]; the bf16 P / dS overwrite the fp32 S / dP they were computed from.
+// Every mbarrier wait is bounded; on expiry the CTA raises an abort flag and all roles leave their loops.
+#include "swin_common.cuh"
+#include "swin_kernels.h"
+#include "tc_common.cuh"
+
+namespace terra {
+
+__device__ int g_bwd_tc_timeout = 0;   // set when a bounded wait expired in any CTA of the kernels below
+
+namespace {
+
+using namespace tc;
+
+constexpr int kMmaWarp = 8;
+constexpr int kLoaderWarp0 = 9;
+constexpr int kLoaderWarps = 3;
+constexpr int kLoaderThreads = kLoaderWarps * 32;
+constexpr int kThreads = (kLoaderWarp0 + kLoaderWarps) * 32;   // 384 = three warpgroups
+constexpr int kRegsLaunch = 168;
+constexpr int kRegsWork = 216;      // elementwise warpgroups after setmaxnreg.inc
+constexpr int kRegsOther = 64;      // MMA + loader warpgroup after setmaxnreg.dec
+static_assert(2 * (kRegsWork - kRegsLaunch) <= (kRegsLaunch - kRegsOther), "register hand-over does not balance");
+
+constexpr int kStages = 2;
+constexpr int kMaxSlots = 256;
+constexpr int kD = 32;
+constexpr int kRowBytes = kD * 2;
+constexpr int kTileBytes = kMaxSlots * kRowBytes;              // 16384
+
+// stage layout (bytes)
+constexpr int kOffQ = 0;
+constexpr int kOffK = kTileBytes;
+constexpr int kOffV = 2 * kTileBytes;
+constexpr int kOffDO = 3 * kTileBytes;
+constexpr int kOffColOff = 4 * kTileBytes;                     // per slot as a column: byte offset into the bias table
+constexpr int kOffLab = kOffColOff + kMaxSlots * 4;            // per slot: shift-mask label (0xff: no token)
+constexpr int kOffCode = kOffLab + kMaxSlots * 4;              // per slot: bias code a * (w + 32) + b
+constexpr int kOffTok = kOffCode + kMaxSlots * 4;              // per slot: grid token, -1 if none
+constexpr int kOffLse = kOffTok + kMaxSlots * 4;               // per slot: lse * log2(e), +inf if none
+constexpr int kOffDelta = kOffLse + kMaxSlots * 4;             // per slot: delta
+constexpr int kStageBytes = ((kOffDelta + kMaxSlots * 4 + 1023) / 1024) * 1024;   // 71680
+// after the stages
+constexpr int kOffBias = kStages * kStageBytes;                // the head's prepared bias table (kFwdBiasFloats floats)
+constexpr int kOffDBias = kOffBias + kFwdBiasFloats * 4;       // query side: bias-gradient table, same indexing
+constexpr int kDBiasFloats = 1536;                             // >= 2 c0 + 1 for w <= 16
+constexpr int kOffBars = kOffDBias + kDBiasFloats * 4;
+constexpr int kSmemBytes = kOffBars + 256;
+
+__device__ __forceinline__ int code_stride(int w) { return w + 32; }
+
+struct Item {
+    int b, win;
+    WindowRef r;
+    int npad;      // slots rounded up to 16
+    int ntiles;    // 128-row tiles in use
+    bool masked;   // the window mixes shift-mask labels
+    bool ragged;   // some row of a 128-row tile, or some column below npad, has no token
+};
+
+__device__ __forceinline__ Item make_item(const Geo& g, long long it) {
+    Item x;
+    const int M = g.Mh * g.Mw;
+    x.win = (int)(it % M);
+    x.b = (int)(it / M);
+    x.r = window_ref(g, x.win);
+    x.npad = (x.r.n + 15) & ~15;
+    x.ntiles = (x.r.n + 127) >> 7;
+    const int r0 = x.r.wr * g.w, c0 = x.r.wc * g.w;
+    const bool mh = !g.ph && g.sh > 0 && r0 < g.H - g.sh && r0 + x.r.eh > g.H - g.sh;
+    const bool mw = !g.pw && g.sw > 0 && c0 < g.W - g.sw && c0 + x.r.ew > g.W - g.sw;
+    x.masked = mh || mw;
+    x.ragged = x.npad != x.r.n || x.r.n != x.ntiles * 128;   // some row of a tile or some column has no token
+    return x;
+}
+
+__device__ __forceinline__ int slot_token_tc(const Geo& g, const WindowRef& r, int slot, int& code, int& label) {
+    const int a = slot / r.ew;
+    const int b = slot - a * r.ew;
+    int u = r.wr * g.w + a + g.sh;
+    if (u >= g.H) u -= g.H;
+    int v = r.wc * g.w + b + g.sw;
+    if (v >= g.W) v -= g.W;
+    label = ((!g.ph && u < g.sh) ? 2 : 0) + ((!g.pw && v < g.sw) ? 1 : 0);
+    code = a * code_stride(g.w) + b;
+    return u * g.W + v;
+}
+
+__device__ __forceinline__ float lds_f32(uint32_t addr) {
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ int4 lds_i4(uint32_t addr) {
+    int4 v;
+    asm volatile("ld.shared.v4.s32 {%0,%1,%2,%3}, [%4];\n" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ float4 lds_f4(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];\n" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ int lds_i32(uint32_t addr) {
+    int v;
+    asm volatile("ld.shared.s32 %0, [%1];\n" : "=r"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void red_global_f32(const float* addr, float v) {
+    asm volatile("red.global.add.f32 [%0], %1;\n" ::"l"(addr), "f"(v) : "memory");
+}
+
+// What one elementwise thread knows about its row.
+struct RowCtx {
+    uint32_t bias_row;   // shared address: bias table + the row's part of the index
+    const char* dbias_row;  // global address: this CTA's bias-gradient table + the row's part of the index (query side)
+    int label;
+    float lse2, delta;   // query side: of this row
+    bool valid;
+};
+
+// 16 columns of one row: P = exp2(S * scale + bias - lse), dS = P * (dP - delta); packs dS (and P) to bf16.
+//   KV = false: rows are queries (lse, delta per row); adds dS into the bias-gradient table.
+//   KV = true : rows are keys    (lse, delta per column).
+template <bool KV, bool MASKED, bool RAGGED>
+__device__ __forceinline__ void bwd_cols16(const uint32_t (&rs)[16], const uint32_t (&rp)[16], uint32_t (&pk_p)[8], uint32_t (&pk_ds)[8],
+                                           int c, const RowCtx& rc, uint32_t st_a, float scale, int dbias_limit) {
+#pragma unroll
+    for (int e4 = 0; e4 < 4; ++e4) {
+        const int4 co4 = lds_i4(st_a + kOffColOff + 4 * (c + e4 * 4));
+        const int co[4] = {co4.x, co4.y, co4.z, co4.w};
+        int kl[4] = {0, 0, 0, 0};
+        if (MASKED) {
+            const int4 kl4 = lds_i4(st_a + kOffLab + 4 * (c + e4 * 4));
+            kl[0] = kl4.x; kl[1] = kl4.y; kl[2] = kl4.z; kl[3] = kl4.w;
+        }
+        float l2[4], dl[4];
+        if (KV) {
+            const float4 a = lds_f4(st_a + kOffLse + 4 * (c + e4 * 4));
+            const float4 b = lds_f4(st_a + kOffDelta + 4 * (c + e4 * 4));
+            l2[0] = a.x; l2[1] = a.y; l2[2] = a.z; l2[3] = a.w;
+            dl[0] = b.x; dl[1] = b.y; dl[2] = b.z; dl[3] = b.w;
+        } else {
+            l2[0] = l2[1] = l2[2] = l2[3] = rc.lse2;
+            dl[0] = dl[1] = dl[2] = dl[3] = rc.delta;
+        }
+        float p[4], ds[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float bv = lds_f32(rc.bias_row + co[e]);
+            float xv = fmaf(__uint_as_float(rs[e4 * 4 + e]), scale, bv) - l2[e];
+            if (MASKED && kl[e] != rc.label) xv = -INFINITY;
+            p[e] = fast_exp2(xv);
+            ds[e] = p[e] * (__uint_as_float(rp[e4 * 4 + e]) - dl[e]);
+            if (!KV) {
+                // one warp instruction touches 32 different table entries (32 different rows, one column)
+                if (RAGGED) {
+                    if (rc.valid && co[e] < dbias_limit) red_global_f32(reinterpret_cast<const float*>(rc.dbias_row + co[e]), ds[e]);
+                } else {
+                    red_global_f32(reinterpret_cast<const float*>(rc.dbias_row + co[e]), ds[e]);
+                }
+            }
+        }
+        if (KV) {
+            pk_p[e4 * 2] = pack_bf16(p[0], p[1]);
+            pk_p[e4 * 2 + 1] = pack_bf16(p[2], p[3]);
+        }
+        pk_ds[e4 * 2] = pack_bf16(ds[0], ds[1]);
+        pk_ds[e4 * 2 + 1] = pack_bf16(ds[2], ds[3]);
+    }
+}
+
+// All columns [0, ncols) of one column block for one row; S at t_s, dP at t_dp (fp32), overwritten in place
+// by bf16 P (key side) and dS.  16 columns per step, the next step's loads in flight.
+template <bool KV, bool MASKED, bool RAGGED>
+__device__ __forceinline__ void bwd_block(uint32_t t_s, uint32_t t_dp, int c_first, int ncols, const RowCtx& rc, uint32_t st_a,
+                                          float scale, int dbias_limit) {
+    uint32_t sa[16], pa[16], sb[16], pb[16];
+    const int nsteps = ncols >> 4;
+    tmem_ld16(t_s, sa);
+    tmem_ld16(t_dp, pa);
+    for (int i = 0; i < nsteps; i += 2) {
+        uint32_t pk_p[8], pk_ds[8];
+        tmem_ld_wait();
+        if (i + 1 < nsteps) {
+            tmem_ld16(t_s + 16 * (i + 1), sb);
+            tmem_ld16(t_dp + 16 * (i + 1), pb);
+        }
+        bwd_cols16<KV, MASKED, RAGGED>(sa, pa, pk_p, pk_ds, c_first + 16 * i, rc, st_a, scale, dbias_limit);
+        if (KV) tmem_st8(t_s + 8 * i, pk_p);
+        tmem_st8(t_dp + 8 * i, pk_ds);
+        if (i + 1 < nsteps) {
+            tmem_ld_wait();
+            if (i + 2 < nsteps) {
+                tmem_ld16(t_s + 16 * (i + 2), sa);
+                tmem_ld16(t_dp + 16 * (i + 2), pa);
+            }
+            bwd_cols16<KV, MASKED, RAGGED>(sb, pb, pk_p, pk_ds, c_first + 16 * (i + 1), rc, st_a, scale, dbias_limit);
+            if (KV) tmem_st8(t_s + 8 * (i + 1), pk_p);
+            tmem_st8(t_dp + 8 * (i + 1), pk_ds);
+        }
+    }
+}
+
+template <bool KV>
+__global__ void __launch_bounds__(kThreads, 1)
+swin_bwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
+                   const __nv_bfloat16* __restrict__ v, const __nv_bfloat16* __restrict__ d_o,
+                   const float* __restrict__ bias_prep, const float* __restrict__ lse, const float* __restrict__ delta,
+                   __nv_bfloat16* __restrict__ out1, __nv_bfloat16* __restrict__ out2, float* __restrict__ dbias,
+                   long long n_items, int ctas_per_head) {
+    constexpr int CB = KV ? 96 : 112;           // columns per block
+    constexpr int kColAcc1 = 2 * CB;            // key side: dV at 192; query side: dQ at 224
+    constexpr int kColAcc2 = 2 * CB + 32;       // key side: dK at 224
+    extern __shared__ __align__(1024) unsigned char smem[];
+    const uint32_t smem0 = smem_u32(smem);
+    const uint32_t bar0 = smem0 + kOffBars;
+    auto bar_full = [&](int s) { return bar0 + 8u * s; };
+    auto bar_empty = [&](int s) { return bar0 + 8u * (kStages + s); };
+    auto bar_sdp = [&](int t) { return bar0 + 8u * (2 * kStages + t); };       // S and dP of a block are in TMEM
+    auto bar_ds = [&](int t) { return bar0 + 8u * (2 * kStages + 2 + t); };    // bf16 P / dS of a block are in TMEM
+    auto bar_acc = [&](int t) { return bar0 + 8u * (2 * kStages + 4 + t); };   // the item's accumulators are final
+    auto bar_free = [&](int t) { return bar0 + 8u * (2 * kStages + 6 + t); };  // the tile's TMEM region may be reused
+    unsigned char* tail = smem + kOffBars + 8 * (2 * kStages + 8);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail);
+    volatile int* cta_abort = reinterpret_cast<volatile int*>(tail + 8);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int head = blockIdx.x % g.heads;
+    const int cta_in_head = blockIdx.x / g.heads;
+
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(bar_full(s), kLoaderThreads);
+            mbar_init(bar_empty(s), 1);
+        }
+        for (int t = 0; t < 2; ++t) {
+            mbar_init(bar_sdp(t), 1);
+            mbar_init(bar_ds(t), 128);
+            mbar_init(bar_acc(t), 1);
+            mbar_init(bar_free(t), 128);
+        }
+        *cta_abort = 0;
+        fence_barrier_init();
+    }
+    // the head's prepared bias table, and a zeroed bias-gradient table
+    for (int i = tid; i < kFwdBiasFloats; i += kThreads)
+        reinterpret_cast<float*>(smem + kOffBias)[i] = bias_prep[(size_t)head * kFwdBiasFloats + i];
+    if (warp == kMmaWarp) {
+        tmem_alloc(smem_u32(tmem_slot), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int cs = code_stride(g.w);
+    const int c0 = (g.w - 1) * (cs + 1);
+    const size_t HW = (size_t)g.H * g.W;
+
+    if (warp >= kMmaWarp) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kRegsOther));
+    if (warp >= kLoaderWarp0) {
+        // ------------------------------------------------------------------ loaders
+        const int lt = tid - kLoaderWarp0 * 32;
+        int kuse = 0, pending_s = -1;
+        for (long long it = cta_in_head; it < n_items; it += ctas_per_head, ++kuse) {
+            const int s = kuse % kStages;
+            // if the next stage is not free yet, publish the copies already issued instead of holding them back
+            if (pending_s >= 0 && !__all_sync(0xffffffffu, mbar_test_wait(bar_empty(s), ((kuse / kStages) & 1) ^ 1))) {
+                cp_async_wait<0>();
+                fence_proxy_async();
+                mbar_arrive(bar_full(pending_s));
+                pending_s = -1;
+            }
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_empty(s), ((kuse / kStages) & 1) ^ 1, cta_abort))) break;
+            const Item x = make_item(g, it);
+            unsigned char* st = smem + s * kStageBytes;
+            const uint32_t st_a = smem0 + s * kStageBytes;
+            const size_t sample_off = (size_t)x.b * HW;
+            // slot metadata; the lse / delta gathers stay in flight while the row copies are issued below
+            constexpr int kSlotIters = (kMaxSlots + kLoaderThreads - 1) / kLoaderThreads;
+            float l2v[kSlotIters], dlv[kSlotIters];
+#pragma unroll
+            for (int i = 0; i < kSlotIters; ++i) {
+                const int slot = lt + i * kLoaderThreads;
+                l2v[i] = INFINITY;                       // no token: P = exp2(.. - inf) = 0
+                dlv[i] = 0.f;
+                if (slot >= kMaxSlots) continue;
+                int code = 0, label = 0xff, tok = -1;
+                // as a column of the query side a slot without a token points into the table's -inf zone
+                int coloff = KV ? 0 : 4 * (2 * c0 + 1);
+                if (slot < x.r.n) {
+                    tok = slot_token_tc(g, x.r, slot, code, label);
+                    const size_t li = (sample_off + (size_t)tok) * g.heads + head;
+                    l2v[i] = __ldg(lse + li);
+                    dlv[i] = __ldg(delta + li);
+                    coloff = KV ? 4 * code : 4 * (c0 - code);
+                }
+                reinterpret_cast<int*>(st + kOffColOff)[slot] = coloff;
+                reinterpret_cast<int*>(st + kOffLab)[slot] = label;
+                reinterpret_cast<int*>(st + kOffCode)[slot] = code;
+                reinterpret_cast<int*>(st + kOffTok)[slot] = tok;
+            }
+            const int chunk = lt & 3;
+            for (int row = lt >> 2; row < x.npad; row += kLoaderThreads / 4) {
+                const __nv_bfloat16 *sq = q, *sk = k, *sv = v, *sg = d_o;
+                int bytes = 0;   // rows past the window's end are written as zeros
+                if (row < x.r.n) {
+                    int code, label;
+                    const int tok = slot_token_tc(g, x.r, row, code, label);
+                    const size_t off = ((sample_off + (size_t)tok) * g.heads + head) * kD + chunk * 8;
+                    sq = q + off; sk = k + off; sv = v + off; sg = d_o + off;
+                    bytes = 16;
+                }
+                const uint32_t so = st_a + tile_off<kD>(row, chunk);
+                cp_async16(so + kOffQ, sq, bytes);
+                cp_async16(so + kOffK, sk, bytes);
+                cp_async16(so + kOffV, sv, bytes);
+                cp_async16(so + kOffDO, sg, bytes);
+            }
+            cp_async_commit();
+#pragma unroll
+            for (int i = 0; i < kSlotIters; ++i) {
+                const int slot = lt + i * kLoaderThreads;
+                if (slot < kMaxSlots) {
+                    reinterpret_cast<float*>(st + kOffLse)[slot] = l2v[i] * kLog2e;
+                    reinterpret_cast<float*>(st + kOffDelta)[slot] = dlv[i];
+                }
+            }
+            if (pending_s >= 0) {
+                cp_async_wait<1>();
+                fence_proxy_async();
+                mbar_arrive(bar_full(pending_s));
+            }
+            pending_s = s;
+        }
+        if (pending_s >= 0) {
+            cp_async_wait<0>();
+            fence_proxy_async();
+            mbar_arrive(bar_full(pending_s));
+        }
+    } else {
+        // ------------------------------------------------------------------ MMA issuer (one lane)
+        if (lane == 0) {
+            const uint32_t idesc_acc = make_idesc_bf16(128, kD, 0, 1);   // A from TMEM, B = 16 rows x 32 (MN-major)
+            // row operands (A of the S-type products) and column operands (their B, and B of the accumulations)
+            const uint32_t off_r1 = KV ? kOffK : kOffQ, off_r2 = KV ? kOffV : kOffDO;
+            const uint32_t off_c1 = KV ? kOffQ : kOffK, off_c2 = KV ? kOffDO : kOffV;
+            const uint64_t d_r1 = make_sdesc_sw64(smem0 + off_r1, 512), d_r2 = make_sdesc_sw64(smem0 + off_r2, 512);
+            const uint64_t d_c1 = make_sdesc_sw64(smem0 + off_c1, 512), d_c2 = make_sdesc_sw64(smem0 + off_c2, 512);
+            int n_sdp[2] = {0, 0}, n_ds[2] = {0, 0}, n_free[2] = {0, 0}, n_acc_used[2] = {0, 0};
+            bool ok = true;
+            // S = R1 C1^T and dP = R2 C2^T for column block cb of tile t
+            auto issue_sdp = [&](int s, int t, int cb, int ncols) {
+                const uint64_t so = (uint64_t)((s * kStageBytes) >> 4);
+                const uint64_t ro = so + (uint64_t)((t * 128 * kRowBytes) >> 4), co = so + (uint64_t)((cb * CB * kRowBytes) >> 4);
+                const uint32_t idesc = make_idesc_bf16(128, ncols, 0, 0);
+                const uint32_t t_s = tmem_base + t * 256, t_dp = tmem_base + t * 256 + CB;
+                mma_ss(t_s, d_r1 + ro, d_c1 + co, idesc, 0u);
+                mma_ss(t_s, d_r1 + ro + 2, d_c1 + co + 2, idesc, 1u);
+                mma_ss(t_dp, d_r2 + ro, d_c2 + co, idesc, 0u);
+                mma_ss(t_dp, d_r2 + ro + 2, d_c2 + co + 2, idesc, 1u);
+                mma_commit(bar_sdp(t));
+            };
+            // accumulations of column block cb: query side dQ += dS C1; key side dV += P C2, dK += dS C1
+            auto issue_acc = [&](int s, int t, int cb, int ncols) {
+                const uint64_t co = (uint64_t)((s * kStageBytes + cb * CB * kRowBytes) >> 4);
+                const uint32_t t_p = tmem_base + t * 256, t_ds = tmem_base + t * 256 + CB;
+                const uint32_t first = cb == 0 ? 0u : 1u;
+                for (int ks = 0; ks < (ncols >> 4); ++ks) {
+                    const uint32_t acc = (ks > 0) ? 1u : first;
+                    if (KV) {
+                        mma_ts(tmem_base + t * 256 + kColAcc1, t_p + ks * 8, d_c2 + co + (uint64_t)(ks * 64), idesc_acc, acc);
+                        mma_ts(tmem_base + t * 256 + kColAcc2, t_ds + ks * 8, d_c1 + co + (uint64_t)(ks * 64), idesc_acc, acc);
+                    } else {
+                        mma_ts(tmem_base + t * 256 + kColAcc1, t_ds + ks * 8, d_c1 + co + (uint64_t)(ks * 64), idesc_acc, acc);
+                    }
+                }
+            };
+            int kuse = 0;
+            for (long long it = cta_in_head; ok && it < n_items; it += ctas_per_head, ++kuse) {
+                const int s = kuse % kStages;
+                const Item x = make_item(g, it);
+                const int ncb = (x.npad + CB - 1) / CB;
+                ok = mbar_wait(bar_full(s), (kuse / kStages) & 1, cta_abort);
+                if (!ok) break;
+                fence_proxy_async();
+                for (int cb = 0; cb < ncb && ok; ++cb) {
+                    const int ncols = min(CB, x.npad - cb * CB);
+#pragma unroll
+                    for (int t = 0; t < 2; ++t) {
+                        if (t >= x.ntiles || !ok) continue;
+                        if (cb == 0) {
+                            // the tile's region is free once its warpgroup has read the previous item's accumulators
+                            if (n_acc_used[t] > n_free[t]) {
+                                ok = mbar_wait(bar_free(t), n_free[t] & 1, cta_abort);
+                                ++n_free[t];
+                            }
+                        } else {
+                            ok = mbar_wait(bar_ds(t), n_ds[t] & 1, cta_abort);
+                            ++n_ds[t];
+                            if (ok) {
+                                tc_fence_after();
+                                issue_acc(s, t, cb - 1, CB);
+                            }
+                        }
+                        if (!ok) continue;
+                        tc_fence_after();
+                        issue_sdp(s, t, cb, ncols);
+                        ++n_sdp[t];
+                    }
+                }
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    if (t >= x.ntiles || !ok) continue;
+                    ok = mbar_wait(bar_ds(t), n_ds[t] & 1, cta_abort);
+                    ++n_ds[t];
+                    if (!ok) continue;
+                    tc_fence_after();
+                    issue_acc(s, t, ncb - 1, x.npad - (ncb - 1) * CB);
+                    mma_commit(bar_acc(t));
+                    ++n_acc_used[t];
+                }
+                if (ok) mma_commit(bar_empty(s));
+            }
+        }
+    }
+    } else {
+        // ------------------------------------------------------------------ elementwise warpgroups
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(kRegsWork));
+        const int wg = warp >> 2;
+        const int row = tid & 127;
+        const int slot = wg * 128 + row;
+        const uint32_t lane_addr = ((uint32_t)(32 * (warp & 3))) << 16;
+        const uint32_t t_reg = tmem_base + lane_addr + wg * 256;
+        const float scale = g.scale_log2e;
+        const float out_scale = g.scale_log2e * kLn2;          // dQ and dK carry the score scale
+        const int dbias_limit = 4 * (2 * c0 + 1);
+        int kuse = 0, n_sdp = 0, n_acc = 0;
+        for (long long it = cta_in_head; it < n_items; it += ctas_per_head, ++kuse) {
+            const Item x = make_item(g, it);
+            if (wg >= x.ntiles) continue;
+            const int s = kuse % kStages;
+            const uint32_t st_a = smem0 + s * kStageBytes;
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_full(s), (kuse / kStages) & 1, cta_abort))) break;
+            const int code_i = lds_i32(st_a + kOffCode + 4 * slot);
+            const int tok = lds_i32(st_a + kOffTok + 4 * slot);
+            RowCtx rc;
+            rc.label = lds_i32(st_a + kOffLab + 4 * slot);
+            rc.valid = tok >= 0;
+            rc.lse2 = lds_f32(st_a + kOffLse + 4 * slot);
+            rc.delta = lds_f32(st_a + kOffDelta + 4 * slot);
+            // bias index = code_query - code_key + c0
+            rc.bias_row = smem0 + kOffBias + (KV ? 4 * (c0 - code_i) : 4 * code_i);
+            rc.dbias_row = reinterpret_cast<const char*>(dbias + (size_t)blockIdx.x * kDBiasFloats + code_i);
+            const int ncb = (x.npad + CB - 1) / CB;
+            bool ok = true;
+            for (int cb = 0; cb < ncb; ++cb) {
+                const int ncols = min(CB, x.npad - cb * CB);
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_sdp(wg), n_sdp & 1, cta_abort));
+                if (!ok) break;
+                ++n_sdp;
+                tc_fence_after();
+                if (x.masked)
+                    bwd_block<KV, true, true>(t_reg, t_reg + CB, cb * CB, ncols, rc, st_a, scale, dbias_limit);
+                else if (x.ragged)
+                    bwd_block<KV, false, true>(t_reg, t_reg + CB, cb * CB, ncols, rc, st_a, scale, dbias_limit);
+                else
+                    bwd_block<KV, false, false>(t_reg, t_reg + CB, cb * CB, ncols, rc, st_a, scale, dbias_limit);
+                tmem_st_wait();
+                tc_fence_before();
+                mbar_arrive(bar_ds(wg));
+            }
+            if (!ok) break;
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_acc(wg), n_acc & 1, cta_abort))) break;
+            ++n_acc;
+            tc_fence_after();
+            uint32_t r1[32], r2[32];
+            if (KV) {
+                tmem_ld32(t_reg + kColAcc1, r1);      // dV
+                tmem_ld32(t_reg + kColAcc2, r2);      // dK
+            } else {
+                tmem_ld32(t_reg + kColAcc1, r2);      // dQ
+            }
+            tmem_ld_wait();
+            tc_fence_before();
+            mbar_arrive(bar_free(wg));
+            if (tok >= 0) {
+                const size_t row_off = (((size_t)x.b * HW + (size_t)tok) * g.heads + head) * kD;
+                if (KV) {
+                    uint4* dv_dst = reinterpret_cast<uint4*>(out2 + row_off);     // dV
+                    uint4* dk_dst = reinterpret_cast<uint4*>(out1 + row_off);     // dK
+#pragma unroll
+                    for (int c4 = 0; c4 < 4; ++c4) {
+                        uint4 a, b;
+                        a.x = pack_bf16(__uint_as_float(r1[c4 * 8 + 0]), __uint_as_float(r1[c4 * 8 + 1]));
+                        a.y = pack_bf16(__uint_as_float(r1[c4 * 8 + 2]), __uint_as_float(r1[c4 * 8 + 3]));
+                        a.z = pack_bf16(__uint_as_float(r1[c4 * 8 + 4]), __uint_as_float(r1[c4 * 8 + 5]));
+                        a.w = pack_bf16(__uint_as_float(r1[c4 * 8 + 6]), __uint_as_float(r1[c4 * 8 + 7]));
+                        b.x = pack_bf16(__uint_as_float(r2[c4 * 8 + 0]) * out_scale, __uint_as_float(r2[c4 * 8 + 1]) * out_scale);
+                        b.y = pack_bf16(__uint_as_float(r2[c4 * 8 + 2]) * out_scale, __uint_as_float(r2[c4 * 8 + 3]) * out_scale);
+                        b.z = pack_bf16(__uint_as_float(r2[c4 * 8 + 4]) * out_scale, __uint_as_float(r2[c4 * 8 + 5]) * out_scale);
+                        b.w = pack_bf16(__uint_as_float(r2[c4 * 8 + 6]) * out_scale, __uint_as_float(r2[c4 * 8 + 7]) * out_scale);
+                        dv_dst[c4] = a;
+                        dk_dst[c4] = b;
+                    }
+                } else {
+                    uint4* dq_dst = reinterpret_cast<uint4*>(out1 + row_off);
+#pragma unroll
+                    for (int c4 = 0; c4 < 4; ++c4) {
+                        uint4 b;
+                        b.x = pack_bf16(__uint_as_float(r2[c4 * 8 + 0]) * out_scale, __uint_as_float(r2[c4 * 8 + 1]) * out_scale);
+                        b.y = pack_bf16(__uint_as_float(r2[c4 * 8 + 2]) * out_scale, __uint_as_float(r2[c4 * 8 + 3]) * out_scale);
+                        b.z = pack_bf16(__uint_as_float(r2[c4 * 8 + 4]) * out_scale, __uint_as_float(r2[c4 * 8 + 5]) * out_scale);
+                        b.w = pack_bf16(__uint_as_float(r2[c4 * 8 + 6]) * out_scale, __uint_as_float(r2[c4 * 8 + 7]) * out_scale);
+                        dq_dst[c4] = b;
+                    }
+                }
+            }
+        }
+    }
+
+    // teardown: every role ends up here, also after an expired wait
+    cp_async_wait<0>();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == kMmaWarp) tmem_dealloc(tmem_base, 512);
+    if (tid == 0 && *cta_abort) atomicExch(&g_bwd_tc_timeout, 1);
+}
+
+// dbias[(da, db), head] = sum over the head's CTAs of their tables (entry (da + w - 1) * cs + (db + w - 1)).
+// Fixed summation order over CTAs.
+__global__ void __launch_bounds__(256)
+swin_bwd_tc_dbias_finalize_kernel(const float* __restrict__ parts, float* __restrict__ dbias, int w, int heads, int ctas_per_head) {
+    const int nw = 2 * w - 1, cs = w + 32;
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;       // (table row, head)
+    if (i >= nw * nw * heads) return;
+    const int head = i % heads, r = i / heads;
+    const int e = (r / nw) * cs + (r % nw);
+    float acc = 0.f;
+    for (int c = 0; c < ctas_per_head; ++c) acc += parts[(size_t)(c * heads + head) * kDBiasFloats + e];
+    dbias[i] = acc;
+}
+
+}  // namespace
+
+cudaError_t read_bwd_tc_status(int* timed_out) {
+    int zero = 0;
+    cudaError_t e = cudaMemcpyFromSymbol(timed_out, g_bwd_tc_timeout, sizeof(int));
+    if (e != cudaSuccess) return e;
+    if (*timed_out) e = cudaMemcpyToSymbol(g_bwd_tc_timeout, &zero, sizeof(int));
+    return e;
+}
+
+constexpr int kMaxGrid = 160;   // CTAs whose bias-gradient tables fit the workspace
+
+bool bwd_tc_supported(const Geo& g) { return g.d == 32 && g.nmax <= kMaxSlots && g.w <= 16 && g.heads <= 148; }
+
+// workspace: delta [B*H*W*heads] fp32, then the prepared bias tables [heads * kFwdBiasFloats] fp32
+size_t bwd_tc_workspace_bytes(const Geo& g) {
+    const size_t delta = (((size_t)g.B * g.H * g.W * g.heads * sizeof(float)) + 255) / 256 * 256;
+    return delta + (size_t)g.heads * kFwdBiasFloats * sizeof(float) + (size_t)kMaxGrid * kDBiasFloats * sizeof(float);
+}
+
+cudaError_t launch_bwd_tc(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
+                          const void* o, const float* lse, const void* d_o, void* dq, void* dk, void* dv, float* dbias,
+                          void* workspace, int sm_count, cudaStream_t stream) {
+    float* delta = reinterpret_cast<float*>(workspace);
+    const size_t delta_bytes = (((size_t)g.B * g.H * g.W * g.heads * sizeof(float)) + 255) / 256 * 256;
+    float* prep = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(workspace) + delta_bytes);
+    cudaError_t e = launch_bwd_delta(g, o, d_o, delta, stream);
+    if (e != cudaSuccess) return e;
+    e = launch_bias_prep(g, bias, prep, stream);
+    if (e != cudaSuccess) return e;
+    float* parts = prep + (size_t)g.heads * kFwdBiasFloats;
+    e = cudaMemsetAsync(parts, 0, sizeof(float) * (size_t)kMaxGrid * kDBiasFloats, stream);
+    if (e != cudaSuccess) return e;
+    const long long items = (long long)g.B * g.Mh * g.Mw;
+    long long cph = (sm_count < kMaxGrid ? sm_count : kMaxGrid) / g.heads;
+    if (cph < 1) cph = 1;
+    if (cph > items) cph = items;
+    const unsigned grid = (unsigned)(cph * g.heads);
+    e = cudaFuncSetAttribute(swin_bwd_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(swin_bwd_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    swin_bwd_tc_kernel<true><<<grid, kThreads, kSmemBytes, stream>>>(
+        g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)d_o, prep, lse, delta,
+        (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, nullptr, items, (int)cph);
+    count_launch();
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    swin_bwd_tc_kernel<false><<<grid, kThreads, kSmemBytes, stream>>>(
+        g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)d_o, prep, lse, delta,
+        (__nv_bfloat16*)dq, nullptr, parts, items, (int)cph);
+    count_launch();
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const int nrows = (2 * g.w - 1) * (2 * g.w - 1) * g.heads;
+    swin_bwd_tc_dbias_finalize_kernel<<<(nrows + 255) / 256, 256, 0, stream>>>(parts, dbias, g.w, g.heads, (int)cph);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace terra

@@ -273,6 +273,13 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
         int kuse = 0, pending_s = -1;
         for (long long it = blockIdx.x; it < n_items; it += gridDim.x, ++kuse) {
             const int s = kuse % kStages;
+            // if the next stage is not free yet, publish the copies already issued instead of holding them back
+            if (pending_s >= 0 && !__all_sync(0xffffffffu, mbar_test_wait(bar_empty(s), ((kuse / kStages) & 1) ^ 1))) {
+                cp_async_wait<0>();
+                fence_proxy_async();
+                mbar_arrive(bar_full(pending_s));
+                pending_s = -1;
+            }
             if (!__all_sync(0xffffffffu, mbar_wait(bar_empty(s), ((kuse / kStages) & 1) ^ 1, cta_abort))) break;
             const Item x = make_item(g, it);
             unsigned char* st = smem + s * kStageBytes;
@@ -535,6 +542,13 @@ cudaError_t launch_fwd_tc(const Geo& g, const void* q, const void* k, const void
     const unsigned grid = (unsigned)(items < sm_count ? items : sm_count);
     swin_fwd_tc_kernel<<<grid, kThreads, kSmemBytes, stream>>>(g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k,
                                                                (const __nv_bfloat16*)v, prep, (__nv_bfloat16*)o, lse, items);
+    count_launch();
+    return cudaGetLastError();
+}
+
+// prepared bias tables for every head (also used by the backward kernels)
+cudaError_t launch_bias_prep(const Geo& g, const float* bias, float* prep, cudaStream_t stream) {
+    swin_fwd_bias_prep_kernel<<<g.heads, 256, 0, stream>>>(bias, prep, g.w, g.heads);
     count_launch();
     return cudaGetLastError();
 }

@@ -25,6 +25,16 @@ cudaError_t launch_fwd_tc(const Geo& g, const void* q, const void* k, const void
 // synchronises the stream, reads and clears the device-side "a bounded wait expired" word
 cudaError_t read_tc_status(int* timed_out, cudaStream_t stream);
 
+cudaError_t launch_bias_prep(const Geo& g, const float* bias, float* prep, cudaStream_t stream);
+
+// tcgen05 backward path (head dim 32, window side <= 16)
+bool bwd_tc_supported(const Geo& g);
+size_t bwd_tc_workspace_bytes(const Geo& g);
+cudaError_t launch_bwd_tc(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
+                          const void* o, const float* lse, const void* d_o, void* dq, void* dk, void* dv, float* dbias,
+                          void* workspace, int sm_count, cudaStream_t stream);
+cudaError_t read_bwd_tc_status(int* timed_out);
+
 // delta[b, token, head] = sum_c dO * O   (fp32, same indexing as lse)
 cudaError_t launch_bwd_delta(const Geo& g, const void* o, const void* d_o, float* delta, cudaStream_t stream);
 
