@@ -8,7 +8,8 @@
 //                            written to TMEM as bf16, dV += P^T dO and dK += dS^T Q.
 // P is recomputed from the saved log-sum-exp, so the column blocks of a row are independent (no running
 // maximum).  Structure as in the forward kernel: persistent CTAs, two 128-row tiles (one per elementwise
-// warpgroup, one thread per row), one MMA-issuing lane, three loader warps gathering the window's rows with
+// warpgroup, one thread per row), one MMA-issuing lane per tile (so one tile's elementwise work never delays the other tile's
+// MMAs), two loader warps gathering the window's rows with
 // cp.async into the 64-byte-swizzled operand layout.  CTAs are bound to one head (grid = heads x CTAs per
 // head), so the head's bias table is staged once per CTA and the bias-gradient table belongs to one head.
 // TMEM, per 128-row tile (256 columns):  query side [S 112 | dP 112 | dQ 32], key side
@@ -26,9 +27,9 @@ namespace {
 
 using namespace tc;
 
-constexpr int kMmaWarp = 8;
-constexpr int kLoaderWarp0 = 9;
-constexpr int kLoaderWarps = 3;
+constexpr int kMmaWarp = 8;         // warps 8 and 9: one MMA-issuing lane per 128-row tile
+constexpr int kLoaderWarp0 = 10;
+constexpr int kLoaderWarps = 2;
 constexpr int kLoaderThreads = kLoaderWarps * 32;
 constexpr int kThreads = (kLoaderWarp0 + kLoaderWarps) * 32;   // 384 = three warpgroups
 constexpr int kRegsLaunch = 168;
@@ -139,48 +140,57 @@ struct RowCtx {
 template <bool KV, bool MASKED, bool RAGGED>
 __device__ __forceinline__ void bwd_cols16(const uint32_t (&rs)[16], const uint32_t (&rp)[16], uint32_t (&pk_p)[8], uint32_t (&pk_ds)[8],
                                            int c, const RowCtx& rc, uint32_t st_a, float scale, int dbias_limit) {
+    // all shared-memory loads first (the explicit loads keep their order), then the arithmetic
+    int co[16], kl[16];
+    float l2[16], dl[16], bv[16];
 #pragma unroll
     for (int e4 = 0; e4 < 4; ++e4) {
         const int4 co4 = lds_i4(st_a + kOffColOff + 4 * (c + e4 * 4));
-        const int co[4] = {co4.x, co4.y, co4.z, co4.w};
-        int kl[4] = {0, 0, 0, 0};
-        if (MASKED) {
+        co[e4 * 4] = co4.x; co[e4 * 4 + 1] = co4.y; co[e4 * 4 + 2] = co4.z; co[e4 * 4 + 3] = co4.w;
+    }
+#pragma unroll
+    for (int e = 0; e < 16; ++e) bv[e] = lds_f32(rc.bias_row + co[e]);
+    if (MASKED) {
+#pragma unroll
+        for (int e4 = 0; e4 < 4; ++e4) {
             const int4 kl4 = lds_i4(st_a + kOffLab + 4 * (c + e4 * 4));
-            kl[0] = kl4.x; kl[1] = kl4.y; kl[2] = kl4.z; kl[3] = kl4.w;
+            kl[e4 * 4] = kl4.x; kl[e4 * 4 + 1] = kl4.y; kl[e4 * 4 + 2] = kl4.z; kl[e4 * 4 + 3] = kl4.w;
         }
-        float l2[4], dl[4];
-        if (KV) {
+    }
+    if (KV) {
+#pragma unroll
+        for (int e4 = 0; e4 < 4; ++e4) {
             const float4 a = lds_f4(st_a + kOffLse + 4 * (c + e4 * 4));
             const float4 b = lds_f4(st_a + kOffDelta + 4 * (c + e4 * 4));
-            l2[0] = a.x; l2[1] = a.y; l2[2] = a.z; l2[3] = a.w;
-            dl[0] = b.x; dl[1] = b.y; dl[2] = b.z; dl[3] = b.w;
-        } else {
-            l2[0] = l2[1] = l2[2] = l2[3] = rc.lse2;
-            dl[0] = dl[1] = dl[2] = dl[3] = rc.delta;
+            l2[e4 * 4] = a.x; l2[e4 * 4 + 1] = a.y; l2[e4 * 4 + 2] = a.z; l2[e4 * 4 + 3] = a.w;
+            dl[e4 * 4] = b.x; dl[e4 * 4 + 1] = b.y; dl[e4 * 4 + 2] = b.z; dl[e4 * 4 + 3] = b.w;
         }
-        float p[4], ds[4];
+    }
+    float p[16], ds[16];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const float bv = lds_f32(rc.bias_row + co[e]);
-            float xv = fmaf(__uint_as_float(rs[e4 * 4 + e]), scale, bv) - l2[e];
-            if (MASKED && kl[e] != rc.label) xv = -INFINITY;
-            p[e] = fast_exp2(xv);
-            ds[e] = p[e] * (__uint_as_float(rp[e4 * 4 + e]) - dl[e]);
-            if (!KV) {
-                // one warp instruction touches 32 different table entries (32 different rows, one column)
-                if (RAGGED) {
-                    if (rc.valid && co[e] < dbias_limit) red_global_f32(reinterpret_cast<const float*>(rc.dbias_row + co[e]), ds[e]);
-                } else {
-                    red_global_f32(reinterpret_cast<const float*>(rc.dbias_row + co[e]), ds[e]);
-                }
+    for (int e = 0; e < 16; ++e) {
+        const float lse_e = KV ? l2[e] : rc.lse2;
+        const float del_e = KV ? dl[e] : rc.delta;
+        float xv = fmaf(__uint_as_float(rs[e]), scale, bv[e]) - lse_e;
+        if (MASKED && kl[e] != rc.label) xv = -INFINITY;
+        p[e] = fast_exp2(xv);
+        ds[e] = p[e] * (__uint_as_float(rp[e]) - del_e);
+    }
+    if (!KV) {
+        // one warp instruction touches 32 different table entries (32 different rows, one column)
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+            if (RAGGED) {
+                if (rc.valid && co[e] < dbias_limit) red_global_f32(reinterpret_cast<const float*>(rc.dbias_row + co[e]), ds[e]);
+            } else {
+                red_global_f32(reinterpret_cast<const float*>(rc.dbias_row + co[e]), ds[e]);
             }
         }
-        if (KV) {
-            pk_p[e4 * 2] = pack_bf16(p[0], p[1]);
-            pk_p[e4 * 2 + 1] = pack_bf16(p[2], p[3]);
-        }
-        pk_ds[e4 * 2] = pack_bf16(ds[0], ds[1]);
-        pk_ds[e4 * 2 + 1] = pack_bf16(ds[2], ds[3]);
+    }
+#pragma unroll
+    for (int e2 = 0; e2 < 8; ++e2) {
+        if (KV) pk_p[e2] = pack_bf16(p[2 * e2], p[2 * e2 + 1]);
+        pk_ds[e2] = pack_bf16(ds[2 * e2], ds[2 * e2 + 1]);
     }
 }
 
@@ -246,7 +256,7 @@ swin_bwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(bar_full(s), kLoaderThreads);
-            mbar_init(bar_empty(s), 1);
+            mbar_init(bar_empty(s), 2);      // one arrival per MMA issuer
         }
         for (int t = 0; t < 2; ++t) {
             mbar_init(bar_sdp(t), 1);
@@ -356,7 +366,7 @@ swin_bwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
             mbar_arrive(bar_full(pending_s));
         }
     } else {
-        // ------------------------------------------------------------------ MMA issuer (one lane)
+        // ------------------------------------------------------------------ MMA issuers (one lane of warp 8 / 9)
         if (lane == 0) {
             const uint32_t idesc_acc = make_idesc_bf16(128, kD, 0, 1);   // A from TMEM, B = 16 rows x 32 (MN-major)
             // row operands (A of the S-type products) and column operands (their B, and B of the accumulations)
@@ -364,7 +374,6 @@ swin_bwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
             const uint32_t off_c1 = KV ? kOffQ : kOffK, off_c2 = KV ? kOffDO : kOffV;
             const uint64_t d_r1 = make_sdesc_sw64(smem0 + off_r1, 512), d_r2 = make_sdesc_sw64(smem0 + off_r2, 512);
             const uint64_t d_c1 = make_sdesc_sw64(smem0 + off_c1, 512), d_c2 = make_sdesc_sw64(smem0 + off_c2, 512);
-            int n_sdp[2] = {0, 0}, n_ds[2] = {0, 0}, n_free[2] = {0, 0}, n_acc_used[2] = {0, 0};
             bool ok = true;
             // S = R1 C1^T and dP = R2 C2^T for column block cb of tile t
             auto issue_sdp = [&](int s, int t, int cb, int ncols) {
@@ -393,51 +402,53 @@ swin_bwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
                     }
                 }
             };
-            int kuse = 0;
+            const int t = warp - kMmaWarp;      // this issuer's tile
+            int kuse = 0, n_ds = 0, n_free = 0, n_acc_used = 0;
             for (long long it = cta_in_head; ok && it < n_items; it += ctas_per_head, ++kuse) {
                 const int s = kuse % kStages;
                 const Item x = make_item(g, it);
                 const int ncb = (x.npad + CB - 1) / CB;
                 ok = mbar_wait(bar_full(s), (kuse / kStages) & 1, cta_abort);
                 if (!ok) break;
+                if (t >= x.ntiles) {            // nothing to issue for this tile: just release the stage
+                    mma_commit(bar_empty(s));
+                    continue;
+                }
                 fence_proxy_async();
                 for (int cb = 0; cb < ncb && ok; ++cb) {
                     const int ncols = min(CB, x.npad - cb * CB);
-#pragma unroll
-                    for (int t = 0; t < 2; ++t) {
-                        if (t >= x.ntiles || !ok) continue;
-                        if (cb == 0) {
-                            // the tile's region is free once its warpgroup has read the previous item's accumulators
-                            if (n_acc_used[t] > n_free[t]) {
-                                ok = mbar_wait(bar_free(t), n_free[t] & 1, cta_abort);
-                                ++n_free[t];
-                            }
-                        } else {
-                            ok = mbar_wait(bar_ds(t), n_ds[t] & 1, cta_abort);
-                            ++n_ds[t];
-                            if (ok) {
-                                tc_fence_after();
-                                issue_acc(s, t, cb - 1, CB);
-                            }
+                    // S / dP columns are free as soon as the previous accumulation MMAs (issued earlier by this
+                    // lane, executed in order) have read them; only the accumulator columns have to wait until
+                    // the warpgroup has read the previous item's results.
+                    if (cb > 0) {
+                        ok = mbar_wait(bar_ds(t), n_ds & 1, cta_abort);
+                        ++n_ds;
+                        if (ok && cb == 1 && n_acc_used > n_free) {
+                            ok = mbar_wait(bar_free(t), n_free & 1, cta_abort);
+                            ++n_free;
                         }
-                        if (!ok) continue;
-                        tc_fence_after();
-                        issue_sdp(s, t, cb, ncols);
-                        ++n_sdp[t];
+                        if (ok) {
+                            tc_fence_after();
+                            issue_acc(s, t, cb - 1, CB);
+                        }
                     }
-                }
-#pragma unroll
-                for (int t = 0; t < 2; ++t) {
-                    if (t >= x.ntiles || !ok) continue;
-                    ok = mbar_wait(bar_ds(t), n_ds[t] & 1, cta_abort);
-                    ++n_ds[t];
-                    if (!ok) continue;
+                    if (!ok) break;
                     tc_fence_after();
-                    issue_acc(s, t, ncb - 1, x.npad - (ncb - 1) * CB);
-                    mma_commit(bar_acc(t));
-                    ++n_acc_used[t];
+                    issue_sdp(s, t, cb, ncols);
                 }
-                if (ok) mma_commit(bar_empty(s));
+                if (!ok) break;
+                ok = mbar_wait(bar_ds(t), n_ds & 1, cta_abort);
+                ++n_ds;
+                if (ok && ncb == 1 && n_acc_used > n_free) {
+                    ok = mbar_wait(bar_free(t), n_free & 1, cta_abort);
+                    ++n_free;
+                }
+                if (!ok) break;
+                tc_fence_after();
+                issue_acc(s, t, ncb - 1, x.npad - (ncb - 1) * CB);
+                mma_commit(bar_acc(t));
+                ++n_acc_used;
+                mma_commit(bar_empty(s));
             }
         }
     }
