@@ -57,9 +57,9 @@ constexpr int kOffDelta = kOffLse + kMaxSlots * 4;             // per slot: delt
 constexpr int kStageBytes = ((kOffDelta + kMaxSlots * 4 + 1023) / 1024) * 1024;   // 71680
 // after the stages
 constexpr int kOffBias = kStages * kStageBytes;                // the head's prepared bias table (kFwdBiasFloats floats)
-constexpr int kOffDBias = kOffBias + kFwdBiasFloats * 4;       // query side: bias-gradient table, same indexing
+constexpr int kOffDBias = kOffBias + kFwdBiasFloats * 4;       // query side: one bias-gradient table per elementwise warp
 constexpr int kDBiasFloats = 1536;                             // >= 2 c0 + 1 for w <= 16
-constexpr int kOffBars = kOffDBias + kDBiasFloats * 4;
+constexpr int kOffBars = kOffDBias + 8 * kDBiasFloats * 4;
 constexpr int kSmemBytes = kOffBars + 256;
 
 __device__ __forceinline__ int code_stride(int w) { return w + 32; }
@@ -121,14 +121,21 @@ __device__ __forceinline__ int lds_i32(uint32_t addr) {
     asm volatile("ld.shared.s32 %0, [%1];\n" : "=r"(v) : "r"(addr));
     return v;
 }
-__device__ __forceinline__ void red_global_f32(const float* addr, float v) {
-    asm volatile("red.global.add.f32 [%0], %1;\n" ::"l"(addr), "f"(v) : "memory");
+// table[addr] += v in the warp's own table.  Not atomic: within one warp instruction the 32 lanes (32
+// different rows, same column) touch 32 different entries, and successive instructions of a warp reach
+// shared memory in program order, so nothing is lost.
+__device__ __forceinline__ void rmw_shared_f32(uint32_t addr, float v) {
+    asm volatile(
+        "{\n\t.reg .f32 t;\n\t"
+        "ld.shared.f32 t, [%0];\n\t"
+        "add.f32 t, t, %1;\n\t"
+        "st.shared.f32 [%0], t;\n\t}\n" ::"r"(addr), "f"(v) : "memory");
 }
 
 // What one elementwise thread knows about its row.
 struct RowCtx {
     uint32_t bias_row;   // shared address: bias table + the row's part of the index
-    const char* dbias_row;  // global address: this CTA's bias-gradient table + the row's part of the index (query side)
+    uint32_t dbias_row;  // shared address: this warp's bias-gradient table + the row's part of the index (query side)
     int label;
     float lse2, delta;   // query side: of this row
     bool valid;
@@ -181,9 +188,9 @@ __device__ __forceinline__ void bwd_cols16(const uint32_t (&rs)[16], const uint3
 #pragma unroll
         for (int e = 0; e < 16; ++e) {
             if (RAGGED) {
-                if (rc.valid && co[e] < dbias_limit) red_global_f32(reinterpret_cast<const float*>(rc.dbias_row + co[e]), ds[e]);
+                if (rc.valid && co[e] < dbias_limit) rmw_shared_f32(rc.dbias_row + co[e], ds[e]);
             } else {
-                red_global_f32(reinterpret_cast<const float*>(rc.dbias_row + co[e]), ds[e]);
+                rmw_shared_f32(rc.dbias_row + co[e], ds[e]);
             }
         }
     }
@@ -270,6 +277,8 @@ swin_bwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
     // the head's prepared bias table, and a zeroed bias-gradient table
     for (int i = tid; i < kFwdBiasFloats; i += kThreads)
         reinterpret_cast<float*>(smem + kOffBias)[i] = bias_prep[(size_t)head * kFwdBiasFloats + i];
+    if (!KV)
+        for (int i = tid; i < 8 * kDBiasFloats; i += kThreads) reinterpret_cast<float*>(smem + kOffDBias)[i] = 0.f;
     if (warp == kMmaWarp) {
         tmem_alloc(smem_u32(tmem_slot), 512);
         tmem_relinquish();
@@ -479,7 +488,7 @@ swin_bwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
             rc.delta = lds_f32(st_a + kOffDelta + 4 * slot);
             // bias index = code_query - code_key + c0
             rc.bias_row = smem0 + kOffBias + (KV ? 4 * (c0 - code_i) : 4 * code_i);
-            rc.dbias_row = reinterpret_cast<const char*>(dbias + (size_t)blockIdx.x * kDBiasFloats + code_i);
+            rc.dbias_row = smem0 + kOffDBias + 4 * (warp * kDBiasFloats + code_i);
             const int ncb = (x.npad + CB - 1) / CB;
             bool ok = true;
             for (int cb = 0; cb < ncb; ++cb) {
@@ -553,11 +562,21 @@ swin_bwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
     __syncthreads();
     tc_fence_after();
     if (warp == kMmaWarp) tmem_dealloc(tmem_base, 512);
+    if (!KV) {
+        // this CTA's table = sum of its warps' tables (fixed order), written to the CTA's slot of the workspace
+        const float* tbl = reinterpret_cast<const float*>(smem + kOffDBias);
+        for (int e = tid; e < kDBiasFloats; e += kThreads) {
+            float acc = 0.f;
+#pragma unroll
+            for (int wq = 0; wq < 8; ++wq) acc += tbl[wq * kDBiasFloats + e];
+            dbias[(size_t)blockIdx.x * kDBiasFloats + e] = acc;
+        }
+    }
     if (tid == 0 && *cta_abort) atomicExch(&g_bwd_tc_timeout, 1);
 }
 
 // dbias[(da, db), head] = sum over the head's CTAs of their tables (entry (da + w - 1) * cs + (db + w - 1)).
-// Fixed summation order over CTAs.
+// Fixed summation order over warps and CTAs: the bias gradient is reproducible run to run.
 __global__ void __launch_bounds__(256)
 swin_bwd_tc_dbias_finalize_kernel(const float* __restrict__ parts, float* __restrict__ dbias, int w, int heads, int ctas_per_head) {
     const int nw = 2 * w - 1, cs = w + 32;
