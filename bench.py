@@ -174,6 +174,24 @@ def run_reference(args, cfg):
     print(json.dumps(line), flush=True)
 
 
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per (batch, window, head) item from the ncu
+# captures summarised under profiles/ (config 3 cut to 254 token rows, 13 056 items); traffic grows in
+# proportion to the item count, so a full launch is this figure times its items.  None = not captured.
+NCU_DRAM_BYTES_PER_ITEM = {
+    "swin_fwd_tc_kernel": 63833,
+    "swin_bwd_tc_kernel<key side>": 96401,
+    "swin_bwd_tc_kernel<query side>": 81609,
+}
+
+
+def ncu_traffic(kernel, cfg):
+    per_item = NCU_DRAM_BYTES_PER_ITEM.get(kernel)
+    if per_item is None or cfg.head_dim != 32 or cfg.window != 16:
+        return None
+    mh, mw = -(-cfg.H // cfg.window), -(-cfg.W // cfg.window)
+    return per_item * cfg.B * mh * mw * cfg.heads
+
+
 def workload_config(cfg, l2_note):
     return {"workload": f"{cfg.name}: B={cfg.B}, token grid {cfg.H}x{cfg.W}, {cfg.heads} heads x d={cfg.head_dim}, "
                         f"window {cfg.window}, shift {cfg.shift_h}, lat non-periodic / lon periodic, fwd+bwd",
@@ -281,6 +299,7 @@ def main():
     sampler = ClockSampler(local_rank)
     sampler.start()
     launches0 = terra.launch_count()
+    terra.profile_enable(True)         # the library brackets each of its main kernels with CUDA events on this stream
     barrier()
     t_start = torch.cuda.Event(enable_timing=True)
     t_end = torch.cuda.Event(enable_timing=True)
@@ -296,6 +315,10 @@ def main():
     t_end.record(stream)
     barrier()
     launches = terra.launch_count() - launches0
+    kernel_ms = {}
+    for kname, kms in terra.profile_read():
+        kernel_ms.setdefault(kname, []).append(kms)
+    terra.profile_enable(False)
     clocks = sampler.stop()
     total_ms = t_start.elapsed_time(t_end)
     t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
@@ -342,10 +365,24 @@ def main():
     if rank == 0:
         peak_tf = peaks["bf16_tflops"]
         peak_bw = peaks["hbm_gbs"]
-        dom_is_bwd = bwd_ms >= fwd_ms
-        dom_flops = wk["flop_bwd"] if dom_is_bwd else wk["flop_fwd"]
-        dom_ms = bwd_ms if dom_is_bwd else fwd_ms
-        achieved = dom_flops / (dom_ms * 1e-3) / 1e12
+        # Algorithmic FLOP per launch of each kernel (strict convention, per allowed pair per head):
+        # forward 4d (QK^T, PV); key side 4d (dV, dK); query side 4d (dP, dQ).  The recomputed S of both
+        # backward kernels and the key side's own dP are not counted.
+        pairs = wk["score_elements"]
+        d = cfg.head_dim
+        kernel_flop = {"swin_fwd_tc_kernel": 4 * d * pairs, "swin_fwd_mma_kernel": 4 * d * pairs,
+                       "swin_bwd_tc_kernel<key side>": 4 * d * pairs, "swin_bwd_tc_kernel<query side>": 4 * d * pairs,
+                       "swin_bwd_mma_kernel<key tiles>": 4 * d * pairs, "swin_bwd_mma_kernel<query tiles>": 4 * d * pairs,
+                       "swin_bwd_delta_kernel": 0}
+        kernels = []
+        for kname, vals in kernel_ms.items():
+            avg = statistics.mean(vals)
+            kernels.append({"kernel": kname, "launches": len(vals), "avg_ms": avg,
+                            "tflops": kernel_flop.get(kname, 0) / (avg * 1e-3) / 1e12,
+                            "dram_bytes_ncu": ncu_traffic(kname, cfg)})
+        kernels.sort(key=lambda r: -r["avg_ms"] * r["launches"])
+        dom = kernels[0] if kernels else {"kernel": "none", "avg_ms": bwd_ms, "tflops": 0.0, "dram_bytes_ncu": None}
+        achieved = dom["tflops"]
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
@@ -359,9 +396,11 @@ def main():
             "breakdown_ms": {"route": route_ms, "fwd": fwd_ms, "bwd": bwd_ms},
             "fwd_tflops": wk["flop_fwd"] / (fwd_ms * 1e-3) / 1e12,
             "bwd_tflops": wk["flop_bwd"] / (bwd_ms * 1e-3) / 1e12,
-            "roofline": {"bound": "tensor", "kernel": "terra_swin_attn_bwd launches" if dom_is_bwd else "terra_swin_attn_fwd launch",
+            "roofline": {"bound": "tensor", "kernel": dom["kernel"], "avg_ms": dom["avg_ms"],
                          "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved / peak_tf,
-                         "traffic": None, "peak_kind": f"{peak_kind} burst bf16"},
+                         "traffic": dom["dram_bytes_ncu"], "peak_kind": f"{peak_kind} burst bf16",
+                         "note": "dominant kernel by time; achieved = its algorithmic FLOP / its CUDA-event duration"},
+            "kernels": kernels,
             "roofline_hbm": {"bound": "hbm", "achieved": (wk["bytes_fwd"] + wk["bytes_bwd"]) / (ms_step * 1e-3) / 1e9,
                              "peak": peak_bw, "unit": "GB/s",
                              "frac": (wk["bytes_fwd"] + wk["bytes_bwd"]) / (ms_step * 1e-3) / 1e9 / peak_bw,

@@ -145,6 +145,17 @@ int terra_swin_attn_fwd_noalloc(const terra_swin_desc* desc, const void* q, cons
  */
 int terra_swin_check(void* stream);
 
+/*
+ * Per-kernel timing for benchmarks (the paper has no counterpart).  While enabled, the library brackets each
+ * of its main kernel launches with CUDA events on the launching stream.  terra_profile_enable(1) clears the
+ * record and starts, (0) clears and stops; terra_profile_count gives the number of recorded launches;
+ * terra_profile_get waits for launch `index` and returns its kernel name (truncated to name_bytes) and
+ * duration in milliseconds.  Host-only; off by default; not meant for use during stream capture.
+ */
+int terra_profile_enable(int on);
+int terra_profile_count(void);
+int terra_profile_get(int index, char* name, int name_bytes, float* ms);
+
 /* Static text for a terra_status.  Host-only. */
 const char* terra_strerror(int status);
 

@@ -17,7 +17,7 @@ from .build import LIB_PATH
 TERRA_OK = 0
 EXPORTS = ("terra_route_sizes", "terra_window_route", "terra_swin_workspace_bytes", "terra_swin_attn_fwd",
            "terra_swin_attn_fwd_noalloc", "terra_swin_attn_bwd", "terra_swin_check", "terra_strerror", "terra_last_cuda_error",
-           "terra_launch_count")
+           "terra_launch_count", "terra_profile_enable", "terra_profile_count", "terra_profile_get")
 
 
 class TerraError(RuntimeError):
@@ -62,6 +62,9 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
     lib.terra_strerror.restype = ctypes.c_char_p
     lib.terra_last_cuda_error.restype = ctypes.c_char_p
     lib.terra_launch_count.restype = ctypes.c_int64
+    lib.terra_profile_enable.argtypes = [ctypes.c_int]
+    lib.terra_profile_count.restype = ctypes.c_int
+    lib.terra_profile_get.argtypes = [ctypes.c_int, ctypes.c_char_p, ctypes.c_int, ctypes.POINTER(ctypes.c_float)]
     if path is None:
         _lib = lib
     return lib
@@ -98,6 +101,22 @@ def _stream() -> ctypes.c_void_p:
 def terra_swin_check() -> None:
     """Waits for the current stream; raises TerraError(6) if a kernel gave up on a bounded wait."""
     _check(load_library().terra_swin_check(_stream()))
+
+
+def profile_enable(on: bool) -> None:
+    load_library().terra_profile_enable(int(on))
+
+
+def profile_read() -> list:
+    """[(kernel name, milliseconds)] of every launch recorded since profile_enable(True)."""
+    lib = load_library()
+    out = []
+    name = ctypes.create_string_buffer(64)
+    ms = ctypes.c_float()
+    for i in range(lib.terra_profile_count()):
+        if lib.terra_profile_get(i, name, 64, ctypes.byref(ms)) == TERRA_OK:
+            out.append((name.value.decode(), float(ms.value)))
+    return out
 
 
 def launch_count() -> int:

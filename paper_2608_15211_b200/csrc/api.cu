@@ -1,5 +1,7 @@
 // C ABI of the shifted-window attention library: argument checks, geometry, launches.
 #include <atomic>
+#include <mutex>
+#include <vector>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
@@ -11,7 +13,34 @@
 namespace terra {
 
 static std::atomic<long long> g_launches{0};
-void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+
+struct ProfEntry { const char* name; cudaEvent_t begin, end; bool closed; };
+static std::mutex g_prof_mutex;
+static bool g_prof_on = false;
+static std::vector<ProfEntry> g_prof;
+
+void prof_begin(const char* name, cudaStream_t stream) {
+    std::lock_guard<std::mutex> lock(g_prof_mutex);
+    if (!g_prof_on) return;
+    ProfEntry e{name, nullptr, nullptr, false};
+    if (cudaEventCreate(&e.begin) != cudaSuccess || cudaEventCreate(&e.end) != cudaSuccess) return;
+    cudaEventRecord(e.begin, stream);
+    g_prof.push_back(e);
+}
+
+void count_launch(cudaStream_t stream) {
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    std::lock_guard<std::mutex> lock(g_prof_mutex);
+    if (g_prof_on && !g_prof.empty() && !g_prof.back().closed) {
+        cudaEventRecord(g_prof.back().end, stream);
+        g_prof.back().closed = true;
+    }
+}
+
+static void prof_clear() {
+    for (auto& e : g_prof) { cudaEventDestroy(e.begin); cudaEventDestroy(e.end); }
+    g_prof.clear();
+}
 
 static thread_local char g_cuda_error[256] = "";
 
@@ -190,6 +219,33 @@ int terra_swin_check(void* stream) {
     e = read_bwd_tc_status(&timed_out_bwd);
     if (e != cudaSuccess) return cuda_fail(e, "terra_swin_check");
     return (timed_out || timed_out_bwd) ? TERRA_ERR_DEVICE_TIMEOUT : TERRA_OK;
+}
+
+int terra_profile_enable(int on) {
+    std::lock_guard<std::mutex> lock(g_prof_mutex);
+    prof_clear();
+    g_prof_on = on != 0;
+    return TERRA_OK;
+}
+
+int terra_profile_count(void) {
+    std::lock_guard<std::mutex> lock(g_prof_mutex);
+    return (int)g_prof.size();
+}
+
+int terra_profile_get(int index, char* name, int name_bytes, float* ms) {
+    std::lock_guard<std::mutex> lock(g_prof_mutex);
+    if (index < 0 || index >= (int)g_prof.size() || !ms) return TERRA_ERR_INVALID_ARG;
+    const ProfEntry& e = g_prof[index];
+    if (!e.closed) return TERRA_ERR_INVALID_ARG;
+    cudaError_t err = cudaEventSynchronize(e.end);
+    if (err == cudaSuccess) err = cudaEventElapsedTime(ms, e.begin, e.end);
+    if (err != cudaSuccess) return cuda_fail(err, "terra_profile_get");
+    if (name && name_bytes > 0) {
+        std::strncpy(name, e.name, (size_t)name_bytes - 1);
+        name[name_bytes - 1] = 0;
+    }
+    return TERRA_OK;
 }
 
 const char* terra_strerror(int status) {

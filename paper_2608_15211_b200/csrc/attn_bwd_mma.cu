@@ -390,10 +390,11 @@ cudaError_t launch_one(const Geo& g, const void* q, const void* k, const void* v
     long long cpg = ((long long)sm_count * occ) / groups;
     if (cpg < 1) cpg = 1;
     if (cpg > items) cpg = items;
+    prof_begin(KV ? "swin_bwd_mma_kernel<key tiles>" : "swin_bwd_mma_kernel<query tiles>", stream);
     kern<<<(unsigned)(cpg * groups), NTHREADS, smem, stream>>>(
         g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)d_o, bias,
         lse, delta, (__nv_bfloat16*)out1, (__nv_bfloat16*)out2, dbias, tiles, (int)cpg, KV ? 0 : acc_stride_for(g));
-    count_launch();
+    count_launch(stream);
     return cudaGetLastError();
 }
 
@@ -404,11 +405,12 @@ cudaError_t launch_bwd_delta(const Geo& g, const void* o, const void* d_o, float
     const int lpr = g.d / 8;
     const long long threads = rows * lpr;
     const unsigned blocks = (unsigned)((threads + 255) / 256);
+    prof_begin("swin_bwd_delta_kernel", stream);
     if (g.d == 32)
         swin_bwd_delta_kernel<32><<<blocks, 256, 0, stream>>>((const __nv_bfloat16*)o, (const __nv_bfloat16*)d_o, delta, rows);
     else
         swin_bwd_delta_kernel<64><<<blocks, 256, 0, stream>>>((const __nv_bfloat16*)o, (const __nv_bfloat16*)d_o, delta, rows);
-    count_launch();
+    count_launch(stream);
     return cudaGetLastError();
 }
 

@@ -631,21 +631,23 @@ cudaError_t launch_bwd_tc(const Geo& g, const void* q, const void* k, const void
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(swin_bwd_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
+    prof_begin("swin_bwd_tc_kernel<key side>", stream);
     swin_bwd_tc_kernel<true><<<grid, kThreads, kSmemBytes, stream>>>(
         g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)d_o, prep, lse, delta,
         (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, nullptr, items, (int)cph);
-    count_launch();
+    count_launch(stream);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
+    prof_begin("swin_bwd_tc_kernel<query side>", stream);
     swin_bwd_tc_kernel<false><<<grid, kThreads, kSmemBytes, stream>>>(
         g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)d_o, prep, lse, delta,
         (__nv_bfloat16*)dq, nullptr, parts, items, (int)cph);
-    count_launch();
+    count_launch(stream);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     const int nrows = (2 * g.w - 1) * (2 * g.w - 1) * g.heads;
     swin_bwd_tc_dbias_finalize_kernel<<<(nrows + 255) / 256, 256, 0, stream>>>(parts, dbias, g.w, g.heads, (int)cph);
-    count_launch();
+    count_launch(stream);
     return cudaGetLastError();
 }
 

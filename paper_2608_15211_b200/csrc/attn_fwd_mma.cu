@@ -247,9 +247,10 @@ cudaError_t launch_fwd_mma(const Geo& g, const void* q, const void* k, const voi
     auto kern = (g.d == 32) ? swin_fwd_mma_kernel<32> : swin_fwd_mma_kernel<64>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
+    prof_begin("swin_fwd_mma_kernel", stream);
     kern<<<(unsigned)items, NTHREADS, smem, stream>>>(g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k,
                                                       (const __nv_bfloat16*)v, bias, (__nv_bfloat16*)o, lse, qtiles);
-    count_launch();
+    count_launch(stream);
     return cudaGetLastError();
 }
 

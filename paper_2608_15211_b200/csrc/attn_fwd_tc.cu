@@ -534,22 +534,23 @@ cudaError_t launch_fwd_tc(const Geo& g, const void* q, const void* k, const void
     const long long items = (long long)g.B * g.Mh * g.Mw * g.heads;
     float* prep = reinterpret_cast<float*>(workspace);
     swin_fwd_bias_prep_kernel<<<g.heads, 256, 0, stream>>>(bias, prep, g.w, g.heads);
-    count_launch();
+    count_launch(stream);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(swin_fwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
     const unsigned grid = (unsigned)(items < sm_count ? items : sm_count);
+    prof_begin("swin_fwd_tc_kernel", stream);
     swin_fwd_tc_kernel<<<grid, kThreads, kSmemBytes, stream>>>(g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k,
                                                                (const __nv_bfloat16*)v, prep, (__nv_bfloat16*)o, lse, items);
-    count_launch();
+    count_launch(stream);
     return cudaGetLastError();
 }
 
 // prepared bias tables for every head (also used by the backward kernels)
 cudaError_t launch_bias_prep(const Geo& g, const float* bias, float* prep, cudaStream_t stream) {
     swin_fwd_bias_prep_kernel<<<g.heads, 256, 0, stream>>>(bias, prep, g.w, g.heads);
-    count_launch();
+    count_launch(stream);
     return cudaGetLastError();
 }
 

@@ -46,14 +46,14 @@ cudaError_t launch_route(const Geo& g, int32_t* perm, int32_t* inv_perm, int32_t
     if (perm || inv_perm || pos || label) {
         const int n = g.H * g.W;
         route_tokens_kernel<<<(n + 255) / 256, 256, 0, stream>>>(g, perm, inv_perm, pos, label);
-        count_launch();
+        count_launch(stream);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
     if (win_offsets) {
         const int n = g.Mh * g.Mw + 1;
         route_offsets_kernel<<<(n + 255) / 256, 256, 0, stream>>>(g, win_offsets);
-        count_launch();
+        count_launch(stream);
         return cudaGetLastError();
     }
     return cudaSuccess;

@@ -8,7 +8,10 @@
 
 namespace terra {
 
-void count_launch();   // bumps the process-wide kernel launch counter
+void count_launch(cudaStream_t stream);   // after every launch: bumps the launch counter, closes an open timing scope
+// Optional per-kernel timing (terra_profile_*): opens a scope (CUDA event on `stream`) that the next
+// count_launch closes.  Does nothing unless profiling is enabled.
+void prof_begin(const char* name, cudaStream_t stream);
 
 cudaError_t launch_route(const Geo& g, int32_t* perm, int32_t* inv_perm, int32_t* win_offsets,
                          int32_t* pos, int32_t* label, cudaStream_t stream);
