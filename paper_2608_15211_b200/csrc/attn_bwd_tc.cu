@@ -12,8 +12,9 @@
 // MMAs), two loader warps gathering the window's rows with
 // cp.async into the 64-byte-swizzled operand layout.  CTAs are bound to one head (grid = heads x CTAs per
 // head), so the head's bias table is staged once per CTA and the bias-gradient table belongs to one head.
-// TMEM, per 128-row tile (256 columns):  query side [S 112 | dP 112 | dQ 32], key side
-// [S^T 96 | dP^T 96 | dV 32 | dK 32]; the bf16 P / dS overwrite the fp32 S / dP they were computed from.
+// TMEM, per 128-row tile (256 columns): two buffers [S 48 | dP 48] for column blocks in flight (the MMAs
+// run up to two blocks ahead of the elementwise warpgroup), then the accumulators: query side dQ (32
+// columns), key side dV and dK (32 each).  The bf16 P / dS overwrite the fp32 S / dP they came from.
 // Every mbarrier wait is bounded; on expiry the CTA raises an abort flag and all roles leave their loops.
 #include "swin_common.cuh"
 #include "swin_kernels.h"
@@ -240,19 +241,20 @@ swin_bwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
                    const float* __restrict__ bias_prep, const float* __restrict__ lse, const float* __restrict__ delta,
                    __nv_bfloat16* __restrict__ out1, __nv_bfloat16* __restrict__ out2, float* __restrict__ dbias,
                    long long n_items, int ctas_per_head) {
-    constexpr int CB = KV ? 96 : 112;           // columns per block
-    constexpr int kColAcc1 = 2 * CB;            // key side: dV at 192; query side: dQ at 224
-    constexpr int kColAcc2 = 2 * CB + 32;       // key side: dK at 224
+    constexpr int CB = 48;                      // columns per block; two blocks (buffers) in flight per tile
+    constexpr int kBufCols = 2 * CB;            // one buffer = [S 48 | dP 48]
+    constexpr int kColAcc1 = 2 * kBufCols;      // key side: dV at 192; query side: dQ at 192
+    constexpr int kColAcc2 = 2 * kBufCols + 32; // key side: dK at 224
     extern __shared__ __align__(1024) unsigned char smem[];
     const uint32_t smem0 = smem_u32(smem);
     const uint32_t bar0 = smem0 + kOffBars;
     auto bar_full = [&](int s) { return bar0 + 8u * s; };
     auto bar_empty = [&](int s) { return bar0 + 8u * (kStages + s); };
-    auto bar_sdp = [&](int t) { return bar0 + 8u * (2 * kStages + t); };       // S and dP of a block are in TMEM
-    auto bar_ds = [&](int t) { return bar0 + 8u * (2 * kStages + 2 + t); };    // bf16 P / dS of a block are in TMEM
-    auto bar_acc = [&](int t) { return bar0 + 8u * (2 * kStages + 4 + t); };   // the item's accumulators are final
-    auto bar_free = [&](int t) { return bar0 + 8u * (2 * kStages + 6 + t); };  // the tile's TMEM region may be reused
-    unsigned char* tail = smem + kOffBars + 8 * (2 * kStages + 8);
+    auto bar_sdp = [&](int t, int b) { return bar0 + 8u * (2 * kStages + 2 * t + b); };      // S and dP of a block are in buffer b
+    auto bar_ds = [&](int t, int b) { return bar0 + 8u * (2 * kStages + 4 + 2 * t + b); };   // bf16 P / dS of a block are in buffer b
+    auto bar_acc = [&](int t) { return bar0 + 8u * (2 * kStages + 8 + t); };    // the item's accumulators are final
+    auto bar_free = [&](int t) { return bar0 + 8u * (2 * kStages + 10 + t); };  // the accumulators have been read back
+    unsigned char* tail = smem + kOffBars + 8 * (2 * kStages + 12);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail);
     volatile int* cta_abort = reinterpret_cast<volatile int*>(tail + 8);
 
@@ -266,8 +268,10 @@ swin_bwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
             mbar_init(bar_empty(s), 2);      // one arrival per MMA issuer
         }
         for (int t = 0; t < 2; ++t) {
-            mbar_init(bar_sdp(t), 1);
-            mbar_init(bar_ds(t), 128);
+            for (int b = 0; b < 2; ++b) {
+                mbar_init(bar_sdp(t, b), 1);
+                mbar_init(bar_ds(t, b), 128);
+            }
             mbar_init(bar_acc(t), 1);
             mbar_init(bar_free(t), 128);
         }
@@ -389,17 +393,17 @@ swin_bwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
                 const uint64_t so = (uint64_t)((s * kStageBytes) >> 4);
                 const uint64_t ro = so + (uint64_t)((t * 128 * kRowBytes) >> 4), co = so + (uint64_t)((cb * CB * kRowBytes) >> 4);
                 const uint32_t idesc = make_idesc_bf16(128, ncols, 0, 0);
-                const uint32_t t_s = tmem_base + t * 256, t_dp = tmem_base + t * 256 + CB;
+                const uint32_t t_s = tmem_base + t * 256 + (cb & 1) * kBufCols, t_dp = t_s + CB;
                 mma_ss(t_s, d_r1 + ro, d_c1 + co, idesc, 0u);
                 mma_ss(t_s, d_r1 + ro + 2, d_c1 + co + 2, idesc, 1u);
                 mma_ss(t_dp, d_r2 + ro, d_c2 + co, idesc, 0u);
                 mma_ss(t_dp, d_r2 + ro + 2, d_c2 + co + 2, idesc, 1u);
-                mma_commit(bar_sdp(t));
+                mma_commit(bar_sdp(t, cb & 1));
             };
             // accumulations of column block cb: query side dQ += dS C1; key side dV += P C2, dK += dS C1
             auto issue_acc = [&](int s, int t, int cb, int ncols) {
                 const uint64_t co = (uint64_t)((s * kStageBytes + cb * CB * kRowBytes) >> 4);
-                const uint32_t t_p = tmem_base + t * 256, t_ds = tmem_base + t * 256 + CB;
+                const uint32_t t_p = tmem_base + t * 256 + (cb & 1) * kBufCols, t_ds = t_p + CB;
                 const uint32_t first = cb == 0 ? 0u : 1u;
                 for (int ks = 0; ks < (ncols >> 4); ++ks) {
                     const uint32_t acc = (ks > 0) ? 1u : first;
@@ -412,7 +416,7 @@ swin_bwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
                 }
             };
             const int t = warp - kMmaWarp;      // this issuer's tile
-            int kuse = 0, n_ds = 0, n_free = 0, n_acc_used = 0;
+            int kuse = 0, n_ds[2] = {0, 0}, n_free = 0, n_acc_used = 0;
             for (long long it = cta_in_head; ok && it < n_items; it += ctas_per_head, ++kuse) {
                 const int s = kuse % kStages;
                 const Item x = make_item(g, it);
@@ -424,37 +428,27 @@ swin_bwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
                     continue;
                 }
                 fence_proxy_async();
+                tc_fence_after();
+                // Both buffers are free here: the previous item's elementwise work is over (its ds barriers
+                // were waited for) and the accumulation MMAs that read the buffers were issued earlier by this
+                // lane, so they execute first.  Run two blocks ahead of the elementwise warpgroup.
+                issue_sdp(s, t, 0, min(CB, x.npad));
+                if (ncb > 1) issue_sdp(s, t, 1, min(CB, x.npad - CB));
                 for (int cb = 0; cb < ncb && ok; ++cb) {
-                    const int ncols = min(CB, x.npad - cb * CB);
-                    // S / dP columns are free as soon as the previous accumulation MMAs (issued earlier by this
-                    // lane, executed in order) have read them; only the accumulator columns have to wait until
-                    // the warpgroup has read the previous item's results.
-                    if (cb > 0) {
-                        ok = mbar_wait(bar_ds(t), n_ds & 1, cta_abort);
-                        ++n_ds;
-                        if (ok && cb == 1 && n_acc_used > n_free) {
-                            ok = mbar_wait(bar_free(t), n_free & 1, cta_abort);
-                            ++n_free;
-                        }
-                        if (ok) {
-                            tc_fence_after();
-                            issue_acc(s, t, cb - 1, CB);
-                        }
+                    const int buf = cb & 1;
+                    ok = mbar_wait(bar_ds(t, buf), n_ds[buf] & 1, cta_abort);
+                    ++n_ds[buf];
+                    if (ok && cb == 0 && n_acc_used > n_free) {
+                        // the first accumulation overwrites the accumulators: the previous item's must have been read
+                        ok = mbar_wait(bar_free(t), n_free & 1, cta_abort);
+                        ++n_free;
                     }
                     if (!ok) break;
                     tc_fence_after();
-                    issue_sdp(s, t, cb, ncols);
+                    issue_acc(s, t, cb, min(CB, x.npad - cb * CB));
+                    if (cb + 2 < ncb) issue_sdp(s, t, cb + 2, min(CB, x.npad - (cb + 2) * CB));
                 }
                 if (!ok) break;
-                ok = mbar_wait(bar_ds(t), n_ds & 1, cta_abort);
-                ++n_ds;
-                if (ok && ncb == 1 && n_acc_used > n_free) {
-                    ok = mbar_wait(bar_free(t), n_free & 1, cta_abort);
-                    ++n_free;
-                }
-                if (!ok) break;
-                tc_fence_after();
-                issue_acc(s, t, ncb - 1, x.npad - (ncb - 1) * CB);
                 mma_commit(bar_acc(t));
                 ++n_acc_used;
                 mma_commit(bar_empty(s));
@@ -472,7 +466,7 @@ swin_bwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
         const float scale = g.scale_log2e;
         const float out_scale = g.scale_log2e * kLn2;          // dQ and dK carry the score scale
         const int dbias_limit = 4 * (2 * c0 + 1);
-        int kuse = 0, n_sdp = 0, n_acc = 0;
+        int kuse = 0, n_sdp[2] = {0, 0}, n_acc = 0;
         for (long long it = cta_in_head; it < n_items; it += ctas_per_head, ++kuse) {
             const Item x = make_item(g, it);
             if (wg >= x.ntiles) continue;
@@ -493,19 +487,21 @@ swin_bwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
             bool ok = true;
             for (int cb = 0; cb < ncb; ++cb) {
                 const int ncols = min(CB, x.npad - cb * CB);
-                ok = __all_sync(0xffffffffu, mbar_wait(bar_sdp(wg), n_sdp & 1, cta_abort));
+                const int buf = cb & 1;
+                const uint32_t t_buf = t_reg + buf * kBufCols;
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_sdp(wg, buf), n_sdp[buf] & 1, cta_abort));
                 if (!ok) break;
-                ++n_sdp;
+                ++n_sdp[buf];
                 tc_fence_after();
                 if (x.masked)
-                    bwd_block<KV, true, true>(t_reg, t_reg + CB, cb * CB, ncols, rc, st_a, scale, dbias_limit);
+                    bwd_block<KV, true, true>(t_buf, t_buf + CB, cb * CB, ncols, rc, st_a, scale, dbias_limit);
                 else if (x.ragged)
-                    bwd_block<KV, false, true>(t_reg, t_reg + CB, cb * CB, ncols, rc, st_a, scale, dbias_limit);
+                    bwd_block<KV, false, true>(t_buf, t_buf + CB, cb * CB, ncols, rc, st_a, scale, dbias_limit);
                 else
-                    bwd_block<KV, false, false>(t_reg, t_reg + CB, cb * CB, ncols, rc, st_a, scale, dbias_limit);
+                    bwd_block<KV, false, false>(t_buf, t_buf + CB, cb * CB, ncols, rc, st_a, scale, dbias_limit);
                 tmem_st_wait();
                 tc_fence_before();
-                mbar_arrive(bar_ds(wg));
+                mbar_arrive(bar_ds(wg, buf));
             }
             if (!ok) break;
             if (!__all_sync(0xffffffffu, mbar_wait(bar_acc(wg), n_acc & 1, cta_abort))) break;
