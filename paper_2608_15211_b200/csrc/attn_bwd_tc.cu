@@ -61,7 +61,8 @@ constexpr int kOffBias = kStages * kStageBytes;                // the head's pre
 constexpr int kOffDBias = kOffBias + kFwdBiasFloats * 4;       // query side: one bias-gradient table per elementwise warp
 constexpr int kDBiasFloats = 1536;                             // >= 2 c0 + 1 for w <= 16
 constexpr int kOffBars = kOffDBias + 8 * kDBiasFloats * 4;
-constexpr int kSmemBytes = kOffBars + 256;
+constexpr int kOffOutStage = kOffBars + 256;                   // per elementwise warp: 32 output rows on their way out (query side)
+constexpr int kSmemBytes = kOffOutStage + 8 * 32 * kRowBytes;
 
 __device__ __forceinline__ int code_stride(int w) { return w + 32; }
 
@@ -517,37 +518,61 @@ swin_bwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
             tmem_ld_wait();
             tc_fence_before();
             mbar_arrive(bar_free(wg));
-            if (tok >= 0) {
-                const size_t row_off = (((size_t)x.b * HW + (size_t)tok) * g.heads + head) * kD;
-                if (KV) {
-                    uint4* dv_dst = reinterpret_cast<uint4*>(out2 + row_off);     // dV
-                    uint4* dk_dst = reinterpret_cast<uint4*>(out1 + row_off);     // dK
+            if (KV) {
+                // Each thread holds one 64-byte row of dV and of dK.  Rows go through a per-warp shared-memory
+                // tile (the bias-gradient area is unused on the key side) so that one store instruction
+                // writes 8 whole rows (4 lanes x 16 bytes each) instead of 32 scattered 16-byte pieces.
+                unsigned char* stg = smem + kOffDBias + warp * 2 * 32 * kRowBytes;
 #pragma unroll
-                    for (int c4 = 0; c4 < 4; ++c4) {
-                        uint4 a, b;
-                        a.x = pack_bf16(__uint_as_float(r1[c4 * 8 + 0]), __uint_as_float(r1[c4 * 8 + 1]));
-                        a.y = pack_bf16(__uint_as_float(r1[c4 * 8 + 2]), __uint_as_float(r1[c4 * 8 + 3]));
-                        a.z = pack_bf16(__uint_as_float(r1[c4 * 8 + 4]), __uint_as_float(r1[c4 * 8 + 5]));
-                        a.w = pack_bf16(__uint_as_float(r1[c4 * 8 + 6]), __uint_as_float(r1[c4 * 8 + 7]));
-                        b.x = pack_bf16(__uint_as_float(r2[c4 * 8 + 0]) * out_scale, __uint_as_float(r2[c4 * 8 + 1]) * out_scale);
-                        b.y = pack_bf16(__uint_as_float(r2[c4 * 8 + 2]) * out_scale, __uint_as_float(r2[c4 * 8 + 3]) * out_scale);
-                        b.z = pack_bf16(__uint_as_float(r2[c4 * 8 + 4]) * out_scale, __uint_as_float(r2[c4 * 8 + 5]) * out_scale);
-                        b.w = pack_bf16(__uint_as_float(r2[c4 * 8 + 6]) * out_scale, __uint_as_float(r2[c4 * 8 + 7]) * out_scale);
-                        dv_dst[c4] = a;
-                        dk_dst[c4] = b;
-                    }
-                } else {
-                    uint4* dq_dst = reinterpret_cast<uint4*>(out1 + row_off);
+                for (int c4 = 0; c4 < 4; ++c4) {
+                    uint4 a, b;
+                    a.x = pack_bf16(__uint_as_float(r1[c4 * 8 + 0]), __uint_as_float(r1[c4 * 8 + 1]));
+                    a.y = pack_bf16(__uint_as_float(r1[c4 * 8 + 2]), __uint_as_float(r1[c4 * 8 + 3]));
+                    a.z = pack_bf16(__uint_as_float(r1[c4 * 8 + 4]), __uint_as_float(r1[c4 * 8 + 5]));
+                    a.w = pack_bf16(__uint_as_float(r1[c4 * 8 + 6]), __uint_as_float(r1[c4 * 8 + 7]));
+                    b.x = pack_bf16(__uint_as_float(r2[c4 * 8 + 0]) * out_scale, __uint_as_float(r2[c4 * 8 + 1]) * out_scale);
+                    b.y = pack_bf16(__uint_as_float(r2[c4 * 8 + 2]) * out_scale, __uint_as_float(r2[c4 * 8 + 3]) * out_scale);
+                    b.z = pack_bf16(__uint_as_float(r2[c4 * 8 + 4]) * out_scale, __uint_as_float(r2[c4 * 8 + 5]) * out_scale);
+                    b.w = pack_bf16(__uint_as_float(r2[c4 * 8 + 6]) * out_scale, __uint_as_float(r2[c4 * 8 + 7]) * out_scale);
+                    *reinterpret_cast<uint4*>(stg + tile_off<kD>(lane, c4)) = a;                       // dV
+                    *reinterpret_cast<uint4*>(stg + 32 * kRowBytes + tile_off<kD>(lane, c4)) = b;      // dK
+                }
+                __syncwarp();
 #pragma unroll
-                    for (int c4 = 0; c4 < 4; ++c4) {
-                        uint4 b;
-                        b.x = pack_bf16(__uint_as_float(r2[c4 * 8 + 0]) * out_scale, __uint_as_float(r2[c4 * 8 + 1]) * out_scale);
-                        b.y = pack_bf16(__uint_as_float(r2[c4 * 8 + 2]) * out_scale, __uint_as_float(r2[c4 * 8 + 3]) * out_scale);
-                        b.z = pack_bf16(__uint_as_float(r2[c4 * 8 + 4]) * out_scale, __uint_as_float(r2[c4 * 8 + 5]) * out_scale);
-                        b.w = pack_bf16(__uint_as_float(r2[c4 * 8 + 6]) * out_scale, __uint_as_float(r2[c4 * 8 + 7]) * out_scale);
-                        dq_dst[c4] = b;
+                for (int j = 0; j < 4; ++j) {
+                    const int rr = 8 * j + (lane >> 2), c4 = lane & 3;
+                    const int tok_r = __shfl_sync(0xffffffffu, tok, rr);
+                    const uint4 a = *reinterpret_cast<const uint4*>(stg + tile_off<kD>(rr, c4));
+                    const uint4 b = *reinterpret_cast<const uint4*>(stg + 32 * kRowBytes + tile_off<kD>(rr, c4));
+                    if (tok_r >= 0) {
+                        const size_t off = (((size_t)x.b * HW + (size_t)tok_r) * g.heads + head) * kD + c4 * 8;
+                        *reinterpret_cast<uint4*>(out2 + off) = a;
+                        *reinterpret_cast<uint4*>(out1 + off) = b;
                     }
                 }
+                __syncwarp();
+            }
+            if (!KV) {
+                unsigned char* stg = smem + kOffOutStage + warp * 32 * kRowBytes;
+#pragma unroll
+                for (int c4 = 0; c4 < 4; ++c4) {
+                    uint4 b;
+                    b.x = pack_bf16(__uint_as_float(r2[c4 * 8 + 0]) * out_scale, __uint_as_float(r2[c4 * 8 + 1]) * out_scale);
+                    b.y = pack_bf16(__uint_as_float(r2[c4 * 8 + 2]) * out_scale, __uint_as_float(r2[c4 * 8 + 3]) * out_scale);
+                    b.z = pack_bf16(__uint_as_float(r2[c4 * 8 + 4]) * out_scale, __uint_as_float(r2[c4 * 8 + 5]) * out_scale);
+                    b.w = pack_bf16(__uint_as_float(r2[c4 * 8 + 6]) * out_scale, __uint_as_float(r2[c4 * 8 + 7]) * out_scale);
+                    *reinterpret_cast<uint4*>(stg + tile_off<kD>(lane, c4)) = b;                       // dQ
+                }
+                __syncwarp();
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int rr = 8 * j + (lane >> 2), c4 = lane & 3;
+                    const int tok_r = __shfl_sync(0xffffffffu, tok, rr);
+                    const uint4 b = *reinterpret_cast<const uint4*>(stg + tile_off<kD>(rr, c4));
+                    if (tok_r >= 0)
+                        *reinterpret_cast<uint4*>(out1 + (((size_t)x.b * HW + (size_t)tok_r) * g.heads + head) * kD + c4 * 8) = b;
+                }
+                __syncwarp();
             }
         }
     }
