@@ -146,9 +146,25 @@ struct RowCtx {
 // 16 columns of one row: P = exp2(S * scale + bias - lse), dS = P * (dP - delta); packs dS (and P) to bf16.
 //   KV = false: rows are queries (lse, delta per row); adds dS into the bias-gradient table.
 //   KV = true : rows are keys    (lse, delta per column).
-template <bool KV, bool MASKED, bool RAGGED>
+// Two table updates whose entries cannot coincide (see bwd_block), issued together so that their
+// load-add-store latencies overlap.
+__device__ __forceinline__ void rmw2_shared_f32(uint32_t addr0, float v0, uint32_t addr1, float v1) {
+    asm volatile(
+        "{\n\t.reg .f32 t0, t1;\n\t"
+        "ld.shared.f32 t0, [%0];\n\t"
+        "ld.shared.f32 t1, [%2];\n\t"
+        "add.f32 t0, t0, %1;\n\t"
+        "add.f32 t1, t1, %3;\n\t"
+        "st.shared.f32 [%0], t0;\n\t"
+        "st.shared.f32 [%2], t1;\n\t}\n" ::"r"(addr0), "f"(v0), "r"(addr1), "f"(v1) : "memory");
+}
+
+// HOLD = 0: add dS into the bias-gradient table now; 1: only hand the 16 (address, dS) pairs back in
+// held_addr / held_ds; 2: add them together with this step's pairs, two entries at a time.
+template <bool KV, bool MASKED, bool RAGGED, int HOLD = 0>
 __device__ __forceinline__ void bwd_cols16(const uint32_t (&rs)[16], const uint32_t (&rp)[16], uint32_t (&pk_p)[8], uint32_t (&pk_ds)[8],
-                                           int c, const RowCtx& rc, uint32_t st_a, float scale, int dbias_limit) {
+                                           int c, const RowCtx& rc, uint32_t st_a, float scale, int dbias_limit,
+                                           uint32_t (&held_addr)[16], float (&held_ds)[16]) {
     // all shared-memory loads first (the explicit loads keep their order), then the arithmetic
     int co[16], kl[16];
     float l2[16], dl[16], bv[16];
@@ -185,7 +201,16 @@ __device__ __forceinline__ void bwd_cols16(const uint32_t (&rs)[16], const uint3
         p[e] = fast_exp2(xv);
         ds[e] = p[e] * (__uint_as_float(rp[e]) - del_e);
     }
-    if (!KV) {
+    if (!KV && HOLD == 1) {
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+            held_addr[e] = rc.dbias_row + co[e];
+            held_ds[e] = ds[e];
+        }
+    } else if (!KV && HOLD == 2) {
+#pragma unroll
+        for (int e = 0; e < 16; ++e) rmw2_shared_f32(held_addr[e], held_ds[e], rc.dbias_row + co[e], ds[e]);
+    } else if (!KV) {
         // one warp instruction touches 32 different table entries (32 different rows, one column)
 #pragma unroll
         for (int e = 0; e < 16; ++e) {
@@ -209,9 +234,37 @@ template <bool KV, bool MASKED, bool RAGGED>
 __device__ __forceinline__ void bwd_block(uint32_t t_s, uint32_t t_dp, int c_first, int ncols, const RowCtx& rc, uint32_t st_a,
                                           float scale, int dbias_limit) {
     uint32_t sa[16], pa[16], sb[16], pb[16];
+    uint32_t held_addr[16];
+    float held_ds[16];
     const int nsteps = ncols >> 4;
     tmem_ld16(t_s, sa);
     tmem_ld16(t_dp, pa);
+    if (!KV && !RAGGED && nsteps == 3) {
+        // Query side, full block of three 16-column steps.  Table updates of one step must stay in program
+        // order with those of the next step (lane l at column j and lane l + 1 at column j + 1 share an
+        // entry), but columns 32 apart never share one inside a warp: bias codes grow with the slot and
+        // determine the slot distance, and a warp spans only 32 slots.  So steps 0 and 2 are updated
+        // together, two independent entries per instruction group, and the serial chain is a third shorter.
+        uint32_t pk_p[8], pk_ds[8];
+        tmem_ld_wait();
+        tmem_ld16(t_s + 16, sb);
+        tmem_ld16(t_dp + 16, pb);
+        bwd_cols16<KV, MASKED, RAGGED, 1>(sa, pa, pk_p, pk_ds, c_first, rc, st_a, scale, dbias_limit, held_addr, held_ds);
+        tmem_st8(t_dp, pk_ds);
+        tmem_ld_wait();
+        tmem_ld16(t_s + 32, sa);
+        tmem_ld16(t_dp + 32, pa);
+        {
+            uint32_t na[16];
+            float nd[16];
+            bwd_cols16<KV, MASKED, RAGGED, 0>(sb, pb, pk_p, pk_ds, c_first + 16, rc, st_a, scale, dbias_limit, na, nd);
+        }
+        tmem_st8(t_dp + 8, pk_ds);
+        tmem_ld_wait();
+        bwd_cols16<KV, MASKED, RAGGED, 2>(sa, pa, pk_p, pk_ds, c_first + 32, rc, st_a, scale, dbias_limit, held_addr, held_ds);
+        tmem_st8(t_dp + 16, pk_ds);
+        return;
+    }
     for (int i = 0; i < nsteps; i += 2) {
         uint32_t pk_p[8], pk_ds[8];
         tmem_ld_wait();
@@ -219,7 +272,7 @@ __device__ __forceinline__ void bwd_block(uint32_t t_s, uint32_t t_dp, int c_fir
             tmem_ld16(t_s + 16 * (i + 1), sb);
             tmem_ld16(t_dp + 16 * (i + 1), pb);
         }
-        bwd_cols16<KV, MASKED, RAGGED>(sa, pa, pk_p, pk_ds, c_first + 16 * i, rc, st_a, scale, dbias_limit);
+        bwd_cols16<KV, MASKED, RAGGED, 0>(sa, pa, pk_p, pk_ds, c_first + 16 * i, rc, st_a, scale, dbias_limit, held_addr, held_ds);
         if (KV) tmem_st8(t_s + 8 * i, pk_p);
         tmem_st8(t_dp + 8 * i, pk_ds);
         if (i + 1 < nsteps) {
@@ -228,7 +281,7 @@ __device__ __forceinline__ void bwd_block(uint32_t t_s, uint32_t t_dp, int c_fir
                 tmem_ld16(t_s + 16 * (i + 2), sa);
                 tmem_ld16(t_dp + 16 * (i + 2), pa);
             }
-            bwd_cols16<KV, MASKED, RAGGED>(sb, pb, pk_p, pk_ds, c_first + 16 * (i + 1), rc, st_a, scale, dbias_limit);
+            bwd_cols16<KV, MASKED, RAGGED, 0>(sb, pb, pk_p, pk_ds, c_first + 16 * (i + 1), rc, st_a, scale, dbias_limit, held_addr, held_ds);
             if (KV) tmem_st8(t_s + 8 * (i + 1), pk_p);
             tmem_st8(t_dp + 8 * (i + 1), pk_ds);
         }
