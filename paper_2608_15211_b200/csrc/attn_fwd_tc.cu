@@ -170,15 +170,24 @@ __device__ __forceinline__ float softmax_row(uint32_t t_s, int npad, uint32_t bi
     const bool tail = (npad & 16) != 0;
     uint32_t ra[32], rb[32];
     float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-    if (nfull > 0) tmem_ld32(t_s, ra);
-    for (int i = 0; i < nfull; i += 2) {
-        tmem_ld_wait();
-        if (i + 1 < nfull) tmem_ld32(t_s + 32 * (i + 1), rb);
-        max_cols<32>(ra, mx4);
-        if (i + 1 < nfull) {
+    {
+        int i = 0;
+        for (; i + 4 <= nfull; i += 4) {      // 128 columns per round trip to TMEM
+            uint32_t rc[32], rd[32];
+            tmem_ld32(t_s + 32 * i, ra);
+            tmem_ld32(t_s + 32 * (i + 1), rb);
+            tmem_ld32(t_s + 32 * (i + 2), rc);
+            tmem_ld32(t_s + 32 * (i + 3), rd);
             tmem_ld_wait();
-            if (i + 2 < nfull) tmem_ld32(t_s + 32 * (i + 2), ra);
+            max_cols<32>(ra, mx4);
             max_cols<32>(rb, mx4);
+            max_cols<32>(rc, mx4);
+            max_cols<32>(rd, mx4);
+        }
+        for (; i < nfull; ++i) {
+            tmem_ld32(t_s + 32 * i, ra);
+            tmem_ld_wait();
+            max_cols<32>(ra, mx4);
         }
     }
     if (tail) {
