@@ -7,9 +7,9 @@
 //   warp 8           issues tcgen05.mma: S = Q K^T (operands in shared memory), O = P V (P from TMEM)
 //   warps 9-11       loaders: undo the roll, gather the window's Q / K / V rows with cp.async into the
 //                    64-byte-swizzled operand layout, stage the head's bias table and the slot metadata
-// TMEM: columns [256 t, 256 t + 256) belong to query tile t: S (fp32) first, then P (bf16, the first 128
-// columns) and four partial O accumulators (fp32, columns 128..255; key step ks adds into accumulator
-// ks mod 4, so consecutive MMAs do not wait on each other's accumulator) once S has been consumed.
+// TMEM: columns [256 t, 256 t + 256) belong to query tile t: S (fp32) first; as pass 2 consumes it, bf16 P of
+// keys 0..127 goes to columns 0..63, the O accumulator to 64..95 and bf16 P of keys 128..255 to 128..191, so
+// that O += P V over the first 128 keys runs while the softmax of the second 128 keys is still going on.
 // The row maximum is replaced by the upper bound max_j(raw score) * scale + max(bias): softmax is shift
 // invariant, so the result is the same; only the exponent range matters.
 // Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, all roles leave their loops,
@@ -58,8 +58,13 @@ constexpr int kStageBytes = ((kOffRowTok + kMaxSlots * 4 + 1023) / 1024) * 1024;
 constexpr int kBarBytes = 256;
 constexpr int kSmemBytes = kStages * kStageBytes + kBarBytes;
 
-constexpr int kColO = 128;       // first O accumulator inside a query tile's 256-column TMEM region
-constexpr int kOAcc = 4;         // partial O accumulators, 32 columns each
+// TMEM columns inside a query tile's 256-column region once S is being consumed: bf16 P of keys 0..127 in
+// [0, 64), the O accumulator in [64, 96) (S columns that the first half of pass 2 has already read), bf16
+// P of keys 128..255 in [128, 192).  The PV product of the first 128 keys is issued while the softmax
+// warpgroup is still working on the second 128 keys.
+constexpr int kColO = 64;
+constexpr int kColP1 = 128;
+__device__ __forceinline__ int p_col(int chunk32) { return chunk32 < 4 ? 16 * chunk32 : kColP1 + 16 * (chunk32 - 4); }
 
 // Bias codes use a row stride of w + 32 instead of 2w - 1: the 32 rows of a warp (consecutive slots of a
 // full-width window) then read 32 different shared-memory banks.
@@ -165,7 +170,7 @@ __device__ __forceinline__ void max_cols(const uint32_t (&r)[N], float (&mx)[4])
 // flight while the current one is processed.  Returns m (log2 domain); the row sum goes to sum_out.
 template <bool MASKED>
 __device__ __forceinline__ float softmax_row(uint32_t t_s, int npad, uint32_t bias_i, uint32_t a_kc, uint32_t a_klab,
-                                             int label_i, float scale, float bmax, float& sum_out) {
+                                             int label_i, float scale, float bmax, float& sum_out, uint32_t bar_half) {
     const int nfull = npad >> 5;
     const bool tail = (npad & 16) != 0;
     uint32_t ra[32], rb[32];
@@ -207,12 +212,18 @@ __device__ __forceinline__ float softmax_row(uint32_t t_s, int npad, uint32_t bi
         tmem_ld_wait();
         if (i + 1 < nfull) tmem_ld32(t_s + 32 * (i + 1), rb);
         sum += softmax_cols<32, MASKED>(ra, pk, 32 * i, bias_i, a_kc, a_klab, label_i, scale, neg_m);
-        tmem_st16(t_s + 16 * i, pk);
+        tmem_st16(t_s + p_col(i), pk);
         if (i + 1 < nfull) {
             tmem_ld_wait();
             if (i + 2 < nfull) tmem_ld32(t_s + 32 * (i + 2), ra);
             sum += softmax_cols<32, MASKED>(rb, pk, 32 * (i + 1), bias_i, a_kc, a_klab, label_i, scale, neg_m);
-            tmem_st16(t_s + 16 * (i + 1), pk);
+            tmem_st16(t_s + p_col(i + 1), pk);
+        }
+        if (i == 2 && npad > 128) {
+            // P of keys 0..127 is complete: let the MMA lane start O += P V on it while this row goes on
+            tmem_st_wait();
+            tc_fence_before();
+            mbar_arrive(bar_half);
         }
     }
     if (tail) {
@@ -220,7 +231,7 @@ __device__ __forceinline__ float softmax_row(uint32_t t_s, int npad, uint32_t bi
         tmem_ld16(t_s + 32 * nfull, rt);
         tmem_ld_wait();
         sum += softmax_cols<16, MASKED>(rt, pk, 32 * nfull, bias_i, a_kc, a_klab, label_i, scale, neg_m);
-        tmem_st8(t_s + 16 * nfull, pk);
+        tmem_st8(t_s + p_col(nfull), pk);
     }
     sum_out = sum;
     return m;
@@ -240,7 +251,8 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
     auto bar_pready = [&](int t) { return bar0 + 8u * (2 * kStages + 2 + t); };
     auto bar_oready = [&](int t) { return bar0 + 8u * (2 * kStages + 4 + t); };
     auto bar_sfree = [&](int t) { return bar0 + 8u * (2 * kStages + 6 + t); };
-    unsigned char* tail = smem + kStages * kStageBytes + 8 * (2 * kStages + 8);
+    auto bar_phalf = [&](int t) { return bar0 + 8u * (2 * kStages + 8 + t); };   // P of the first 128 keys is in TMEM
+    unsigned char* tail = smem + kStages * kStageBytes + 8 * (2 * kStages + 10);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail);
     volatile int* cta_abort = reinterpret_cast<volatile int*>(tail + 8);
 
@@ -256,6 +268,7 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
             mbar_init(bar_pready(t), 128);
             mbar_init(bar_oready(t), 1);
             mbar_init(bar_sfree(t), 128);
+            mbar_init(bar_phalf(t), 128);
         }
         *cta_abort = 0;
         fence_barrier_init();
@@ -360,12 +373,12 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
                            idesc, ks > 0 ? 1u : 0u);
                 mma_commit(bar_sready(t));
             };
-            auto issue_pv = [&](const Item& x, int s, int t) {
+            // O += P V over key steps [ks0, ks1) of 16 keys; P of step ks sits at TMEM column p_col(ks / 2) + 8 (ks & 1)
+            auto issue_pv = [&](const Item& x, int s, int t, int ks0, int ks1) {
                 const uint32_t va = smem0 + s * kStageBytes + kOffV;
-                for (int ks = 0; ks < x.npad / 16; ++ks)
-                    mma_ts(tmem_base + t * 256 + kColO + 32 * (ks & (kOAcc - 1)), tmem_base + t * 256 + ks * 8,
-                           make_sdesc_sw64(va + ks * 16 * kRowBytes, 512), idesc_pv, ks >= kOAcc ? 1u : 0u);
-                mma_commit(bar_oready(t));
+                for (int ks = ks0; ks < ks1; ++ks)
+                    mma_ts(tmem_base + t * 256 + kColO, tmem_base + t * 256 + p_col(ks >> 1) + 8 * (ks & 1),
+                           make_sdesc_sw64(va + ks * 16 * kRowBytes, 512), idesc_pv, ks > 0 ? 1u : 0u);
             };
             long long it = blockIdx.x;
             Item cur;
@@ -386,6 +399,16 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
                 const int sn = (kuse + 1) % kStages;
                 if (has_next) nx = make_item(g, nxt);
                 bool next_ready = false;
+                const int nks = cur.npad >> 4;
+                // first 128 keys of each tile, as soon as their P is there
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    if (!ok || t >= cur.ntiles) continue;
+                    ok = mbar_wait(bar_phalf(t), use_t[t] & 1, cta_abort);
+                    if (!ok) continue;
+                    tc_fence_after();
+                    issue_pv(cur, s, t, 0, min(8, nks));
+                }
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
                     if (!ok) break;
@@ -393,7 +416,8 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
                         ok = mbar_wait(bar_pready(t), use_t[t] & 1, cta_abort);   // use_t[t] still counts earlier uses only
                         if (!ok) break;
                         tc_fence_after();
-                        issue_pv(cur, s, t);
+                        issue_pv(cur, s, t, 8, nks);
+                        mma_commit(bar_oready(t));
                         if (t == cur.ntiles - 1) mma_commit(bar_empty(s));   // all operands of this stage consumed
                     }
                     if (has_next && t < nx.ntiles) {
@@ -445,31 +469,22 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
             if (!__all_sync(0xffffffffu, mbar_wait(bar_sready(wg), use & 1, cta_abort))) break;
             tc_fence_after();
             float m, sum;
-            if (x.masked) m = softmax_row<true>(t_s, x.npad, bias_i, st_a + kOffKc, st_a + kOffKlab, label_i, scale, bmax, sum);
-            else m = softmax_row<false>(t_s, x.npad, bias_i, st_a + kOffKc, st_a + kOffKlab, label_i, scale, bmax, sum);
+            if (x.masked) m = softmax_row<true>(t_s, x.npad, bias_i, st_a + kOffKc, st_a + kOffKlab, label_i, scale, bmax, sum, bar_phalf(wg));
+            else m = softmax_row<false>(t_s, x.npad, bias_i, st_a + kOffKc, st_a + kOffKlab, label_i, scale, bmax, sum, bar_phalf(wg));
             tmem_st_wait();
             tc_fence_before();
+            if (x.npad <= 128) mbar_arrive(bar_phalf(wg));      // short rows: both halves at once
             mbar_arrive(bar_pready(wg));
 
             const size_t row_off = ((size_t)x.b * HW + (size_t)(tok < 0 ? 0 : tok)) * g.heads + x.head;
             if (tok >= 0) lse[row_off] = (m + log2f(sum)) * kLn2;
             const float inv = 1.f / sum;
-            const int nacc = min(kOAcc, x.npad >> 4);
 
             if (!__all_sync(0xffffffffu, mbar_wait(bar_oready(wg), use & 1, cta_abort))) break;
             tc_fence_after();
             uint32_t ro[32];
             tmem_ld32(t_s + kColO, ro);
             tmem_ld_wait();
-#pragma unroll
-            for (int a = 1; a < kOAcc; ++a) {
-                if (a >= nacc) break;
-                uint32_t rx[32];
-                tmem_ld32(t_s + kColO + 32 * a, rx);
-                tmem_ld_wait();
-#pragma unroll
-                for (int e = 0; e < 32; ++e) ro[e] = __float_as_uint(__uint_as_float(ro[e]) + __uint_as_float(rx[e]));
-            }
             tc_fence_before();
             mbar_arrive(bar_sfree(wg));
             ++use;
