@@ -134,6 +134,7 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
     unsigned char* s_c1 = s_r2 + TILE_BYTES;          // two stages
     unsigned char* s_c2 = s_c1 + 2 * TILE_BYTES;      // two stages
     float* s_acc = reinterpret_cast<float*>(s_c2 + 2 * TILE_BYTES);   // 64 x acc_stride image of summed dS (query tiles only)
+    float* s_stage = s_acc + BM * acc_stride;                         // 4 warps x 16 x (BN + 1) staging tile (query tiles only)
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int gq = lane >> 2, tq = lane & 3;
@@ -278,15 +279,25 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
                         cell0[nt * 4 + 4 * acc_stride] = cur[nt][1];
                     }
                 } else {
+                    // The warp's 16 x 64 dS tile goes through a staging tile so that one atomic instruction
+                    // covers 32 consecutive columns of one row: 32 different table entries, no retries inside
+                    // the warp (in the MMA fragment layout a warp instruction hits only 14 distinct entries).
+                    float* stage = s_stage + warp * 16 * (BN + 1);
 #pragma unroll
                     for (int nt = 0; nt < BN / 8; ++nt) {
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const int mc = s_meta[blk * BN + nt * 8 + 2 * tq + (e & 1)];
-                            const int mr = meta_r[e >> 1];
-                            if (acc_dp[nt][e] != 0.f) atomicAdd(&s_dbias[meta_code(mr) - meta_code(mc) + c0], acc_dp[nt][e]);
-                        }
+                        for (int e = 0; e < 4; ++e)
+                            stage[(gq + 8 * (e >> 1)) * (BN + 1) + nt * 8 + 2 * tq + (e & 1)] = acc_dp[nt][e];
                     }
+                    __syncwarp();
+                    const int code_c0 = meta_code(s_meta[blk * BN + lane]), code_c1 = meta_code(s_meta[blk * BN + lane + 32]);
+                    for (int rr = 0; rr < 16; ++rr) {
+                        const int code_r = meta_code(s_meta[r0 + warp * 16 + rr]) + c0;
+                        const float v0 = stage[rr * (BN + 1) + lane], v1 = stage[rr * (BN + 1) + lane + 32];
+                        if (v0 != 0.f) atomicAdd(&s_dbias[code_r - code_c0], v0);
+                        if (v1 != 0.f) atomicAdd(&s_dbias[code_r - code_c1], v1);
+                    }
+                    __syncwarp();
                 }
             }
             if constexpr (KV) {
@@ -368,7 +379,7 @@ size_t bwd_smem_bytes(const Geo& g, bool query_side) {
     int npad_max = ((g.nmax + BN - 1) / BN) * BN;
     int nbias = (2 * g.w - 1) * (2 * g.w - 1);
     size_t head = (((size_t)npad_max * 16 + (size_t)nbias * 8 + 127) / 128) * 128;
-    size_t acc = query_side ? (size_t)BM * acc_stride_for(g) * sizeof(float) : 0;
+    size_t acc = query_side ? ((size_t)BM * acc_stride_for(g) + (size_t)BM * (BN + 1)) * sizeof(float) : 0;
     return head + 6 * (size_t)BN * g.d * 2 + acc;
 }
 
