@@ -57,7 +57,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
             return
@@ -178,9 +178,9 @@ def run_reference(args, cfg):
 # captures summarised under profiles/ (config 3 cut to 254 token rows, 13 056 items); traffic grows in
 # proportion to the item count, so a full launch is this figure times its items.  None = not captured.
 NCU_DRAM_BYTES_PER_ITEM = {
-    "swin_fwd_tc_kernel": 63833,
-    "swin_bwd_tc_kernel<key side>": 96401,
-    "swin_bwd_tc_kernel<query side>": 81609,
+    "swin_fwd_tc_kernel": 63629,
+    "swin_bwd_tc_kernel<key side>": 96647,
+    "swin_bwd_tc_kernel<query side>": 81558,
 }
 
 
@@ -202,7 +202,7 @@ def workload_config(cfg, l2_note):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", default="cfg3")
     ap.add_argument("--impl", default="terra", choices=["terra", "reference"])

@@ -146,6 +146,14 @@ int terra_swin_attn_fwd_noalloc(const terra_swin_desc* desc, const void* q, cons
 int terra_swin_check(void* stream);
 
 /*
+ * Self-test of the failure report above (the paper has no counterpart): launches one small CTA that waits on
+ * a barrier nobody arrives on, with a limit of `limit_cycles` SM clocks (1 .. 2e9).  The wait expires, the
+ * kernel ends normally, and the next terra_swin_check returns TERRA_ERR_DEVICE_TIMEOUT.  Nothing hangs or
+ * faults; the context stays usable.
+ */
+int terra_selftest_bounded_wait(long long limit_cycles, void* stream);
+
+/*
  * Per-kernel timing for benchmarks (the paper has no counterpart).  While enabled, the library brackets each
  * of its main kernel launches with CUDA events on the launching stream.  terra_profile_enable(1) clears the
  * record and starts, (0) clears and stops; terra_profile_count gives the number of recorded launches;

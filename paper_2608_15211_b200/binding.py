@@ -17,7 +17,7 @@ from .build import LIB_PATH
 TERRA_OK = 0
 EXPORTS = ("terra_route_sizes", "terra_window_route", "terra_swin_workspace_bytes", "terra_swin_attn_fwd",
            "terra_swin_attn_fwd_noalloc", "terra_swin_attn_bwd", "terra_swin_check", "terra_strerror", "terra_last_cuda_error",
-           "terra_launch_count", "terra_profile_enable", "terra_profile_count", "terra_profile_get")
+           "terra_launch_count", "terra_selftest_bounded_wait", "terra_profile_enable", "terra_profile_count", "terra_profile_get")
 
 
 class TerraError(RuntimeError):
@@ -62,6 +62,8 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
     lib.terra_strerror.restype = ctypes.c_char_p
     lib.terra_last_cuda_error.restype = ctypes.c_char_p
     lib.terra_launch_count.restype = ctypes.c_int64
+    lib.terra_selftest_bounded_wait.argtypes = [ctypes.c_longlong, vp]
+    lib.terra_selftest_bounded_wait.restype = ctypes.c_int
     lib.terra_profile_enable.argtypes = [ctypes.c_int]
     lib.terra_profile_count.restype = ctypes.c_int
     lib.terra_profile_get.argtypes = [ctypes.c_int, ctypes.c_char_p, ctypes.c_int, ctypes.POINTER(ctypes.c_float)]
@@ -117,6 +119,11 @@ def profile_read() -> list:
         if lib.terra_profile_get(i, name, 64, ctypes.byref(ms)) == TERRA_OK:
             out.append((name.value.decode(), float(ms.value)))
     return out
+
+
+def selftest_bounded_wait(limit_cycles: int = 1_000_000) -> None:
+    """Launches the kernel whose bounded wait must expire (see include/terra.h); check with terra_swin_check()."""
+    _check(load_library().terra_selftest_bounded_wait(int(limit_cycles), _stream()))
 
 
 def launch_count() -> int:

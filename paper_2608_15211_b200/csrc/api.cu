@@ -211,6 +211,15 @@ int terra_swin_attn_bwd(const terra_swin_desc* desc, const void* q, const void* 
     return e == cudaSuccess ? TERRA_OK : cuda_fail(e, "terra_swin_attn_bwd");
 }
 
+int terra_selftest_bounded_wait(long long limit_cycles, void* stream) {
+    if (limit_cycles <= 0 || limit_cycles > 2000000000LL) return TERRA_ERR_INVALID_ARG;
+    int sms = 0;
+    int rc = device_props(&sms);
+    if (rc) return rc;
+    cudaError_t e = launch_bounded_wait_selftest(limit_cycles, (cudaStream_t)stream);
+    return e == cudaSuccess ? TERRA_OK : cuda_fail(e, "terra_selftest_bounded_wait");
+}
+
 int terra_swin_check(void* stream) {
     int timed_out = 0;
     cudaError_t e = read_tc_status(&timed_out, (cudaStream_t)stream);

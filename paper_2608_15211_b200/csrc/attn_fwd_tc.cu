@@ -571,6 +571,28 @@ cudaError_t launch_fwd_tc(const Geo& g, const void* q, const void* k, const void
     return cudaGetLastError();
 }
 
+// Self-test of the failure report: one CTA waits, with a short cycle limit, on a barrier that nothing ever
+// arrives on; the wait gives up, the kernel raises the device status word and returns normally.
+__global__ void bounded_wait_selftest_kernel(long long limit_cycles) {
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        tc::mbar_init(smem_u32(&bar), 1);
+        abort_flag = 0;
+        tc::fence_barrier_init();
+    }
+    __syncthreads();
+    const bool ok = tc::mbar_wait(smem_u32(&bar), 0, &abort_flag, limit_cycles);
+    __syncthreads();
+    if (threadIdx.x == 0 && (!ok || abort_flag)) atomicExch(&g_tc_timeout, 1);
+}
+
+cudaError_t launch_bounded_wait_selftest(long long limit_cycles, cudaStream_t stream) {
+    bounded_wait_selftest_kernel<<<1, 32, 0, stream>>>(limit_cycles);
+    count_launch(stream);
+    return cudaGetLastError();
+}
+
 // prepared bias tables for every head (also used by the backward kernels)
 cudaError_t launch_bias_prep(const Geo& g, const float* bias, float* prep, cudaStream_t stream) {
     swin_fwd_bias_prep_kernel<<<g.heads, 256, 0, stream>>>(bias, prep, g.w, g.heads);

@@ -28,6 +28,7 @@ cudaError_t launch_fwd_tc(const Geo& g, const void* q, const void* k, const void
 // synchronises the stream, reads and clears the device-side "a bounded wait expired" word
 cudaError_t read_tc_status(int* timed_out, cudaStream_t stream);
 
+cudaError_t launch_bounded_wait_selftest(long long limit_cycles, cudaStream_t stream);
 cudaError_t launch_bias_prep(const Geo& g, const float* bias, float* prep, cudaStream_t stream);
 
 // tcgen05 backward path (head dim 32, window side <= 16)

@@ -192,3 +192,18 @@ def test_alignment_and_workspace_errors():
                                   workspace=torch.empty(16, dtype=torch.uint8, device="cuda"))
     assert e.value.status == 4
     torch.cuda.synchronize()
+
+
+def test_expired_bounded_wait_is_reported_and_the_context_stays_usable():
+    """A kernel wait that nothing satisfies gives up after its cycle limit and the host sees it; afterwards the
+    library works as before (no hang, no fault)."""
+    terra.terra_swin_check()                       # clean slate
+    terra.selftest_bounded_wait(2_000_000)         # about a millisecond of SM clocks
+    with pytest.raises(terra.TerraError) as e:
+        terra.terra_swin_check()
+    assert e.value.status == 6
+    terra.terra_swin_check()                       # the word was cleared by the failed check
+    cfg = small_config("after", 1, 16, 16, 2, 32, 8, 4, 4)
+    x = make_inputs(cfg)
+    d, o, lse = _run_fwd(cfg, _to_gpu(x))
+    _check_forward(cfg, x, o, lse, None)
