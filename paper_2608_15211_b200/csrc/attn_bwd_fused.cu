@@ -1,0 +1,781 @@
+// Backward shifted-window attention on the tcgen05 tensor cores, one pass (head dim 32, windows of <= 256
+// tokens): P and dS of a (window, head) item are computed once and feed all three gradients.
+//
+// Orientation: TMEM lanes (rows) = keys of a 128-key tile, columns = queries, 64 query columns per block.
+//   S^T  = K Q^T, dP^T = V dO^T                      (SS MMAs, N = the block's columns)
+//   P^T  = exp2(S^T scale + bias - lse_q), dS^T = P^T (dP^T - delta_q)       (elementwise warps, one key row per thread)
+//   dV  += P^T dO, dK += dS^T Q                      (A = bf16 P^T / dS^T read from TMEM, per block)
+//   dQ  += dS K                                      (A = dS^T from shared memory, read transposed (MN-major),
+//                                                     per pair of blocks = 128 queries)
+//   dBias: every elementwise warp adds its dS into a private shared-memory table (plain load-add-store: the
+//          32 lanes of one instruction are 32 different keys at one query = 32 different entries).
+// The eight elementwise warps work on ONE key tile at a time: warps w and w + 4 share the 32 key rows of TMEM
+// lane quarter w & 3 and split each block's four 16-column steps (steps 0, 2 and steps 1, 3).
+// TMEM columns: two [S 64 | dP 64] buffers (the MMAs run two blocks ahead), two (dV, dK) accumulator sets
+// (so a tile's read-out overlaps the next tile), two dQ accumulators (queries 0..127 and 128..255).
+// Outputs leave through the item's own operand tiles in shared memory (dK over the K rows, dV over V, dQ
+// over Q, once the MMAs that read them are complete), so that whole 64-byte rows are stored.
+// CTAs are bound to one head (grid = heads x CTAs per head): the head's bias table is staged once per CTA
+// and the bias-gradient tables belong to one head; they are summed in a fixed order (reproducible dBias).
+// Every mbarrier wait is bounded; on expiry the CTA raises an abort flag and all roles leave their loops.
+#include "swin_common.cuh"
+#include "swin_kernels.h"
+#include "tc_common.cuh"
+
+namespace terra {
+
+__device__ int g_bwd_tc_timeout = 0;   // set when a bounded wait expired in any CTA of the kernel below
+
+namespace {
+
+using namespace tc;
+
+constexpr int kMmaWarp = 8;         // warp 8: one MMA-issuing lane
+constexpr int kLoaderWarp0 = 9;
+constexpr int kLoaderWarps = 3;
+constexpr int kLoaderThreads = kLoaderWarps * 32;
+constexpr int kThreads = (kLoaderWarp0 + kLoaderWarps) * 32;   // 384 = three warpgroups
+constexpr int kWorkWarps = 8;              // elementwise warps; each arrives once per barrier phase
+constexpr int kRegsLaunch = 168;
+constexpr int kRegsWork = 216;      // elementwise warpgroups after setmaxnreg.inc
+constexpr int kRegsOther = 72;      // MMA + loader warpgroup after setmaxnreg.dec
+static_assert(2 * (kRegsWork - kRegsLaunch) <= (kRegsLaunch - kRegsOther), "register hand-over does not balance");
+
+constexpr int kStages = 2;
+constexpr int kMaxSlots = 256;
+constexpr int kD = 32;
+constexpr int kRowBytes = kD * 2;
+constexpr int kTileBytes = kMaxSlots * kRowBytes;              // 16384
+constexpr int CB = 64;                                         // query columns per block
+
+// stage layout (bytes)
+constexpr int kOffQ = 0;
+constexpr int kOffK = kTileBytes;
+constexpr int kOffV = 2 * kTileBytes;
+constexpr int kOffDO = 3 * kTileBytes;
+constexpr int kOffColOff = 4 * kTileBytes;                     // per slot: 4 * bias code, code = a * (w + 32) + b (0 if no token)
+constexpr int kOffLab = kOffColOff + kMaxSlots * 4;            // per slot: shift-mask label (0xff: no token)
+constexpr int kOffTok = kOffLab + kMaxSlots * 4;               // per slot: grid token, -1 if none
+constexpr int kOffLse = kOffTok + kMaxSlots * 4;               // per slot: lse * log2(e), +inf if none
+constexpr int kOffDelta = kOffLse + kMaxSlots * 4;             // per slot: delta
+constexpr int kStageBytes = kOffDelta + kMaxSlots * 4;         // 70656
+static_assert(kStageBytes % 1024 == 0, "stages keep the swizzle alignment");
+// after the stages
+constexpr int kOffBias = kStages * kStageBytes;                // the head's prepared bias table (kFwdBiasFloats floats)
+constexpr int kDBiasEntries = 1472;                            // >= 2 c0 + 1 for w <= 16
+constexpr int kDBiasFloats = kDBiasEntries + 32;               // + one scratch float per lane (where pairs without a token add their 0)
+constexpr int kOffDBias = kOffBias + kFwdBiasFloats * 4;       // one bias-gradient table per elementwise warp
+constexpr int kOffDS = kOffDBias + 8 * kDBiasFloats * 4;       // dS^T of one pair of blocks: [128 keys][128 queries] bf16
+static_assert(kOffDS % 1024 == 0, "the dS tile keeps the swizzle alignment");
+constexpr int kDSGroupBytes = 128 * kRowBytes;                 // 32 queries x 128 keys
+constexpr int kOffBars = kOffDS + 4 * kDSGroupBytes;
+constexpr int kSmemBytes = kOffBars + 256;
+static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
+
+// TMEM columns
+constexpr int kColBuf = 128;        // buffer b at b * 128: S at +0, dP at +64
+constexpr int kColDV = 256;         // accumulator set s: dV at 256 + 64 s, dK at 288 + 64 s
+constexpr int kColDK = 288;
+constexpr int kColDQ = 384;         // dQ of query pair p at 384 + 32 p
+
+__device__ __forceinline__ int code_stride(int w) { return w + 32; }
+
+struct Item {
+    int b, win;
+    WindowRef r;
+    int npad;      // slots rounded up to 16
+    int ntiles;    // 128-key tiles in use
+    int nblk;      // 64-query blocks in use
+    bool masked;   // the window mixes shift-mask labels
+    bool ragged;   // some row of a key tile, or some column below npad, has no token
+};
+
+__device__ __forceinline__ Item make_item(const Geo& g, long long it) {
+    Item x;
+    const int M = g.Mh * g.Mw;
+    x.win = (int)(it % M);
+    x.b = (int)(it / M);
+    x.r = window_ref(g, x.win);
+    x.npad = (x.r.n + 15) & ~15;
+    x.ntiles = (x.r.n + 127) >> 7;
+    x.nblk = (x.npad + CB - 1) / CB;
+    const int r0 = x.r.wr * g.w, c0 = x.r.wc * g.w;
+    const bool mh = !g.ph && g.sh > 0 && r0 < g.H - g.sh && r0 + x.r.eh > g.H - g.sh;
+    const bool mw = !g.pw && g.sw > 0 && c0 < g.W - g.sw && c0 + x.r.ew > g.W - g.sw;
+    x.masked = mh || mw;
+    x.ragged = x.npad != x.r.n || x.r.n != x.ntiles * 128;
+    return x;
+}
+
+__device__ __forceinline__ int slot_token_tc(const Geo& g, const WindowRef& r, int slot, int& code, int& label) {
+    const int a = slot / r.ew;
+    const int b = slot - a * r.ew;
+    int u = r.wr * g.w + a + g.sh;
+    if (u >= g.H) u -= g.H;
+    int v = r.wc * g.w + b + g.sw;
+    if (v >= g.W) v -= g.W;
+    label = ((!g.ph && u < g.sh) ? 2 : 0) + ((!g.pw && v < g.sw) ? 1 : 0);
+    code = a * code_stride(g.w) + b;
+    return u * g.W + v;
+}
+
+__device__ __forceinline__ float lds_f32(uint32_t addr) {
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ int4 lds_i4(uint32_t addr) {
+    int4 v;
+    asm volatile("ld.shared.v4.s32 {%0,%1,%2,%3}, [%4];\n" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ float4 lds_f4(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];\n" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ int lds_i32(uint32_t addr) {
+    int v;
+    asm volatile("ld.shared.s32 %0, [%1];\n" : "=r"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void sts_u4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};\n" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+// table[addr] += v in the warp's own table.  Not atomic: within one warp instruction the 32 lanes (32
+// different keys, same query) touch 32 different entries, and successive instructions of a warp reach
+// shared memory in program order, so nothing is lost.
+__device__ __forceinline__ void rmw_shared_f32(uint32_t addr, float v) {
+    asm volatile(
+        "{\n\t.reg .f32 t;\n\t"
+        "ld.shared.f32 t, [%0];\n\t"
+        "add.f32 t, t, %1;\n\t"
+        "st.shared.f32 [%0], t;\n\t}\n" ::"r"(addr), "f"(v) : "memory");
+}
+// G table updates of one lane, issued together so that their load-add-store latencies overlap.  Allowed only
+// where no two of the warp's 32 x G updates can meet in one entry (see the key-row order in the kernel).
+__device__ __forceinline__ void rmw4_shared_f32(const uint32_t* a, const float* v) {
+    asm volatile(
+        "{\n\t.reg .f32 t0, t1, t2, t3;\n\t"
+        "ld.shared.f32 t0, [%0];\n\tld.shared.f32 t1, [%1];\n\tld.shared.f32 t2, [%2];\n\tld.shared.f32 t3, [%3];\n\t"
+        "add.f32 t0, t0, %4;\n\tadd.f32 t1, t1, %5;\n\tadd.f32 t2, t2, %6;\n\tadd.f32 t3, t3, %7;\n\t"
+        "st.shared.f32 [%0], t0;\n\tst.shared.f32 [%1], t1;\n\tst.shared.f32 [%2], t2;\n\tst.shared.f32 [%3], t3;\n\t}\n"
+        ::"r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]) : "memory");
+}
+__device__ __forceinline__ void rmw8_shared_f32(const uint32_t* a, const float* v) {
+    asm volatile(
+        "{\n\t.reg .f32 t0, t1, t2, t3, t4, t5, t6, t7;\n\t"
+        "ld.shared.f32 t0, [%0];\n\tld.shared.f32 t1, [%1];\n\tld.shared.f32 t2, [%2];\n\tld.shared.f32 t3, [%3];\n\t"
+        "ld.shared.f32 t4, [%4];\n\tld.shared.f32 t5, [%5];\n\tld.shared.f32 t6, [%6];\n\tld.shared.f32 t7, [%7];\n\t"
+        "add.f32 t0, t0, %8;\n\tadd.f32 t1, t1, %9;\n\tadd.f32 t2, t2, %10;\n\tadd.f32 t3, t3, %11;\n\t"
+        "add.f32 t4, t4, %12;\n\tadd.f32 t5, t5, %13;\n\tadd.f32 t6, t6, %14;\n\tadd.f32 t7, t7, %15;\n\t"
+        "st.shared.f32 [%0], t0;\n\tst.shared.f32 [%1], t1;\n\tst.shared.f32 [%2], t2;\n\tst.shared.f32 [%3], t3;\n\t"
+        "st.shared.f32 [%4], t4;\n\tst.shared.f32 [%5], t5;\n\tst.shared.f32 [%6], t6;\n\tst.shared.f32 [%7], t7;\n\t}\n"
+        ::"r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(a[4]), "r"(a[5]), "r"(a[6]), "r"(a[7]),
+          "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]) : "memory");
+}
+// mode 8 / 4: groups of 8 / 4 consecutive columns at once; else one column at a time
+__device__ __forceinline__ void dbias_add16(int mode, const uint32_t (&addr)[16], const float (&ds)[16]) {
+    if (mode == 8) {
+        rmw8_shared_f32(&addr[0], &ds[0]);
+        rmw8_shared_f32(&addr[8], &ds[8]);
+    } else if (mode == 4) {
+#pragma unroll
+        for (int e = 0; e < 16; e += 4) rmw4_shared_f32(&addr[e], &ds[e]);
+    } else {
+#pragma unroll
+        for (int e = 0; e < 16; ++e) rmw_shared_f32(addr[e], ds[e]);
+    }
+}
+
+// What one elementwise thread knows about its key row.
+struct RowCtx {
+    uint32_t bias_row;   // shared address: bias table + the row's part of the index (the -inf zone if the row has no token)
+    uint32_t dbias_row;  // shared address: this warp's bias-gradient table + the row's part of the index
+    uint32_t scratch;    // shared address: this lane's scratch float behind the table
+    int label;
+    bool valid;
+};
+
+// 16 query columns [c, c + 16) of one key row: P = exp2(S scale + bias - lse), dS = P (dP - delta), both
+// packed to bf16; dS also in fp32 with the shared address of its bias-gradient entry (the lane's scratch
+// float for a pair without a token, whose dS is 0).
+template <bool MASKED, bool RAGGED>
+__device__ __forceinline__ void cols16(const uint32_t (&rs)[16], const uint32_t (&rp)[16], int c, const RowCtx& rc, uint32_t st_a,
+                                       float scale, uint32_t (&pk_p)[8], uint32_t (&pk_ds)[8], float (&ds)[16], uint32_t (&addr)[16]) {
+    int co[16], kl[16];
+    float l2[16], dl[16], bv[16];
+#pragma unroll
+    for (int e4 = 0; e4 < 4; ++e4) {
+        const int4 co4 = lds_i4(st_a + kOffColOff + 4 * (c + e4 * 4));
+        co[e4 * 4] = co4.x; co[e4 * 4 + 1] = co4.y; co[e4 * 4 + 2] = co4.z; co[e4 * 4 + 3] = co4.w;
+    }
+#pragma unroll
+    for (int e = 0; e < 16; ++e) bv[e] = lds_f32(rc.bias_row + co[e]);
+    if (MASKED) {
+#pragma unroll
+        for (int e4 = 0; e4 < 4; ++e4) {
+            const int4 kl4 = lds_i4(st_a + kOffLab + 4 * (c + e4 * 4));
+            kl[e4 * 4] = kl4.x; kl[e4 * 4 + 1] = kl4.y; kl[e4 * 4 + 2] = kl4.z; kl[e4 * 4 + 3] = kl4.w;
+        }
+    }
+#pragma unroll
+    for (int e4 = 0; e4 < 4; ++e4) {
+        const float4 a = lds_f4(st_a + kOffLse + 4 * (c + e4 * 4));
+        const float4 b = lds_f4(st_a + kOffDelta + 4 * (c + e4 * 4));
+        l2[e4 * 4] = a.x; l2[e4 * 4 + 1] = a.y; l2[e4 * 4 + 2] = a.z; l2[e4 * 4 + 3] = a.w;
+        dl[e4 * 4] = b.x; dl[e4 * 4 + 1] = b.y; dl[e4 * 4 + 2] = b.z; dl[e4 * 4 + 3] = b.w;
+    }
+    float p[16];
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
+        float xv = fmaf(__uint_as_float(rs[e]), scale, bv[e]) - l2[e];
+        if (MASKED && kl[e] != rc.label) xv = -INFINITY;
+        p[e] = fast_exp2(xv);
+        ds[e] = p[e] * (__uint_as_float(rp[e]) - dl[e]);
+        addr[e] = rc.dbias_row + co[e];
+        if (RAGGED && (!rc.valid || l2[e] == INFINITY)) addr[e] = rc.scratch;
+    }
+#pragma unroll
+    for (int e2 = 0; e2 < 8; ++e2) {
+        pk_p[e2] = pack_bf16(p[2 * e2], p[2 * e2 + 1]);
+        pk_ds[e2] = pack_bf16(ds[2 * e2], ds[2 * e2 + 1]);
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
+                      const __nv_bfloat16* __restrict__ v, const __nv_bfloat16* __restrict__ d_o,
+                      const float* __restrict__ bias_prep, const float* __restrict__ lse, const float* __restrict__ delta,
+                      __nv_bfloat16* __restrict__ dq, __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv,
+                      float* __restrict__ dbias_parts, long long n_items, int ctas_per_head) {
+    extern __shared__ __align__(1024) unsigned char smem[];
+    const uint32_t smem0 = smem_u32(smem);
+    const uint32_t bar0 = smem0 + kOffBars;
+    auto bar_full = [&](int s) { return bar0 + 8u * s; };           // stage s holds an item's operands
+    auto bar_empty = [&](int s) { return bar0 + 8u * (2 + s); };    // stage s may be overwritten
+    auto bar_sdp = [&](int b) { return bar0 + 8u * (4 + b); };      // S and dP of a block are in buffer b
+    auto bar_ds = [&](int b) { return bar0 + 8u * (6 + b); };       // bf16 P / dS of a block are in buffer b (and dS in shared memory)
+    auto bar_acc = [&](int s) { return bar0 + 8u * (8 + s); };      // dV / dK of a key tile are final in accumulator set s
+    auto bar_accfree = [&](int s) { return bar0 + 8u * (10 + s); }; // ... and have been read back
+    const uint32_t bar_dsfree = bar0 + 8u * 12;                      // the dQ MMAs of a block pair have read the shared dS tile
+    const uint32_t bar_dq = bar0 + 8u * 13;                          // every MMA of the item is complete (dQ final)
+    const uint32_t bar_dqfree = bar0 + 8u * 14;                      // dQ has been read back
+    unsigned char* tail = smem + kOffBars + 8 * 16;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail);
+    volatile int* cta_abort = reinterpret_cast<volatile int*>(tail + 8);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int head = blockIdx.x % g.heads;
+    const int cta_in_head = blockIdx.x / g.heads;
+
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(bar_full(s), kLoaderThreads);
+            mbar_init(bar_empty(s), kWorkWarps);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bar_sdp(b), 1);
+            mbar_init(bar_ds(b), kWorkWarps);
+            mbar_init(bar_acc(b), 1);
+            mbar_init(bar_accfree(b), kWorkWarps);
+        }
+        mbar_init(bar_dsfree, 1);
+        mbar_init(bar_dq, 1);
+        mbar_init(bar_dqfree, kWorkWarps);
+        *cta_abort = 0;
+        fence_barrier_init();
+    }
+    // the head's prepared bias table, and zeroed bias-gradient tables
+    for (int i = tid; i < kFwdBiasFloats; i += kThreads)
+        reinterpret_cast<float*>(smem + kOffBias)[i] = bias_prep[(size_t)head * kFwdBiasFloats + i];
+    for (int i = tid; i < 8 * kDBiasFloats; i += kThreads) reinterpret_cast<float*>(smem + kOffDBias)[i] = 0.f;
+    // the shared dS tile starts finite: columns that no block writes only reach dQ rows that are never stored
+    for (int i = tid; i < 4 * kDSGroupBytes / 4; i += kThreads) reinterpret_cast<uint32_t*>(smem + kOffDS)[i] = 0u;
+    fence_proxy_async();
+    if (warp == kMmaWarp) {
+        tmem_alloc(smem_u32(tmem_slot), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int cs = code_stride(g.w);
+    const int c0 = (g.w - 1) * (cs + 1);
+    const size_t HW = (size_t)g.H * g.W;
+
+    if (warp >= kMmaWarp) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kRegsOther));
+    if (warp >= kLoaderWarp0) {
+        // ------------------------------------------------------------------ loaders
+        const int lt = tid - kLoaderWarp0 * 32;
+        int kuse = 0, pending_s = -1;
+        for (long long it = cta_in_head; it < n_items; it += ctas_per_head, ++kuse) {
+            const int s = kuse % kStages;
+            // if the next stage is not free yet, publish the copies already issued instead of holding them back
+            if (pending_s >= 0 && !__all_sync(0xffffffffu, mbar_test_wait(bar_empty(s), ((kuse / kStages) & 1) ^ 1))) {
+                cp_async_wait<0>();
+                fence_proxy_async();
+                mbar_arrive(bar_full(pending_s));
+                pending_s = -1;
+            }
+            if (!mbar_wait_warp(bar_empty(s), ((kuse / kStages) & 1) ^ 1, cta_abort)) break;
+            const Item x = make_item(g, it);
+            unsigned char* st = smem + s * kStageBytes;
+            const uint32_t st_a = smem0 + s * kStageBytes;
+            const size_t sample_off = (size_t)x.b * HW;
+            // slot metadata; the lse / delta gathers stay in flight while the row copies are issued below
+            constexpr int kSlotIters = (kMaxSlots + kLoaderThreads - 1) / kLoaderThreads;
+            float l2v[kSlotIters], dlv[kSlotIters];
+#pragma unroll
+            for (int i = 0; i < kSlotIters; ++i) {
+                const int slot = lt + i * kLoaderThreads;
+                l2v[i] = INFINITY;                       // no token: P = exp2(.. - inf) = 0
+                dlv[i] = 0.f;
+                if (slot >= kMaxSlots) continue;
+                int code = 0, label = 0xff, tok = -1;
+                if (slot < x.r.n) {
+                    tok = slot_token_tc(g, x.r, slot, code, label);
+                    const size_t li = (sample_off + (size_t)tok) * g.heads + head;
+                    l2v[i] = __ldg(lse + li);
+                    dlv[i] = __ldg(delta + li);
+                }
+                reinterpret_cast<int*>(st + kOffColOff)[slot] = 4 * code;
+                reinterpret_cast<int*>(st + kOffLab)[slot] = label;
+                reinterpret_cast<int*>(st + kOffTok)[slot] = tok;
+            }
+            // K and V rows of every key tile in use (rows without a token as zeros: they are MMA operands and
+            // must stay finite); Q and dO rows up to the padded column count
+            // Key rows are interleaved: with M = 4 * (tiles in use) 32-slot groups, lane l of elementwise warp
+            // W = 4 t + qd (key row 128 t + 32 qd + l) holds slot 32 ((W + l) mod M) + l (see the bias-gradient updates).
+            const int chunk = lt & 3;
+            const int nrows = x.ntiles * 128;
+            const int M = 4 * x.ntiles;
+            for (int row = lt >> 2; row < nrows; row += kLoaderThreads / 4) {
+                const int kl = row & 31, kw = ((row >> 5) - kl) & (M - 1), krow = 128 * (kw >> 2) + 32 * (kw & 3) + kl;
+                const __nv_bfloat16 *sq = q, *sk = k, *sv = v, *sg = d_o;
+                int bytes = 0;
+                if (row < x.r.n) {
+                    int code, label;
+                    const int tok = slot_token_tc(g, x.r, row, code, label);
+                    const size_t off = ((sample_off + (size_t)tok) * g.heads + head) * kD + chunk * 8;
+                    sq = q + off; sk = k + off; sv = v + off; sg = d_o + off;
+                    bytes = 16;
+                }
+                const uint32_t so = st_a + tile_off<kD>(row, chunk), sok = st_a + tile_off<kD>(krow, chunk);
+                cp_async16(sok + kOffK, sk, bytes);
+                cp_async16(sok + kOffV, sv, bytes);
+                if (row < x.npad) {
+                    cp_async16(so + kOffQ, sq, bytes);
+                    cp_async16(so + kOffDO, sg, bytes);
+                }
+            }
+            cp_async_commit();
+#pragma unroll
+            for (int i = 0; i < kSlotIters; ++i) {
+                const int slot = lt + i * kLoaderThreads;
+                if (slot < kMaxSlots) {
+                    reinterpret_cast<float*>(st + kOffLse)[slot] = l2v[i] * kLog2e;
+                    reinterpret_cast<float*>(st + kOffDelta)[slot] = dlv[i];
+                }
+            }
+            if (pending_s >= 0) {
+                cp_async_wait<1>();
+                fence_proxy_async();
+                mbar_arrive(bar_full(pending_s));
+            }
+            pending_s = s;
+        }
+        if (pending_s >= 0) {
+            cp_async_wait<0>();
+            fence_proxy_async();
+            mbar_arrive(bar_full(pending_s));
+        }
+    } else {
+        // ------------------------------------------------------------------ MMA issuer (warp 8)
+        // The whole warp runs the loop (warp-uniform control flow and operands); one elected lane issues.
+        {
+            const uint32_t idesc_acc = make_idesc_bf16(128, kD, 0, 1);   // A from TMEM, B = 16 rows x 32 (MN-major)
+            const uint32_t idesc_dq = make_idesc_bf16(128, kD, 1, 1);    // A = dS^T tile read transposed, B = 16 K rows x 32
+            // shared-memory descriptors: one common high word, low words = start address (16-byte units)
+            const uint32_t d_hi = sdesc_hi(make_sdesc_sw64(smem0, 512));
+            const uint32_t d_q = sdesc_lo(make_sdesc_sw64(smem0 + kOffQ, 512)), d_k = sdesc_lo(make_sdesc_sw64(smem0 + kOffK, 512));
+            const uint32_t d_v = sdesc_lo(make_sdesc_sw64(smem0 + kOffV, 512)), d_do = sdesc_lo(make_sdesc_sw64(smem0 + kOffDO, 512));
+            const uint32_t d_ds = sdesc_lo(make_sdesc_sw64_mn(smem0 + kOffDS, kDSGroupBytes, 512));
+            bool ok = true;
+            int kuse = 0, n_tile = 0;
+            uint32_t ph_ds = 0;          // bit b: parity of the next completion of bar_ds(b)
+            for (long long it = cta_in_head; ok && it < n_items; it += ctas_per_head, ++kuse) {
+                const int s = kuse % kStages;
+                int npad, ntiles, nblk;
+                {
+                    const Item x = make_item(g, it);
+                    npad = x.npad; ntiles = x.ntiles; nblk = x.nblk;
+                }
+                const int nb_total = ntiles * nblk;
+                const uint32_t so = (uint32_t)((s * kStageBytes) >> 4);
+                ok = mbar_wait_warp(bar_full(s), (kuse / kStages) & 1, cta_abort);
+                if (!ok) break;
+                fence_proxy_async();
+                tc_fence_after();
+                // S^T = K Q^T and dP^T = V dO^T of query block b of key tile t into buffer `buf`
+                auto issue_sdp = [&](int t, int b, int buf) {
+                    const int ncols = min(CB, npad - b * CB);
+                    const uint32_t ro = so + (uint32_t)((t * 128 * kRowBytes) >> 4), co = so + (uint32_t)((b * CB * kRowBytes) >> 4);
+                    const uint32_t idesc = make_idesc_bf16(128, ncols, 0, 0);
+                    const uint32_t t_s = tmem_base + buf * kColBuf, t_dp = t_s + CB;
+                    if (elect_one()) {
+                        mma_ss_h<false>(t_s, d_k + ro, d_q + co, d_hi, idesc);
+                        mma_ss_h<true>(t_s, d_k + ro + 2, d_q + co + 2, d_hi, idesc);
+                        mma_ss_h<false>(t_dp, d_v + ro, d_do + co, d_hi, idesc);
+                        mma_ss_h<true>(t_dp, d_v + ro + 2, d_do + co + 2, d_hi, idesc);
+                        mma_commit(bar_sdp(buf));
+                    }
+                    __syncwarp();
+                };
+                // Both buffers are free here: the previous item's elementwise work is over (its ds barriers were
+                // waited for) and the MMAs that read the buffers were issued earlier by this warp.
+                issue_sdp(0, 0, 0);
+                int t2 = 0, b2 = 1;                        // block j + 1, then j + 2: the look-ahead position
+                if (b2 == nblk) { t2 = 1; b2 = 0; }
+                if (nb_total > 1) issue_sdp(t2, b2, 1);
+                int j = 0;
+                for (int t = 0; t < ntiles && ok; ++t) {
+                    const int set = n_tile & 1;
+                    const uint32_t ro = so + (uint32_t)((t * 128 * kRowBytes) >> 4);
+                    for (int b = 0; b < nblk; ++b, ++j) {
+                        const int buf = j & 1;
+                        const int nks = min(CB, npad - b * CB) >> 4;
+                        ok = mbar_wait_warp(bar_ds(buf), (ph_ds >> buf) & 1, cta_abort);
+                        ph_ds ^= 1u << buf;
+                        if (ok && b == 0 && n_tile >= 2)     // the accumulator set must have been read back (tile n_tile - 2)
+                            ok = mbar_wait_warp(bar_accfree(set), ((n_tile >> 1) - 1) & 1, cta_abort);
+                        if (!ok) break;
+                        tc_fence_after();
+                        // dV += P^T dO, dK += dS^T Q over the block's query columns
+                        const uint32_t co = so + (uint32_t)((b * CB * kRowBytes) >> 4);
+                        const uint32_t t_p = tmem_base + buf * kColBuf, t_dst = t_p + CB;
+                        if (elect_one()) {
+                            const uint32_t a_dv = tmem_base + kColDV + 64 * set, a_dk = tmem_base + kColDK + 64 * set;
+                            const uint32_t b_do = d_do + co, b_q = d_q + co;
+                            if (b == 0) {
+                                mma_ts_h<false>(a_dv, t_p, b_do, d_hi, idesc_acc);
+                                mma_ts_h<false>(a_dk, t_dst, b_q, d_hi, idesc_acc);
+                            } else {
+                                mma_ts_h<true>(a_dv, t_p, b_do, d_hi, idesc_acc);
+                                mma_ts_h<true>(a_dk, t_dst, b_q, d_hi, idesc_acc);
+                            }
+                            if (nks == 4) {
+                                mma_ts_h<true>(a_dv, t_p + 16, b_do + 64, d_hi, idesc_acc);
+                                mma_ts_h<true>(a_dk, t_dst + 16, b_q + 64, d_hi, idesc_acc);
+                                mma_ts_h<true>(a_dv, t_p + 32, b_do + 128, d_hi, idesc_acc);
+                                mma_ts_h<true>(a_dk, t_dst + 32, b_q + 128, d_hi, idesc_acc);
+                                mma_ts_h<true>(a_dv, t_p + 48, b_do + 192, d_hi, idesc_acc);
+                                mma_ts_h<true>(a_dk, t_dst + 48, b_q + 192, d_hi, idesc_acc);
+                            } else {
+                                for (int ks = 1; ks < nks; ++ks) {
+                                    mma_ts_h<true>(a_dv, t_p + 16 * ks, b_do + 64 * ks, d_hi, idesc_acc);
+                                    mma_ts_h<true>(a_dk, t_dst + 16 * ks, b_q + 64 * ks, d_hi, idesc_acc);
+                                }
+                            }
+                        }
+                        __syncwarp();
+                        // look ahead two blocks
+                        if (++b2 == nblk) { ++t2; b2 = 0; }
+                        if (j + 2 < nb_total) issue_sdp(t2, b2, buf);
+                        if ((b & 1) || b == nblk - 1) {
+                            // dQ (queries of this pair of blocks) += dS K over the tile's keys
+                            if (t == 0 && b < 2 && kuse > 0) {   // the item's first write of dQ: the previous item's was read
+                                ok = mbar_wait_warp(bar_dqfree, (kuse - 1) & 1, cta_abort);
+                                if (!ok) break;
+                                tc_fence_after();
+                            }
+                            if (elect_one()) {
+                                const uint32_t a_dq = tmem_base + kColDQ + 32 * (b >> 1);
+                                const uint32_t b_k = d_k + ro;
+                                if (t == 0) mma_ss_h<false>(a_dq, d_ds, b_k, d_hi, idesc_dq);
+                                else mma_ss_h<true>(a_dq, d_ds, b_k, d_hi, idesc_dq);
+#pragma unroll
+                                for (int ks = 1; ks < 8; ++ks)     // all 8 key steps: the interleaved key order spreads the keys over all rows
+                                    mma_ss_h<true>(a_dq, d_ds + 64 * ks, b_k + 64 * ks, d_hi, idesc_dq);
+                                mma_commit(bar_dsfree);
+                                if (b == nblk - 1) mma_commit(bar_acc(set));   // covers the dQ MMAs too: they read this tile's K rows
+                            }
+                            __syncwarp();
+                        }
+                    }
+                    ++n_tile;
+                }
+                if (!ok) break;
+                if (elect_one()) mma_commit(bar_dq);
+                __syncwarp();
+            }
+        }
+    }
+    } else {
+        // ------------------------------------------------------------------ elementwise warps
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(kRegsWork));
+        const int h = warp >> 2;                 // which 16-column steps of a block: h and h + 2
+        const int quarter = warp & 3;            // TMEM lane quarter = 32 key rows of the tile
+        const uint32_t lane_addr = ((uint32_t)(32 * quarter)) << 16;
+        const float scale = g.scale_log2e;
+        const float out_scale = g.scale_log2e * kLn2;          // dQ and dK carry the score scale
+        int kuse = 0, n_tile = 0, n_pair = 0;
+        uint32_t ph_sdp = 0;             // bit b: parity of the next completion of bar_sdp(b)
+        bool ok = true;
+
+        for (long long it = cta_in_head; ok && it < n_items; it += ctas_per_head, ++kuse) {
+            const Item x = make_item(g, it);
+            const int s = kuse % kStages;
+            unsigned char* st = smem + s * kStageBytes;
+            const uint32_t st_a = smem0 + s * kStageBytes;
+            if (!mbar_wait_warp(bar_full(s), (kuse / kStages) & 1, cta_abort)) break;
+            for (int t = 0; t < x.ntiles && ok; ++t) {
+                const int krow = 32 * quarter + lane;            // key row inside the tile
+                const int M = 4 * x.ntiles;
+                const int slot = 32 * ((4 * t + quarter + lane) & (M - 1)) + lane;     // interleaved key order
+                // Bias-gradient updates.  In a full-width window (width = w) the bias code of a slot is the slot
+                // number plus 32 per window row, so code mod 32 = slot mod 32 = lane: the 32 updates of one warp
+                // instruction (32 keys, one query) fall into 32 different banks and entries.  If w also divides 32
+                // (window rows never straddle a 32-slot group), two keys of a warp in the same window row lie in
+                // the same group with lanes congruent mod M, i.e. >= M slots = codes apart, keys in different rows
+                // are >= 33 codes apart, and G <= min(M, w) consecutive queries of a group aligned to G sit in one
+                // window row 1 .. G - 1 codes apart: the 32 x G updates of such a query group never meet and are
+                // issued together.  Other windows are updated one query at a time.
+                int rmw_mode = 1;
+                if (x.r.ew == g.w && (32 % g.w) == 0 && g.w >= 4) rmw_mode = (M == 8 && g.w >= 8) ? 8 : 4;
+                const int coloff_i = lds_i32(st_a + kOffColOff + 4 * slot);
+                const int tok = lds_i32(st_a + kOffTok + 4 * slot);
+                RowCtx rc;
+                rc.label = lds_i32(st_a + kOffLab + 4 * slot);
+                rc.valid = tok >= 0;
+                // bias index = code_query - code_key + c0; a key row without a token reads the table's -inf zone
+                rc.bias_row = smem0 + kOffBias + (rc.valid ? 4 * c0 - coloff_i : 4 * (2 * c0 + 1));
+                rc.dbias_row = smem0 + kOffDBias + 4 * (warp * kDBiasFloats + c0) - coloff_i;
+                rc.scratch = smem0 + kOffDBias + 4 * (warp * kDBiasFloats + kDBiasEntries + lane);
+                for (int b = 0; b < x.nblk; ++b) {
+                    const int j = t * x.nblk + b, buf = j & 1;
+                    const int nsteps = min(CB, x.npad - b * CB) >> 4;
+                    const bool has_a = h < nsteps, has_b = h + 2 < nsteps;
+                    ok = mbar_wait_warp(bar_sdp(buf), (ph_sdp >> buf) & 1, cta_abort);
+                    if (!ok) break;
+                    ph_sdp ^= 1u << buf;
+                    tc_fence_after();
+                    const uint32_t t_s = tmem_base + lane_addr + buf * kColBuf, t_dp = t_s + CB;
+                    // step h: load, compute, write back; the loads of step h + 2 are in flight during the
+                    // bias-gradient updates of step h
+                    uint32_t sa[16], pa[16], pk_p[8], pk_dsa[8], pk_dsb[8], addr[16];
+                    float ds[16];
+                    const int ca = b * CB + 16 * h, cb2 = ca + 32;
+                    if (has_a) {
+                        tmem_ld16(t_s + 16 * h, sa);
+                        tmem_ld16(t_dp + 16 * h, pa);
+                        tmem_ld_wait();
+                        if (x.masked) cols16<true, true>(sa, pa, ca, rc, st_a, scale, pk_p, pk_dsa, ds, addr);
+                        else if (x.ragged) cols16<false, true>(sa, pa, ca, rc, st_a, scale, pk_p, pk_dsa, ds, addr);
+                        else cols16<false, false>(sa, pa, ca, rc, st_a, scale, pk_p, pk_dsa, ds, addr);
+                        tmem_st8(t_s + 16 * h, pk_p);
+                        tmem_st8(t_dp + 16 * h, pk_dsa);
+                        if (has_b) {
+                            tmem_ld16(t_s + 16 * (h + 2), sa);
+                            tmem_ld16(t_dp + 16 * (h + 2), pa);
+                        }
+                        dbias_add16(rmw_mode, addr, ds);
+                    }
+                    if (has_b) {
+                        tmem_ld_wait();
+                        if (x.masked) cols16<true, true>(sa, pa, cb2, rc, st_a, scale, pk_p, pk_dsb, ds, addr);
+                        else if (x.ragged) cols16<false, true>(sa, pa, cb2, rc, st_a, scale, pk_p, pk_dsb, ds, addr);
+                        else cols16<false, false>(sa, pa, cb2, rc, st_a, scale, pk_p, pk_dsb, ds, addr);
+                        tmem_st8(t_s + 16 * (h + 2), pk_p);
+                        tmem_st8(t_dp + 16 * (h + 2), pk_dsb);
+                        dbias_add16(rmw_mode, addr, ds);
+                    }
+                    // dS^T into the shared tile of this pair of blocks (32-query groups 2 (b & 1) and 2 (b & 1) + 1;
+                    // step h -> group 2 (b & 1), step h + 2 -> the next group; 16-byte chunks 2 h and 2 h + 1)
+                    if ((b & 1) == 0 && n_pair > 0) {
+                        ok = mbar_wait_warp(bar_dsfree, (n_pair - 1) & 1, cta_abort);
+                        if (!ok) break;
+                    }
+                    {
+                        const uint32_t base = smem0 + kOffDS + 2 * (b & 1) * kDSGroupBytes;
+                        if (has_a) {
+                            sts_u4(base + tile_off<kD>(krow, 2 * h), pk_dsa[0], pk_dsa[1], pk_dsa[2], pk_dsa[3]);
+                            sts_u4(base + tile_off<kD>(krow, 2 * h + 1), pk_dsa[4], pk_dsa[5], pk_dsa[6], pk_dsa[7]);
+                        }
+                        if (has_b) {
+                            sts_u4(base + kDSGroupBytes + tile_off<kD>(krow, 2 * h), pk_dsb[0], pk_dsb[1], pk_dsb[2], pk_dsb[3]);
+                            sts_u4(base + kDSGroupBytes + tile_off<kD>(krow, 2 * h + 1), pk_dsb[4], pk_dsb[5], pk_dsb[6], pk_dsb[7]);
+                        }
+                    }
+                    if ((b & 1) || b == x.nblk - 1) ++n_pair;
+                    tmem_st_wait();
+                    tc_fence_before();
+                    fence_proxy_async();
+                    mbar_arrive_warp(bar_ds(buf));
+                }
+                if (!ok) break;
+                // ---- the tile's dV (warps 0..3) / dK (warps 4..7): one 64-byte row per thread
+                const int set = n_tile & 1;
+                ok = mbar_wait_warp(bar_acc(set), (n_tile >> 1) & 1, cta_abort);
+                if (!ok) break;
+                ++n_tile;
+                tc_fence_after();
+                uint32_t r[32];
+                tmem_ld32(tmem_base + lane_addr + (h == 0 ? kColDV : kColDK) + 64 * set, r);
+                tmem_ld_wait();
+                tc_fence_before();
+                mbar_arrive_warp(bar_accfree(set));
+                {
+                    const float f = h == 0 ? 1.f : out_scale;
+                    // the tile's own V (K) rows are dead now: stage the output rows there, then store whole rows
+                    unsigned char* stg = st + (h == 0 ? kOffV : kOffK) + (t * 128 + 32 * quarter) * kRowBytes;
+                    __nv_bfloat16* out = h == 0 ? dv : dk;
+#pragma unroll
+                    for (int c4 = 0; c4 < 4; ++c4) {
+                        uint4 a;
+                        a.x = pack_bf16(__uint_as_float(r[c4 * 8 + 0]) * f, __uint_as_float(r[c4 * 8 + 1]) * f);
+                        a.y = pack_bf16(__uint_as_float(r[c4 * 8 + 2]) * f, __uint_as_float(r[c4 * 8 + 3]) * f);
+                        a.z = pack_bf16(__uint_as_float(r[c4 * 8 + 4]) * f, __uint_as_float(r[c4 * 8 + 5]) * f);
+                        a.w = pack_bf16(__uint_as_float(r[c4 * 8 + 6]) * f, __uint_as_float(r[c4 * 8 + 7]) * f);
+                        *reinterpret_cast<uint4*>(stg + tile_off<kD>(lane, c4)) = a;
+                    }
+                    __syncwarp();
+#pragma unroll
+                    for (int jj = 0; jj < 4; ++jj) {
+                        const int rr = 8 * jj + (lane >> 2), c4 = lane & 3;
+                        const int tok_r = __shfl_sync(0xffffffffu, tok, rr);
+                        const uint4 a = *reinterpret_cast<const uint4*>(stg + tile_off<kD>(rr, c4));
+                        if (tok_r >= 0)
+                            *reinterpret_cast<uint4*>(out + (((size_t)x.b * HW + (size_t)tok_r) * g.heads + head) * kD + c4 * 8) = a;
+                    }
+                    __syncwarp();
+                }
+            }
+            if (!ok) break;
+            // ---- dQ: queries 0..127 by warps 0..3, queries 128..255 by warps 4..7
+            if (!mbar_wait_warp(bar_dq, kuse & 1, cta_abort)) break;
+            tc_fence_after();
+            const bool have_q = h * 128 < x.npad;
+            uint32_t r[32];
+            if (have_q) {
+                tmem_ld32(tmem_base + lane_addr + kColDQ + 32 * h, r);
+                tmem_ld_wait();
+            }
+            tc_fence_before();
+            mbar_arrive_warp(bar_dqfree);
+            if (have_q) {
+                const int tokq = lds_i32(st_a + kOffTok + 4 * (h * 128 + 32 * quarter + lane));
+                unsigned char* stg = st + kOffQ + (h * 128 + 32 * quarter) * kRowBytes;
+#pragma unroll
+                for (int c4 = 0; c4 < 4; ++c4) {
+                    uint4 a;
+                    a.x = pack_bf16(__uint_as_float(r[c4 * 8 + 0]) * out_scale, __uint_as_float(r[c4 * 8 + 1]) * out_scale);
+                    a.y = pack_bf16(__uint_as_float(r[c4 * 8 + 2]) * out_scale, __uint_as_float(r[c4 * 8 + 3]) * out_scale);
+                    a.z = pack_bf16(__uint_as_float(r[c4 * 8 + 4]) * out_scale, __uint_as_float(r[c4 * 8 + 5]) * out_scale);
+                    a.w = pack_bf16(__uint_as_float(r[c4 * 8 + 6]) * out_scale, __uint_as_float(r[c4 * 8 + 7]) * out_scale);
+                    *reinterpret_cast<uint4*>(stg + tile_off<kD>(lane, c4)) = a;
+                }
+                __syncwarp();
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj) {
+                    const int rr = 8 * jj + (lane >> 2), c4 = lane & 3;
+                    const int tok_r = __shfl_sync(0xffffffffu, tokq, rr);
+                    const uint4 a = *reinterpret_cast<const uint4*>(stg + tile_off<kD>(rr, c4));
+                    if (tok_r >= 0)
+                        *reinterpret_cast<uint4*>(dq + (((size_t)x.b * HW + (size_t)tok_r) * g.heads + head) * kD + c4 * 8) = a;
+                }
+                __syncwarp();
+            }
+            mbar_arrive_warp(bar_empty(s));       // this warp no longer touches the stage
+        }
+    }
+
+    // teardown: every role ends up here, also after an expired wait
+    cp_async_wait<0>();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == kMmaWarp) tmem_dealloc(tmem_base, 512);
+    {
+        // this CTA's table = sum of its warps' tables (fixed order), written to the CTA's slot of the workspace
+        const float* tbl = reinterpret_cast<const float*>(smem + kOffDBias);
+        for (int e = tid; e < kDBiasFloats; e += kThreads) {
+            float acc = 0.f;
+#pragma unroll
+            for (int wq = 0; wq < 8; ++wq) acc += tbl[wq * kDBiasFloats + e];
+            dbias_parts[(size_t)blockIdx.x * kDBiasFloats + e] = acc;
+        }
+    }
+    if (tid == 0 && *cta_abort) atomicExch(&g_bwd_tc_timeout, 1);
+}
+
+// dbias[(da, db), head] = sum over the head's CTAs of their tables (entry (da + w - 1) * cs + (db + w - 1)).
+// Fixed summation order over warps and CTAs: the bias gradient is reproducible run to run.
+__global__ void __launch_bounds__(256)
+swin_bwd_dbias_finalize_kernel(const float* __restrict__ parts, float* __restrict__ dbias, int w, int heads, int ctas_per_head) {
+    const int nw = 2 * w - 1, cs = w + 32;
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;       // (table row, head)
+    if (i >= nw * nw * heads) return;
+    const int head = i % heads, r = i / heads;
+    const int e = (r / nw) * cs + (r % nw);
+    float acc = 0.f;
+    for (int c = 0; c < ctas_per_head; ++c) acc += parts[(size_t)(c * heads + head) * kDBiasFloats + e];
+    dbias[i] = acc;
+}
+
+}  // namespace
+
+cudaError_t read_bwd_tc_status(int* timed_out) {
+    int zero = 0;
+    cudaError_t e = cudaMemcpyFromSymbol(timed_out, g_bwd_tc_timeout, sizeof(int));
+    if (e != cudaSuccess) return e;
+    if (*timed_out) e = cudaMemcpyToSymbol(g_bwd_tc_timeout, &zero, sizeof(int));
+    return e;
+}
+
+constexpr int kMaxGrid = 160;   // CTAs whose bias-gradient tables fit the workspace
+
+bool bwd_tc_supported(const Geo& g) { return g.d == 32 && g.nmax <= kMaxSlots && g.w <= 16 && g.heads <= 148; }
+
+// workspace: delta [B*H*W*heads] fp32, the prepared bias tables [heads * kFwdBiasFloats] fp32, one
+// bias-gradient table per CTA
+size_t bwd_tc_workspace_bytes(const Geo& g) {
+    const size_t delta = (((size_t)g.B * g.H * g.W * g.heads * sizeof(float)) + 255) / 256 * 256;
+    return delta + (size_t)g.heads * kFwdBiasFloats * sizeof(float) + (size_t)kMaxGrid * kDBiasFloats * sizeof(float);
+}
+
+cudaError_t launch_bwd_tc(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
+                          const void* o, const float* lse, const void* d_o, void* dq, void* dk, void* dv, float* dbias,
+                          void* workspace, int sm_count, cudaStream_t stream) {
+    float* delta = reinterpret_cast<float*>(workspace);
+    const size_t delta_bytes = (((size_t)g.B * g.H * g.W * g.heads * sizeof(float)) + 255) / 256 * 256;
+    float* prep = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(workspace) + delta_bytes);
+    cudaError_t e = launch_bwd_delta(g, o, d_o, delta, stream);
+    if (e != cudaSuccess) return e;
+    e = launch_bias_prep(g, bias, prep, stream);
+    if (e != cudaSuccess) return e;
+    float* parts = prep + (size_t)g.heads * kFwdBiasFloats;
+    const long long items = (long long)g.B * g.Mh * g.Mw;
+    long long cph = (sm_count < kMaxGrid ? sm_count : kMaxGrid) / g.heads;
+    if (cph < 1) cph = 1;
+    if (cph > items) cph = items;
+    const unsigned grid = (unsigned)(cph * g.heads);
+    e = cudaFuncSetAttribute(swin_bwd_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    prof_begin("swin_bwd_fused_kernel", stream);
+    swin_bwd_fused_kernel<<<grid, kThreads, kSmemBytes, stream>>>(
+        g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)d_o, prep, lse, delta,
+        (__nv_bfloat16*)dq, (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, parts, items, (int)cph);
+    count_launch(stream);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const int nrows = (2 * g.w - 1) * (2 * g.w - 1) * g.heads;
+    swin_bwd_dbias_finalize_kernel<<<(nrows + 255) / 256, 256, 0, stream>>>(parts, dbias, g.w, g.heads, (int)cph);
+    count_launch(stream);
+    return cudaGetLastError();
+}
+
+}  // namespace terra
