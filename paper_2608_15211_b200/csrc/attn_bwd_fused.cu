@@ -30,8 +30,11 @@ namespace {
 
 using namespace tc;
 
-constexpr int kMmaWarp = 8;         // warp 8: one MMA-issuing lane
-constexpr int kLoaderWarp0 = 9;
+// Roles by role number; the role of a hardware warp is (warp + 8) mod 12, so that the MMA issuer is hardware
+// warp 0: it shares a scheduler with two elementwise warps that are rarely stalled, and as a late warp it
+// was given an issue slot only every few dozen cycles.
+constexpr int kIssuerWarp = 8;      // role 8: MMA issuer (also owns the TMEM allocation)
+constexpr int kLoaderWarp0 = 9;     // roles 9..11: loaders
 constexpr int kLoaderWarps = 3;
 constexpr int kLoaderThreads = kLoaderWarps * 32;
 constexpr int kThreads = (kLoaderWarp0 + kLoaderWarps) * 32;   // 384 = three warpgroups
@@ -265,7 +268,8 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail);
     volatile int* cta_abort = reinterpret_cast<volatile int*>(tail + 8);
 
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int warp = ((tid >> 5) + 8) % 12;      // role number (see the constants above)
     const int head = blockIdx.x % g.heads;
     const int cta_in_head = blockIdx.x / g.heads;
 
@@ -293,7 +297,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
     // the shared dS tile starts finite: columns that no block writes only reach dQ rows that are never stored
     for (int i = tid; i < 4 * kDSGroupBytes / 4; i += kThreads) reinterpret_cast<uint32_t*>(smem + kOffDS)[i] = 0u;
     fence_proxy_async();
-    if (warp == kMmaWarp) {
+    if (warp == kIssuerWarp) {
         tmem_alloc(smem_u32(tmem_slot), 512);
         tmem_relinquish();
     }
@@ -306,11 +310,12 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
     const int c0 = (g.w - 1) * (cs + 1);
     const size_t HW = (size_t)g.H * g.W;
 
-    if (warp >= kMmaWarp) {
+    if (warp >= kIssuerWarp) {
+    // hardware warps 0..3 = one warpgroup (issuer + loaders) give registers back: one instruction for the whole warpgroup
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kRegsOther));
     if (warp >= kLoaderWarp0) {
         // ------------------------------------------------------------------ loaders
-        const int lt = tid - kLoaderWarp0 * 32;
+        const int lt = (warp - kLoaderWarp0) * 32 + lane;
         int kuse = 0, pending_s = -1;
         for (long long it = cta_in_head; it < n_items; it += ctas_per_head, ++kuse) {
             const int s = kuse % kStages;
@@ -394,123 +399,145 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
             mbar_arrive(bar_full(pending_s));
         }
     } else {
-        // ------------------------------------------------------------------ MMA issuer (warp 8)
+        // ------------------------------------------------------------------ MMA issuer
         // The whole warp runs the loop (warp-uniform control flow and operands); one elected lane issues.
-        {
-            const uint32_t idesc_acc = make_idesc_bf16(128, kD, 0, 1);   // A from TMEM, B = 16 rows x 32 (MN-major)
-            const uint32_t idesc_dq = make_idesc_bf16(128, kD, 1, 1);    // A = dS^T tile read transposed, B = 16 K rows x 32
-            // shared-memory descriptors: one common high word, low words = start address (16-byte units)
-            const uint32_t d_hi = sdesc_hi(make_sdesc_sw64(smem0, 512));
-            const uint32_t d_q = sdesc_lo(make_sdesc_sw64(smem0 + kOffQ, 512)), d_k = sdesc_lo(make_sdesc_sw64(smem0 + kOffK, 512));
-            const uint32_t d_v = sdesc_lo(make_sdesc_sw64(smem0 + kOffV, 512)), d_do = sdesc_lo(make_sdesc_sw64(smem0 + kOffDO, 512));
-            const uint32_t d_ds = sdesc_lo(make_sdesc_sw64_mn(smem0 + kOffDS, kDSGroupBytes, 512));
-            bool ok = true;
-            int kuse = 0, n_tile = 0;
-            uint32_t ph_ds = 0;          // bit b: parity of the next completion of bar_ds(b)
-            for (long long it = cta_in_head; ok && it < n_items; it += ctas_per_head, ++kuse) {
-                const int s = kuse % kStages;
-                int npad, ntiles, nblk;
-                {
-                    const Item x = make_item(g, it);
-                    npad = x.npad; ntiles = x.ntiles; nblk = x.nblk;
+        // The CTA's blocks form one sequence across tiles and items: block J uses S / dP buffer J & 1, and its
+        // S^T / dP^T are issued two blocks ahead (from the previous item's last blocks where needed, as soon as
+        // the item's stage is loaded), so the elementwise warps find them ready.
+        const uint32_t idesc_acc = make_idesc_bf16(128, kD, 0, 1);   // A from TMEM, B = 16 rows x 32 (MN-major)
+        const uint32_t idesc_dq = make_idesc_bf16(128, kD, 1, 1);    // A = dS^T tile read transposed, B = 16 K rows x 32
+        // shared-memory descriptors: one common high word, low words = start address (16-byte units)
+        const uint32_t d_hi = sdesc_hi(make_sdesc_sw64(smem0, 512));
+        const uint32_t d_q = sdesc_lo(make_sdesc_sw64(smem0 + kOffQ, 512)), d_k = sdesc_lo(make_sdesc_sw64(smem0 + kOffK, 512));
+        const uint32_t d_v = sdesc_lo(make_sdesc_sw64(smem0 + kOffV, 512)), d_do = sdesc_lo(make_sdesc_sw64(smem0 + kOffDO, 512));
+        const uint32_t d_ds = sdesc_lo(make_sdesc_sw64_mn(smem0 + kOffDS, kDSGroupBytes, 512));
+        uint32_t ph_ds = 0;              // bit b: parity of the next completion of bar_ds(b)
+        int J = 0;                       // number of the current block in the CTA's sequence
+        int n_issued = 0;                // S^T / dP^T have been issued for blocks [0, n_issued)
+        int kuse = 0, n_tile = 0;
+        bool ok = true;
+        // S^T = K Q^T and dP^T = V dO^T of query block b of key tile t (item in stage `stage`, npad_i columns) into buffer `buf`
+        auto issue_sdp = [&](int stage, int npad_i, int t, int b, int buf) {
+            const int ncols = min(CB, npad_i - b * CB);
+            const uint32_t so = (uint32_t)((stage * kStageBytes) >> 4);
+            const uint32_t ro = so + (uint32_t)((t * 128 * kRowBytes) >> 4), co = so + (uint32_t)((b * CB * kRowBytes) >> 4);
+            const uint32_t idesc = make_idesc_bf16(128, ncols, 0, 0);
+            const uint32_t t_s = tmem_base + buf * kColBuf, t_dp = t_s + CB;
+            if (elect_one()) {
+                mma_ss_h<false>(t_s, d_k + ro, d_q + co, d_hi, idesc);
+                mma_ss_h<true>(t_s, d_k + ro + 2, d_q + co + 2, d_hi, idesc);
+                mma_ss_h<false>(t_dp, d_v + ro, d_do + co, d_hi, idesc);
+                mma_ss_h<true>(t_dp, d_v + ro + 2, d_do + co + 2, d_hi, idesc);
+                mma_commit(bar_sdp(buf));
+            }
+            __syncwarp();
+        };
+        for (long long it = cta_in_head; ok && it < n_items; it += ctas_per_head, ++kuse) {
+            const int s = kuse % kStages;
+            int npad, ntiles, nblk;
+            {
+                const Item x = make_item(g, it);
+                npad = x.npad; ntiles = x.ntiles; nblk = x.nblk;
+            }
+            const int nb = ntiles * nblk;
+            // the item after this one
+            int nb_n = 0, npad_n = 0, nblk_n = 1;
+            if (it + ctas_per_head < n_items) {
+                const Item xn = make_item(g, it + ctas_per_head);
+                nb_n = xn.ntiles * xn.nblk; npad_n = xn.npad; nblk_n = xn.nblk;
+            }
+            const int J0 = J;
+            ok = mbar_wait_warp(bar_full(s), (kuse / kStages) & 1, cta_abort);
+            if (!ok) break;
+            fence_proxy_async();
+            tc_fence_after();
+            // S / dP of blocks [n_issued, limit): blocks of this item, or of the next one (other stage, once it is loaded)
+            auto issue_upto = [&](int limit) -> bool {
+                for (int jt = n_issued; jt < limit; ++jt) {
+                    int local = jt - J0;
+                    if (local < nb) {
+                        const int t = local >= nblk ? 1 : 0;
+                        issue_sdp(s, npad, t, local - t * nblk, jt & 1);
+                    } else {
+                        local -= nb;
+                        const int sn = (kuse + 1) % kStages;
+                        if (!mbar_wait_warp(bar_full(sn), ((kuse + 1) / kStages) & 1, cta_abort)) return false;
+                        fence_proxy_async();
+                        const int t = local >= nblk_n ? 1 : 0;
+                        issue_sdp(sn, npad_n, t, local - t * nblk_n, jt & 1);
+                    }
                 }
-                const int nb_total = ntiles * nblk;
-                const uint32_t so = (uint32_t)((s * kStageBytes) >> 4);
-                ok = mbar_wait_warp(bar_full(s), (kuse / kStages) & 1, cta_abort);
-                if (!ok) break;
-                fence_proxy_async();
-                tc_fence_after();
-                // S^T = K Q^T and dP^T = V dO^T of query block b of key tile t into buffer `buf`
-                auto issue_sdp = [&](int t, int b, int buf) {
-                    const int ncols = min(CB, npad - b * CB);
-                    const uint32_t ro = so + (uint32_t)((t * 128 * kRowBytes) >> 4), co = so + (uint32_t)((b * CB * kRowBytes) >> 4);
-                    const uint32_t idesc = make_idesc_bf16(128, ncols, 0, 0);
-                    const uint32_t t_s = tmem_base + buf * kColBuf, t_dp = t_s + CB;
+                if (limit > n_issued) n_issued = limit;
+                return true;
+            };
+            if (kuse == 0) ok = issue_upto(min(2, nb + nb_n));     // the first two blocks have no earlier block to be issued from
+            const uint32_t so = (uint32_t)((s * kStageBytes) >> 4);
+            for (int t = 0; t < ntiles && ok; ++t) {
+                const int set = n_tile & 1;
+                for (int b = 0; b < nblk; ++b, ++J) {
+                    const int buf = J & 1;
+                    const int nks = min(CB, npad - b * CB) >> 4;
+                    ok = mbar_wait_warp(bar_ds(buf), (ph_ds >> buf) & 1, cta_abort);          // all eight warps are done with block J
+                    ph_ds ^= 1u << buf;
+                    if (ok && b == 0 && n_tile >= 2)     // the accumulator set must have been read back (tile n_tile - 2)
+                        ok = mbar_wait_warp(bar_accfree(set), ((n_tile >> 1) - 1) & 1, cta_abort);
+                    if (!ok) break;
+                    tc_fence_after();
+                    // dV += P^T dO, dK += dS^T Q over the block's query columns
                     if (elect_one()) {
-                        mma_ss_h<false>(t_s, d_k + ro, d_q + co, d_hi, idesc);
-                        mma_ss_h<true>(t_s, d_k + ro + 2, d_q + co + 2, d_hi, idesc);
-                        mma_ss_h<false>(t_dp, d_v + ro, d_do + co, d_hi, idesc);
-                        mma_ss_h<true>(t_dp, d_v + ro + 2, d_do + co + 2, d_hi, idesc);
-                        mma_commit(bar_sdp(buf));
+                        const uint32_t a_dv = tmem_base + kColDV + 64 * set, a_dk = tmem_base + kColDK + 64 * set;
+                        const uint32_t t_p = tmem_base + buf * kColBuf, t_dst = t_p + CB;
+                        const uint32_t b_do = d_do + so + (uint32_t)((b * CB * kRowBytes) >> 4), b_q = d_q + so + (uint32_t)((b * CB * kRowBytes) >> 4);
+                        if (b == 0) {
+                            mma_ts_h<false>(a_dv, t_p, b_do, d_hi, idesc_acc);
+                            mma_ts_h<false>(a_dk, t_dst, b_q, d_hi, idesc_acc);
+                        } else {
+                            mma_ts_h<true>(a_dv, t_p, b_do, d_hi, idesc_acc);
+                            mma_ts_h<true>(a_dk, t_dst, b_q, d_hi, idesc_acc);
+                        }
+                        if (nks == 4) {
+                            mma_ts_h<true>(a_dv, t_p + 16, b_do + 64, d_hi, idesc_acc);
+                            mma_ts_h<true>(a_dk, t_dst + 16, b_q + 64, d_hi, idesc_acc);
+                            mma_ts_h<true>(a_dv, t_p + 32, b_do + 128, d_hi, idesc_acc);
+                            mma_ts_h<true>(a_dk, t_dst + 32, b_q + 128, d_hi, idesc_acc);
+                            mma_ts_h<true>(a_dv, t_p + 48, b_do + 192, d_hi, idesc_acc);
+                            mma_ts_h<true>(a_dk, t_dst + 48, b_q + 192, d_hi, idesc_acc);
+                        } else {
+                            for (int ks = 1; ks < nks; ++ks) {
+                                mma_ts_h<true>(a_dv, t_p + 16 * ks, b_do + 64 * ks, d_hi, idesc_acc);
+                                mma_ts_h<true>(a_dk, t_dst + 16 * ks, b_q + 64 * ks, d_hi, idesc_acc);
+                            }
+                        }
                     }
                     __syncwarp();
-                };
-                // Both buffers are free here: the previous item's elementwise work is over (its ds barriers were
-                // waited for) and the MMAs that read the buffers were issued earlier by this warp.
-                issue_sdp(0, 0, 0);
-                int t2 = 0, b2 = 1;                        // block j + 1, then j + 2: the look-ahead position
-                if (b2 == nblk) { t2 = 1; b2 = 0; }
-                if (nb_total > 1) issue_sdp(t2, b2, 1);
-                int j = 0;
-                for (int t = 0; t < ntiles && ok; ++t) {
-                    const int set = n_tile & 1;
-                    const uint32_t ro = so + (uint32_t)((t * 128 * kRowBytes) >> 4);
-                    for (int b = 0; b < nblk; ++b, ++j) {
-                        const int buf = j & 1;
-                        const int nks = min(CB, npad - b * CB) >> 4;
-                        ok = mbar_wait_warp(bar_ds(buf), (ph_ds >> buf) & 1, cta_abort);
-                        ph_ds ^= 1u << buf;
-                        if (ok && b == 0 && n_tile >= 2)     // the accumulator set must have been read back (tile n_tile - 2)
-                            ok = mbar_wait_warp(bar_accfree(set), ((n_tile >> 1) - 1) & 1, cta_abort);
-                        if (!ok) break;
-                        tc_fence_after();
-                        // dV += P^T dO, dK += dS^T Q over the block's query columns
-                        const uint32_t co = so + (uint32_t)((b * CB * kRowBytes) >> 4);
-                        const uint32_t t_p = tmem_base + buf * kColBuf, t_dst = t_p + CB;
+                    // S^T / dP^T two blocks ahead (this buffer is free again: its P / dS reads were issued just above)
+                    ok = issue_upto(min(J + 3, J0 + nb + nb_n));
+                    if (!ok) break;
+                    if ((b & 1) || b == nblk - 1) {
+                        // dQ (queries of this pair of blocks) += dS K over the tile's keys
+                        if (t == 0 && b < 2 && kuse > 0) {   // the item's first write of dQ: the previous item's was read
+                            ok = mbar_wait_warp(bar_dqfree, (kuse - 1) & 1, cta_abort);
+                            if (!ok) break;
+                            tc_fence_after();
+                        }
                         if (elect_one()) {
-                            const uint32_t a_dv = tmem_base + kColDV + 64 * set, a_dk = tmem_base + kColDK + 64 * set;
-                            const uint32_t b_do = d_do + co, b_q = d_q + co;
-                            if (b == 0) {
-                                mma_ts_h<false>(a_dv, t_p, b_do, d_hi, idesc_acc);
-                                mma_ts_h<false>(a_dk, t_dst, b_q, d_hi, idesc_acc);
-                            } else {
-                                mma_ts_h<true>(a_dv, t_p, b_do, d_hi, idesc_acc);
-                                mma_ts_h<true>(a_dk, t_dst, b_q, d_hi, idesc_acc);
-                            }
-                            if (nks == 4) {
-                                mma_ts_h<true>(a_dv, t_p + 16, b_do + 64, d_hi, idesc_acc);
-                                mma_ts_h<true>(a_dk, t_dst + 16, b_q + 64, d_hi, idesc_acc);
-                                mma_ts_h<true>(a_dv, t_p + 32, b_do + 128, d_hi, idesc_acc);
-                                mma_ts_h<true>(a_dk, t_dst + 32, b_q + 128, d_hi, idesc_acc);
-                                mma_ts_h<true>(a_dv, t_p + 48, b_do + 192, d_hi, idesc_acc);
-                                mma_ts_h<true>(a_dk, t_dst + 48, b_q + 192, d_hi, idesc_acc);
-                            } else {
-                                for (int ks = 1; ks < nks; ++ks) {
-                                    mma_ts_h<true>(a_dv, t_p + 16 * ks, b_do + 64 * ks, d_hi, idesc_acc);
-                                    mma_ts_h<true>(a_dk, t_dst + 16 * ks, b_q + 64 * ks, d_hi, idesc_acc);
-                                }
+                            const uint32_t a_dq = tmem_base + kColDQ + 32 * (b >> 1);
+                            const uint32_t b_k = d_k + so + (uint32_t)((t * 128 * kRowBytes) >> 4);
+                            if (t == 0) mma_ss_h<false>(a_dq, d_ds, b_k, d_hi, idesc_dq);
+                            else mma_ss_h<true>(a_dq, d_ds, b_k, d_hi, idesc_dq);
+#pragma unroll
+                            for (int ks = 1; ks < 8; ++ks)     // all 8 key steps: the interleaved key order spreads the keys over all rows
+                                mma_ss_h<true>(a_dq, d_ds + 64 * ks, b_k + 64 * ks, d_hi, idesc_dq);
+                            mma_commit(bar_dsfree);
+                            if (b == nblk - 1) {
+                                mma_commit(bar_acc(set));                  // the tile's dV / dK (and the dQ MMAs, which read its K rows)
+                                if (t == ntiles - 1) mma_commit(bar_dq);   // the item's last MMAs
                             }
                         }
                         __syncwarp();
-                        // look ahead two blocks
-                        if (++b2 == nblk) { ++t2; b2 = 0; }
-                        if (j + 2 < nb_total) issue_sdp(t2, b2, buf);
-                        if ((b & 1) || b == nblk - 1) {
-                            // dQ (queries of this pair of blocks) += dS K over the tile's keys
-                            if (t == 0 && b < 2 && kuse > 0) {   // the item's first write of dQ: the previous item's was read
-                                ok = mbar_wait_warp(bar_dqfree, (kuse - 1) & 1, cta_abort);
-                                if (!ok) break;
-                                tc_fence_after();
-                            }
-                            if (elect_one()) {
-                                const uint32_t a_dq = tmem_base + kColDQ + 32 * (b >> 1);
-                                const uint32_t b_k = d_k + ro;
-                                if (t == 0) mma_ss_h<false>(a_dq, d_ds, b_k, d_hi, idesc_dq);
-                                else mma_ss_h<true>(a_dq, d_ds, b_k, d_hi, idesc_dq);
-#pragma unroll
-                                for (int ks = 1; ks < 8; ++ks)     // all 8 key steps: the interleaved key order spreads the keys over all rows
-                                    mma_ss_h<true>(a_dq, d_ds + 64 * ks, b_k + 64 * ks, d_hi, idesc_dq);
-                                mma_commit(bar_dsfree);
-                                if (b == nblk - 1) mma_commit(bar_acc(set));   // covers the dQ MMAs too: they read this tile's K rows
-                            }
-                            __syncwarp();
-                        }
                     }
-                    ++n_tile;
                 }
-                if (!ok) break;
-                if (elect_one()) mma_commit(bar_dq);
-                __syncwarp();
+                ++n_tile;
             }
         }
     }
@@ -525,11 +552,92 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
         int kuse = 0, n_tile = 0, n_pair = 0;
         uint32_t ph_sdp = 0;             // bit b: parity of the next completion of bar_sdp(b)
         bool ok = true;
+        // Read-outs are deferred: a tile's dV / dK (and, after an item's last tile, its dQ) are read one block
+        // later, after the first block of the next tile or item, so that the last MMAs of the tile have had a
+        // block's time to complete and no elementwise warp sits waiting for them.
+        int pend_tile = -1, pend_tile_s = 0, pend_tile_b = 0, pend_tile_tok = -1, pend_tile_seq = 0;   // tile index; its stage, sample, key token, tile number
+        int pend_item_s = -1, pend_item_b = 0, pend_item_npad = 0, pend_item_use = 0;                 // stage (-1: none), sample, columns, item number
+        auto flush_pending = [&]() -> bool {
+            if (pend_tile >= 0) {
+                // ---- the tile's dV (warps 0..3) / dK (warps 4..7): one 64-byte row per thread
+                const int set = pend_tile_seq & 1;
+                if (!mbar_wait_warp(bar_acc(set), (pend_tile_seq >> 1) & 1, cta_abort)) return false;
+                tc_fence_after();
+                uint32_t r[32];
+                tmem_ld32(tmem_base + lane_addr + (h == 0 ? kColDV : kColDK) + 64 * set, r);
+                tmem_ld_wait();
+                tc_fence_before();
+                mbar_arrive_warp(bar_accfree(set));
+                const float f = h == 0 ? 1.f : out_scale;
+                // the tile's own V (K) rows are dead now: stage the output rows there, then store whole rows
+                unsigned char* stg = smem + pend_tile_s * kStageBytes + (h == 0 ? kOffV : kOffK) + (pend_tile * 128 + 32 * quarter) * kRowBytes;
+                __nv_bfloat16* out = h == 0 ? dv : dk;
+#pragma unroll
+                for (int c4 = 0; c4 < 4; ++c4) {
+                    uint4 a;
+                    a.x = pack_bf16(__uint_as_float(r[c4 * 8 + 0]) * f, __uint_as_float(r[c4 * 8 + 1]) * f);
+                    a.y = pack_bf16(__uint_as_float(r[c4 * 8 + 2]) * f, __uint_as_float(r[c4 * 8 + 3]) * f);
+                    a.z = pack_bf16(__uint_as_float(r[c4 * 8 + 4]) * f, __uint_as_float(r[c4 * 8 + 5]) * f);
+                    a.w = pack_bf16(__uint_as_float(r[c4 * 8 + 6]) * f, __uint_as_float(r[c4 * 8 + 7]) * f);
+                    *reinterpret_cast<uint4*>(stg + tile_off<kD>(lane, c4)) = a;
+                }
+                __syncwarp();
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj) {
+                    const int rr = 8 * jj + (lane >> 2), c4 = lane & 3;
+                    const int tok_r = __shfl_sync(0xffffffffu, pend_tile_tok, rr);
+                    const uint4 a = *reinterpret_cast<const uint4*>(stg + tile_off<kD>(rr, c4));
+                    if (tok_r >= 0)
+                        *reinterpret_cast<uint4*>(out + (((size_t)pend_tile_b * HW + (size_t)tok_r) * g.heads + head) * kD + c4 * 8) = a;
+                }
+                __syncwarp();
+                pend_tile = -1;
+            }
+            if (pend_item_s >= 0) {
+                // ---- dQ: queries 0..127 by warps 0..3, queries 128..255 by warps 4..7
+                if (!mbar_wait_warp(bar_dq, pend_item_use & 1, cta_abort)) return false;
+                tc_fence_after();
+                const bool have_q = h * 128 < pend_item_npad;
+                uint32_t r[32];
+                if (have_q) {
+                    tmem_ld32(tmem_base + lane_addr + kColDQ + 32 * h, r);
+                    tmem_ld_wait();
+                }
+                tc_fence_before();
+                mbar_arrive_warp(bar_dqfree);
+                if (have_q) {
+                    const int tokq = lds_i32(smem0 + pend_item_s * kStageBytes + kOffTok + 4 * (h * 128 + 32 * quarter + lane));
+                    unsigned char* stg = smem + pend_item_s * kStageBytes + kOffQ + (h * 128 + 32 * quarter) * kRowBytes;
+#pragma unroll
+                    for (int c4 = 0; c4 < 4; ++c4) {
+                        uint4 a;
+                        a.x = pack_bf16(__uint_as_float(r[c4 * 8 + 0]) * out_scale, __uint_as_float(r[c4 * 8 + 1]) * out_scale);
+                        a.y = pack_bf16(__uint_as_float(r[c4 * 8 + 2]) * out_scale, __uint_as_float(r[c4 * 8 + 3]) * out_scale);
+                        a.z = pack_bf16(__uint_as_float(r[c4 * 8 + 4]) * out_scale, __uint_as_float(r[c4 * 8 + 5]) * out_scale);
+                        a.w = pack_bf16(__uint_as_float(r[c4 * 8 + 6]) * out_scale, __uint_as_float(r[c4 * 8 + 7]) * out_scale);
+                        *reinterpret_cast<uint4*>(stg + tile_off<kD>(lane, c4)) = a;
+                    }
+                    __syncwarp();
+#pragma unroll
+                    for (int jj = 0; jj < 4; ++jj) {
+                        const int rr = 8 * jj + (lane >> 2), c4 = lane & 3;
+                        const int tok_r = __shfl_sync(0xffffffffu, tokq, rr);
+                        const uint4 a = *reinterpret_cast<const uint4*>(stg + tile_off<kD>(rr, c4));
+                        if (tok_r >= 0)
+                            *reinterpret_cast<uint4*>(dq + (((size_t)pend_item_b * HW + (size_t)tok_r) * g.heads + head) * kD + c4 * 8) = a;
+                    }
+                    __syncwarp();
+                }
+                mbar_arrive_warp(bar_empty(pend_item_s));       // this warp no longer touches that stage
+                pend_item_s = -1;
+            }
+            return true;
+        };
 
+        int J = 0;                       // number of this block in the CTA's sequence; its S / dP buffer is J & 1
         for (long long it = cta_in_head; ok && it < n_items; it += ctas_per_head, ++kuse) {
             const Item x = make_item(g, it);
             const int s = kuse % kStages;
-            unsigned char* st = smem + s * kStageBytes;
             const uint32_t st_a = smem0 + s * kStageBytes;
             if (!mbar_wait_warp(bar_full(s), (kuse / kStages) & 1, cta_abort)) break;
             for (int t = 0; t < x.ntiles && ok; ++t) {
@@ -556,7 +664,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                 rc.dbias_row = smem0 + kOffDBias + 4 * (warp * kDBiasFloats + c0) - coloff_i;
                 rc.scratch = smem0 + kOffDBias + 4 * (warp * kDBiasFloats + kDBiasEntries + lane);
                 for (int b = 0; b < x.nblk; ++b) {
-                    const int j = t * x.nblk + b, buf = j & 1;
+                    const int buf = J & 1;
                     const int nsteps = min(CB, x.npad - b * CB) >> 4;
                     const bool has_a = h < nsteps, has_b = h + 2 < nsteps;
                     ok = mbar_wait_warp(bar_sdp(buf), (ph_sdp >> buf) & 1, cta_abort);
@@ -615,82 +723,20 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                     tc_fence_before();
                     fence_proxy_async();
                     mbar_arrive_warp(bar_ds(buf));
+                    ++J;
+                    if (b == 0) {
+                        ok = flush_pending();      // the previous tile's / item's read-out
+                        if (!ok) break;
+                    }
                 }
                 if (!ok) break;
-                // ---- the tile's dV (warps 0..3) / dK (warps 4..7): one 64-byte row per thread
-                const int set = n_tile & 1;
-                ok = mbar_wait_warp(bar_acc(set), (n_tile >> 1) & 1, cta_abort);
-                if (!ok) break;
+                pend_tile = t; pend_tile_s = s; pend_tile_b = x.b; pend_tile_tok = tok; pend_tile_seq = n_tile;
                 ++n_tile;
-                tc_fence_after();
-                uint32_t r[32];
-                tmem_ld32(tmem_base + lane_addr + (h == 0 ? kColDV : kColDK) + 64 * set, r);
-                tmem_ld_wait();
-                tc_fence_before();
-                mbar_arrive_warp(bar_accfree(set));
-                {
-                    const float f = h == 0 ? 1.f : out_scale;
-                    // the tile's own V (K) rows are dead now: stage the output rows there, then store whole rows
-                    unsigned char* stg = st + (h == 0 ? kOffV : kOffK) + (t * 128 + 32 * quarter) * kRowBytes;
-                    __nv_bfloat16* out = h == 0 ? dv : dk;
-#pragma unroll
-                    for (int c4 = 0; c4 < 4; ++c4) {
-                        uint4 a;
-                        a.x = pack_bf16(__uint_as_float(r[c4 * 8 + 0]) * f, __uint_as_float(r[c4 * 8 + 1]) * f);
-                        a.y = pack_bf16(__uint_as_float(r[c4 * 8 + 2]) * f, __uint_as_float(r[c4 * 8 + 3]) * f);
-                        a.z = pack_bf16(__uint_as_float(r[c4 * 8 + 4]) * f, __uint_as_float(r[c4 * 8 + 5]) * f);
-                        a.w = pack_bf16(__uint_as_float(r[c4 * 8 + 6]) * f, __uint_as_float(r[c4 * 8 + 7]) * f);
-                        *reinterpret_cast<uint4*>(stg + tile_off<kD>(lane, c4)) = a;
-                    }
-                    __syncwarp();
-#pragma unroll
-                    for (int jj = 0; jj < 4; ++jj) {
-                        const int rr = 8 * jj + (lane >> 2), c4 = lane & 3;
-                        const int tok_r = __shfl_sync(0xffffffffu, tok, rr);
-                        const uint4 a = *reinterpret_cast<const uint4*>(stg + tile_off<kD>(rr, c4));
-                        if (tok_r >= 0)
-                            *reinterpret_cast<uint4*>(out + (((size_t)x.b * HW + (size_t)tok_r) * g.heads + head) * kD + c4 * 8) = a;
-                    }
-                    __syncwarp();
-                }
             }
             if (!ok) break;
-            // ---- dQ: queries 0..127 by warps 0..3, queries 128..255 by warps 4..7
-            if (!mbar_wait_warp(bar_dq, kuse & 1, cta_abort)) break;
-            tc_fence_after();
-            const bool have_q = h * 128 < x.npad;
-            uint32_t r[32];
-            if (have_q) {
-                tmem_ld32(tmem_base + lane_addr + kColDQ + 32 * h, r);
-                tmem_ld_wait();
-            }
-            tc_fence_before();
-            mbar_arrive_warp(bar_dqfree);
-            if (have_q) {
-                const int tokq = lds_i32(st_a + kOffTok + 4 * (h * 128 + 32 * quarter + lane));
-                unsigned char* stg = st + kOffQ + (h * 128 + 32 * quarter) * kRowBytes;
-#pragma unroll
-                for (int c4 = 0; c4 < 4; ++c4) {
-                    uint4 a;
-                    a.x = pack_bf16(__uint_as_float(r[c4 * 8 + 0]) * out_scale, __uint_as_float(r[c4 * 8 + 1]) * out_scale);
-                    a.y = pack_bf16(__uint_as_float(r[c4 * 8 + 2]) * out_scale, __uint_as_float(r[c4 * 8 + 3]) * out_scale);
-                    a.z = pack_bf16(__uint_as_float(r[c4 * 8 + 4]) * out_scale, __uint_as_float(r[c4 * 8 + 5]) * out_scale);
-                    a.w = pack_bf16(__uint_as_float(r[c4 * 8 + 6]) * out_scale, __uint_as_float(r[c4 * 8 + 7]) * out_scale);
-                    *reinterpret_cast<uint4*>(stg + tile_off<kD>(lane, c4)) = a;
-                }
-                __syncwarp();
-#pragma unroll
-                for (int jj = 0; jj < 4; ++jj) {
-                    const int rr = 8 * jj + (lane >> 2), c4 = lane & 3;
-                    const int tok_r = __shfl_sync(0xffffffffu, tokq, rr);
-                    const uint4 a = *reinterpret_cast<const uint4*>(stg + tile_off<kD>(rr, c4));
-                    if (tok_r >= 0)
-                        *reinterpret_cast<uint4*>(dq + (((size_t)x.b * HW + (size_t)tok_r) * g.heads + head) * kD + c4 * 8) = a;
-                }
-                __syncwarp();
-            }
-            mbar_arrive_warp(bar_empty(s));       // this warp no longer touches the stage
+            pend_item_s = s; pend_item_b = x.b; pend_item_npad = x.npad; pend_item_use = kuse;
         }
+        if (ok) flush_pending();
     }
 
     // teardown: every role ends up here, also after an expired wait
@@ -698,7 +744,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    if (warp == kMmaWarp) tmem_dealloc(tmem_base, 512);
+    if (warp == kIssuerWarp) tmem_dealloc(tmem_base, 512);
     {
         // this CTA's table = sum of its warps' tables (fixed order), written to the CTA's slot of the workspace
         const float* tbl = reinterpret_cast<const float*>(smem + kOffDBias);
