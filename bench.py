@@ -179,8 +179,7 @@ def run_reference(args, cfg):
 # proportion to the item count, so a full launch is this figure times its items.  None = not captured.
 NCU_DRAM_BYTES_PER_ITEM = {
     "swin_fwd_tc_kernel": 63629,
-    "swin_bwd_tc_kernel<key side>": 96647,
-    "swin_bwd_tc_kernel<query side>": 81558,
+    "swin_bwd_fused_kernel": None,
 }
 
 
@@ -366,12 +365,12 @@ def main():
         peak_tf = peaks["bf16_tflops"]
         peak_bw = peaks["hbm_gbs"]
         # Algorithmic FLOP per launch of each kernel (strict convention, per allowed pair per head):
-        # forward 4d (QK^T, PV); key side 4d (dV, dK); query side 4d (dP, dQ).  The recomputed S of both
-        # backward kernels and the key side's own dP are not counted.
+        # forward 4d (QK^T, PV); one-pass backward 8d (dP, dV, dK, dQ; the recomputed S is not counted); the
+        # register-tile backward kernels 4d each (key tiles: dV, dK; query tiles: dP, dQ).
         pairs = wk["score_elements"]
         d = cfg.head_dim
         kernel_flop = {"swin_fwd_tc_kernel": 4 * d * pairs, "swin_fwd_mma_kernel": 4 * d * pairs,
-                       "swin_bwd_tc_kernel<key side>": 4 * d * pairs, "swin_bwd_tc_kernel<query side>": 4 * d * pairs,
+                       "swin_bwd_fused_kernel": 8 * d * pairs,
                        "swin_bwd_mma_kernel<key tiles>": 4 * d * pairs, "swin_bwd_mma_kernel<query tiles>": 4 * d * pairs,
                        "swin_bwd_delta_kernel": 0}
         kernels = []

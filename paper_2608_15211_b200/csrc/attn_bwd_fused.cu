@@ -164,6 +164,7 @@ __device__ __forceinline__ void rmw4_shared_f32(const uint32_t* a, const float* 
         "add.f32 t0, t0, %4;\n\tadd.f32 t1, t1, %5;\n\tadd.f32 t2, t2, %6;\n\tadd.f32 t3, t3, %7;\n\t"
         "st.shared.f32 [%0], t0;\n\tst.shared.f32 [%1], t1;\n\tst.shared.f32 [%2], t2;\n\tst.shared.f32 [%3], t3;\n\t}\n"
         ::"r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]) : "memory");
+    __syncwarp();   // later groups stay behind these stores (see rmw8_consecutive_f32)
 }
 __device__ __forceinline__ void rmw8_shared_f32(const uint32_t* a, const float* v) {
     asm volatile(
@@ -176,6 +177,28 @@ __device__ __forceinline__ void rmw8_shared_f32(const uint32_t* a, const float* 
         "st.shared.f32 [%4], t4;\n\tst.shared.f32 [%5], t5;\n\tst.shared.f32 [%6], t6;\n\tst.shared.f32 [%7], t7;\n\t}\n"
         ::"r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(a[4]), "r"(a[5]), "r"(a[6]), "r"(a[7]),
           "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]) : "memory");
+    __syncwarp();   // later groups stay behind these stores (see rmw8_consecutive_f32)
+}
+// The same for 8 consecutive entries (one address register, immediate offsets).  The warp barrier at the end
+// keeps the next group's loads behind these stores: with base + immediate addresses the assembler can see that
+// one THREAD's next loads do not touch these entries and would hoist them, but another lane's do.
+__device__ __forceinline__ void rmw8_consecutive_f32(uint32_t a, const float* v) {
+    asm volatile(
+        "{\n\t.reg .f32 t0, t1, t2, t3, t4, t5, t6, t7;\n\t"
+        "ld.shared.f32 t0, [%0];\n\tld.shared.f32 t1, [%0+4];\n\tld.shared.f32 t2, [%0+8];\n\tld.shared.f32 t3, [%0+12];\n\t"
+        "ld.shared.f32 t4, [%0+16];\n\tld.shared.f32 t5, [%0+20];\n\tld.shared.f32 t6, [%0+24];\n\tld.shared.f32 t7, [%0+28];\n\t"
+        "add.f32 t0, t0, %1;\n\tadd.f32 t1, t1, %2;\n\tadd.f32 t2, t2, %3;\n\tadd.f32 t3, t3, %4;\n\t"
+        "add.f32 t4, t4, %5;\n\tadd.f32 t5, t5, %6;\n\tadd.f32 t6, t6, %7;\n\tadd.f32 t7, t7, %8;\n\t"
+        "st.shared.f32 [%0], t0;\n\tst.shared.f32 [%0+4], t1;\n\tst.shared.f32 [%0+8], t2;\n\tst.shared.f32 [%0+12], t3;\n\t"
+        "st.shared.f32 [%0+16], t4;\n\tst.shared.f32 [%0+20], t5;\n\tst.shared.f32 [%0+24], t6;\n\tst.shared.f32 [%0+28], t7;\n\t}\n"
+        ::"r"(a), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]) : "memory");
+    __syncwarp();
+}
+template <int OFF>
+__device__ __forceinline__ float lds_f32_at(uint32_t addr) {
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1+%2];\n" : "=f"(v) : "r"(addr), "n"(OFF));
+    return v;
 }
 // mode 8 / 4: groups of 8 / 4 consecutive columns at once; else one column at a time
 __device__ __forceinline__ void dbias_add16(int mode, const uint32_t (&addr)[16], const float (&ds)[16]) {
@@ -244,6 +267,40 @@ __device__ __forceinline__ void cols16(const uint32_t (&rs)[16], const uint32_t 
         pk_p[e2] = pack_bf16(p[2 * e2], p[2 * e2 + 1]);
         pk_ds[e2] = pack_bf16(ds[2 * e2], ds[2 * e2 + 1]);
     }
+}
+
+// The same for a full 16 x 16 window without mask labels: the 16 columns [c, c + 16) are one window row, so
+// their bias codes are consecutive and every table address is one base plus an immediate offset (no per-column
+// offsets to load, no address arithmetic).  `code0x4` = 4 * bias code of column c.  Returns the shared
+// address of the first column's bias-gradient entry; the others follow 4 bytes apart.
+__device__ __forceinline__ uint32_t cols16_row(const uint32_t (&rs)[16], const uint32_t (&rp)[16], int c, int code0x4, const RowCtx& rc,
+                                               uint32_t st_a, float scale, uint32_t (&pk_p)[8], uint32_t (&pk_ds)[8], float (&ds)[16]) {
+    float l2[16], dl[16], bv[16];
+    const uint32_t bb = rc.bias_row + code0x4;
+    bv[0] = lds_f32_at<0>(bb);   bv[1] = lds_f32_at<4>(bb);   bv[2] = lds_f32_at<8>(bb);   bv[3] = lds_f32_at<12>(bb);
+    bv[4] = lds_f32_at<16>(bb);  bv[5] = lds_f32_at<20>(bb);  bv[6] = lds_f32_at<24>(bb);  bv[7] = lds_f32_at<28>(bb);
+    bv[8] = lds_f32_at<32>(bb);  bv[9] = lds_f32_at<36>(bb);  bv[10] = lds_f32_at<40>(bb); bv[11] = lds_f32_at<44>(bb);
+    bv[12] = lds_f32_at<48>(bb); bv[13] = lds_f32_at<52>(bb); bv[14] = lds_f32_at<56>(bb); bv[15] = lds_f32_at<60>(bb);
+#pragma unroll
+    for (int e4 = 0; e4 < 4; ++e4) {
+        const float4 a = lds_f4(st_a + kOffLse + 4 * (c + e4 * 4));
+        const float4 b = lds_f4(st_a + kOffDelta + 4 * (c + e4 * 4));
+        l2[e4 * 4] = a.x; l2[e4 * 4 + 1] = a.y; l2[e4 * 4 + 2] = a.z; l2[e4 * 4 + 3] = a.w;
+        dl[e4 * 4] = b.x; dl[e4 * 4 + 1] = b.y; dl[e4 * 4 + 2] = b.z; dl[e4 * 4 + 3] = b.w;
+    }
+    float p[16];
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
+        const float xv = fmaf(__uint_as_float(rs[e]), scale, bv[e]) - l2[e];
+        p[e] = fast_exp2(xv);
+        ds[e] = p[e] * (__uint_as_float(rp[e]) - dl[e]);
+    }
+#pragma unroll
+    for (int e2 = 0; e2 < 8; ++e2) {
+        pk_p[e2] = pack_bf16(p[2 * e2], p[2 * e2 + 1]);
+        pk_ds[e2] = pack_bf16(ds[2 * e2], ds[2 * e2 + 1]);
+    }
+    return rc.dbias_row + code0x4;
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -654,6 +711,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                 // issued together.  Other windows are updated one query at a time.
                 int rmw_mode = 1;
                 if (x.r.ew == g.w && (32 % g.w) == 0 && g.w >= 4) rmw_mode = (M == 8 && g.w >= 8) ? 8 : 4;
+                const bool row16 = g.w == 16 && x.r.n == 256 && !x.masked;    // full 16 x 16 window: update groups of 8 apply as well
                 const int coloff_i = lds_i32(st_a + kOffColOff + 4 * slot);
                 const int tok = lds_i32(st_a + kOffTok + 4 * slot);
                 RowCtx rc;
@@ -677,7 +735,25 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                     uint32_t sa[16], pa[16], pk_p[8], pk_dsa[8], pk_dsb[8], addr[16];
                     float ds[16];
                     const int ca = b * CB + 16 * h, cb2 = ca + 32;
-                    if (has_a) {
+                    if (row16) {
+                        // full 16 x 16 window (four steps per block, no mask): one window row per step
+                        tmem_ld16(t_s + 16 * h, sa);
+                        tmem_ld16(t_dp + 16 * h, pa);
+                        tmem_ld_wait();
+                        uint32_t a0 = cols16_row(sa, pa, ca, 4 * cs * (ca >> 4), rc, st_a, scale, pk_p, pk_dsa, ds);
+                        tmem_st8(t_s + 16 * h, pk_p);
+                        tmem_st8(t_dp + 16 * h, pk_dsa);
+                        tmem_ld16(t_s + 16 * (h + 2), sa);
+                        tmem_ld16(t_dp + 16 * (h + 2), pa);
+                        rmw8_consecutive_f32(a0, &ds[0]);
+                        rmw8_consecutive_f32(a0 + 32, &ds[8]);
+                        tmem_ld_wait();
+                        a0 = cols16_row(sa, pa, cb2, 4 * cs * (cb2 >> 4), rc, st_a, scale, pk_p, pk_dsb, ds);
+                        tmem_st8(t_s + 16 * (h + 2), pk_p);
+                        tmem_st8(t_dp + 16 * (h + 2), pk_dsb);
+                        rmw8_consecutive_f32(a0, &ds[0]);
+                        rmw8_consecutive_f32(a0 + 32, &ds[8]);
+                    } else if (has_a) {
                         tmem_ld16(t_s + 16 * h, sa);
                         tmem_ld16(t_dp + 16 * h, pa);
                         tmem_ld_wait();
@@ -692,7 +768,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                         }
                         dbias_add16(rmw_mode, addr, ds);
                     }
-                    if (has_b) {
+                    if (has_b && !row16) {
                         tmem_ld_wait();
                         if (x.masked) cols16<true, true>(sa, pa, cb2, rc, st_a, scale, pk_p, pk_dsb, ds, addr);
                         else if (x.ragged) cols16<false, true>(sa, pa, cb2, rc, st_a, scale, pk_p, pk_dsb, ds, addr);
