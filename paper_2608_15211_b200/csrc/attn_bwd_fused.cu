@@ -30,14 +30,11 @@ namespace {
 
 using namespace tc;
 
-// Roles by role number; the role of a hardware warp is (warp + 8) mod 12, so that the MMA issuer is hardware
-// warp 0: it shares a scheduler with two elementwise warps that are rarely stalled, and as a late warp it
-// was given an issue slot only every few dozen cycles.
-constexpr int kIssuerWarp = 8;      // role 8: MMA issuer (also owns the TMEM allocation)
-constexpr int kLoaderWarp0 = 9;     // roles 9..11: loaders
+constexpr int kIssuerWarp = 8;      // warp 8: MMA issuer (also owns the TMEM allocation)
+constexpr int kLoaderWarp0 = 9;     // warps 9..11: loaders
 constexpr int kLoaderWarps = 3;
 constexpr int kLoaderThreads = kLoaderWarps * 32;
-constexpr int kThreads = (kLoaderWarp0 + kLoaderWarps) * 32;   // 384 = three warpgroups
+constexpr int kThreads = 12 * 32;                               // 384 = three warpgroups
 constexpr int kWorkWarps = 8;              // elementwise warps; each arrives once per barrier phase
 constexpr int kRegsLaunch = 168;
 constexpr int kRegsWork = 216;      // elementwise warpgroups after setmaxnreg.inc
@@ -326,7 +323,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
     volatile int* cta_abort = reinterpret_cast<volatile int*>(tail + 8);
 
     const int tid = threadIdx.x, lane = tid & 31;
-    const int warp = ((tid >> 5) + 8) % 12;      // role number (see the constants above)
+    const int warp = tid >> 5;                   // role number = hardware warp
     const int head = blockIdx.x % g.heads;
     const int cta_in_head = blockIdx.x / g.heads;
 
@@ -368,9 +365,9 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
     const size_t HW = (size_t)g.H * g.W;
 
     if (warp >= kIssuerWarp) {
-    // hardware warps 0..3 = one warpgroup (issuer + loaders) give registers back: one instruction for the whole warpgroup
+    // warpgroup 2 (issuer + loaders) gives registers back: one instruction for the whole warpgroup
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kRegsOther));
-    if (warp >= kLoaderWarp0) {
+    if (warp != kIssuerWarp) {
         // ------------------------------------------------------------------ loaders
         const int lt = (warp - kLoaderWarp0) * 32 + lane;
         int kuse = 0, pending_s = -1;

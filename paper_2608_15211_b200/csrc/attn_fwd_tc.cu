@@ -256,7 +256,8 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail);
     volatile int* cta_abort = reinterpret_cast<volatile int*>(tail + 8);
 
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int warp = tid >> 5;
 
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -291,7 +292,7 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kRegsOther));
     if (warp >= kLoaderWarp0) {
         // ------------------------------------------------------------------ loaders
-        const int lt = tid - kLoaderWarp0 * 32;
+        const int lt = (warp - kLoaderWarp0) * 32 + lane;
         int kuse = 0, pending_s = -1;
         for (long long it = blockIdx.x; it < n_items; it += gridDim.x, ++kuse) {
             const int s = kuse % kStages;
@@ -374,11 +375,18 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
                 mma_commit(bar_sready(t));
             };
             // O += P V over key steps [ks0, ks1) of 16 keys; P of step ks sits at TMEM column p_col(ks / 2) + 8 (ks & 1)
+            const uint32_t d_hi = sdesc_hi(make_sdesc_sw64(smem0, 512));
             auto issue_pv = [&](const Item& x, int s, int t, int ks0, int ks1) {
-                const uint32_t va = smem0 + s * kStageBytes + kOffV;
-                for (int ks = ks0; ks < ks1; ++ks)
-                    mma_ts(tmem_base + t * 256 + kColO, tmem_base + t * 256 + p_col(ks >> 1) + 8 * (ks & 1),
-                           make_sdesc_sw64(va + ks * 16 * kRowBytes, 512), idesc_pv, ks > 0 ? 1u : 0u);
+                // descriptor low word = start address in 16-byte units; one key step = 16 rows of 64 bytes
+                const uint32_t v_lo = sdesc_lo(make_sdesc_sw64(smem0 + s * kStageBytes + kOffV, 512));
+                const uint32_t t_o = tmem_base + t * 256 + kColO, t_p = tmem_base + t * 256;
+                int ks = ks0;
+                if (ks == 0 && ks < ks1) {
+                    mma_ts_h<false>(t_o, t_p + p_col(0), v_lo, d_hi, idesc_pv);
+                    ks = 1;
+                }
+                for (; ks < ks1; ++ks)
+                    mma_ts_h<true>(t_o, t_p + p_col(ks >> 1) + 8 * (ks & 1), v_lo + 64 * ks, d_hi, idesc_pv);
             };
             long long it = blockIdx.x;
             Item cur;
@@ -448,7 +456,7 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
         // ------------------------------------------------------------------ softmax warpgroups
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(kRegsSoftmax));
         const int wg = warp >> 2;
-        const int row = tid & 127;
+        const int row = (warp & 3) * 32 + lane;
         const int slot = wg * 128 + row;
         const uint32_t lane_addr = ((uint32_t)(32 * (warp & 3))) << 16;
         const uint32_t t_s = tmem_base + lane_addr + wg * 256;
