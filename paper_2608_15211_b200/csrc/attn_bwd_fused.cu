@@ -275,9 +275,8 @@ __device__ __forceinline__ void cols16(const uint32_t (&rs)[16], const uint32_t 
 // their bias codes are consecutive and every table address is one base plus an immediate offset (no per-column
 // offsets to load, no address arithmetic).  `code0x4` = 4 * bias code of column c.  Returns the shared
 // address of the first column's bias-gradient entry; the others follow 4 bytes apart.
-__device__ __forceinline__ uint32_t cols16_row(const uint32_t (&rs)[16], const uint32_t (&rp)[16], int c, int code0x4, const RowCtx& rc,
-                                               uint32_t st_a, float scale, uint32_t (&pk_p)[8], uint32_t (&pk_ds)[8], float (&ds)[16]) {
-    float l2[16], dl[16], bv[16];
+__device__ __forceinline__ void load16_row(int c, int code0x4, const RowCtx& rc, uint32_t st_a, float (&bv)[16], float (&l2)[16],
+                                           float (&dl)[16]) {
     const uint32_t bb = rc.bias_row + code0x4;
     bv[0] = lds_f32_at<0>(bb);   bv[1] = lds_f32_at<4>(bb);   bv[2] = lds_f32_at<8>(bb);   bv[3] = lds_f32_at<12>(bb);
     bv[4] = lds_f32_at<16>(bb);  bv[5] = lds_f32_at<20>(bb);  bv[6] = lds_f32_at<24>(bb);  bv[7] = lds_f32_at<28>(bb);
@@ -290,6 +289,9 @@ __device__ __forceinline__ uint32_t cols16_row(const uint32_t (&rs)[16], const u
         l2[e4 * 4] = a.x; l2[e4 * 4 + 1] = a.y; l2[e4 * 4 + 2] = a.z; l2[e4 * 4 + 3] = a.w;
         dl[e4 * 4] = b.x; dl[e4 * 4 + 1] = b.y; dl[e4 * 4 + 2] = b.z; dl[e4 * 4 + 3] = b.w;
     }
+}
+__device__ __forceinline__ void math16_row(const uint32_t (&rs)[16], const uint32_t (&rp)[16], const float (&bv)[16], const float (&l2)[16],
+                                           const float (&dl)[16], float scale, uint32_t (&pk_p)[8], uint32_t (&pk_ds)[8], float (&ds)[16]) {
     float p[16];
 #pragma unroll
     for (int e = 0; e < 16; ++e) {
@@ -302,7 +304,6 @@ __device__ __forceinline__ uint32_t cols16_row(const uint32_t (&rs)[16], const u
         pk_p[e2] = pack_bf16(p[2 * e2], p[2 * e2 + 1]);
         pk_ds[e2] = pack_bf16(ds[2 * e2], ds[2 * e2 + 1]);
     }
-    return rc.dbias_row + code0x4;
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -742,15 +743,21 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                         tmem_ld16(t_s + 16 * h, sa);
                         tmem_ld16(t_dp + 16 * h, pa);
                         tmem_ld_wait();
-                        uint32_t a0 = cols16_row(sa, pa, ca, 4 * cs * (ca >> 4), rc, st_a, scale, pk_p, pk_dsa, ds);
+                        float bv[16], l2[16], dl[16];
+                        const int code_a = 4 * cs * (ca >> 4), code_b = 4 * cs * (cb2 >> 4);
+                        load16_row(ca, code_a, rc, st_a, bv, l2, dl);
+                        math16_row(sa, pa, bv, l2, dl, scale, pk_p, pk_dsa, ds);
+                        uint32_t a0 = rc.dbias_row + code_a;
                         tmem_st8(t_s + 16 * h, pk_p);
                         tmem_st8(t_dp + 16 * h, pk_dsa);
                         tmem_ld16(t_s + 16 * (h + 2), sa);
                         tmem_ld16(t_dp + 16 * (h + 2), pa);
+                        load16_row(cb2, code_b, rc, st_a, bv, l2, dl);       // the second step's table values, in flight during the updates
                         rmw8_consecutive_f32(a0, &ds[0]);
                         rmw8_consecutive_f32(a0 + 32, &ds[8]);
                         tmem_ld_wait();
-                        a0 = cols16_row(sa, pa, cb2, 4 * cs * (cb2 >> 4), rc, st_a, scale, pk_p, pk_dsb, ds);
+                        math16_row(sa, pa, bv, l2, dl, scale, pk_p, pk_dsb, ds);
+                        a0 = rc.dbias_row + code_b;
                         tmem_st8(t_s + 16 * (h + 2), pk_p);
                         tmem_st8(t_dp + 16 * (h + 2), pk_dsb);
                         rmw8_consecutive_f32(a0, &ds[0]);

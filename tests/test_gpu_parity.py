@@ -23,6 +23,9 @@ EDGE = [
     ("w32_d32", 1, 40, 70, 1, 32, 32, 16, 16, 0, 1),
     ("w20_d64", 2, 45, 50, 2, 64, 20, 10, 10, 0, 1),
     ("shift_ge_grid", 1, 12, 16, 2, 32, 4, 12 + 2, 16 * 3 + 1, 0, 1),
+    ("w12_three_blocks", 2, 30, 40, 3, 32, 12, 6, 6, 0, 1),     # 144-token windows: two key tiles, an odd number of query blocks
+    ("w16_wrap_and_rem", 1, 40, 48, 2, 32, 16, 8, 8, 0, 1),      # full, masked (latitude wrap) and truncated 16-wide windows
+    ("w8_nonperiodic", 2, 24, 40, 2, 32, 8, 4, 4, 0, 0),         # 64-token windows, masks on both axes, several items per CTA
 ]
 
 
