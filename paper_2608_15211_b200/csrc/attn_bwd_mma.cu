@@ -290,12 +290,40 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
                             stage[(gq + 8 * (e >> 1)) * (BN + 1) + nt * 8 + 2 * tq + (e & 1)] = acc_dp[nt][e];
                     }
                     __syncwarp();
-                    const int code_c0 = meta_code(s_meta[blk * BN + lane]), code_c1 = meta_code(s_meta[blk * BN + lane + 32]);
-                    for (int rr = 0; rr < 16; ++rr) {
-                        const int code_r = meta_code(s_meta[r0 + warp * 16 + rr]) + c0;
-                        const float v0 = stage[rr * (BN + 1) + lane], v1 = stage[rr * (BN + 1) + lane + 32];
-                        if (v0 != 0.f) atomicAdd(&s_dbias[code_r - code_c0], v0);
-                        if (v1 != 0.f) atomicAdd(&s_dbias[code_r - code_c1], v1);
+                    if (g.w == 32 && r.ew == 32) {
+                        // Full-width 32-wide window: the warp's 16 rows are consecutive offsets b_q of one window row
+                        // a_q, and each 32-column half of the block is one window row a_k of keys with b_k = 0..31.
+                        // All pairs of a half with the same b_q - b_k share one table entry: sum each of the 47
+                        // diagonals first (lane j and lane j + 32 take diagonal j), then one atomic per diagonal
+                        // instead of one per pair.
+                        const int slot0 = r0 + warp * 16;
+                        const int a_q = slot0 >> 5, bq0 = slot0 & 31;
+#pragma unroll
+                        for (int half = 0; half < 2; ++half) {
+                            const int a_k = 2 * blk + half;
+                            const int row_base = (a_q - a_k) * (2 * g.w - 1) + c0;
+#pragma unroll
+                            for (int jj = 0; jj < 2; ++jj) {
+                                const int j = lane + 32 * jj;              // diagonal: b_q - b_k = bq0 - 31 + j
+                                if (j < 47) {
+                                    float sum = 0.f;
+#pragma unroll
+                                    for (int rr = 0; rr < 16; ++rr) {
+                                        const int bk = 31 - j + rr;
+                                        if (bk >= 0 && bk < 32) sum += stage[rr * (BN + 1) + half * 32 + bk];
+                                    }
+                                    if (sum != 0.f) atomicAdd(&s_dbias[row_base + bq0 - 31 + j], sum);
+                                }
+                            }
+                        }
+                    } else {
+                        const int code_c0 = meta_code(s_meta[blk * BN + lane]), code_c1 = meta_code(s_meta[blk * BN + lane + 32]);
+                        for (int rr = 0; rr < 16; ++rr) {
+                            const int code_r = meta_code(s_meta[r0 + warp * 16 + rr]) + c0;
+                            const float v0 = stage[rr * (BN + 1) + lane], v1 = stage[rr * (BN + 1) + lane + 32];
+                            if (v0 != 0.f) atomicAdd(&s_dbias[code_r - code_c0], v0);
+                            if (v1 != 0.f) atomicAdd(&s_dbias[code_r - code_c1], v1);
+                        }
                     }
                     __syncwarp();
                 }
