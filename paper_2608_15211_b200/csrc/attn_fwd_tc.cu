@@ -56,7 +56,12 @@ constexpr int kOffRowMeta = kOffKlab + kMaxSlots * 4;          // per query slot
 constexpr int kOffRowTok = kOffRowMeta + kMaxSlots * 4;        // grid token of the slot, -1 if none
 constexpr int kStageBytes = ((kOffRowTok + kMaxSlots * 4 + 1023) / 1024) * 1024;
 constexpr int kBarBytes = 256;
-constexpr int kSmemBytes = kStages * kStageBytes + kBarBytes;
+// After the stages and barriers: a constant block that extends V by 16 columns of ones (256 key rows x 64 bytes
+// in the operand layout, the first 16 bf16 of a row = 1).  O = P V then carries the row sums of the bf16 P in
+// its columns 32..47, and the softmax threads need not add them up.
+constexpr int kOffOnes = kStages * kStageBytes + 1024;
+constexpr int kSmemBytes = kOffOnes + kMaxSlots * kRowBytes;
+constexpr int kNO = kD + 16;                                   // columns of the O accumulator
 
 // TMEM columns inside a query tile's 256-column region once S is being consumed: bf16 P of keys 0..127 in
 // [0, 64), the O accumulator in [64, 96) (S columns that the first half of pass 2 has already read), bf16
@@ -274,6 +279,12 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
         *cta_abort = 0;
         fence_barrier_init();
     }
+    for (int i = tid; i < kMaxSlots * 4; i += kThreads) {          // (row, 16-byte chunk): chunks 0, 1 = ones, 2, 3 = zeros
+        const int row = i >> 2, chunk = i & 3;
+        const uint32_t val = chunk < 2 ? 0x3F803F80u : 0u;
+        *reinterpret_cast<uint4*>(smem + kOffOnes + tile_off<kD>(row, chunk)) = make_uint4(val, val, val, val);
+    }
+    fence_proxy_async();
     if (warp == kMmaWarp) {
         tmem_alloc(smem_u32(tmem_slot), 512);
         tmem_relinquish();
@@ -361,7 +372,7 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
     } else {
         // ------------------------------------------------------------------ MMA issuer (one lane)
         if (lane == 0) {
-            const uint32_t idesc_pv = make_idesc_bf16(128, kD, 0, 1);
+            const uint32_t idesc_pv = make_idesc_bf16(128, kNO, 0, 1);   // B = [V | ones]: 32 + 16 columns
             int kuse = 0, use_t[2] = {0, 0}, freed_t[2] = {0, 0};   // uses begun / s_free phases consumed
             bool ok = true;
             auto issue_qk = [&](const Item& x, int s, int t) {
@@ -378,7 +389,8 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
             const uint32_t d_hi = sdesc_hi(make_sdesc_sw64(smem0, 512));
             auto issue_pv = [&](const Item& x, int s, int t, int ks0, int ks1) {
                 // descriptor low word = start address in 16-byte units; one key step = 16 rows of 64 bytes
-                const uint32_t v_lo = sdesc_lo(make_sdesc_sw64(smem0 + s * kStageBytes + kOffV, 512));
+                // the second 32-column group of B (the ones block) lies one leading-dimension stride behind V
+                const uint32_t v_lo = sdesc_lo(make_sdesc_sw64_mn(smem0 + s * kStageBytes + kOffV, kOffOnes - (s * kStageBytes + kOffV), 512));
                 const uint32_t t_o = tmem_base + t * 256 + kColO, t_p = tmem_base + t * 256;
                 int ks = ks0;
                 if (ks == 0 && ks < ks1) {
@@ -485,14 +497,16 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
             mbar_arrive(bar_pready(wg));
 
             const size_t row_off = ((size_t)x.b * HW + (size_t)(tok < 0 ? 0 : tok)) * g.heads + x.head;
-            if (tok >= 0) lse[row_off] = (m + log2f(sum)) * kLn2;
-            const float inv = 1.f / sum;
 
             if (!__all_sync(0xffffffffu, mbar_wait(bar_oready(wg), use & 1, cta_abort))) break;
             tc_fence_after();
-            uint32_t ro[32];
+            uint32_t ro[32], rsum;
             tmem_ld32(t_s + kColO, ro);
+            tmem_ld1(t_s + kColO + kD, rsum);       // row sum of P (as rounded to bf16), from the ones columns
             tmem_ld_wait();
+            sum = __uint_as_float(rsum);
+            if (tok >= 0) lse[row_off] = (m + log2f(sum)) * kLn2;
+            const float inv = 1.f / sum;
             tc_fence_before();
             mbar_arrive(bar_sfree(wg));
             ++use;
