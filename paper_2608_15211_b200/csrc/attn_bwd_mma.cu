@@ -134,7 +134,7 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
     unsigned char* s_c1 = s_r2 + TILE_BYTES;          // two stages
     unsigned char* s_c2 = s_c1 + 2 * TILE_BYTES;      // two stages
     float* s_acc = reinterpret_cast<float*>(s_c2 + 2 * TILE_BYTES);   // 64 x acc_stride image of summed dS (query tiles only)
-    float* s_stage = s_acc + BM * acc_stride;                         // 4 warps x 16 x (BN + 1) staging tile (query tiles only)
+    float* s_stage = s_acc + BM * acc_stride;                         // 4 warps x 16 x 33 staging tile (query tiles only)
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int gq = lane >> 2, tq = lane & 3;
@@ -282,24 +282,24 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
                     // The warp's 16 x 64 dS tile goes through a staging tile so that one atomic instruction
                     // covers 32 consecutive columns of one row: 32 different table entries, no retries inside
                     // the warp (in the MMA fragment layout a warp instruction hits only 14 distinct entries).
-                    float* stage = s_stage + warp * 16 * (BN + 1);
+                    // The staging tile holds 32 columns: the block's two halves go through it one after the other.
+                    float* stage = s_stage + warp * 16 * 33;
+                    const int slot0 = r0 + warp * 16;
 #pragma unroll
-                    for (int nt = 0; nt < BN / 8; ++nt) {
+                    for (int half = 0; half < 2; ++half) {
 #pragma unroll
-                        for (int e = 0; e < 4; ++e)
-                            stage[(gq + 8 * (e >> 1)) * (BN + 1) + nt * 8 + 2 * tq + (e & 1)] = acc_dp[nt][e];
-                    }
-                    __syncwarp();
-                    if (g.w == 32 && r.ew == 32) {
-                        // Full-width 32-wide window: the warp's 16 rows are consecutive offsets b_q of one window row
-                        // a_q, and each 32-column half of the block is one window row a_k of keys with b_k = 0..31.
-                        // All pairs of a half with the same b_q - b_k share one table entry: sum each of the 47
-                        // diagonals first (lane j and lane j + 32 take diagonal j), then one atomic per diagonal
-                        // instead of one per pair.
-                        const int slot0 = r0 + warp * 16;
-                        const int a_q = slot0 >> 5, bq0 = slot0 & 31;
+                        for (int nt = 4 * half; nt < 4 * half + 4; ++nt) {
 #pragma unroll
-                        for (int half = 0; half < 2; ++half) {
+                            for (int e = 0; e < 4; ++e)
+                                stage[(gq + 8 * (e >> 1)) * 33 + (nt - 4 * half) * 8 + 2 * tq + (e & 1)] = acc_dp[nt][e];
+                        }
+                        __syncwarp();
+                        if (g.w == 32 && r.ew == 32) {
+                            // Full-width 32-wide window: the warp's 16 rows are consecutive offsets b_q of one window row
+                            // a_q, and this half of the block is one window row a_k of keys with b_k = 0..31.  All pairs
+                            // with the same b_q - b_k share one table entry: sum each of the 47 diagonals first (lane j
+                            // and lane j + 32 take diagonal j), then one atomic per diagonal instead of one per pair.
+                            const int a_q = slot0 >> 5, bq0 = slot0 & 31;
                             const int a_k = 2 * blk + half;
                             const int row_base = (a_q - a_k) * (2 * g.w - 1) + c0;
 #pragma unroll
@@ -310,22 +310,21 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
 #pragma unroll
                                     for (int rr = 0; rr < 16; ++rr) {
                                         const int bk = 31 - j + rr;
-                                        if (bk >= 0 && bk < 32) sum += stage[rr * (BN + 1) + half * 32 + bk];
+                                        if (bk >= 0 && bk < 32) sum += stage[rr * 33 + bk];
                                     }
                                     if (sum != 0.f) atomicAdd(&s_dbias[row_base + bq0 - 31 + j], sum);
                                 }
                             }
+                        } else {
+                            const int code_c = meta_code(s_meta[blk * BN + half * 32 + lane]);
+                            for (int rr = 0; rr < 16; ++rr) {
+                                const int code_r = meta_code(s_meta[slot0 + rr]) + c0;
+                                const float v0 = stage[rr * 33 + lane];
+                                if (v0 != 0.f) atomicAdd(&s_dbias[code_r - code_c], v0);
+                            }
                         }
-                    } else {
-                        const int code_c0 = meta_code(s_meta[blk * BN + lane]), code_c1 = meta_code(s_meta[blk * BN + lane + 32]);
-                        for (int rr = 0; rr < 16; ++rr) {
-                            const int code_r = meta_code(s_meta[r0 + warp * 16 + rr]) + c0;
-                            const float v0 = stage[rr * (BN + 1) + lane], v1 = stage[rr * (BN + 1) + lane + 32];
-                            if (v0 != 0.f) atomicAdd(&s_dbias[code_r - code_c0], v0);
-                            if (v1 != 0.f) atomicAdd(&s_dbias[code_r - code_c1], v1);
-                        }
+                        __syncwarp();
                     }
-                    __syncwarp();
                 }
             }
             if constexpr (KV) {
@@ -407,7 +406,7 @@ size_t bwd_smem_bytes(const Geo& g, bool query_side) {
     int npad_max = ((g.nmax + BN - 1) / BN) * BN;
     int nbias = (2 * g.w - 1) * (2 * g.w - 1);
     size_t head = (((size_t)npad_max * 16 + (size_t)nbias * 8 + 127) / 128) * 128;
-    size_t acc = query_side ? ((size_t)BM * acc_stride_for(g) + (size_t)BM * (BN + 1)) * sizeof(float) : 0;
+    size_t acc = query_side ? ((size_t)BM * acc_stride_for(g) + (size_t)BM * 33) * sizeof(float) : 0;
     return head + 6 * (size_t)BN * g.d * 2 + acc;
 }
 
