@@ -40,7 +40,7 @@ constexpr int kLoaderWarp0 = 9;     // warps 9..11: loaders
 constexpr int kLoaderWarps = 3;
 constexpr int kLoaderThreads = kLoaderWarps * 32;
 constexpr int kThreads = 12 * 32;                               // 384 = three warpgroups
-constexpr int kWorkWarps = 8;              // elementwise warps; each arrives once per barrier phase
+constexpr int kWorkThreads = 256;          // elementwise threads; each arrives once per barrier phase
 constexpr int kRegsLaunch = 168;
 constexpr int kRegsWork = 216;      // elementwise warpgroups after setmaxnreg.inc
 constexpr int kRegsOther = 72;      // MMA + loader warpgroup after setmaxnreg.dec
@@ -336,17 +336,17 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(bar_full(s), kLoaderThreads);
-            mbar_init(bar_empty(s), kWorkWarps);
+            mbar_init(bar_empty(s), kWorkThreads);
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar_sdp(b), 1);
-            mbar_init(bar_ds(b), kWorkWarps);
+            mbar_init(bar_ds(b), kWorkThreads);
             mbar_init(bar_acc(b), 1);
-            mbar_init(bar_accfree(b), kWorkWarps);
+            mbar_init(bar_accfree(b), kWorkThreads);
         }
         mbar_init(bar_dsfree, 1);
         mbar_init(bar_dq, 1);
-        mbar_init(bar_dqfree, kWorkWarps);
+        mbar_init(bar_dqfree, kWorkThreads);
         *cta_abort = 0;
         fence_barrier_init();
     }
@@ -386,7 +386,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                 mbar_arrive(bar_full(pending_s));
                 pending_s = -1;
             }
-            if (!mbar_wait_warp(bar_empty(s), ((kuse / kStages) & 1) ^ 1, cta_abort)) break;
+            if (!mbar_wait_all(bar_empty(s), ((kuse / kStages) & 1) ^ 1, cta_abort)) break;
             const Item x = make_item(g, it);
             unsigned char* st = smem + s * kStageBytes;
             const uint32_t st_a = smem0 + s * kStageBytes;
@@ -507,7 +507,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                 nb_n = xn.ntiles * xn.nblk; npad_n = xn.npad; nblk_n = xn.nblk;
             }
             const int J0 = J;
-            ok = mbar_wait_warp(bar_full(s), (kuse / kStages) & 1, cta_abort);
+            ok = mbar_wait_all(bar_full(s), (kuse / kStages) & 1, cta_abort);
             if (!ok) break;
             fence_proxy_async();
             tc_fence_after();
@@ -521,7 +521,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                     } else {
                         local -= nb;
                         const int sn = (kuse + 1) % kStages;
-                        if (!mbar_wait_warp(bar_full(sn), ((kuse + 1) / kStages) & 1, cta_abort)) return false;
+                        if (!mbar_wait_all(bar_full(sn), ((kuse + 1) / kStages) & 1, cta_abort)) return false;
                         fence_proxy_async();
                         const int t = local >= nblk_n ? 1 : 0;
                         issue_sdp(sn, npad_n, t, local - t * nblk_n, jt & 1);
@@ -537,10 +537,10 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                 for (int b = 0; b < nblk; ++b, ++J) {
                     const int buf = J & 1;
                     const int nks = min(CB, npad - b * CB) >> 4;
-                    ok = mbar_wait_warp(bar_ds(buf), (ph_ds >> buf) & 1, cta_abort);          // all eight warps are done with block J
+                    ok = mbar_wait_all(bar_ds(buf), (ph_ds >> buf) & 1, cta_abort);          // all eight warps are done with block J
                     ph_ds ^= 1u << buf;
                     if (ok && b == 0 && n_tile >= 2)     // the accumulator set must have been read back (tile n_tile - 2)
-                        ok = mbar_wait_warp(bar_accfree(set), ((n_tile >> 1) - 1) & 1, cta_abort);
+                        ok = mbar_wait_all(bar_accfree(set), ((n_tile >> 1) - 1) & 1, cta_abort);
                     if (!ok) break;
                     tc_fence_after();
                     // dV += P^T dO, dK += dS^T Q over the block's query columns
@@ -576,7 +576,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                     if ((b & 1) || b == nblk - 1) {
                         // dQ (queries of this pair of blocks) += dS K over the tile's keys
                         if (t == 0 && b < 2 && kuse > 0) {   // the item's first write of dQ: the previous item's was read
-                            ok = mbar_wait_warp(bar_dqfree, (kuse - 1) & 1, cta_abort);
+                            ok = mbar_wait_all(bar_dqfree, (kuse - 1) & 1, cta_abort);
                             if (!ok) break;
                             tc_fence_after();
                         }
@@ -621,13 +621,13 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
             if (pend_tile >= 0) {
                 // ---- the tile's dV (warps 0..3) / dK (warps 4..7): one 64-byte row per thread
                 const int set = pend_tile_seq & 1;
-                if (!mbar_wait_warp(bar_acc(set), (pend_tile_seq >> 1) & 1, cta_abort)) return false;
+                if (!mbar_wait_all(bar_acc(set), (pend_tile_seq >> 1) & 1, cta_abort)) return false;
                 tc_fence_after();
                 uint32_t r[32];
                 tmem_ld32(tmem_base + lane_addr + (h == 0 ? kColDV : kColDK) + 64 * set, r);
                 tmem_ld_wait();
                 tc_fence_before();
-                mbar_arrive_warp(bar_accfree(set));
+                mbar_arrive(bar_accfree(set));
                 const float f = h == 0 ? 1.f : out_scale;
                 // the tile's own V (K) rows are dead now: stage the output rows there, then store whole rows
                 unsigned char* stg = smem + pend_tile_s * kStageBytes + (h == 0 ? kOffV : kOffK) + (pend_tile * 128 + 32 * quarter) * kRowBytes;
@@ -655,7 +655,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
             }
             if (pend_item_s >= 0) {
                 // ---- dQ: queries 0..127 by warps 0..3, queries 128..255 by warps 4..7
-                if (!mbar_wait_warp(bar_dq, pend_item_use & 1, cta_abort)) return false;
+                if (!mbar_wait_all(bar_dq, pend_item_use & 1, cta_abort)) return false;
                 tc_fence_after();
                 const bool have_q = h * 128 < pend_item_npad;
                 uint32_t r[32];
@@ -664,7 +664,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                     tmem_ld_wait();
                 }
                 tc_fence_before();
-                mbar_arrive_warp(bar_dqfree);
+                mbar_arrive(bar_dqfree);
                 if (have_q) {
                     const int tokq = lds_i32(smem0 + pend_item_s * kStageBytes + kOffTok + 4 * (h * 128 + 32 * quarter + lane));
                     unsigned char* stg = smem + pend_item_s * kStageBytes + kOffQ + (h * 128 + 32 * quarter) * kRowBytes;
@@ -688,7 +688,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                     }
                     __syncwarp();
                 }
-                mbar_arrive_warp(bar_empty(pend_item_s));       // this warp no longer touches that stage
+                mbar_arrive(bar_empty(pend_item_s));       // this thread no longer touches that stage
                 pend_item_s = -1;
             }
             return true;
@@ -699,7 +699,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
             const Item x = make_item(g, it);
             const int s = kuse % kStages;
             const uint32_t st_a = smem0 + s * kStageBytes;
-            if (!mbar_wait_warp(bar_full(s), (kuse / kStages) & 1, cta_abort)) break;
+            if (!mbar_wait_all(bar_full(s), (kuse / kStages) & 1, cta_abort)) break;
             for (int t = 0; t < x.ntiles && ok; ++t) {
                 const int krow = 32 * quarter + lane;            // key row inside the tile
                 const int M = 4 * x.ntiles;
@@ -728,7 +728,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                     const int buf = J & 1;
                     const int nsteps = min(CB, x.npad - b * CB) >> 4;
                     const bool has_a = h < nsteps, has_b = h + 2 < nsteps;
-                    ok = mbar_wait_warp(bar_sdp(buf), (ph_sdp >> buf) & 1, cta_abort);
+                    ok = mbar_wait_all(bar_sdp(buf), (ph_sdp >> buf) & 1, cta_abort);
                     if (!ok) break;
                     ph_sdp ^= 1u << buf;
                     tc_fence_after();
@@ -789,7 +789,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                     // dS^T into the shared tile of this pair of blocks (32-query groups 2 (b & 1) and 2 (b & 1) + 1;
                     // step h -> group 2 (b & 1), step h + 2 -> the next group; 16-byte chunks 2 h and 2 h + 1)
                     if ((b & 1) == 0 && n_pair > 0) {
-                        ok = mbar_wait_warp(bar_dsfree, (n_pair - 1) & 1, cta_abort);
+                        ok = mbar_wait_all(bar_dsfree, (n_pair - 1) & 1, cta_abort);
                         if (!ok) break;
                     }
                     {
@@ -807,7 +807,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                     tmem_st_wait();
                     tc_fence_before();
                     fence_proxy_async();
-                    mbar_arrive_warp(bar_ds(buf));
+                    mbar_arrive(bar_ds(buf));
                     ++J;
                     if (b == 0) {
                         ok = flush_pending();      // the previous tile's / item's read-out
