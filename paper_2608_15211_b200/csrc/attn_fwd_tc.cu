@@ -55,7 +55,6 @@ constexpr int kOffKlab = kOffKc + kMaxSlots * 4;               // per key slot: 
 constexpr int kOffRowMeta = kOffKlab + kMaxSlots * 4;          // per query slot: code | label << 16
 constexpr int kOffRowTok = kOffRowMeta + kMaxSlots * 4;        // grid token of the slot, -1 if none
 constexpr int kStageBytes = ((kOffRowTok + kMaxSlots * 4 + 1023) / 1024) * 1024;
-constexpr int kBarBytes = 256;
 // After the stages and barriers: a constant block that extends V by 16 columns of ones (256 key rows x 64 bytes
 // in the operand layout, the first 16 bf16 of a row = 1).  O = P V then carries the row sums of the bf16 P in
 // its columns 32..47, and the softmax threads need not add them up.
@@ -370,8 +369,10 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
             mbar_arrive(bar_full(pending_s));
         }
     } else {
-        // ------------------------------------------------------------------ MMA issuer (one lane)
-        if (lane == 0) {
+        // ------------------------------------------------------------------ MMA issuer
+        // The whole warp runs the loop and waits (a warp whose 32 lanes wait together is parked and woken as a
+        // whole); one elected lane issues the MMAs and commits.
+        {
             const uint32_t idesc_pv = make_idesc_bf16(128, kNO, 0, 1);   // B = [V | ones]: 32 + 16 columns
             int kuse = 0, use_t[2] = {0, 0}, freed_t[2] = {0, 0};   // uses begun / s_free phases consumed
             bool ok = true;
@@ -379,11 +380,14 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
                 const uint32_t qa = smem0 + s * kStageBytes + kOffQ + t * 128 * kRowBytes;
                 const uint32_t ka = smem0 + s * kStageBytes + kOffK;
                 const uint32_t idesc = make_idesc_bf16(128, x.npad, 0, 0);
+                if (elect_one()) {
 #pragma unroll
-                for (int ks = 0; ks < kD / 16; ++ks)
-                    mma_ss(tmem_base + t * 256, make_sdesc_sw64(qa + ks * 32, 512), make_sdesc_sw64(ka + ks * 32, 512),
-                           idesc, ks > 0 ? 1u : 0u);
-                mma_commit(bar_sready(t));
+                    for (int ks = 0; ks < kD / 16; ++ks)
+                        mma_ss(tmem_base + t * 256, make_sdesc_sw64(qa + ks * 32, 512), make_sdesc_sw64(ka + ks * 32, 512),
+                               idesc, ks > 0 ? 1u : 0u);
+                    mma_commit(bar_sready(t));
+                }
+                __syncwarp();
             };
             // O += P V over key steps [ks0, ks1) of 16 keys; P of step ks sits at TMEM column p_col(ks / 2) + 8 (ks & 1)
             const uint32_t d_hi = sdesc_hi(make_sdesc_sw64(smem0, 512));
@@ -392,19 +396,22 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
                 // the second 32-column group of B (the ones block) lies one leading-dimension stride behind V
                 const uint32_t v_lo = sdesc_lo(make_sdesc_sw64_mn(smem0 + s * kStageBytes + kOffV, kOffOnes - (s * kStageBytes + kOffV), 512));
                 const uint32_t t_o = tmem_base + t * 256 + kColO, t_p = tmem_base + t * 256;
-                int ks = ks0;
-                if (ks == 0 && ks < ks1) {
-                    mma_ts_h<false>(t_o, t_p + p_col(0), v_lo, d_hi, idesc_pv);
-                    ks = 1;
+                if (elect_one()) {
+                    int ks = ks0;
+                    if (ks == 0 && ks < ks1) {
+                        mma_ts_h<false>(t_o, t_p + p_col(0), v_lo, d_hi, idesc_pv);
+                        ks = 1;
+                    }
+                    for (; ks < ks1; ++ks)
+                        mma_ts_h<true>(t_o, t_p + p_col(ks >> 1) + 8 * (ks & 1), v_lo + 64 * ks, d_hi, idesc_pv);
                 }
-                for (; ks < ks1; ++ks)
-                    mma_ts_h<true>(t_o, t_p + p_col(ks >> 1) + 8 * (ks & 1), v_lo + 64 * ks, d_hi, idesc_pv);
+                __syncwarp();
             };
             long long it = blockIdx.x;
             Item cur;
             if (it < n_items) {
                 cur = make_item(g, it);
-                ok = mbar_wait(bar_full(0), 0, cta_abort);
+                ok = mbar_wait_all(bar_full(0), 0, cta_abort);
                 if (ok) {
                     fence_proxy_async();
                     tc_fence_after();
@@ -424,7 +431,7 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
                     if (!ok || t >= cur.ntiles) continue;
-                    ok = mbar_wait(bar_phalf(t), use_t[t] & 1, cta_abort);
+                    ok = mbar_wait_all(bar_phalf(t), use_t[t] & 1, cta_abort);
                     if (!ok) continue;
                     tc_fence_after();
                     issue_pv(cur, s, t, 0, min(8, nks));
@@ -433,16 +440,19 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
                 for (int t = 0; t < 2; ++t) {
                     if (!ok) break;
                     if (t < cur.ntiles) {
-                        ok = mbar_wait(bar_pready(t), use_t[t] & 1, cta_abort);   // use_t[t] still counts earlier uses only
+                        ok = mbar_wait_all(bar_pready(t), use_t[t] & 1, cta_abort);   // use_t[t] still counts earlier uses only
                         if (!ok) break;
                         tc_fence_after();
                         issue_pv(cur, s, t, 8, nks);
-                        mma_commit(bar_oready(t));
-                        if (t == cur.ntiles - 1) mma_commit(bar_empty(s));   // all operands of this stage consumed
+                        if (elect_one()) {
+                            mma_commit(bar_oready(t));
+                            if (t == cur.ntiles - 1) mma_commit(bar_empty(s));   // all operands of this stage consumed
+                        }
+                        __syncwarp();
                     }
                     if (has_next && t < nx.ntiles) {
                         if (!next_ready) {
-                            ok = mbar_wait(bar_full(sn), ((kuse + 1) / kStages) & 1, cta_abort);
+                            ok = mbar_wait_all(bar_full(sn), ((kuse + 1) / kStages) & 1, cta_abort);
                             if (!ok) break;
                             fence_proxy_async();
                             next_ready = true;
@@ -450,7 +460,7 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
                         if (t < cur.ntiles) ++use_t[t];
                         // region t is free once its softmax warpgroup has read O of the last item that used it
                         while (ok && freed_t[t] < use_t[t]) {
-                            ok = mbar_wait(bar_sfree(t), freed_t[t] & 1, cta_abort);
+                            ok = mbar_wait_all(bar_sfree(t), freed_t[t] & 1, cta_abort);
                             ++freed_t[t];
                         }
                         if (!ok) break;
