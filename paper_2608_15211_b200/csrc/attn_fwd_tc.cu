@@ -160,6 +160,30 @@ __device__ __forceinline__ float softmax_cols(const uint32_t (&r)[N], uint32_t (
     return s0 + s1;
 }
 
+template <int OFF>
+__device__ __forceinline__ float lds_f32_at(uint32_t addr) {
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1+%2];\n" : "=f"(v) : "r"(addr), "n"(OFF));
+    return v;
+}
+// 16 key columns that are one window row of a full 16 x 16 window without mask labels: their bias entries are
+// consecutive (descending with the key), so each address is one base plus an immediate offset.  `top` = shared
+// address of the entry of the row's first key.
+__device__ __forceinline__ void softmax_cols16_row(const uint32_t* r, uint32_t* pk, uint32_t top, float scale, float neg_m) {
+    const uint32_t bb = top - 60;
+    float bv[16];
+    bv[0] = lds_f32_at<60>(bb);  bv[1] = lds_f32_at<56>(bb);  bv[2] = lds_f32_at<52>(bb);  bv[3] = lds_f32_at<48>(bb);
+    bv[4] = lds_f32_at<44>(bb);  bv[5] = lds_f32_at<40>(bb);  bv[6] = lds_f32_at<36>(bb);  bv[7] = lds_f32_at<32>(bb);
+    bv[8] = lds_f32_at<28>(bb);  bv[9] = lds_f32_at<24>(bb);  bv[10] = lds_f32_at<20>(bb); bv[11] = lds_f32_at<16>(bb);
+    bv[12] = lds_f32_at<12>(bb); bv[13] = lds_f32_at<8>(bb);  bv[14] = lds_f32_at<4>(bb);  bv[15] = lds_f32_at<0>(bb);
+#pragma unroll
+    for (int e2 = 0; e2 < 8; ++e2) {
+        const float p0 = fast_exp2(fmaf(__uint_as_float(r[2 * e2]), scale, bv[2 * e2]) + neg_m);
+        const float p1 = fast_exp2(fmaf(__uint_as_float(r[2 * e2 + 1]), scale, bv[2 * e2 + 1]) + neg_m);
+        pk[e2] = pack_bf16(p0, p1);
+    }
+}
+
 template <int N>
 __device__ __forceinline__ void max_cols(const uint32_t (&r)[N], float (&mx)[4]) {
 #pragma unroll
@@ -172,9 +196,12 @@ __device__ __forceinline__ void max_cols(const uint32_t (&r)[N], float (&mx)[4])
 
 // One softmax row: two passes over the row's S columns in TMEM, 32 columns per load, the next load in
 // flight while the current one is processed.  Returns m (log2 domain); the row sum goes to sum_out.
-template <bool MASKED>
+// ROW16: full 16 x 16 window without mask labels (npad = 256); `top0` = shared address of the bias entry of key 0
+// for this query, `row_step` = bytes between the entries of keys one window row apart.
+template <bool MASKED, bool ROW16 = false>
 __device__ __forceinline__ float softmax_row(uint32_t t_s, int npad, uint32_t bias_i, uint32_t a_kc, uint32_t a_klab,
-                                             int label_i, float scale, float bmax, float& sum_out, uint32_t bar_half) {
+                                             int label_i, float scale, float bmax, float& sum_out, uint32_t bar_half,
+                                             uint32_t top0 = 0, uint32_t row_step = 0) {
     const int nfull = npad >> 5;
     const bool tail = (npad & 16) != 0;
     uint32_t ra[32], rb[32];
@@ -215,12 +242,22 @@ __device__ __forceinline__ float softmax_row(uint32_t t_s, int npad, uint32_t bi
         uint32_t pk[16];
         tmem_ld_wait();
         if (i + 1 < nfull) tmem_ld32(t_s + 32 * (i + 1), rb);
-        sum += softmax_cols<32, MASKED>(ra, pk, 32 * i, bias_i, a_kc, a_klab, label_i, scale, neg_m);
+        if (ROW16) {
+            softmax_cols16_row(&ra[0], &pk[0], top0 - (2 * i) * row_step, scale, neg_m);
+            softmax_cols16_row(&ra[16], &pk[8], top0 - (2 * i + 1) * row_step, scale, neg_m);
+        } else {
+            sum += softmax_cols<32, MASKED>(ra, pk, 32 * i, bias_i, a_kc, a_klab, label_i, scale, neg_m);
+        }
         tmem_st16(t_s + p_col(i), pk);
         if (i + 1 < nfull) {
             tmem_ld_wait();
             if (i + 2 < nfull) tmem_ld32(t_s + 32 * (i + 2), ra);
-            sum += softmax_cols<32, MASKED>(rb, pk, 32 * (i + 1), bias_i, a_kc, a_klab, label_i, scale, neg_m);
+            if (ROW16) {
+                softmax_cols16_row(&rb[0], &pk[0], top0 - (2 * i + 2) * row_step, scale, neg_m);
+                softmax_cols16_row(&rb[16], &pk[8], top0 - (2 * i + 3) * row_step, scale, neg_m);
+            } else {
+                sum += softmax_cols<32, MASKED>(rb, pk, 32 * (i + 1), bias_i, a_kc, a_klab, label_i, scale, neg_m);
+            }
             tmem_st16(t_s + p_col(i + 1), pk);
         }
         if (i == 2 && npad > 128) {
@@ -241,6 +278,10 @@ __device__ __forceinline__ float softmax_row(uint32_t t_s, int npad, uint32_t bi
     return m;
 }
 
+// W16 = the window side is 16: full unmasked windows take the immediate-offset table addressing, every other
+// window of that grid (shift-mask labels, truncated at the grid's edge) the label-compare path, which also
+// covers key slots without a token (their label never matches).  Two softmax paths per kernel either way.
+template <bool W16>
 __global__ void __launch_bounds__(kThreads, 1)
 swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                    const __nv_bfloat16* __restrict__ v, const float* __restrict__ bias_prep,
@@ -499,8 +540,16 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
             if (!__all_sync(0xffffffffu, mbar_wait(bar_sready(wg), use & 1, cta_abort))) break;
             tc_fence_after();
             float m, sum;
-            if (x.masked) m = softmax_row<true>(t_s, x.npad, bias_i, st_a + kOffKc, st_a + kOffKlab, label_i, scale, bmax, sum, bar_phalf(wg));
-            else m = softmax_row<false>(t_s, x.npad, bias_i, st_a + kOffKc, st_a + kOffKlab, label_i, scale, bmax, sum, bar_phalf(wg));
+            if (W16) {
+                if (x.masked || x.r.n != 256)
+                    m = softmax_row<true>(t_s, x.npad, bias_i, st_a + kOffKc, st_a + kOffKlab, label_i, scale, bmax, sum, bar_phalf(wg));
+                else
+                    m = softmax_row<false, true>(t_s, x.npad, bias_i, st_a + kOffKc, st_a + kOffKlab, label_i, scale, bmax, sum, bar_phalf(wg),
+                                                 bias_i + 4 * c0, 4 * cs);
+            } else {
+                if (x.masked) m = softmax_row<true>(t_s, x.npad, bias_i, st_a + kOffKc, st_a + kOffKlab, label_i, scale, bmax, sum, bar_phalf(wg));
+                else m = softmax_row<false>(t_s, x.npad, bias_i, st_a + kOffKc, st_a + kOffKlab, label_i, scale, bmax, sum, bar_phalf(wg));
+            }
             tmem_st_wait();
             tc_fence_before();
             if (x.npad <= 128) mbar_arrive(bar_phalf(wg));      // short rows: both halves at once
@@ -593,12 +642,17 @@ cudaError_t launch_fwd_tc(const Geo& g, const void* q, const void* k, const void
     count_launch(stream);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(swin_fwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    e = cudaFuncSetAttribute(g.w == 16 ? swin_fwd_tc_kernel<true> : swin_fwd_tc_kernel<false>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
     const unsigned grid = (unsigned)(items < sm_count ? items : sm_count);
     prof_begin("swin_fwd_tc_kernel", stream);
-    swin_fwd_tc_kernel<<<grid, kThreads, kSmemBytes, stream>>>(g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k,
-                                                               (const __nv_bfloat16*)v, prep, (__nv_bfloat16*)o, lse, items);
+    if (g.w == 16)
+        swin_fwd_tc_kernel<true><<<grid, kThreads, kSmemBytes, stream>>>(g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k,
+                                                                         (const __nv_bfloat16*)v, prep, (__nv_bfloat16*)o, lse, items);
+    else
+        swin_fwd_tc_kernel<false><<<grid, kThreads, kSmemBytes, stream>>>(g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k,
+                                                                          (const __nv_bfloat16*)v, prep, (__nv_bfloat16*)o, lse, items);
     count_launch(stream);
     return cudaGetLastError();
 }
