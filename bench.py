@@ -226,6 +226,7 @@ def main():
 
     import paper_2608_15211_b200 as terra
     from paper_2608_15211_b200.accounting import work
+    from paper_2608_15211_b200.replicas import max_over_ranks, whole_job_tflops
     from paper_2608_15211_b200.build import build
     from paper_2608_15211_b200.workloads import make_activation, make_bias_table
 
@@ -319,16 +320,12 @@ def main():
         kernel_ms.setdefault(kname, []).append(kms)
     terra.profile_enable(False)
     clocks = sampler.stop()
-    total_ms = t_start.elapsed_time(t_end)
-    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms = float(t.item())
+    total_ms = max_over_ranks(t_start.elapsed_time(t_end), dev)     # the job is as slow as its slowest replica
     ms_step = total_ms / args.steps
     route_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in ev)
     fwd_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in ev)
     bwd_ms = statistics.mean(e[2].elapsed_time(e[3]) for e in ev)
-    value = world * flops / (ms_step * 1e-3) / 1e12
+    value = whole_job_tflops(flops, world, ms_step)
 
     # end to end through the C ABI from pinned HOST buffers: every step copies its inputs host -> device, runs, and
     # copies its results device -> host.  Two device buffer sets and three streams, as an application would do
@@ -387,10 +384,8 @@ def main():
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e2e_steps(n_e2e, a, b)
         barrier()
-        te = torch.tensor([a.elapsed_time(b) / n_e2e], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(te, op=dist.ReduceOp.MAX)
-        e2e = {"value": world * flops / (float(te.item()) * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": float(te.item()),
+        e2e_ms = max_over_ranks(a.elapsed_time(b) / n_e2e, dev)
+        e2e = {"value": whole_job_tflops(flops, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                "note": "pinned host buffers; H2D, kernels and D2H of consecutive steps overlap (two device buffer sets)"}
 
