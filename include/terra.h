@@ -102,8 +102,10 @@ int terra_swin_attn_fwd(const terra_swin_desc* desc, const void* q, const void* 
  *   q, k, v, o, lse   as given to / produced by the forward call
  *   d_o               bf16 [B, H, W, heads, head_dim]   upstream gradient
  *   dq, dk, dv        bf16 [B, H, W, heads, head_dim]   overwritten
- *   dbias             fp32 [(2w-1)^2, heads]            overwritten (summed over batch and windows;
- *                                                       the summation order is not fixed)
+ *   dbias             fp32 [(2w-1)^2, heads]            overwritten (summed over batch and windows; in a fixed
+ *                                                       order, hence reproducible run to run, for head_dim 32
+ *                                                       with window <= 16; with atomics, hence in no fixed
+ *                                                       order, for the other shapes)
  *   workspace         >= terra_swin_workspace_bytes(desc, 1) bytes
  */
 int terra_swin_attn_bwd(const terra_swin_desc* desc, const void* q, const void* k, const void* v,
