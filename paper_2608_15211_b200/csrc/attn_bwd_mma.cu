@@ -297,24 +297,22 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
                         if (g.w == 32 && r.ew == 32) {
                             // Full-width 32-wide window: the warp's 16 rows are consecutive offsets b_q of one window row
                             // a_q, and this half of the block is one window row a_k of keys with b_k = 0..31.  All pairs
-                            // with the same b_q - b_k share one table entry: sum each of the 47 diagonals first (lane j
-                            // and lane j + 32 take diagonal j), then one atomic per diagonal instead of one per pair.
+                            // with the same b_q - b_k share one table entry: sum each of the 47 diagonals first, then one
+                            // atomic per diagonal instead of one per pair.
                             const int a_q = slot0 >> 5, bq0 = slot0 & 31;
                             const int a_k = 2 * blk + half;
                             const int row_base = (a_q - a_k) * (2 * g.w - 1) + c0;
+                            // lane l sums diagonal l (rows rr <= l) and, for l < 15, diagonal l + 32 (rows rr > l): 16 loads
+                            // per lane cover all 47 diagonals
+                            float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-                            for (int jj = 0; jj < 2; ++jj) {
-                                const int j = lane + 32 * jj;              // diagonal: b_q - b_k = bq0 - 31 + j
-                                if (j < 47) {
-                                    float sum = 0.f;
-#pragma unroll
-                                    for (int rr = 0; rr < 16; ++rr) {
-                                        const int bk = 31 - j + rr;
-                                        if (bk >= 0 && bk < 32) sum += stage[rr * 33 + bk];
-                                    }
-                                    if (sum != 0.f) atomicAdd(&s_dbias[row_base + bq0 - 31 + j], sum);
-                                }
+                            for (int rr = 0; rr < 16; ++rr) {
+                                const bool first = rr <= lane;
+                                const float val = stage[rr * 33 + (first ? 31 - lane + rr : rr - lane - 1)];
+                                if (first) s0 += val; else s1 += val;
                             }
+                            if (s0 != 0.f) atomicAdd(&s_dbias[row_base + bq0 - 31 + lane], s0);
+                            if (lane < 15 && s1 != 0.f) atomicAdd(&s_dbias[row_base + bq0 + 1 + lane], s1);
                         } else {
                             const int code_c = meta_code(s_meta[blk * BN + half * 32 + lane]);
                             for (int rr = 0; rr < 16; ++rr) {
