@@ -109,6 +109,8 @@ __device__ __forceinline__ void scatter_rows(const unsigned char* tile, __nv_bfl
 
 // KV = true : CTA owns 64 keys   (own tiles K, V;  streams Q, dO) -> dK, dV
 // KV = false: CTA owns 64 queries (own tiles Q, dO; streams K, V) -> dQ, dBias
+constexpr int kStageStride = 40;   // floats per row of the dS staging tile (32 columns used)
+
 template <int D, bool KV>
 __global__ void __launch_bounds__(NTHREADS)
 swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
@@ -134,7 +136,7 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
     unsigned char* s_c1 = s_r2 + TILE_BYTES;          // two stages
     unsigned char* s_c2 = s_c1 + 2 * TILE_BYTES;      // two stages
     float* s_acc = reinterpret_cast<float*>(s_c2 + 2 * TILE_BYTES);   // 64 x acc_stride image of summed dS (query tiles only)
-    float* s_stage = s_acc + BM * acc_stride;                         // 4 warps x 16 x 33 staging tile (query tiles only)
+    float* s_stage = s_acc + BM * acc_stride;                         // 4 warps x 16 x kStageStride staging tile (query tiles only)
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int gq = lane >> 2, tq = lane & 3;
@@ -283,15 +285,16 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
                     // covers 32 consecutive columns of one row: 32 different table entries, no retries inside
                     // the warp (in the MMA fragment layout a warp instruction hits only 14 distinct entries).
                     // The staging tile holds 32 columns: the block's two halves go through it one after the other.
-                    float* stage = s_stage + warp * 16 * 33;
+                    float* stage = s_stage + warp * 16 * kStageStride;
                     const int slot0 = r0 + warp * 16;
 #pragma unroll
                     for (int half = 0; half < 2; ++half) {
 #pragma unroll
                         for (int nt = 4 * half; nt < 4 * half + 4; ++nt) {
-#pragma unroll
-                            for (int e = 0; e < 4; ++e)
-                                stage[(gq + 8 * (e >> 1)) * 33 + (nt - 4 * half) * 8 + 2 * tq + (e & 1)] = acc_dp[nt][e];
+                            // 8-byte stores; with a row stride of 40 floats the 16 lanes of a half warp hit 32 different banks
+                            const int col = (nt - 4 * half) * 8 + 2 * tq;
+                            *reinterpret_cast<float2*>(stage + gq * kStageStride + col) = make_float2(acc_dp[nt][0], acc_dp[nt][1]);
+                            *reinterpret_cast<float2*>(stage + (gq + 8) * kStageStride + col) = make_float2(acc_dp[nt][2], acc_dp[nt][3]);
                         }
                         __syncwarp();
                         if (g.w == 32 && r.ew == 32) {
@@ -308,7 +311,7 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
 #pragma unroll
                             for (int rr = 0; rr < 16; ++rr) {
                                 const bool first = rr <= lane;
-                                const float val = stage[rr * 33 + (first ? 31 - lane + rr : rr - lane - 1)];
+                                const float val = stage[rr * kStageStride + (first ? 31 - lane + rr : rr - lane - 1)];
                                 if (first) s0 += val; else s1 += val;
                             }
                             if (s0 != 0.f) atomicAdd(&s_dbias[row_base + bq0 - 31 + lane], s0);
@@ -317,7 +320,7 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
                             const int code_c = meta_code(s_meta[blk * BN + half * 32 + lane]);
                             for (int rr = 0; rr < 16; ++rr) {
                                 const int code_r = meta_code(s_meta[slot0 + rr]) + c0;
-                                const float v0 = stage[rr * 33 + lane];
+                                const float v0 = stage[rr * kStageStride + lane];
                                 if (v0 != 0.f) atomicAdd(&s_dbias[code_r - code_c], v0);
                             }
                         }
@@ -404,7 +407,7 @@ size_t bwd_smem_bytes(const Geo& g, bool query_side) {
     int npad_max = ((g.nmax + BN - 1) / BN) * BN;
     int nbias = (2 * g.w - 1) * (2 * g.w - 1);
     size_t head = (((size_t)npad_max * 16 + (size_t)nbias * 8 + 127) / 128) * 128;
-    size_t acc = query_side ? ((size_t)BM * acc_stride_for(g) + (size_t)BM * 33) * sizeof(float) : 0;
+    size_t acc = query_side ? ((size_t)BM * acc_stride_for(g) + (size_t)BM * kStageStride) * sizeof(float) : 0;
     return head + 6 * (size_t)BN * g.d * 2 + acc;
 }
 
