@@ -4,11 +4,13 @@
 //   warps 0-3 / 4-7  softmax warpgroups: one thread per query row of the first / second 128-row tile;
 //                    S is read from TMEM, P = exp2(S*scale + bias - m) is written back to TMEM as bf16,
 //                    O is read from TMEM, normalised and stored straight to the token's grid position
-//   warp 8           issues tcgen05.mma: S = Q K^T (operands in shared memory), O = P V (P from TMEM)
+//   warp 8           issues tcgen05.mma (the whole warp runs the loop and waits, one elected lane issues):
+//                    S = Q K^T (operands in shared memory), O = P [V | 1] (P from TMEM; 16 columns of ones behind
+//                    V make the accumulator carry the row sums of P in its columns 32..47)
 //   warps 9-11       loaders: undo the roll, gather the window's Q / K / V rows with cp.async into the
 //                    64-byte-swizzled operand layout, stage the head's bias table and the slot metadata
 // TMEM: columns [256 t, 256 t + 256) belong to query tile t: S (fp32) first; as pass 2 consumes it, bf16 P of
-// keys 0..127 goes to columns 0..63, the O accumulator to 64..95 and bf16 P of keys 128..255 to 128..191, so
+// keys 0..127 goes to columns 0..63, the O accumulator to 64..111 and bf16 P of keys 128..255 to 128..191, so
 // that O += P V over the first 128 keys runs while the softmax of the second 128 keys is still going on.
 // The row maximum is replaced by the upper bound max_j(raw score) * scale + max(bias): softmax is shift
 // invariant, so the result is the same; only the exponent range matters.
@@ -63,7 +65,7 @@ constexpr int kSmemBytes = kOffOnes + kMaxSlots * kRowBytes;
 constexpr int kNO = kD + 16;                                   // columns of the O accumulator
 
 // TMEM columns inside a query tile's 256-column region once S is being consumed: bf16 P of keys 0..127 in
-// [0, 64), the O accumulator in [64, 96) (S columns that the first half of pass 2 has already read), bf16
+// [0, 64), the O accumulator (with the row sums) in [64, 112) (S columns that the first half of pass 2 has already read), bf16
 // P of keys 128..255 in [128, 192).  The PV product of the first 128 keys is issued while the softmax
 // warpgroup is still working on the second 128 keys.
 constexpr int kColO = 64;
