@@ -392,6 +392,7 @@ def main():
     if rank == 0:
         peak_tf = peaks["bf16_tflops"]
         peak_bw = peaks["hbm_gbs"]
+        sm_count = torch.cuda.get_device_properties(local_rank).multi_processor_count
         # Algorithmic FLOP per launch of each kernel (strict convention, per allowed pair per head):
         # forward 4d (QK^T, PV); one-pass backward 8d (dP, dV, dK, dQ; the recomputed S is not counted); the
         # register-tile backward kernels 4d each (key tiles: dV, dK; query tiles: dP, dQ).
@@ -432,8 +433,19 @@ def main():
                              "peak": peak_bw, "unit": "GB/s",
                              "frac": (wk["bytes_fwd"] + wk["bytes_bwd"]) / (ms_step * 1e-3) / 1e9 / peak_bw,
                              "note": "algorithmic bytes of the whole step / step time"},
+            # The tcgen05 kernels are limited by the elementwise warps, not by the tensor pipe: one exp2 per
+            # (query, key) pair per head on the special-function unit (16 per clock per SM) and about 11 lane
+            # instructions per pair (128 lanes per clock per SM) in the dominant kernel.
+            "roofline_alu": {"bound": "alu", "kernel": dom["kernel"], "unit": "G pairs/s",
+                             "achieved": pairs / (dom["avg_ms"] * 1e-3) / 1e9,
+                             "peak_exp_unit": 16 * sm_count * (clocks.get("sm_mhz") or 1965.0) * 1e6 / 1e9,
+                             "peak_issue_slots": 128 * sm_count * (clocks.get("sm_mhz") or 1965.0) * 1e6 / 11.0 / 1e9,
+                             "note": "peaks derived from unit counts and the sampled SM clock; achieved = allowed pairs of one launch / its duration"},
             "clocks": clocks, "gpu_launches": launches, "e2e": e2e,
         }
+        ra = line["roofline_alu"]
+        ra["frac_exp_unit"] = ra["achieved"] / ra["peak_exp_unit"]
+        ra["frac_issue_slots"] = ra["achieved"] / ra["peak_issue_slots"]
         if not args.no_cpu_baseline and world == 1:
             line["cpu_baseline"] = cpu_baseline(cfg)
         elif world > 1:
