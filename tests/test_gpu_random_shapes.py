@@ -1,0 +1,55 @@
+"""Seeded random small shapes through the C ABI against the oracle: window sides 1..16 at head dim 32 (the
+tcgen05 kernels: every tile / block / mask / truncation combination the shapes happen to hit) and larger
+windows or head dim 64 (the register-tile kernels)."""
+import random
+
+import pytest
+import torch
+
+import oracle
+from paper_2608_15211_b200.workloads import make_inputs, small_config
+from tests._parity import gate, gpu_rows
+from tests.test_gpu_parity import _run_bwd, _run_fwd, _to_gpu
+
+pytestmark = pytest.mark.gpu
+
+
+def _shapes():
+    rng = random.Random(20260815)
+    out = []
+    for i in range(14):                      # head dim 32, window side <= 16
+        w = rng.choice([1, 3, 4, 5, 7, 8, 8, 9, 11, 12, 13, 14, 14, 15, 16, 16, 16])
+        H, W = rng.randint(1, 6 * w + 7), rng.randint(1, 6 * w + 9)
+        out.append((f"r{i}_w{w}", rng.choice([1, 1, 2, 3]), H, W, rng.choice([1, 2, 3, 5]), 32, w,
+                    rng.randint(0, H + 2), rng.randint(0, W + 2), rng.randint(0, 1), rng.randint(0, 1)))
+    for i in range(6):                       # head dim 64 and / or windows larger than 16
+        d = rng.choice([64, 64, 32])
+        w = rng.choice([32, 32, 24, 20, 17])
+        H, W = rng.randint(w // 2, 2 * w + 9), rng.randint(w // 2, 3 * w + 5)
+        out.append((f"g{i}_d{d}_w{w}", rng.choice([1, 2]), H, W, rng.choice([1, 2, 3]), d, w,
+                    rng.randint(0, H), rng.randint(0, W), rng.randint(0, 1), rng.randint(0, 1)))
+    return out
+
+
+SHAPES = _shapes()
+
+
+@pytest.mark.parametrize("case", SHAPES, ids=[c[0] for c in SHAPES])
+def test_random_shape_forward_backward(case):
+    cfg = small_config(*case)
+    x = make_inputs(cfg)
+    x["bias"] = x["bias"] * 25.0          # make the bias matter (std 0.5)
+    xg = _to_gpu(x)
+    d, o, lse = _run_fwd(cfg, xg)
+    dq, dk, dv, dbias = _run_bwd(cfg, d, xg, o, lse)
+    torch.cuda.synchronize()
+    bias64 = x["bias"].double().numpy()
+    ro, rl = oracle.attn_fwd(cfg, x["q"], x["k"], x["v"], bias64)
+    rq, rk, rv, rb = oracle.attn_bwd(cfg, x["q"], x["k"], x["v"], x["do"], bias64)
+    tok = oracle.selection_tokens(cfg, None)
+    # the two gates of the tolerance statement; the tighter diagnostic gate is kept for the fixed cases, where a
+    # single element a hair above it on a 150-token window would not be a finding
+    for name, got, ref in (("o", gpu_rows(o, cfg, tok), ro), ("lse", gpu_rows(lse, cfg, tok), rl),
+                           ("dq", gpu_rows(dq, cfg, tok), rq), ("dk", gpu_rows(dk, cfg, tok), rk),
+                           ("dv", gpu_rows(dv, cfg, tok), rv), ("dbias", dbias.cpu().double().numpy(), rb)):
+        gate(name, got, ref, strict=False)
