@@ -39,12 +39,15 @@ constexpr int kIssuerWarp = 8;      // warp 8: MMA issuer (also owns the TMEM al
 constexpr int kLoaderWarp0 = 9;     // warps 9..11: loaders
 constexpr int kLoaderWarps = 3;
 constexpr int kLoaderThreads = kLoaderWarps * 32;
-constexpr int kThreads = 12 * 32;                               // 384 = three warpgroups
+constexpr int kEpiWarp0 = 12;       // warps 12..15: read-out of the accumulators (one warp per TMEM lane quarter)
+constexpr int kEpiThreads = 128;
+constexpr int kThreads = 16 * 32;                               // 512 = four warpgroups
 constexpr int kWorkThreads = 256;          // elementwise threads; each arrives once per barrier phase
-constexpr int kRegsLaunch = 168;
-constexpr int kRegsWork = 216;      // elementwise warpgroups after setmaxnreg.inc
+constexpr int kRegsLaunch = 128;
+constexpr int kRegsWork = 192;      // elementwise warpgroups after setmaxnreg.inc
 constexpr int kRegsOther = 72;      // MMA + loader warpgroup after setmaxnreg.dec
-static_assert(2 * (kRegsWork - kRegsLaunch) <= (kRegsLaunch - kRegsOther), "register hand-over does not balance");
+constexpr int kRegsEpi = 56;        // read-out warpgroup after setmaxnreg.dec
+static_assert(2 * (kRegsWork - kRegsLaunch) <= (kRegsLaunch - kRegsOther) + (kRegsLaunch - kRegsEpi), "register hand-over does not balance");
 
 constexpr int kStages = 2;
 constexpr int kMaxSlots = 256;
@@ -336,17 +339,17 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(bar_full(s), kLoaderThreads);
-            mbar_init(bar_empty(s), kWorkThreads);
+            mbar_init(bar_empty(s), kEpiThreads);
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar_sdp(b), 1);
             mbar_init(bar_ds(b), kWorkThreads);
             mbar_init(bar_acc(b), 1);
-            mbar_init(bar_accfree(b), kWorkThreads);
+            mbar_init(bar_accfree(b), kEpiThreads);
         }
         mbar_init(bar_dsfree, 1);
         mbar_init(bar_dq, 1);
-        mbar_init(bar_dqfree, kWorkThreads);
+        mbar_init(bar_dqfree, kEpiThreads);
         *cta_abort = 0;
         fence_barrier_init();
     }
@@ -370,7 +373,88 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
     const int c0 = (g.w - 1) * (cs + 1);
     const size_t HW = (size_t)g.H * g.W;
 
-    if (warp >= kIssuerWarp) {
+    if (warp >= kEpiWarp0) {
+        // ------------------------------------------------------------------ read-out warps
+        // A tile's dV / dK and an item's dQ leave tensor memory here, as soon as their last MMA has completed,
+        // while the elementwise warps are already working on the next blocks.  Each output row (64 bytes) is
+        // staged in the item's own V / K / Q row, which no MMA reads any more, and stored from there as whole rows.
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kRegsEpi));
+        const int quarter = warp & 3;
+        const uint32_t tq = tmem_base + (((uint32_t)(32 * quarter)) << 16);
+        const float out_scale = g.scale_log2e * kLn2;          // dQ and dK carry the score scale
+        // 32 accumulator columns of this lane's row -> bf16 -> the row's place in the staging tile
+        auto stage_row = [&](uint32_t taddr, uint32_t rows_a, float f) {
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                uint32_t r[16];
+                tmem_ld16(taddr + 16 * half, r);
+                tmem_ld_wait();
+                sts_u4(rows_a + tile_off<kD>(lane, 2 * half),
+                       pack_bf16(__uint_as_float(r[0]) * f, __uint_as_float(r[1]) * f), pack_bf16(__uint_as_float(r[2]) * f, __uint_as_float(r[3]) * f),
+                       pack_bf16(__uint_as_float(r[4]) * f, __uint_as_float(r[5]) * f), pack_bf16(__uint_as_float(r[6]) * f, __uint_as_float(r[7]) * f));
+                sts_u4(rows_a + tile_off<kD>(lane, 2 * half + 1),
+                       pack_bf16(__uint_as_float(r[8]) * f, __uint_as_float(r[9]) * f), pack_bf16(__uint_as_float(r[10]) * f, __uint_as_float(r[11]) * f),
+                       pack_bf16(__uint_as_float(r[12]) * f, __uint_as_float(r[13]) * f), pack_bf16(__uint_as_float(r[14]) * f, __uint_as_float(r[15]) * f));
+            }
+        };
+        // the warp's 32 staged rows -> global memory, four lanes per row; `tok` = this lane's row's grid token (-1: none)
+        auto store_rows = [&](uint32_t rows_a, __nv_bfloat16* out, size_t sample_off, int tok) {
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj) {
+                const int rr = 8 * jj + (lane >> 2), c4 = lane & 3;
+                const int tok_r = __shfl_sync(0xffffffffu, tok, rr);
+                const int4 a = lds_i4(rows_a + tile_off<kD>(rr, c4));
+                if (tok_r >= 0)
+                    *reinterpret_cast<int4*>(out + ((sample_off + (size_t)tok_r) * g.heads + head) * kD + c4 * 8) = a;
+            }
+        };
+        int kuse = 0, n_tile = 0;
+        bool ok = true;
+        for (long long it = cta_in_head; ok && it < n_items; it += ctas_per_head, ++kuse) {
+            int npad, ntiles;
+            size_t sample_off;
+            {
+                const Item x = make_item(g, it);
+                npad = x.npad; ntiles = x.ntiles; sample_off = (size_t)x.b * HW;
+            }
+            const int s = kuse % kStages;
+            const uint32_t st_a = smem0 + s * kStageBytes;
+            if (!mbar_wait_all(bar_full(s), (kuse / kStages) & 1, cta_abort)) break;      // the slot -> token table of the stage
+            for (int t = 0; t < ntiles; ++t, ++n_tile) {
+                const int set = n_tile & 1;
+                ok = mbar_wait_all(bar_acc(set), (n_tile >> 1) & 1, cta_abort);
+                if (!ok) break;
+                tc_fence_after();
+                const int slot = 32 * ((4 * t + quarter + lane) & (4 * ntiles - 1)) + lane;      // interleaved key order
+                const int tok = lds_i32(st_a + kOffTok + 4 * slot);
+                const uint32_t rows_a = st_a + (uint32_t)((t * 128 + 32 * quarter) * kRowBytes);
+                stage_row(tq + kColDV + 64 * set, rows_a + kOffV, 1.f);
+                stage_row(tq + kColDK + 64 * set, rows_a + kOffK, out_scale);
+                tc_fence_before();
+                mbar_arrive(bar_accfree(set));
+                __syncwarp();
+                store_rows(rows_a + kOffV, dv, sample_off, tok);
+                store_rows(rows_a + kOffK, dk, sample_off, tok);
+            }
+            if (!ok) break;
+            ok = mbar_wait_all(bar_dq, kuse & 1, cta_abort);
+            if (!ok) break;
+            tc_fence_after();
+#pragma unroll
+            for (int hq = 0; hq < 2; ++hq)
+                if (hq * 128 < npad) stage_row(tq + kColDQ + 32 * hq, st_a + kOffQ + (uint32_t)((hq * 128 + 32 * quarter) * kRowBytes), out_scale);
+            tc_fence_before();
+            mbar_arrive(bar_dqfree);
+            __syncwarp();
+#pragma unroll
+            for (int hq = 0; hq < 2; ++hq)
+                if (hq * 128 < npad) {
+                    const int tokq = lds_i32(st_a + kOffTok + 4 * (hq * 128 + 32 * quarter + lane));
+                    store_rows(st_a + kOffQ + (uint32_t)((hq * 128 + 32 * quarter) * kRowBytes), dq, sample_off, tokq);
+                }
+            mbar_arrive(bar_empty(s));       // the stage's rows and tables are not needed any more
+        }
+    } else if (warp >= kIssuerWarp) {
     // warpgroup 2 (issuer + loaders) gives registers back: one instruction for the whole warpgroup
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kRegsOther));
     if (warp != kIssuerWarp) {
@@ -608,92 +692,9 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
         const int quarter = warp & 3;            // TMEM lane quarter = 32 key rows of the tile
         const uint32_t lane_addr = ((uint32_t)(32 * quarter)) << 16;
         const float scale = g.scale_log2e;
-        const float out_scale = g.scale_log2e * kLn2;          // dQ and dK carry the score scale
-        int kuse = 0, n_tile = 0, n_pair = 0;
+        int kuse = 0, n_pair = 0;
         uint32_t ph_sdp = 0;             // bit b: parity of the next completion of bar_sdp(b)
         bool ok = true;
-        // Read-outs are deferred: a tile's dV / dK (and, after an item's last tile, its dQ) are read one block
-        // later, after the first block of the next tile or item, so that the last MMAs of the tile have had a
-        // block's time to complete and no elementwise warp sits waiting for them.
-        int pend_tile = -1, pend_tile_s = 0, pend_tile_b = 0, pend_tile_tok = -1, pend_tile_seq = 0;   // tile index; its stage, sample, key token, tile number
-        int pend_item_s = -1, pend_item_b = 0, pend_item_npad = 0, pend_item_use = 0;                 // stage (-1: none), sample, columns, item number
-        auto flush_pending = [&]() -> bool {
-            if (pend_tile >= 0) {
-                // ---- the tile's dV (warps 0..3) / dK (warps 4..7): one 64-byte row per thread
-                const int set = pend_tile_seq & 1;
-                if (!mbar_wait_all(bar_acc(set), (pend_tile_seq >> 1) & 1, cta_abort)) return false;
-                tc_fence_after();
-                uint32_t r[32];
-                tmem_ld32(tmem_base + lane_addr + (h == 0 ? kColDV : kColDK) + 64 * set, r);
-                tmem_ld_wait();
-                tc_fence_before();
-                mbar_arrive(bar_accfree(set));
-                const float f = h == 0 ? 1.f : out_scale;
-                // the tile's own V (K) rows are dead now: stage the output rows there, then store whole rows
-                unsigned char* stg = smem + pend_tile_s * kStageBytes + (h == 0 ? kOffV : kOffK) + (pend_tile * 128 + 32 * quarter) * kRowBytes;
-                __nv_bfloat16* out = h == 0 ? dv : dk;
-#pragma unroll
-                for (int c4 = 0; c4 < 4; ++c4) {
-                    uint4 a;
-                    a.x = pack_bf16(__uint_as_float(r[c4 * 8 + 0]) * f, __uint_as_float(r[c4 * 8 + 1]) * f);
-                    a.y = pack_bf16(__uint_as_float(r[c4 * 8 + 2]) * f, __uint_as_float(r[c4 * 8 + 3]) * f);
-                    a.z = pack_bf16(__uint_as_float(r[c4 * 8 + 4]) * f, __uint_as_float(r[c4 * 8 + 5]) * f);
-                    a.w = pack_bf16(__uint_as_float(r[c4 * 8 + 6]) * f, __uint_as_float(r[c4 * 8 + 7]) * f);
-                    *reinterpret_cast<uint4*>(stg + tile_off<kD>(lane, c4)) = a;
-                }
-                __syncwarp();
-#pragma unroll
-                for (int jj = 0; jj < 4; ++jj) {
-                    const int rr = 8 * jj + (lane >> 2), c4 = lane & 3;
-                    const int tok_r = __shfl_sync(0xffffffffu, pend_tile_tok, rr);
-                    const uint4 a = *reinterpret_cast<const uint4*>(stg + tile_off<kD>(rr, c4));
-                    if (tok_r >= 0)
-                        *reinterpret_cast<uint4*>(out + (((size_t)pend_tile_b * HW + (size_t)tok_r) * g.heads + head) * kD + c4 * 8) = a;
-                }
-                __syncwarp();
-                pend_tile = -1;
-            }
-            if (pend_item_s >= 0) {
-                // ---- dQ: queries 0..127 by warps 0..3, queries 128..255 by warps 4..7
-                if (!mbar_wait_all(bar_dq, pend_item_use & 1, cta_abort)) return false;
-                tc_fence_after();
-                const bool have_q = h * 128 < pend_item_npad;
-                uint32_t r[32];
-                if (have_q) {
-                    tmem_ld32(tmem_base + lane_addr + kColDQ + 32 * h, r);
-                    tmem_ld_wait();
-                }
-                tc_fence_before();
-                mbar_arrive(bar_dqfree);
-                if (have_q) {
-                    const int tokq = lds_i32(smem0 + pend_item_s * kStageBytes + kOffTok + 4 * (h * 128 + 32 * quarter + lane));
-                    unsigned char* stg = smem + pend_item_s * kStageBytes + kOffQ + (h * 128 + 32 * quarter) * kRowBytes;
-#pragma unroll
-                    for (int c4 = 0; c4 < 4; ++c4) {
-                        uint4 a;
-                        a.x = pack_bf16(__uint_as_float(r[c4 * 8 + 0]) * out_scale, __uint_as_float(r[c4 * 8 + 1]) * out_scale);
-                        a.y = pack_bf16(__uint_as_float(r[c4 * 8 + 2]) * out_scale, __uint_as_float(r[c4 * 8 + 3]) * out_scale);
-                        a.z = pack_bf16(__uint_as_float(r[c4 * 8 + 4]) * out_scale, __uint_as_float(r[c4 * 8 + 5]) * out_scale);
-                        a.w = pack_bf16(__uint_as_float(r[c4 * 8 + 6]) * out_scale, __uint_as_float(r[c4 * 8 + 7]) * out_scale);
-                        *reinterpret_cast<uint4*>(stg + tile_off<kD>(lane, c4)) = a;
-                    }
-                    __syncwarp();
-#pragma unroll
-                    for (int jj = 0; jj < 4; ++jj) {
-                        const int rr = 8 * jj + (lane >> 2), c4 = lane & 3;
-                        const int tok_r = __shfl_sync(0xffffffffu, tokq, rr);
-                        const uint4 a = *reinterpret_cast<const uint4*>(stg + tile_off<kD>(rr, c4));
-                        if (tok_r >= 0)
-                            *reinterpret_cast<uint4*>(dq + (((size_t)pend_item_b * HW + (size_t)tok_r) * g.heads + head) * kD + c4 * 8) = a;
-                    }
-                    __syncwarp();
-                }
-                mbar_arrive(bar_empty(pend_item_s));       // this thread no longer touches that stage
-                pend_item_s = -1;
-            }
-            return true;
-        };
-
         int J = 0;                       // number of this block in the CTA's sequence; its S / dP buffer is J & 1
         for (long long it = cta_in_head; ok && it < n_items; it += ctas_per_head, ++kuse) {
             const Item x = make_item(g, it);
@@ -809,19 +810,10 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                     fence_proxy_async();
                     mbar_arrive(bar_ds(buf));
                     ++J;
-                    if (b == 0) {
-                        ok = flush_pending();      // the previous tile's / item's read-out
-                        if (!ok) break;
-                    }
                 }
                 if (!ok) break;
-                pend_tile = t; pend_tile_s = s; pend_tile_b = x.b; pend_tile_tok = tok; pend_tile_seq = n_tile;
-                ++n_tile;
             }
-            if (!ok) break;
-            pend_item_s = s; pend_item_b = x.b; pend_item_npad = x.npad; pend_item_use = kuse;
         }
-        if (ok) flush_pending();
     }
 
     // teardown: every role ends up here, also after an expired wait
