@@ -654,9 +654,6 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                         }
                     }
                     __syncwarp();
-                    // S^T / dP^T two blocks ahead (this buffer is free again: its P / dS reads were issued just above)
-                    ok = issue_upto(min(J + 3, J0 + nb + nb_n));
-                    if (!ok) break;
                     if ((b & 1) || b == nblk - 1) {
                         // dQ (queries of this pair of blocks) += dS K over the tile's keys
                         if (t == 0 && b < 2 && kuse > 0) {   // the item's first write of dQ: the previous item's was read
@@ -680,6 +677,11 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                         }
                         __syncwarp();
                     }
+                    // S^T / dP^T two blocks ahead (this buffer is free again: its P / dS reads were issued above).  They
+                    // come after the dQ MMAs: the elementwise warps need the shared dS tile back one block from
+                    // now, the new S / dP only two blocks from now.
+                    ok = issue_upto(min(J + 3, J0 + nb + nb_n));
+                    if (!ok) break;
                 }
                 ++n_tile;
             }
