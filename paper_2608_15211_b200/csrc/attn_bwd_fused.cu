@@ -44,9 +44,9 @@ constexpr int kEpiThreads = 128;
 constexpr int kThreads = 16 * 32;                               // 512 = four warpgroups
 constexpr int kWorkThreads = 256;          // elementwise threads; each arrives once per barrier phase
 constexpr int kRegsLaunch = 128;
-constexpr int kRegsWork = 192;      // elementwise warpgroups after setmaxnreg.inc
-constexpr int kRegsOther = 72;      // MMA + loader warpgroup after setmaxnreg.dec
-constexpr int kRegsEpi = 56;        // read-out warpgroup after setmaxnreg.dec
+constexpr int kRegsWork = 184;      // elementwise warpgroups after setmaxnreg.inc
+constexpr int kRegsOther = 80;      // MMA + loader warpgroup after setmaxnreg.dec
+constexpr int kRegsEpi = 64;        // read-out warpgroup after setmaxnreg.dec
 static_assert(2 * (kRegsWork - kRegsLaunch) <= (kRegsLaunch - kRegsOther) + (kRegsLaunch - kRegsEpi), "register hand-over does not balance");
 
 constexpr int kStages = 2;
@@ -98,12 +98,11 @@ struct Item {
     bool ragged;   // some row of a key tile, or some column below npad, has no token
 };
 
-__device__ __forceinline__ Item make_item(const Geo& g, long long it) {
+__device__ __forceinline__ Item make_item(const Geo& g, const ItemCursor& c) {
     Item x;
-    const int M = g.Mh * g.Mw;
-    x.win = (int)(it % M);
-    x.b = (int)(it / M);
-    x.r = window_ref(g, x.win);
+    x.win = c.wr * g.Mw + c.wc;
+    x.b = c.b;
+    x.r = window_ref_rc(g, c.wr, c.wc);
     x.npad = (x.r.n + 15) & ~15;
     x.ntiles = (x.r.n + 127) >> 7;
     x.nblk = (x.npad + CB - 1) / CB;
@@ -410,11 +409,12 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
         };
         int kuse = 0, n_tile = 0;
         bool ok = true;
-        for (long long it = cta_in_head; ok && it < n_items; it += ctas_per_head, ++kuse) {
+        ItemCursor cur_it = cursor_init(cta_in_head, ctas_per_head, 1, g.Mw, g.Mh);
+        for (long long it = cta_in_head; ok && it < n_items; it += ctas_per_head, ++kuse, cursor_advance(cur_it, 1, g.Mw, g.Mh)) {
             int npad, ntiles;
             size_t sample_off;
             {
-                const Item x = make_item(g, it);
+                const Item x = make_item(g, cur_it);
                 npad = x.npad; ntiles = x.ntiles; sample_off = (size_t)x.b * HW;
             }
             const int s = kuse % kStages;
@@ -461,7 +461,8 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
         // ------------------------------------------------------------------ loaders
         const int lt = (warp - kLoaderWarp0) * 32 + lane;
         int kuse = 0, pending_s = -1;
-        for (long long it = cta_in_head; it < n_items; it += ctas_per_head, ++kuse) {
+        ItemCursor cur_it = cursor_init(cta_in_head, ctas_per_head, 1, g.Mw, g.Mh);
+        for (long long it = cta_in_head; it < n_items; it += ctas_per_head, ++kuse, cursor_advance(cur_it, 1, g.Mw, g.Mh)) {
             const int s = kuse % kStages;
             // if the next stage is not free yet, publish the copies already issued instead of holding them back
             if (pending_s >= 0 && !__all_sync(0xffffffffu, mbar_test_wait(bar_empty(s), ((kuse / kStages) & 1) ^ 1))) {
@@ -471,7 +472,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                 pending_s = -1;
             }
             if (!mbar_wait_all(bar_empty(s), ((kuse / kStages) & 1) ^ 1, cta_abort)) break;
-            const Item x = make_item(g, it);
+            const Item x = make_item(g, cur_it);
             unsigned char* st = smem + s * kStageBytes;
             const uint32_t st_a = smem0 + s * kStageBytes;
             const size_t sample_off = (size_t)x.b * HW;
@@ -576,19 +577,22 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
             }
             __syncwarp();
         };
+        ItemCursor nx_it = cursor_init(cta_in_head, ctas_per_head, 1, g.Mw, g.Mh);     // runs one item ahead
+        int npad = 0, ntiles = 0, nblk = 1;
+        if (cta_in_head < n_items) {
+            const Item x = make_item(g, nx_it);
+            npad = x.npad; ntiles = x.ntiles; nblk = x.nblk;
+            cursor_advance(nx_it, 1, g.Mw, g.Mh);
+        }
         for (long long it = cta_in_head; ok && it < n_items; it += ctas_per_head, ++kuse) {
             const int s = kuse % kStages;
-            int npad, ntiles, nblk;
-            {
-                const Item x = make_item(g, it);
-                npad = x.npad; ntiles = x.ntiles; nblk = x.nblk;
-            }
             const int nb = ntiles * nblk;
             // the item after this one
-            int nb_n = 0, npad_n = 0, nblk_n = 1;
+            int nb_n = 0, npad_n = 0, nblk_n = 1, ntiles_n = 0;
             if (it + ctas_per_head < n_items) {
-                const Item xn = make_item(g, it + ctas_per_head);
-                nb_n = xn.ntiles * xn.nblk; npad_n = xn.npad; nblk_n = xn.nblk;
+                const Item xn = make_item(g, nx_it);
+                cursor_advance(nx_it, 1, g.Mw, g.Mh);
+                nb_n = xn.ntiles * xn.nblk; npad_n = xn.npad; nblk_n = xn.nblk; ntiles_n = xn.ntiles;
             }
             const int J0 = J;
             ok = mbar_wait_all(bar_full(s), (kuse / kStages) & 1, cta_abort);
@@ -685,6 +689,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                 }
                 ++n_tile;
             }
+            npad = npad_n; ntiles = ntiles_n; nblk = nblk_n;     // the next item becomes the current one
         }
     }
     } else {
@@ -698,8 +703,9 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
         uint32_t ph_sdp = 0;             // bit b: parity of the next completion of bar_sdp(b)
         bool ok = true;
         int J = 0;                       // number of this block in the CTA's sequence; its S / dP buffer is J & 1
-        for (long long it = cta_in_head; ok && it < n_items; it += ctas_per_head, ++kuse) {
-            const Item x = make_item(g, it);
+        ItemCursor cur_it = cursor_init(cta_in_head, ctas_per_head, 1, g.Mw, g.Mh);
+        for (long long it = cta_in_head; ok && it < n_items; it += ctas_per_head, ++kuse, cursor_advance(cur_it, 1, g.Mw, g.Mh)) {
+            const Item x = make_item(g, cur_it);
             const int s = kuse % kStages;
             const uint32_t st_a = smem0 + s * kStageBytes;
             if (!mbar_wait_all(bar_full(s), (kuse / kStages) & 1, cta_abort)) break;

@@ -84,14 +84,12 @@ struct Item {
     bool masked;   // the window mixes shift-mask labels
 };
 
-__device__ __forceinline__ Item make_item(const Geo& g, long long it) {
+__device__ __forceinline__ Item make_item(const Geo& g, const ItemCursor& c) {
     Item x;
-    x.head = (int)(it % g.heads);
-    long long rest = it / g.heads;
-    const int M = g.Mh * g.Mw;
-    x.win = (int)(rest % M);
-    x.b = (int)(rest / M);
-    x.r = window_ref(g, x.win);
+    x.head = c.head;
+    x.win = c.wr * g.Mw + c.wc;
+    x.b = c.b;
+    x.r = window_ref_rc(g, c.wr, c.wc);
     x.npad = (x.r.n + 15) & ~15;
     x.ntiles = (x.r.n + 127) >> 7;
     // rolled rows >= H - sh (columns >= W - sw) hold the tokens that wrapped across a non-periodic edge
@@ -347,7 +345,8 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
         // ------------------------------------------------------------------ loaders
         const int lt = (warp - kLoaderWarp0) * 32 + lane;
         int kuse = 0, pending_s = -1;
-        for (long long it = blockIdx.x; it < n_items; it += gridDim.x, ++kuse) {
+        ItemCursor cur_it = cursor_init(blockIdx.x, gridDim.x, g.heads, g.Mw, g.Mh);
+        for (long long it = blockIdx.x; it < n_items; it += gridDim.x, ++kuse, cursor_advance(cur_it, g.heads, g.Mw, g.Mh)) {
             const int s = kuse % kStages;
             // if the next stage is not free yet, publish the copies already issued instead of holding them back
             if (pending_s >= 0 && !__all_sync(0xffffffffu, mbar_test_wait(bar_empty(s), ((kuse / kStages) & 1) ^ 1))) {
@@ -357,7 +356,7 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
                 pending_s = -1;
             }
             if (!__all_sync(0xffffffffu, mbar_wait(bar_empty(s), ((kuse / kStages) & 1) ^ 1, cta_abort))) break;
-            const Item x = make_item(g, it);
+            const Item x = make_item(g, cur_it);
             unsigned char* st = smem + s * kStageBytes;
             const uint32_t st_a = smem0 + s * kStageBytes;
             int* s_kc = reinterpret_cast<int*>(st + kOffKc);
@@ -451,9 +450,11 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
                 __syncwarp();
             };
             long long it = blockIdx.x;
+            ItemCursor nx_it = cursor_init(blockIdx.x, gridDim.x, g.heads, g.Mw, g.Mh);     // runs one item ahead
             Item cur;
             if (it < n_items) {
-                cur = make_item(g, it);
+                cur = make_item(g, nx_it);
+                cursor_advance(nx_it, g.heads, g.Mw, g.Mh);
                 ok = mbar_wait_all(bar_full(0), 0, cta_abort);
                 if (ok) {
                     fence_proxy_async();
@@ -467,7 +468,10 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
                 const bool has_next = nxt < n_items;
                 Item nx;
                 const int sn = (kuse + 1) % kStages;
-                if (has_next) nx = make_item(g, nxt);
+                if (has_next) {
+                    nx = make_item(g, nx_it);
+                    cursor_advance(nx_it, g.heads, g.Mw, g.Mh);
+                }
                 bool next_ready = false;
                 const int nks = cur.npad >> 4;
                 // first 128 keys of each tile, as soon as their P is there
@@ -527,8 +531,9 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
         const uint32_t t_s = tmem_base + lane_addr + wg * 256;
         const float scale = g.scale_log2e;
         int kuse = 0, use = 0;
-        for (long long it = blockIdx.x; it < n_items; it += gridDim.x, ++kuse) {
-            const Item x = make_item(g, it);
+        ItemCursor cur_it = cursor_init(blockIdx.x, gridDim.x, g.heads, g.Mw, g.Mh);
+        for (long long it = blockIdx.x; it < n_items; it += gridDim.x, ++kuse, cursor_advance(cur_it, g.heads, g.Mw, g.Mh)) {
+            const Item x = make_item(g, cur_it);
             if (wg >= x.ntiles) continue;
             const int s = kuse % kStages;
             const uint32_t st_a = smem0 + s * kStageBytes;

@@ -26,6 +26,19 @@ constexpr float kLn2 = 0.6931471805599453f;
 __device__ __forceinline__ int meta_code(int m) { return m & 0xffff; }
 __device__ __forceinline__ int meta_label(int m) { return m >> 16; }
 
+// it = quo * div + rem.  Item numbers almost always fit 32 bits, where the division is a handful of
+// instructions; the 64-bit one (a long software routine) is kept for the sizes that need it.
+__device__ __forceinline__ void split_item(long long it, int div, long long& quo, int& rem) {
+    if (((unsigned long long)it >> 32) == 0) {
+        const unsigned i = (unsigned)it, q = i / (unsigned)div;
+        quo = q;
+        rem = (int)(i - q * (unsigned)div);
+    } else {
+        quo = it / div;
+        rem = (int)(it - quo * div);
+    }
+}
+
 struct WindowRef {
     int wr, wc;   // window row / column
     int eh, ew;   // true extent (truncated at the last row / column)
@@ -40,6 +53,50 @@ __device__ __forceinline__ WindowRef window_ref(const Geo& g, int win) {
     r.ew = min(g.w, g.W - r.wc * g.w);
     r.n = r.eh * r.ew;
     return r;
+}
+
+__device__ __forceinline__ WindowRef window_ref_rc(const Geo& g, int wr, int wc) {
+    WindowRef r;
+    r.wr = wr;
+    r.wc = wc;
+    r.eh = min(g.w, g.H - wr * g.w);
+    r.ew = min(g.w, g.W - wc * g.w);
+    r.n = r.eh * r.ew;
+    return r;
+}
+
+// A persistent CTA's items are it0, it0 + step, it0 + 2 step, ...  The item number is kept as mixed-radix
+// digits (head | window column | window row | sample, fastest first; radix of the head digit 1 where the head
+// is fixed), and going to the next item adds the step's digits with carries: no division per item (an integer
+// division is a long dependent chain through the reciprocal unit, which the softmax warps keep busy).
+struct ItemCursor {
+    int head, wc, wr, b;
+    int s_head, s_wc, s_wr, s_b;
+};
+__device__ __forceinline__ void cursor_digits(long long it, int heads_radix, int Mw, int Mh, int& head, int& wc, int& wr, int& b) {
+    long long rest, rest2, rest3;
+    split_item(it, heads_radix, rest, head);
+    split_item(rest, Mw, rest2, wc);
+    split_item(rest2, Mh, rest3, wr);
+    b = (int)rest3;
+}
+__device__ __forceinline__ ItemCursor cursor_init(long long it0, long long step, int heads_radix, int Mw, int Mh) {
+    ItemCursor c;
+    cursor_digits(it0, heads_radix, Mw, Mh, c.head, c.wc, c.wr, c.b);
+    cursor_digits(step, heads_radix, Mw, Mh, c.s_head, c.s_wc, c.s_wr, c.s_b);
+    return c;
+}
+__device__ __forceinline__ void cursor_advance(ItemCursor& c, int heads_radix, int Mw, int Mh) {
+    c.head += c.s_head;
+    int carry = c.head >= heads_radix;
+    c.head -= carry ? heads_radix : 0;
+    c.wc += c.s_wc + carry;
+    carry = c.wc >= Mw;
+    c.wc -= carry ? Mw : 0;
+    c.wr += c.s_wr + carry;
+    carry = c.wr >= Mh;
+    c.wr -= carry ? Mh : 0;
+    c.b += c.s_b + carry;
 }
 
 // Slot of a window -> grid token u * W + v (undoing the roll) and packed metadata.
