@@ -100,10 +100,8 @@ __device__ __forceinline__ Item make_item(const Geo& g, const ItemCursor& c) {
     return x;
 }
 
-// slot -> grid token, bias code a * (w + 32) + b and shift-mask label
-__device__ __forceinline__ int slot_token_tc(const Geo& g, const WindowRef& r, int slot, int& code, int& label) {
-    const int a = slot / r.ew;
-    const int b = slot - a * r.ew;
+// window offset (a, b) -> grid token, bias code a * (w + 32) + b and shift-mask label
+__device__ __forceinline__ int offset_token_tc(const Geo& g, const WindowRef& r, int a, int b, int& code, int& label) {
     int u = r.wr * g.w + a + g.sh;
     if (u >= g.H) u -= g.H;
     int v = r.wc * g.w + b + g.sw;
@@ -365,26 +363,35 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
             int* s_rowtok = reinterpret_cast<int*>(st + kOffRowTok);
             const size_t sample_off = (size_t)x.b * HW;
 
+            // Slots advance by a fixed step, so their window offsets (a, b) = (slot / width, slot mod width) are
+            // carried along instead of divided out each time (a division is a long chain through the reciprocal unit).
+            const int ew = x.r.ew;
+            const int q_s = kLoaderThreads / ew, r_s = kLoaderThreads - q_s * ew;              // slot loop: step of kLoaderThreads
+            const int q_r = (kLoaderThreads / 4) / ew, r_r = (kLoaderThreads / 4) - q_r * ew;  // row loop: step of kLoaderThreads / 4
+            int a_s = lt / ew, b_s = lt - a_s * ew;
             for (int slot = lt; slot < kMaxSlots; slot += kLoaderThreads) {
                 // a slot without a token: as a key its bias index lands in the table's -inf zone
                 int code = 0, label = 0xff, tok = -1, kc = 4 * (2 * c0 + 1);
                 if (slot < x.r.n) {
-                    tok = slot_token_tc(g, x.r, slot, code, label);
+                    tok = offset_token_tc(g, x.r, a_s, b_s, code, label);
                     kc = 4 * (c0 - code);
                 }
                 s_kc[slot] = kc;
                 s_klab[slot] = label;
                 s_rowmeta[slot] = code | (label << 16);
                 s_rowtok[slot] = tok;
+                a_s += q_s; b_s += r_s;
+                if (b_s >= ew) { b_s -= ew; ++a_s; }
             }
-            // rows: this thread owns 16-byte chunk (lt & 3) of rows (lt >> 2) + 32 i
+            // rows: this thread owns 16-byte chunk (lt & 3) of rows (lt >> 2) + (kLoaderThreads / 4) i
             const int chunk = lt & 3;
+            int a_r = (lt >> 2) / ew, b_r = (lt >> 2) - a_r * ew;
             for (int row = lt >> 2; row < x.npad; row += kLoaderThreads / 4) {
                 const __nv_bfloat16 *sq = q, *sk = k, *sv = v;
                 int bytes = 0;   // rows past the window's end are written as zeros
                 if (row < x.r.n) {
                     int code, label;
-                    const int tok = slot_token_tc(g, x.r, row, code, label);
+                    const int tok = offset_token_tc(g, x.r, a_r, b_r, code, label);
                     const size_t off = ((sample_off + (size_t)tok) * g.heads + x.head) * kD + chunk * 8;
                     sq = q + off; sk = k + off; sv = v + off;
                     bytes = 16;
@@ -393,6 +400,8 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
                 cp_async16(so + kOffQ, sq, bytes);
                 cp_async16(so + kOffK, sk, bytes);
                 cp_async16(so + kOffV, sv, bytes);
+                a_r += q_r; b_r += r_r;
+                if (b_r >= ew) { b_r -= ew; ++a_r; }
             }
             const float* bsrc = bias_prep + (size_t)x.head * kFwdBiasFloats;
             for (int c = lt; c < kFwdBiasFloats / 4; c += kLoaderThreads)
