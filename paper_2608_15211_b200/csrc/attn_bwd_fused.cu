@@ -114,9 +114,8 @@ __device__ __forceinline__ Item make_item(const Geo& g, const ItemCursor& c) {
     return x;
 }
 
-__device__ __forceinline__ int slot_token_tc(const Geo& g, const WindowRef& r, int slot, int& code, int& label) {
-    const int a = slot / r.ew;
-    const int b = slot - a * r.ew;
+// window offset (a, b) -> grid token, bias code and shift-mask label
+__device__ __forceinline__ int offset_token_tc(const Geo& g, const WindowRef& r, int a, int b, int& code, int& label) {
     int u = r.wr * g.w + a + g.sh;
     if (u >= g.H) u -= g.H;
     int v = r.wc * g.w + b + g.sw;
@@ -479,15 +478,22 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
             // slot metadata; the lse / delta gathers stay in flight while the row copies are issued below
             constexpr int kSlotIters = (kMaxSlots + kLoaderThreads - 1) / kLoaderThreads;
             float l2v[kSlotIters], dlv[kSlotIters];
+            // Slots advance by a fixed step, so their window offsets (a, b) = (slot / width, slot mod width) are
+            // carried along instead of divided out each time (a division is a long chain through the reciprocal unit).
+            const int ew = x.r.ew;
+            const int q_s = kLoaderThreads / ew, r_s = kLoaderThreads - q_s * ew;              // slot loop: step of kLoaderThreads
+            const int q_r = (kLoaderThreads / 4) / ew, r_r = (kLoaderThreads / 4) - q_r * ew;  // row loop: step of kLoaderThreads / 4
+            int a_s = lt / ew, b_s = lt - a_s * ew;
 #pragma unroll
-            for (int i = 0; i < kSlotIters; ++i) {
+            for (int i = 0; i < kSlotIters; ++i, a_s += q_s, b_s += r_s) {
+                if (b_s >= ew) { b_s -= ew; ++a_s; }
                 const int slot = lt + i * kLoaderThreads;
                 l2v[i] = INFINITY;                       // no token: P = exp2(.. - inf) = 0
                 dlv[i] = 0.f;
                 if (slot >= kMaxSlots) continue;
                 int code = 0, label = 0xff, tok = -1;
                 if (slot < x.r.n) {
-                    tok = slot_token_tc(g, x.r, slot, code, label);
+                    tok = offset_token_tc(g, x.r, a_s, b_s, code, label);
                     const size_t li = (sample_off + (size_t)tok) * g.heads + head;
                     l2v[i] = __ldg(lse + li);
                     dlv[i] = __ldg(delta + li);
@@ -503,13 +509,15 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
             const int chunk = lt & 3;
             const int nrows = x.ntiles * 128;
             const int M = 4 * x.ntiles;
-            for (int row = lt >> 2; row < nrows; row += kLoaderThreads / 4) {
+            int a_r = (lt >> 2) / ew, b_r = (lt >> 2) - a_r * ew;
+            for (int row = lt >> 2; row < nrows; row += kLoaderThreads / 4, a_r += q_r, b_r += r_r) {
+                if (b_r >= ew) { b_r -= ew; ++a_r; }
                 const int kl = row & 31, kw = ((row >> 5) - kl) & (M - 1), krow = 128 * (kw >> 2) + 32 * (kw & 3) + kl;
                 const __nv_bfloat16 *sq = q, *sk = k, *sv = v, *sg = d_o;
                 int bytes = 0;
                 if (row < x.r.n) {
                     int code, label;
-                    const int tok = slot_token_tc(g, x.r, row, code, label);
+                    const int tok = offset_token_tc(g, x.r, a_r, b_r, code, label);
                     const size_t off = ((sample_off + (size_t)tok) * g.heads + head) * kD + chunk * 8;
                     sq = q + off; sk = k + off; sv = v + off; sg = d_o + off;
                     bytes = 16;
