@@ -166,6 +166,27 @@ int terra_profile_enable(int on);
 int terra_profile_count(void);
 int terra_profile_get(int index, char* name, int name_bytes, float* ms);
 
+/*
+ * Window ownership across window-parallel (WP) ranks (Section V-A).  Host-only integer helpers; they launch
+ * nothing and touch no device.  This library runs one GPU; these state which windows a rank of a WP group
+ * would own, so that a caller sharding windows over several processes uses the paper's rule.
+ *
+ * terra_fixed_assignment_padding (Eq. 3): the fixed round-robin assignment over an m x n WP mesh needs every
+ * rank to hold the same number of complete windows, so the INPUT field (H x W grid points, before patching) is
+ * padded to  H_hat = ceil(H / (p alpha w m)) p alpha w m,  W_hat = ceil(W / (p alpha w n)) p alpha w n
+ * (p patch size, alpha sampling factor, w window side in tokens).  m = n = 1 gives the padding to complete
+ * windows alone, which is all the ragged assignment needs.  All arguments >= 1; results via H_hat, W_hat
+ * (either may be NULL).  TERRA_ERR_INVALID_ARG on a non-positive argument or a product that overflows int64.
+ *
+ * terra_ragged_window_range (Eq. 4): with the M = M_h M_w complete windows numbered row-major, rank r of
+ * `ranks` owns the contiguous range [L, R),  L = floor(r M / ranks),  R = floor((r + 1) M / ranks).  Every
+ * window is owned exactly once and two ranks' counts differ by at most one.  M >= 0, ranks >= 1,
+ * 0 <= r < ranks; else TERRA_ERR_INVALID_ARG.  Either output may be NULL.
+ */
+int terra_fixed_assignment_padding(int64_t H, int64_t W, int32_t p, int32_t alpha, int32_t w, int32_t m, int32_t n,
+                                   int64_t* H_hat, int64_t* W_hat);
+int terra_ragged_window_range(int64_t M, int32_t ranks, int32_t r, int64_t* L, int64_t* R);
+
 /* Static text for a terra_status.  Host-only. */
 const char* terra_strerror(int status);
 

@@ -17,7 +17,8 @@ from .build import LIB_PATH
 TERRA_OK = 0
 EXPORTS = ("terra_route_sizes", "terra_window_route", "terra_swin_workspace_bytes", "terra_swin_attn_fwd",
            "terra_swin_attn_fwd_noalloc", "terra_swin_attn_bwd", "terra_swin_check", "terra_strerror", "terra_last_cuda_error",
-           "terra_launch_count", "terra_selftest_bounded_wait", "terra_profile_enable", "terra_profile_count", "terra_profile_get")
+           "terra_launch_count", "terra_selftest_bounded_wait", "terra_profile_enable", "terra_profile_count", "terra_profile_get",
+           "terra_fixed_assignment_padding", "terra_ragged_window_range")
 
 
 class TerraError(RuntimeError):
@@ -67,6 +68,10 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
     lib.terra_profile_enable.argtypes = [ctypes.c_int]
     lib.terra_profile_count.restype = ctypes.c_int
     lib.terra_profile_get.argtypes = [ctypes.c_int, ctypes.c_char_p, ctypes.c_int, ctypes.POINTER(ctypes.c_float)]
+    lib.terra_fixed_assignment_padding.argtypes = [ctypes.c_int64, ctypes.c_int64] + [ctypes.c_int32] * 5 + [i64p, i64p]
+    lib.terra_fixed_assignment_padding.restype = ctypes.c_int
+    lib.terra_ragged_window_range.argtypes = [ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, i64p, i64p]
+    lib.terra_ragged_window_range.restype = ctypes.c_int
     if path is None:
         _lib = lib
     return lib
@@ -128,6 +133,20 @@ def selftest_bounded_wait(limit_cycles: int = 1_000_000) -> None:
 
 def launch_count() -> int:
     return int(load_library().terra_launch_count())
+
+
+def terra_fixed_assignment_padding(H: int, W: int, p: int, alpha: int, w: int, m: int = 1, n: int = 1):
+    """(H_hat, W_hat) of Eq. 3: the input field padded so that an m x n WP mesh holds equal window counts."""
+    hh, ww = ctypes.c_int64(), ctypes.c_int64()
+    _check(load_library().terra_fixed_assignment_padding(H, W, p, alpha, w, m, n, ctypes.byref(hh), ctypes.byref(ww)))
+    return hh.value, ww.value
+
+
+def terra_ragged_window_range(M: int, ranks: int, r: int):
+    """[L, R) of Eq. 4: the row-major window range that rank r of `ranks` owns."""
+    lo, hi = ctypes.c_int64(), ctypes.c_int64()
+    _check(load_library().terra_ragged_window_range(M, ranks, r, ctypes.byref(lo), ctypes.byref(hi)))
+    return lo.value, hi.value
 
 
 def terra_route_sizes(desc: terra_swin_desc):
