@@ -207,6 +207,7 @@ def main():
     ap.add_argument("--impl", default="terra", choices=["terra", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-packed", action="store_true", help="skip the packed-QKV leg")
     ap.add_argument("--rows", type=int, default=0,
                     help="profiling aid: keep the configuration but use this many token rows (a smaller case of the "
                          "same kernels for ncu captures); the JSON names the changed grid")
@@ -327,6 +328,32 @@ def main():
     bwd_ms = statistics.mean(e[2].elapsed_time(e[3]) for e in ev)
     value = whole_job_tflops(flops, world, ms_step)
 
+    # the same step on the packed layout of a fused QKV projection ([B, H, W, 3, heads, d] in, the gradient in
+    # the same layout out): same kernels, only the token stride differs
+    packed = None
+    if not args.no_packed:
+        qkv = torch.stack([q, k, v], dim=3).contiguous()
+        dqkv = torch.empty_like(qkv)
+        for _ in range(3):
+            terra.terra_swin_attn_fwd_packed(desc, qkv, bias, o, lse, ws)
+            terra.terra_swin_attn_bwd_packed(desc, qkv, bias, o, lse, d_o, dqkv, dbias, ws)
+        n_packed = max(4, min(args.steps, 20))
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        a.record()
+        for _ in range(n_packed):
+            terra.terra_swin_attn_fwd_packed(desc, qkv, bias, o, lse, ws)
+            terra.terra_swin_attn_bwd_packed(desc, qkv, bias, o, lse, d_o, dqkv, dbias, ws)
+        b.record()
+        barrier()
+        packed_ms = max_over_ranks(a.elapsed_time(b) / n_packed, dev)
+        packed = {"value": whole_job_tflops(flops, world, packed_ms), "unit": UNIT, "ms_per_step": packed_ms, "steps": n_packed,
+                  "note": "terra_swin_attn_fwd_packed + terra_swin_attn_bwd_packed on qkv / dqkv [B, H, W, 3, heads, d]"}
+        del qkv, dqkv
+        # restore the outputs of the unpacked step for whatever reads them below
+        call_fwd()
+        call_bwd()
+
     # end to end through the C ABI from pinned HOST buffers: every step copies its inputs host -> device, runs, and
     # copies its results device -> host.  Two device buffer sets and three streams, as an application would do
     # it: the H2D copy of step i + 1 and the D2H copy of step i - 1 overlap step i's kernels.
@@ -443,6 +470,8 @@ def main():
                              "note": "peaks derived from unit counts and the sampled SM clock; achieved = allowed pairs of one launch / its duration"},
             "clocks": clocks, "gpu_launches": launches, "e2e": e2e,
         }
+        if packed is not None:
+            line["packed_qkv"] = packed
         ra = line["roofline_alu"]
         ra["frac_exp_unit"] = ra["achieved"] / ra["peak_exp_unit"]
         ra["frac_issue_slots"] = ra["achieved"] / ra["peak_issue_slots"]

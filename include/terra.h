@@ -114,6 +114,23 @@ int terra_swin_attn_bwd(const terra_swin_desc* desc, const void* q, const void* 
                         void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The same two passes on the packed layout of a fused QKV projection (the block sits between that GEMM and the
+ * output projection, Section IV-A; the paper has no layout statement, this is the library's): the GEMM's output
+ * is consumed in place and the gradient comes back in the layout that GEMM's backward reads, with no re-layout
+ * pass in between.
+ *   qkv    bf16 [B, H, W, 3, heads, head_dim]   q = [..., 0, :, :], k = [..., 1, :, :], v = [..., 2, :, :]
+ *   dqkv   bf16 [B, H, W, 3, heads, head_dim]   overwritten: dq, dk, dv in the same three slots
+ *   o, lse, d_o, bias_table, dbias, workspace   as in terra_swin_attn_fwd / terra_swin_attn_bwd (o and d_o dense
+ *                                               [B, H, W, heads, head_dim]); same sizes from terra_swin_workspace_bytes
+ * Results are those of the unpacked calls on the three slices, bit for bit; same error codes.
+ */
+int terra_swin_attn_fwd_packed(const terra_swin_desc* desc, const void* qkv, const float* bias_table, void* o, float* lse,
+                               void* workspace, size_t workspace_bytes, void* stream);
+int terra_swin_attn_bwd_packed(const terra_swin_desc* desc, const void* qkv, const float* bias_table, const void* o,
+                               const float* lse, const void* d_o, void* dqkv, float* dbias,
+                               void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Forward pass without a workspace argument.  (The paper has no counterpart: this exists for the way the
  * library is embedded, not for the method.)
  *

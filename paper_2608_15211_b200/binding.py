@@ -18,7 +18,7 @@ TERRA_OK = 0
 EXPORTS = ("terra_route_sizes", "terra_window_route", "terra_swin_workspace_bytes", "terra_swin_attn_fwd",
            "terra_swin_attn_fwd_noalloc", "terra_swin_attn_bwd", "terra_swin_check", "terra_strerror", "terra_last_cuda_error",
            "terra_launch_count", "terra_selftest_bounded_wait", "terra_profile_enable", "terra_profile_count", "terra_profile_get",
-           "terra_fixed_assignment_padding", "terra_ragged_window_range")
+           "terra_fixed_assignment_padding", "terra_ragged_window_range", "terra_swin_attn_fwd_packed", "terra_swin_attn_bwd_packed")
 
 
 class TerraError(RuntimeError):
@@ -54,8 +54,10 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
     lib.terra_swin_attn_fwd.argtypes = [dp] + [vp] * 6 + [vp, ctypes.c_size_t, vp]
     lib.terra_swin_attn_bwd.argtypes = [dp] + [vp] * 11 + [vp, ctypes.c_size_t, vp]
     lib.terra_swin_attn_fwd_noalloc.argtypes = [dp] + [vp] * 6 + [vp]
+    lib.terra_swin_attn_fwd_packed.argtypes = [dp] + [vp] * 4 + [vp, ctypes.c_size_t, vp]
+    lib.terra_swin_attn_bwd_packed.argtypes = [dp] + [vp] * 7 + [vp, ctypes.c_size_t, vp]
     for n in ("terra_route_sizes", "terra_window_route", "terra_swin_workspace_bytes", "terra_swin_attn_fwd",
-              "terra_swin_attn_fwd_noalloc", "terra_swin_attn_bwd"):
+              "terra_swin_attn_fwd_noalloc", "terra_swin_attn_bwd", "terra_swin_attn_fwd_packed", "terra_swin_attn_bwd_packed"):
         getattr(lib, n).restype = ctypes.c_int
     lib.terra_swin_check.argtypes = [vp]
     lib.terra_swin_check.restype = ctypes.c_int
@@ -234,3 +236,44 @@ def terra_swin_attn_bwd(desc, q, k, v, bias_table, o, lse, d_o, dq=None, dk=None
                                               _ptr(o), _ptr(lse), _ptr(d_o), _ptr(dq), _ptr(dk), _ptr(dv),
                                               _ptr(dbias), _ptr(workspace), ws_bytes, _stream()))
     return dq, dk, dv, dbias
+
+
+def terra_swin_attn_fwd_packed(desc, qkv, bias_table, o=None, lse=None, workspace=None):
+    """Forward on the packed projection output.  qkv bf16 [B, H, W, 3, heads, head_dim] (q, k, v in that order);
+    returns (o bf16 [B, H, W, heads, head_dim], lse fp32 [B, H, W, heads])."""
+    n = desc.B * desc.H * desc.W * desc.heads
+    _expect(qkv, torch.bfloat16, 3 * n * desc.head_dim, "qkv")
+    _expect(bias_table, torch.float32, (2 * desc.window - 1) ** 2 * desc.heads, "bias_table")
+    if o is None:
+        o = torch.empty((desc.B, desc.H, desc.W, desc.heads, desc.head_dim), dtype=torch.bfloat16, device=qkv.device)
+    if lse is None:
+        lse = torch.empty((desc.B, desc.H, desc.W, desc.heads), dtype=torch.float32, device=qkv.device)
+    _expect(o, torch.bfloat16, n * desc.head_dim, "o")
+    _expect(lse, torch.float32, n, "lse")
+    if workspace is None:
+        need = terra_swin_workspace_bytes(desc, False)
+        workspace = torch.empty(need, dtype=torch.uint8, device=qkv.device) if need else None
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(load_library().terra_swin_attn_fwd_packed(ctypes.byref(desc), _ptr(qkv), _ptr(bias_table), _ptr(o), _ptr(lse),
+                                                     _ptr(workspace), ws_bytes, _stream()))
+    return o, lse
+
+
+def terra_swin_attn_bwd_packed(desc, qkv, bias_table, o, lse, d_o, dqkv=None, dbias=None, workspace=None):
+    """Backward on the packed layout.  Returns (dqkv bf16 like qkv, dbias fp32 like bias_table)."""
+    n = desc.B * desc.H * desc.W * desc.heads
+    _expect(qkv, torch.bfloat16, 3 * n * desc.head_dim, "qkv")
+    for name, t in (("o", o), ("d_o", d_o)):
+        _expect(t, torch.bfloat16, n * desc.head_dim, name)
+    _expect(lse, torch.float32, n, "lse")
+    _expect(bias_table, torch.float32, (2 * desc.window - 1) ** 2 * desc.heads, "bias_table")
+    dqkv = torch.empty_like(qkv) if dqkv is None else dqkv
+    dbias = torch.empty_like(bias_table) if dbias is None else dbias
+    _expect(dqkv, torch.bfloat16, 3 * n * desc.head_dim, "dqkv")
+    _expect(dbias, torch.float32, bias_table.numel(), "dbias")
+    if workspace is None:
+        workspace = torch.empty(terra_swin_workspace_bytes(desc, True), dtype=torch.uint8, device=qkv.device)
+    ws_bytes = workspace.numel() * workspace.element_size()
+    _check(load_library().terra_swin_attn_bwd_packed(ctypes.byref(desc), _ptr(qkv), _ptr(bias_table), _ptr(o), _ptr(lse),
+                                                     _ptr(d_o), _ptr(dqkv), _ptr(dbias), _ptr(workspace), ws_bytes, _stream()))
+    return dqkv, dbias

@@ -69,6 +69,7 @@ static int make_geo(const terra_swin_desc* d, bool for_attention, Geo* out) {
     Geo g;
     g.B = d->B; g.H = d->H; g.W = d->W;
     g.heads = d->heads; g.d = d->head_dim; g.w = d->window;
+    g.ts = d->heads * d->head_dim;
     g.sh = d->shift_h % d->H; g.sw = d->shift_w % d->W;
     g.ph = d->periodic_h != 0; g.pw = d->periodic_w != 0;
     g.Mh = (d->H + d->window - 1) / d->window;
@@ -159,12 +160,11 @@ int terra_swin_workspace_bytes(const terra_swin_desc* desc, int backward, size_t
     return TERRA_OK;
 }
 
-int terra_swin_attn_fwd(const terra_swin_desc* desc, const void* q, const void* k, const void* v,
-                        const float* bias_table, void* o, float* lse,
-                        void* workspace, size_t workspace_bytes, void* stream) {
-    Geo g;
-    int rc = make_geo(desc, true, &g);
-    if (rc) return rc;
+// forward with q, k, v given as three pointers and one token stride (g.ts elements)
+static int fwd_call(const Geo& g, const void* q, const void* k, const void* v,
+                    const float* bias_table, void* o, float* lse,
+                    void* workspace, size_t workspace_bytes, void* stream) {
+    int rc;
     if (!q || !k || !v || !bias_table || !o || !lse) return TERRA_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o) || !aligned16(bias_table) || !aligned16(lse))
         return TERRA_ERR_ALIGNMENT;
@@ -182,13 +182,33 @@ int terra_swin_attn_fwd(const terra_swin_desc* desc, const void* q, const void* 
     return e == cudaSuccess ? TERRA_OK : cuda_fail(e, "terra_swin_attn_fwd");
 }
 
-int terra_swin_attn_bwd(const terra_swin_desc* desc, const void* q, const void* k, const void* v,
-                        const float* bias_table, const void* o, const float* lse, const void* d_o,
-                        void* dq, void* dk, void* dv, float* dbias,
+int terra_swin_attn_fwd(const terra_swin_desc* desc, const void* q, const void* k, const void* v,
+                        const float* bias_table, void* o, float* lse,
                         void* workspace, size_t workspace_bytes, void* stream) {
     Geo g;
     int rc = make_geo(desc, true, &g);
     if (rc) return rc;
+    return fwd_call(g, q, k, v, bias_table, o, lse, workspace, workspace_bytes, stream);
+}
+
+int terra_swin_attn_fwd_packed(const terra_swin_desc* desc, const void* qkv, const float* bias_table, void* o, float* lse,
+                               void* workspace, size_t workspace_bytes, void* stream) {
+    Geo g;
+    int rc = make_geo(desc, true, &g);
+    if (rc) return rc;
+    if (!qkv) return TERRA_ERR_INVALID_ARG;
+    const size_t hd = (size_t)g.heads * g.d;
+    g.ts = (int)(3 * hd);
+    const __nv_bfloat16* base = reinterpret_cast<const __nv_bfloat16*>(qkv);
+    return fwd_call(g, base, base + hd, base + 2 * hd, bias_table, o, lse, workspace, workspace_bytes, stream);
+}
+
+// backward with q, k, v and dq, dk, dv given as pointers and one token stride (g.ts elements)
+static int bwd_call(const Geo& g, const void* q, const void* k, const void* v,
+                    const float* bias_table, const void* o, const float* lse, const void* d_o,
+                    void* dq, void* dk, void* dv, float* dbias,
+                    void* workspace, size_t workspace_bytes, void* stream) {
+    int rc;
     if (!q || !k || !v || !bias_table || !o || !lse || !d_o || !dq || !dk || !dv || !dbias)
         return TERRA_ERR_INVALID_ARG;
     const void* ptrs[] = {q, k, v, bias_table, o, lse, d_o, dq, dk, dv, dbias};
@@ -209,6 +229,31 @@ int terra_swin_attn_bwd(const terra_swin_desc* desc, const void* q, const void* 
     if (e != cudaSuccess) return cuda_fail(e, "terra_swin_attn_bwd (delta)");
     e = launch_bwd_mma(g, q, k, v, bias_table, lse, delta, d_o, dq, dk, dv, dbias, sms, st);
     return e == cudaSuccess ? TERRA_OK : cuda_fail(e, "terra_swin_attn_bwd");
+}
+
+int terra_swin_attn_bwd(const terra_swin_desc* desc, const void* q, const void* k, const void* v,
+                        const float* bias_table, const void* o, const float* lse, const void* d_o,
+                        void* dq, void* dk, void* dv, float* dbias,
+                        void* workspace, size_t workspace_bytes, void* stream) {
+    Geo g;
+    int rc = make_geo(desc, true, &g);
+    if (rc) return rc;
+    return bwd_call(g, q, k, v, bias_table, o, lse, d_o, dq, dk, dv, dbias, workspace, workspace_bytes, stream);
+}
+
+int terra_swin_attn_bwd_packed(const terra_swin_desc* desc, const void* qkv, const float* bias_table, const void* o,
+                               const float* lse, const void* d_o, void* dqkv, float* dbias,
+                               void* workspace, size_t workspace_bytes, void* stream) {
+    Geo g;
+    int rc = make_geo(desc, true, &g);
+    if (rc) return rc;
+    if (!qkv || !dqkv) return TERRA_ERR_INVALID_ARG;
+    const size_t hd = (size_t)g.heads * g.d;
+    g.ts = (int)(3 * hd);
+    const __nv_bfloat16* base = reinterpret_cast<const __nv_bfloat16*>(qkv);
+    __nv_bfloat16* gbase = reinterpret_cast<__nv_bfloat16*>(dqkv);
+    return bwd_call(g, base, base + hd, base + 2 * hd, bias_table, o, lse, d_o, gbase, gbase + hd, gbase + 2 * hd, dbias,
+                    workspace, workspace_bytes, stream);
 }
 
 int terra_selftest_bounded_wait(long long limit_cycles, void* stream) {

@@ -45,8 +45,8 @@ constexpr int kThreads = 16 * 32;                               // 512 = four wa
 constexpr int kWorkThreads = 256;          // elementwise threads; each arrives once per barrier phase
 constexpr int kRegsLaunch = 128;
 constexpr int kRegsWork = 184;      // elementwise warpgroups after setmaxnreg.inc
-constexpr int kRegsOther = 80;      // MMA + loader warpgroup after setmaxnreg.dec
-constexpr int kRegsEpi = 64;        // read-out warpgroup after setmaxnreg.dec
+constexpr int kRegsOther = 88;      // MMA + loader warpgroup after setmaxnreg.dec
+constexpr int kRegsEpi = 56;        // read-out warpgroup after setmaxnreg.dec
 static_assert(2 * (kRegsWork - kRegsLaunch) <= (kRegsLaunch - kRegsOther) + (kRegsLaunch - kRegsEpi), "register hand-over does not balance");
 
 constexpr int kStages = 2;
@@ -403,7 +403,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                 const int tok_r = __shfl_sync(0xffffffffu, tok, rr);
                 const int4 a = lds_i4(rows_a + tile_off<kD>(rr, c4));
                 if (tok_r >= 0)
-                    *reinterpret_cast<int4*>(out + ((sample_off + (size_t)tok_r) * g.heads + head) * kD + c4 * 8) = a;
+                    *reinterpret_cast<int4*>(out + (sample_off + (size_t)tok_r) * g.ts + head * kD + c4 * 8) = a;
             }
         };
         int kuse = 0, n_tile = 0;
@@ -507,6 +507,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
             // Key rows are interleaved: with M = 4 * (tiles in use) 32-slot groups, lane l of elementwise warp
             // W = 4 t + qd (key row 128 t + 32 qd + l) holds slot 32 ((W + l) mod M) + l (see the bias-gradient updates).
             const int chunk = lt & 3;
+            const int hc = head * kD + chunk * 8;
             const int nrows = x.ntiles * 128;
             const int M = 4 * x.ntiles;
             int a_r = (lt >> 2) / ew, b_r = (lt >> 2) - a_r * ew;
@@ -518,8 +519,10 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                 if (row < x.r.n) {
                     int code, label;
                     const int tok = offset_token_tc(g, x.r, a_r, b_r, code, label);
-                    const size_t off = ((sample_off + (size_t)tok) * g.heads + head) * kD + chunk * 8;
-                    sq = q + off; sk = k + off; sv = v + off; sg = d_o + off;
+                    const size_t t_abs = sample_off + (size_t)tok;
+                    const size_t off = t_abs * g.ts + hc;
+                    sq = q + off; sk = k + off; sv = v + off;
+                    sg = d_o + t_abs * (g.heads * kD) + hc;            // dO is dense even where q, k, v are packed
                     bytes = 16;
                 }
                 const uint32_t so = st_a + tile_off<kD>(row, chunk), sok = st_a + tile_off<kD>(krow, chunk);

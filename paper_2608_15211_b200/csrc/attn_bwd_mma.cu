@@ -24,7 +24,7 @@ constexpr int NTHREADS = 128;
 
 template <int D>
 __device__ __forceinline__ void load_rows(unsigned char* s_tile, const __nv_bfloat16* base, const int* s_tok,
-                                          int slot0, size_t sample_off, int heads, int head, int tid) {
+                                          int slot0, size_t sample_off, int tstride, int head, int tid) {
     constexpr int CPR = D / 8;
     for (int idx = tid; idx < BN * CPR; idx += NTHREADS) {
         int row = idx / CPR, chunk = idx - row * CPR;
@@ -32,7 +32,7 @@ __device__ __forceinline__ void load_rows(unsigned char* s_tile, const __nv_bflo
         const __nv_bfloat16* src = base;
         int bytes = 0;
         if (tok >= 0) {
-            src = base + ((sample_off + (size_t)tok) * heads + head) * D + chunk * 8;
+            src = base + (sample_off + (size_t)tok) * tstride + head * D + chunk * 8;
             bytes = 16;
         }
         cp_async16(smem_u32(s_tile + tile_off<D>(row, chunk)), src, bytes);
@@ -95,14 +95,14 @@ __device__ __forceinline__ void stage_rows(unsigned char* tile, const float (&ac
 
 template <int D>
 __device__ __forceinline__ void scatter_rows(const unsigned char* tile, __nv_bfloat16* dst, const int* s_tok, int slot0,
-                                             int n, size_t sample_off, int heads, int head, int tid) {
+                                             int n, size_t sample_off, int tstride, int head, int tid) {
     constexpr int CPR = D / 8;
     for (int idx = tid; idx < BM * CPR; idx += NTHREADS) {
         int row = idx / CPR, chunk = idx - row * CPR;
         int slot = slot0 + row;
         if (slot < n) {
             uint4 val = *reinterpret_cast<const uint4*>(tile + tile_off<D>(row, chunk));
-            *reinterpret_cast<uint4*>(dst + ((sample_off + (size_t)s_tok[slot]) * heads + head) * D + chunk * 8) = val;
+            *reinterpret_cast<uint4*>(dst + (sample_off + (size_t)s_tok[slot]) * tstride + head * D + chunk * 8) = val;
         }
     }
 }
@@ -155,6 +155,8 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
     const __nv_bfloat16* own2 = KV ? v : d_o;
     const __nv_bfloat16* str1 = KV ? q : k;
     const __nv_bfloat16* str2 = KV ? d_o : v;
+    // token strides: q, k, v and the gradients may be slices of a packed tensor; dO is dense
+    const int ts_own2 = KV ? g.ts : g.heads * D, ts_str2 = KV ? g.heads * D : g.ts;
 
     for (int i = tid; i < nbias; i += NTHREADS) {
         s_bias[i] = bias[(size_t)i * g.heads + head] * kLog2e;
@@ -191,10 +193,10 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
         }
         __syncthreads();
 
-        load_rows<D>(s_r1, own1, s_tok, r0, sample_off, g.heads, head, tid);
-        load_rows<D>(s_r2, own2, s_tok, r0, sample_off, g.heads, head, tid);
-        load_rows<D>(s_c1, str1, s_tok, 0, sample_off, g.heads, head, tid);
-        load_rows<D>(s_c2, str2, s_tok, 0, sample_off, g.heads, head, tid);
+        load_rows<D>(s_r1, own1, s_tok, r0, sample_off, g.ts, head, tid);
+        load_rows<D>(s_r2, own2, s_tok, r0, sample_off, ts_own2, head, tid);
+        load_rows<D>(s_c1, str1, s_tok, 0, sample_off, g.ts, head, tid);
+        load_rows<D>(s_c2, str2, s_tok, 0, sample_off, ts_str2, head, tid);
         cp_async_commit();
 
         uint32_t f1[KS][4], f2[KS][4];
@@ -216,8 +218,8 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
         for (int blk = 0; blk < nblk; ++blk) {
             const int stage = blk & 1;
             if (blk + 1 < nblk) {
-                load_rows<D>(s_c1 + (stage ^ 1) * TILE_BYTES, str1, s_tok, (blk + 1) * BN, sample_off, g.heads, head, tid);
-                load_rows<D>(s_c2 + (stage ^ 1) * TILE_BYTES, str2, s_tok, (blk + 1) * BN, sample_off, g.heads, head, tid);
+                load_rows<D>(s_c1 + (stage ^ 1) * TILE_BYTES, str1, s_tok, (blk + 1) * BN, sample_off, g.ts, head, tid);
+                load_rows<D>(s_c2 + (stage ^ 1) * TILE_BYTES, str2, s_tok, (blk + 1) * BN, sample_off, ts_str2, head, tid);
                 cp_async_commit();
                 cp_async_wait<1>();
             } else {
@@ -342,8 +344,8 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
         stage_rows<D>(s_r1, acc1, scale, warp, gq, tq);
         if constexpr (KV) stage_rows<D>(s_r2, acc2, 1.f, warp, gq, tq);
         __syncthreads();
-        scatter_rows<D>(s_r1, out1, s_tok, r0, r.n, sample_off, g.heads, head, tid);
-        if constexpr (KV) scatter_rows<D>(s_r2, out2, s_tok, r0, r.n, sample_off, g.heads, head, tid);
+        scatter_rows<D>(s_r1, out1, s_tok, r0, r.n, sample_off, g.ts, head, tid);
+        if constexpr (KV) scatter_rows<D>(s_r2, out2, s_tok, r0, r.n, sample_off, g.ts, head, tid);
     }
 
     if (!KV) {

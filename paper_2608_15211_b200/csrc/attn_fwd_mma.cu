@@ -19,7 +19,7 @@ constexpr int NTHREADS = 128;
 
 template <int D>
 __device__ __forceinline__ void load_rows(unsigned char* s_tile, const __nv_bfloat16* base, const int* s_tok,
-                                          int slot0, size_t sample_off, int heads, int head, int tid) {
+                                          int slot0, size_t sample_off, int tstride, int head, int tid) {
     constexpr int CPR = D / 8;
     for (int idx = tid; idx < BN * CPR; idx += NTHREADS) {
         int row = idx / CPR, chunk = idx - row * CPR;
@@ -27,7 +27,7 @@ __device__ __forceinline__ void load_rows(unsigned char* s_tile, const __nv_bflo
         const __nv_bfloat16* src = base;
         int bytes = 0;
         if (tok >= 0) {
-            src = base + ((sample_off + (size_t)tok) * heads + head) * D + chunk * 8;
+            src = base + (sample_off + (size_t)tok) * tstride + head * D + chunk * 8;
             bytes = 16;
         }
         cp_async16(smem_u32(s_tile + tile_off<D>(row, chunk)), src, bytes);
@@ -78,9 +78,9 @@ swin_fwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
     for (int i = tid; i < nbias; i += NTHREADS) s_bias[i] = bias[(size_t)i * g.heads + head] * kLog2e;
     __syncthreads();
 
-    load_rows<D>(s_q, q, s_tok, q0, sample_off, g.heads, head, tid);
-    load_rows<D>(s_k, k, s_tok, 0, sample_off, g.heads, head, tid);
-    load_rows<D>(s_v, v, s_tok, 0, sample_off, g.heads, head, tid);
+    load_rows<D>(s_q, q, s_tok, q0, sample_off, g.ts, head, tid);
+    load_rows<D>(s_k, k, s_tok, 0, sample_off, g.ts, head, tid);
+    load_rows<D>(s_v, v, s_tok, 0, sample_off, g.ts, head, tid);
     cp_async_commit();
 
     uint32_t qf[KS][4];
@@ -98,8 +98,8 @@ swin_fwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
     for (int kb = 0; kb < nkb; ++kb) {
         const int stage = kb & 1;
         if (kb + 1 < nkb) {
-            load_rows<D>(s_k + (stage ^ 1) * TILE_BYTES, k, s_tok, (kb + 1) * BN, sample_off, g.heads, head, tid);
-            load_rows<D>(s_v + (stage ^ 1) * TILE_BYTES, v, s_tok, (kb + 1) * BN, sample_off, g.heads, head, tid);
+            load_rows<D>(s_k + (stage ^ 1) * TILE_BYTES, k, s_tok, (kb + 1) * BN, sample_off, g.ts, head, tid);
+            load_rows<D>(s_v + (stage ^ 1) * TILE_BYTES, v, s_tok, (kb + 1) * BN, sample_off, g.ts, head, tid);
             cp_async_commit();
             cp_async_wait<1>();
         } else {

@@ -392,7 +392,7 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
                 if (row < x.r.n) {
                     int code, label;
                     const int tok = offset_token_tc(g, x.r, a_r, b_r, code, label);
-                    const size_t off = ((sample_off + (size_t)tok) * g.heads + x.head) * kD + chunk * 8;
+                    const size_t off = (sample_off + (size_t)tok) * g.ts + x.head * kD + chunk * 8;
                     sq = q + off; sk = k + off; sv = v + off;
                     bytes = 16;
                 }

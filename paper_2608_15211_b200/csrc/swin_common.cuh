@@ -10,6 +10,8 @@ namespace terra {
 struct Geo {
     int B, H, W;          // batch, token grid (H_T x W_T)
     int heads, d;         // heads, head dim
+    int ts;               // elements between consecutive tokens of q, k, v (and of dq, dk, dv): heads * d for separate
+                          // dense tensors, 3 * heads * d for the packed [B, H, W, 3, heads, d] layout; o, dO, lse are dense
     int w;                // window side
     int sh, sw;           // shifts, already reduced mod H / mod W
     int ph, pw;           // periodic flags
