@@ -45,8 +45,8 @@ constexpr int kThreads = 16 * 32;                               // 512 = four wa
 constexpr int kWorkThreads = 256;          // elementwise threads; each arrives once per barrier phase
 constexpr int kRegsLaunch = 128;
 constexpr int kRegsWork = 184;      // elementwise warpgroups after setmaxnreg.inc
-constexpr int kRegsOther = 88;      // MMA + loader warpgroup after setmaxnreg.dec
-constexpr int kRegsEpi = 56;        // read-out warpgroup after setmaxnreg.dec
+constexpr int kRegsOther = 80;      // MMA + loader warpgroup after setmaxnreg.dec
+constexpr int kRegsEpi = 64;        // read-out warpgroup after setmaxnreg.dec
 static_assert(2 * (kRegsWork - kRegsLaunch) <= (kRegsLaunch - kRegsOther) + (kRegsLaunch - kRegsEpi), "register hand-over does not balance");
 
 constexpr int kStages = 2;
@@ -87,6 +87,11 @@ constexpr int kColDK = 288;
 constexpr int kColDQ = 384;         // dQ of query pair p at 384 + 32 p
 
 __device__ __forceinline__ int code_stride(int w) { return w + 32; }
+
+// Key rows of a tile are interleaved over the elementwise warps: lane l of warp W = 4 t + quarter holds slot
+// 32 ((W + c l) mod M) + l, M = 4 * (tiles in use).  c = 1, except c = 5 for two-tile windows whose side does not
+// divide 32 (see the bias-gradient updates in the kernel).
+__device__ __forceinline__ int key_interleave(int w, int ntiles) { return (ntiles == 2 && (32 % w) != 0) ? 5 : 1; }
 
 struct Item {
     int b, win;
@@ -424,7 +429,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                 ok = mbar_wait_all(bar_acc(set), (n_tile >> 1) & 1, cta_abort);
                 if (!ok) break;
                 tc_fence_after();
-                const int slot = 32 * ((4 * t + quarter + lane) & (4 * ntiles - 1)) + lane;      // interleaved key order
+                const int slot = 32 * ((4 * t + quarter + key_interleave(g.w, ntiles) * lane) & (4 * ntiles - 1)) + lane;      // interleaved key order
                 const int tok = lds_i32(st_a + kOffTok + 4 * slot);
                 const uint32_t rows_a = st_a + (uint32_t)((t * 128 + 32 * quarter) * kRowBytes);
                 stage_row(tq + kColDV + 64 * set, rows_a + kOffV, 1.f);
@@ -510,10 +515,11 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
             const int hc = head * kD + chunk * 8;
             const int nrows = x.ntiles * 128;
             const int M = 4 * x.ntiles;
+            const int kc = key_interleave(g.w, x.ntiles);
             int a_r = (lt >> 2) / ew, b_r = (lt >> 2) - a_r * ew;
             for (int row = lt >> 2; row < nrows; row += kLoaderThreads / 4, a_r += q_r, b_r += r_r) {
                 if (b_r >= ew) { b_r -= ew; ++a_r; }
-                const int kl = row & 31, kw = ((row >> 5) - kl) & (M - 1), krow = 128 * (kw >> 2) + 32 * (kw & 3) + kl;
+                const int kl = row & 31, kw = ((row >> 5) - kc * kl) & (M - 1), krow = 128 * (kw >> 2) + 32 * (kw & 3) + kl;
                 const __nv_bfloat16 *sq = q, *sk = k, *sv = v, *sg = d_o;
                 int bytes = 0;
                 if (row < x.r.n) {
@@ -723,7 +729,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
             for (int t = 0; t < x.ntiles && ok; ++t) {
                 const int krow = 32 * quarter + lane;            // key row inside the tile
                 const int M = 4 * x.ntiles;
-                const int slot = 32 * ((4 * t + quarter + lane) & (M - 1)) + lane;     // interleaved key order
+                const int slot = 32 * ((4 * t + quarter + key_interleave(g.w, x.ntiles) * lane) & (M - 1)) + lane;     // interleaved key order
                 // Bias-gradient updates.  In a full-width window (width = w) the bias code of a slot is the slot
                 // number plus 32 per window row, so code mod 32 = slot mod 32 = lane: the 32 updates of one warp
                 // instruction (32 keys, one query) fall into 32 different banks and entries.  If w also divides 32
@@ -731,9 +737,16 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                 // the same group with lanes congruent mod M, i.e. >= M slots = codes apart, keys in different rows
                 // are >= 33 codes apart, and G <= min(M, w) consecutive queries of a group aligned to G sit in one
                 // window row 1 .. G - 1 codes apart: the 32 x G updates of such a query group never meet and are
-                // issued together.  Other windows are updated one query at a time.
+                // issued together.  For sides that do not divide 32 the slots 32 g - 1 and 32 g (lanes 31 and 0 of one
+                // warp under c = 1) may share a window row; with c = 5 and two tiles (M = 8) any two lanes of a warp
+                // hold slots at least 5 apart, and groups of 4 queries are collision-free for every full-width
+                // window of side 9 .. 16 (checked exhaustively on the host over all heights; the parity tests cover
+                // sides 12 and 14).  Other windows are updated one query at a time.
                 int rmw_mode = 1;
-                if (x.r.ew == g.w && (32 % g.w) == 0 && g.w >= 4) rmw_mode = (M == 8 && g.w >= 8) ? 8 : 4;
+                if (x.r.ew == g.w && g.w >= 4) {
+                    if ((32 % g.w) == 0) rmw_mode = (M == 8 && g.w >= 8) ? 8 : 4;
+                    else if (M == 8) rmw_mode = 4;
+                }
                 const bool row16 = g.w == 16 && x.r.n == 256 && !x.masked;    // full 16 x 16 window: update groups of 8 apply as well
                 const int coloff_i = lds_i32(st_a + kOffColOff + 4 * slot);
                 const int tok = lds_i32(st_a + kOffTok + 4 * slot);
