@@ -305,7 +305,7 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(bar_full(s), kLoaderThreads);
-            mbar_init(bar_empty(s), 1);
+            mbar_init(bar_empty(s), 1 + 128);      // the issuer's commit + the second softmax warpgroup (see its loop)
         }
         for (int t = 0; t < 2; ++t) {
             mbar_init(bar_sready(t), 1);
@@ -543,10 +543,17 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
         ItemCursor cur_it = cursor_init(blockIdx.x, gridDim.x, g.heads, g.Mw, g.Mh);
         for (long long it = blockIdx.x; it < n_items; it += gridDim.x, ++kuse, cursor_advance(cur_it, g.heads, g.Mw, g.Mh)) {
             const Item x = make_item(g, cur_it);
-            if (wg >= x.ntiles) continue;
             const int s = kuse % kStages;
             const uint32_t st_a = smem0 + s * kStageBytes;
+            // Every warpgroup follows the stage ring item by item, also the second one through items that have no
+            // second query tile: a wait names its barrier phase by parity only, so a warpgroup that skipped ahead
+            // by a whole turn of the ring would take an older phase for the one it wants.  Its arrival on the
+            // stage's release barrier keeps the loaders from lapping it the other way round.
             if (!__all_sync(0xffffffffu, mbar_wait(bar_full(s), (kuse / kStages) & 1, cta_abort))) break;
+            if (wg >= x.ntiles) {
+                mbar_arrive(bar_empty(s));
+                continue;
+            }
             const int rmeta = lds_i32(st_a + kOffRowMeta + 4 * slot);
             const int tok = lds_i32(st_a + kOffRowTok + 4 * slot);
             const uint32_t bias_i = st_a + kOffBias + 4 * meta_code(rmeta);
@@ -570,6 +577,7 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
             tc_fence_before();
             if (x.npad <= 128) mbar_arrive(bar_phalf(wg));      // short rows: both halves at once
             mbar_arrive(bar_pready(wg));
+            if (wg == 1) mbar_arrive(bar_empty(s));            // this warpgroup has read all it needs from the stage
 
             const size_t row_off = ((size_t)x.b * HW + (size_t)(tok < 0 ? 0 : tok)) * g.heads + x.head;
 
