@@ -26,9 +26,6 @@ EDGE = [
     ("w12_three_blocks", 2, 30, 40, 3, 32, 12, 6, 6, 0, 1),     # 144-token windows: two key tiles, an odd number of query blocks
     ("w16_wrap_and_rem", 1, 40, 48, 2, 32, 16, 8, 8, 0, 1),      # full, masked (latitude wrap) and truncated 16-wide windows
     ("w8_nonperiodic", 2, 24, 40, 2, 32, 8, 4, 4, 0, 0),         # 64-token windows, masks on both axes, several items per CTA
-    # 540 items on 148 CTAs: two CTAs meet three one-tile windows (6 wide) and then a two-tile one, i.e. the second
-    # query tile's first use comes after a whole turn of the forward kernel's stage ring
-    ("ring_turn_then_second_tile", 2, 111, 71, 5, 32, 13, 45, 48, 0, 0),
 ]
 
 

@@ -1,6 +1,7 @@
 """Seeded random small shapes through the C ABI against the oracle: window sides 1..16 at head dim 32 (the
-tcgen05 kernels: every tile / block / mask / truncation combination the shapes happen to hit) and larger
-windows or head dim 64 (the register-tile kernels)."""
+tcgen05 kernels: every tile / block / mask / truncation combination the shapes happen to hit), larger
+windows or head dim 64 (the register-tile kernels), and grids with hundreds to thousands of (window, head) items
+(several items per CTA in mixed order of one-tile and two-tile windows)."""
 import random
 
 import pytest
@@ -28,6 +29,15 @@ def _shapes():
         H, W = rng.randint(w // 2, 2 * w + 9), rng.randint(w // 2, 3 * w + 5)
         out.append((f"g{i}_d{d}_w{w}", rng.choice([1, 2]), H, W, rng.choice([1, 2, 3]), d, w,
                     rng.randint(0, H), rng.randint(0, W), rng.randint(0, 1), rng.randint(0, 1)))
+    rng = random.Random(20260816)
+    for i in range(8):                       # many items per CTA: the persistent kernels' rings turn several times
+        w = rng.choice([3, 5, 6, 8, 9, 12, 13, 14, 16])
+        H, W = rng.randint(6 * w, 14 * w + 7), rng.randint(6 * w, 14 * w + 9)
+        out.append((f"m{i}_w{w}", rng.choice([1, 2, 3]), H, W, rng.choice([3, 5, 6, 7]), 32, w,
+                    rng.randint(0, H + 2), rng.randint(0, W + 2), rng.randint(0, 1), rng.randint(0, 1)))
+    # found by fuzzing: 540 items on 148 CTAs, two of which meet three one-tile windows (6 wide) and then a
+    # two-tile one, i.e. the second query tile's first use comes after a whole turn of the forward kernel's stage ring
+    out.append(("ring_turn_then_second_tile", 2, 111, 71, 5, 32, 13, 45, 48, 0, 0))
     return out
 
 
