@@ -11,13 +11,14 @@
 //          32 lanes of one instruction are 32 different keys at one query = 32 different entries; the keys of
 //          a tile are interleaved over the warps so that 4 or 8 consecutive queries can be updated together).
 // Roles: warps 0..7 elementwise, warp 8 issues every MMA (the whole warp runs the loop, one elected lane
-// issues), warps 9..11 gather the window's rows with cp.async into the 64-byte-swizzled operand layout.
+// issues), warps 9..11 gather the window's rows with cp.async into the 64-byte-swizzled operand layout,
+// warps 12..15 read the finished accumulators out of TMEM and store them.
 // The eight elementwise warps work on ONE key tile at a time: warps w and w + 4 share the 32 key rows of TMEM
 // lane quarter w & 3 and split each block's four 16-column steps (steps 0, 2 and steps 1, 3).
 // The CTA's blocks form one sequence across tiles and items; S^T / dP^T of a block are issued two blocks ahead.
 // TMEM columns: two [S 64 | dP 64] buffers, two (dV, dK) accumulator sets, two dQ accumulators (queries
-// 0..127 and 128..255).  A tile's dV / dK and an item's dQ are read out one block later, so that no
-// elementwise warp waits for the last MMAs of the tile.
+// 0..127 and 128..255).  A tile's dV / dK and an item's dQ are read out by the read-out warps as soon as their
+// last MMA has completed; the elementwise warps never wait for them.
 // Outputs leave through the item's own operand tiles in shared memory (dK over the K rows, dV over V, dQ
 // over Q, once the MMAs that read them are complete), so that whole 64-byte rows are stored.
 // CTAs are bound to one head (grid = heads x CTAs per head): the head's bias table is staged once per CTA
