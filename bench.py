@@ -178,8 +178,8 @@ def run_reference(args, cfg):
 # captures summarised under profiles/ (config 3 cut to 254 token rows, 13 056 items); traffic grows in
 # proportion to the item count, so a full launch is this figure times its items.  None = not captured.
 NCU_DRAM_BYTES_PER_ITEM = {
-    "swin_fwd_tc_kernel": 63616,
-    "swin_bwd_fused_kernel": 112215,
+    "swin_fwd_tc_kernel": 63620,
+    "swin_bwd_fused_kernel": 112255,
 }
 
 
