@@ -108,8 +108,13 @@ static bool force_register_path() {
     return on;
 }
 
+static bool use_fwd_tc64(const Geo& g) { return fwd_tc64_supported(g) && !force_register_path(); }
+
 static size_t fwd_bytes(const Geo& g) {
-    return (fwd_tc_supported(g) && !force_register_path()) ? align_up(fwd_tc_workspace_bytes(g), 256) : 0;
+    if (force_register_path()) return 0;
+    if (fwd_tc_supported(g)) return align_up(fwd_tc_workspace_bytes(g), 256);
+    if (use_fwd_tc64(g)) return align_up(fwd_tc64_workspace_bytes(g), 256);
+    return 0;
 }
 
 static bool use_bwd_tc(const Geo& g) { return bwd_tc_supported(g) && !force_register_path(); }
@@ -175,7 +180,9 @@ static int fwd_call(const Geo& g, const void* q, const void* k, const void* v,
     rc = device_props(&sms);
     if (rc) return rc;
     cudaError_t e;
-    if (need > 0)
+    if (need > 0 && use_fwd_tc64(g) && !fwd_tc_supported(g))
+        e = launch_fwd_tc64(g, q, k, v, bias_table, o, lse, workspace, sms, (cudaStream_t)stream);
+    else if (need > 0)
         e = launch_fwd_tc(g, q, k, v, bias_table, o, lse, workspace, sms, (cudaStream_t)stream);
     else
         e = launch_fwd_mma(g, q, k, v, bias_table, o, lse, (cudaStream_t)stream);
@@ -272,7 +279,10 @@ int terra_swin_check(void* stream) {
     int timed_out_bwd = 0;
     e = read_bwd_tc_status(&timed_out_bwd);
     if (e != cudaSuccess) return cuda_fail(e, "terra_swin_check");
-    return (timed_out || timed_out_bwd) ? TERRA_ERR_DEVICE_TIMEOUT : TERRA_OK;
+    int timed_out_64 = 0;
+    e = read_fwd_tc64_status(&timed_out_64);
+    if (e != cudaSuccess) return cuda_fail(e, "terra_swin_check");
+    return (timed_out || timed_out_bwd || timed_out_64) ? TERRA_ERR_DEVICE_TIMEOUT : TERRA_OK;
 }
 
 int terra_profile_enable(int on) {

@@ -1,0 +1,628 @@
+// Forward shifted-window attention on the tcgen05 tensor cores for head dim 64 and windows of up to 1024 tokens
+// (window side <= 32): the large-window regime, where a score row no longer fits tensor memory.
+//
+// One persistent CTA per SM, bound to one head, walks over (batch, window, pair of 128-row query tiles) items.
+// The window's keys are streamed in chunks of 128 through a ring of shared-memory slots, twice:
+//   pass A   S = Q K_c^T per chunk, the softmax threads only take the row maximum of the raw scores
+//            (the same upper bound max_j(raw) * scale + max(bias) as in the small-window kernel);
+//   pass B   S = Q K_c^T again, P = exp2(S * scale + bias - m) written back over S as bf16, O += P [V_c | 1]
+//            (16 columns of ones behind V: the accumulator's columns 64..79 carry the row sums of P).
+// Recomputing S costs tensor-pipe time, of which there is plenty next to the exp work, and spares the running
+// rescale of O of an online softmax.
+// Roles: warps 0-3 / 4-7 softmax warpgroups (one thread per query row of the pair's first / second tile),
+// warp 8 issues every tcgen05.mma (whole warp runs the loop, one elected lane issues), warps 9-11 gather rows
+// with cp.async, undoing the roll.  Head dim 64 is kept as two 32-column halves in the 64-byte-swizzled operand
+// layout of the small-window kernels (lo | hi regions), so that the same descriptors serve.
+// TMEM: columns [256 t, 256 t + 256) belong to query tile t of the pair: S chunk (fp32, 128 columns), overwritten
+// in place by bf16 P (64 columns); the O accumulator (64 + 16 columns) at +128.
+// Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, all roles leave their loops, TMEM is
+// released and the host reads the device status word.  Every role follows every ring item by item.
+#include "swin_common.cuh"
+#include "swin_kernels.h"
+#include "tc_common.cuh"
+
+namespace terra {
+
+__device__ int g_fwd_tc64_timeout = 0;   // set when a bounded wait expired in any CTA of the kernel below
+
+namespace {
+
+using namespace tc;
+
+constexpr int kMmaWarp = 8;
+constexpr int kLoaderWarp0 = 9;
+constexpr int kLoaderThreads = 96;
+constexpr int kThreads = 384;
+constexpr int kRegsLaunch = 168, kRegsSoftmax = 216, kRegsOther = 64;
+static_assert(2 * (kRegsSoftmax - kRegsLaunch) <= (kRegsLaunch - kRegsOther), "register hand-over does not balance");
+
+constexpr int kD = 64;
+constexpr int kHalfBytes = 64;                        // one 32-column half of a row
+constexpr int kQRows = 256, kChunk = 128;
+constexpr int kQStages = 2, kSlots = 3;
+constexpr int kQHalf = kQRows * kHalfBytes;           // 16384
+constexpr int kQStageBytes = 2 * kQHalf;              // Q lo | Q hi
+constexpr int kKHalf = kChunk * kHalfBytes;           // 8192
+constexpr int kOffKlo = 0, kOffKhi = kKHalf, kOffVlo = 2 * kKHalf, kOffVhi = 3 * kKHalf, kOffOnes = 4 * kKHalf;
+constexpr int kSlotBytes = 5 * kKHalf;                // 40960
+constexpr int kOffSlots = kQStages * kQStageBytes;                      // 65536
+constexpr int kOffKeyMeta = kOffSlots + kSlots * kSlotBytes;            // per slot: kc[128], klab[128]
+constexpr int kOffRowMeta = kOffKeyMeta + kSlots * 1024;                // per Q stage: rowmeta[256], rowtok[256]
+constexpr int kBiasFloats = 6048;                     // 3 c0 + 3 with c0 = 31 * 65 (window side 32)
+constexpr int kOffBias = kOffRowMeta + kQStages * 2048;
+constexpr int kOffBars = ((kOffBias + kBiasFloats * 4 + 1023) / 1024) * 1024;
+constexpr int kSmemBytes = kOffBars + 1024;
+static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
+constexpr int kColO = 128;
+constexpr int kNO = kD + 16;
+
+__device__ __forceinline__ int code_stride(int w) { return w + 32; }
+
+struct Item {
+    int b, pair;
+    WindowRef r;
+    int npad;      // key slots rounded up to 16
+    int nch;       // 128-key chunks
+    int ntiles;    // query tiles of this pair that exist (0, 1 or 2)
+    bool masked;
+};
+
+__device__ __forceinline__ Item make_item(const Geo& g, const ItemCursor& c) {
+    Item x;
+    x.pair = c.head;                                  // the cursor's fastest digit counts tile pairs here
+    x.b = c.b;
+    x.r = window_ref_rc(g, c.wr, c.wc);
+    x.npad = (x.r.n + 15) & ~15;
+    x.nch = (x.npad + kChunk - 1) / kChunk;
+    const int tiles = (x.r.n + 127) >> 7;
+    x.ntiles = min(2, max(0, tiles - 2 * x.pair));
+    const int r0 = x.r.wr * g.w, c0 = x.r.wc * g.w;
+    const bool mh = !g.ph && g.sh > 0 && r0 < g.H - g.sh && r0 + x.r.eh > g.H - g.sh;
+    const bool mw = !g.pw && g.sw > 0 && c0 < g.W - g.sw && c0 + x.r.ew > g.W - g.sw;
+    x.masked = mh || mw;
+    return x;
+}
+
+__device__ __forceinline__ int offset_token(const Geo& g, const WindowRef& r, int a, int b, int& code, int& label) {
+    int u = r.wr * g.w + a + g.sh;
+    if (u >= g.H) u -= g.H;
+    int v = r.wc * g.w + b + g.sw;
+    if (v >= g.W) v -= g.W;
+    label = ((!g.ph && u < g.sh) ? 2 : 0) + ((!g.pw && v < g.sw) ? 1 : 0);
+    code = a * code_stride(g.w) + b;
+    return u * g.W + v;
+}
+
+__device__ __forceinline__ float lds_f32(uint32_t addr) {
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ int4 lds_i4(uint32_t addr) {
+    int4 v;
+    asm volatile("ld.shared.v4.s32 {%0,%1,%2,%3}, [%4];\n" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ int lds_i32(uint32_t addr) {
+    int v;
+    asm volatile("ld.shared.s32 %0, [%1];\n" : "=r"(v) : "r"(addr));
+    return v;
+}
+
+// P for N consecutive key columns of the chunk starting at local column c: exp2(raw * scale + bias - m), packed
+template <int N, bool MASKED>
+__device__ __forceinline__ void softmax_cols(const uint32_t (&r)[N], uint32_t (&pk)[N / 2], int c, uint32_t bias_i,
+                                             uint32_t a_kc, uint32_t a_klab, int label_i, float scale, float neg_m) {
+#pragma unroll
+    for (int e4 = 0; e4 < N / 4; ++e4) {
+        const int4 kc4 = lds_i4(a_kc + 4 * (c + e4 * 4));
+        const int kc[4] = {kc4.x, kc4.y, kc4.z, kc4.w};
+        int kl[4] = {0, 0, 0, 0};
+        if (MASKED) {
+            const int4 kl4 = lds_i4(a_klab + 4 * (c + e4 * 4));
+            kl[0] = kl4.x; kl[1] = kl4.y; kl[2] = kl4.z; kl[3] = kl4.w;
+        }
+        float p[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float bv = lds_f32(bias_i + kc[e]);
+            float xv = fmaf(__uint_as_float(r[e4 * 4 + e]), scale, bv) + neg_m;
+            if (MASKED && kl[e] != label_i) xv = -INFINITY;
+            p[e] = fast_exp2(xv);
+        }
+        pk[e4 * 2] = pack_bf16(p[0], p[1]);
+        pk[e4 * 2 + 1] = pack_bf16(p[2], p[3]);
+    }
+}
+
+template <int N>
+__device__ __forceinline__ void max_cols(const uint32_t (&r)[N], float (&mx)[4]) {
+#pragma unroll
+    for (int e = 0; e < N; e += 8) {
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+            mx[a] = fmaxf(mx[a], fmaxf(__uint_as_float(r[e + 2 * a]), __uint_as_float(r[e + 2 * a + 1])));
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
+                     const __nv_bfloat16* __restrict__ v, const float* __restrict__ bias_prep,
+                     __nv_bfloat16* __restrict__ o, float* __restrict__ lse, long long n_items, int ctas_per_head,
+                     int max_pairs) {
+    extern __shared__ __align__(1024) unsigned char smem[];
+    const uint32_t smem0 = smem_u32(smem);
+    const uint32_t bar0 = smem0 + kOffBars;
+    auto bar_qfull = [&](int s) { return bar0 + 8u * s; };               // Q rows and row tables of an item are there
+    auto bar_qempty = [&](int s) { return bar0 + 8u * (2 + s); };        // ... and no longer needed
+    auto bar_kvfull = [&](int s) { return bar0 + 8u * (4 + s); };        // a key chunk is in ring slot s
+    auto bar_kvempty = [&](int s) { return bar0 + 8u * (7 + s); };       // ... and every MMA that reads it is complete
+    auto bar_sready = [&](int t) { return bar0 + 8u * (10 + t); };       // S of a chunk is in tile t's columns
+    auto bar_sfree = [&](int t) { return bar0 + 8u * (12 + t); };        // pass A: the softmax threads have read it
+    auto bar_pready = [&](int t) { return bar0 + 8u * (14 + t); };       // pass B: P of the chunk is in TMEM
+    auto bar_oready = [&](int t) { return bar0 + 8u * (16 + t); };       // O of the item is final
+    auto bar_ofree = [&](int t) { return bar0 + 8u * (18 + t); };        // ... and has been read
+    unsigned char* tail = smem + kOffBars + 8 * 20;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail);
+    volatile int* cta_abort = reinterpret_cast<volatile int*>(tail + 8);
+
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int warp = tid >> 5;
+    const int head = blockIdx.x % g.heads;
+    const int cta_in_head = blockIdx.x / g.heads;
+
+    if (tid == 0) {
+        for (int s = 0; s < kQStages; ++s) {
+            mbar_init(bar_qfull(s), kLoaderThreads);
+            mbar_init(bar_qempty(s), 1 + 256);        // the issuer's commit + every softmax thread
+        }
+        for (int s = 0; s < kSlots; ++s) {
+            mbar_init(bar_kvfull(s), kLoaderThreads);
+            mbar_init(bar_kvempty(s), 1);
+        }
+        for (int t = 0; t < 2; ++t) {
+            mbar_init(bar_sready(t), 1);
+            mbar_init(bar_sfree(t), 128);
+            mbar_init(bar_pready(t), 128);
+            mbar_init(bar_oready(t), 1);
+            mbar_init(bar_ofree(t), 128);
+        }
+        *cta_abort = 0;
+        fence_barrier_init();
+    }
+    // the head's prepared bias table; the ones block of every ring slot (first 16 bf16 of a row = 1)
+    for (int i = tid; i < kBiasFloats; i += kThreads)
+        reinterpret_cast<float*>(smem + kOffBias)[i] = bias_prep[(size_t)head * kBiasFloats + i];
+    for (int i = tid; i < kSlots * kChunk * 4; i += kThreads) {
+        const int s = i / (kChunk * 4), rem = i - s * (kChunk * 4), row = rem >> 2, chunk = rem & 3;
+        const uint32_t val = chunk < 2 ? 0x3F803F80u : 0u;
+        *reinterpret_cast<uint4*>(smem + kOffSlots + s * kSlotBytes + kOffOnes + tile_off<32>(row, chunk)) = make_uint4(val, val, val, val);
+    }
+    fence_proxy_async();
+    if (warp == kMmaWarp) {
+        tmem_alloc(smem_u32(tmem_slot), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int cs = code_stride(g.w);
+    const int c0 = (g.w - 1) * (cs + 1);
+    const size_t HW = (size_t)g.H * g.W;
+
+    if (warp >= kMmaWarp) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kRegsOther));
+    if (warp >= kLoaderWarp0) {
+        // ------------------------------------------------------------------ loaders
+        const int lt = (warp - kLoaderWarp0) * 32 + lane;
+        const int j8 = lt & 7;                            // 16-byte chunk of the 128-byte row this thread copies
+        const uint32_t half_off = (j8 >> 2) ? 1u : 0u;    // lo or hi half
+        const int c4 = j8 & 3;
+        int kuse = 0;
+        long long ru = 0;                                 // ring uses so far
+        ItemCursor cur = cursor_init(cta_in_head, ctas_per_head, max_pairs, g.Mw, g.Mh);
+        for (long long it = cta_in_head; it < n_items; it += ctas_per_head, cursor_advance(cur, max_pairs, g.Mw, g.Mh)) {
+            const Item x = make_item(g, cur);
+            if (x.ntiles == 0) continue;
+            const int qs = kuse % kQStages;
+            if (!mbar_wait_all(bar_qempty(qs), ((kuse / kQStages) & 1) ^ 1, cta_abort)) break;
+            const size_t sample_off = (size_t)x.b * HW;
+            const int ew = x.r.ew;
+            // ---- Q rows of the pair (rows without a token as zeros) and the row tables
+            {
+                const uint32_t qb = smem0 + qs * kQStageBytes;
+                int* rowmeta = reinterpret_cast<int*>(smem + kOffRowMeta + qs * 2048);
+                int* rowtok = rowmeta + 256;
+                const int slot0 = x.pair * kQRows;
+                for (int row = lt; row < kQRows; row += kLoaderThreads) {
+                    const int slot = slot0 + row;
+                    int code = 0, label = 0xff, tok = -1;
+                    if (slot < x.r.n) {
+                        const int a = slot / ew;
+                        tok = offset_token(g, x.r, a, slot - a * ew, code, label);
+                    }
+                    rowmeta[row] = code | (label << 16);
+                    rowtok[row] = tok;
+                }
+                const int nrows = x.ntiles * 128;
+                const int q_r = 12 / ew, r_r = 12 - q_r * ew;
+                int slot = slot0 + (lt >> 3);
+                int a_r = slot / ew, b_r = slot - a_r * ew;
+                for (int row = lt >> 3; row < nrows; row += 12, a_r += q_r, b_r += r_r) {
+                    if (b_r >= ew) { b_r -= ew; ++a_r; }
+                    const __nv_bfloat16* src = q;
+                    int bytes = 0;
+                    if (slot0 + row < x.r.n) {
+                        int code, label;
+                        const int tok = offset_token(g, x.r, a_r, b_r, code, label);
+                        src = q + (sample_off + (size_t)tok) * g.ts + head * kD + j8 * 8;
+                        bytes = 16;
+                    }
+                    cp_async16(qb + half_off * kQHalf + tile_off<32>(row, c4), src, bytes);
+                }
+                cp_async_commit();
+                cp_async_wait<0>();
+                fence_proxy_async();
+                mbar_arrive(bar_qfull(qs));
+            }
+            // ---- the key chunks: pass A needs K only, pass B K and V
+            for (int pass = 0; pass < 2; ++pass) {
+                for (int c = 0; c < x.nch; ++c, ++ru) {
+                    const int s = (int)(ru % kSlots);
+                    if (!mbar_wait_all(bar_kvempty(s), (int)((ru / kSlots) & 1) ^ 1, cta_abort)) goto done_loader;
+                    const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes;
+                    const int ncols = min(kChunk, x.npad - c * kChunk);
+                    if (pass == 1) {
+                        int* kcs = reinterpret_cast<int*>(smem + kOffKeyMeta + s * 1024);
+                        int* klab = kcs + 128;
+                        for (int row = lt; row < kChunk; row += kLoaderThreads) {
+                            const int slot = c * kChunk + row;
+                            int code = 0, label = 0xff, kc = 4 * (2 * c0 + 1);
+                            if (slot < x.r.n) {
+                                const int a = slot / ew;
+                                offset_token(g, x.r, a, slot - a * ew, code, label);
+                                kc = 4 * (c0 - code);
+                            }
+                            kcs[row] = kc;
+                            klab[row] = label;
+                        }
+                    }
+                    const int q_r = 12 / ew, r_r = 12 - q_r * ew;
+                    const int slot_first = c * kChunk + (lt >> 3);
+                    int a_r = slot_first / ew, b_r = slot_first - a_r * ew;
+                    for (int row = lt >> 3; row < ncols; row += 12, a_r += q_r, b_r += r_r) {
+                        if (b_r >= ew) { b_r -= ew; ++a_r; }
+                        const __nv_bfloat16 *sk = k, *sv = v;
+                        int bytes = 0;
+                        if (c * kChunk + row < x.r.n) {
+                            int code, label;
+                            const int tok = offset_token(g, x.r, a_r, b_r, code, label);
+                            const size_t off = (sample_off + (size_t)tok) * g.ts + head * kD + j8 * 8;
+                            sk = k + off; sv = v + off;
+                            bytes = 16;
+                        }
+                        const uint32_t so = tile_off<32>(row, c4);
+                        cp_async16(sb + (half_off ? kOffKhi : kOffKlo) + so, sk, bytes);
+                        if (pass == 1) cp_async16(sb + (half_off ? kOffVhi : kOffVlo) + so, sv, bytes);
+                    }
+                    cp_async_commit();
+                    cp_async_wait<0>();
+                    fence_proxy_async();
+                    mbar_arrive(bar_kvfull(s));
+                }
+            }
+            ++kuse;
+        }
+    done_loader:;
+    } else {
+        // ------------------------------------------------------------------ MMA issuer
+        const uint32_t idesc_pv = make_idesc_bf16(128, kNO, 0, 1);
+        int kuse = 0;
+        long long ru = 0;
+        int n_s[2] = {0, 0}, n_free[2] = {0, 0}, n_p[2] = {0, 0}, n_items_t[2] = {0, 0};
+        bool ok = true;
+        ItemCursor cur = cursor_init(cta_in_head, ctas_per_head, max_pairs, g.Mw, g.Mh);
+        for (long long it = cta_in_head; ok && it < n_items; it += ctas_per_head, cursor_advance(cur, max_pairs, g.Mw, g.Mh)) {
+            const Item x = make_item(g, cur);
+            if (x.ntiles == 0) continue;
+            const int qs = kuse % kQStages;
+            ok = mbar_wait_all(bar_qfull(qs), (kuse / kQStages) & 1, cta_abort);
+            if (!ok) break;
+            fence_proxy_async();
+            tc_fence_after();
+            const uint32_t qb = smem0 + qs * kQStageBytes;
+            // S = Q_t K_c^T into tile t's columns
+            auto issue_qk = [&](int t, uint32_t sb, int ncols) {
+                const uint32_t idesc = make_idesc_bf16(128, ncols, 0, 0);
+                if (elect_one()) {
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) {
+                        const uint32_t qa = qb + (ks >> 1) * kQHalf + t * 128 * kHalfBytes + (ks & 1) * 32;
+                        const uint32_t ka = sb + (ks >> 1) * kKHalf + (ks & 1) * 32;
+                        mma_ss(tmem_base + t * 256, make_sdesc_sw64(qa, 512), make_sdesc_sw64(ka, 512), idesc, ks > 0 ? 1u : 0u);
+                    }
+                    mma_commit(bar_sready(t));
+                }
+                __syncwarp();
+            };
+            for (int pass = 0; pass < 2 && ok; ++pass) {
+                for (int c = 0; c < x.nch && ok; ++c, ++ru) {
+                    const int s = (int)(ru % kSlots);
+                    ok = mbar_wait_all(bar_kvfull(s), (int)((ru / kSlots) & 1), cta_abort);
+                    if (!ok) break;
+                    fence_proxy_async();
+                    const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes;
+                    const int ncols = min(kChunk, x.npad - c * kChunk);
+                    for (int t = 0; t < x.ntiles && ok; ++t) {
+                        // tile t's S columns are free: in pass A once the softmax threads have read the chunk before
+                        // this one (every S of pass A is read and released), in pass B by the order of the MMAs (the
+                        // chunk before this one was consumed by its PV product, issued earlier from this thread)
+                        while (ok && n_free[t] < n_s[t]) {
+                            ok = mbar_wait_all(bar_sfree(t), n_free[t] & 1, cta_abort);
+                            ++n_free[t];
+                        }
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_qk(t, sb, ncols);
+                        if (pass == 0) ++n_s[t];
+                    }
+                    if (!ok) break;
+                    if (pass == 1) {
+                        for (int t = 0; t < x.ntiles && ok; ++t) {
+                            ok = mbar_wait_all(bar_pready(t), n_p[t] & 1, cta_abort);
+                            ++n_p[t];
+                            if (ok && c == 0 && n_items_t[t] > 0)      // the accumulator still holds the tile's previous O
+                                ok = mbar_wait_all(bar_ofree(t), (n_items_t[t] - 1) & 1, cta_abort);
+                            if (!ok) break;
+                            tc_fence_after();
+                            const uint32_t v_lo = sdesc_lo(make_sdesc_sw64_mn(sb + kOffVlo, kKHalf, 512));
+                            const uint32_t d_hi = sdesc_hi(make_sdesc_sw64_mn(sb + kOffVlo, kKHalf, 512));
+                            const uint32_t t_o = tmem_base + t * 256 + kColO, t_p = tmem_base + t * 256;
+                            const int nks = ncols >> 4;
+                            if (elect_one()) {
+                                int ks = 0;
+                                if (c == 0) {
+                                    mma_ts_h<false>(t_o, t_p, v_lo, d_hi, idesc_pv);
+                                    ks = 1;
+                                }
+                                for (; ks < nks; ++ks) mma_ts_h<true>(t_o, t_p + 8 * ks, v_lo + 64 * ks, d_hi, idesc_pv);
+                                if (c == x.nch - 1) mma_commit(bar_oready(t));
+                            }
+                            __syncwarp();
+                            if (c == x.nch - 1) ++n_items_t[t];
+                        }
+                        if (!ok) break;
+                    }
+                    if (elect_one()) mma_commit(bar_kvempty(s));     // the slot is free once the MMAs issued so far are complete
+                    __syncwarp();
+                }
+            }
+            if (!ok) break;
+            if (elect_one()) mma_commit(bar_qempty(qs));
+            __syncwarp();
+            ++kuse;
+        }
+    }
+    } else {
+        // ------------------------------------------------------------------ softmax warpgroups
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(kRegsSoftmax));
+        const int wg = warp >> 2;
+        const int row = (warp & 3) * 32 + lane;
+        const uint32_t lane_addr = ((uint32_t)(32 * (warp & 3))) << 16;
+        const uint32_t t_s = tmem_base + lane_addr + wg * 256;
+        const float scale = g.scale_log2e;
+        int kuse = 0, n_s = 0, n_o = 0;
+        long long ru = 0;
+        ItemCursor cur = cursor_init(cta_in_head, ctas_per_head, max_pairs, g.Mw, g.Mh);
+        for (long long it = cta_in_head; it < n_items; it += ctas_per_head, cursor_advance(cur, max_pairs, g.Mw, g.Mh)) {
+            const Item x = make_item(g, cur);
+            if (x.ntiles == 0) continue;
+            const int qs = kuse % kQStages;
+            if (!mbar_wait_all(bar_qfull(qs), (kuse / kQStages) & 1, cta_abort)) break;
+            const int rmeta = lds_i32(smem0 + kOffRowMeta + qs * 2048 + 4 * (wg * 128 + row));
+            const int tok = lds_i32(smem0 + kOffRowMeta + qs * 2048 + 1024 + 4 * (wg * 128 + row));
+            mbar_arrive(bar_qempty(qs));                  // this thread has what it needs from the stage
+            ++kuse;
+            const long long ru0 = ru;
+            ru += 2 * x.nch;
+            if (wg >= x.ntiles) continue;                 // the pair's second tile does not exist in this window
+            const uint32_t bias_i = smem0 + kOffBias + 4 * meta_code(rmeta);
+            const int label_i = meta_label(rmeta);
+            const float bmax = lds_f32(smem0 + kOffBias + 4 * (kBiasFloats - 1));
+            bool ok = true;
+            // ---- pass A: row maximum of the raw scores over all chunks
+            float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            for (int c = 0; c < x.nch; ++c) {
+                const int ncols = min(kChunk, x.npad - c * kChunk);
+                ok = mbar_wait_all(bar_sready(wg), n_s & 1, cta_abort);
+                if (!ok) break;
+                ++n_s;
+                tc_fence_after();
+                uint32_t ra[32], rb[32];
+                int cc = 0;
+                for (; cc + 64 <= ncols; cc += 64) {
+                    tmem_ld32(t_s + cc, ra);
+                    tmem_ld32(t_s + cc + 32, rb);
+                    tmem_ld_wait();
+                    max_cols<32>(ra, mx4);
+                    max_cols<32>(rb, mx4);
+                }
+                if (cc + 32 <= ncols) {
+                    tmem_ld32(t_s + cc, ra);
+                    tmem_ld_wait();
+                    max_cols<32>(ra, mx4);
+                    cc += 32;
+                }
+                if (cc < ncols) {
+                    uint32_t rt[16];
+                    tmem_ld16(t_s + cc, rt);
+                    tmem_ld_wait();
+                    max_cols<16>(rt, mx4);
+                }
+                tc_fence_before();
+                mbar_arrive(bar_sfree(wg));
+            }
+            if (!ok) break;
+            const float m = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale + bmax;
+            const float neg_m = -m;
+            // ---- pass B: P chunk by chunk
+            for (int c = 0; c < x.nch; ++c) {
+                const int ncols = min(kChunk, x.npad - c * kChunk);
+                const int s = (int)((ru0 + x.nch + c) % kSlots);
+                const uint32_t a_kc = smem0 + kOffKeyMeta + s * 1024, a_klab = a_kc + 512;
+                ok = mbar_wait_all(bar_sready(wg), n_s & 1, cta_abort);
+                if (!ok) break;
+                ++n_s;
+                tc_fence_after();
+                const int nfull = ncols >> 5;
+                uint32_t ra[32], rb[32];
+                if (nfull > 0) tmem_ld32(t_s, ra);
+                for (int i = 0; i < nfull; i += 2) {
+                    uint32_t pk[16];
+                    tmem_ld_wait();
+                    if (i + 1 < nfull) tmem_ld32(t_s + 32 * (i + 1), rb);
+                    if (x.masked) softmax_cols<32, true>(ra, pk, 32 * i, bias_i, a_kc, a_klab, label_i, scale, neg_m);
+                    else softmax_cols<32, false>(ra, pk, 32 * i, bias_i, a_kc, a_klab, label_i, scale, neg_m);
+                    tmem_st16(t_s + 16 * i, pk);
+                    if (i + 1 < nfull) {
+                        tmem_ld_wait();
+                        if (i + 2 < nfull) tmem_ld32(t_s + 32 * (i + 2), ra);
+                        if (x.masked) softmax_cols<32, true>(rb, pk, 32 * (i + 1), bias_i, a_kc, a_klab, label_i, scale, neg_m);
+                        else softmax_cols<32, false>(rb, pk, 32 * (i + 1), bias_i, a_kc, a_klab, label_i, scale, neg_m);
+                        tmem_st16(t_s + 16 * (i + 1), pk);
+                    }
+                }
+                if (ncols & 16) {
+                    uint32_t rt[16], pk[8];
+                    tmem_ld16(t_s + 32 * nfull, rt);
+                    tmem_ld_wait();
+                    if (x.masked) softmax_cols<16, true>(rt, pk, 32 * nfull, bias_i, a_kc, a_klab, label_i, scale, neg_m);
+                    else softmax_cols<16, false>(rt, pk, 32 * nfull, bias_i, a_kc, a_klab, label_i, scale, neg_m);
+                    tmem_st8(t_s + 16 * nfull, pk);
+                }
+                tmem_st_wait();
+                tc_fence_before();
+                mbar_arrive(bar_pready(wg));
+            }
+            if (!ok) break;
+            // ---- O and the row sum
+            if (!mbar_wait_all(bar_oready(wg), n_o & 1, cta_abort)) break;
+            ++n_o;
+            tc_fence_after();
+            uint32_t ro[32], ro2[32], rsum;
+            tmem_ld32(t_s + kColO, ro);
+            tmem_ld32(t_s + kColO + 32, ro2);
+            tmem_ld1(t_s + kColO + kD, rsum);
+            tmem_ld_wait();
+            tc_fence_before();
+            mbar_arrive(bar_ofree(wg));
+            if (tok >= 0) {
+                const float sum = __uint_as_float(rsum);
+                const size_t row_off = ((size_t)x.b * HW + (size_t)tok) * g.heads + head;
+                lse[row_off] = (m + log2f(sum)) * kLn2;
+                const float inv = 1.f / sum;
+                uint4* dst = reinterpret_cast<uint4*>(o + row_off * kD);
+#pragma unroll
+                for (int c4 = 0; c4 < 4; ++c4) {
+                    uint4 val;
+                    val.x = pack_bf16(__uint_as_float(ro[c4 * 8 + 0]) * inv, __uint_as_float(ro[c4 * 8 + 1]) * inv);
+                    val.y = pack_bf16(__uint_as_float(ro[c4 * 8 + 2]) * inv, __uint_as_float(ro[c4 * 8 + 3]) * inv);
+                    val.z = pack_bf16(__uint_as_float(ro[c4 * 8 + 4]) * inv, __uint_as_float(ro[c4 * 8 + 5]) * inv);
+                    val.w = pack_bf16(__uint_as_float(ro[c4 * 8 + 6]) * inv, __uint_as_float(ro[c4 * 8 + 7]) * inv);
+                    dst[c4] = val;
+                }
+#pragma unroll
+                for (int c4 = 0; c4 < 4; ++c4) {
+                    uint4 val;
+                    val.x = pack_bf16(__uint_as_float(ro2[c4 * 8 + 0]) * inv, __uint_as_float(ro2[c4 * 8 + 1]) * inv);
+                    val.y = pack_bf16(__uint_as_float(ro2[c4 * 8 + 2]) * inv, __uint_as_float(ro2[c4 * 8 + 3]) * inv);
+                    val.z = pack_bf16(__uint_as_float(ro2[c4 * 8 + 4]) * inv, __uint_as_float(ro2[c4 * 8 + 5]) * inv);
+                    val.w = pack_bf16(__uint_as_float(ro2[c4 * 8 + 6]) * inv, __uint_as_float(ro2[c4 * 8 + 7]) * inv);
+                    dst[4 + c4] = val;
+                }
+            }
+        }
+    }
+
+    // teardown: every role ends up here, also after an expired wait
+    cp_async_wait<0>();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == kMmaWarp) tmem_dealloc(tmem_base, 512);
+    if (tid == 0 && *cta_abort) atomicExch(&g_fwd_tc64_timeout, 1);
+}
+
+// The prepared bias table of the small-window kernel, sized for window sides up to 32: per head
+//   table[(da + w - 1) * cs + (db + w - 1)] = T[(da + w - 1) * (2w - 1) + (db + w - 1), head] * log2(e)   (cs = w + 32),
+//   table[2 c0 + 1 .. 3 c0 + 1] = -inf (where key slots without a token point), the head's largest entry in the last float.
+__global__ void __launch_bounds__(256)
+swin_fwd_bias_prep64_kernel(const float* __restrict__ bias, float* __restrict__ prep, int w, int heads) {
+    const int head = blockIdx.x;
+    const int cs = w + 32, nw = 2 * w - 1;
+    const int c0 = (w - 1) * (cs + 1);
+    float* dst = prep + (size_t)head * kBiasFloats;
+    float mx = -INFINITY;
+    for (int e = threadIdx.x; e < kBiasFloats - 1; e += blockDim.x) {
+        float val = 0.f;
+        if (e > 2 * c0) {
+            val = -INFINITY;
+        } else {
+            const int ra = e / cs, rb = e - ra * cs;
+            if (rb < nw && ra < nw) {
+                val = bias[(size_t)(ra * nw + rb) * heads + head] * kLog2e;
+                mx = fmaxf(mx, val);
+            }
+        }
+        dst[e] = val;
+    }
+    __shared__ float red[8];
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = mx;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int i = 1; i < 8; ++i) mx = fmaxf(mx, red[i]);
+        dst[kBiasFloats - 1] = mx;
+    }
+}
+
+}  // namespace
+
+cudaError_t read_fwd_tc64_status(int* timed_out) {
+    int zero = 0;
+    cudaError_t e = cudaMemcpyFromSymbol(timed_out, g_fwd_tc64_timeout, sizeof(int));
+    if (e != cudaSuccess) return e;
+    if (*timed_out) e = cudaMemcpyToSymbol(g_fwd_tc64_timeout, &zero, sizeof(int));
+    return e;
+}
+
+bool fwd_tc64_supported(const Geo& g) { return g.d == 64 && g.w <= 32 && g.nmax <= 1024 && g.heads <= 148; }
+
+size_t fwd_tc64_workspace_bytes(const Geo& g) { return (size_t)g.heads * kBiasFloats * sizeof(float); }
+
+cudaError_t launch_fwd_tc64(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
+                            void* o, float* lse, void* workspace, int sm_count, cudaStream_t stream) {
+    float* prep = reinterpret_cast<float*>(workspace);
+    swin_fwd_bias_prep64_kernel<<<g.heads, 256, 0, stream>>>(bias, prep, g.w, g.heads);
+    count_launch(stream);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const int max_pairs = (((g.nmax + 127) >> 7) + 1) / 2;
+    const long long items = (long long)g.B * g.Mh * g.Mw * max_pairs;
+    long long cph = sm_count / g.heads;
+    if (cph < 1) cph = 1;
+    if (cph > items) cph = items;
+    e = cudaFuncSetAttribute(swin_fwd_tc64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    prof_begin("swin_fwd_tc64_kernel", stream);
+    swin_fwd_tc64_kernel<<<(unsigned)(cph * g.heads), kThreads, kSmemBytes, stream>>>(
+        g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, prep, (__nv_bfloat16*)o, lse,
+        items, (int)cph, max_pairs);
+    count_launch(stream);
+    return cudaGetLastError();
+}
+
+}  // namespace terra

@@ -28,6 +28,13 @@ cudaError_t launch_fwd_tc(const Geo& g, const void* q, const void* k, const void
 // synchronises the stream, reads and clears the device-side "a bounded wait expired" word
 cudaError_t read_tc_status(int* timed_out, cudaStream_t stream);
 
+// tcgen05 forward path for head dim 64 and windows of up to 1024 tokens (keys streamed in chunks, two passes)
+bool fwd_tc64_supported(const Geo& g);
+size_t fwd_tc64_workspace_bytes(const Geo& g);
+cudaError_t launch_fwd_tc64(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
+                            void* o, float* lse, void* workspace, int sm_count, cudaStream_t stream);
+cudaError_t read_fwd_tc64_status(int* timed_out);     // after the stream has been synchronised
+
 cudaError_t launch_bounded_wait_selftest(long long limit_cycles, cudaStream_t stream);
 cudaError_t launch_bias_prep(const Geo& g, const float* bias, float* prep, cudaStream_t stream);
 
