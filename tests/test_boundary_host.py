@@ -50,7 +50,7 @@ def test_workspace_sizes(lib):
     cfg = CONFIGS["cfg3"]
     d = terra.make_desc(cfg)
     assert terra.terra_swin_workspace_bytes(d, False) >= cfg.heads * 8192     # prepared bias tables
-    assert terra.terra_swin_workspace_bytes(terra.make_desc(CONFIGS["cfg4"]), False) == 0
+    assert terra.terra_swin_workspace_bytes(terra.make_desc(CONFIGS["cfg4"]), False) >= CONFIGS["cfg4"].heads * 6048 * 4    # tables for window side 32
     assert terra.terra_swin_workspace_bytes(d, True) >= cfg.tokens * cfg.heads * 4
 
 
