@@ -216,23 +216,51 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kRegsOther));
     if (warp >= kLoaderWarp0) {
         // ------------------------------------------------------------------ loaders
+        // Two lanes per row: lane parity picks the row's lo / hi half, each lane issues the half's four 16-byte
+        // copies with one address computation.  A chunk is published (its barrier arrived on) only when the next
+        // one has been issued, so that two chunks are in flight; if the ring has no free slot the pending chunk is
+        // published first, or the consumers could never free one.
         const int lt = (warp - kLoaderWarp0) * 32 + lane;
-        const int j8 = lt & 7;                            // 16-byte chunk of the 128-byte row this thread copies
-        const uint32_t half_off = (j8 >> 2) ? 1u : 0u;    // lo or hi half
-        const int c4 = j8 & 3;
+        const int hf = lt & 1;                            // which 32-column half of the row this thread copies
+        const int lrow = lt >> 1;                         // 0 .. 47
+        constexpr int kRowsPerIter = kLoaderThreads / 2;  // 48
         int kuse = 0;
         long long ru = 0;                                 // ring uses so far
+        uint32_t pending_bar = 0;                         // barrier of the group of copies issued last (0: none)
+        bool ok = true;
+        // waits for `bar` (a slot's or stage's release); publishes the pending copies first if that is not immediate
+        auto acquire = [&](uint32_t bar, uint32_t parity) -> bool {
+            if (pending_bar && !__all_sync(0xffffffffu, mbar_test_wait(bar, parity))) {
+                cp_async_wait<0>();
+                fence_proxy_async();
+                mbar_arrive(pending_bar);
+                pending_bar = 0;
+            }
+            return mbar_wait_all(bar, parity, cta_abort);
+        };
+        // the copies just issued become the pending group; the group before them is complete and is published
+        auto issued = [&](uint32_t bar) {
+            cp_async_commit();
+            if (pending_bar) {
+                cp_async_wait<1>();
+                fence_proxy_async();
+                mbar_arrive(pending_bar);
+            }
+            pending_bar = bar;
+        };
         ItemCursor cur = cursor_init(cta_in_head, ctas_per_head, max_pairs, g.Mw, g.Mh);
-        for (long long it = cta_in_head; it < n_items; it += ctas_per_head, cursor_advance(cur, max_pairs, g.Mw, g.Mh)) {
+        for (long long it = cta_in_head; ok && it < n_items; it += ctas_per_head, cursor_advance(cur, max_pairs, g.Mw, g.Mh)) {
             const Item x = make_item(g, cur);
             if (x.ntiles == 0) continue;
             const int qs = kuse % kQStages;
-            if (!mbar_wait_all(bar_qempty(qs), ((kuse / kQStages) & 1) ^ 1, cta_abort)) break;
+            ok = acquire(bar_qempty(qs), ((kuse / kQStages) & 1) ^ 1);
+            if (!ok) break;
             const size_t sample_off = (size_t)x.b * HW;
             const int ew = x.r.ew;
+            const int q_r = kRowsPerIter / ew, r_r = kRowsPerIter - q_r * ew;       // window-offset step of 48 slots
             // ---- Q rows of the pair (rows without a token as zeros) and the row tables
             {
-                const uint32_t qb = smem0 + qs * kQStageBytes;
+                const uint32_t qb = smem0 + qs * kQStageBytes + hf * kQHalf;
                 int* rowmeta = reinterpret_cast<int*>(smem + kOffRowMeta + qs * 2048);
                 int* rowtok = rowmeta + 256;
                 const int slot0 = x.pair * kQRows;
@@ -247,32 +275,29 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                     rowtok[row] = tok;
                 }
                 const int nrows = x.ntiles * 128;
-                const int q_r = 12 / ew, r_r = 12 - q_r * ew;
-                int slot = slot0 + (lt >> 3);
-                int a_r = slot / ew, b_r = slot - a_r * ew;
-                for (int row = lt >> 3; row < nrows; row += 12, a_r += q_r, b_r += r_r) {
+                int a_r = (slot0 + lrow) / ew, b_r = (slot0 + lrow) - a_r * ew;
+                for (int row = lrow; row < nrows; row += kRowsPerIter, a_r += q_r, b_r += r_r) {
                     if (b_r >= ew) { b_r -= ew; ++a_r; }
                     const __nv_bfloat16* src = q;
                     int bytes = 0;
                     if (slot0 + row < x.r.n) {
                         int code, label;
                         const int tok = offset_token(g, x.r, a_r, b_r, code, label);
-                        src = q + (sample_off + (size_t)tok) * g.ts + head * kD + j8 * 8;
+                        src = q + (sample_off + (size_t)tok) * g.ts + head * kD + hf * 32;
                         bytes = 16;
                     }
-                    cp_async16(qb + half_off * kQHalf + tile_off<32>(row, c4), src, bytes);
+#pragma unroll
+                    for (int c4 = 0; c4 < 4; ++c4) cp_async16(qb + tile_off<32>(row, c4), bytes ? src + c4 * 8 : src, bytes);
                 }
-                cp_async_commit();
-                cp_async_wait<0>();
-                fence_proxy_async();
-                mbar_arrive(bar_qfull(qs));
+                issued(bar_qfull(qs));
             }
             // ---- the key chunks: pass A needs K only, pass B K and V
-            for (int pass = 0; pass < 2; ++pass) {
+            for (int pass = 0; pass < 2 && ok; ++pass) {
                 for (int c = 0; c < x.nch; ++c, ++ru) {
                     const int s = (int)(ru % kSlots);
-                    if (!mbar_wait_all(bar_kvempty(s), (int)((ru / kSlots) & 1) ^ 1, cta_abort)) goto done_loader;
-                    const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes;
+                    ok = acquire(bar_kvempty(s), (uint32_t)((ru / kSlots) & 1) ^ 1u);
+                    if (!ok) break;
+                    const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes + hf * kKHalf;
                     const int ncols = min(kChunk, x.npad - c * kChunk);
                     if (pass == 1) {
                         int* kcs = reinterpret_cast<int*>(smem + kOffKeyMeta + s * 1024);
@@ -289,33 +314,36 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                             klab[row] = label;
                         }
                     }
-                    const int q_r = 12 / ew, r_r = 12 - q_r * ew;
-                    const int slot_first = c * kChunk + (lt >> 3);
+                    const int slot_first = c * kChunk + lrow;
                     int a_r = slot_first / ew, b_r = slot_first - a_r * ew;
-                    for (int row = lt >> 3; row < ncols; row += 12, a_r += q_r, b_r += r_r) {
+                    for (int row = lrow; row < ncols; row += kRowsPerIter, a_r += q_r, b_r += r_r) {
                         if (b_r >= ew) { b_r -= ew; ++a_r; }
                         const __nv_bfloat16 *sk = k, *sv = v;
                         int bytes = 0;
                         if (c * kChunk + row < x.r.n) {
                             int code, label;
                             const int tok = offset_token(g, x.r, a_r, b_r, code, label);
-                            const size_t off = (sample_off + (size_t)tok) * g.ts + head * kD + j8 * 8;
+                            const size_t off = (sample_off + (size_t)tok) * g.ts + head * kD + hf * 32;
                             sk = k + off; sv = v + off;
                             bytes = 16;
                         }
-                        const uint32_t so = tile_off<32>(row, c4);
-                        cp_async16(sb + (half_off ? kOffKhi : kOffKlo) + so, sk, bytes);
-                        if (pass == 1) cp_async16(sb + (half_off ? kOffVhi : kOffVlo) + so, sv, bytes);
+#pragma unroll
+                        for (int c4 = 0; c4 < 4; ++c4) {
+                            const uint32_t so = tile_off<32>(row, c4);
+                            cp_async16(sb + kOffKlo + so, bytes ? sk + c4 * 8 : sk, bytes);
+                            if (pass == 1) cp_async16(sb + kOffVlo + so, bytes ? sv + c4 * 8 : sv, bytes);
+                        }
                     }
-                    cp_async_commit();
-                    cp_async_wait<0>();
-                    fence_proxy_async();
-                    mbar_arrive(bar_kvfull(s));
+                    issued(bar_kvfull(s));
                 }
             }
             ++kuse;
         }
-    done_loader:;
+        if (pending_bar) {
+            cp_async_wait<0>();
+            fence_proxy_async();
+            mbar_arrive(pending_bar);
+        }
     } else {
         // ------------------------------------------------------------------ MMA issuer
         const uint32_t idesc_pv = make_idesc_bf16(128, kNO, 0, 1);
