@@ -375,57 +375,85 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                 }
                 __syncwarp();
             };
-            for (int pass = 0; pass < 2 && ok; ++pass) {
-                for (int c = 0; c < x.nch && ok; ++c, ++ru) {
-                    const int s = (int)(ru % kSlots);
-                    ok = mbar_wait_all(bar_kvfull(s), (int)((ru / kSlots) & 1), cta_abort);
-                    if (!ok) break;
-                    fence_proxy_async();
-                    const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes;
-                    const int ncols = min(kChunk, x.npad - c * kChunk);
-                    for (int t = 0; t < x.ntiles && ok; ++t) {
-                        // tile t's S columns are free: in pass A once the softmax threads have read the chunk before
-                        // this one (every S of pass A is read and released), in pass B by the order of the MMAs (the
-                        // chunk before this one was consumed by its PV product, issued earlier from this thread)
-                        while (ok && n_free[t] < n_s[t]) {
-                            ok = mbar_wait_all(bar_sfree(t), n_free[t] & 1, cta_abort);
-                            ++n_free[t];
-                        }
-                        if (!ok) break;
-                        tc_fence_after();
-                        issue_qk(t, sb, ncols);
-                        if (pass == 0) ++n_s[t];
-                    }
-                    if (!ok) break;
-                    if (pass == 1) {
-                        for (int t = 0; t < x.ntiles && ok; ++t) {
-                            ok = mbar_wait_all(bar_pready(t), n_p[t] & 1, cta_abort);
-                            ++n_p[t];
-                            if (ok && c == 0 && n_items_t[t] > 0)      // the accumulator still holds the tile's previous O
-                                ok = mbar_wait_all(bar_ofree(t), (n_items_t[t] - 1) & 1, cta_abort);
-                            if (!ok) break;
-                            tc_fence_after();
-                            const uint32_t v_lo = sdesc_lo(make_sdesc_sw64_mn(sb + kOffVlo, kKHalf, 512));
-                            const uint32_t d_hi = sdesc_hi(make_sdesc_sw64_mn(sb + kOffVlo, kKHalf, 512));
-                            const uint32_t t_o = tmem_base + t * 256 + kColO, t_p = tmem_base + t * 256;
-                            const int nks = ncols >> 4;
-                            if (elect_one()) {
-                                int ks = 0;
-                                if (c == 0) {
-                                    mma_ts_h<false>(t_o, t_p, v_lo, d_hi, idesc_pv);
-                                    ks = 1;
-                                }
-                                for (; ks < nks; ++ks) mma_ts_h<true>(t_o, t_p + 8 * ks, v_lo + 64 * ks, d_hi, idesc_pv);
-                                if (c == x.nch - 1) mma_commit(bar_oready(t));
-                            }
-                            __syncwarp();
-                            if (c == x.nch - 1) ++n_items_t[t];
-                        }
-                        if (!ok) break;
-                    }
-                    if (elect_one()) mma_commit(bar_kvempty(s));     // the slot is free once the MMAs issued so far are complete
-                    __syncwarp();
+            // tile t's S columns are free for a new QK product: after pass-A chunks once the softmax threads have read
+            // the chunk before (every S of pass A is read and released); after pass-B chunks by the order of the MMAs
+            // (the P that replaced S was consumed by its PV product, issued earlier from this thread)
+            auto s_free = [&](int t) -> bool {
+                while (n_free[t] < n_s[t]) {
+                    if (!mbar_wait_all(bar_sfree(t), n_free[t] & 1, cta_abort)) return false;
+                    ++n_free[t];
                 }
+                tc_fence_after();
+                return true;
+            };
+            auto chunk_ready = [&](long long use) -> bool {
+                if (!mbar_wait_all(bar_kvfull((int)(use % kSlots)), (uint32_t)((use / kSlots) & 1), cta_abort)) return false;
+                fence_proxy_async();
+                return true;
+            };
+            // ---- pass A: S of every chunk, for the row maxima
+            for (int c = 0; c < x.nch && ok; ++c, ++ru) {
+                const int s = (int)(ru % kSlots);
+                ok = chunk_ready(ru);
+                if (!ok) break;
+                const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes;
+                const int ncols = min(kChunk, x.npad - c * kChunk);
+                for (int t = 0; t < x.ntiles && ok; ++t) {
+                    ok = s_free(t);
+                    if (!ok) break;
+                    issue_qk(t, sb, ncols);
+                    ++n_s[t];
+                }
+                if (!ok) break;
+                if (elect_one()) mma_commit(bar_kvempty(s));     // the slot is free once the MMAs issued so far are complete
+                __syncwarp();
+            }
+            if (!ok) break;
+            // ---- pass B: per tile, PV of chunk c is followed at once by QK of chunk c + 1, so that a tile's softmax
+            // threads wait for one PV and one QK product only, whatever the other tile is doing
+            ok = chunk_ready(ru);
+            for (int t = 0; t < x.ntiles && ok; ++t) {
+                ok = s_free(t);
+                if (ok) issue_qk(t, smem0 + kOffSlots + (int)(ru % kSlots) * kSlotBytes, min(kChunk, x.npad));
+            }
+            for (int c = 0; c < x.nch && ok; ++c, ++ru) {
+                const int s = (int)(ru % kSlots);
+                const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes;
+                const int ncols = min(kChunk, x.npad - c * kChunk);
+                const bool has_next = c + 1 < x.nch;
+                if (has_next) {
+                    ok = chunk_ready(ru + 1);
+                    if (!ok) break;
+                }
+                const uint32_t sb_n = smem0 + kOffSlots + (int)((ru + 1) % kSlots) * kSlotBytes;
+                const int ncols_n = min(kChunk, x.npad - (c + 1) * kChunk);
+                for (int t = 0; t < x.ntiles && ok; ++t) {
+                    ok = mbar_wait_all(bar_pready(t), n_p[t] & 1, cta_abort);
+                    ++n_p[t];
+                    if (ok && c == 0 && n_items_t[t] > 0)      // the accumulator still holds the tile's previous O
+                        ok = mbar_wait_all(bar_ofree(t), (n_items_t[t] - 1) & 1, cta_abort);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint64_t vd = make_sdesc_sw64_mn(sb + kOffVlo, kKHalf, 512);
+                    const uint32_t v_lo = sdesc_lo(vd), d_hi = sdesc_hi(vd);
+                    const uint32_t t_o = tmem_base + t * 256 + kColO, t_p = tmem_base + t * 256;
+                    const int nks = ncols >> 4;
+                    if (elect_one()) {
+                        int ks = 0;
+                        if (c == 0) {
+                            mma_ts_h<false>(t_o, t_p, v_lo, d_hi, idesc_pv);
+                            ks = 1;
+                        }
+                        for (; ks < nks; ++ks) mma_ts_h<true>(t_o, t_p + 8 * ks, v_lo + 64 * ks, d_hi, idesc_pv);
+                        if (!has_next) mma_commit(bar_oready(t));
+                    }
+                    __syncwarp();
+                    if (!has_next) ++n_items_t[t];
+                    else issue_qk(t, sb_n, ncols_n);
+                }
+                if (!ok) break;
+                if (elect_one()) mma_commit(bar_kvempty(s));
+                __syncwarp();
             }
             if (!ok) break;
             if (elect_one()) mma_commit(bar_qempty(qs));
