@@ -135,6 +135,58 @@ __device__ __forceinline__ void softmax_cols(const uint32_t (&r)[N], uint32_t (&
     }
 }
 
+template <int OFF>
+__device__ __forceinline__ float lds_f32_at(uint32_t addr) {
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1+%2];\n" : "=f"(v) : "r"(addr), "n"(OFF));
+    return v;
+}
+// 32 key columns that are one window row of a full-width 32-wide window without mask labels: their bias entries are
+// consecutive (descending with the key), so each address is one base plus an immediate offset: no per-key offsets to
+// load, no address arithmetic.  `top` = shared address of the entry of the row's first key.
+__device__ __forceinline__ void softmax_cols32_row(const uint32_t (&r)[32], uint32_t (&pk)[16], uint32_t top, float scale, float neg_m) {
+    const uint32_t bb = top - 124;
+    float bv[32];
+    bv[0] = lds_f32_at<124>(bb);
+    bv[1] = lds_f32_at<120>(bb);
+    bv[2] = lds_f32_at<116>(bb);
+    bv[3] = lds_f32_at<112>(bb);
+    bv[4] = lds_f32_at<108>(bb);
+    bv[5] = lds_f32_at<104>(bb);
+    bv[6] = lds_f32_at<100>(bb);
+    bv[7] = lds_f32_at<96>(bb);
+    bv[8] = lds_f32_at<92>(bb);
+    bv[9] = lds_f32_at<88>(bb);
+    bv[10] = lds_f32_at<84>(bb);
+    bv[11] = lds_f32_at<80>(bb);
+    bv[12] = lds_f32_at<76>(bb);
+    bv[13] = lds_f32_at<72>(bb);
+    bv[14] = lds_f32_at<68>(bb);
+    bv[15] = lds_f32_at<64>(bb);
+    bv[16] = lds_f32_at<60>(bb);
+    bv[17] = lds_f32_at<56>(bb);
+    bv[18] = lds_f32_at<52>(bb);
+    bv[19] = lds_f32_at<48>(bb);
+    bv[20] = lds_f32_at<44>(bb);
+    bv[21] = lds_f32_at<40>(bb);
+    bv[22] = lds_f32_at<36>(bb);
+    bv[23] = lds_f32_at<32>(bb);
+    bv[24] = lds_f32_at<28>(bb);
+    bv[25] = lds_f32_at<24>(bb);
+    bv[26] = lds_f32_at<20>(bb);
+    bv[27] = lds_f32_at<16>(bb);
+    bv[28] = lds_f32_at<12>(bb);
+    bv[29] = lds_f32_at<8>(bb);
+    bv[30] = lds_f32_at<4>(bb);
+    bv[31] = lds_f32_at<0>(bb);
+#pragma unroll
+    for (int e2 = 0; e2 < 16; ++e2) {
+        const float p0 = fast_exp2(fmaf(__uint_as_float(r[2 * e2]), scale, bv[2 * e2]) + neg_m);
+        const float p1 = fast_exp2(fmaf(__uint_as_float(r[2 * e2 + 1]), scale, bv[2 * e2 + 1]) + neg_m);
+        pk[e2] = pack_bf16(p0, p1);
+    }
+}
+
 template <int N>
 __device__ __forceinline__ void max_cols(const uint32_t (&r)[N], float (&mx)[4]) {
 #pragma unroll
@@ -487,6 +539,7 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             const uint32_t bias_i = smem0 + kOffBias + 4 * meta_code(rmeta);
             const int label_i = meta_label(rmeta);
             const float bmax = lds_f32(smem0 + kOffBias + 4 * (kBiasFloats - 1));
+            const bool row32 = g.w == 32 && x.r.ew == 32 && !x.masked;       // then every key slot holds a token, too
             bool ok = true;
             // ---- pass A: row maximum of the raw scores over all chunks
             float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
@@ -535,17 +588,21 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                 const int nfull = ncols >> 5;
                 uint32_t ra[32], rb[32];
                 if (nfull > 0) tmem_ld32(t_s, ra);
+                // full-width 32-wide window without mask labels: 32-column group i of chunk c is key row 4 c + i
+                const uint32_t top_c = bias_i + 4 * (c0 - 4 * c * cs);
                 for (int i = 0; i < nfull; i += 2) {
                     uint32_t pk[16];
                     tmem_ld_wait();
                     if (i + 1 < nfull) tmem_ld32(t_s + 32 * (i + 1), rb);
-                    if (x.masked) softmax_cols<32, true>(ra, pk, 32 * i, bias_i, a_kc, a_klab, label_i, scale, neg_m);
+                    if (row32) softmax_cols32_row(ra, pk, top_c - 4 * i * cs, scale, neg_m);
+                    else if (x.masked) softmax_cols<32, true>(ra, pk, 32 * i, bias_i, a_kc, a_klab, label_i, scale, neg_m);
                     else softmax_cols<32, false>(ra, pk, 32 * i, bias_i, a_kc, a_klab, label_i, scale, neg_m);
                     tmem_st16(t_s + 16 * i, pk);
                     if (i + 1 < nfull) {
                         tmem_ld_wait();
                         if (i + 2 < nfull) tmem_ld32(t_s + 32 * (i + 2), ra);
-                        if (x.masked) softmax_cols<32, true>(rb, pk, 32 * (i + 1), bias_i, a_kc, a_klab, label_i, scale, neg_m);
+                        if (row32) softmax_cols32_row(rb, pk, top_c - 4 * (i + 1) * cs, scale, neg_m);
+                        else if (x.masked) softmax_cols<32, true>(rb, pk, 32 * (i + 1), bias_i, a_kc, a_klab, label_i, scale, neg_m);
                         else softmax_cols<32, false>(rb, pk, 32 * (i + 1), bias_i, a_kc, a_klab, label_i, scale, neg_m);
                         tmem_st16(t_s + 16 * (i + 1), pk);
                     }
