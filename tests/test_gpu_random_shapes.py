@@ -38,6 +38,14 @@ def _shapes():
     # found by fuzzing: 540 items on 148 CTAs, two of which meet three one-tile windows (6 wide) and then a
     # two-tile one, i.e. the second query tile's first use comes after a whole turn of the forward kernel's stage ring
     out.append(("ring_turn_then_second_tile", 2, 111, 71, 5, 32, 13, 45, 48, 0, 0))
+    # head dim 64 on the chunked tcgen05 forward: 1, 3, 5 and 8 query tiles per window (a pair's second tile missing
+    # for the odd counts), truncated and masked 32-wide windows, sides below 32, several items per CTA
+    out += [("d64_w32_full", 1, 64, 96, 2, 64, 32, 16, 16, 0, 1),
+            ("d64_w32_rows9", 2, 41, 64, 3, 64, 32, 5, 7, 0, 0),         # last window row 9 high: 288 tokens, 3 tiles
+            ("d64_w24", 1, 60, 72, 2, 64, 24, 12, 12, 0, 1),             # 576 tokens: 5 tiles
+            ("d64_w17", 2, 40, 50, 3, 64, 17, 8, 9, 1, 0),               # 289 tokens: 3 tiles, ragged chunks
+            ("d64_w8_many", 2, 64, 96, 5, 64, 8, 4, 4, 0, 1),            # one-tile windows, 960 items
+            ("d64_w32_narrow", 1, 70, 45, 2, 64, 32, 20, 30, 0, 0)]      # 13-wide last column, 6-high last row
     return out
 
 
