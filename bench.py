@@ -425,7 +425,7 @@ def main():
         # register-tile backward kernels 4d each (key tiles: dV, dK; query tiles: dP, dQ).
         pairs = wk["score_elements"]
         d = cfg.head_dim
-        kernel_flop = {"swin_fwd_tc_kernel": 4 * d * pairs, "swin_fwd_mma_kernel": 4 * d * pairs,
+        kernel_flop = {"swin_fwd_tc_kernel": 4 * d * pairs, "swin_fwd_tc64_kernel": 4 * d * pairs, "swin_fwd_mma_kernel": 4 * d * pairs,
                        "swin_bwd_fused_kernel": 8 * d * pairs,
                        "swin_bwd_mma_kernel<key tiles>": 4 * d * pairs, "swin_bwd_mma_kernel<query tiles>": 4 * d * pairs,
                        "swin_bwd_delta_kernel": 0}
