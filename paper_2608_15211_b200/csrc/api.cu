@@ -119,9 +119,13 @@ static size_t fwd_bytes(const Geo& g) {
 
 static bool use_bwd_tc(const Geo& g) { return bwd_tc_supported(g) && !force_register_path(); }
 
+static bool use_bwd_kv64(const Geo& g) { return bwd_kv64_supported(g) && !force_register_path(); }
+
 static size_t delta_bytes(const Geo& g) {
     if (use_bwd_tc(g)) return align_up(bwd_tc_workspace_bytes(g), 256);
-    return align_up(sizeof(float) * (size_t)g.B * g.H * g.W * g.heads, 256);
+    const size_t delta = align_up(sizeof(float) * (size_t)g.B * g.H * g.W * g.heads, 256);
+    // the tcgen05 key-side kernel of the head-dim-64 regime also wants the prepared bias tables
+    return use_bwd_kv64(g) ? delta + align_up(fwd_tc64_workspace_bytes(g), 256) : delta;
 }
 
 // Descriptor check + geometry, and the SM count of the current device, for entry points that live in
@@ -234,6 +238,15 @@ static int bwd_call(const Geo& g, const void* q, const void* k, const void* v,
     float* delta = reinterpret_cast<float*>(workspace);
     cudaError_t e = launch_bwd_delta(g, o, d_o, delta, st);
     if (e != cudaSuccess) return cuda_fail(e, "terra_swin_attn_bwd (delta)");
+    if (use_bwd_kv64(g)) {
+        // key side (dK, dV) on tcgen05, query side (dQ, dBias) on the register-tile kernel
+        float* prep = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(workspace) +
+                                               align_up(sizeof(float) * (size_t)g.B * g.H * g.W * g.heads, 256));
+        e = launch_bias_prep64(g, bias_table, prep, st);
+        if (e == cudaSuccess) e = launch_bwd_kv64(g, q, k, v, d_o, prep, lse, delta, dk, dv, sms, st);
+        if (e == cudaSuccess) e = launch_bwd_mma(g, q, k, v, bias_table, lse, delta, d_o, dq, dk, dv, dbias, sms, st, true);
+        return e == cudaSuccess ? TERRA_OK : cuda_fail(e, "terra_swin_attn_bwd");
+    }
     e = launch_bwd_mma(g, q, k, v, bias_table, lse, delta, d_o, dq, dk, dv, dbias, sms, st);
     return e == cudaSuccess ? TERRA_OK : cuda_fail(e, "terra_swin_attn_bwd");
 }
@@ -282,7 +295,10 @@ int terra_swin_check(void* stream) {
     int timed_out_64 = 0;
     e = read_fwd_tc64_status(&timed_out_64);
     if (e != cudaSuccess) return cuda_fail(e, "terra_swin_check");
-    return (timed_out || timed_out_bwd || timed_out_64) ? TERRA_ERR_DEVICE_TIMEOUT : TERRA_OK;
+    int timed_out_kv = 0;
+    e = read_bwd_kv64_status(&timed_out_kv);
+    if (e != cudaSuccess) return cuda_fail(e, "terra_swin_check");
+    return (timed_out || timed_out_bwd || timed_out_64 || timed_out_kv) ? TERRA_ERR_DEVICE_TIMEOUT : TERRA_OK;
 }
 
 int terra_profile_enable(int on) {

@@ -1,0 +1,537 @@
+// Key side of the backward pass (dK, dV) on the tcgen05 tensor cores for head dim 64 and windows of up to 1024
+// tokens (window side <= 32).  The query side (dQ, dBias) of this regime runs the register-tile kernel.
+//
+// One persistent CTA per SM, bound to one head, walks over (batch, window, 128-key tile) items.  The tile's K and V
+// rows stay in shared memory; the window's queries stream through a ring of slots in chunks of 128 (Q, dO rows and
+// per-query lse, delta, bias code, mask label).  Orientation as in the small-window backward kernel: TMEM lanes =
+// keys, columns = queries.  Per chunk:
+//   S^T = K Q_c^T, dP^T = V dO_c^T                                   (SS MMAs, N = the chunk's queries)
+//   P^T = exp2(S^T scale + bias - lse_q), dS^T = P^T (dP^T - delta_q)   (elementwise warps, one key row per thread,
+//                                                                      written back over S^T / dP^T as bf16)
+//   dV += P^T dO_c, dK += dS^T Q_c                                   (A from TMEM, B = the chunk's rows, MN-major)
+// P is recomputed from the saved log-sum-exp, so the chunks are independent.
+// Roles: warps 0-7 elementwise (warps w and w + 4 share TMEM lane quarter w & 3 and take the chunk's first / second
+// 64 query columns), warp 8 issues every MMA, warps 9-11 gather rows with cp.async.  Head dim 64 is kept as two
+// 32-column halves in the 64-byte-swizzled operand layout (lo | hi regions), as in the forward kernel of this regime.
+// TMEM columns: S^T 0..127, dP^T 128..255, dV 256..319, dK 320..383.
+// Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, all roles leave their loops, TMEM is
+// released and the host reads the device status word.  Every role follows every ring item by item.
+#include "swin_common.cuh"
+#include "swin_kernels.h"
+#include "tc_common.cuh"
+
+namespace terra {
+
+__device__ int g_bwd_kv64_timeout = 0;   // set when a bounded wait expired in any CTA of the kernel below
+
+namespace {
+
+using namespace tc;
+
+constexpr int kMmaWarp = 8;
+constexpr int kLoaderWarp0 = 9;
+constexpr int kLoaderThreads = 96;
+constexpr int kThreads = 384;
+constexpr int kWorkThreads = 256;
+constexpr int kRegsLaunch = 168, kRegsWork = 208, kRegsOther = 80;
+static_assert(2 * (kRegsWork - kRegsLaunch) <= (kRegsLaunch - kRegsOther), "register hand-over does not balance");
+
+constexpr int kD = 64;
+constexpr int kHalfBytes = 64;
+constexpr int kTile = 128;                            // keys per item, queries per chunk
+constexpr int kHalf = kTile * kHalfBytes;             // 8192: one 32-column half of 128 rows
+constexpr int kKvStages = 2, kSlots = 3;
+// key stage: K lo | K hi | V lo | V hi, then per key row: 4 * bias code, label, token
+constexpr int kOffKlo = 0, kOffKhi = kHalf, kOffVlo = 2 * kHalf, kOffVhi = 3 * kHalf;
+constexpr int kKvRows = 4 * kHalf;                    // 32768
+constexpr int kOffKCode = kKvRows, kOffKLab = kKvRows + 512, kOffKTok = kKvRows + 1024;
+constexpr int kKvStageBytes = kKvRows + 2048;
+// query slot: Q lo | Q hi | dO lo | dO hi, then per query column: 4 * bias code, label, lse * log2(e), delta
+constexpr int kOffQlo = 0, kOffQhi = kHalf, kOffGlo = 2 * kHalf, kOffGhi = 3 * kHalf;
+constexpr int kOffQCode = 4 * kHalf, kOffQLab = kOffQCode + 512, kOffQLse = kOffQCode + 1024, kOffQDelta = kOffQCode + 1536;
+constexpr int kSlotBytes = 4 * kHalf + 2048;          // 34816
+constexpr int kOffSlots = kKvStages * kKvStageBytes;  // 69632
+constexpr int kBiasFloats = 6048;
+constexpr int kOffBias = kOffSlots + kSlots * kSlotBytes;
+constexpr int kOffBars = ((kOffBias + kBiasFloats * 4 + 1023) / 1024) * 1024;
+constexpr int kSmemBytes = kOffBars + 1024;
+static_assert(kKvStageBytes % 1024 == 0 && kSlotBytes % 1024 == 0, "tiles keep the swizzle alignment");
+static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
+constexpr int kColS = 0, kColDP = 128, kColDV = 256, kColDK = 320;
+
+__device__ __forceinline__ int code_stride(int w) { return w + 32; }
+
+struct Item {
+    int b, kt;
+    WindowRef r;
+    int npad;      // query slots rounded up to 16
+    int nch;       // 128-query chunks
+    bool has;      // the window has this key tile
+    bool masked;
+};
+
+__device__ __forceinline__ Item make_item(const Geo& g, const ItemCursor& c) {
+    Item x;
+    x.kt = c.head;                                    // the cursor's fastest digit counts key tiles here
+    x.b = c.b;
+    x.r = window_ref_rc(g, c.wr, c.wc);
+    x.npad = (x.r.n + 15) & ~15;
+    x.nch = (x.npad + kTile - 1) / kTile;
+    x.has = x.kt * kTile < x.r.n;
+    const int r0 = x.r.wr * g.w, c0 = x.r.wc * g.w;
+    const bool mh = !g.ph && g.sh > 0 && r0 < g.H - g.sh && r0 + x.r.eh > g.H - g.sh;
+    const bool mw = !g.pw && g.sw > 0 && c0 < g.W - g.sw && c0 + x.r.ew > g.W - g.sw;
+    x.masked = mh || mw;
+    return x;
+}
+
+__device__ __forceinline__ int offset_token(const Geo& g, const WindowRef& r, int a, int b, int& code, int& label) {
+    int u = r.wr * g.w + a + g.sh;
+    if (u >= g.H) u -= g.H;
+    int v = r.wc * g.w + b + g.sw;
+    if (v >= g.W) v -= g.W;
+    label = ((!g.ph && u < g.sh) ? 2 : 0) + ((!g.pw && v < g.sw) ? 1 : 0);
+    code = a * code_stride(g.w) + b;
+    return u * g.W + v;
+}
+
+__device__ __forceinline__ float lds_f32(uint32_t addr) {
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ int4 lds_i4(uint32_t addr) {
+    int4 v;
+    asm volatile("ld.shared.v4.s32 {%0,%1,%2,%3}, [%4];\n" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ float4 lds_f4(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];\n" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ int lds_i32(uint32_t addr) {
+    int v;
+    asm volatile("ld.shared.s32 %0, [%1];\n" : "=r"(v) : "r"(addr));
+    return v;
+}
+
+// 16 query columns [c, c + 16) of one key row: P = exp2(S scale + bias - lse), dS = P (dP - delta), packed to bf16.
+// `bias_row` = shared address of the bias table + the key row's part of the index (the -inf zone if the row has no
+// token); a query column without a token has lse = +inf, so its P is 0.
+template <bool MASKED>
+__device__ __forceinline__ void cols16(const uint32_t (&rs)[16], const uint32_t (&rp)[16], int c, uint32_t bias_row, int klabel,
+                                       uint32_t sl_a, float scale, uint32_t (&pk_p)[8], uint32_t (&pk_ds)[8]) {
+    float p[16], ds[16];
+#pragma unroll
+    for (int e4 = 0; e4 < 4; ++e4) {
+        const int4 co = lds_i4(sl_a + kOffQCode + 4 * (c + e4 * 4));
+        const float4 l2 = lds_f4(sl_a + kOffQLse + 4 * (c + e4 * 4));
+        const float4 dl = lds_f4(sl_a + kOffQDelta + 4 * (c + e4 * 4));
+        int4 ql = make_int4(0, 0, 0, 0);
+        if (MASKED) ql = lds_i4(sl_a + kOffQLab + 4 * (c + e4 * 4));
+        const int cov[4] = {co.x, co.y, co.z, co.w}, qlv[4] = {ql.x, ql.y, ql.z, ql.w};
+        const float l2v[4] = {l2.x, l2.y, l2.z, l2.w}, dlv[4] = {dl.x, dl.y, dl.z, dl.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int i = e4 * 4 + e;
+            float xv = fmaf(__uint_as_float(rs[i]), scale, lds_f32(bias_row + cov[e])) - l2v[e];
+            if (MASKED && qlv[e] != klabel) xv = -INFINITY;
+            p[i] = fast_exp2(xv);
+            ds[i] = p[i] * (__uint_as_float(rp[i]) - dlv[e]);
+        }
+    }
+#pragma unroll
+    for (int e2 = 0; e2 < 8; ++e2) {
+        pk_p[e2] = pack_bf16(p[2 * e2], p[2 * e2 + 1]);
+        pk_ds[e2] = pack_bf16(ds[2 * e2], ds[2 * e2 + 1]);
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
+                     const __nv_bfloat16* __restrict__ v, const __nv_bfloat16* __restrict__ d_o,
+                     const float* __restrict__ bias_prep, const float* __restrict__ lse, const float* __restrict__ delta,
+                     __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv, long long n_items, int ctas_per_head,
+                     int max_tiles) {
+    extern __shared__ __align__(1024) unsigned char smem[];
+    const uint32_t smem0 = smem_u32(smem);
+    const uint32_t bar0 = smem0 + kOffBars;
+    auto bar_kvfull = [&](int s) { return bar0 + 8u * s; };              // the tile's K, V rows and key tables are there
+    auto bar_kvempty = [&](int s) { return bar0 + 8u * (2 + s); };       // ... and no longer needed
+    auto bar_qfull = [&](int s) { return bar0 + 8u * (4 + s); };         // a query chunk is in ring slot s
+    auto bar_qempty = [&](int s) { return bar0 + 8u * (7 + s); };        // ... and every MMA that reads it is complete
+    const uint32_t bar_sdp = bar0 + 8u * 10;                              // S^T and dP^T of a chunk are in TMEM
+    const uint32_t bar_ds = bar0 + 8u * 11;                               // bf16 P^T and dS^T of the chunk are in TMEM
+    const uint32_t bar_acc = bar0 + 8u * 12;                              // dV, dK of the item are final
+    const uint32_t bar_accfree = bar0 + 8u * 13;                          // ... and have been read
+    unsigned char* tail = smem + kOffBars + 8 * 14;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail);
+    volatile int* cta_abort = reinterpret_cast<volatile int*>(tail + 8);
+
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int warp = tid >> 5;
+    const int head = blockIdx.x % g.heads;
+    const int cta_in_head = blockIdx.x / g.heads;
+
+    if (tid == 0) {
+        for (int s = 0; s < kKvStages; ++s) {
+            mbar_init(bar_kvfull(s), kLoaderThreads);
+            mbar_init(bar_kvempty(s), 1 + kWorkThreads);   // the issuer's commit + every elementwise thread
+        }
+        for (int s = 0; s < kSlots; ++s) {
+            mbar_init(bar_qfull(s), kLoaderThreads);
+            mbar_init(bar_qempty(s), 1);
+        }
+        mbar_init(bar_sdp, 1);
+        mbar_init(bar_ds, kWorkThreads);
+        mbar_init(bar_acc, 1);
+        mbar_init(bar_accfree, kWorkThreads);
+        *cta_abort = 0;
+        fence_barrier_init();
+    }
+    for (int i = tid; i < kBiasFloats; i += kThreads)
+        reinterpret_cast<float*>(smem + kOffBias)[i] = bias_prep[(size_t)head * kBiasFloats + i];
+    fence_proxy_async();
+    if (warp == kMmaWarp) {
+        tmem_alloc(smem_u32(tmem_slot), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int cs = code_stride(g.w);
+    const int c0 = (g.w - 1) * (cs + 1);
+    const size_t HW = (size_t)g.H * g.W;
+
+    if (warp >= kMmaWarp) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kRegsOther));
+    if (warp >= kLoaderWarp0) {
+        // ------------------------------------------------------------------ loaders
+        // Two lanes per row (lane parity = the row's lo / hi half, four 16-byte copies each).  A group of copies is
+        // published when the next one has been issued; if a ring has no free place the pending group is published first.
+        const int lt = (warp - kLoaderWarp0) * 32 + lane;
+        const int hf = lt & 1;
+        const int lrow = lt >> 1;
+        constexpr int kRowsPerIter = kLoaderThreads / 2;      // 48
+        int kuse = 0;
+        long long ru = 0;
+        uint32_t pending_bar = 0;
+        bool ok = true;
+        auto acquire = [&](uint32_t bar, uint32_t parity) -> bool {
+            if (pending_bar && !__all_sync(0xffffffffu, mbar_test_wait(bar, parity))) {
+                cp_async_wait<0>();
+                fence_proxy_async();
+                mbar_arrive(pending_bar);
+                pending_bar = 0;
+            }
+            return mbar_wait_all(bar, parity, cta_abort);
+        };
+        auto issued = [&](uint32_t bar) {
+            cp_async_commit();
+            if (pending_bar) {
+                cp_async_wait<1>();
+                fence_proxy_async();
+                mbar_arrive(pending_bar);
+            }
+            pending_bar = bar;
+        };
+        ItemCursor cur = cursor_init(cta_in_head, ctas_per_head, max_tiles, g.Mw, g.Mh);
+        for (long long it = cta_in_head; ok && it < n_items; it += ctas_per_head, cursor_advance(cur, max_tiles, g.Mw, g.Mh)) {
+            const Item x = make_item(g, cur);
+            if (!x.has) continue;
+            const int ks = kuse % kKvStages;
+            ok = acquire(bar_kvempty(ks), ((kuse / kKvStages) & 1) ^ 1);
+            if (!ok) break;
+            const size_t sample_off = (size_t)x.b * HW;
+            const int ew = x.r.ew;
+            const int q_r = kRowsPerIter / ew, r_r = kRowsPerIter - q_r * ew;
+            // ---- the key tile: K, V rows (rows without a token as zeros) and the key tables
+            {
+                unsigned char* st = smem + ks * kKvStageBytes;
+                const uint32_t sb = smem0 + ks * kKvStageBytes + hf * kHalf;
+                const int slot0 = x.kt * kTile;
+                for (int row = lt; row < kTile; row += kLoaderThreads) {
+                    const int slot = slot0 + row;
+                    int code = 0, label = 0xff, tok = -1;
+                    if (slot < x.r.n) {
+                        const int a = slot / ew;
+                        tok = offset_token(g, x.r, a, slot - a * ew, code, label);
+                    }
+                    reinterpret_cast<int*>(st + kOffKCode)[row] = 4 * code;
+                    reinterpret_cast<int*>(st + kOffKLab)[row] = label;
+                    reinterpret_cast<int*>(st + kOffKTok)[row] = tok;
+                }
+                int a_r = (slot0 + lrow) / ew, b_r = (slot0 + lrow) - a_r * ew;
+                for (int row = lrow; row < kTile; row += kRowsPerIter, a_r += q_r, b_r += r_r) {
+                    if (b_r >= ew) { b_r -= ew; ++a_r; }
+                    const __nv_bfloat16 *sk = k, *sv = v;
+                    int bytes = 0;
+                    if (slot0 + row < x.r.n) {
+                        int code, label;
+                        const int tok = offset_token(g, x.r, a_r, b_r, code, label);
+                        const size_t off = (sample_off + (size_t)tok) * g.ts + head * kD + hf * 32;
+                        sk = k + off; sv = v + off;
+                        bytes = 16;
+                    }
+#pragma unroll
+                    for (int c4 = 0; c4 < 4; ++c4) {
+                        const uint32_t so = tile_off<32>(row, c4);
+                        cp_async16(sb + kOffKlo + so, bytes ? sk + c4 * 8 : sk, bytes);
+                        cp_async16(sb + kOffVlo + so, bytes ? sv + c4 * 8 : sv, bytes);
+                    }
+                }
+                issued(bar_kvfull(ks));
+            }
+            // ---- the window's queries, chunk by chunk
+            for (int c = 0; c < x.nch; ++c, ++ru) {
+                const int s = (int)(ru % kSlots);
+                ok = acquire(bar_qempty(s), (uint32_t)((ru / kSlots) & 1) ^ 1u);
+                if (!ok) break;
+                unsigned char* sl = smem + kOffSlots + s * kSlotBytes;
+                const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes + hf * kHalf;
+                const int ncols = min(kTile, x.npad - c * kTile);
+                for (int row = lt; row < kTile; row += kLoaderThreads) {
+                    const int slot = c * kTile + row;
+                    int code = 0, label = 0xff;
+                    float l2 = INFINITY, dl = 0.f;              // no token: P = exp2(.. - inf) = 0
+                    if (slot < x.r.n) {
+                        const int a = slot / ew;
+                        const int tok = offset_token(g, x.r, a, slot - a * ew, code, label);
+                        const size_t li = (sample_off + (size_t)tok) * g.heads + head;
+                        l2 = __ldg(lse + li) * kLog2e;
+                        dl = __ldg(delta + li);
+                    }
+                    reinterpret_cast<int*>(sl + kOffQCode)[row] = 4 * code;
+                    reinterpret_cast<int*>(sl + kOffQLab)[row] = label;
+                    reinterpret_cast<float*>(sl + kOffQLse)[row] = l2;
+                    reinterpret_cast<float*>(sl + kOffQDelta)[row] = dl;
+                }
+                const int slot_first = c * kTile + lrow;
+                int a_r = slot_first / ew, b_r = slot_first - a_r * ew;
+                for (int row = lrow; row < ncols; row += kRowsPerIter, a_r += q_r, b_r += r_r) {
+                    if (b_r >= ew) { b_r -= ew; ++a_r; }
+                    const __nv_bfloat16 *sq = q, *sg = d_o;
+                    int bytes = 0;
+                    if (c * kTile + row < x.r.n) {
+                        int code, label;
+                        const int tok = offset_token(g, x.r, a_r, b_r, code, label);
+                        sq = q + (sample_off + (size_t)tok) * g.ts + head * kD + hf * 32;
+                        sg = d_o + ((sample_off + (size_t)tok) * g.heads + head) * kD + hf * 32;
+                        bytes = 16;
+                    }
+#pragma unroll
+                    for (int c4 = 0; c4 < 4; ++c4) {
+                        const uint32_t so = tile_off<32>(row, c4);
+                        cp_async16(sb + kOffQlo + so, bytes ? sq + c4 * 8 : sq, bytes);
+                        cp_async16(sb + kOffGlo + so, bytes ? sg + c4 * 8 : sg, bytes);
+                    }
+                }
+                issued(bar_qfull(s));
+            }
+            ++kuse;
+        }
+        if (pending_bar) {
+            cp_async_wait<0>();
+            fence_proxy_async();
+            mbar_arrive(pending_bar);
+        }
+    } else {
+        // ------------------------------------------------------------------ MMA issuer
+        const uint32_t idesc_acc = make_idesc_bf16(128, kD, 0, 1);       // A from TMEM, B = 16 rows x 64 (MN-major)
+        int kuse = 0, n_chunk = 0;
+        long long ru = 0;
+        bool ok = true;
+        ItemCursor cur = cursor_init(cta_in_head, ctas_per_head, max_tiles, g.Mw, g.Mh);
+        for (long long it = cta_in_head; ok && it < n_items; it += ctas_per_head, cursor_advance(cur, max_tiles, g.Mw, g.Mh)) {
+            const Item x = make_item(g, cur);
+            if (!x.has) continue;
+            const int ks = kuse % kKvStages;
+            ok = mbar_wait_all(bar_kvfull(ks), (kuse / kKvStages) & 1, cta_abort);
+            if (!ok) break;
+            fence_proxy_async();
+            const uint32_t kb = smem0 + ks * kKvStageBytes;
+            for (int c = 0; c < x.nch && ok; ++c, ++ru, ++n_chunk) {
+                const int s = (int)(ru % kSlots);
+                ok = mbar_wait_all(bar_qfull(s), (uint32_t)((ru / kSlots) & 1), cta_abort);
+                if (!ok) break;
+                fence_proxy_async();
+                tc_fence_after();
+                const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes;
+                const int ncols = min(kTile, x.npad - c * kTile);
+                // S^T = K Q_c^T, dP^T = V dO_c^T.  The buffers are free: the products that read the chunk before
+                // (as bf16 P^T / dS^T) were issued earlier from this thread.
+                const uint32_t idesc = make_idesc_bf16(128, ncols, 0, 0);
+                if (elect_one()) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint32_t off = (j >> 1) * kHalf + (j & 1) * 32;
+                        mma_ss(tmem_base + kColS, make_sdesc_sw64(kb + kOffKlo + off, 512), make_sdesc_sw64(sb + kOffQlo + off, 512), idesc, j > 0 ? 1u : 0u);
+                    }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint32_t off = (j >> 1) * kHalf + (j & 1) * 32;
+                        mma_ss(tmem_base + kColDP, make_sdesc_sw64(kb + kOffVlo + off, 512), make_sdesc_sw64(sb + kOffGlo + off, 512), idesc, j > 0 ? 1u : 0u);
+                    }
+                    mma_commit(bar_sdp);
+                }
+                __syncwarp();
+                ok = mbar_wait_all(bar_ds, n_chunk & 1, cta_abort);
+                if (ok && c == 0 && kuse > 0) ok = mbar_wait_all(bar_accfree, (kuse - 1) & 1, cta_abort);
+                if (!ok) break;
+                tc_fence_after();
+                // dV += P^T dO_c, dK += dS^T Q_c over the chunk's query columns
+                {
+                    const uint64_t gd = make_sdesc_sw64_mn(sb + kOffGlo, kHalf, 512), qd = make_sdesc_sw64_mn(sb + kOffQlo, kHalf, 512);
+                    const uint32_t g_lo = sdesc_lo(gd), q_lo = sdesc_lo(qd), d_hi = sdesc_hi(gd);
+                    const int nks = ncols >> 4;
+                    if (elect_one()) {
+                        int j = 0;
+                        if (c == 0) {
+                            mma_ts_h<false>(tmem_base + kColDV, tmem_base + kColS, g_lo, d_hi, idesc_acc);
+                            mma_ts_h<false>(tmem_base + kColDK, tmem_base + kColDP, q_lo, d_hi, idesc_acc);
+                            j = 1;
+                        }
+                        for (; j < nks; ++j) {
+                            mma_ts_h<true>(tmem_base + kColDV, tmem_base + kColS + 16 * j, g_lo + 64 * j, d_hi, idesc_acc);
+                            mma_ts_h<true>(tmem_base + kColDK, tmem_base + kColDP + 16 * j, q_lo + 64 * j, d_hi, idesc_acc);
+                        }
+                        mma_commit(bar_qempty(s));
+                        if (c == x.nch - 1) {
+                            mma_commit(bar_acc);
+                            mma_commit(bar_kvempty(ks));
+                        }
+                    }
+                    __syncwarp();
+                }
+            }
+            ++kuse;
+        }
+    }
+    } else {
+        // ------------------------------------------------------------------ elementwise warps
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(kRegsWork));
+        const int hcol = warp >> 2;                       // which 64 query columns of a chunk
+        const int quarter = warp & 3;
+        const int krow = 32 * quarter + lane;             // key row inside the tile
+        const uint32_t lane_addr = ((uint32_t)(32 * quarter)) << 16;
+        const float scale = g.scale_log2e;
+        const float out_scale = g.scale_log2e * kLn2;     // dK carries the score scale
+        int kuse = 0, n_chunk = 0;
+        long long ru = 0;
+        bool ok = true;
+        ItemCursor cur = cursor_init(cta_in_head, ctas_per_head, max_tiles, g.Mw, g.Mh);
+        for (long long it = cta_in_head; ok && it < n_items; it += ctas_per_head, cursor_advance(cur, max_tiles, g.Mw, g.Mh)) {
+            const Item x = make_item(g, cur);
+            if (!x.has) continue;
+            const int ks = kuse % kKvStages;
+            if (!mbar_wait_all(bar_kvfull(ks), (kuse / kKvStages) & 1, cta_abort)) break;
+            const uint32_t st_a = smem0 + ks * kKvStageBytes;
+            const int kcode4 = lds_i32(st_a + kOffKCode + 4 * krow);
+            const int klabel = lds_i32(st_a + kOffKLab + 4 * krow);
+            const int ktok = lds_i32(st_a + kOffKTok + 4 * krow);
+            mbar_arrive(bar_kvempty(ks));                 // this thread has what it needs from the key stage
+            // bias index = code_query - code_key + c0; a key row without a token reads the table's -inf zone
+            const uint32_t bias_row = smem0 + kOffBias + (ktok >= 0 ? 4 * c0 - kcode4 : 4 * (2 * c0 + 1));
+            for (int c = 0; c < x.nch && ok; ++c, ++ru, ++n_chunk) {
+                const int s = (int)(ru % kSlots);
+                const uint32_t sl_a = smem0 + kOffSlots + s * kSlotBytes;
+                const int ncols = min(kTile, x.npad - c * kTile);
+                ok = mbar_wait_all(bar_sdp, n_chunk & 1, cta_abort);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t t_s = tmem_base + lane_addr + kColS, t_dp = tmem_base + lane_addr + kColDP;
+                const int col_end = min(ncols, 64 * hcol + 64);
+                for (int cc = 64 * hcol; cc < col_end; cc += 16) {
+                    uint32_t rs[16], rp[16], pk_p[8], pk_ds[8];
+                    tmem_ld16(t_s + cc, rs);
+                    tmem_ld16(t_dp + cc, rp);
+                    tmem_ld_wait();
+                    if (x.masked) cols16<true>(rs, rp, cc, bias_row, klabel, sl_a, scale, pk_p, pk_ds);
+                    else cols16<false>(rs, rp, cc, bias_row, klabel, sl_a, scale, pk_p, pk_ds);
+                    tmem_st8(t_s + cc, pk_p);              // 16 queries -> 8 packed columns at the group's own place
+                    tmem_st8(t_dp + cc, pk_ds);
+                }
+                tmem_st_wait();
+                tc_fence_before();
+                mbar_arrive(bar_ds);
+            }
+            if (!ok) break;
+            // ---- read-out: dV rows by warps 0-3, dK rows by warps 4-7
+            if (!mbar_wait_all(bar_acc, kuse & 1, cta_abort)) break;
+            tc_fence_after();
+            uint32_t r0[32], r1[32];
+            tmem_ld32(tmem_base + lane_addr + (hcol == 0 ? kColDV : kColDK), r0);
+            tmem_ld32(tmem_base + lane_addr + (hcol == 0 ? kColDV : kColDK) + 32, r1);
+            tmem_ld_wait();
+            tc_fence_before();
+            mbar_arrive(bar_accfree);
+            if (ktok >= 0) {
+                const float f = hcol == 0 ? 1.f : out_scale;
+                __nv_bfloat16* out = hcol == 0 ? dv : dk;
+                uint4* dst = reinterpret_cast<uint4*>(out + ((size_t)x.b * HW + (size_t)ktok) * g.ts + head * kD);
+#pragma unroll
+                for (int c4 = 0; c4 < 4; ++c4) {
+                    uint4 a;
+                    a.x = pack_bf16(__uint_as_float(r0[c4 * 8 + 0]) * f, __uint_as_float(r0[c4 * 8 + 1]) * f);
+                    a.y = pack_bf16(__uint_as_float(r0[c4 * 8 + 2]) * f, __uint_as_float(r0[c4 * 8 + 3]) * f);
+                    a.z = pack_bf16(__uint_as_float(r0[c4 * 8 + 4]) * f, __uint_as_float(r0[c4 * 8 + 5]) * f);
+                    a.w = pack_bf16(__uint_as_float(r0[c4 * 8 + 6]) * f, __uint_as_float(r0[c4 * 8 + 7]) * f);
+                    dst[c4] = a;
+                }
+#pragma unroll
+                for (int c4 = 0; c4 < 4; ++c4) {
+                    uint4 a;
+                    a.x = pack_bf16(__uint_as_float(r1[c4 * 8 + 0]) * f, __uint_as_float(r1[c4 * 8 + 1]) * f);
+                    a.y = pack_bf16(__uint_as_float(r1[c4 * 8 + 2]) * f, __uint_as_float(r1[c4 * 8 + 3]) * f);
+                    a.z = pack_bf16(__uint_as_float(r1[c4 * 8 + 4]) * f, __uint_as_float(r1[c4 * 8 + 5]) * f);
+                    a.w = pack_bf16(__uint_as_float(r1[c4 * 8 + 6]) * f, __uint_as_float(r1[c4 * 8 + 7]) * f);
+                    dst[4 + c4] = a;
+                }
+            }
+            ++kuse;
+        }
+    }
+
+    // teardown: every role ends up here, also after an expired wait
+    cp_async_wait<0>();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == kMmaWarp) tmem_dealloc(tmem_base, 512);
+    if (tid == 0 && *cta_abort) atomicExch(&g_bwd_kv64_timeout, 1);
+}
+
+}  // namespace
+
+cudaError_t read_bwd_kv64_status(int* timed_out) {
+    int zero = 0;
+    cudaError_t e = cudaMemcpyFromSymbol(timed_out, g_bwd_kv64_timeout, sizeof(int));
+    if (e != cudaSuccess) return e;
+    if (*timed_out) e = cudaMemcpyToSymbol(g_bwd_kv64_timeout, &zero, sizeof(int));
+    return e;
+}
+
+bool bwd_kv64_supported(const Geo& g) { return g.d == 64 && g.w <= 32 && g.nmax <= 1024 && g.heads <= 148; }
+
+// `prep` = the prepared bias tables of the head-dim-64 forward kernel (kBiasFloats per head), filled by the caller
+cudaError_t launch_bwd_kv64(const Geo& g, const void* q, const void* k, const void* v, const void* d_o, const float* prep,
+                            const float* lse, const float* delta, void* dk, void* dv, int sm_count, cudaStream_t stream) {
+    const int max_tiles = (g.nmax + 127) >> 7;
+    const long long items = (long long)g.B * g.Mh * g.Mw * max_tiles;
+    long long cph = sm_count / g.heads;
+    if (cph < 1) cph = 1;
+    if (cph > items) cph = items;
+    cudaError_t e = cudaFuncSetAttribute(swin_bwd_kv64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    prof_begin("swin_bwd_kv64_kernel", stream);
+    swin_bwd_kv64_kernel<<<(unsigned)(cph * g.heads), kThreads, kSmemBytes, stream>>>(
+        g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)d_o, prep, lse, delta,
+        (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, items, (int)cph, max_tiles);
+    count_launch(stream);
+    return cudaGetLastError();
+}
+
+}  // namespace terra

@@ -457,9 +457,13 @@ cudaError_t launch_bwd_delta(const Geo& g, const void* o, const void* d_o, float
 
 cudaError_t launch_bwd_mma(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
                            const float* lse, const float* delta, const void* d_o,
-                           void* dq, void* dk, void* dv, float* dbias, int sm_count, cudaStream_t stream) {
+                           void* dq, void* dk, void* dv, float* dbias, int sm_count, cudaStream_t stream,
+                           bool query_side_only) {
     cudaError_t e = cudaMemsetAsync(dbias, 0, sizeof(float) * (size_t)(2 * g.w - 1) * (2 * g.w - 1) * g.heads, stream);
     if (e != cudaSuccess) return e;
+    if (query_side_only)      // dK, dV come from another kernel
+        return g.d == 32 ? launch_one<32, false>(g, q, k, v, d_o, bias, lse, delta, dq, nullptr, dbias, sm_count, stream)
+                         : launch_one<64, false>(g, q, k, v, d_o, bias, lse, delta, dq, nullptr, dbias, sm_count, stream);
     if (g.d == 32) {
         e = launch_one<32, true>(g, q, k, v, d_o, bias, lse, delta, dk, dv, nullptr, sm_count, stream);
         if (e != cudaSuccess) return e;

@@ -712,6 +712,13 @@ cudaError_t read_fwd_tc64_status(int* timed_out) {
     return e;
 }
 
+// prepared bias tables (kBiasFloats = 6048 floats per head) for the kernels of the head-dim-64 regime
+cudaError_t launch_bias_prep64(const Geo& g, const float* bias, float* prep, cudaStream_t stream) {
+    swin_fwd_bias_prep64_kernel<<<g.heads, 256, 0, stream>>>(bias, prep, g.w, g.heads);
+    count_launch(stream);
+    return cudaGetLastError();
+}
+
 bool fwd_tc64_supported(const Geo& g) { return g.d == 64 && g.w <= 32 && g.nmax <= 1024 && g.heads <= 148; }
 
 size_t fwd_tc64_workspace_bytes(const Geo& g) { return (size_t)g.heads * kBiasFloats * sizeof(float); }

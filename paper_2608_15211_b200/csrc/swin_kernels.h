@@ -34,6 +34,14 @@ size_t fwd_tc64_workspace_bytes(const Geo& g);
 cudaError_t launch_fwd_tc64(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
                             void* o, float* lse, void* workspace, int sm_count, cudaStream_t stream);
 cudaError_t read_fwd_tc64_status(int* timed_out);     // after the stream has been synchronised
+cudaError_t launch_bias_prep64(const Geo& g, const float* bias, float* prep, cudaStream_t stream);
+
+// tcgen05 key side (dK, dV) of the backward pass for head dim 64 and windows of up to 1024 tokens; `prep` = the
+// tables of launch_bias_prep64, `delta` as for the register-tile kernels
+bool bwd_kv64_supported(const Geo& g);
+cudaError_t launch_bwd_kv64(const Geo& g, const void* q, const void* k, const void* v, const void* d_o, const float* prep,
+                            const float* lse, const float* delta, void* dk, void* dv, int sm_count, cudaStream_t stream);
+cudaError_t read_bwd_kv64_status(int* timed_out);
 
 cudaError_t launch_bounded_wait_selftest(long long limit_cycles, cudaStream_t stream);
 cudaError_t launch_bias_prep(const Geo& g, const float* bias, float* prep, cudaStream_t stream);
@@ -52,6 +60,7 @@ cudaError_t launch_bwd_delta(const Geo& g, const void* o, const void* d_o, float
 // dK, dV (key-tile CTAs) and dQ, dBias (query-tile CTAs)
 cudaError_t launch_bwd_mma(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
                            const float* lse, const float* delta, const void* d_o,
-                           void* dq, void* dk, void* dv, float* dbias, int sm_count, cudaStream_t stream);
+                           void* dq, void* dk, void* dv, float* dbias, int sm_count, cudaStream_t stream,
+                           bool query_side_only = false);
 
 }  // namespace terra
