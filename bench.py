@@ -428,6 +428,7 @@ def main():
         kernel_flop = {"swin_fwd_tc_kernel": 4 * d * pairs, "swin_fwd_tc64_kernel": 4 * d * pairs, "swin_fwd_mma_kernel": 4 * d * pairs,
                        "swin_bwd_fused_kernel": 8 * d * pairs,
                        "swin_bwd_mma_kernel<key tiles>": 4 * d * pairs, "swin_bwd_mma_kernel<query tiles>": 4 * d * pairs,
+                       "swin_bwd_kv64_kernel": 4 * d * pairs,
                        "swin_bwd_delta_kernel": 0}
         kernels = []
         for kname, vals in kernel_ms.items():
