@@ -122,24 +122,37 @@ __device__ __forceinline__ int lds_i32(uint32_t addr) {
 template <bool MASKED>
 __device__ __forceinline__ void cols16(const uint32_t (&rs)[16], const uint32_t (&rp)[16], int c, uint32_t bias_row, int klabel,
                                        uint32_t sl_a, float scale, uint32_t (&pk_p)[8], uint32_t (&pk_ds)[8]) {
-    float p[16], ds[16];
+    // all table loads first (they are issued in program order), then the gathers that depend on them, then the math
+    int co[16], ql[16];
+    float l2[16], dl[16], bv[16];
 #pragma unroll
     for (int e4 = 0; e4 < 4; ++e4) {
-        const int4 co = lds_i4(sl_a + kOffQCode + 4 * (c + e4 * 4));
-        const float4 l2 = lds_f4(sl_a + kOffQLse + 4 * (c + e4 * 4));
-        const float4 dl = lds_f4(sl_a + kOffQDelta + 4 * (c + e4 * 4));
-        int4 ql = make_int4(0, 0, 0, 0);
-        if (MASKED) ql = lds_i4(sl_a + kOffQLab + 4 * (c + e4 * 4));
-        const int cov[4] = {co.x, co.y, co.z, co.w}, qlv[4] = {ql.x, ql.y, ql.z, ql.w};
-        const float l2v[4] = {l2.x, l2.y, l2.z, l2.w}, dlv[4] = {dl.x, dl.y, dl.z, dl.w};
+        const int4 c4 = lds_i4(sl_a + kOffQCode + 4 * (c + e4 * 4));
+        co[e4 * 4] = c4.x; co[e4 * 4 + 1] = c4.y; co[e4 * 4 + 2] = c4.z; co[e4 * 4 + 3] = c4.w;
+    }
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const int i = e4 * 4 + e;
-            float xv = fmaf(__uint_as_float(rs[i]), scale, lds_f32(bias_row + cov[e])) - l2v[e];
-            if (MASKED && qlv[e] != klabel) xv = -INFINITY;
-            p[i] = fast_exp2(xv);
-            ds[i] = p[i] * (__uint_as_float(rp[i]) - dlv[e]);
+    for (int e4 = 0; e4 < 4; ++e4) {
+        const float4 a = lds_f4(sl_a + kOffQLse + 4 * (c + e4 * 4));
+        const float4 b = lds_f4(sl_a + kOffQDelta + 4 * (c + e4 * 4));
+        l2[e4 * 4] = a.x; l2[e4 * 4 + 1] = a.y; l2[e4 * 4 + 2] = a.z; l2[e4 * 4 + 3] = a.w;
+        dl[e4 * 4] = b.x; dl[e4 * 4 + 1] = b.y; dl[e4 * 4 + 2] = b.z; dl[e4 * 4 + 3] = b.w;
+    }
+    if (MASKED) {
+#pragma unroll
+        for (int e4 = 0; e4 < 4; ++e4) {
+            const int4 q4 = lds_i4(sl_a + kOffQLab + 4 * (c + e4 * 4));
+            ql[e4 * 4] = q4.x; ql[e4 * 4 + 1] = q4.y; ql[e4 * 4 + 2] = q4.z; ql[e4 * 4 + 3] = q4.w;
         }
+    }
+#pragma unroll
+    for (int e = 0; e < 16; ++e) bv[e] = lds_f32(bias_row + co[e]);
+    float p[16], ds[16];
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
+        float xv = fmaf(__uint_as_float(rs[e]), scale, bv[e]) - l2[e];
+        if (MASKED && ql[e] != klabel) xv = -INFINITY;
+        p[e] = fast_exp2(xv);
+        ds[e] = p[e] * (__uint_as_float(rp[e]) - dl[e]);
     }
 #pragma unroll
     for (int e2 = 0; e2 < 8; ++e2) {
@@ -444,15 +457,33 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                 tc_fence_after();
                 const uint32_t t_s = tmem_base + lane_addr + kColS, t_dp = tmem_base + lane_addr + kColDP;
                 const int col_end = min(ncols, 64 * hcol + 64);
-                for (int cc = 64 * hcol; cc < col_end; cc += 16) {
-                    uint32_t rs[16], rp[16], pk_p[8], pk_ds[8];
-                    tmem_ld16(t_s + cc, rs);
-                    tmem_ld16(t_dp + cc, rp);
+                // groups of 16 columns; the next group's S^T / dP^T travel from TMEM while this one is worked on
+                uint32_t rs[16], rp[16], rs2[16], rp2[16], pk_p[8], pk_ds[8];
+                if (64 * hcol < col_end) {
+                    tmem_ld16(t_s + 64 * hcol, rs);
+                    tmem_ld16(t_dp + 64 * hcol, rp);
+                }
+                for (int cc = 64 * hcol; cc < col_end; cc += 32) {
                     tmem_ld_wait();
+                    if (cc + 16 < col_end) {
+                        tmem_ld16(t_s + cc + 16, rs2);
+                        tmem_ld16(t_dp + cc + 16, rp2);
+                    }
                     if (x.masked) cols16<true>(rs, rp, cc, bias_row, klabel, sl_a, scale, pk_p, pk_ds);
                     else cols16<false>(rs, rp, cc, bias_row, klabel, sl_a, scale, pk_p, pk_ds);
                     tmem_st8(t_s + cc, pk_p);              // 16 queries -> 8 packed columns at the group's own place
                     tmem_st8(t_dp + cc, pk_ds);
+                    if (cc + 16 < col_end) {
+                        tmem_ld_wait();
+                        if (cc + 32 < col_end) {
+                            tmem_ld16(t_s + cc + 32, rs);
+                            tmem_ld16(t_dp + cc + 32, rp);
+                        }
+                        if (x.masked) cols16<true>(rs2, rp2, cc + 16, bias_row, klabel, sl_a, scale, pk_p, pk_ds);
+                        else cols16<false>(rs2, rp2, cc + 16, bias_row, klabel, sl_a, scale, pk_p, pk_ds);
+                        tmem_st8(t_s + cc + 16, pk_p);
+                        tmem_st8(t_dp + cc + 16, pk_ds);
+                    }
                 }
                 tmem_st_wait();
                 tc_fence_before();
