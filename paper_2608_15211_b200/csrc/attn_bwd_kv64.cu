@@ -174,11 +174,13 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
     auto bar_kvempty = [&](int s) { return bar0 + 8u * (2 + s); };       // ... and no longer needed
     auto bar_qfull = [&](int s) { return bar0 + 8u * (4 + s); };         // a query chunk is in ring slot s
     auto bar_qempty = [&](int s) { return bar0 + 8u * (7 + s); };        // ... and every MMA that reads it is complete
-    const uint32_t bar_sdp = bar0 + 8u * 10;                              // S^T and dP^T of a chunk are in TMEM
-    const uint32_t bar_ds = bar0 + 8u * 11;                               // bf16 P^T and dS^T of the chunk are in TMEM
-    const uint32_t bar_acc = bar0 + 8u * 12;                              // dV, dK of the item are final
-    const uint32_t bar_accfree = bar0 + 8u * 13;                          // ... and have been read
-    unsigned char* tail = smem + kOffBars + 8 * 14;
+    // a chunk's two 64-query halves are separate buffers (columns 64 h of S^T and dP^T) with their own hand-overs:
+    // half h belongs to elementwise warps 4 h .. 4 h + 3, and the MMAs of one half run while the other is worked on
+    auto bar_sdp = [&](int h) { return bar0 + 8u * (10 + h); };          // S^T and dP^T of a half chunk are in TMEM
+    auto bar_ds = [&](int h) { return bar0 + 8u * (12 + h); };           // bf16 P^T and dS^T of the half chunk are in TMEM
+    const uint32_t bar_acc = bar0 + 8u * 14;                              // dV, dK of the item are final
+    const uint32_t bar_accfree = bar0 + 8u * 15;                          // ... and have been read
+    unsigned char* tail = smem + kOffBars + 8 * 16;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail);
     volatile int* cta_abort = reinterpret_cast<volatile int*>(tail + 8);
 
@@ -196,8 +198,10 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             mbar_init(bar_qfull(s), kLoaderThreads);
             mbar_init(bar_qempty(s), 1);
         }
-        mbar_init(bar_sdp, 1);
-        mbar_init(bar_ds, kWorkThreads);
+        for (int h = 0; h < 2; ++h) {
+            mbar_init(bar_sdp(h), 1);
+            mbar_init(bar_ds(h), kWorkThreads / 2);
+        }
         mbar_init(bar_acc, 1);
         mbar_init(bar_accfree, kWorkThreads);
         *cta_abort = 0;
@@ -354,7 +358,9 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
     } else {
         // ------------------------------------------------------------------ MMA issuer
         const uint32_t idesc_acc = make_idesc_bf16(128, kD, 0, 1);       // A from TMEM, B = 16 rows x 64 (MN-major)
-        int kuse = 0, n_chunk = 0;
+        const uint32_t sd_hi = sdesc_hi(make_sdesc_sw64(smem0, 512));    // common high word of the K-major descriptors
+        int kuse = 0;
+        int n_ds[2] = {0, 0};
         long long ru = 0;
         bool ok = true;
         ItemCursor cur = cursor_init(cta_in_head, ctas_per_head, max_tiles, g.Mw, g.Mh);
@@ -366,59 +372,89 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             if (!ok) break;
             fence_proxy_async();
             const uint32_t kb = smem0 + ks * kKvStageBytes;
-            for (int c = 0; c < x.nch && ok; ++c, ++ru, ++n_chunk) {
-                const int s = (int)(ru % kSlots);
-                ok = mbar_wait_all(bar_qfull(s), (uint32_t)((ru / kSlots) & 1), cta_abort);
-                if (!ok) break;
+            // queries of half h of chunk c (a multiple of 16; 0: the half does not exist)
+            auto half_cols = [&](int c, int h) { return max(0, min(64, x.npad - c * kTile - 64 * h)); };
+            auto chunk_ready = [&](long long use) -> bool {
+                if (!mbar_wait_all(bar_qfull((int)(use % kSlots)), (uint32_t)((use / kSlots) & 1), cta_abort)) return false;
                 fence_proxy_async();
+                return true;
+            };
+            // S^T = K Q^T, dP^T = V dO^T for the 64 queries of half h of the chunk in ring slot `sb`
+            // (descriptor low words = start address in 16-byte units: + 2 per 32-byte K step, + kHalf / 16 for the hi half)
+            const uint32_t k_lo = sdesc_lo(make_sdesc_sw64(kb + kOffKlo, 512)), v_lo = sdesc_lo(make_sdesc_sw64(kb + kOffVlo, 512));
+            auto issue_sdp = [&](int h, uint32_t sb, int nc) {
+                const uint32_t idesc = make_idesc_bf16(128, nc, 0, 0);
+                const uint32_t q_lo = sdesc_lo(make_sdesc_sw64(sb + kOffQlo + h * 64 * kHalfBytes, 512));
+                const uint32_t g_lo = sdesc_lo(make_sdesc_sw64(sb + kOffGlo + h * 64 * kHalfBytes, 512));
+                const uint32_t t_s = tmem_base + kColS + 64 * h, t_dp = tmem_base + kColDP + 64 * h;
+                constexpr uint32_t kHi = kHalf >> 4;
                 tc_fence_after();
-                const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes;
-                const int ncols = min(kTile, x.npad - c * kTile);
-                // S^T = K Q_c^T, dP^T = V dO_c^T.  The buffers are free: the products that read the chunk before
-                // (as bf16 P^T / dS^T) were issued earlier from this thread.
-                const uint32_t idesc = make_idesc_bf16(128, ncols, 0, 0);
                 if (elect_one()) {
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const uint32_t off = (j >> 1) * kHalf + (j & 1) * 32;
-                        mma_ss(tmem_base + kColS, make_sdesc_sw64(kb + kOffKlo + off, 512), make_sdesc_sw64(sb + kOffQlo + off, 512), idesc, j > 0 ? 1u : 0u);
-                    }
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const uint32_t off = (j >> 1) * kHalf + (j & 1) * 32;
-                        mma_ss(tmem_base + kColDP, make_sdesc_sw64(kb + kOffVlo + off, 512), make_sdesc_sw64(sb + kOffGlo + off, 512), idesc, j > 0 ? 1u : 0u);
-                    }
-                    mma_commit(bar_sdp);
+                    mma_ss_h<false>(t_s, k_lo, q_lo, sd_hi, idesc);
+                    mma_ss_h<true>(t_s, k_lo + 2, q_lo + 2, sd_hi, idesc);
+                    mma_ss_h<true>(t_s, k_lo + kHi, q_lo + kHi, sd_hi, idesc);
+                    mma_ss_h<true>(t_s, k_lo + kHi + 2, q_lo + kHi + 2, sd_hi, idesc);
+                    mma_ss_h<false>(t_dp, v_lo, g_lo, sd_hi, idesc);
+                    mma_ss_h<true>(t_dp, v_lo + 2, g_lo + 2, sd_hi, idesc);
+                    mma_ss_h<true>(t_dp, v_lo + kHi, g_lo + kHi, sd_hi, idesc);
+                    mma_ss_h<true>(t_dp, v_lo + kHi + 2, g_lo + kHi + 2, sd_hi, idesc);
+                    mma_commit(bar_sdp(h));
                 }
                 __syncwarp();
-                ok = mbar_wait_all(bar_ds, n_chunk & 1, cta_abort);
-                if (ok && c == 0 && kuse > 0) ok = mbar_wait_all(bar_accfree, (kuse - 1) & 1, cta_abort);
-                if (!ok) break;
-                tc_fence_after();
-                // dV += P^T dO_c, dK += dS^T Q_c over the chunk's query columns
-                {
-                    const uint64_t gd = make_sdesc_sw64_mn(sb + kOffGlo, kHalf, 512), qd = make_sdesc_sw64_mn(sb + kOffQlo, kHalf, 512);
+            };
+            ok = chunk_ready(ru);
+            if (!ok) break;
+            for (int h = 0; h < 2; ++h)
+                if (half_cols(0, h) > 0) issue_sdp(h, smem0 + kOffSlots + (int)(ru % kSlots) * kSlotBytes, half_cols(0, h));
+            for (int c = 0; c < x.nch && ok; ++c, ++ru) {
+                const int s = (int)(ru % kSlots);
+                const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes;
+                const bool has_next = c + 1 < x.nch;
+                if (has_next) {
+                    ok = chunk_ready(ru + 1);
+                    if (!ok) break;
+                }
+                const uint32_t sb_n = smem0 + kOffSlots + (int)((ru + 1) % kSlots) * kSlotBytes;
+                for (int h = 0; h < 2 && ok; ++h) {
+                    const int nc = half_cols(c, h);
+                    if (nc == 0) continue;
+                    ok = mbar_wait_all(bar_ds(h), n_ds[h] & 1, cta_abort);
+                    ++n_ds[h];
+                    if (ok && c == 0 && h == 0 && kuse > 0) ok = mbar_wait_all(bar_accfree, (kuse - 1) & 1, cta_abort);
+                    if (!ok) break;
+                    tc_fence_after();
+                    // dV += P^T dO, dK += dS^T Q over the half chunk's query columns
+                    const uint64_t gd = make_sdesc_sw64_mn(sb + kOffGlo + h * 64 * kHalfBytes, kHalf, 512);
+                    const uint64_t qd = make_sdesc_sw64_mn(sb + kOffQlo + h * 64 * kHalfBytes, kHalf, 512);
                     const uint32_t g_lo = sdesc_lo(gd), q_lo = sdesc_lo(qd), d_hi = sdesc_hi(gd);
-                    const int nks = ncols >> 4;
+                    const uint32_t t_p = tmem_base + kColS + 64 * h, t_ds = tmem_base + kColDP + 64 * h;
+                    const int nks = nc >> 4;
                     if (elect_one()) {
                         int j = 0;
-                        if (c == 0) {
-                            mma_ts_h<false>(tmem_base + kColDV, tmem_base + kColS, g_lo, d_hi, idesc_acc);
-                            mma_ts_h<false>(tmem_base + kColDK, tmem_base + kColDP, q_lo, d_hi, idesc_acc);
+                        if (c == 0 && h == 0) {
+                            mma_ts_h<false>(tmem_base + kColDV, t_p, g_lo, d_hi, idesc_acc);
+                            mma_ts_h<false>(tmem_base + kColDK, t_ds, q_lo, d_hi, idesc_acc);
                             j = 1;
                         }
                         for (; j < nks; ++j) {
-                            mma_ts_h<true>(tmem_base + kColDV, tmem_base + kColS + 16 * j, g_lo + 64 * j, d_hi, idesc_acc);
-                            mma_ts_h<true>(tmem_base + kColDK, tmem_base + kColDP + 16 * j, q_lo + 64 * j, d_hi, idesc_acc);
-                        }
-                        mma_commit(bar_qempty(s));
-                        if (c == x.nch - 1) {
-                            mma_commit(bar_acc);
-                            mma_commit(bar_kvempty(ks));
+                            mma_ts_h<true>(tmem_base + kColDV, t_p + 16 * j, g_lo + 64 * j, d_hi, idesc_acc);
+                            mma_ts_h<true>(tmem_base + kColDK, t_ds + 16 * j, q_lo + 64 * j, d_hi, idesc_acc);
                         }
                     }
                     __syncwarp();
+                    // the half's buffers are free again (the products that read them were issued just above): the
+                    // next chunk's scores for this half follow at once, while the other half is being worked on
+                    if (has_next && half_cols(c + 1, h) > 0) issue_sdp(h, sb_n, half_cols(c + 1, h));
                 }
+                if (!ok) break;
+                if (elect_one()) {
+                    mma_commit(bar_qempty(s));
+                    if (!has_next) {
+                        mma_commit(bar_acc);
+                        mma_commit(bar_kvempty(ks));
+                    }
+                }
+                __syncwarp();
             }
             ++kuse;
         }
@@ -432,7 +468,7 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
         const uint32_t lane_addr = ((uint32_t)(32 * quarter)) << 16;
         const float scale = g.scale_log2e;
         const float out_scale = g.scale_log2e * kLn2;     // dK carries the score scale
-        int kuse = 0, n_chunk = 0;
+        int kuse = 0, n_half = 0;                       // items; half chunks this group has worked on
         long long ru = 0;
         bool ok = true;
         ItemCursor cur = cursor_init(cta_in_head, ctas_per_head, max_tiles, g.Mw, g.Mh);
@@ -448,12 +484,14 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             mbar_arrive(bar_kvempty(ks));                 // this thread has what it needs from the key stage
             // bias index = code_query - code_key + c0; a key row without a token reads the table's -inf zone
             const uint32_t bias_row = smem0 + kOffBias + (ktok >= 0 ? 4 * c0 - kcode4 : 4 * (2 * c0 + 1));
-            for (int c = 0; c < x.nch && ok; ++c, ++ru, ++n_chunk) {
+            for (int c = 0; c < x.nch && ok; ++c, ++ru) {
                 const int s = (int)(ru % kSlots);
                 const uint32_t sl_a = smem0 + kOffSlots + s * kSlotBytes;
                 const int ncols = min(kTile, x.npad - c * kTile);
-                ok = mbar_wait_all(bar_sdp, n_chunk & 1, cta_abort);
+                if (ncols <= 64 * hcol) continue;          // this group's half of the chunk does not exist
+                ok = mbar_wait_all(bar_sdp(hcol), n_half & 1, cta_abort);
                 if (!ok) break;
+                ++n_half;
                 tc_fence_after();
                 const uint32_t t_s = tmem_base + lane_addr + kColS, t_dp = tmem_base + lane_addr + kColDP;
                 const int col_end = min(ncols, 64 * hcol + 64);
@@ -487,7 +525,7 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                 }
                 tmem_st_wait();
                 tc_fence_before();
-                mbar_arrive(bar_ds);
+                mbar_arrive(bar_ds(hcol));
             }
             if (!ok) break;
             // ---- read-out: dV rows by warps 0-3, dK rows by warps 4-7

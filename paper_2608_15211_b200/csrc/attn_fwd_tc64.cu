@@ -414,15 +414,18 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             tc_fence_after();
             const uint32_t qb = smem0 + qs * kQStageBytes;
             // S = Q_t K_c^T into tile t's columns
+            // (descriptor low words = start address in 16-byte units: + 2 per 32-byte K step, + half / 16 for the hi half)
+            const uint32_t sd_hi = sdesc_hi(make_sdesc_sw64(smem0, 512));
+            const uint32_t q_lo0 = sdesc_lo(make_sdesc_sw64(qb, 512));
             auto issue_qk = [&](int t, uint32_t sb, int ncols) {
                 const uint32_t idesc = make_idesc_bf16(128, ncols, 0, 0);
+                const uint32_t q_lo = q_lo0 + ((t * 128 * kHalfBytes) >> 4), k_lo = sdesc_lo(make_sdesc_sw64(sb, 512));
+                const uint32_t t_d = tmem_base + t * 256;
                 if (elect_one()) {
-#pragma unroll
-                    for (int ks = 0; ks < 4; ++ks) {
-                        const uint32_t qa = qb + (ks >> 1) * kQHalf + t * 128 * kHalfBytes + (ks & 1) * 32;
-                        const uint32_t ka = sb + (ks >> 1) * kKHalf + (ks & 1) * 32;
-                        mma_ss(tmem_base + t * 256, make_sdesc_sw64(qa, 512), make_sdesc_sw64(ka, 512), idesc, ks > 0 ? 1u : 0u);
-                    }
+                    mma_ss_h<false>(t_d, q_lo, k_lo, sd_hi, idesc);
+                    mma_ss_h<true>(t_d, q_lo + 2, k_lo + 2, sd_hi, idesc);
+                    mma_ss_h<true>(t_d, q_lo + (kQHalf >> 4), k_lo + (kKHalf >> 4), sd_hi, idesc);
+                    mma_ss_h<true>(t_d, q_lo + (kQHalf >> 4) + 2, k_lo + (kKHalf >> 4) + 2, sd_hi, idesc);
                     mma_commit(bar_sready(t));
                 }
                 __syncwarp();
