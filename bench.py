@@ -422,13 +422,13 @@ def main():
         sm_count = torch.cuda.get_device_properties(local_rank).multi_processor_count
         # Algorithmic FLOP per launch of each kernel (strict convention, per allowed pair per head):
         # forward 4d (QK^T, PV); one-pass backward 8d (dP, dV, dK, dQ; the recomputed S is not counted); the
-        # register-tile backward kernels 4d each (key tiles: dV, dK; query tiles: dP, dQ).
+        # two-kernel backward paths 4d each (key side: dV, dK; query side: dP, dQ).
         pairs = wk["score_elements"]
         d = cfg.head_dim
         kernel_flop = {"swin_fwd_tc_kernel": 4 * d * pairs, "swin_fwd_tc64_kernel": 4 * d * pairs, "swin_fwd_mma_kernel": 4 * d * pairs,
                        "swin_bwd_fused_kernel": 8 * d * pairs,
                        "swin_bwd_mma_kernel<key tiles>": 4 * d * pairs, "swin_bwd_mma_kernel<query tiles>": 4 * d * pairs,
-                       "swin_bwd_kv64_kernel": 4 * d * pairs,
+                       "swin_bwd_kv64_kernel": 4 * d * pairs, "swin_bwd_q64_kernel": 4 * d * pairs,
                        "swin_bwd_delta_kernel": 0}
         kernels = []
         for kname, vals in kernel_ms.items():

@@ -239,12 +239,16 @@ static int bwd_call(const Geo& g, const void* q, const void* k, const void* v,
     cudaError_t e = launch_bwd_delta(g, o, d_o, delta, st);
     if (e != cudaSuccess) return cuda_fail(e, "terra_swin_attn_bwd (delta)");
     if (use_bwd_kv64(g)) {
-        // key side (dK, dV) on tcgen05, query side (dQ, dBias) on the register-tile kernel
+        // key side (dK, dV) on tcgen05
         float* prep = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(workspace) +
                                                align_up(sizeof(float) * (size_t)g.B * g.H * g.W * g.heads, 256));
         e = launch_bias_prep64(g, bias_table, prep, st);
         if (e == cudaSuccess) e = launch_bwd_kv64(g, q, k, v, d_o, prep, lse, delta, dk, dv, sms, st);
-        if (e == cudaSuccess) e = launch_bwd_mma(g, q, k, v, bias_table, lse, delta, d_o, dq, dk, dv, dbias, sms, st, true);
+        if (e == cudaSuccess) {
+            // query side (dQ, dBias): tcgen05 for complete 32 x 32 windows, else the register-tile kernel
+            if (bwd_q64_supported(g)) e = launch_bwd_q64(g, q, k, v, d_o, prep, lse, delta, dq, dbias, sms, st);
+            else e = launch_bwd_mma(g, q, k, v, bias_table, lse, delta, d_o, dq, dk, dv, dbias, sms, st, true);
+        }
         return e == cudaSuccess ? TERRA_OK : cuda_fail(e, "terra_swin_attn_bwd");
     }
     e = launch_bwd_mma(g, q, k, v, bias_table, lse, delta, d_o, dq, dk, dv, dbias, sms, st);
@@ -298,7 +302,10 @@ int terra_swin_check(void* stream) {
     int timed_out_kv = 0;
     e = read_bwd_kv64_status(&timed_out_kv);
     if (e != cudaSuccess) return cuda_fail(e, "terra_swin_check");
-    return (timed_out || timed_out_bwd || timed_out_64 || timed_out_kv) ? TERRA_ERR_DEVICE_TIMEOUT : TERRA_OK;
+    int timed_out_q = 0;
+    e = read_bwd_q64_status(&timed_out_q);
+    if (e != cudaSuccess) return cuda_fail(e, "terra_swin_check");
+    return (timed_out || timed_out_bwd || timed_out_64 || timed_out_kv || timed_out_q) ? TERRA_ERR_DEVICE_TIMEOUT : TERRA_OK;
 }
 
 int terra_profile_enable(int on) {

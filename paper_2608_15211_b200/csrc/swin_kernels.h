@@ -43,6 +43,13 @@ cudaError_t launch_bwd_kv64(const Geo& g, const void* q, const void* k, const vo
                             const float* lse, const float* delta, void* dk, void* dv, int sm_count, cudaStream_t stream);
 cudaError_t read_bwd_kv64_status(int* timed_out);
 
+// tcgen05 query side (dQ, dBias) of the same regime for complete 32 x 32 windows (window side 32, grid extents
+// multiples of 32); dbias is overwritten
+bool bwd_q64_supported(const Geo& g);
+cudaError_t launch_bwd_q64(const Geo& g, const void* q, const void* k, const void* v, const void* d_o, const float* prep,
+                           const float* lse, const float* delta, void* dq, float* dbias, int sm_count, cudaStream_t stream);
+cudaError_t read_bwd_q64_status(int* timed_out);
+
 cudaError_t launch_bounded_wait_selftest(long long limit_cycles, cudaStream_t stream);
 cudaError_t launch_bias_prep(const Geo& g, const float* bias, float* prep, cudaStream_t stream);
 
