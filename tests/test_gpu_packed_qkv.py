@@ -16,6 +16,7 @@ CASES = [
     small_config("packed_w8", 2, 24, 40, 3, 32, 8, 4, 4, 0, 0),        # tcgen05 kernels, several items per CTA
     small_config("packed_w14", 1, 45, 50, 2, 32, 14, 7, 7, 0, 1),      # generic table addressing
     small_config("packed_d64", 1, 45, 50, 2, 64, 20, 10, 10, 0, 1),    # register-tile kernels
+    small_config("packed_d64_w32", 1, 64, 64, 2, 64, 32, 16, 16, 0, 1),  # chunked tcgen05 kernels, complete windows
     small_config("packed_noshift", 1, 32, 32, 2, 32, 16, 0, 0, 0, 1),  # the unshifted W-MSA sibling of the block
 ]
 

@@ -1,6 +1,6 @@
 """Seeded random small shapes through the C ABI against the oracle: window sides 1..16 at head dim 32 (the
 tcgen05 kernels: every tile / block / mask / truncation combination the shapes happen to hit), larger
-windows or head dim 64 (the register-tile kernels), and grids with hundreds to thousands of (window, head) items
+windows or head dim 64 (the chunked tcgen05 kernels and the register-tile kernels), and grids with hundreds to thousands of (window, head) items
 (several items per CTA in mixed order of one-tile and two-tile windows)."""
 import random
 
@@ -46,6 +46,13 @@ def _shapes():
             ("d64_w17", 2, 40, 50, 3, 64, 17, 8, 9, 1, 0),               # 289 tokens: 3 tiles, ragged chunks
             ("d64_w8_many", 2, 64, 96, 5, 64, 8, 4, 4, 0, 1),            # one-tile windows, 960 items
             ("d64_w32_narrow", 1, 70, 45, 2, 64, 32, 20, 30, 0, 0)]      # 13-wide last column, 6-high last row
+    # complete 32 x 32 windows at head dim 64: the tcgen05 query side of the backward pass (dQ, dBias).  One item per
+    # CTA; both masks and two samples; CTAs whose item range crosses a query-tile boundary (their bias-gradient tables
+    # are flushed in mid-run); one or two items per CTA with 29 CTAs per head
+    out += [("d64_w32_one_window", 1, 32, 32, 1, 64, 32, 0, 0, 1, 1),
+            ("d64_w32_masks_b2", 2, 64, 96, 3, 64, 32, 5, 9, 0, 0),
+            ("d64_w32_heads12", 1, 96, 160, 12, 64, 32, 16, 16, 0, 1),
+            ("d64_w32_heads5", 1, 64, 64, 5, 64, 32, 40, 3, 0, 1)]
     return out
 
 
