@@ -20,7 +20,12 @@
 // Roles: warps 0-7 elementwise (warps w and w + 4 share lane quarter w & 3 and take the chunk's first / second 64 key
 // columns), warp 8 issues every MMA, warps 9-11 gather rows with cp.async.  Head dim 64 is kept as two 32-column
 // halves in the 64-byte-swizzled operand layout (lo | hi regions).
-// TMEM columns: S 0..127, dP 128..255, dQ 256..319.
+// A chunk's two 64-key halves are separate units of work ("half chunks", 16 per item, numbered through the whole
+// run); half chunk n belongs to elementwise warps 4 (n % 2) .. 4 (n % 2) + 3 and lives in TMEM buffer n % 3 (S in the
+// buffer's first 64 columns, dP in the second).  With three buffers for two groups of warps the scores of a group's
+// next half chunk are issued while it still works on the current one (as soon as the other group's previous half
+// chunk has been consumed), so the MMA round trip is hidden behind the elementwise work.
+// TMEM columns: buffers 0..127, 128..255, 256..383; dQ 384..447.
 // Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, all roles leave their loops, TMEM is
 // released and the host reads the device status word.  Every role follows every ring item by item.
 #include "swin_common.cuh"
@@ -40,6 +45,7 @@ constexpr int kLoaderWarp0 = 9;
 constexpr int kLoaderThreads = 96;
 constexpr int kThreads = 384;
 constexpr int kWorkThreads = 256;
+// every SM sub-partition holds two elementwise warps and one of warps 8-11: 2 * 192 + 112 <= 512 registers per lane
 constexpr int kRegsLaunch = 168, kRegsWork = 192, kRegsOther = 112;
 static_assert(2 * (kRegsWork - kRegsLaunch) <= (kRegsLaunch - kRegsOther), "register hand-over does not balance");
 
@@ -50,7 +56,7 @@ constexpr int kTile = 128;                            // queries per item, keys 
 constexpr int kHalf = kTile * kHalfBytes;             // 8192: one 32-column half of 128 rows
 constexpr int kTiles = kW * kW / kTile;               // 8 query tiles = 8 key chunks per window
 constexpr int kQStages = 2, kSlots = 3;
-// query stage: Q lo | Q hi | dO lo | dO hi, then per query row: 4 * bias code, label, token, lse * log2(e), delta
+// query stage: Q lo | Q hi | dO lo | dO hi, then per query row: 4 * bias code, label, token, lse, delta
 constexpr int kOffQlo = 0, kOffGlo = 2 * kHalf;     // hi halves follow at + kHalf
 constexpr int kRows = 4 * kHalf;                      // 32768
 constexpr int kOffQCode = kRows, kOffQLab = kRows + 512, kOffQTok = kRows + 1024, kOffQLse = kRows + 1536, kOffQDelta = kRows + 2048;
@@ -69,7 +75,8 @@ constexpr int kOffBars = ((kOffTab + 4 * kTabFloats * 4 + 1023) / 1024) * 1024;
 constexpr int kSmemBytes = kOffBars + 1024;
 static_assert(kQStageBytes % 1024 == 0 && kSlotBytes % 1024 == 0, "tiles keep the swizzle alignment");
 static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
-constexpr int kColS = 0, kColDP = 128, kColDQ = 256;
+constexpr int kBufCols = 128, kColDQ = 384;           // buffer b: S at 128 b, dP at 128 b + 64
+constexpr int kHalfChunks = 2 * kTiles;               // per item
 
 constexpr int kCodeStride = kW + 32;
 constexpr int kC0 = (kW - 1) * (kCodeStride + 1);
@@ -120,6 +127,9 @@ __device__ __forceinline__ int slot_token(const Geo& g, const Cursor& c, int slo
     return u * g.W + v;
 }
 
+__device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" ::"r"(dst), "l"(src));
+}
 __device__ __forceinline__ float lds_f32(uint32_t addr) {
     float v;
     asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(v) : "r"(addr) : "memory");
@@ -188,16 +198,15 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
     const uint32_t bar0 = smem0 + kOffBars;
     auto bar_qfull = [&](int s) { return bar0 + 8u * s; };               // the tile's Q, dO rows and row tables are there
     auto bar_qempty = [&](int s) { return bar0 + 8u * (2 + s); };        // ... and no longer needed
-    auto bar_kfull = [&](int s) { return bar0 + 8u * (4 + s); };         // a key chunk is in ring slot s
-    auto bar_kempty = [&](int s) { return bar0 + 8u * (7 + s); };        // ... and every MMA that reads it is complete
-    // a chunk's two 64-key halves are separate buffers (columns 64 h of S and dP) with their own hand-overs: half h
-    // belongs to elementwise warps 4 h .. 4 h + 3, and the MMAs of one half run while the other is worked on
-    auto bar_sdp = [&](int h) { return bar0 + 8u * (10 + h); };          // S and dP of a half chunk are in TMEM
-    auto bar_ds = [&](int h) { return bar0 + 8u * (12 + h); };           // bf16 dS of the half chunk is in TMEM
-    const uint32_t bar_acc = bar0 + 8u * 14;                              // dQ of the item is final
-    const uint32_t bar_accfree = bar0 + 8u * 15;                          // ... and has been read
-    const uint32_t bar_flush = bar0 + 8u * 16;                            // the elementwise warps meet around a table flush
-    unsigned char* tail = smem + kOffBars + 8 * 17;
+    // the ring is handed over in half slots: half chunk number p sits in rows 64 (p % 2) .. of slot (p / 2) % 3
+    auto bar_kfull = [&](int hs) { return bar0 + 8u * (4 + hs); };       // half slot hs = p % 6 holds its 64 keys
+    auto bar_kempty = [&](int hs) { return bar0 + 8u * (10 + hs); };     // ... and every MMA that reads them is complete
+    auto bar_sdp = [&](int b) { return bar0 + 8u * (16 + b); };          // S and dP of a half chunk are in TMEM buffer b
+    auto bar_ds = [&](int b) { return bar0 + 8u * (19 + b); };           // bf16 dS of the half chunk is in TMEM buffer b
+    const uint32_t bar_acc = bar0 + 8u * 22;                              // dQ of the item is final
+    const uint32_t bar_accfree = bar0 + 8u * 23;                          // ... and has been read
+    const uint32_t bar_flush = bar0 + 8u * 24;                            // the elementwise warps meet around a table flush
+    unsigned char* tail = smem + kOffBars + 8 * 25;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail);
     volatile int* cta_abort = reinterpret_cast<volatile int*>(tail + 8);
 
@@ -213,13 +222,13 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
             mbar_init(bar_qfull(s), kLoaderThreads);
             mbar_init(bar_qempty(s), 1 + kWorkThreads);    // the issuer's commit + every elementwise thread
         }
-        for (int s = 0; s < kSlots; ++s) {
-            mbar_init(bar_kfull(s), kLoaderThreads);
-            mbar_init(bar_kempty(s), 1);
+        for (int hs = 0; hs < 2 * kSlots; ++hs) {
+            mbar_init(bar_kfull(hs), kLoaderThreads);
+            mbar_init(bar_kempty(hs), 1);
         }
-        for (int h = 0; h < 2; ++h) {
-            mbar_init(bar_sdp(h), 1);
-            mbar_init(bar_ds(h), kWorkThreads / 2);
+        for (int b = 0; b < 3; ++b) {
+            mbar_init(bar_sdp(b), 1);
+            mbar_init(bar_ds(b), kWorkThreads / 2);
         }
         mbar_init(bar_acc, 1);
         mbar_init(bar_accfree, kWorkThreads);
@@ -246,25 +255,28 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kRegsOther));
     if (warp >= kLoaderWarp0) {
         // ------------------------------------------------------------------ loaders
-        // Two lanes per row (lane parity = the row's lo / hi half, four 16-byte copies each).  A group of copies is
-        // published when the next one has been issued; if a ring has no free place the pending group is published first.
         const int lt = (warp - kLoaderWarp0) * 32 + lane;
-        const int hf = lt & 1;
-        const int lrow = lt >> 1;
-        constexpr int kRowsPerIter = kLoaderThreads / 2;      // 48
+        // Eight lanes per row, one 16-byte piece of the row's 128 bytes each (pieces 0-3: the lo half, 4-7: the hi
+        // half), twelve rows per step: a warp's copy instruction reads four whole rows.
+        const int piece = lt & 7, rsub = lt >> 3;
+        constexpr int kRowsPerStep = kLoaderThreads / 8;      // 12
+        const uint32_t piece_off = (uint32_t)(piece >> 2) * kHalf;
         int quse = 0;
-        long long ru = 0;
-        uint32_t pending_bar = 0;
+        long long ru = 0;                                 // half chunks so far
+        uint32_t pending_bar = 0;                         // barrier of the group in flight
         bool ok = true;
+        auto publish = [&]() {
+            cp_async_wait<0>();
+            fence_proxy_async();
+            mbar_arrive(pending_bar);
+            pending_bar = 0;
+        };
+        // no free place yet: the group in flight is published first
         auto acquire = [&](uint32_t bar, uint32_t parity) -> bool {
-            if (pending_bar && !__all_sync(0xffffffffu, mbar_test_wait(bar, parity))) {
-                cp_async_wait<0>();
-                fence_proxy_async();
-                mbar_arrive(pending_bar);
-                pending_bar = 0;
-            }
+            if (pending_bar && !__all_sync(0xffffffffu, mbar_test_wait(bar, parity))) publish();
             return mbar_wait_all(bar, parity, cta_abort);
         };
+        // a group is published when the next one has been issued
         auto issued = [&](uint32_t bar) {
             cp_async_commit();
             if (pending_bar) {
@@ -283,72 +295,65 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
             // ---- the query tile: Q, dO rows and the row tables
             {
                 unsigned char* st = smem + qs * kQStageBytes;
-                const uint32_t sb = smem0 + qs * kQStageBytes + hf * kHalf;
+                const uint32_t sb = smem0 + qs * kQStageBytes + piece_off;
                 const int slot0 = cur.qt * kTile;
-                for (int row = lt; row < kTile; row += kLoaderThreads) {
-                    int code, label;
-                    const int tok = slot_token(g, cur, slot0 + row, code, label);
-                    const size_t li = (sample_off + (size_t)tok) * g.heads + head;
-                    reinterpret_cast<int*>(st + kOffQCode)[row] = 4 * code;
-                    reinterpret_cast<int*>(st + kOffQLab)[row] = label;
-                    reinterpret_cast<int*>(st + kOffQTok)[row] = tok;
-                    reinterpret_cast<float*>(st + kOffQLse)[row] = __ldg(lse + li) * kLog2e;
-                    reinterpret_cast<float*>(st + kOffQDelta)[row] = __ldg(delta + li);
-                }
-                for (int row = lrow; row < kTile; row += kRowsPerIter) {
-                    int code, label;
-                    const int tok = slot_token(g, cur, slot0 + row, code, label);
-                    const __nv_bfloat16* sq = q + (sample_off + (size_t)tok) * g.ts + head * kD + hf * 32;
-                    const __nv_bfloat16* sg = d_o + ((sample_off + (size_t)tok) * g.heads + head) * kD + hf * 32;
-#pragma unroll
-                    for (int c4 = 0; c4 < 4; ++c4) {
-                        const uint32_t so = tile_off<32>(row, c4);
-                        cp_async16(sb + kOffQlo + so, sq + c4 * 8, 16);
-                        cp_async16(sb + kOffGlo + so, sg + c4 * 8, 16);
+#pragma unroll 1
+                for (int step = 0; step < (kTile + kRowsPerStep - 1) / kRowsPerStep; ++step) {
+                    const int row = rsub + kRowsPerStep * step;
+                    if (row < kTile) {
+                        int code, label;
+                        const int tok = slot_token(g, cur, slot0 + row, code, label);
+                        const size_t li = (sample_off + (size_t)tok) * g.heads + head;
+                        if (piece == 0) {
+                            reinterpret_cast<int*>(st + kOffQCode)[row] = 4 * code;
+                            reinterpret_cast<int*>(st + kOffQLab)[row] = label;
+                            reinterpret_cast<int*>(st + kOffQTok)[row] = tok;
+                            // lse and delta travel with the rows (no load the loader would have to wait for)
+                            cp_async4(smem0 + qs * kQStageBytes + kOffQLse + 4 * row, lse + li);
+                            cp_async4(smem0 + qs * kQStageBytes + kOffQDelta + 4 * row, delta + li);
+                        }
+                        const uint32_t so = tile_off<32>(row, piece & 3);
+                        cp_async16(sb + kOffQlo + so, q + (sample_off + (size_t)tok) * g.ts + head * kD + piece * 8, 16);
+                        cp_async16(sb + kOffGlo + so, d_o + li * kD + piece * 8, 16);
                     }
                 }
                 issued(bar_qfull(qs));
             }
-            // ---- the window's keys, chunk by chunk
-            for (int c = 0; c < kTiles; ++c, ++ru) {
-                const int s = (int)(ru % kSlots);
-                ok = acquire(bar_kempty(s), (uint32_t)((ru / kSlots) & 1) ^ 1u);
+            // ---- the window's keys, half chunk by half chunk
+            for (int n = 0; n < kHalfChunks; ++n, ++ru) {
+                const int hs = (int)(ru % (2 * kSlots));
+                ok = acquire(bar_kempty(hs), (uint32_t)((ru / (2 * kSlots)) & 1) ^ 1u);
                 if (!ok) break;
-                unsigned char* sl = smem + kOffSlots + s * kSlotBytes;
-                const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes + hf * kHalf;
-                for (int row = lt; row < kTile; row += kLoaderThreads) {
-                    int code, label;
-                    slot_token(g, cur, chunk_slot(c, row), code, label);
-                    reinterpret_cast<int*>(sl + kOffKCode)[row] = 4 * (kC0 - code);
-                    reinterpret_cast<int*>(sl + kOffKLab)[row] = label;
-                }
-                for (int row = lrow; row < kTile; row += kRowsPerIter) {
-                    int code, label;
-                    const int tok = slot_token(g, cur, chunk_slot(c, row), code, label);
-                    const size_t off = (sample_off + (size_t)tok) * g.ts + head * kD + hf * 32;
+                unsigned char* sl = smem + kOffSlots + (hs >> 1) * kSlotBytes;
+                const uint32_t sb = smem0 + kOffSlots + (hs >> 1) * kSlotBytes + piece_off;
+                const int c = n >> 1, row0 = 64 * (n & 1);
 #pragma unroll
-                    for (int c4 = 0; c4 < 4; ++c4) {
-                        const uint32_t so = tile_off<32>(row, c4);
-                        cp_async16(sb + kOffKlo + so, k + off + c4 * 8, 16);
-                        cp_async16(sb + kOffVlo + so, v + off + c4 * 8, 16);
+                for (int step = 0; step < (64 + kRowsPerStep - 1) / kRowsPerStep; ++step) {
+                    const int r = rsub + kRowsPerStep * step;
+                    if (r < 64) {
+                        const int row = row0 + r;
+                        int code, label;
+                        const int tok = slot_token(g, cur, chunk_slot(c, row), code, label);
+                        if (piece == 0) {
+                            reinterpret_cast<int*>(sl + kOffKCode)[row] = 4 * (kC0 - code);
+                            reinterpret_cast<int*>(sl + kOffKLab)[row] = label;
+                        }
+                        const size_t off = (sample_off + (size_t)tok) * g.ts + head * kD + piece * 8;
+                        const uint32_t so = tile_off<32>(row, piece & 3);
+                        cp_async16(sb + kOffKlo + so, k + off, 16);
+                        cp_async16(sb + kOffVlo + so, v + off, 16);
                     }
                 }
-                issued(bar_kfull(s));
+                issued(bar_kfull(hs));
             }
         }
-        if (pending_bar) {
-            cp_async_wait<0>();
-            fence_proxy_async();
-            mbar_arrive(pending_bar);
-        }
+        if (pending_bar) publish();
     } else {
         // ------------------------------------------------------------------ MMA issuer
         const uint32_t idesc_s = make_idesc_bf16(128, 64, 0, 0);
         const uint32_t idesc_acc = make_idesc_bf16(128, kD, 0, 1);       // A from TMEM, B = 16 rows x 64 (MN-major)
         const uint32_t sd_hi = sdesc_hi(make_sdesc_sw64(smem0, 512));    // common high word of the K-major descriptors
         int quse = 0;
-        int n_ds[2] = {0, 0};
-        long long ru = 0;
         bool ok = true;
         for (long long it = it_lo; ok && it < it_hi; ++it, ++quse) {
             const int qs = quse % kQStages;
@@ -356,18 +361,22 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
             if (!ok) break;
             fence_proxy_async();
             const uint32_t qb = smem0 + qs * kQStageBytes;
-            auto chunk_ready = [&](long long use) -> bool {
-                if (!mbar_wait_all(bar_kfull((int)(use % kSlots)), (uint32_t)((use / kSlots) & 1), cta_abort)) return false;
+            const long long n0 = (long long)quse * kHalfChunks;   // number of the item's half chunk 0
+            auto half_ready = [&](int n) -> bool {        // the keys of the item's half chunk n are in their half slot
+                const long long p = n0 + n;
+                if (!mbar_wait_all(bar_kfull((int)(p % (2 * kSlots))), (uint32_t)((p / (2 * kSlots)) & 1), cta_abort)) return false;
                 fence_proxy_async();
                 return true;
             };
-            // S = Q K^T, dP = dO V^T for the 64 keys of half h of the chunk in ring slot `sb`
+            // S = Q K^T, dP = dO V^T for half chunk n of the item (chunk n / 2, keys 64 (n % 2) ..), into its buffer
             // (descriptor low words = start address in 16-byte units: + 2 per 32-byte K step, + kHalf / 16 for the hi half)
             const uint32_t q_lo = sdesc_lo(make_sdesc_sw64(qb + kOffQlo, 512)), g_lo = sdesc_lo(make_sdesc_sw64(qb + kOffGlo, 512));
-            auto issue_sdp = [&](int h, uint32_t sb) {
-                const uint32_t k_lo = sdesc_lo(make_sdesc_sw64(sb + kOffKlo + h * 64 * kHalfBytes, 512));
-                const uint32_t v_lo = sdesc_lo(make_sdesc_sw64(sb + kOffVlo + h * 64 * kHalfBytes, 512));
-                const uint32_t t_s = tmem_base + kColS + 64 * h, t_dp = tmem_base + kColDP + 64 * h;
+            auto issue_sdp = [&](int n) {
+                const uint32_t sb = smem0 + kOffSlots + (int)(((n0 + n) >> 1) % kSlots) * kSlotBytes + (n & 1) * 64 * kHalfBytes;
+                const int buf = (int)((n0 + n) % 3);
+                const uint32_t k_lo = sdesc_lo(make_sdesc_sw64(sb + kOffKlo, 512));
+                const uint32_t v_lo = sdesc_lo(make_sdesc_sw64(sb + kOffVlo, 512));
+                const uint32_t t_s = tmem_base + kBufCols * buf, t_dp = t_s + 64;
                 constexpr uint32_t kHi = kHalf >> 4;
                 tc_fence_after();
                 if (elect_one()) {
@@ -379,54 +388,49 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
                     mma_ss_h<true>(t_dp, g_lo + 2, v_lo + 2, sd_hi, idesc_s);
                     mma_ss_h<true>(t_dp, g_lo + kHi, v_lo + kHi, sd_hi, idesc_s);
                     mma_ss_h<true>(t_dp, g_lo + kHi + 2, v_lo + kHi + 2, sd_hi, idesc_s);
-                    mma_commit(bar_sdp(h));
+                    mma_commit(bar_sdp(buf));
                 }
                 __syncwarp();
             };
-            ok = chunk_ready(ru);
+            // the item's first three half chunks (every buffer is free: the previous item's were all consumed)
+            for (int n = 0; n < 3 && ok; ++n) {
+                ok = half_ready(n);
+                if (ok) issue_sdp(n);
+            }
             if (!ok) break;
-            for (int h = 0; h < 2; ++h) issue_sdp(h, smem0 + kOffSlots + (int)(ru % kSlots) * kSlotBytes);
-            for (int c = 0; c < kTiles && ok; ++c, ++ru) {
-                const int s = (int)(ru % kSlots);
-                const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes;
-                const bool has_next = c + 1 < kTiles;
-                if (has_next) {
-                    ok = chunk_ready(ru + 1);
-                    if (!ok) break;
-                }
-                const uint32_t sb_n = smem0 + kOffSlots + (int)((ru + 1) % kSlots) * kSlotBytes;
-                for (int h = 0; h < 2 && ok; ++h) {
-                    ok = mbar_wait_all(bar_ds(h), n_ds[h] & 1, cta_abort);
-                    ++n_ds[h];
-                    if (ok && c == 0 && h == 0 && quse > 0) ok = mbar_wait_all(bar_accfree, (quse - 1) & 1, cta_abort);
-                    if (!ok) break;
-                    tc_fence_after();
-                    // dQ += dS K over the half chunk's key columns
-                    const uint64_t kd = make_sdesc_sw64_mn(sb + kOffKlo + h * 64 * kHalfBytes, kHalf, 512);
-                    const uint32_t k_lo = sdesc_lo(kd), d_hi = sdesc_hi(kd);
-                    const uint32_t t_ds = tmem_base + kColDP + 64 * h;
-                    if (elect_one()) {
-                        int j = 0;
-                        if (c == 0 && h == 0) {
-                            mma_ts_h<false>(tmem_base + kColDQ, t_ds, k_lo, d_hi, idesc_acc);
-                            j = 1;
-                        }
-                        for (; j < 4; ++j) mma_ts_h<true>(tmem_base + kColDQ, t_ds + 16 * j, k_lo + 64 * j, d_hi, idesc_acc);
-                    }
-                    __syncwarp();
-                    // the half's buffers are free again (the product that reads them was issued just above): the next
-                    // chunk's scores for this half follow at once, while the other half is being worked on
-                    if (has_next) issue_sdp(h, sb_n);
-                }
+            for (int n = 0; n < kHalfChunks && ok; ++n) {
+                const long long ng = n0 + n;
+                const int buf = (int)(ng % 3);
+                ok = mbar_wait_all(bar_ds(buf), (uint32_t)((ng / 3) & 1), cta_abort);
+                if (ok && n == 0 && quse > 0) ok = mbar_wait_all(bar_accfree, (quse - 1) & 1, cta_abort);
                 if (!ok) break;
+                tc_fence_after();
+                // dQ += dS K over the half chunk's key columns
+                const uint32_t sb = smem0 + kOffSlots + (int)((ng >> 1) % kSlots) * kSlotBytes + (n & 1) * 64 * kHalfBytes;
+                const uint64_t kd = make_sdesc_sw64_mn(sb + kOffKlo, kHalf, 512);
+                const uint32_t k_lo = sdesc_lo(kd), d_hi = sdesc_hi(kd);
+                const uint32_t t_ds = tmem_base + kBufCols * buf + 64;
                 if (elect_one()) {
-                    mma_commit(bar_kempty(s));
-                    if (!has_next) {
+                    int j = 0;
+                    if (n == 0) {
+                        mma_ts_h<false>(tmem_base + kColDQ, t_ds, k_lo, d_hi, idesc_acc);
+                        j = 1;
+                    }
+                    for (; j < 4; ++j) mma_ts_h<true>(tmem_base + kColDQ, t_ds + 16 * j, k_lo + 64 * j, d_hi, idesc_acc);
+                    mma_commit(bar_kempty((int)(ng % (2 * kSlots))));   // the half slot's last reader: it goes back at once
+                    if (n + 1 == kHalfChunks) {
                         mma_commit(bar_acc);
                         mma_commit(bar_qempty(qs));
                     }
                 }
                 __syncwarp();
+                // the buffer is free again (the product that reads it was issued just above): the scores of the half
+                // chunk three further on follow at once
+                if (n + 3 < kHalfChunks) {
+                    ok = half_ready(n + 3);
+                    if (!ok) break;
+                    issue_sdp(n + 3);
+                }
             }
         }
     }
@@ -442,7 +446,7 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
         const uint32_t tab0 = smem0 + kOffTab;
         // this lane's entry for key (a_k = 16 hcol, b_k = 0): [a_k][lane + 31]; b_k lies b_k floats below, a_k rows above
         const uint32_t tab_lane = tab0 + 4 * (quarter * kTabFloats + 16 * hcol * 64 + lane + 31);
-        int quse = 0, n_half = 0, n_flush = 0;
+        int quse = 0, n_flush = 0;
         int tab_qt = -1;                                  // the tile whose gradients the tables hold
         long long ru = 0;
         bool ok = true;
@@ -480,19 +484,21 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
             const int qcode4 = lds_i32(st_a + kOffQCode + 4 * qrow);
             const int qlabel = lds_i32(st_a + kOffQLab + 4 * qrow);
             const int qtok = lds_i32(st_a + kOffQTok + 4 * qrow);
-            const float l2 = lds_f32(st_a + kOffQLse + 4 * qrow);
+            const float l2 = lds_f32(st_a + kOffQLse + 4 * qrow) * kLog2e;
             const float dl = lds_f32(st_a + kOffQDelta + 4 * qrow);
             mbar_arrive(bar_qempty(qs));                  // this thread has what it needs from the query stage
             // bias index = code_query - code_key + c0
             const uint32_t bias_row = smem0 + kOffBias + qcode4;
             for (int c = 0; c < kTiles && ok; ++c, ++ru) {
-                const int s = (int)(ru % kSlots);
+                const int s = (int)(ru % kSlots);         // the chunk's slot: half chunk p is in slot (p / 2) % 3
                 const uint32_t sl_a = smem0 + kOffSlots + s * kSlotBytes;
-                ok = mbar_wait_all(bar_sdp(hcol), n_half & 1, cta_abort);
+                const long long ng = (long long)quse * kHalfChunks + 2 * c + hcol;   // this group's half chunk
+                const int buf = (int)(ng % 3);
+                ok = mbar_wait_all(bar_sdp(buf), (uint32_t)((ng / 3) & 1), cta_abort);
                 if (!ok) break;
-                ++n_half;
                 tc_fence_after();
-                const uint32_t t_s = tmem_base + lane_addr + kColS, t_dp = tmem_base + lane_addr + kColDP;
+                // buffer columns of key column cc of the chunk: S at cc - 64 hcol, dP 64 further
+                const uint32_t t_s = tmem_base + lane_addr + kBufCols * buf - 64 * hcol, t_dp = t_s + 64;
                 // a 16-column group is key rows 16 hcol .. 16 hcol + 15 at b_k = 4 c + (column / 16) % 4
                 auto tab_of = [&](int col) { return tab_lane - 4 * (4 * c + ((col >> 4) & 3)); };
                 // groups of 16 columns; the next group's S / dP travel from TMEM while this one is worked on
@@ -519,7 +525,7 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
                 }
                 tmem_st_wait();
                 tc_fence_before();
-                mbar_arrive(bar_ds(hcol));
+                mbar_arrive(bar_ds(buf));
             }
             if (!ok) break;
             // ---- read-out: dQ columns 0..31 by warps 0-3, 32..63 by warps 4-7
