@@ -46,7 +46,7 @@ constexpr int kOffKlo = 0, kOffKhi = kHalf, kOffVlo = 2 * kHalf, kOffVhi = 3 * k
 constexpr int kKvRows = 4 * kHalf;                    // 32768
 constexpr int kOffKCode = kKvRows, kOffKLab = kKvRows + 512, kOffKTok = kKvRows + 1024;
 constexpr int kKvStageBytes = kKvRows + 2048;
-// query slot: Q lo | Q hi | dO lo | dO hi, then per query column: 4 * bias code, label, lse * log2(e), delta
+// query slot: Q lo | Q hi | dO lo | dO hi, then per query column: 4 * bias code, label, lse, delta
 constexpr int kOffQlo = 0, kOffQhi = kHalf, kOffGlo = 2 * kHalf, kOffGhi = 3 * kHalf;
 constexpr int kOffQCode = 4 * kHalf, kOffQLab = kOffQCode + 512, kOffQLse = kOffQCode + 1024, kOffQDelta = kOffQCode + 1536;
 constexpr int kSlotBytes = 4 * kHalf + 2048;          // 34816
@@ -95,6 +95,9 @@ __device__ __forceinline__ int offset_token(const Geo& g, const WindowRef& r, in
     return u * g.W + v;
 }
 
+__device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" ::"r"(dst), "l"(src));
+}
 __device__ __forceinline__ float lds_f32(uint32_t addr) {
     float v;
     asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(v) : "r"(addr));
@@ -149,7 +152,7 @@ __device__ __forceinline__ void cols16(const uint32_t (&rs)[16], const uint32_t 
     float p[16], ds[16];
 #pragma unroll
     for (int e = 0; e < 16; ++e) {
-        float xv = fmaf(__uint_as_float(rs[e]), scale, bv[e]) - l2[e];
+        float xv = fmaf(-l2[e], kLog2e, fmaf(__uint_as_float(rs[e]), scale, bv[e]));
         if (MASKED && ql[e] != klabel) xv = -INFINITY;
         p[e] = fast_exp2(xv);
         ds[e] = p[e] * (__uint_as_float(rp[e]) - dl[e]);
@@ -313,18 +316,19 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                 for (int row = lt; row < kTile; row += kLoaderThreads) {
                     const int slot = c * kTile + row;
                     int code = 0, label = 0xff;
-                    float l2 = INFINITY, dl = 0.f;              // no token: P = exp2(.. - inf) = 0
                     if (slot < x.r.n) {
+                        // lse and delta travel with the rows (no load the loader would have to wait for)
                         const int a = slot / ew;
                         const int tok = offset_token(g, x.r, a, slot - a * ew, code, label);
                         const size_t li = (sample_off + (size_t)tok) * g.heads + head;
-                        l2 = __ldg(lse + li) * kLog2e;
-                        dl = __ldg(delta + li);
+                        cp_async4(smem0 + kOffSlots + s * kSlotBytes + kOffQLse + 4 * row, lse + li);
+                        cp_async4(smem0 + kOffSlots + s * kSlotBytes + kOffQDelta + 4 * row, delta + li);
+                    } else {
+                        reinterpret_cast<float*>(sl + kOffQLse)[row] = INFINITY;   // no token: P = exp2(.. - inf) = 0
+                        reinterpret_cast<float*>(sl + kOffQDelta)[row] = 0.f;
                     }
                     reinterpret_cast<int*>(sl + kOffQCode)[row] = 4 * code;
                     reinterpret_cast<int*>(sl + kOffQLab)[row] = label;
-                    reinterpret_cast<float*>(sl + kOffQLse)[row] = l2;
-                    reinterpret_cast<float*>(sl + kOffQDelta)[row] = dl;
                 }
                 const int slot_first = c * kTile + lrow;
                 int a_r = slot_first / ew, b_r = slot_first - a_r * ew;
