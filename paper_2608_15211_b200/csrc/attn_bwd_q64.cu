@@ -61,9 +61,9 @@ constexpr int kOffQlo = 0, kOffGlo = 2 * kHalf;     // hi halves follow at + kHa
 constexpr int kRows = 4 * kHalf;                      // 32768
 constexpr int kOffQCode = kRows, kOffQLab = kRows + 512, kOffQTok = kRows + 1024, kOffQLse = kRows + 1536, kOffQDelta = kRows + 2048;
 constexpr int kQStageBytes = kRows + 3072;
-// key slot: K lo | K hi | V lo | V hi, then per key column: 4 * (c0 - bias code), label
+// key slot: K lo | K hi | V lo | V hi, then per key column: label
 constexpr int kOffKlo = 0, kOffVlo = 2 * kHalf;     // hi halves follow at + kHalf
-constexpr int kOffKCode = kRows, kOffKLab = kRows + 512;
+constexpr int kOffKLab = kRows;
 constexpr int kSlotBytes = kRows + 1024;
 constexpr int kOffSlots = kQStages * kQStageBytes;
 constexpr int kBiasFloats = 6048;
@@ -152,16 +152,13 @@ __device__ __forceinline__ int lds_i32(uint32_t addr) {
 // 16 key columns [c, c + 16) of one query row: P = exp2(S scale + bias - lse), dS = P (dP - delta); dS is packed to
 // bf16 for the dQ product and added, in fp32, to the row's 16 entries of the bias-gradient table (`tab` = address of
 // the entry of column c; the following columns are the following key rows, one table row further each).
+// `bias_grp` = address of the bias entry of column c: the group's columns are 16 consecutive key rows at one b_k, so
+// the following entries lie one code stride below each (no per-key table is read for them).
 template <bool MASKED>
-__device__ __forceinline__ void cols16(const uint32_t (&rs)[16], const uint32_t (&rp)[16], int c, uint32_t bias_row, int qlabel,
+__device__ __forceinline__ void cols16(const uint32_t (&rs)[16], const uint32_t (&rp)[16], int c, uint32_t bias_grp, int qlabel,
                                        float l2, float dl, uint32_t sl_a, float scale, uint32_t tab, uint32_t (&pk_ds)[8]) {
-    int co[16], kl[16];
+    int kl[16];
     float bv[16], tv[16];
-#pragma unroll
-    for (int e4 = 0; e4 < 4; ++e4) {
-        const int4 c4 = lds_i4(sl_a + kOffKCode + 4 * (c + e4 * 4));
-        co[e4 * 4] = c4.x; co[e4 * 4 + 1] = c4.y; co[e4 * 4 + 2] = c4.z; co[e4 * 4 + 3] = c4.w;
-    }
     if (MASKED) {
 #pragma unroll
         for (int e4 = 0; e4 < 4; ++e4) {
@@ -170,7 +167,7 @@ __device__ __forceinline__ void cols16(const uint32_t (&rs)[16], const uint32_t 
         }
     }
 #pragma unroll
-    for (int e = 0; e < 16; ++e) bv[e] = lds_f32(bias_row + co[e]);
+    for (int e = 0; e < 16; ++e) bv[e] = lds_f32(bias_grp - 4 * kCodeStride * e);
     float ds[16];
 #pragma unroll
     for (int e = 0; e < 16; ++e) {
@@ -334,10 +331,7 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
                         const int row = row0 + r;
                         int code, label;
                         const int tok = slot_token(g, cur, chunk_slot(c, row), code, label);
-                        if (piece == 0) {
-                            reinterpret_cast<int*>(sl + kOffKCode)[row] = 4 * (kC0 - code);
-                            reinterpret_cast<int*>(sl + kOffKLab)[row] = label;
-                        }
+                        if (piece == 0) reinterpret_cast<int*>(sl + kOffKLab)[row] = label;
                         const size_t off = (sample_off + (size_t)tok) * g.ts + head * kD + piece * 8;
                         const uint32_t so = tile_off<32>(row, piece & 3);
                         cp_async16(sb + kOffKlo + so, k + off, 16);
@@ -487,7 +481,6 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
             const float l2 = lds_f32(st_a + kOffQLse + 4 * qrow) * kLog2e;
             const float dl = lds_f32(st_a + kOffQDelta + 4 * qrow);
             mbar_arrive(bar_qempty(qs));                  // this thread has what it needs from the query stage
-            // bias index = code_query - code_key + c0
             const uint32_t bias_row = smem0 + kOffBias + qcode4;
             for (int c = 0; c < kTiles && ok; ++c, ++ru) {
                 const int s = (int)(ru % kSlots);         // the chunk's slot: half chunk p is in slot (p / 2) % 3
@@ -501,6 +494,8 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
                 const uint32_t t_s = tmem_base + lane_addr + kBufCols * buf - 64 * hcol, t_dp = t_s + 64;
                 // a 16-column group is key rows 16 hcol .. 16 hcol + 15 at b_k = 4 c + (column / 16) % 4
                 auto tab_of = [&](int col) { return tab_lane - 4 * (4 * c + ((col >> 4) & 3)); };
+                // bias index = code_query - code_key + c0 with code_key = (16 hcol + e) * stride + b_k
+                auto bias_of = [&](int col) { return bias_row + 4 * (kC0 - 16 * hcol * kCodeStride - 4 * c - ((col >> 4) & 3)); };
                 // groups of 16 columns; the next group's S / dP travel from TMEM while this one is worked on
                 uint32_t rs[16], rp[16], rs2[16], rp2[16], pk_ds[8];
                 const int col0 = 64 * hcol;
@@ -511,16 +506,16 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
                     tmem_ld_wait();
                     tmem_ld16(t_s + cc + 16, rs2);
                     tmem_ld16(t_dp + cc + 16, rp2);
-                    if (masked) cols16<true>(rs, rp, cc, bias_row, qlabel, l2, dl, sl_a, scale, tab_of(cc), pk_ds);
-                    else cols16<false>(rs, rp, cc, bias_row, qlabel, l2, dl, sl_a, scale, tab_of(cc), pk_ds);
+                    if (masked) cols16<true>(rs, rp, cc, bias_of(cc), qlabel, l2, dl, sl_a, scale, tab_of(cc), pk_ds);
+                    else cols16<false>(rs, rp, cc, bias_of(cc), qlabel, l2, dl, sl_a, scale, tab_of(cc), pk_ds);
                     tmem_st8(t_dp + cc, pk_ds);            // 16 keys -> 8 packed columns at the group's own place
                     tmem_ld_wait();
                     if (cc + 32 < col0 + 64) {
                         tmem_ld16(t_s + cc + 32, rs);
                         tmem_ld16(t_dp + cc + 32, rp);
                     }
-                    if (masked) cols16<true>(rs2, rp2, cc + 16, bias_row, qlabel, l2, dl, sl_a, scale, tab_of(cc + 16), pk_ds);
-                    else cols16<false>(rs2, rp2, cc + 16, bias_row, qlabel, l2, dl, sl_a, scale, tab_of(cc + 16), pk_ds);
+                    if (masked) cols16<true>(rs2, rp2, cc + 16, bias_of(cc + 16), qlabel, l2, dl, sl_a, scale, tab_of(cc + 16), pk_ds);
+                    else cols16<false>(rs2, rp2, cc + 16, bias_of(cc + 16), qlabel, l2, dl, sl_a, scale, tab_of(cc + 16), pk_ds);
                     tmem_st8(t_dp + cc + 16, pk_ds);
                 }
                 tmem_st_wait();
