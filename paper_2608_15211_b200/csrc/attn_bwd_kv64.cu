@@ -122,16 +122,20 @@ __device__ __forceinline__ int lds_i32(uint32_t addr) {
 // 16 query columns [c, c + 16) of one key row: P = exp2(S scale + bias - lse), dS = P (dP - delta), packed to bf16.
 // `bias_row` = shared address of the bias table + the key row's part of the index (the -inf zone if the row has no
 // token); a query column without a token has lse = +inf, so its P is 0.
-template <bool MASKED>
+// ROW32: the window is 32 tokens wide, so the group's 16 queries sit in one window row and their bias codes are
+// consecutive: `code4` = 4 * code of column c, no per-query code table is read.
+template <bool MASKED, bool ROW32 = false>
 __device__ __forceinline__ void cols16(const uint32_t (&rs)[16], const uint32_t (&rp)[16], int c, uint32_t bias_row, int klabel,
-                                       uint32_t sl_a, float scale, uint32_t (&pk_p)[8], uint32_t (&pk_ds)[8]) {
+                                       uint32_t sl_a, float scale, uint32_t (&pk_p)[8], uint32_t (&pk_ds)[8], int code4 = 0) {
     // all table loads first (they are issued in program order), then the gathers that depend on them, then the math
     int co[16], ql[16];
     float l2[16], dl[16], bv[16];
+    if (!ROW32) {
 #pragma unroll
-    for (int e4 = 0; e4 < 4; ++e4) {
-        const int4 c4 = lds_i4(sl_a + kOffQCode + 4 * (c + e4 * 4));
-        co[e4 * 4] = c4.x; co[e4 * 4 + 1] = c4.y; co[e4 * 4 + 2] = c4.z; co[e4 * 4 + 3] = c4.w;
+        for (int e4 = 0; e4 < 4; ++e4) {
+            const int4 c4 = lds_i4(sl_a + kOffQCode + 4 * (c + e4 * 4));
+            co[e4 * 4] = c4.x; co[e4 * 4 + 1] = c4.y; co[e4 * 4 + 2] = c4.z; co[e4 * 4 + 3] = c4.w;
+        }
     }
 #pragma unroll
     for (int e4 = 0; e4 < 4; ++e4) {
@@ -148,7 +152,7 @@ __device__ __forceinline__ void cols16(const uint32_t (&rs)[16], const uint32_t 
         }
     }
 #pragma unroll
-    for (int e = 0; e < 16; ++e) bv[e] = lds_f32(bias_row + co[e]);
+    for (int e = 0; e < 16; ++e) bv[e] = ROW32 ? lds_f32(bias_row + code4 + 4 * e) : lds_f32(bias_row + co[e]);
     float p[16], ds[16];
 #pragma unroll
     for (int e = 0; e < 16; ++e) {
@@ -488,6 +492,7 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             mbar_arrive(bar_kvempty(ks));                 // this thread has what it needs from the key stage
             // bias index = code_query - code_key + c0; a key row without a token reads the table's -inf zone
             const uint32_t bias_row = smem0 + kOffBias + (ktok >= 0 ? 4 * c0 - kcode4 : 4 * (2 * c0 + 1));
+            const bool row32 = x.r.ew == 32;
             for (int c = 0; c < x.nch && ok; ++c, ++ru) {
                 const int s = (int)(ru % kSlots);
                 const uint32_t sl_a = smem0 + kOffSlots + s * kSlotBytes;
@@ -499,6 +504,8 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                 tc_fence_after();
                 const uint32_t t_s = tmem_base + lane_addr + kColS, t_dp = tmem_base + lane_addr + kColDP;
                 const int col_end = min(ncols, 64 * hcol + 64);
+                // 4 * bias code of query column `col` of this chunk in a 32-wide window: slot = 128 c + col = 32 a + b
+                auto code4_of = [&](int col) { return 4 * ((4 * c + (col >> 5)) * cs + (col & 31)); };
                 // groups of 16 columns; the next group's S^T / dP^T travel from TMEM while this one is worked on
                 uint32_t rs[16], rp[16], rs2[16], rp2[16], pk_p[8], pk_ds[8];
                 if (64 * hcol < col_end) {
@@ -512,6 +519,7 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                         tmem_ld16(t_dp + cc + 16, rp2);
                     }
                     if (x.masked) cols16<true>(rs, rp, cc, bias_row, klabel, sl_a, scale, pk_p, pk_ds);
+                    else if (row32) cols16<false, true>(rs, rp, cc, bias_row, klabel, sl_a, scale, pk_p, pk_ds, code4_of(cc));
                     else cols16<false>(rs, rp, cc, bias_row, klabel, sl_a, scale, pk_p, pk_ds);
                     tmem_st8(t_s + cc, pk_p);              // 16 queries -> 8 packed columns at the group's own place
                     tmem_st8(t_dp + cc, pk_ds);
@@ -522,6 +530,7 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                             tmem_ld16(t_dp + cc + 32, rp);
                         }
                         if (x.masked) cols16<true>(rs2, rp2, cc + 16, bias_row, klabel, sl_a, scale, pk_p, pk_ds);
+                        else if (row32) cols16<false, true>(rs2, rp2, cc + 16, bias_row, klabel, sl_a, scale, pk_p, pk_ds, code4_of(cc + 16));
                         else cols16<false>(rs2, rp2, cc + 16, bias_row, klabel, sl_a, scale, pk_p, pk_ds);
                         tmem_st8(t_s + cc + 16, pk_p);
                         tmem_st8(t_dp + cc + 16, pk_ds);
