@@ -177,6 +177,7 @@ def run_reference(args, cfg):
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per (batch, window, head) item from the ncu
 # captures summarised under profiles/ (config 3 cut to 254 token rows, 13 056 items); traffic grows in
 # proportion to the item count, so a full launch is this figure times its items.  None = not captured.
+TRAFFIC_SOURCE = "stored ncu capture (profiles/swin_*_cfg3_rows254.md), scaled by the item count; not measured in this run"
 NCU_DRAM_BYTES_PER_ITEM = {
     "swin_fwd_tc_kernel": 63620,
     "swin_bwd_fused_kernel": 112255,
@@ -293,6 +294,7 @@ def main():
     for _ in range(max(3, args.warmup)):
         step()
     barrier()
+    terra.terra_swin_check()           # raises if any kernel of the warm-up gave up on a bounded wait
 
     wk = work(cfg)
     flops = wk["flop_fwd"] + wk["flop_bwd"]
@@ -315,6 +317,9 @@ def main():
         ev[i][3].record(stream)
     t_end.record(stream)
     barrier()
+    # a CTA whose bounded wait expired leaves its loops early and the launch still returns TERRA_OK: a timed
+    # region that saw that is not a measurement, so it ends the run with an error instead of a line
+    terra.terra_swin_check()
     launches = terra.launch_count() - launches0
     kernel_ms = {}
     for kname, kms in terra.profile_read():
@@ -346,6 +351,7 @@ def main():
             terra.terra_swin_attn_bwd_packed(desc, qkv, bias, o, lse, d_o, dqkv, dbias, ws)
         b.record()
         barrier()
+        terra.terra_swin_check()
         packed_ms = max_over_ranks(a.elapsed_time(b) / n_packed, dev)
         packed = {"value": whole_job_tflops(flops, world, packed_ms), "unit": UNIT, "ms_per_step": packed_ms, "steps": n_packed,
                   "note": "terra_swin_attn_fwd_packed + terra_swin_attn_bwd_packed on qkv / dqkv [B, H, W, 3, heads, d]"}
@@ -411,6 +417,7 @@ def main():
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e2e_steps(n_e2e, a, b)
         barrier()
+        terra.terra_swin_check()
         e2e_ms = max_over_ranks(a.elapsed_time(b) / n_e2e, dev)
         e2e = {"value": whole_job_tflops(flops, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -454,7 +461,8 @@ def main():
             "bwd_tflops": wk["flop_bwd"] / (bwd_ms * 1e-3) / 1e12,
             "roofline": {"bound": "tensor", "kernel": dom["kernel"], "avg_ms": dom["avg_ms"],
                          "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved / peak_tf,
-                         "traffic": dom["dram_bytes_ncu"], "peak_kind": f"{peak_kind} burst bf16",
+                         "traffic": dom["dram_bytes_ncu"], "traffic_source": TRAFFIC_SOURCE if dom["dram_bytes_ncu"] else None,
+                         "peak_kind": f"{peak_kind} burst bf16",
                          "note": "dominant kernel by time; achieved = its algorithmic FLOP / its CUDA-event duration"},
             "kernels": kernels,
             "roofline_hbm": {"bound": "hbm", "achieved": (wk["bytes_fwd"] + wk["bytes_bwd"]) / (ms_step * 1e-3) / 1e9,

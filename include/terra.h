@@ -18,6 +18,9 @@
  *     with (a, b) the in-window offsets; masked pairs get probability exactly zero.
  *
  * All pointers are DEVICE pointers unless stated otherwise, 16-byte aligned, owned by the caller.
+ * The device that holds them must be the CURRENT device of the calling thread (cudaSetDevice): every entry
+ * point launches on the current device and takes its SM count, and the built-in scratch of
+ * terra_swin_attn_fwd_noalloc, from it.
  * Calls enqueue work on `stream` (a cudaStream_t passed as void*; NULL = the legacy default stream)
  * and return without synchronising.  No call allocates device memory; scratch comes from the
  * caller's workspace.  Every function returns a terra_status; nothing throws, nothing falls back to
@@ -139,10 +142,18 @@ int terra_swin_attn_bwd_packed(const terra_swin_desc* desc, const void* qkv, con
  * buffers up front, a callback from which cudaMalloc is off limits.  Such a caller still brings the inputs
  * and outputs, but has nowhere to get the forward kernel's scratch (one prepared bias table per head) from.
  * Here that scratch is a fixed array compiled into the library: TERRA_NOALLOC_MAX_HEADS * 9216 bytes
- * (576 KiB) on every GPU that loads the library, held until the process exits.  The call allocates nothing:
- * no cudaMalloc / cudaFree, no allocating library routine.
+ * (576 KiB) on every GPU that loads the library, held until the process exits.  The call itself allocates
+ * nothing: no cudaMalloc / cudaFree, no allocating library routine.  One thing happens once per device: under
+ * CUDA's lazy module loading the FIRST call on a device is what makes the driver load the code module that
+ * holds the array and place it in that device's memory.  So make one warm-up call per device during
+ * initialisation -- outside any callback, real-time section or stream capture -- and only later calls are
+ * free of loading and allocation.
  *
- * Arguments, layouts, results and error codes are those of terra_swin_attn_fwd; the output is the same.
+ * Arguments, layouts and error codes are those of terra_swin_attn_fwd.  Results: the same within the
+ * library's tolerance; bit-equal to terra_swin_attn_fwd for head_dim 32 with window <= 16, where both run the
+ * same tensor-core kernel.  For every other shape this entry point runs the register-tile forward kernel
+ * (`swin_fwd_mma_kernel`, which needs no scratch) while terra_swin_attn_fwd may pick a faster chunked
+ * tensor-core kernel that does need a workspace: equal within tolerance, not bit for bit, and slower.
  * Extra rules:
  *   - heads > TERRA_NOALLOC_MAX_HEADS is refused with TERRA_ERR_NOALLOC_LIMIT when the shape uses the
  *     scratch (head_dim 32, window <= 16); other shapes need no scratch and are not limited;

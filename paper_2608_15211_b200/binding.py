@@ -100,6 +100,10 @@ def _ptr(t) -> ctypes.c_void_p:
         raise ValueError("terra: tensors must be CUDA tensors (the library has no CPU path)")
     if not t.is_contiguous():
         raise ValueError("terra: tensors must be contiguous")
+    if t.device.index != torch.cuda.current_device():
+        # the library launches on the current device (its stream, SM count and built-in scratch are that device's)
+        raise ValueError(f"terra: tensor lives on {t.device} but the current device is cuda:{torch.cuda.current_device()}; "
+                         "make the tensors' device current (torch.cuda.device(...)) around the call")
     return ctypes.c_void_p(t.data_ptr())
 
 

@@ -2,8 +2,6 @@
 import numpy as np
 import torch
 
-import oracle
-
 # Gates for bf16 outputs against the fp64 oracle (stated by the benchmark spec for this path):
 #   G1  max |err| <= 2e-2 * max |ref|
 #   G2  |err_i| <= 2e-2 * max |ref| + 3e-2 * |ref_i|  for every element
@@ -37,17 +35,3 @@ def gpu_rows(t, cfg, tokens):
     flat = t.reshape(cfg.B * cfg.H * cfg.W, *t.shape[3:])
     idx = torch.from_numpy(np.asarray(tokens)).to(t.device)
     return flat[idx].float().cpu().double().numpy()
-
-
-def sample_windows(cfg, count, seed=0):
-    """(batch * n_windows + window) ids: the four corner windows (edge classes, seam, latitude wrap),
-    the rest drawn at random."""
-    _, nw, _ = oracle.route_sizes(cfg)
-    mw = -(-cfg.W // cfg.window)
-    mh = nw // mw
-    fixed = {0, mw - 1, (mh - 1) * mw, nw - 1, (mh - 1) * mw + mw // 2, (mh // 2) * mw + mw - 1}
-    ids = {(cfg.B - 1) * nw + g for g in fixed}
-    rng = np.random.default_rng(seed)
-    while len(ids) < min(count, cfg.B * nw):
-        ids.add(int(rng.integers(0, cfg.B * nw)))
-    return np.array(sorted(ids), dtype=np.int64)

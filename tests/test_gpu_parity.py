@@ -6,7 +6,7 @@ import torch
 import oracle
 import paper_2608_15211_b200 as terra
 from paper_2608_15211_b200.workloads import CONFIGS, make_inputs, small_config
-from tests._parity import gate, gpu_rows, sample_windows
+from tests._parity import gate, gpu_rows
 
 pytestmark = pytest.mark.gpu
 
@@ -46,22 +46,22 @@ def _run_bwd(cfg, d, xg, o, lse):
     return out
 
 
-def _check_forward(cfg, x, o, lse, sel, scale=0.0):
+def _check_forward(cfg, x, o, lse, sel, scale=0.0, strict=True):
     ro, rl = oracle.attn_fwd(cfg, x["q"], x["k"], x["v"], x["bias"].double().numpy(), sel=sel, scale=scale)
     tok = oracle.selection_tokens(cfg, sel)
-    gate("o", gpu_rows(o, cfg, tok), ro)
-    gate("lse", gpu_rows(lse, cfg, tok), rl)
+    gate("o", gpu_rows(o, cfg, tok), ro, strict)
+    gate("lse", gpu_rows(lse, cfg, tok), rl, strict)
 
 
-def _check_backward(cfg, x, grads, sel, dbias_ref_is_total, scale=0.0):
+def _check_backward(cfg, x, grads, sel, dbias_ref_is_total, scale=0.0, strict=True):
     dq, dk, dv, dbias = grads
     rq, rk, rv, rb = oracle.attn_bwd(cfg, x["q"], x["k"], x["v"], x["do"], x["bias"].double().numpy(), sel=sel, scale=scale)
     tok = oracle.selection_tokens(cfg, sel)
-    gate("dq", gpu_rows(dq, cfg, tok), rq)
-    gate("dk", gpu_rows(dk, cfg, tok), rk)
-    gate("dv", gpu_rows(dv, cfg, tok), rv)
+    gate("dq", gpu_rows(dq, cfg, tok), rq, strict)
+    gate("dk", gpu_rows(dk, cfg, tok), rk, strict)
+    gate("dv", gpu_rows(dv, cfg, tok), rv, strict)
     if dbias_ref_is_total:
-        gate("dbias", dbias.cpu().double().numpy(), rb)
+        gate("dbias", dbias.cpu().double().numpy(), rb, strict)
 
 
 @pytest.mark.parametrize("name", ["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
@@ -136,32 +136,83 @@ def test_full_tensors_forward_backward(name):
     _check_backward(cfg, x, grads, None, True)
 
 
-@pytest.mark.parametrize("name,count", [("cfg4", 8), ("cfg5", 48)])
-def test_full_size_sampled_windows(name, count):
-    """Full-size launch; the oracle recomputes a sample of windows (every edge class included).
-    dBias sums over all windows, so it is checked on a second backward launch whose upstream gradient
-    is zero outside the sampled windows: there the full sum equals the oracle's sum over the sample."""
-    cfg = CONFIGS[name]
+def test_cfg4_full_tensors_forward_backward():
+    """Config 4 at full size, every one of its 128 windows against the oracle (O, LSE, dQ, dK, dV, dBias)."""
+    cfg = CONFIGS["cfg4"]
     x = make_inputs(cfg)
     xg = _to_gpu(x)
-    sel = sample_windows(cfg, count)
     d, o, lse = _run_fwd(cfg, xg)
-    _check_forward(cfg, x, o, lse, sel)
+    _check_forward(cfg, x, o, lse, None)
     grads = _run_bwd(cfg, d, xg, o, lse)
-    _check_backward(cfg, x, grads, sel, False)
-    # property that holds at any size: every softmax row's dS sums to zero, hence so does dT per head
-    # (up to the rounding of the saved bf16 O that enters delta: a random walk over all query rows)
-    dbias = grads[3].double()
-    assert torch.all(dbias.sum(0).abs() <= 2e-3 * dbias.abs().sum(0))
-    del grads
-    tok = torch.from_numpy(oracle.selection_tokens(cfg, sel)).cuda()
-    do_sparse = torch.zeros_like(xg["do"])
-    flat_src = xg["do"].reshape(cfg.tokens, cfg.heads, cfg.head_dim)
-    do_sparse.reshape(cfg.tokens, cfg.heads, cfg.head_dim)[tok] = flat_src[tok]
-    xs = dict(xg, do=do_sparse)
-    grads = _run_bwd(cfg, d, xs, o, lse)
-    x2 = dict(x, do=do_sparse.cpu())
-    _check_backward(cfg, x2, grads, sel, True)
+    _check_backward(cfg, x, grads, None, True)
+
+
+def test_cfg5_full_size_every_window_in_chunks():
+    """Config 5 at full size: ONE forward and ONE backward launch over all 22 630 windows; the oracle then walks
+    over the windows in chunks (its fp64 results for the whole problem would not fit in host memory at once).
+    Every output row of every chunk is compared, and the oracle's bias gradient, which is additive over
+    selections of windows, is summed over the chunks and compared with the launch's full dBias."""
+    cfg = CONFIGS["cfg5"]
+    x = make_inputs(cfg)
+    xg = _to_gpu(x)
+    d, o, lse = _run_fwd(cfg, xg)
+    dq, dk, dv, dbias = _run_bwd(cfg, d, xg, o, lse)
+    _, nw, _ = oracle.route_sizes(cfg)
+    total = cfg.B * nw
+    bias64 = x["bias"].double().numpy()
+    rb_sum = np.zeros((cfg.bias_rows, cfg.heads))
+    n_chunks = 24
+    for c in range(n_chunks):
+        sel = np.arange(c * total // n_chunks, (c + 1) * total // n_chunks, dtype=np.int64)
+        tok = oracle.selection_tokens(cfg, sel)
+        ro, rl = oracle.attn_fwd(cfg, x["q"], x["k"], x["v"], bias64, sel=sel)
+        gate(f"o[{c}]", gpu_rows(o, cfg, tok), ro)
+        gate(f"lse[{c}]", gpu_rows(lse, cfg, tok), rl)
+        del ro, rl
+        rq, rk, rv, rb = oracle.attn_bwd(cfg, x["q"], x["k"], x["v"], x["do"], bias64, sel=sel)
+        gate(f"dq[{c}]", gpu_rows(dq, cfg, tok), rq)
+        gate(f"dk[{c}]", gpu_rows(dk, cfg, tok), rk)
+        gate(f"dv[{c}]", gpu_rows(dv, cfg, tok), rv)
+        rb_sum += rb
+        del rq, rk, rv
+    gate("dbias", dbias.cpu().double().numpy(), rb_sum)
+
+
+# Activations far from N(0, 1): scores of tens to thousands of nats, a bias table with one entry of +200 and a
+# wide spread, and grids whose windows mix shift-mask groups and end in truncated windows.  The keys a query may
+# not see (the other mask group, slots past the window's extent) then carry scores that exceed every allowed one by
+# hundreds of nats: a softmax that takes its maximum over them would underflow to 0 / 0.
+LARGE = [
+    # name,            B, H,  W,  heads, d,  w,  sh, sw, ph, pw, q/k factor
+    ("x8_w16_masks", 1, 40, 56, 2, 32, 16, 8, 8, 0, 0, 8.0),
+    ("x32_w16_masks", 1, 40, 56, 2, 32, 16, 8, 8, 0, 0, 32.0),
+    ("x8_w14", 2, 37, 45, 3, 32, 14, 7, 7, 0, 1, 8.0),
+    ("x32_w8", 1, 24, 40, 2, 32, 8, 4, 4, 0, 0, 32.0),
+    ("x8_d64_w32", 1, 70, 80, 2, 64, 32, 16, 16, 0, 0, 8.0),
+    ("x32_d64_w32", 1, 70, 80, 2, 64, 32, 16, 16, 0, 0, 32.0),
+    ("x8_d64_w20", 1, 45, 50, 2, 64, 20, 10, 10, 0, 1, 8.0),
+]
+
+
+@pytest.mark.parametrize("case", LARGE, ids=[c[0] for c in LARGE])
+def test_large_magnitude_scores_and_wide_bias_stay_finite_and_exact(case):
+    cfg = small_config(*case[:-1])
+    f = case[-1]
+    x = make_inputs(cfg)
+    x["q"] = (x["q"].float() * f).to(torch.bfloat16)
+    x["k"] = (x["k"].float() * f).to(torch.bfloat16)
+    x["bias"] = x["bias"] * 25.0
+    x["bias"][3, 0] = 200.0                 # one entry far above the rest
+    x["bias"][5, :] = -150.0                # and a row far below
+    xg = _to_gpu(x)
+    d, o, lse = _run_fwd(cfg, xg)
+    assert torch.isfinite(o.float()).all() and torch.isfinite(lse).all()
+    _check_forward(cfg, x, o, lse, None)
+    # backward: the two gates of the tolerance statement.  With nearly one-hot softmax rows dS = P (dP - delta) is
+    # the difference of two nearly equal numbers, of which delta is taken from the saved bf16 O, so the tighter
+    # diagnostic gate (which budgets only bf16 rounding of the outputs) does not apply here.
+    grads = _run_bwd(cfg, d, xg, o, lse)
+    _check_backward(cfg, x, grads, None, True, strict=False)
 
 
 def test_outputs_are_reproducible_and_inputs_untouched():
