@@ -12,8 +12,11 @@
 // TMEM: columns [256 t, 256 t + 256) belong to query tile t: S (fp32) first; as pass 2 consumes it, bf16 P of
 // keys 0..127 goes to columns 0..63, the O accumulator to 64..111 and bf16 P of keys 128..255 to 128..191, so
 // that O += P V over the first 128 keys runs while the softmax of the second 128 keys is still going on.
-// The row maximum is replaced by the upper bound max_j(raw score) * scale + max(bias): softmax is shift
-// invariant, so the result is the same; only the exponent range matters.
+// Row maximum: windows without mask labels use the upper bound max_j(raw score) * scale + max(bias) over the key
+// slots that hold a token (softmax is shift invariant, so the result is the same; only the exponent range
+// matters: the bound exceeds the true maximum by at most the spread of the head's bias table, and a head whose
+// table spreads over more than 64 octaves takes the exact path); windows that mix shift-mask labels take the
+// exact maximum over the keys the row may see.
 // Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, all roles leave their loops,
 // TMEM is released and the host reads the device status word.
 #include "swin_common.cuh"
@@ -132,7 +135,6 @@ __device__ __forceinline__ int lds_i32(uint32_t addr) {
 template <int N, bool MASKED>
 __device__ __forceinline__ float softmax_cols(const uint32_t (&r)[N], uint32_t (&pk)[N / 2], int c, uint32_t bias_i,
                                               uint32_t a_kc, uint32_t a_klab, int label_i, float scale, float neg_m) {
-    float s0 = 0.f, s1 = 0.f;
 #pragma unroll
     for (int e4 = 0; e4 < N / 4; ++e4) {
         const int4 kc4 = lds_i4(a_kc + 4 * (c + e4 * 4));
@@ -143,19 +145,50 @@ __device__ __forceinline__ float softmax_cols(const uint32_t (&r)[N], uint32_t (
             kl[0] = kl4.x; kl[1] = kl4.y; kl[2] = kl4.z; kl[3] = kl4.w;
         }
         float p[4];
+        if (MASKED) {
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const float bv = lds_f32(bias_i + kc[e]);
-            float xv = fmaf(__uint_as_float(r[e4 * 4 + e]), scale, bv) + neg_m;
-            if (MASKED && kl[e] != label_i) xv = -INFINITY;
-            p[e] = fast_exp2(xv);
+            for (int e = 0; e < 4; ++e) {
+                const float bv = lds_f32(bias_i + kc[e]);
+                float xv = fmaf(__uint_as_float(r[e4 * 4 + e]), scale, bv) + neg_m;
+                if (kl[e] != label_i) xv = -INFINITY;
+                p[e] = fast_exp2(xv);
+            }
+        } else {
+            float bv[4], xv[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) bv[e] = lds_f32(bias_i + kc[e]);
+#pragma unroll
+            for (int e = 0; e < 4; e += 2) {
+                fma2(xv[e], xv[e + 1], __uint_as_float(r[e4 * 4 + e]), __uint_as_float(r[e4 * 4 + e + 1]), scale, bv[e], bv[e + 1]);
+                add2(xv[e], xv[e + 1], xv[e], xv[e + 1], neg_m);
+                p[e] = fast_exp2(xv[e]);
+                p[e + 1] = fast_exp2(xv[e + 1]);
+            }
         }
-        s0 += p[0] + p[1];
-        s1 += p[2] + p[3];
         pk[e4 * 2] = pack_bf16(p[0], p[1]);
         pk[e4 * 2 + 1] = pack_bf16(p[2], p[3]);
     }
-    return s0 + s1;
+    return 0.f;       // the row sum comes from the ones columns of the P V product
+}
+
+// exact maximum of scale * raw + bias (log2 domain) over the keys of N columns that the row may see: a key of another
+// mask group, or a slot without a token (its label matches no query's), gives -inf
+template <int N>
+__device__ __forceinline__ float score_max_cols(const uint32_t (&r)[N], int c, uint32_t bias_i, uint32_t a_kc, uint32_t a_klab,
+                                                int label_i, float scale, float mx) {
+#pragma unroll
+    for (int e4 = 0; e4 < N / 4; ++e4) {
+        const int4 kc4 = lds_i4(a_kc + 4 * (c + e4 * 4));
+        const int4 kl4 = lds_i4(a_klab + 4 * (c + e4 * 4));
+        const int kc[4] = {kc4.x, kc4.y, kc4.z, kc4.w};
+        const int kl[4] = {kl4.x, kl4.y, kl4.z, kl4.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float xv = fmaf(__uint_as_float(r[e4 * 4 + e]), scale, lds_f32(bias_i + kc[e]));
+            mx = fmaxf(mx, kl[e] == label_i ? xv : -INFINITY);
+        }
+    }
+    return mx;
 }
 
 template <int OFF>
@@ -176,9 +209,10 @@ __device__ __forceinline__ void softmax_cols16_row(const uint32_t* r, uint32_t* 
     bv[12] = lds_f32_at<12>(bb); bv[13] = lds_f32_at<8>(bb);  bv[14] = lds_f32_at<4>(bb);  bv[15] = lds_f32_at<0>(bb);
 #pragma unroll
     for (int e2 = 0; e2 < 8; ++e2) {
-        const float p0 = fast_exp2(fmaf(__uint_as_float(r[2 * e2]), scale, bv[2 * e2]) + neg_m);
-        const float p1 = fast_exp2(fmaf(__uint_as_float(r[2 * e2 + 1]), scale, bv[2 * e2 + 1]) + neg_m);
-        pk[e2] = pack_bf16(p0, p1);
+        float x0, x1;
+        fma2(x0, x1, __uint_as_float(r[2 * e2]), __uint_as_float(r[2 * e2 + 1]), scale, bv[2 * e2], bv[2 * e2 + 1]);
+        add2(x0, x1, x0, x1, neg_m);
+        pk[e2] = pack_bf16(fast_exp2(x0), fast_exp2(x1));
     }
 }
 
@@ -188,8 +222,14 @@ __device__ __forceinline__ void max_cols(const uint32_t (&r)[N], float (&mx)[4])
     for (int e = 0; e < N; e += 8) {
 #pragma unroll
         for (int a = 0; a < 4; ++a)
-            mx[a] = fmaxf(mx[a], fmaxf(__uint_as_float(r[e + 2 * a]), __uint_as_float(r[e + 2 * a + 1])));
+            mx[a] = max3(mx[a], __uint_as_float(r[e + 2 * a]), __uint_as_float(r[e + 2 * a + 1]));
     }
+}
+// the same over the first `nv` of N columns only (the others are key slots without a token: zero rows, raw score 0)
+template <int N>
+__device__ __forceinline__ void max_cols_limit(const uint32_t (&r)[N], int nv, float (&mx)[4]) {
+#pragma unroll
+    for (int e = 0; e < N; ++e) mx[e & 3] = fmaxf(mx[e & 3], e < nv ? __uint_as_float(r[e]) : -INFINITY);
 }
 
 // One softmax row: two passes over the row's S columns in TMEM, 32 columns per load, the next load in
@@ -197,16 +237,35 @@ __device__ __forceinline__ void max_cols(const uint32_t (&r)[N], float (&mx)[4])
 // ROW16: full 16 x 16 window without mask labels (npad = 256); `top0` = shared address of the bias entry of key 0
 // for this query, `row_step` = bytes between the entries of keys one window row apart.
 template <bool MASKED, bool ROW16 = false>
-__device__ __forceinline__ float softmax_row(uint32_t t_s, int npad, uint32_t bias_i, uint32_t a_kc, uint32_t a_klab,
+__device__ __forceinline__ float softmax_row(uint32_t t_s, int npad, int nvalid, uint32_t bias_i, uint32_t a_kc, uint32_t a_klab,
                                              int label_i, float scale, float bmax, float& sum_out, uint32_t bar_half,
                                              uint32_t top0 = 0, uint32_t row_step = 0) {
     const int nfull = npad >> 5;
     const bool tail = (npad & 16) != 0;
     uint32_t ra[32], rb[32];
-    float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-    {
+    float m;
+    if (MASKED) {
+        // exact maximum over the keys this row may see (bias included)
+        float mx = -INFINITY;
+        for (int i = 0; i < nfull; ++i) {
+            tmem_ld32(t_s + 32 * i, ra);
+            tmem_ld_wait();
+            mx = score_max_cols<32>(ra, 32 * i, bias_i, a_kc, a_klab, label_i, scale, mx);
+        }
+        if (tail) {
+            uint32_t rt[16];
+            tmem_ld16(t_s + 32 * nfull, rt);
+            tmem_ld_wait();
+            mx = score_max_cols<16>(rt, 32 * nfull, bias_i, a_kc, a_klab, label_i, scale, mx);
+        }
+        m = (mx == -INFINITY) ? 0.f : mx;     // a row without a token sees no key: its P is formed against 0 and is exactly 0
+    } else {
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+        // key slots without a token (zero rows, raw score 0) sit in the row's last 16 columns only and are left out
+        const bool limit = nvalid < npad;
+        const int nplain = (limit && !tail) ? nfull - 1 : nfull;
         int i = 0;
-        for (; i + 4 <= nfull; i += 4) {      // 128 columns per round trip to TMEM
+        for (; i + 4 <= nplain; i += 4) {      // 128 columns per round trip to TMEM
             uint32_t rc[32], rd[32];
             tmem_ld32(t_s + 32 * i, ra);
             tmem_ld32(t_s + 32 * (i + 1), rb);
@@ -218,20 +277,26 @@ __device__ __forceinline__ float softmax_row(uint32_t t_s, int npad, uint32_t bi
             max_cols<32>(rc, mx4);
             max_cols<32>(rd, mx4);
         }
-        for (; i < nfull; ++i) {
+        for (; i < nplain; ++i) {
             tmem_ld32(t_s + 32 * i, ra);
             tmem_ld_wait();
             max_cols<32>(ra, mx4);
         }
+        if (i < nfull) {                       // last full group, with a ragged end
+            tmem_ld32(t_s + 32 * i, ra);
+            tmem_ld_wait();
+            max_cols_limit<32>(ra, nvalid - 32 * i, mx4);
+        }
+        if (tail) {
+            uint32_t rt[16];
+            tmem_ld16(t_s + 32 * nfull, rt);
+            tmem_ld_wait();
+            if (limit) max_cols_limit<16>(rt, nvalid - 32 * nfull, mx4);
+            else max_cols<16>(rt, mx4);
+        }
+        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+        m = mx * scale + bmax;   // scale > 0: max of the scaled scores plus the largest bias
     }
-    if (tail) {
-        uint32_t rt[16];
-        tmem_ld16(t_s + 32 * nfull, rt);
-        tmem_ld_wait();
-        max_cols<16>(rt, mx4);
-    }
-    const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-    const float m = mx * scale + bmax;   // scale > 0: max of the scaled scores plus the largest bias
     const float neg_m = -m;
 
     float sum = 0.f;
@@ -563,15 +628,16 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
             if (!__all_sync(0xffffffffu, mbar_wait(bar_sready(wg), use & 1, cta_abort))) break;
             tc_fence_after();
             float m, sum;
+            const bool wide = bmax == INFINITY;      // the head's bias table spreads too far for the bound on the row maximum
             if (W16) {
-                if (x.masked || x.r.n != 256)
-                    m = softmax_row<true>(t_s, x.npad, bias_i, st_a + kOffKc, st_a + kOffKlab, label_i, scale, bmax, sum, bar_phalf(wg));
+                if (x.masked || x.r.n != 256 || wide)
+                    m = softmax_row<true>(t_s, x.npad, x.r.n, bias_i, st_a + kOffKc, st_a + kOffKlab, label_i, scale, bmax, sum, bar_phalf(wg));
                 else
-                    m = softmax_row<false, true>(t_s, x.npad, bias_i, st_a + kOffKc, st_a + kOffKlab, label_i, scale, bmax, sum, bar_phalf(wg),
+                    m = softmax_row<false, true>(t_s, x.npad, x.r.n, bias_i, st_a + kOffKc, st_a + kOffKlab, label_i, scale, bmax, sum, bar_phalf(wg),
                                                  bias_i + 4 * c0, 4 * cs);
             } else {
-                if (x.masked) m = softmax_row<true>(t_s, x.npad, bias_i, st_a + kOffKc, st_a + kOffKlab, label_i, scale, bmax, sum, bar_phalf(wg));
-                else m = softmax_row<false>(t_s, x.npad, bias_i, st_a + kOffKc, st_a + kOffKlab, label_i, scale, bmax, sum, bar_phalf(wg));
+                if (x.masked || wide) m = softmax_row<true>(t_s, x.npad, x.r.n, bias_i, st_a + kOffKc, st_a + kOffKlab, label_i, scale, bmax, sum, bar_phalf(wg));
+                else m = softmax_row<false>(t_s, x.npad, x.r.n, bias_i, st_a + kOffKc, st_a + kOffKlab, label_i, scale, bmax, sum, bar_phalf(wg));
             }
             tmem_st_wait();
             tc_fence_before();
@@ -620,14 +686,15 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
 // Per head, with code stride cs = w + 32 and c0 = (w - 1) * (cs + 1):
 //   table[(da + w - 1) * cs + (db + w - 1)] = T[(da + w - 1) * (2w - 1) + (db + w - 1), head] * log2(e)
 //   for |da|, |db| < w (unused gaps 0), table[2 c0 + 1 .. 3 c0 + 1] = -inf (where key slots without a
-//   token point), and the head's largest entry in the last float.
+//   token point), and the head's largest entry in the last float (+inf instead if the head's entries spread over
+//   more than 64 octaves: the forward kernel then takes exact row maxima).
 __global__ void __launch_bounds__(256)
 swin_fwd_bias_prep_kernel(const float* __restrict__ bias, float* __restrict__ prep, int w, int heads) {
     const int head = blockIdx.x;
     const int cs = w + 32, nw = 2 * w - 1;
     const int c0 = (w - 1) * (cs + 1);
     float* dst = prep + (size_t)head * kFwdBiasFloats;
-    float mx = -INFINITY;
+    float mx = -INFINITY, mn = INFINITY;
     for (int e = threadIdx.x; e < kFwdBiasFloats - 1; e += blockDim.x) {
         float val = 0.f;
         if (e > 2 * c0) {
@@ -637,18 +704,22 @@ swin_fwd_bias_prep_kernel(const float* __restrict__ bias, float* __restrict__ pr
             if (rb < nw) {
                 val = bias[(size_t)(ra * nw + rb) * heads + head] * kLog2e;
                 mx = fmaxf(mx, val);
+                mn = fminf(mn, val);
             }
         }
         dst[e] = val;
     }
-    __shared__ float red[8];
+    __shared__ float red[8], red_mn[8];
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = mx;
+    for (int off = 16; off > 0; off >>= 1) {
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, off));
+    }
+    if ((threadIdx.x & 31) == 0) { red[threadIdx.x >> 5] = mx; red_mn[threadIdx.x >> 5] = mn; }
     __syncthreads();
     if (threadIdx.x == 0) {
-        for (int i = 1; i < 8; ++i) mx = fmaxf(mx, red[i]);
-        dst[kFwdBiasFloats - 1] = mx;
+        for (int i = 1; i < 8; ++i) { mx = fmaxf(mx, red[i]); mn = fminf(mn, red_mn[i]); }
+        dst[kFwdBiasFloats - 1] = (mx - mn <= 64.f) ? mx : INFINITY;
     }
 }
 

@@ -3,8 +3,11 @@
 //
 // One persistent CTA per SM, bound to one head, walks over (batch, window, pair of 128-row query tiles) items.
 // The window's keys are streamed in chunks of 128 through a ring of shared-memory slots, twice:
-//   pass A   S = Q K_c^T per chunk, the softmax threads only take the row maximum of the raw scores
-//            (the same upper bound max_j(raw) * scale + max(bias) as in the small-window kernel);
+//   pass A   S = Q K_c^T per chunk, the softmax threads only take the row maximum: for complete windows without mask
+//            labels the upper bound max_j(raw) * scale + max(bias) of the small-window kernel; for windows that mix
+//            mask labels or hold slots without a token, and for heads whose bias table spreads over more than 64
+//            octaves, the exact maximum over the keys the row may see (the chunk's key tables are then staged in
+//            pass A as well, and its ring slot is released only when the softmax threads have read them);
 //   pass B   S = Q K_c^T again, P = exp2(S * scale + bias - m) written back over S as bf16, O += P [V_c | 1]
 //            (16 columns of ones behind V: the accumulator's columns 64..79 carry the row sums of P).
 // Recomputing S costs tensor-pipe time, of which there is plenty next to the exp work, and spares the running
@@ -187,6 +190,26 @@ __device__ __forceinline__ void softmax_cols32_row(const uint32_t (&r)[32], uint
     }
 }
 
+// exact maximum of scale * raw + bias over the keys of N columns that the row may see (others, and slots without a
+// token, give -inf)
+template <int N>
+__device__ __forceinline__ float score_max_cols(const uint32_t* r, int c, uint32_t bias_i, uint32_t a_kc, uint32_t a_klab,
+                                                int label_i, float scale, float mx) {
+#pragma unroll
+    for (int e4 = 0; e4 < N / 4; ++e4) {
+        const int4 kc4 = lds_i4(a_kc + 4 * (c + e4 * 4));
+        const int4 kl4 = lds_i4(a_klab + 4 * (c + e4 * 4));
+        const int kc[4] = {kc4.x, kc4.y, kc4.z, kc4.w};
+        const int kl[4] = {kl4.x, kl4.y, kl4.z, kl4.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float xv = fmaf(__uint_as_float(r[e4 * 4 + e]), scale, lds_f32(bias_i + kc[e]));
+            mx = fmaxf(mx, kl[e] == label_i ? xv : -INFINITY);
+        }
+    }
+    return mx;
+}
+
 template <int N>
 __device__ __forceinline__ void max_cols(const uint32_t (&r)[N], float (&mx)[4]) {
 #pragma unroll
@@ -263,6 +286,10 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
     const int cs = code_stride(g.w);
     const int c0 = (g.w - 1) * (cs + 1);
     const size_t HW = (size_t)g.H * g.W;
+    // the table's last float: the head's largest entry, or +inf if the table spreads too far for the bound on the row maximum
+    const bool wide = reinterpret_cast<const float*>(smem + kOffBias)[kBiasFloats - 1] == INFINITY;
+    // windows whose row maxima are taken exactly (every role derives this the same way)
+    auto exact_max = [&](const Item& x) { return x.masked || x.npad != x.r.n || wide; };
 
     if (warp >= kMmaWarp) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kRegsOther));
@@ -343,7 +370,8 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                 }
                 issued(bar_qfull(qs));
             }
-            // ---- the key chunks: pass A needs K only, pass B K and V
+            // ---- the key chunks: pass A needs K only (and the key tables if the row maxima are taken exactly), pass B K and V
+            const int first_meta_pass = exact_max(x) ? 0 : 1;
             for (int pass = 0; pass < 2 && ok; ++pass) {
                 for (int c = 0; c < x.nch; ++c, ++ru) {
                     const int s = (int)(ru % kSlots);
@@ -351,7 +379,7 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                     if (!ok) break;
                     const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes + hf * kKHalf;
                     const int ncols = min(kChunk, x.npad - c * kChunk);
-                    if (pass == 1) {
+                    if (pass >= first_meta_pass) {
                         int* kcs = reinterpret_cast<int*>(smem + kOffKeyMeta + s * 1024);
                         int* klab = kcs + 128;
                         for (int row = lt; row < kChunk; row += kLoaderThreads) {
@@ -447,6 +475,10 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                 return true;
             };
             // ---- pass A: S of every chunk, for the row maxima
+            // Exact row maxima: the softmax threads also read the chunk's key tables from the ring slot, so the slot is
+            // released (plain arrival) only after they have given the chunk's S columns back, one chunk later.
+            const bool exact = exact_max(x);
+            int held = -1;                                       // exact: slot of the chunk before, not released yet
             for (int c = 0; c < x.nch && ok; ++c, ++ru) {
                 const int s = (int)(ru % kSlots);
                 ok = chunk_ready(ru);
@@ -460,17 +492,24 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                     ++n_s[t];
                 }
                 if (!ok) break;
-                if (elect_one()) mma_commit(bar_kvempty(s));     // the slot is free once the MMAs issued so far are complete
+                if (elect_one()) {
+                    if (!exact) mma_commit(bar_kvempty(s));      // the slot is free once the MMAs issued so far are complete
+                    else if (held >= 0) mbar_arrive(bar_kvempty(held));   // every tile's softmax threads are done with it
+                }
                 __syncwarp();
+                held = exact ? s : -1;
             }
             if (!ok) break;
             // ---- pass B: per tile, PV of chunk c is followed at once by QK of chunk c + 1, so that a tile's softmax
             // threads wait for one PV and one QK product only, whatever the other tile is doing
             ok = chunk_ready(ru);
-            for (int t = 0; t < x.ntiles && ok; ++t) {
-                ok = s_free(t);
-                if (ok) issue_qk(t, smem0 + kOffSlots + (int)(ru % kSlots) * kSlotBytes, min(kChunk, x.npad));
+            for (int t = 0; t < x.ntiles && ok; ++t) ok = s_free(t);
+            if (ok && held >= 0) {
+                if (elect_one()) mbar_arrive(bar_kvempty(held));
+                __syncwarp();
             }
+            for (int t = 0; t < x.ntiles && ok; ++t)
+                issue_qk(t, smem0 + kOffSlots + (int)(ru % kSlots) * kSlotBytes, min(kChunk, x.npad));
             for (int c = 0; c < x.nch && ok; ++c, ++ru) {
                 const int s = (int)(ru % kSlots);
                 const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes;
@@ -543,9 +582,11 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             const int label_i = meta_label(rmeta);
             const float bmax = lds_f32(smem0 + kOffBias + 4 * (kBiasFloats - 1));
             const bool row32 = g.w == 32 && x.r.ew == 32 && !x.masked;       // then every key slot holds a token, too
+            const bool exact = exact_max(x);
             bool ok = true;
-            // ---- pass A: row maximum of the raw scores over all chunks
+            // ---- pass A: row maximum over all chunks
             float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            float mxe = -INFINITY;
             for (int c = 0; c < x.nch; ++c) {
                 const int ncols = min(kChunk, x.npad - c * kChunk);
                 ok = mbar_wait_all(bar_sready(wg), n_s & 1, cta_abort);
@@ -554,6 +595,21 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                 tc_fence_after();
                 uint32_t ra[32], rb[32];
                 int cc = 0;
+                if (exact) {
+                    const uint32_t a_kc = smem0 + kOffKeyMeta + (int)((ru0 + c) % kSlots) * 1024, a_klab = a_kc + 512;
+                    for (; cc + 32 <= ncols; cc += 32) {
+                        tmem_ld32(t_s + cc, ra);
+                        tmem_ld_wait();
+                        mxe = score_max_cols<32>(ra, cc, bias_i, a_kc, a_klab, label_i, scale, mxe);
+                    }
+                    if (cc < ncols) {
+                        uint32_t rt[16];
+                        tmem_ld16(t_s + cc, rt);
+                        tmem_ld_wait();
+                        mxe = score_max_cols<16>(rt, cc, bias_i, a_kc, a_klab, label_i, scale, mxe);
+                        cc = ncols;
+                    }
+                }
                 for (; cc + 64 <= ncols; cc += 64) {
                     tmem_ld32(t_s + cc, ra);
                     tmem_ld32(t_s + cc + 32, rb);
@@ -577,7 +633,8 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                 mbar_arrive(bar_sfree(wg));
             }
             if (!ok) break;
-            const float m = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale + bmax;
+            // a row without a token sees no key: its P is formed against 0 and is exactly 0
+            const float m = exact ? (mxe == -INFINITY ? 0.f : mxe) : fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale + bmax;
             const float neg_m = -m;
             // ---- pass B: P chunk by chunk
             for (int c = 0; c < x.nch; ++c) {
@@ -673,14 +730,15 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
 
 // The prepared bias table of the small-window kernel, sized for window sides up to 32: per head
 //   table[(da + w - 1) * cs + (db + w - 1)] = T[(da + w - 1) * (2w - 1) + (db + w - 1), head] * log2(e)   (cs = w + 32),
-//   table[2 c0 + 1 .. 3 c0 + 1] = -inf (where key slots without a token point), the head's largest entry in the last float.
+//   table[2 c0 + 1 .. 3 c0 + 1] = -inf (where key slots without a token point), the head's largest entry in the last float
+//   (+inf instead if the head's entries spread over more than 64 octaves).
 __global__ void __launch_bounds__(256)
 swin_fwd_bias_prep64_kernel(const float* __restrict__ bias, float* __restrict__ prep, int w, int heads) {
     const int head = blockIdx.x;
     const int cs = w + 32, nw = 2 * w - 1;
     const int c0 = (w - 1) * (cs + 1);
     float* dst = prep + (size_t)head * kBiasFloats;
-    float mx = -INFINITY;
+    float mx = -INFINITY, mn = INFINITY;
     for (int e = threadIdx.x; e < kBiasFloats - 1; e += blockDim.x) {
         float val = 0.f;
         if (e > 2 * c0) {
@@ -690,18 +748,24 @@ swin_fwd_bias_prep64_kernel(const float* __restrict__ bias, float* __restrict__ 
             if (rb < nw && ra < nw) {
                 val = bias[(size_t)(ra * nw + rb) * heads + head] * kLog2e;
                 mx = fmaxf(mx, val);
+                mn = fminf(mn, val);
             }
         }
         dst[e] = val;
     }
-    __shared__ float red[8];
+    __shared__ float red[8], red_mn[8];
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = mx;
+    for (int off = 16; off > 0; off >>= 1) {
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, off));
+    }
+    if ((threadIdx.x & 31) == 0) { red[threadIdx.x >> 5] = mx; red_mn[threadIdx.x >> 5] = mn; }
     __syncthreads();
     if (threadIdx.x == 0) {
-        for (int i = 1; i < 8; ++i) mx = fmaxf(mx, red[i]);
-        dst[kBiasFloats - 1] = mx;
+        for (int i = 1; i < 8; ++i) { mx = fmaxf(mx, red[i]); mn = fminf(mn, red_mn[i]); }
+        // a table that spreads over more than 64 octaves makes the bound max(raw) * scale + max(bias) on the row
+        // maximum too loose for the exponent range: +inf here tells the forward kernel to take exact row maxima
+        dst[kBiasFloats - 1] = (mx - mn <= 64.f) ? mx : INFINITY;
     }
 }
 

@@ -195,6 +195,42 @@ __device__ __forceinline__ void tmem_ld1(uint32_t taddr, uint32_t& r) {
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory"); }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory"); }
 
+// ---- two-wide fp32 arithmetic and three-input maximum (sm_100) ------------------------------------------
+// One instruction per pair of elements: the elementwise warps are bound by the instructions they issue.
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;\n" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+// (x0, x1) = (a0, a1) * s + (b0, b1)
+__device__ __forceinline__ void fma2(float& x0, float& x1, float a0, float a1, float s, float b0, float b1) {
+    asm("{\n\t.reg .b64 ra, rs, rb, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rs, {%4, %4};\n\tmov.b64 rb, {%5, %6};\n\t"
+        "fma.rn.f32x2 rd, ra, rs, rb;\n\t"
+        "mov.b64 {%0, %1}, rd;\n\t}\n" : "=f"(x0), "=f"(x1) : "f"(a0), "f"(a1), "f"(s), "f"(b0), "f"(b1));
+}
+// (x0, x1) = (a0, a1) + (b, b)
+__device__ __forceinline__ void add2(float& x0, float& x1, float a0, float a1, float b) {
+    asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %4};\n\t"
+        "add.rn.f32x2 rd, ra, rb;\n\t"
+        "mov.b64 {%0, %1}, rd;\n\t}\n" : "=f"(x0), "=f"(x1) : "f"(a0), "f"(a1), "f"(b));
+}
+// (x0, x1) = (a0, a1) - (b0, b1)
+__device__ __forceinline__ void sub2(float& x0, float& x1, float a0, float a1, float b0, float b1) {
+    asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+        "sub.rn.f32x2 rd, ra, rb;\n\t"
+        "mov.b64 {%0, %1}, rd;\n\t}\n" : "=f"(x0), "=f"(x1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+}
+// (x0, x1) = (a0, a1) * (b0, b1)
+__device__ __forceinline__ void mul2(float& x0, float& x1, float a0, float a1, float b0, float b1) {
+    asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+        "mul.rn.f32x2 rd, ra, rb;\n\t"
+        "mov.b64 {%0, %1}, rd;\n\t}\n" : "=f"(x0), "=f"(x1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+}
+
 __device__ __forceinline__ bool elect_one() {
     uint32_t pred;
     asm volatile(
