@@ -39,7 +39,7 @@ extern "C" {
 typedef enum {
     TERRA_OK = 0,
     TERRA_ERR_INVALID_ARG = 1,   /* null pointer, non-positive size, element count out of range   */
-    TERRA_ERR_UNSUPPORTED = 2,   /* head_dim not in {32, 64}, window too large, not an sm_100 GPU */
+    TERRA_ERR_UNSUPPORTED = 2,   /* head_dim not in {32, 64, 128}, window too large, not an sm_100 GPU */
     TERRA_ERR_ALIGNMENT = 3,     /* a pointer is not 16-byte aligned                              */
     TERRA_ERR_WORKSPACE = 4,     /* workspace NULL or smaller than terra_swin_workspace_bytes     */
     TERRA_ERR_CUDA = 5,          /* a CUDA call failed; text via terra_last_cuda_error            */
@@ -54,7 +54,7 @@ typedef enum {
 typedef struct {
     int32_t B;                      /* batch (samples / rollout steps), >= 1                      */
     int32_t H, W;                   /* token grid: latitude rows x longitude columns              */
-    int32_t heads, head_dim;        /* attention heads; per-head width, 32 or 64                  */
+    int32_t heads, head_dim;        /* attention heads; per-head width: 32, 64 or 128 (Table V)   */
     int32_t window;                 /* w: square window side, 1 <= w <= 32                        */
     int32_t shift_h, shift_w;       /* >= 0, taken mod H and mod W                                */
     int32_t periodic_h, periodic_w; /* 0 / 1; the paper's grids: latitude 0, longitude 1          */

@@ -424,10 +424,10 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
             }
             const int s = kuse % kStages;
             const uint32_t st_a = smem0 + s * kStageBytes;
-            if (!mbar_wait_all(bar_full(s), (kuse / kStages) & 1, cta_abort)) break;      // the slot -> token table of the stage
+            if (!mbar_wait_all_relaxed(bar_full(s), (kuse / kStages) & 1, cta_abort)) break;      // the slot -> token table of the stage
             for (int t = 0; t < ntiles; ++t, ++n_tile) {
                 const int set = n_tile & 1;
-                ok = mbar_wait_all(bar_acc(set), (n_tile >> 1) & 1, cta_abort);
+                ok = mbar_wait_all_relaxed(bar_acc(set), (n_tile >> 1) & 1, cta_abort);
                 if (!ok) break;
                 tc_fence_after();
                 const int slot = 32 * ((4 * t + quarter + key_interleave(g.w, ntiles) * lane) & (4 * ntiles - 1)) + lane;      // interleaved key order
@@ -442,7 +442,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                 store_rows(rows_a + kOffK, dk, sample_off, tok);
             }
             if (!ok) break;
-            ok = mbar_wait_all(bar_dq, kuse & 1, cta_abort);
+            ok = mbar_wait_all_relaxed(bar_dq, kuse & 1, cta_abort);
             if (!ok) break;
             tc_fence_after();
 #pragma unroll
@@ -476,7 +476,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                 mbar_arrive(bar_full(pending_s));
                 pending_s = -1;
             }
-            if (!mbar_wait_all(bar_empty(s), ((kuse / kStages) & 1) ^ 1, cta_abort)) break;
+            if (!mbar_wait_all_relaxed(bar_empty(s), ((kuse / kStages) & 1) ^ 1, cta_abort)) break;
             const Item x = make_item(g, cur_it);
             unsigned char* st = smem + s * kStageBytes;
             const uint32_t st_a = smem0 + s * kStageBytes;

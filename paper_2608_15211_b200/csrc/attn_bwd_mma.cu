@@ -39,23 +39,36 @@ __device__ __forceinline__ void load_rows(unsigned char* s_tile, const __nv_bflo
     }
 }
 
-// acc (16 x 64 per warp) = own rows (fragments in registers) x streamed block^T
+// Head dim 128: the fragments of the CTA's own rows (two operands x 8 k-steps) and two 16 x 128 accumulators do not
+// fit the register file together, so the own-row fragments are re-read from their shared-memory tiles at each use.
 template <int D>
-__device__ __forceinline__ void rows_times_block_t(float (&acc)[BN / 8][4], const uint32_t (&af)[D / 16][4],
-                                                   const unsigned char* blk, int lane) {
+constexpr bool kFragsInRegs = D <= 64;
+
+// acc (16 x 64 per warp) = own rows x streamed block^T; the own rows' fragments come from registers (af) or, for
+// head dim 128, from their shared-memory tile (own)
+template <int D>
+__device__ __forceinline__ void rows_times_block_t(float (&acc)[BN / 8][4], const uint32_t (&af)[kFragsInRegs<D> ? D / 16 : 1][4],
+                                                   const unsigned char* own, const unsigned char* blk, int warp, int lane) {
 #pragma unroll
     for (int i = 0; i < BN / 8; ++i)
 #pragma unroll
         for (int e = 0; e < 4; ++e) acc[i][e] = 0.f;
 #pragma unroll
     for (int ks = 0; ks < D / 16; ++ks) {
+        uint32_t a[4];
+        if constexpr (kFragsInRegs<D>) {
+            a[0] = af[ks][0]; a[1] = af[ks][1]; a[2] = af[ks][2]; a[3] = af[ks][3];
+        } else {
+            const int row = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+            ldmatrix_x4(a, smem_u32(own + tile_off<D>(row, 2 * ks + (lane >> 4))));
+        }
 #pragma unroll
         for (int np = 0; np < BN / 16; ++np) {
             uint32_t bf[4];
             int r = np * 16 + (lane & 7) + (lane >> 4) * 8;
             ldmatrix_x4(bf, smem_u32(blk + tile_off<D>(r, 2 * ks + ((lane >> 3) & 1))));
-            mma_bf16(acc[2 * np], af[ks], bf[0], bf[1]);
-            mma_bf16(acc[2 * np + 1], af[ks], bf[2], bf[3]);
+            mma_bf16(acc[2 * np], a, bf[0], bf[1]);
+            mma_bf16(acc[2 * np + 1], a, bf[2], bf[3]);
         }
     }
 }
@@ -199,7 +212,7 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
         load_rows<D>(s_c2, str2, s_tok, 0, sample_off, ts_str2, head, tid);
         cp_async_commit();
 
-        uint32_t f1[KS][4], f2[KS][4];
+        uint32_t f1[kFragsInRegs<D> ? KS : 1][4], f2[kFragsInRegs<D> ? KS : 1][4];
         float acc1[DT][4], acc2[KV ? DT : 1][4];
 #pragma unroll
         for (int i = 0; i < DT; ++i)
@@ -226,20 +239,22 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
                 cp_async_wait<0>();
             }
             __syncthreads();
-            if (blk == 0) {
+            if constexpr (kFragsInRegs<D>) {
+                if (blk == 0) {
 #pragma unroll
-                for (int ks = 0; ks < KS; ++ks) {
-                    int row = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
-                    ldmatrix_x4(f1[ks], smem_u32(s_r1 + tile_off<D>(row, 2 * ks + (lane >> 4))));
-                    ldmatrix_x4(f2[ks], smem_u32(s_r2 + tile_off<D>(row, 2 * ks + (lane >> 4))));
+                    for (int ks = 0; ks < KS; ++ks) {
+                        int row = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+                        ldmatrix_x4(f1[ks], smem_u32(s_r1 + tile_off<D>(row, 2 * ks + (lane >> 4))));
+                        ldmatrix_x4(f2[ks], smem_u32(s_r2 + tile_off<D>(row, 2 * ks + (lane >> 4))));
+                    }
                 }
             }
             const unsigned char* c1 = s_c1 + stage * TILE_BYTES;
             const unsigned char* c2 = s_c2 + stage * TILE_BYTES;
 
             float acc_s[BN / 8][4], acc_dp[BN / 8][4];
-            rows_times_block_t<D>(acc_s, f1, c1, lane);     // S (or S^T) before scale and bias
-            rows_times_block_t<D>(acc_dp, f2, c2, lane);    // dP (or dP^T)
+            rows_times_block_t<D>(acc_s, f1, s_r1, c1, warp, lane);     // S (or S^T) before scale and bias
+            rows_times_block_t<D>(acc_dp, f2, s_r2, c2, warp, lane);    // dP (or dP^T)
 
             // P = exp2(S * scale * log2e + bias * log2e - lse * log2e);  dS = P * (dP - delta)
 #pragma unroll
@@ -449,8 +464,10 @@ cudaError_t launch_bwd_delta(const Geo& g, const void* o, const void* d_o, float
     prof_begin("swin_bwd_delta_kernel", stream);
     if (g.d == 32)
         swin_bwd_delta_kernel<32><<<blocks, 256, 0, stream>>>((const __nv_bfloat16*)o, (const __nv_bfloat16*)d_o, delta, rows);
-    else
+    else if (g.d == 64)
         swin_bwd_delta_kernel<64><<<blocks, 256, 0, stream>>>((const __nv_bfloat16*)o, (const __nv_bfloat16*)d_o, delta, rows);
+    else
+        swin_bwd_delta_kernel<128><<<blocks, 256, 0, stream>>>((const __nv_bfloat16*)o, (const __nv_bfloat16*)d_o, delta, rows);
     count_launch(stream);
     return cudaGetLastError();
 }
@@ -461,6 +478,11 @@ cudaError_t launch_bwd_mma(const Geo& g, const void* q, const void* k, const voi
                            bool query_side_only) {
     cudaError_t e = cudaMemsetAsync(dbias, 0, sizeof(float) * (size_t)(2 * g.w - 1) * (2 * g.w - 1) * g.heads, stream);
     if (e != cudaSuccess) return e;
+    if (g.d == 128) {
+        e = launch_one<128, true>(g, q, k, v, d_o, bias, lse, delta, dk, dv, nullptr, sm_count, stream);
+        if (e != cudaSuccess) return e;
+        return launch_one<128, false>(g, q, k, v, d_o, bias, lse, delta, dq, nullptr, dbias, sm_count, stream);
+    }
     if (query_side_only)      // dK, dV come from another kernel
         return g.d == 32 ? launch_one<32, false>(g, q, k, v, d_o, bias, lse, delta, dq, nullptr, dbias, sm_count, stream)
                          : launch_one<64, false>(g, q, k, v, d_o, bias, lse, delta, dq, nullptr, dbias, sm_count, stream);

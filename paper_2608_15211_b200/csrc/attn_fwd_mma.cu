@@ -5,7 +5,7 @@
 // Roll, window gather, shift mask, relative-position bias, softmax, PV and the scatter back to the
 // contiguous grid all happen here; nothing window-major is ever written to global memory.
 // This path covers every window class (truncated edges, the split latitude-wrap row, w up to 32,
-// head dim 32 / 64).
+// head dim 32 / 64 / 128; head dim 128, the width of the paper's Table V models, runs here only).
 #include "swin_common.cuh"
 #include "swin_kernels.h"
 
@@ -244,7 +244,7 @@ cudaError_t launch_fwd_mma(const Geo& g, const void* q, const void* k, const voi
     const int qtiles = (g.nmax + BM - 1) / BM;
     const long long items = (long long)g.B * g.Mh * g.Mw * g.heads * qtiles;
     const size_t smem = fwd_smem_bytes(g);
-    auto kern = (g.d == 32) ? swin_fwd_mma_kernel<32> : swin_fwd_mma_kernel<64>;
+    auto kern = (g.d == 32) ? swin_fwd_mma_kernel<32> : (g.d == 64) ? swin_fwd_mma_kernel<64> : swin_fwd_mma_kernel<128>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     prof_begin("swin_fwd_mma_kernel", stream);

@@ -418,7 +418,7 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
                 mbar_arrive(bar_full(pending_s));
                 pending_s = -1;
             }
-            if (!__all_sync(0xffffffffu, mbar_wait(bar_empty(s), ((kuse / kStages) & 1) ^ 1, cta_abort))) break;
+            if (!mbar_wait_all_relaxed(bar_empty(s), ((kuse / kStages) & 1) ^ 1, cta_abort)) break;
             const Item x = make_item(g, cur_it);
             unsigned char* st = smem + s * kStageBytes;
             const uint32_t st_a = smem0 + s * kStageBytes;

@@ -40,21 +40,58 @@ __device__ __forceinline__ void fence_proxy_async() {
     asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
 }
 
+// One round of polling: up to 64 try_waits in a loop of five instructions.  A try_wait that finds the phase open
+// comes back after a hardware time slice of the order of a hundred cycles, so a waiting warp executes a handful of
+// instructions per slice; with many warps waiting at any time (issuer, loaders, read-out, the elementwise warps
+// between hand-overs) a longer loop body costs the working warps a noticeable share of the issue slots.
+// SLEEP_NS > 0 adds a nanosleep between polls, for roles that run stages ahead and can afford to wake up late.
+template <int SLEEP_NS>
+__device__ __forceinline__ bool mbar_poll_round(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    if (SLEEP_NS > 0) {
+        asm volatile(
+            "{\n\t.reg .pred p, q;\n\t.reg .u32 n;\n\t"
+            "mov.u32 n, 0;\n"
+            "TERRA_WAIT_S:\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "@p bra TERRA_DONE_S;\n\t"
+            "nanosleep.u32 %3;\n\t"
+            "add.u32 n, n, 1;\n\t"
+            "setp.lt.u32 q, n, 64;\n\t"
+            "@q bra TERRA_WAIT_S;\n"
+            "TERRA_DONE_S:\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}\n"
+            : "=r"(ok) : "r"(bar), "r"(parity), "n"(SLEEP_NS) : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p, q;\n\t.reg .u32 n;\n\t"
+            "mov.u32 n, 0;\n"
+            "TERRA_WAIT:\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "@p bra TERRA_DONE;\n\t"
+            "add.u32 n, n, 1;\n\t"
+            "setp.lt.u32 q, n, 64;\n\t"
+            "@q bra TERRA_WAIT;\n"
+            "TERRA_DONE:\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}\n"
+            : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    }
+    return ok != 0;
+}
+
 // Bounded wait: gives up after `limit_cycles` SM clocks (or when another thread of the CTA already gave
 // up), raises the CTA's abort flag and returns false.  No trap, no endless spin.
+template <int SLEEP_NS = 0>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* cta_abort,
                                           long long limit_cycles = 4000000000LL) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
-    int polls = 0;
     while (true) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((++polls & 255) == 0) {
-            if (*cta_abort) return false;
-            if (clock64() - t0 > limit_cycles) {
-                *cta_abort = 1;
-                return false;
-            }
+        if (mbar_poll_round<SLEEP_NS>(bar, parity)) return true;
+        if (*cta_abort) return false;
+        if (clock64() - t0 > limit_cycles) {
+            *cta_abort = 1;
+            return false;
         }
     }
 }
@@ -62,7 +99,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 // All 32 lanes of a warp wait together: a warp whose lanes all sit in try_wait is put to sleep and woken as a
 // whole.  (One polling lane with the other 31 parked at a warp barrier was measured 25 % slower end to end.)
 __device__ __forceinline__ bool mbar_wait_all(uint32_t bar, uint32_t parity, volatile int* cta_abort) {
-    return __all_sync(0xffffffffu, mbar_wait(bar, parity, cta_abort));
+    return __all_sync(0xffffffffu, mbar_wait<0>(bar, parity, cta_abort));
+}
+// The same for roles that work stages ahead of their consumers (loaders, read-out warps): they sleep between polls.
+__device__ __forceinline__ bool mbar_wait_all_relaxed(uint32_t bar, uint32_t parity, volatile int* cta_abort) {
+    return __all_sync(0xffffffffu, mbar_wait<128>(bar, parity, cta_abort));
 }
 
 // ---- tcgen05: TMEM allocation -----------------------------------------------------------------------

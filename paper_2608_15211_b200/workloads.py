@@ -56,6 +56,11 @@ CONFIGS = {
     "cfg3": SwinConfig("cfg3", 1, 510, 1080, 12, 32, 16, 8, 8, index=3),   # Wenhai-shaped, patch 4
     "cfg4": SwinConfig("cfg4", 1, 256, 512, 12, 64, 32, 16, 16, index=4),  # large window
     "cfg5": SwinConfig("cfg5", 2, 1020, 2160, 8, 32, 14, 7, 7, index=5),   # fine patch, batch 2
+    # The paper's own model shapes (Table V: 128 channels per head; patch 4, sampling factor 2 on the field padded to
+    # 2304 x 4352, i.e. a 288 x 544 token grid in the Transformer blocks, Section VII-B): small, medium and large model.
+    "tv_small": SwinConfig("tv_small", 1, 288, 544, 8, 128, 8, 4, 4, index=6),
+    "tv_medium": SwinConfig("tv_medium", 1, 288, 544, 32, 128, 8, 4, 4, index=7),
+    "tv_large": SwinConfig("tv_large", 1, 288, 544, 64, 128, 32, 16, 16, index=8),
 }
 
 TENSOR_INDEX = {"q": 0, "k": 1, "v": 2, "do": 3, "bias": 4}
