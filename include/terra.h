@@ -47,6 +47,15 @@ typedef enum {
     TERRA_ERR_NOALLOC_LIMIT = 7  /* terra_swin_attn_fwd_noalloc: more heads than its fixed scratch holds */
 } terra_status;
 
+/*
+ * Element type of the activations and their gradients.  bf16 is the type the tensor-core kernels of this library
+ * are written for; fp16 is what the paper trains in (Section VII-A: FP16 mixed precision) and runs on the
+ * register-tile kernels for every shape.  Scores, softmax, accumulation, lse, bias_table and dbias are fp32 either
+ * way.  A descriptor zero-initialised beyond `scale` selects bf16.
+ */
+#define TERRA_DTYPE_BF16 0
+#define TERRA_DTYPE_F16 1
+
 /* Largest `heads` terra_swin_attn_fwd_noalloc accepts on the shapes that need scratch. */
 #define TERRA_NOALLOC_MAX_HEADS 64
 
@@ -59,6 +68,7 @@ typedef struct {
     int32_t shift_h, shift_w;       /* >= 0, taken mod H and mod W                                */
     int32_t periodic_h, periodic_w; /* 0 / 1; the paper's grids: latitude 0, longitude 1          */
     float scale;                    /* score scale; <= 0 selects 1/sqrt(head_dim)                 */
+    int32_t dtype;                  /* element type of q, k, v, o, d_o, dq, dk, dv: TERRA_DTYPE_*   */
 } terra_swin_desc;
 
 /*
@@ -90,7 +100,8 @@ int terra_swin_workspace_bytes(const terra_swin_desc* desc, int backward, size_t
 /*
  * Forward shifted-window attention (Section IV-A W-MSA / SW-MSA; route + attention + inverse route
  * in one pass).
- *   q, k, v      bf16 [B, H, W, heads, head_dim], innermost contiguous (the contiguous grid layout)
+ *   q, k, v      bf16 (fp16 with TERRA_DTYPE_F16, like every "bf16" below) [B, H, W, heads, head_dim], innermost
+ *                contiguous (the contiguous grid layout)
  *   bias_table   fp32 [(2w-1)^2, heads]
  *   o            bf16 [B, H, W, heads, head_dim]   attention output at the token's grid position
  *   lse          fp32 [B, H, W, heads]             natural-log sum-exp of each score row (for bwd)

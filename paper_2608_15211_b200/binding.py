@@ -30,7 +30,9 @@ class TerraError(RuntimeError):
 class terra_swin_desc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in
                 ("B", "H", "W", "heads", "head_dim", "window", "shift_h", "shift_w", "periodic_h", "periodic_w")] + \
-               [("scale", ctypes.c_float)]
+               [("scale", ctypes.c_float), ("dtype", ctypes.c_int32)]
+
+TERRA_DTYPE_BF16, TERRA_DTYPE_F16 = 0, 1
 
 
 _lib = None
@@ -79,10 +81,18 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
     return lib
 
 
-def make_desc(cfg, scale: float = 0.0) -> terra_swin_desc:
-    """Descriptor from any object with B, H, W, heads, head_dim, window, shift_*, periodic_* fields."""
+def make_desc(cfg, scale: float = 0.0, dtype=torch.bfloat16) -> terra_swin_desc:
+    """Descriptor from any object with B, H, W, heads, head_dim, window, shift_*, periodic_* fields; `dtype` is the
+    element type of the activations (torch.bfloat16 or torch.float16)."""
+    if dtype not in (torch.bfloat16, torch.float16):
+        raise ValueError("terra: activations are bf16 or fp16")
     return terra_swin_desc(cfg.B, cfg.H, cfg.W, cfg.heads, cfg.head_dim, cfg.window, cfg.shift_h, cfg.shift_w,
-                           cfg.periodic_h, cfg.periodic_w, float(scale))
+                           cfg.periodic_h, cfg.periodic_w, float(scale),
+                           TERRA_DTYPE_F16 if dtype == torch.float16 else TERRA_DTYPE_BF16)
+
+
+def _act_dtype(desc):
+    return torch.float16 if desc.dtype == TERRA_DTYPE_F16 else torch.bfloat16
 
 
 def _check(status: int) -> None:
@@ -187,13 +197,13 @@ def terra_swin_attn_fwd(desc, q, k, v, bias_table, o=None, lse=None, workspace=N
     Returns (o bf16 like q, lse fp32 [B, H, W, heads]); pass o / lse / workspace to reuse buffers."""
     n = desc.B * desc.H * desc.W * desc.heads
     for name, t in (("q", q), ("k", k), ("v", v)):
-        _expect(t, torch.bfloat16, n * desc.head_dim, name)
+        _expect(t, _act_dtype(desc), n * desc.head_dim, name)
     _expect(bias_table, torch.float32, (2 * desc.window - 1) ** 2 * desc.heads, "bias_table")
     if o is None:
         o = torch.empty_like(q)
     if lse is None:
         lse = torch.empty((desc.B, desc.H, desc.W, desc.heads), dtype=torch.float32, device=q.device)
-    _expect(o, torch.bfloat16, n * desc.head_dim, "o")
+    _expect(o, _act_dtype(desc), n * desc.head_dim, "o")
     _expect(lse, torch.float32, n, "lse")
     if workspace is None:
         need = terra_swin_workspace_bytes(desc, False)
@@ -210,7 +220,7 @@ def terra_swin_attn_fwd_noalloc(desc, q, k, v, bias_table, o, lse):
     for its limits: at most TERRA_NOALLOC_MAX_HEADS heads, calls on one device must not overlap)."""
     n = desc.B * desc.H * desc.W * desc.heads
     for name, t in (("q", q), ("k", k), ("v", v), ("o", o)):
-        _expect(t, torch.bfloat16, n * desc.head_dim, name)
+        _expect(t, _act_dtype(desc), n * desc.head_dim, name)
     _expect(bias_table, torch.float32, (2 * desc.window - 1) ** 2 * desc.heads, "bias_table")
     _expect(lse, torch.float32, n, "lse")
     _check(load_library().terra_swin_attn_fwd_noalloc(ctypes.byref(desc), _ptr(q), _ptr(k), _ptr(v), _ptr(bias_table),
@@ -223,7 +233,7 @@ def terra_swin_attn_bwd(desc, q, k, v, bias_table, o, lse, d_o, dq=None, dk=None
     """Backward.  Returns (dq, dk, dv bf16 like q, dbias fp32 like bias_table)."""
     n = desc.B * desc.H * desc.W * desc.heads
     for name, t in (("q", q), ("k", k), ("v", v), ("o", o), ("d_o", d_o)):
-        _expect(t, torch.bfloat16, n * desc.head_dim, name)
+        _expect(t, _act_dtype(desc), n * desc.head_dim, name)
     _expect(lse, torch.float32, n, "lse")
     _expect(bias_table, torch.float32, (2 * desc.window - 1) ** 2 * desc.heads, "bias_table")
     dq = torch.empty_like(q) if dq is None else dq
@@ -231,7 +241,7 @@ def terra_swin_attn_bwd(desc, q, k, v, bias_table, o, lse, d_o, dq=None, dk=None
     dv = torch.empty_like(q) if dv is None else dv
     dbias = torch.empty_like(bias_table) if dbias is None else dbias
     for name, t in (("dq", dq), ("dk", dk), ("dv", dv)):
-        _expect(t, torch.bfloat16, n * desc.head_dim, name)
+        _expect(t, _act_dtype(desc), n * desc.head_dim, name)
     _expect(dbias, torch.float32, bias_table.numel(), "dbias")
     if workspace is None:
         workspace = torch.empty(terra_swin_workspace_bytes(desc, True), dtype=torch.uint8, device=q.device)
@@ -246,13 +256,13 @@ def terra_swin_attn_fwd_packed(desc, qkv, bias_table, o=None, lse=None, workspac
     """Forward on the packed projection output.  qkv bf16 [B, H, W, 3, heads, head_dim] (q, k, v in that order);
     returns (o bf16 [B, H, W, heads, head_dim], lse fp32 [B, H, W, heads])."""
     n = desc.B * desc.H * desc.W * desc.heads
-    _expect(qkv, torch.bfloat16, 3 * n * desc.head_dim, "qkv")
+    _expect(qkv, _act_dtype(desc), 3 * n * desc.head_dim, "qkv")
     _expect(bias_table, torch.float32, (2 * desc.window - 1) ** 2 * desc.heads, "bias_table")
     if o is None:
-        o = torch.empty((desc.B, desc.H, desc.W, desc.heads, desc.head_dim), dtype=torch.bfloat16, device=qkv.device)
+        o = torch.empty((desc.B, desc.H, desc.W, desc.heads, desc.head_dim), dtype=_act_dtype(desc), device=qkv.device)
     if lse is None:
         lse = torch.empty((desc.B, desc.H, desc.W, desc.heads), dtype=torch.float32, device=qkv.device)
-    _expect(o, torch.bfloat16, n * desc.head_dim, "o")
+    _expect(o, _act_dtype(desc), n * desc.head_dim, "o")
     _expect(lse, torch.float32, n, "lse")
     if workspace is None:
         need = terra_swin_workspace_bytes(desc, False)
@@ -266,14 +276,14 @@ def terra_swin_attn_fwd_packed(desc, qkv, bias_table, o=None, lse=None, workspac
 def terra_swin_attn_bwd_packed(desc, qkv, bias_table, o, lse, d_o, dqkv=None, dbias=None, workspace=None):
     """Backward on the packed layout.  Returns (dqkv bf16 like qkv, dbias fp32 like bias_table)."""
     n = desc.B * desc.H * desc.W * desc.heads
-    _expect(qkv, torch.bfloat16, 3 * n * desc.head_dim, "qkv")
+    _expect(qkv, _act_dtype(desc), 3 * n * desc.head_dim, "qkv")
     for name, t in (("o", o), ("d_o", d_o)):
-        _expect(t, torch.bfloat16, n * desc.head_dim, name)
+        _expect(t, _act_dtype(desc), n * desc.head_dim, name)
     _expect(lse, torch.float32, n, "lse")
     _expect(bias_table, torch.float32, (2 * desc.window - 1) ** 2 * desc.heads, "bias_table")
     dqkv = torch.empty_like(qkv) if dqkv is None else dqkv
     dbias = torch.empty_like(bias_table) if dbias is None else dbias
-    _expect(dqkv, torch.bfloat16, 3 * n * desc.head_dim, "dqkv")
+    _expect(dqkv, _act_dtype(desc), 3 * n * desc.head_dim, "dqkv")
     _expect(dbias, torch.float32, bias_table.numel(), "dbias")
     if workspace is None:
         workspace = torch.empty(terra_swin_workspace_bytes(desc, True), dtype=torch.uint8, device=qkv.device)

@@ -65,6 +65,7 @@ static int make_geo(const terra_swin_desc* d, bool for_attention, Geo* out) {
         if (d->head_dim != 32 && d->head_dim != 64 && d->head_dim != 128) return TERRA_ERR_UNSUPPORTED;
         if (d->window > 32) return TERRA_ERR_UNSUPPORTED;
         if (!(d->scale == d->scale) || std::isinf(d->scale)) return TERRA_ERR_INVALID_ARG;
+        if (d->dtype != TERRA_DTYPE_BF16 && d->dtype != TERRA_DTYPE_F16) return TERRA_ERR_INVALID_ARG;
     }
     Geo g;
     g.B = d->B; g.H = d->H; g.W = d->W;
@@ -75,6 +76,7 @@ static int make_geo(const terra_swin_desc* d, bool for_attention, Geo* out) {
     g.Mh = (d->H + d->window - 1) / d->window;
     g.Mw = (d->W + d->window - 1) / d->window;
     g.nmax = (d->window < d->H ? d->window : d->H) * (d->window < d->W ? d->window : d->W);
+    g.f16 = for_attention && d->dtype == TERRA_DTYPE_F16;
     const float scale = d->scale > 0.f ? d->scale : 1.0f / std::sqrt((float)d->head_dim);
     g.scale_log2e = scale * kLog2e;
     *out = g;
@@ -108,18 +110,20 @@ static bool force_register_path() {
     return on;
 }
 
-static bool use_fwd_tc64(const Geo& g) { return fwd_tc64_supported(g) && !force_register_path(); }
+// the tcgen05 kernels are written for bf16 operands; fp16 runs on the register-tile kernels
+static bool use_fwd_tc(const Geo& g) { return fwd_tc_supported(g) && !g.f16; }
+static bool use_fwd_tc64(const Geo& g) { return fwd_tc64_supported(g) && !force_register_path() && !g.f16; }
 
 static size_t fwd_bytes(const Geo& g) {
-    if (force_register_path()) return 0;
+    if (force_register_path() || g.f16) return 0;
     if (fwd_tc_supported(g)) return align_up(fwd_tc_workspace_bytes(g), 256);
     if (use_fwd_tc64(g)) return align_up(fwd_tc64_workspace_bytes(g), 256);
     return 0;
 }
 
-static bool use_bwd_tc(const Geo& g) { return bwd_tc_supported(g) && !force_register_path(); }
+static bool use_bwd_tc(const Geo& g) { return bwd_tc_supported(g) && !force_register_path() && !g.f16; }
 
-static bool use_bwd_kv64(const Geo& g) { return bwd_kv64_supported(g) && !force_register_path(); }
+static bool use_bwd_kv64(const Geo& g) { return bwd_kv64_supported(g) && !force_register_path() && !g.f16; }
 
 static size_t delta_bytes(const Geo& g) {
     if (use_bwd_tc(g)) return align_up(bwd_tc_workspace_bytes(g), 256);
@@ -184,7 +188,9 @@ static int fwd_call(const Geo& g, const void* q, const void* k, const void* v,
     rc = device_props(&sms);
     if (rc) return rc;
     cudaError_t e;
-    if (need > 0 && use_fwd_tc64(g) && !fwd_tc_supported(g))
+    if (g.f16)
+        e = launch_fwd_mma_f16(g, q, k, v, bias_table, o, lse, (cudaStream_t)stream);
+    else if (need > 0 && use_fwd_tc64(g) && !use_fwd_tc(g))
         e = launch_fwd_tc64(g, q, k, v, bias_table, o, lse, workspace, sms, (cudaStream_t)stream);
     else if (need > 0)
         e = launch_fwd_tc(g, q, k, v, bias_table, o, lse, workspace, sms, (cudaStream_t)stream);
@@ -236,6 +242,11 @@ static int bwd_call(const Geo& g, const void* q, const void* k, const void* v,
         return et == cudaSuccess ? TERRA_OK : cuda_fail(et, "terra_swin_attn_bwd");
     }
     float* delta = reinterpret_cast<float*>(workspace);
+    if (g.f16) {
+        cudaError_t ef = launch_bwd_delta_f16(g, o, d_o, delta, st);
+        if (ef == cudaSuccess) ef = launch_bwd_mma_f16(g, q, k, v, bias_table, lse, delta, d_o, dq, dk, dv, dbias, sms, st);
+        return ef == cudaSuccess ? TERRA_OK : cuda_fail(ef, "terra_swin_attn_bwd");
+    }
     cudaError_t e = launch_bwd_delta(g, o, d_o, delta, st);
     if (e != cudaSuccess) return cuda_fail(e, "terra_swin_attn_bwd (delta)");
     if (use_bwd_kv64(g)) {

@@ -1,4 +1,5 @@
 // Backward shifted-window attention, register-tile path (warp-level mma.sync).
+// The file is compiled for bf16 and, through attn_bwd_mma_f16.cu, for fp16 activations.
 //
 // Three launches: (1) delta = rowsum(dO * O); (2) key-tile CTAs produce dK and dV; (3) query-tile
 // CTAs produce dQ and the relative-position-bias gradient.  (2) and (3) are one kernel template: a
@@ -67,8 +68,8 @@ __device__ __forceinline__ void rows_times_block_t(float (&acc)[BN / 8][4], cons
             uint32_t bf[4];
             int r = np * 16 + (lane & 7) + (lane >> 4) * 8;
             ldmatrix_x4(bf, smem_u32(blk + tile_off<D>(r, 2 * ks + ((lane >> 3) & 1))));
-            mma_bf16(acc[2 * np], a, bf[0], bf[1]);
-            mma_bf16(acc[2 * np + 1], a, bf[2], bf[3]);
+            mma_elem(acc[2 * np], a, bf[0], bf[1]);
+            mma_elem(acc[2 * np + 1], a, bf[2], bf[3]);
         }
     }
 }
@@ -80,17 +81,17 @@ __device__ __forceinline__ void coef_times_block(float (&out)[D / 8][4], const f
 #pragma unroll
     for (int ks = 0; ks < BN / 16; ++ks) {
         uint32_t pf[4];
-        pf[0] = pack_bf16(coef[2 * ks][0], coef[2 * ks][1]);
-        pf[1] = pack_bf16(coef[2 * ks][2], coef[2 * ks][3]);
-        pf[2] = pack_bf16(coef[2 * ks + 1][0], coef[2 * ks + 1][1]);
-        pf[3] = pack_bf16(coef[2 * ks + 1][2], coef[2 * ks + 1][3]);
+        pf[0] = pack_elem(coef[2 * ks][0], coef[2 * ks][1]);
+        pf[1] = pack_elem(coef[2 * ks][2], coef[2 * ks][3]);
+        pf[2] = pack_elem(coef[2 * ks + 1][0], coef[2 * ks + 1][1]);
+        pf[3] = pack_elem(coef[2 * ks + 1][2], coef[2 * ks + 1][3]);
 #pragma unroll
         for (int dp = 0; dp < D / 16; ++dp) {
             uint32_t bf[4];
             int r = ks * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
             ldmatrix_x4_trans(bf, smem_u32(blk + tile_off<D>(r, 2 * dp + (lane >> 4))));
-            mma_bf16(out[2 * dp], pf, bf[0], bf[1]);
-            mma_bf16(out[2 * dp + 1], pf, bf[2], bf[3]);
+            mma_elem(out[2 * dp], pf, bf[0], bf[1]);
+            mma_elem(out[2 * dp + 1], pf, bf[2], bf[3]);
         }
     }
 }
@@ -101,8 +102,8 @@ __device__ __forceinline__ void stage_rows(unsigned char* tile, const float (&ac
 #pragma unroll
     for (int i = 0; i < D / 8; ++i) {
         int lr = warp * 16 + gq;
-        *reinterpret_cast<uint32_t*>(tile + tile_off<D>(lr, i) + tq * 4) = pack_bf16(acc[i][0] * mul, acc[i][1] * mul);
-        *reinterpret_cast<uint32_t*>(tile + tile_off<D>(lr + 8, i) + tq * 4) = pack_bf16(acc[i][2] * mul, acc[i][3] * mul);
+        *reinterpret_cast<uint32_t*>(tile + tile_off<D>(lr, i) + tq * 4) = pack_elem(acc[i][0] * mul, acc[i][1] * mul);
+        *reinterpret_cast<uint32_t*>(tile + tile_off<D>(lr + 8, i) + tq * 4) = pack_elem(acc[i][2] * mul, acc[i][3] * mul);
     }
 }
 
@@ -400,11 +401,11 @@ swin_bwd_delta_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloat16* 
     if (row < rows) {
         uint4 a = *reinterpret_cast<const uint4*>(o + row * D + chunk * 8);
         uint4 b = *reinterpret_cast<const uint4*>(d_o + row * D + chunk * 8);
-        const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&a);
-        const __nv_bfloat162* pb = reinterpret_cast<const __nv_bfloat162*>(&b);
+        const uint32_t* pa = reinterpret_cast<const uint32_t*>(&a);
+        const uint32_t* pb = reinterpret_cast<const uint32_t*>(&b);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            float2 x = __bfloat1622float2(pa[i]), y = __bfloat1622float2(pb[i]);
+            float2 x = elem2_to_float2(pa[i]), y = elem2_to_float2(pb[i]);
             acc += x.x * y.x + x.y * y.y;
         }
     }
@@ -456,7 +457,7 @@ cudaError_t launch_one(const Geo& g, const void* q, const void* k, const void* v
 
 }  // namespace
 
-cudaError_t launch_bwd_delta(const Geo& g, const void* o, const void* d_o, float* delta, cudaStream_t stream) {
+cudaError_t TERRA_ELEM_FN(launch_bwd_delta)(const Geo& g, const void* o, const void* d_o, float* delta, cudaStream_t stream) {
     const long long rows = (long long)g.B * g.H * g.W * g.heads;
     const int lpr = g.d / 8;
     const long long threads = rows * lpr;
@@ -472,7 +473,7 @@ cudaError_t launch_bwd_delta(const Geo& g, const void* o, const void* d_o, float
     return cudaGetLastError();
 }
 
-cudaError_t launch_bwd_mma(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
+cudaError_t TERRA_ELEM_FN(launch_bwd_mma)(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
                            const float* lse, const float* delta, const void* d_o,
                            void* dq, void* dk, void* dv, float* dbias, int sm_count, cudaStream_t stream,
                            bool query_side_only) {

@@ -4,6 +4,7 @@
 // shared memory in 64-key blocks with an online softmax, so any window size up to 32 x 32 fits.
 // Roll, window gather, shift mask, relative-position bias, softmax, PV and the scatter back to the
 // contiguous grid all happen here; nothing window-major is ever written to global memory.
+// The file is compiled for bf16 and, through attn_fwd_mma_f16.cu, for fp16 activations.
 // This path covers every window class (truncated edges, the split latitude-wrap row, w up to 32,
 // head dim 32 / 64 / 128; head dim 128, the width of the paper's Table V models, runs here only).
 #include "swin_common.cuh"
@@ -128,8 +129,8 @@ swin_fwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
                 uint32_t bf[4];
                 int key = np * 16 + (lane & 7) + (lane >> 4) * 8;
                 ldmatrix_x4(bf, smem_u32(sk + tile_off<D>(key, 2 * ks + ((lane >> 3) & 1))));
-                mma_bf16(acc_s[2 * np], qf[ks], bf[0], bf[1]);
-                mma_bf16(acc_s[2 * np + 1], qf[ks], bf[2], bf[3]);
+                mma_elem(acc_s[2 * np], qf[ks], bf[0], bf[1]);
+                mma_elem(acc_s[2 * np + 1], qf[ks], bf[2], bf[3]);
             }
         }
 
@@ -177,17 +178,17 @@ swin_fwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
 #pragma unroll
         for (int ks = 0; ks < BN / 16; ++ks) {
             uint32_t pf[4];
-            pf[0] = pack_bf16(acc_s[2 * ks][0], acc_s[2 * ks][1]);
-            pf[1] = pack_bf16(acc_s[2 * ks][2], acc_s[2 * ks][3]);
-            pf[2] = pack_bf16(acc_s[2 * ks + 1][0], acc_s[2 * ks + 1][1]);
-            pf[3] = pack_bf16(acc_s[2 * ks + 1][2], acc_s[2 * ks + 1][3]);
+            pf[0] = pack_elem(acc_s[2 * ks][0], acc_s[2 * ks][1]);
+            pf[1] = pack_elem(acc_s[2 * ks][2], acc_s[2 * ks][3]);
+            pf[2] = pack_elem(acc_s[2 * ks + 1][0], acc_s[2 * ks + 1][1]);
+            pf[3] = pack_elem(acc_s[2 * ks + 1][2], acc_s[2 * ks + 1][3]);
 #pragma unroll
             for (int dp = 0; dp < DT / 2; ++dp) {
                 uint32_t bf[4];
                 int key = ks * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
                 ldmatrix_x4_trans(bf, smem_u32(sv + tile_off<D>(key, 2 * dp + (lane >> 4))));
-                mma_bf16(acc_o[2 * dp], pf, bf[0], bf[1]);
-                mma_bf16(acc_o[2 * dp + 1], pf, bf[2], bf[3]);
+                mma_elem(acc_o[2 * dp], pf, bf[0], bf[1]);
+                mma_elem(acc_o[2 * dp + 1], pf, bf[2], bf[3]);
             }
         }
         __syncthreads();
@@ -207,8 +208,8 @@ swin_fwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
     for (int i = 0; i < DT; ++i) {
         int lr = warp * 16 + gq;
         // chunk i holds columns 8i..8i+7; this thread owns columns 2tq, 2tq+1 of it
-        *reinterpret_cast<uint32_t*>(s_q + tile_off<D>(lr, i) + tq * 4) = pack_bf16(acc_o[i][0] * inv[0], acc_o[i][1] * inv[0]);
-        *reinterpret_cast<uint32_t*>(s_q + tile_off<D>(lr + 8, i) + tq * 4) = pack_bf16(acc_o[i][2] * inv[1], acc_o[i][3] * inv[1]);
+        *reinterpret_cast<uint32_t*>(s_q + tile_off<D>(lr, i) + tq * 4) = pack_elem(acc_o[i][0] * inv[0], acc_o[i][1] * inv[0]);
+        *reinterpret_cast<uint32_t*>(s_q + tile_off<D>(lr + 8, i) + tq * 4) = pack_elem(acc_o[i][2] * inv[1], acc_o[i][3] * inv[1]);
     }
     if (tq == 0) {
 #pragma unroll
@@ -239,7 +240,7 @@ size_t fwd_smem_bytes(const Geo& g) {
 
 }  // namespace
 
-cudaError_t launch_fwd_mma(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
+cudaError_t TERRA_ELEM_FN(launch_fwd_mma)(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
                            void* o, float* lse, cudaStream_t stream) {
     const int qtiles = (g.nmax + BM - 1) / BM;
     const long long items = (long long)g.B * g.Mh * g.Mw * g.heads * qtiles;

@@ -1,6 +1,7 @@
 // Shared device-side definitions of the shifted-window attention kernels (sm_100a).
 #pragma once
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -17,6 +18,7 @@ struct Geo {
     int ph, pw;           // periodic flags
     int Mh, Mw;           // window grid: ceil(H / w) x ceil(W / w)
     int nmax;             // tokens in a full window: min(w, H) * min(w, W)
+    int f16;              // activations and gradients are fp16 instead of bf16 (the paper trains in fp16 mixed precision)
     float scale_log2e;    // score scale * log2(e)
 };
 
@@ -144,6 +146,29 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
 }
+// D (16x8, fp32) += A (16x16, fp16, row) * B (16x8, fp16, col)
+__device__ __forceinline__ void mma_f16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+    __half2 v = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+// The register-tile kernel files are compiled twice, for bf16 and (with TERRA_ELEM_F16 defined by a one-line wrapper
+// file) for fp16 activations: same code, the element type enters through these three operations and the name suffix.
+#ifdef TERRA_ELEM_F16
+#define TERRA_ELEM_FN(name) name##_f16
+#define mma_elem mma_f16
+#define pack_elem pack_f16
+__device__ __forceinline__ float2 elem2_to_float2(uint32_t v) { return __half22float2(*reinterpret_cast<const __half2*>(&v)); }
+#else
+#define TERRA_ELEM_FN(name) name
+#define mma_elem mma_bf16
+#define pack_elem pack_bf16
+__device__ __forceinline__ float2 elem2_to_float2(uint32_t v) { return __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&v)); }
+#endif
 __device__ __forceinline__ float fast_exp2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));

@@ -18,6 +18,14 @@ cudaError_t launch_route(const Geo& g, int32_t* perm, int32_t* inv_perm, int32_t
 
 cudaError_t launch_fwd_mma(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
                            void* o, float* lse, cudaStream_t stream);
+// the register-tile kernels for fp16 activations and gradients (same arguments)
+cudaError_t launch_fwd_mma_f16(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
+                               void* o, float* lse, cudaStream_t stream);
+cudaError_t launch_bwd_delta_f16(const Geo& g, const void* o, const void* d_o, float* delta, cudaStream_t stream);
+cudaError_t launch_bwd_mma_f16(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
+                               const float* lse, const float* delta, const void* d_o,
+                               void* dq, void* dk, void* dv, float* dbias, int sm_count, cudaStream_t stream,
+                               bool query_side_only = false);
 
 // tcgen05 forward path (head dim 32, window side <= 16)
 constexpr int kFwdBiasFloats = 2304;   // prepared bias table per head (padded rows, -inf zone, maximum in the last float)
