@@ -64,7 +64,7 @@ typedef struct {
     int32_t B;                      /* batch (samples / rollout steps), >= 1                      */
     int32_t H, W;                   /* token grid: latitude rows x longitude columns              */
     int32_t heads, head_dim;        /* attention heads; per-head width: 32, 64 or 128 (Table V)   */
-    int32_t window;                 /* w: square window side, 1 <= w <= 32                        */
+    int32_t window;                 /* w: square window side, 1 <= w <= 128                       */
     int32_t shift_h, shift_w;       /* >= 0, taken mod H and mod W                                */
     int32_t periodic_h, periodic_w; /* 0 / 1; the paper's grids: latitude 0, longitude 1          */
     float scale;                    /* score scale; <= 0 selects 1/sqrt(head_dim)                 */

@@ -63,7 +63,7 @@ static int make_geo(const terra_swin_desc* d, bool for_attention, Geo* out) {
     if ((long long)d->B * d->H * d->W * d->heads > (1LL << 40)) return TERRA_ERR_INVALID_ARG;
     if (for_attention) {
         if (d->head_dim != 32 && d->head_dim != 64 && d->head_dim != 128) return TERRA_ERR_UNSUPPORTED;
-        if (d->window > 32) return TERRA_ERR_UNSUPPORTED;
+        if (d->window > 128) return TERRA_ERR_UNSUPPORTED;
         if (!(d->scale == d->scale) || std::isinf(d->scale)) return TERRA_ERR_INVALID_ARG;
         if (d->dtype != TERRA_DTYPE_BF16 && d->dtype != TERRA_DTYPE_F16) return TERRA_ERR_INVALID_ARG;
     }
@@ -350,7 +350,7 @@ const char* terra_strerror(int status) {
     switch (status) {
         case TERRA_OK: return "ok";
         case TERRA_ERR_INVALID_ARG: return "invalid argument (null pointer, non-positive size, or size out of range)";
-        case TERRA_ERR_UNSUPPORTED: return "unsupported configuration (head_dim must be 32, 64 or 128, window <= 32, GPU must be sm_100)";
+        case TERRA_ERR_UNSUPPORTED: return "unsupported configuration (head_dim must be 32, 64 or 128, window <= 128, GPU must be sm_100)";
         case TERRA_ERR_ALIGNMENT: return "pointer is not 16-byte aligned";
         case TERRA_ERR_WORKSPACE: return "workspace missing or too small (see terra_swin_workspace_bytes)";
         case TERRA_ERR_CUDA: return "CUDA error (see terra_last_cuda_error)";

@@ -125,7 +125,11 @@ __device__ __forceinline__ void scatter_rows(const unsigned char* tile, __nv_bfl
 // KV = false: CTA owns 64 queries (own tiles Q, dO; streams K, V) -> dQ, dBias
 constexpr int kStageStride = 40;   // floats per row of the dS staging tile (32 columns used)
 
-template <int D, bool KV>
+// BIG = windows of more than 1024 tokens (window sides 33 .. 128): the slot tables cover the CTA's own 64 rows plus
+// the streamed block in flight (two stages) instead of the whole window, the bias is read from the caller's table in
+// global memory, and the bias gradient goes to global memory with atomics (summed over diagonals first where the
+// window is complete along its width).
+template <int D, bool KV, bool BIG>
 __global__ void __launch_bounds__(NTHREADS)
 swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                     const __nv_bfloat16* __restrict__ v, const __nv_bfloat16* __restrict__ d_o,
@@ -139,13 +143,15 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
 
     const int nbias = (2 * g.w - 1) * (2 * g.w - 1);
     const int npad_max = ((g.nmax + BN - 1) / BN) * BN;
+    // tables: small windows [npad_max] slots of the window; BIG: [0, 64) the CTA's own rows, [64, 192) two streamed blocks
+    const int ntab = BIG ? 3 * BN : npad_max;
     int* s_tok = reinterpret_cast<int*>(smem);
-    int* s_meta = s_tok + npad_max;
-    float* s_lse = reinterpret_cast<float*>(s_meta + npad_max);
-    float* s_delta = s_lse + npad_max;
-    float* s_bias = s_delta + npad_max;
-    float* s_dbias = s_bias + nbias;
-    unsigned char* s_r1 = smem + (((size_t)npad_max * 16 + (size_t)nbias * 8 + 127) / 128) * 128;
+    int* s_meta = s_tok + ntab;
+    float* s_lse = reinterpret_cast<float*>(s_meta + ntab);
+    float* s_delta = s_lse + ntab;
+    float* s_bias = s_delta + ntab;
+    float* s_dbias = s_bias + (BIG ? 0 : nbias);
+    unsigned char* s_r1 = smem + (((size_t)ntab * 16 + (BIG ? 0 : (size_t)nbias * 8) + 127) / 128) * 128;
     unsigned char* s_r2 = s_r1 + TILE_BYTES;
     unsigned char* s_c1 = s_r2 + TILE_BYTES;          // two stages
     unsigned char* s_c2 = s_c1 + 2 * TILE_BYTES;      // two stages
@@ -172,10 +178,11 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
     // token strides: q, k, v and the gradients may be slices of a packed tensor; dO is dense
     const int ts_own2 = KV ? g.ts : g.heads * D, ts_str2 = KV ? g.heads * D : g.ts;
 
-    for (int i = tid; i < nbias; i += NTHREADS) {
-        s_bias[i] = bias[(size_t)i * g.heads + head] * kLog2e;
-        s_dbias[i] = 0.f;
-    }
+    if (!BIG)
+        for (int i = tid; i < nbias; i += NTHREADS) {
+            s_bias[i] = bias[(size_t)i * g.heads + head] * kLog2e;
+            s_dbias[i] = 0.f;
+        }
     if (use_acc)
         for (int i = tid; i < BM * acc_stride; i += NTHREADS) s_acc[i] = 0.f;
 
@@ -191,26 +198,39 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
         const size_t sample_off = (size_t)b * g.H * g.W;
 
         __syncthreads();   // previous item's readers of the slot tables and tiles are done
-        for (int s = tid; s < npad; s += NTHREADS) {
-            int meta = 0xff << 16, tok = -1;
-            float l2 = INFINITY, dl = 0.f;      // padded queries: P = exp2(x - inf) = 0
-            if (s < r.n) {
-                tok = slot_token(g, r, s, meta);
-                size_t li = (sample_off + (size_t)tok) * g.heads + head;
-                l2 = lse[li] * kLog2e;
-                dl = delta[li];
+        // fills `count` table entries at `base` with the window's slots first .. first + count - 1
+        auto fill_table = [&](int base, int first, int count) {
+            for (int i = tid; i < count; i += NTHREADS) {
+                const int sl = first + i;
+                int meta = 0xff << 16, tok = -1;
+                float l2 = INFINITY, dl = 0.f;      // padded queries: P = exp2(x - inf) = 0
+                if (sl < r.n) {
+                    tok = slot_token(g, r, sl, meta);
+                    size_t li = (sample_off + (size_t)tok) * g.heads + head;
+                    l2 = lse[li] * kLog2e;
+                    dl = delta[li];
+                }
+                s_tok[base + i] = tok;
+                s_meta[base + i] = meta;
+                s_lse[base + i] = l2;
+                s_delta[base + i] = dl;
             }
-            s_tok[s] = tok;
-            s_meta[s] = meta;
-            s_lse[s] = l2;
-            s_delta[s] = dl;
+        };
+        if (BIG) {
+            fill_table(0, r0, BM);
+            fill_table(BM, 0, BN);
+        } else {
+            fill_table(0, 0, npad);
         }
         __syncthreads();
+        // table index of the CTA's own rows / of the rows of streamed block blk
+        const int obase = BIG ? 0 : r0;
+        auto cbase = [&](int blk) { return BIG ? BM + (blk & 1) * BN : blk * BN; };
 
-        load_rows<D>(s_r1, own1, s_tok, r0, sample_off, g.ts, head, tid);
-        load_rows<D>(s_r2, own2, s_tok, r0, sample_off, ts_own2, head, tid);
-        load_rows<D>(s_c1, str1, s_tok, 0, sample_off, g.ts, head, tid);
-        load_rows<D>(s_c2, str2, s_tok, 0, sample_off, ts_str2, head, tid);
+        load_rows<D>(s_r1, own1, s_tok, obase, sample_off, g.ts, head, tid);
+        load_rows<D>(s_r2, own2, s_tok, obase, sample_off, ts_own2, head, tid);
+        load_rows<D>(s_c1, str1, s_tok, cbase(0), sample_off, g.ts, head, tid);
+        load_rows<D>(s_c2, str2, s_tok, cbase(0), sample_off, ts_str2, head, tid);
         cp_async_commit();
 
         uint32_t f1[kFragsInRegs<D> ? KS : 1][4], f2[kFragsInRegs<D> ? KS : 1][4];
@@ -224,16 +244,20 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
 #pragma unroll
             for (int e = 0; e < 4; ++e) acc2[i][e] = 0.f;
 
-        const int row_slot[2] = {r0 + warp * 16 + gq, r0 + warp * 16 + gq + 8};
-        const int meta_r[2] = {s_meta[row_slot[0]], s_meta[row_slot[1]]};
-        const float lse_r[2] = {s_lse[row_slot[0]], s_lse[row_slot[1]]};
-        const float del_r[2] = {s_delta[row_slot[0]], s_delta[row_slot[1]]};
+        const int row_tab[2] = {obase + warp * 16 + gq, obase + warp * 16 + gq + 8};
+        const int meta_r[2] = {s_meta[row_tab[0]], s_meta[row_tab[1]]};
+        const float lse_r[2] = {s_lse[row_tab[0]], s_lse[row_tab[1]]};
+        const float del_r[2] = {s_delta[row_tab[0]], s_delta[row_tab[1]]};
 
         for (int blk = 0; blk < nblk; ++blk) {
             const int stage = blk & 1;
             if (blk + 1 < nblk) {
-                load_rows<D>(s_c1 + (stage ^ 1) * TILE_BYTES, str1, s_tok, (blk + 1) * BN, sample_off, g.ts, head, tid);
-                load_rows<D>(s_c2 + (stage ^ 1) * TILE_BYTES, str2, s_tok, (blk + 1) * BN, sample_off, ts_str2, head, tid);
+                if (BIG) {   // the other stage's table is free: its block was finished before the barrier that ended the last step
+                    fill_table(cbase(blk + 1), (blk + 1) * BN, BN);
+                    __syncthreads();
+                }
+                load_rows<D>(s_c1 + (stage ^ 1) * TILE_BYTES, str1, s_tok, cbase(blk + 1), sample_off, g.ts, head, tid);
+                load_rows<D>(s_c2 + (stage ^ 1) * TILE_BYTES, str2, s_tok, cbase(blk + 1), sample_off, ts_str2, head, tid);
                 cp_async_commit();
                 cp_async_wait<1>();
             } else {
@@ -262,7 +286,7 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
             for (int nt = 0; nt < BN / 8; ++nt) {
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    const int col = blk * BN + nt * 8 + 2 * tq + (e & 1);
+                    const int col = cbase(blk) + nt * 8 + 2 * tq + (e & 1);
                     const int mc = s_meta[col];
                     const int mr = meta_r[e >> 1];
                     const bool ok = meta_label(mr) == meta_label(mc);
@@ -270,7 +294,8 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
                     const int bidx = KV ? (meta_code(mc) - meta_code(mr) + c0) : (meta_code(mr) - meta_code(mc) + c0);
                     const float l2 = KV ? s_lse[col] : lse_r[e >> 1];
                     const float dl = KV ? s_delta[col] : del_r[e >> 1];
-                    float p = fast_exp2(acc_s[nt][e] * g.scale_log2e + s_bias[bidx] - l2);
+                    const float bv = BIG ? (ok ? __ldg(bias + (size_t)bidx * g.heads + head) * kLog2e : 0.f) : s_bias[bidx];
+                    float p = fast_exp2(acc_s[nt][e] * g.scale_log2e + bv - l2);
                     p = ok ? p : 0.f;
                     const float ds = p * (acc_dp[nt][e] - dl);
                     acc_s[nt][e] = p;
@@ -315,7 +340,34 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
                             *reinterpret_cast<float2*>(stage + (gq + 8) * kStageStride + col) = make_float2(acc_dp[nt][2], acc_dp[nt][3]);
                         }
                         __syncwarp();
-                        if (g.w == 32 && r.ew == 32) {
+                        if (BIG) {
+                            if (r.ew == g.w && (g.w & 31) == 0) {
+                                // Complete along the width, side a multiple of 32: the warp's 16 rows are consecutive offsets
+                                // b_q of one window row a_q, and this half of the block is 32 consecutive offsets b_k of one
+                                // window row a_k.  All pairs with the same b_q - b_k share one table entry: sum each of the
+                                // 47 diagonals, then one global atomic per diagonal.
+                                const int a_q = slot0 / g.w, bq0 = slot0 - a_q * g.w;
+                                const int k0 = blk * BN + half * 32;
+                                const int a_k = k0 / g.w, bk0 = k0 - a_k * g.w;
+                                const int row_base = (a_q - a_k) * (2 * g.w - 1) + c0 + bq0 - bk0;
+                                float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+                                for (int rr = 0; rr < 16; ++rr) {
+                                    const bool first = rr <= lane;
+                                    const float val = stage[rr * kStageStride + (first ? 31 - lane + rr : rr - lane - 1)];
+                                    if (first) s0 += val; else s1 += val;
+                                }
+                                if (s0 != 0.f) atomicAdd(&dbias[(size_t)(row_base - 31 + lane) * g.heads + head], s0);
+                                if (lane < 15 && s1 != 0.f) atomicAdd(&dbias[(size_t)(row_base + 1 + lane) * g.heads + head], s1);
+                            } else {
+                                const int code_c = meta_code(s_meta[cbase(blk) + half * 32 + lane]);
+                                for (int rr = 0; rr < 16; ++rr) {
+                                    const int code_r = meta_code(s_meta[obase + warp * 16 + rr]) + c0;
+                                    const float v0 = stage[rr * kStageStride + lane];
+                                    if (v0 != 0.f) atomicAdd(&dbias[(size_t)(code_r - code_c) * g.heads + head], v0);
+                                }
+                            }
+                        } else if (g.w == 32 && r.ew == 32) {
                             // Full-width 32-wide window: the warp's 16 rows are consecutive offsets b_q of one window row
                             // a_q, and this half of the block is one window row a_k of keys with b_k = 0..31.  All pairs
                             // with the same b_q - b_k share one table entry: sum each of the 47 diagonals first, then one
@@ -335,9 +387,9 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
                             if (s0 != 0.f) atomicAdd(&s_dbias[row_base + bq0 - 31 + lane], s0);
                             if (lane < 15 && s1 != 0.f) atomicAdd(&s_dbias[row_base + bq0 + 1 + lane], s1);
                         } else {
-                            const int code_c = meta_code(s_meta[blk * BN + half * 32 + lane]);
+                            const int code_c = meta_code(s_meta[cbase(blk) + half * 32 + lane]);
                             for (int rr = 0; rr < 16; ++rr) {
-                                const int code_r = meta_code(s_meta[slot0 + rr]) + c0;
+                                const int code_r = meta_code(s_meta[obase + warp * 16 + rr]) + c0;
                                 const float v0 = stage[rr * kStageStride + lane];
                                 if (v0 != 0.f) atomicAdd(&s_dbias[code_r - code_c], v0);
                             }
@@ -360,8 +412,8 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
         stage_rows<D>(s_r1, acc1, scale, warp, gq, tq);
         if constexpr (KV) stage_rows<D>(s_r2, acc2, 1.f, warp, gq, tq);
         __syncthreads();
-        scatter_rows<D>(s_r1, out1, s_tok, r0, r.n, sample_off, g.ts, head, tid);
-        if constexpr (KV) scatter_rows<D>(s_r2, out2, s_tok, r0, r.n, sample_off, g.ts, head, tid);
+        scatter_rows<D>(s_r1, out1, s_tok + obase - r0, r0, r.n, sample_off, g.ts, head, tid);
+        if constexpr (KV) scatter_rows<D>(s_r2, out2, s_tok + obase - r0, r0, r.n, sample_off, g.ts, head, tid);
     }
 
     if (!KV) {
@@ -381,10 +433,11 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
             }
             __syncthreads();
         }
-        for (int i = tid; i < nbias; i += NTHREADS) {
-            float val = s_dbias[i];
-            if (val != 0.f) atomicAdd(&dbias[(size_t)i * g.heads + head], val);
-        }
+        if (!BIG)
+            for (int i = tid; i < nbias; i += NTHREADS) {
+                float val = s_dbias[i];
+                if (val != 0.f) atomicAdd(&dbias[(size_t)i * g.heads + head], val);
+            }
     }
 }
 
@@ -424,16 +477,16 @@ int acc_stride_for(const Geo& g) {
 size_t bwd_smem_bytes(const Geo& g, bool query_side) {
     int npad_max = ((g.nmax + BN - 1) / BN) * BN;
     int nbias = (2 * g.w - 1) * (2 * g.w - 1);
-    size_t head = (((size_t)npad_max * 16 + (size_t)nbias * 8 + 127) / 128) * 128;
+    size_t head = g.w > 32 ? (size_t)3 * BN * 16 : (((size_t)npad_max * 16 + (size_t)nbias * 8 + 127) / 128) * 128;
     size_t acc = query_side ? ((size_t)BM * acc_stride_for(g) + (size_t)BM * kStageStride) * sizeof(float) : 0;
     return head + 6 * (size_t)BN * g.d * 2 + acc;
 }
 
-template <int D, bool KV>
-cudaError_t launch_one(const Geo& g, const void* q, const void* k, const void* v, const void* d_o, const float* bias,
+template <int D, bool KV, bool BIG>
+cudaError_t launch_one_sized(const Geo& g, const void* q, const void* k, const void* v, const void* d_o, const float* bias,
                        const float* lse, const float* delta, void* out1, void* out2, float* dbias, int sm_count,
                        cudaStream_t stream) {
-    auto kern = swin_bwd_mma_kernel<D, KV>;
+    auto kern = swin_bwd_mma_kernel<D, KV, BIG>;
     const size_t smem = bwd_smem_bytes(g, !KV);
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
@@ -453,6 +506,14 @@ cudaError_t launch_one(const Geo& g, const void* q, const void* k, const void* v
         lse, delta, (__nv_bfloat16*)out1, (__nv_bfloat16*)out2, dbias, tiles, (int)cpg, KV ? 0 : acc_stride_for(g));
     count_launch(stream);
     return cudaGetLastError();
+}
+
+template <int D, bool KV>
+cudaError_t launch_one(const Geo& g, const void* q, const void* k, const void* v, const void* d_o, const float* bias,
+                       const float* lse, const float* delta, void* out1, void* out2, float* dbias, int sm_count,
+                       cudaStream_t stream) {
+    return g.w > 32 ? launch_one_sized<D, KV, true>(g, q, k, v, d_o, bias, lse, delta, out1, out2, dbias, sm_count, stream)
+                    : launch_one_sized<D, KV, false>(g, q, k, v, d_o, bias, lse, delta, out1, out2, dbias, sm_count, stream);
 }
 
 }  // namespace

@@ -35,7 +35,10 @@ __device__ __forceinline__ void load_rows(unsigned char* s_tile, const __nv_bflo
     }
 }
 
-template <int D>
+// BIG = windows of more than 1024 tokens (window sides 33 .. 128): the slot tables of a whole window and the head's
+// bias table no longer fit shared memory, so the tables cover the CTA's 64 query rows plus the key block in flight
+// (two stages) and the bias is read from the caller's table in global memory.
+template <int D, bool BIG>
 __global__ void __launch_bounds__(NTHREADS)
 swin_fwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                     const __nv_bfloat16* __restrict__ v, const float* __restrict__ bias,
@@ -59,10 +62,12 @@ swin_fwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
     const int nbias = (2 * g.w - 1) * (2 * g.w - 1);
     const int npad_max = ((g.nmax + BN - 1) / BN) * BN;
 
+    // table layout: small windows [npad_max] slots of the window; BIG: [0, 64) the query rows, [64, 192) two key blocks
+    const int ntab = BIG ? 3 * BN : npad_max;
     int* s_tok = reinterpret_cast<int*>(smem);
-    int* s_meta = s_tok + npad_max;
-    float* s_bias = reinterpret_cast<float*>(s_meta + npad_max);
-    unsigned char* s_q = smem + (((size_t)npad_max * 8 + (size_t)nbias * 4 + 127) / 128) * 128;
+    int* s_meta = s_tok + ntab;
+    float* s_bias = reinterpret_cast<float*>(s_meta + ntab);
+    unsigned char* s_q = smem + (((size_t)ntab * 8 + (BIG ? 0 : (size_t)nbias * 4) + 127) / 128) * 128;
     unsigned char* s_k = s_q + TILE_BYTES;           // two stages
     unsigned char* s_v = s_k + 2 * TILE_BYTES;       // two stages
 
@@ -70,18 +75,35 @@ swin_fwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
     const int gq = lane >> 2, tq = lane & 3;
     const size_t sample_off = (size_t)b * g.H * g.W;
 
-    for (int s = tid; s < npad; s += NTHREADS) {
-        int meta = 0xff << 16, tok = -1;
-        if (s < r.n) tok = slot_token(g, r, s, meta);
-        s_tok[s] = tok;
-        s_meta[s] = meta;
+    // fills 64 table entries at `base` with the window's slots first .. first + 63
+    auto fill_table = [&](int base, int first) {
+        if (tid < BN) {
+            int meta = 0xff << 16, tok = -1;
+            if (first + tid < r.n) tok = slot_token(g, r, first + tid, meta);
+            s_tok[base + tid] = tok;
+            s_meta[base + tid] = meta;
+        }
+    };
+    if (BIG) {
+        fill_table(0, q0);
+        fill_table(BN, 0);
+    } else {
+        for (int s = tid; s < npad; s += NTHREADS) {
+            int meta = 0xff << 16, tok = -1;
+            if (s < r.n) tok = slot_token(g, r, s, meta);
+            s_tok[s] = tok;
+            s_meta[s] = meta;
+        }
+        for (int i = tid; i < nbias; i += NTHREADS) s_bias[i] = bias[(size_t)i * g.heads + head] * kLog2e;
     }
-    for (int i = tid; i < nbias; i += NTHREADS) s_bias[i] = bias[(size_t)i * g.heads + head] * kLog2e;
     __syncthreads();
+    // table index of query row `row` of this CTA / of row `row` of key block kb
+    const int qbase = BIG ? 0 : q0;
+    auto kbase = [&](int kb) { return BIG ? BN + (kb & 1) * BN : kb * BN; };
 
-    load_rows<D>(s_q, q, s_tok, q0, sample_off, g.ts, head, tid);
-    load_rows<D>(s_k, k, s_tok, 0, sample_off, g.ts, head, tid);
-    load_rows<D>(s_v, v, s_tok, 0, sample_off, g.ts, head, tid);
+    load_rows<D>(s_q, q, s_tok, qbase, sample_off, g.ts, head, tid);
+    load_rows<D>(s_k, k, s_tok, kbase(0), sample_off, g.ts, head, tid);
+    load_rows<D>(s_v, v, s_tok, kbase(0), sample_off, g.ts, head, tid);
     cp_async_commit();
 
     uint32_t qf[KS][4];
@@ -93,14 +115,18 @@ swin_fwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
     float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
 
     const int row_slot[2] = {q0 + warp * 16 + gq, q0 + warp * 16 + gq + 8};
-    const int meta_r[2] = {s_meta[row_slot[0]], s_meta[row_slot[1]]};
+    const int meta_r[2] = {s_meta[qbase + warp * 16 + gq], s_meta[qbase + warp * 16 + gq + 8]};
     const int c0 = (g.w - 1) * 2 * g.w;
 
     for (int kb = 0; kb < nkb; ++kb) {
         const int stage = kb & 1;
         if (kb + 1 < nkb) {
-            load_rows<D>(s_k + (stage ^ 1) * TILE_BYTES, k, s_tok, (kb + 1) * BN, sample_off, g.ts, head, tid);
-            load_rows<D>(s_v + (stage ^ 1) * TILE_BYTES, v, s_tok, (kb + 1) * BN, sample_off, g.ts, head, tid);
+            if (BIG) {       // the other stage's table is free: its block was finished before the barrier that ended the last step
+                fill_table(kbase(kb + 1), (kb + 1) * BN);
+                __syncthreads();
+            }
+            load_rows<D>(s_k + (stage ^ 1) * TILE_BYTES, k, s_tok, kbase(kb + 1), sample_off, g.ts, head, tid);
+            load_rows<D>(s_v + (stage ^ 1) * TILE_BYTES, v, s_tok, kbase(kb + 1), sample_off, g.ts, head, tid);
             cp_async_commit();
             cp_async_wait<1>();
         } else {
@@ -140,10 +166,12 @@ swin_fwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
         for (int nt = 0; nt < BN / 8; ++nt) {
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                int mj = s_meta[kb * BN + nt * 8 + 2 * tq + (e & 1)];
+                int mj = s_meta[kbase(kb) + nt * 8 + 2 * tq + (e & 1)];
                 int mi = meta_r[e >> 1];
                 bool ok = meta_label(mi) == meta_label(mj);
-                float sc = acc_s[nt][e] * g.scale_log2e + s_bias[meta_code(mi) - meta_code(mj) + c0];
+                const int bidx = meta_code(mi) - meta_code(mj) + c0;
+                const float bv = BIG ? (ok ? __ldg(bias + (size_t)bidx * g.heads + head) * kLog2e : 0.f) : s_bias[bidx];
+                float sc = acc_s[nt][e] * g.scale_log2e + bv;
                 sc = ok ? sc : -INFINITY;
                 acc_s[nt][e] = sc;
                 mx[e >> 1] = fmaxf(mx[e >> 1], sc);
@@ -216,7 +244,7 @@ swin_fwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
         for (int h = 0; h < 2; ++h) {
             int slot = row_slot[h];
             if (slot < r.n)
-                lse[(sample_off + (size_t)s_tok[slot]) * g.heads + head] = (m_run[h] + log2f(l_run[h])) * kLn2;
+                lse[(sample_off + (size_t)s_tok[slot - q0 + qbase]) * g.heads + head] = (m_run[h] + log2f(l_run[h])) * kLn2;
         }
     }
     __syncthreads();
@@ -226,7 +254,7 @@ swin_fwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
         int slot = q0 + row;
         if (slot < r.n) {
             uint4 val = *reinterpret_cast<const uint4*>(s_q + tile_off<D>(row, chunk));
-            *reinterpret_cast<uint4*>(o + ((sample_off + (size_t)s_tok[slot]) * g.heads + head) * D + chunk * 8) = val;
+            *reinterpret_cast<uint4*>(o + ((sample_off + (size_t)s_tok[qbase + row]) * g.heads + head) * D + chunk * 8) = val;
         }
     }
 }
@@ -234,7 +262,7 @@ swin_fwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
 size_t fwd_smem_bytes(const Geo& g) {
     int npad_max = ((g.nmax + BN - 1) / BN) * BN;
     int nbias = (2 * g.w - 1) * (2 * g.w - 1);
-    size_t head = (((size_t)npad_max * 8 + (size_t)nbias * 4 + 127) / 128) * 128;
+    size_t head = g.w > 32 ? (size_t)3 * BN * 8 : (((size_t)npad_max * 8 + (size_t)nbias * 4 + 127) / 128) * 128;
     return head + 5 * (size_t)BN * g.d * 2;
 }
 
@@ -245,7 +273,8 @@ cudaError_t TERRA_ELEM_FN(launch_fwd_mma)(const Geo& g, const void* q, const voi
     const int qtiles = (g.nmax + BM - 1) / BM;
     const long long items = (long long)g.B * g.Mh * g.Mw * g.heads * qtiles;
     const size_t smem = fwd_smem_bytes(g);
-    auto kern = (g.d == 32) ? swin_fwd_mma_kernel<32> : (g.d == 64) ? swin_fwd_mma_kernel<64> : swin_fwd_mma_kernel<128>;
+    auto kern = g.w > 32 ? ((g.d == 32) ? swin_fwd_mma_kernel<32, true> : (g.d == 64) ? swin_fwd_mma_kernel<64, true> : swin_fwd_mma_kernel<128, true>)
+                         : ((g.d == 32) ? swin_fwd_mma_kernel<32, false> : (g.d == 64) ? swin_fwd_mma_kernel<64, false> : swin_fwd_mma_kernel<128, false>);
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     prof_begin("swin_fwd_mma_kernel", stream);

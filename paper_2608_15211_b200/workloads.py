@@ -61,6 +61,9 @@ CONFIGS = {
     "tv_small": SwinConfig("tv_small", 1, 288, 544, 8, 128, 8, 4, 4, index=6),
     "tv_medium": SwinConfig("tv_medium", 1, 288, 544, 32, 128, 8, 4, 4, index=7),
     "tv_large": SwinConfig("tv_large", 1, 288, 544, 64, 128, 32, 16, 16, index=8),
+    # The window-assignment study's largest window (Section VII-E: small model, w = 128; the 2041 x 4320 field at
+    # patch 4 and sampling factor 2 padded to a 2 x 5 grid of 128 x 128 windows, i.e. 256 x 640 tokens)
+    "tv_small_w128": SwinConfig("tv_small_w128", 1, 256, 640, 8, 128, 128, 64, 64, index=9),
 }
 
 TENSOR_INDEX = {"q": 0, "k": 1, "v": 2, "do": 3, "bias": 4}

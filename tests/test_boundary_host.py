@@ -71,7 +71,7 @@ def test_bad_descriptor_is_rejected_on_the_host(lib, kw, status):
     assert e.value.status == status
 
 
-@pytest.mark.parametrize("kw", [dict(head_dim=48), dict(head_dim=256), dict(window=33)])
+@pytest.mark.parametrize("kw", [dict(head_dim=48), dict(head_dim=256), dict(window=129)])
 def test_unsupported_shapes(lib, kw):
     with pytest.raises(terra.TerraError) as e:
         terra.terra_swin_workspace_bytes(_desc(**kw), True)
