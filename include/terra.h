@@ -206,6 +206,25 @@ int terra_profile_count(void);
 int terra_profile_get(int index, char* name, int name_bytes, float* ms);
 
 /*
+ * Complete-window ("padded") mode (Section IV-B and Eq. 3: the paper pads the grid so that every window is complete,
+ * and the padded tokens are ordinary tokens of the Transformer blocks).  The attention entry points truncate the last
+ * window row / column of a grid that the window side does not divide; a caller who wants the paper's padded
+ * execution instead keeps its activations on the padded token grid H_pad x W_pad (multiples of the window side; for
+ * the fixed assignment of Eq. 3 multiples of w m and w n) and describes THAT grid to the attention calls.  These two
+ * calls move a tensor between the two grids:
+ *   terra_pad_grid   y [B, H_pad, W_pad, token_bytes] = x [B, H, W, token_bytes] in the top-left corner, zeros elsewhere
+ *   terra_crop_grid  x [B, H, W, token_bytes] = the top-left corner of y (the backward of the padding, and the way
+ *                    results leave the padded grid)
+ * token_bytes = bytes per token (for [.., heads, head_dim] bf16: heads * head_dim * 2; for lse: heads * 4), a multiple of 4; device
+ * pointers, 16-byte aligned, no overlap.  H_pad >= H, W_pad >= W.  Errors: TERRA_ERR_INVALID_ARG,
+ * TERRA_ERR_ALIGNMENT, TERRA_ERR_CUDA.
+ */
+int terra_pad_grid(const void* x, void* y, int32_t B, int32_t H, int32_t W, int32_t H_pad, int32_t W_pad,
+                   int64_t token_bytes, void* stream);
+int terra_crop_grid(const void* y, void* x, int32_t B, int32_t H, int32_t W, int32_t H_pad, int32_t W_pad,
+                    int64_t token_bytes, void* stream);
+
+/*
  * Window ownership across window-parallel (WP) ranks (Section V-A).  Host-only integer helpers; they launch
  * nothing and touch no device.  This library runs one GPU; these state which windows a rank of a WP group
  * would own, so that a caller sharding windows over several processes uses the paper's rule.

@@ -18,7 +18,8 @@ TERRA_OK = 0
 EXPORTS = ("terra_route_sizes", "terra_window_route", "terra_swin_workspace_bytes", "terra_swin_attn_fwd",
            "terra_swin_attn_fwd_noalloc", "terra_swin_attn_bwd", "terra_swin_check", "terra_strerror", "terra_last_cuda_error",
            "terra_launch_count", "terra_selftest_bounded_wait", "terra_profile_enable", "terra_profile_count", "terra_profile_get",
-           "terra_fixed_assignment_padding", "terra_ragged_window_range", "terra_swin_attn_fwd_packed", "terra_swin_attn_bwd_packed")
+           "terra_fixed_assignment_padding", "terra_ragged_window_range", "terra_swin_attn_fwd_packed", "terra_swin_attn_bwd_packed",
+           "terra_pad_grid", "terra_crop_grid")
 
 
 class TerraError(RuntimeError):
@@ -76,6 +77,9 @@ def load_library(path: str | None = None) -> ctypes.CDLL:
     lib.terra_fixed_assignment_padding.restype = ctypes.c_int
     lib.terra_ragged_window_range.argtypes = [ctypes.c_int64, ctypes.c_int32, ctypes.c_int32, i64p, i64p]
     lib.terra_ragged_window_range.restype = ctypes.c_int
+    for n in ("terra_pad_grid", "terra_crop_grid"):
+        getattr(lib, n).argtypes = [vp, vp] + [ctypes.c_int32] * 5 + [ctypes.c_int64, vp]
+        getattr(lib, n).restype = ctypes.c_int
     if path is None:
         _lib = lib
     return lib
@@ -291,3 +295,26 @@ def terra_swin_attn_bwd_packed(desc, qkv, bias_table, o, lse, d_o, dqkv=None, db
     _check(load_library().terra_swin_attn_bwd_packed(ctypes.byref(desc), _ptr(qkv), _ptr(bias_table), _ptr(o), _ptr(lse),
                                                      _ptr(d_o), _ptr(dqkv), _ptr(dbias), _ptr(workspace), ws_bytes, _stream()))
     return dqkv, dbias
+
+
+def padded_extent(extent: int, window: int) -> int:
+    """The extent rounded up to complete windows."""
+    return -(-extent // window) * window
+
+
+def terra_pad_grid(x, H_pad: int, W_pad: int):
+    """x [B, H, W, ...] -> zero-padded [B, H_pad, W_pad, ...] (complete-window mode, see include/terra.h)."""
+    B, H, W = x.shape[:3]
+    token_bytes = x[0, 0, 0].numel() * x.element_size()
+    y = torch.empty((B, H_pad, W_pad) + tuple(x.shape[3:]), dtype=x.dtype, device=x.device)
+    _check(load_library().terra_pad_grid(_ptr(x), _ptr(y), B, H, W, H_pad, W_pad, token_bytes, _stream()))
+    return y
+
+
+def terra_crop_grid(y, H: int, W: int):
+    """y [B, H_pad, W_pad, ...] -> its top-left [B, H, W, ...] corner as a dense tensor."""
+    B, H_pad, W_pad = y.shape[:3]
+    token_bytes = y[0, 0, 0].numel() * y.element_size()
+    x = torch.empty((B, H, W) + tuple(y.shape[3:]), dtype=y.dtype, device=y.device)
+    _check(load_library().terra_crop_grid(_ptr(y), _ptr(x), B, H, W, H_pad, W_pad, token_bytes, _stream()))
+    return x
