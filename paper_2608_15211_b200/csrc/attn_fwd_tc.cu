@@ -19,6 +19,10 @@
 // exact maximum over the keys the row may see.
 // Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, all roles leave their loops,
 // TMEM is released and the host reads the device status word.
+#include <cuda.h>
+#include <cstdlib>
+#include <cstring>
+
 #include "swin_common.cuh"
 #include "swin_kernels.h"
 #include "tc_common.cuh"
@@ -344,11 +348,21 @@ __device__ __forceinline__ float softmax_row(uint32_t t_s, int npad, int nvalid,
 // W16 = the window side is 16: full unmasked windows take the immediate-offset table addressing, every other
 // window of that grid (shift-mask labels, truncated at the grid's edge) the label-compare path, which also
 // covers key slots without a token (their label never matches).  Two softmax paths per kernel either way.
-template <bool W16>
+// Tensor maps of the TMA variant: q, k, v as 2-D tensors [tokens][channels of the tensor] with a box of one head's 32
+// channels x one window row of tokens (16, or 8 in the grid's last window column), 64-byte swizzle.
+struct FwdMaps {
+    CUtensorMap q16, k16, v16, q8, k8, v8;
+};
+
+// TMA = the window rows are fetched by tiled tensor copies (one per window row and tensor, issued by the lanes of
+// ONE producer warp, the head's bias table by one bulk copy) instead of 16-byte cp.async copies from three loader
+// warps.  For grids of 16-wide windows whose every window row is one run of consecutive tokens in memory.
+template <bool W16, bool TMA>
 __global__ void __launch_bounds__(kThreads, 1)
 swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                    const __nv_bfloat16* __restrict__ v, const float* __restrict__ bias_prep,
-                   __nv_bfloat16* __restrict__ o, float* __restrict__ lse, long long n_items) {
+                   __nv_bfloat16* __restrict__ o, float* __restrict__ lse, long long n_items,
+                   const __grid_constant__ FwdMaps maps) {
     extern __shared__ __align__(1024) unsigned char smem[];
     const uint32_t smem0 = smem_u32(smem);
     const uint32_t bar0 = smem0 + kStages * kStageBytes;
@@ -369,7 +383,7 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
 
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(bar_full(s), kLoaderThreads);
+            mbar_init(bar_full(s), TMA ? 32 : kLoaderThreads);
             mbar_init(bar_empty(s), 1 + 128);      // the issuer's commit + the second softmax warpgroup (see its loop)
         }
         for (int t = 0; t < 2; ++t) {
@@ -404,7 +418,67 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
     if (warp >= kMmaWarp) {
     // warpgroup 2 (MMA issuer + loaders) gives registers back: one instruction for the whole warpgroup
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kRegsOther));
-    if (warp >= kLoaderWarp0) {
+    if (TMA && warp >= kLoaderWarp0) {
+        // ------------------------------------------------------------------ producer warp (TMA)
+        if (warp == kLoaderWarp0) {
+            int kuse = 0;
+            ItemCursor cur_it = cursor_init(blockIdx.x, gridDim.x, g.heads, g.Mw, g.Mh);
+            for (long long it = blockIdx.x; it < n_items; it += gridDim.x, ++kuse, cursor_advance(cur_it, g.heads, g.Mw, g.Mh)) {
+                const int s = kuse % kStages;
+                if (!mbar_wait_all(bar_empty(s), ((kuse / kStages) & 1) ^ 1, cta_abort)) break;
+                const Item x = make_item(g, cur_it);
+                unsigned char* st = smem + s * kStageBytes;
+                const uint32_t st_a = smem0 + s * kStageBytes;
+                const int ew = x.r.ew;                       // 16, or 8 in the last window column
+                // lane a < eh: the three tensors' copies of window row a (ew consecutive tokens, this head's 64 bytes each)
+                if (lane < x.r.eh) {
+                    int u = x.r.wr * g.w + lane + g.sh;
+                    if (u >= g.H) u -= g.H;
+                    int v0 = x.r.wc * g.w + g.sw;
+                    if (v0 >= g.W) v0 -= g.W;
+                    const int y = (int)((size_t)x.b * HW + (size_t)u * g.W + v0), xc = x.head * kD;
+                    const uint32_t dst = st_a + (uint32_t)(lane * ew * kRowBytes);
+                    if (ew == 16) {
+                        tma_load_2d(dst + kOffQ, &maps.q16, xc, y, bar_full(s));
+                        tma_load_2d(dst + kOffK, &maps.k16, xc, y, bar_full(s));
+                        tma_load_2d(dst + kOffV, &maps.v16, xc, y, bar_full(s));
+                    } else {
+                        tma_load_2d(dst + kOffQ, &maps.q8, xc, y, bar_full(s));
+                        tma_load_2d(dst + kOffK, &maps.k8, xc, y, bar_full(s));
+                        tma_load_2d(dst + kOffV, &maps.v8, xc, y, bar_full(s));
+                    }
+                }
+                if (lane == 31) bulk_load(st_a + kOffBias, bias_prep + (size_t)x.head * kFwdBiasFloats, kFwdBiasFloats * 4, bar_full(s));
+                // slot tables: 8 consecutive slots per lane
+                {
+                    int a_s = (8 * lane) / ew, b_s = 8 * lane - a_s * ew;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int slot = 8 * lane + i;
+                        int code = 0, label = 0xff, tok = -1, kc = 4 * (2 * c0 + 1);
+                        if (slot < x.r.n) {
+                            tok = offset_token_tc(g, x.r, a_s, b_s, code, label);
+                            kc = 4 * (c0 - code);
+                        }
+                        reinterpret_cast<int*>(st + kOffKc)[slot] = kc;
+                        reinterpret_cast<int*>(st + kOffKlab)[slot] = label;
+                        reinterpret_cast<int*>(st + kOffRowMeta)[slot] = code | (label << 16);
+                        reinterpret_cast<int*>(st + kOffRowTok)[slot] = tok;
+                        if (++b_s == ew) { b_s = 0; ++a_s; }
+                    }
+                }
+                // operand rows between the window's end and the next multiple of 16 must read as zeros
+                for (int i = lane; i < (x.npad - x.r.n) * 12; i += 32) {
+                    const int row = x.r.n + i / 12, piece = i % 12;
+                    *reinterpret_cast<uint4*>(st + (piece >> 2) * (kMaxSlots * kRowBytes) + tile_off<kD>(row, piece & 3)) = make_uint4(0u, 0u, 0u, 0u);
+                }
+                fence_proxy_async();
+                // 32 arrivals complete the phase once the copies' bytes have landed as well
+                if (lane == 0) mbar_arrive_expect_tx(bar_full(s), (uint32_t)(3 * x.r.n * kRowBytes + kFwdBiasFloats * 4));
+                else mbar_arrive(bar_full(s));
+            }
+        }
+    } else if (warp >= kLoaderWarp0) {
         // ------------------------------------------------------------------ loaders
         const int lt = (warp - kLoaderWarp0) * 32 + lane;
         int kuse = 0, pending_s = -1;
@@ -727,6 +801,51 @@ swin_fwd_bias_prep_kernel(const float* __restrict__ bias, float* __restrict__ pr
 
 bool fwd_tc_supported(const Geo& g) { return g.d == 32 && g.nmax <= kMaxSlots && g.w <= 16; }
 
+namespace {
+
+// The TMA variant fetches a window row with one tiled copy: every window row must be one run of consecutive tokens
+// (the longitude roll may not cut through a window) of 16 tokens, or 8 in the last window column.
+bool fwd_tma_shape(const Geo& g) {
+    if (g.w != 16 || g.d != 32 || g.W < 16 || (g.W % 16 != 0 && g.W % 16 != 8)) return false;
+    if ((long long)g.B * g.H * g.W >= 0x7fffffffLL) return false;       // token coordinate of the tensor map is int32
+    for (int wc = 0; wc < g.Mw; ++wc) {
+        const int ew = g.W - wc * 16 < 16 ? g.W - wc * 16 : 16;
+        const int v0 = (wc * 16 + g.sw) % g.W;
+        if (v0 + ew > g.W) return false;
+    }
+    return true;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver's encoder, looked up through the runtime (the library does not link against the driver library).
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess || qres != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+// [tokens][channels] bf16 with a token stride of g.ts elements; box = 32 channels x `box_tokens` tokens, 64-byte swizzle
+bool make_map(CUtensorMap* m, const Geo& g, const void* base, int box_tokens) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)g.heads * g.d, (cuuint64_t)g.B * g.H * g.W};
+    const cuuint64_t strides[1] = {(cuuint64_t)g.ts * 2};
+    const cuuint32_t box[2] = {32u, (cuuint32_t)box_tokens};
+    const cuuint32_t estr[2] = {1u, 1u};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
 size_t fwd_tc_workspace_bytes(const Geo& g) { return (size_t)g.heads * kFwdBiasFloats * sizeof(float); }
 
 cudaError_t launch_fwd_tc(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
@@ -737,17 +856,18 @@ cudaError_t launch_fwd_tc(const Geo& g, const void* q, const void* k, const void
     count_launch(stream);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(g.w == 16 ? swin_fwd_tc_kernel<true> : swin_fwd_tc_kernel<false>,
-                             cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    FwdMaps maps;
+    std::memset(&maps, 0, sizeof maps);
+    static const bool tma_off = [] { const char* e_ = std::getenv("TERRA_NO_TMA"); return e_ && e_[0] == '1'; }();
+    const bool tma = !tma_off && fwd_tma_shape(g) && make_map(&maps.q16, g, q, 16) && make_map(&maps.k16, g, k, 16) && make_map(&maps.v16, g, v, 16) &&
+                     make_map(&maps.q8, g, q, 8) && make_map(&maps.k8, g, k, 8) && make_map(&maps.v8, g, v, 8);
+    auto kern = tma ? swin_fwd_tc_kernel<true, true> : (g.w == 16 ? swin_fwd_tc_kernel<true, false> : swin_fwd_tc_kernel<false, false>);
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
     const unsigned grid = (unsigned)(items < sm_count ? items : sm_count);
     prof_begin("swin_fwd_tc_kernel", stream);
-    if (g.w == 16)
-        swin_fwd_tc_kernel<true><<<grid, kThreads, kSmemBytes, stream>>>(g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k,
-                                                                         (const __nv_bfloat16*)v, prep, (__nv_bfloat16*)o, lse, items);
-    else
-        swin_fwd_tc_kernel<false><<<grid, kThreads, kSmemBytes, stream>>>(g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k,
-                                                                          (const __nv_bfloat16*)v, prep, (__nv_bfloat16*)o, lse, items);
+    kern<<<grid, kThreads, kSmemBytes, stream>>>(g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, prep,
+                                                 (__nv_bfloat16*)o, lse, items, maps);
     count_launch(stream);
     return cudaGetLastError();
 }

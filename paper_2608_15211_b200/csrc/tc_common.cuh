@@ -106,6 +106,26 @@ __device__ __forceinline__ bool mbar_wait_all_relaxed(uint32_t bar, uint32_t par
     return __all_sync(0xffffffffu, mbar_wait<128>(bar, parity, cta_abort));
 }
 
+// ---- TMA: tiled tensor copies and plain bulk copies, global -> shared, completing on an mbarrier ---------------
+// 2-D tiled load: the box at coordinates (x, y) of the tensor map (a kernel parameter: its generic address) lands at
+// `dst` (128-byte aligned; the map's swizzle mode is applied from the address bits); the bytes are counted on `bar`.
+// x times the element size must be a multiple of 16 bytes.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const void* tmap, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n"
+        ::"r"(dst), "l"(tmap), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+// contiguous copy of `bytes` (a multiple of 16; both addresses 16-byte aligned)
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+// one arrival that also announces `tx` bytes of asynchronous copies to the barrier's current phase
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t tx) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(tx) : "memory");
+}
+
 // ---- tcgen05: TMEM allocation -----------------------------------------------------------------------
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_dst), "r"(ncols) : "memory");

@@ -26,6 +26,10 @@ EDGE = [
     ("w12_three_blocks", 2, 30, 40, 3, 32, 12, 6, 6, 0, 1),     # 144-token windows: two key tiles, an odd number of query blocks
     ("w16_wrap_and_rem", 1, 40, 48, 2, 32, 16, 8, 8, 0, 1),      # full, masked (latitude wrap) and truncated 16-wide windows
     ("w8_nonperiodic", 2, 24, 40, 2, 32, 8, 4, 4, 0, 0),         # 64-token windows, masks on both axes, several items per CTA
+    # 16-wide windows whose rows are runs of consecutive tokens: the forward fetches them with tiled TMA copies
+    ("tma_rows_wrap_lat", 2, 30, 56, 3, 32, 16, 8, 8, 0, 1),     # last column 8 wide, last row 14 high, latitude wrap + mask
+    ("tma_nonperiodic", 1, 46, 64, 2, 32, 16, 8, 16, 0, 0),      # masks on both axes
+    ("tma_noshift", 1, 32, 40, 2, 32, 16, 0, 0, 0, 1),
 ]
 
 
