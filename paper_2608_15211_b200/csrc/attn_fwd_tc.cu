@@ -801,11 +801,9 @@ swin_fwd_bias_prep_kernel(const float* __restrict__ bias, float* __restrict__ pr
 
 bool fwd_tc_supported(const Geo& g) { return g.d == 32 && g.nmax <= kMaxSlots && g.w <= 16; }
 
-namespace {
-
-// The TMA variant fetches a window row with one tiled copy: every window row must be one run of consecutive tokens
+// The TMA variants fetch a window row with one tiled copy: every window row must be one run of consecutive tokens
 // (the longitude roll may not cut through a window) of 16 tokens, or 8 in the last window column.
-bool fwd_tma_shape(const Geo& g) {
+bool tma_row_shape(const Geo& g) {
     if (g.w != 16 || g.d != 32 || g.W < 16 || (g.W % 16 != 0 && g.W % 16 != 8)) return false;
     if ((long long)g.B * g.H * g.W >= 0x7fffffffLL) return false;       // token coordinate of the tensor map is int32
     for (int wc = 0; wc < g.Mw; ++wc) {
@@ -815,6 +813,8 @@ bool fwd_tma_shape(const Geo& g) {
     }
     return true;
 }
+
+namespace {
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -832,19 +832,21 @@ EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-// [tokens][channels] bf16 with a token stride of g.ts elements; box = 32 channels x `box_tokens` tokens, 64-byte swizzle
-bool make_map(CUtensorMap* m, const Geo& g, const void* base, int box_tokens) {
+}  // namespace
+
+// [tokens][channels] bf16 with a token stride of `token_stride` elements; box = 32 channels x `box_tokens` tokens,
+// 64-byte swizzle.  `map` points to a CUtensorMap.
+bool make_row_map(void* map, const Geo& g, const void* base, int token_stride, int box_tokens) {
+    CUtensorMap* m = reinterpret_cast<CUtensorMap*>(map);
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)g.heads * g.d, (cuuint64_t)g.B * g.H * g.W};
-    const cuuint64_t strides[1] = {(cuuint64_t)g.ts * 2};
+    const cuuint64_t strides[1] = {(cuuint64_t)token_stride * 2};
     const cuuint32_t box[2] = {32u, (cuuint32_t)box_tokens};
     const cuuint32_t estr[2] = {1u, 1u};
     return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
-
-}  // namespace
 
 size_t fwd_tc_workspace_bytes(const Geo& g) { return (size_t)g.heads * kFwdBiasFloats * sizeof(float); }
 
@@ -859,8 +861,9 @@ cudaError_t launch_fwd_tc(const Geo& g, const void* q, const void* k, const void
     FwdMaps maps;
     std::memset(&maps, 0, sizeof maps);
     static const bool tma_off = [] { const char* e_ = std::getenv("TERRA_NO_TMA"); return e_ && e_[0] == '1'; }();
-    const bool tma = !tma_off && fwd_tma_shape(g) && make_map(&maps.q16, g, q, 16) && make_map(&maps.k16, g, k, 16) && make_map(&maps.v16, g, v, 16) &&
-                     make_map(&maps.q8, g, q, 8) && make_map(&maps.k8, g, k, 8) && make_map(&maps.v8, g, v, 8);
+    const bool tma = !tma_off && tma_row_shape(g) && make_row_map(&maps.q16, g, q, g.ts, 16) && make_row_map(&maps.k16, g, k, g.ts, 16) &&
+                     make_row_map(&maps.v16, g, v, g.ts, 16) && make_row_map(&maps.q8, g, q, g.ts, 8) && make_row_map(&maps.k8, g, k, g.ts, 8) &&
+                     make_row_map(&maps.v8, g, v, g.ts, 8);
     auto kern = tma ? swin_fwd_tc_kernel<true, true> : (g.w == 16 ? swin_fwd_tc_kernel<true, false> : swin_fwd_tc_kernel<false, false>);
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;

@@ -36,6 +36,11 @@ cudaError_t launch_fwd_tc(const Geo& g, const void* q, const void* k, const void
 // synchronises the stream, reads and clears the device-side "a bounded wait expired" word
 cudaError_t read_tc_status(int* timed_out, cudaStream_t stream);
 
+// TMA variants of the two kernels above (grids of 16-wide windows whose window rows are runs of consecutive tokens):
+// the shape test, and the encoder of a [tokens][channels] tensor map with a box of 32 channels x box_tokens tokens
+bool tma_row_shape(const Geo& g);
+bool make_row_map(void* cu_tensor_map, const Geo& g, const void* base, int token_stride, int box_tokens);
+
 // tcgen05 forward path for head dim 64 and windows of up to 1024 tokens (keys streamed in chunks, two passes)
 bool fwd_tc64_supported(const Geo& g);
 size_t fwd_tc64_workspace_bytes(const Geo& g);
