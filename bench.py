@@ -179,8 +179,8 @@ def run_reference(args, cfg):
 # proportion to the item count, so a full launch is this figure times its items.  None = not captured.
 TRAFFIC_SOURCE = "stored ncu capture (profiles/swin_*_cfg3_rows254.md), scaled by the item count; not measured in this run"
 NCU_DRAM_BYTES_PER_ITEM = {
-    "swin_fwd_tc_kernel": 63620,
-    "swin_bwd_fused_kernel": 112255,
+    "swin_fwd_tc_kernel": 63575,
+    "swin_bwd_fused_kernel": 112166,
 }
 
 
