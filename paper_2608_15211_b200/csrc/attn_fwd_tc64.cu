@@ -20,6 +20,10 @@
 // in place by bf16 P (64 columns); the O accumulator (64 + 16 columns) at +128.
 // Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, all roles leave their loops, TMEM is
 // released and the host reads the device status word.  Every role follows every ring item by item.
+#include <cuda.h>
+#include <cstdlib>
+#include <cstring>
+
 #include "swin_common.cuh"
 #include "swin_kernels.h"
 #include "tc_common.cuh"
@@ -36,28 +40,38 @@ constexpr int kMmaWarp = 8;
 constexpr int kLoaderWarp0 = 9;
 constexpr int kLoaderThreads = 96;
 constexpr int kThreads = 384;
-constexpr int kRegsLaunch = 168, kRegsSoftmax = 216, kRegsOther = 64;
+constexpr int kRegsLaunch = 168, kRegsSoftmax = 216, kRegsOther = 72;
 static_assert(2 * (kRegsSoftmax - kRegsLaunch) <= (kRegsLaunch - kRegsOther), "register hand-over does not balance");
 
-constexpr int kD = 64;
-constexpr int kHalfBytes = 64;                        // one 32-column half of a row
+constexpr int kPartBytes = 64;                        // one 32-column part of a row
 constexpr int kQRows = 256, kChunk = 128;
-constexpr int kQStages = 2, kSlots = 3;
-constexpr int kQHalf = kQRows * kHalfBytes;           // 16384
-constexpr int kQStageBytes = 2 * kQHalf;              // Q lo | Q hi
-constexpr int kKHalf = kChunk * kHalfBytes;           // 8192
-constexpr int kOffKlo = 0, kOffKhi = kKHalf, kOffVlo = 2 * kKHalf, kOffVhi = 3 * kKHalf, kOffOnes = 4 * kKHalf;
-constexpr int kSlotBytes = 5 * kKHalf;                // 40960
-constexpr int kOffSlots = kQStages * kQStageBytes;                      // 65536
-constexpr int kOffKeyMeta = kOffSlots + kSlots * kSlotBytes;            // per slot: kc[128], klab[128]
-constexpr int kOffRowMeta = kOffKeyMeta + kSlots * 1024;                // per Q stage: rowmeta[256], rowtok[256]
+constexpr int kQPart = kQRows * kPartBytes;           // 16384: the region of one 32-column part of the Q rows
+constexpr int kKPart = kChunk * kPartBytes;           // 8192:  ... of a key chunk
 constexpr int kBiasFloats = 6048;                     // 3 c0 + 3 with c0 = 31 * 65 (window side 32)
-constexpr int kOffBias = kOffRowMeta + kQStages * 2048;
-constexpr int kOffBars = ((kOffBias + kBiasFloats * 4 + 1023) / 1024) * 1024;
-constexpr int kSmemBytes = kOffBars + 1024;
-static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
 constexpr int kColO = 128;
-constexpr int kNO = kD + 16;
+
+// Shared-memory plan per head dim D (64 or 128): a row is kept as D / 32 parts of 32 columns, each part a region in the
+// 64-byte-swizzled operand layout.  Head dim 64: two Q stages, three ring slots of K | V | ones.  Head dim 128: rows
+// are twice as long, so one Q stage and two ring slots of K | V, and no ones block: tensor memory has no columns
+// left for the row sums next to a 128-column accumulator, the softmax threads add them up themselves.
+template <int D>
+struct Lay {
+    static constexpr int kParts = D / 32;
+    static constexpr bool kOnes = D == 64;
+    static constexpr int kQStages = D == 64 ? 2 : 1, kSlots = D == 64 ? 3 : 2;
+    static constexpr int kQStageBytes = kParts * kQPart;
+    static constexpr int kOffK = 0, kOffV = kParts * kKPart, kOffOnes = 2 * kParts * kKPart;
+    static constexpr int kSlotBytes = (2 * kParts + (kOnes ? 1 : 0)) * kKPart;
+    static constexpr int kOffSlots = kQStages * kQStageBytes;
+    static constexpr int kOffKeyMeta = kOffSlots + kSlots * kSlotBytes;            // per slot: kc[128], klab[128]
+    static constexpr int kOffRowMeta = kOffKeyMeta + kSlots * 1024;                // per Q stage: rowmeta[256], rowtok[256]
+    static constexpr int kOffBias = kOffRowMeta + kQStages * 2048;
+    static constexpr int kOffBars = ((kOffBias + kBiasFloats * 4 + 1023) / 1024) * 1024;
+    static constexpr int kSmemBytes = kOffBars + 1024;
+    static constexpr int kNO = kOnes ? D + 16 : D;    // columns of the PV product
+    static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
+    static_assert(kColO + kNO <= 256, "tensor memory columns of one query tile");
+};
 
 __device__ __forceinline__ int code_stride(int w) { return w + 32; }
 
@@ -113,9 +127,11 @@ __device__ __forceinline__ int lds_i32(uint32_t addr) {
 }
 
 // P for N consecutive key columns of the chunk starting at local column c: exp2(raw * scale + bias - m), packed
-template <int N, bool MASKED>
+// (SUM: also adds the values, before rounding, onto `sum`)
+template <int N, bool MASKED, bool SUM>
 __device__ __forceinline__ void softmax_cols(const uint32_t (&r)[N], uint32_t (&pk)[N / 2], int c, uint32_t bias_i,
-                                             uint32_t a_kc, uint32_t a_klab, int label_i, float scale, float neg_m) {
+                                             uint32_t a_kc, uint32_t a_klab, int label_i, float scale, float neg_m,
+                                             float (&sum)[2]) {
 #pragma unroll
     for (int e4 = 0; e4 < N / 4; ++e4) {
         const int4 kc4 = lds_i4(a_kc + 4 * (c + e4 * 4));
@@ -135,6 +151,10 @@ __device__ __forceinline__ void softmax_cols(const uint32_t (&r)[N], uint32_t (&
         }
         pk[e4 * 2] = pack_bf16(p[0], p[1]);
         pk[e4 * 2 + 1] = pack_bf16(p[2], p[3]);
+        if (SUM) {
+            sum[0] += p[0] + p[2];
+            sum[1] += p[1] + p[3];
+        }
     }
 }
 
@@ -147,7 +167,9 @@ __device__ __forceinline__ float lds_f32_at(uint32_t addr) {
 // 32 key columns that are one window row of a full-width 32-wide window without mask labels: their bias entries are
 // consecutive (descending with the key), so each address is one base plus an immediate offset: no per-key offsets to
 // load, no address arithmetic.  `top` = shared address of the entry of the row's first key.
-__device__ __forceinline__ void softmax_cols32_row(const uint32_t (&r)[32], uint32_t (&pk)[16], uint32_t top, float scale, float neg_m) {
+template <bool SUM>
+__device__ __forceinline__ void softmax_cols32_row(const uint32_t (&r)[32], uint32_t (&pk)[16], uint32_t top, float scale, float neg_m,
+                                                   float (&sum)[2]) {
     const uint32_t bb = top - 124;
     float bv[32];
     bv[0] = lds_f32_at<124>(bb);
@@ -187,6 +209,10 @@ __device__ __forceinline__ void softmax_cols32_row(const uint32_t (&r)[32], uint
         const float p0 = fast_exp2(fmaf(__uint_as_float(r[2 * e2]), scale, bv[2 * e2]) + neg_m);
         const float p1 = fast_exp2(fmaf(__uint_as_float(r[2 * e2 + 1]), scale, bv[2 * e2 + 1]) + neg_m);
         pk[e2] = pack_bf16(p0, p1);
+        if (SUM) {
+            sum[0] += p0;
+            sum[1] += p1;
+        }
     }
 }
 
@@ -210,6 +236,19 @@ __device__ __forceinline__ float score_max_cols(const uint32_t* r, int c, uint32
     return mx;
 }
 
+// 32 accumulator columns of one row, scaled by 1 / row sum, as 64 bytes of bf16
+__device__ __forceinline__ void store_o32(uint4* dst, const uint32_t (&ro)[32], float inv) {
+#pragma unroll
+    for (int c4 = 0; c4 < 4; ++c4) {
+        uint4 val;
+        val.x = pack_bf16(__uint_as_float(ro[c4 * 8 + 0]) * inv, __uint_as_float(ro[c4 * 8 + 1]) * inv);
+        val.y = pack_bf16(__uint_as_float(ro[c4 * 8 + 2]) * inv, __uint_as_float(ro[c4 * 8 + 3]) * inv);
+        val.z = pack_bf16(__uint_as_float(ro[c4 * 8 + 4]) * inv, __uint_as_float(ro[c4 * 8 + 5]) * inv);
+        val.w = pack_bf16(__uint_as_float(ro[c4 * 8 + 6]) * inv, __uint_as_float(ro[c4 * 8 + 7]) * inv);
+        dst[c4] = val;
+    }
+}
+
 template <int N>
 __device__ __forceinline__ void max_cols(const uint32_t (&r)[N], float (&mx)[4]) {
 #pragma unroll
@@ -220,11 +259,30 @@ __device__ __forceinline__ void max_cols(const uint32_t (&r)[N], float (&mx)[4])
     }
 }
 
+// tensor maps over the token stream of one tensor ([tokens, heads * d], 64-byte-swizzled boxes of 32 columns) with
+// boxes of 32, 16 and 8 tokens
+struct RowMaps3 {
+    CUtensorMap m[3];
+};
+struct FwdMaps64 {
+    RowMaps3 q, k, v;
+};
+
+// TMA: the grid consists of complete windows of side 16 or 32 and the longitude shift is a multiple of 8: a window row
+// is then one run of tokens (two where it wraps around the longitude seam), and one loader warp fetches every row with
+// tiled bulk copies; otherwise three loader warps gather the rows with 16-byte cp.async copies.
+template <int D, bool TMA>
 __global__ void __launch_bounds__(kThreads, 1)
 swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                      const __nv_bfloat16* __restrict__ v, const float* __restrict__ bias_prep,
                      __nv_bfloat16* __restrict__ o, float* __restrict__ lse, long long n_items, int ctas_per_head,
-                     int max_pairs) {
+                     int max_pairs, const __grid_constant__ FwdMaps64 maps) {
+    using L = Lay<D>;
+    constexpr int kParts = L::kParts, kQStages = L::kQStages, kSlots = L::kSlots, kQStageBytes = L::kQStageBytes;
+    constexpr int kOffK = L::kOffK, kOffV = L::kOffV, kSlotBytes = L::kSlotBytes, kOffSlots = L::kOffSlots;
+    constexpr int kOffKeyMeta = L::kOffKeyMeta, kOffRowMeta = L::kOffRowMeta, kOffBias = L::kOffBias, kOffBars = L::kOffBars;
+    constexpr int kNO = L::kNO;
+    constexpr bool kSum = !L::kOnes;                    // row sums of P are added up by the softmax threads
     extern __shared__ __align__(1024) unsigned char smem[];
     const uint32_t smem0 = smem_u32(smem);
     const uint32_t bar0 = smem0 + kOffBars;
@@ -248,11 +306,11 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
 
     if (tid == 0) {
         for (int s = 0; s < kQStages; ++s) {
-            mbar_init(bar_qfull(s), kLoaderThreads);
+            mbar_init(bar_qfull(s), TMA ? 32 : kLoaderThreads);
             mbar_init(bar_qempty(s), 1 + 256);        // the issuer's commit + every softmax thread
         }
         for (int s = 0; s < kSlots; ++s) {
-            mbar_init(bar_kvfull(s), kLoaderThreads);
+            mbar_init(bar_kvfull(s), TMA ? 32 : kLoaderThreads);
             mbar_init(bar_kvempty(s), 1);
         }
         for (int t = 0; t < 2; ++t) {
@@ -268,10 +326,12 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
     // the head's prepared bias table; the ones block of every ring slot (first 16 bf16 of a row = 1)
     for (int i = tid; i < kBiasFloats; i += kThreads)
         reinterpret_cast<float*>(smem + kOffBias)[i] = bias_prep[(size_t)head * kBiasFloats + i];
-    for (int i = tid; i < kSlots * kChunk * 4; i += kThreads) {
-        const int s = i / (kChunk * 4), rem = i - s * (kChunk * 4), row = rem >> 2, chunk = rem & 3;
-        const uint32_t val = chunk < 2 ? 0x3F803F80u : 0u;
-        *reinterpret_cast<uint4*>(smem + kOffSlots + s * kSlotBytes + kOffOnes + tile_off<32>(row, chunk)) = make_uint4(val, val, val, val);
+    if (L::kOnes) {
+        for (int i = tid; i < kSlots * kChunk * 4; i += kThreads) {
+            const int s = i / (kChunk * 4), rem = i - s * (kChunk * 4), row = rem >> 2, chunk = rem & 3;
+            const uint32_t val = chunk < 2 ? 0x3F803F80u : 0u;
+            *reinterpret_cast<uint4*>(smem + kOffSlots + s * kSlotBytes + L::kOffOnes + tile_off<32>(row, chunk)) = make_uint4(val, val, val, val);
+        }
     }
     fence_proxy_async();
     if (warp == kMmaWarp) {
@@ -293,16 +353,116 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
 
     if (warp >= kMmaWarp) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kRegsOther));
-    if (warp >= kLoaderWarp0) {
+    if (TMA && warp >= kLoaderWarp0) {
+        // ------------------------------------------------------------------ loader warp (TMA); the other two have no work
+        if (warp == kLoaderWarp0) {
+            const int wrows = kChunk / g.w;                   // window rows per 128 slots
+            int v0 = 0;                                       // first token column of the current window's rows
+            int xb = 0, xwr = 0;
+            // the copies of window row `a`, part `part` of a row: w consecutive slots from `dst` on
+            auto copy_row = [&](const RowMaps3& m3, uint32_t dst, int a, int part, uint32_t bar) {
+                int u = xwr * g.w + a + g.sh;
+                if (u >= g.H) u -= g.H;
+                const int y0 = (xb * g.H + u) * g.W, xc = head * D + part * 32;
+                const int n1 = min(g.w, g.W - v0);            // tokens up to the seam; the rest starts at column 0
+                int y = y0 + v0, n = n1;
+#pragma unroll
+                for (int seg = 0; seg < 2; ++seg) {
+                    if (n >= 32) { tma_load_2d(dst, &m3.m[0], xc, y, bar); dst += 32 * kPartBytes; y += 32; n -= 32; }
+                    if (n >= 16) { tma_load_2d(dst, &m3.m[1], xc, y, bar); dst += 16 * kPartBytes; y += 16; n -= 16; }
+                    if (n >= 8) { tma_load_2d(dst, &m3.m[2], xc, y, bar); dst += 8 * kPartBytes; }
+                    y = y0;
+                    n = g.w - n1;
+                }
+            };
+            int kuse = 0;
+            long long ru = 0;
+            bool ok = true;
+            ItemCursor cur = cursor_init(cta_in_head, ctas_per_head, max_pairs, g.Mw, g.Mh);
+            for (long long it = cta_in_head; ok && it < n_items; it += ctas_per_head, cursor_advance(cur, max_pairs, g.Mw, g.Mh)) {
+                const Item x = make_item(g, cur);
+                if (x.ntiles == 0) continue;
+                const int qs = kuse % kQStages;
+                ok = mbar_wait_all(bar_qempty(qs), ((kuse / kQStages) & 1) ^ 1, cta_abort);
+                if (!ok) break;
+                xb = x.b;
+                xwr = x.r.wr;
+                v0 = x.r.wc * g.w + g.sw;
+                if (v0 >= g.W) v0 -= g.W;
+                const int ew = x.r.ew;                        // = w: the windows are complete
+                // ---- Q rows of the pair and the row tables
+                {
+                    int* rowmeta = reinterpret_cast<int*>(smem + kOffRowMeta + qs * 2048);
+                    int* rowtok = rowmeta + 256;
+                    const int slot0 = x.pair * kQRows;
+                    for (int row = lane; row < kQRows; row += 32) {
+                        const int slot = slot0 + row;
+                        int code = 0, label = 0xff, tok = -1;
+                        if (slot < x.r.n) {
+                            const int a = slot / ew;
+                            tok = offset_token(g, x.r, a, slot - a * ew, code, label);
+                        }
+                        rowmeta[row] = code | (label << 16);
+                        rowtok[row] = tok;
+                    }
+                    const uint32_t qb = smem0 + qs * kQStageBytes;
+                    const int a0 = slot0 / g.w, combos = x.ntiles * wrows * kParts;
+                    for (int i = lane; i < combos; i += 32) {
+                        const int ar = i / kParts, part = i - ar * kParts;
+                        copy_row(maps.q, qb + part * kQPart + ar * g.w * kPartBytes, a0 + ar, part, bar_qfull(qs));
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_expect_tx(bar_qfull(qs), (uint32_t)(x.ntiles * 128 * D * 2));
+                    else mbar_arrive(bar_qfull(qs));
+                }
+                // ---- the key chunks: pass A needs K only (and the key tables if the row maxima are taken exactly), pass B K and V
+                const int first_meta_pass = exact_max(x) ? 0 : 1;
+                for (int pass = 0; pass < 2 && ok; ++pass) {
+                    for (int c = 0; c < x.nch; ++c, ++ru) {
+                        const int s = (int)(ru % kSlots);
+                        ok = mbar_wait_all(bar_kvempty(s), (uint32_t)((ru / kSlots) & 1) ^ 1u, cta_abort);
+                        if (!ok) break;
+                        if (pass >= first_meta_pass) {
+                            int* kcs = reinterpret_cast<int*>(smem + kOffKeyMeta + s * 1024);
+                            int* klab = kcs + 128;
+                            for (int row = lane; row < kChunk; row += 32) {
+                                const int slot = c * kChunk + row;
+                                int code = 0, label = 0xff, kc = 4 * (2 * c0 + 1);
+                                if (slot < x.r.n) {
+                                    const int a = slot / ew;
+                                    offset_token(g, x.r, a, slot - a * ew, code, label);
+                                    kc = 4 * (c0 - code);
+                                }
+                                kcs[row] = kc;
+                                klab[row] = label;
+                            }
+                        }
+                        const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes;
+                        const int per_tensor = wrows * kParts, combos = per_tensor * (pass + 1);
+                        for (int i = lane; i < combos; i += 32) {
+                            const int tsr = i >= per_tensor ? 1 : 0, rem = i - tsr * per_tensor;
+                            const int ar = rem / kParts, part = rem - ar * kParts;
+                            copy_row(tsr ? maps.v : maps.k, sb + (tsr ? kOffV : kOffK) + part * kKPart + ar * g.w * kPartBytes,
+                                     c * wrows + ar, part, bar_kvfull(s));
+                        }
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive_expect_tx(bar_kvfull(s), (uint32_t)(kChunk * D * 2 * (pass + 1)));
+                        else mbar_arrive(bar_kvfull(s));
+                    }
+                }
+                ++kuse;
+            }
+        }
+    } else if (warp >= kLoaderWarp0) {
         // ------------------------------------------------------------------ loaders
-        // Two lanes per row: lane parity picks the row's lo / hi half, each lane issues the half's four 16-byte
-        // copies with one address computation.  A chunk is published (its barrier arrived on) only when the next
+        // D / 32 lanes per row: each takes one 32-column part of the row and issues its four 16-byte copies with one
+        // address computation.  A chunk is published (its barrier arrived on) only when the next
         // one has been issued, so that two chunks are in flight; if the ring has no free slot the pending chunk is
         // published first, or the consumers could never free one.
         const int lt = (warp - kLoaderWarp0) * 32 + lane;
-        const int hf = lt & 1;                            // which 32-column half of the row this thread copies
-        const int lrow = lt >> 1;                         // 0 .. 47
-        constexpr int kRowsPerIter = kLoaderThreads / 2;  // 48
+        const int hf = lt % kParts;                       // which 32-column part of the row this thread copies
+        const int lrow = lt / kParts;
+        constexpr int kRowsPerIter = kLoaderThreads / kParts;
         int kuse = 0;
         long long ru = 0;                                 // ring uses so far
         uint32_t pending_bar = 0;                         // barrier of the group of copies issued last (0: none)
@@ -339,7 +499,7 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             const int q_r = kRowsPerIter / ew, r_r = kRowsPerIter - q_r * ew;       // window-offset step of 48 slots
             // ---- Q rows of the pair (rows without a token as zeros) and the row tables
             {
-                const uint32_t qb = smem0 + qs * kQStageBytes + hf * kQHalf;
+                const uint32_t qb = smem0 + qs * kQStageBytes + hf * kQPart;
                 int* rowmeta = reinterpret_cast<int*>(smem + kOffRowMeta + qs * 2048);
                 int* rowtok = rowmeta + 256;
                 const int slot0 = x.pair * kQRows;
@@ -362,7 +522,7 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                     if (slot0 + row < x.r.n) {
                         int code, label;
                         const int tok = offset_token(g, x.r, a_r, b_r, code, label);
-                        src = q + (sample_off + (size_t)tok) * g.ts + head * kD + hf * 32;
+                        src = q + (sample_off + (size_t)tok) * g.ts + head * D + hf * 32;
                         bytes = 16;
                     }
 #pragma unroll
@@ -377,7 +537,7 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                     const int s = (int)(ru % kSlots);
                     ok = acquire(bar_kvempty(s), (uint32_t)((ru / kSlots) & 1) ^ 1u);
                     if (!ok) break;
-                    const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes + hf * kKHalf;
+                    const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes + hf * kKPart;
                     const int ncols = min(kChunk, x.npad - c * kChunk);
                     if (pass >= first_meta_pass) {
                         int* kcs = reinterpret_cast<int*>(smem + kOffKeyMeta + s * 1024);
@@ -403,15 +563,15 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                         if (c * kChunk + row < x.r.n) {
                             int code, label;
                             const int tok = offset_token(g, x.r, a_r, b_r, code, label);
-                            const size_t off = (sample_off + (size_t)tok) * g.ts + head * kD + hf * 32;
+                            const size_t off = (sample_off + (size_t)tok) * g.ts + head * D + hf * 32;
                             sk = k + off; sv = v + off;
                             bytes = 16;
                         }
 #pragma unroll
                         for (int c4 = 0; c4 < 4; ++c4) {
                             const uint32_t so = tile_off<32>(row, c4);
-                            cp_async16(sb + kOffKlo + so, bytes ? sk + c4 * 8 : sk, bytes);
-                            if (pass == 1) cp_async16(sb + kOffVlo + so, bytes ? sv + c4 * 8 : sv, bytes);
+                            cp_async16(sb + kOffK + so, bytes ? sk + c4 * 8 : sk, bytes);
+                            if (pass == 1) cp_async16(sb + kOffV + so, bytes ? sv + c4 * 8 : sv, bytes);
                         }
                     }
                     issued(bar_kvfull(s));
@@ -442,18 +602,21 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             tc_fence_after();
             const uint32_t qb = smem0 + qs * kQStageBytes;
             // S = Q_t K_c^T into tile t's columns
-            // (descriptor low words = start address in 16-byte units: + 2 per 32-byte K step, + half / 16 for the hi half)
+            // (descriptor low words = start address in 16-byte units: + 2 per 32-byte K step, + region / 16 per 32-column part)
             const uint32_t sd_hi = sdesc_hi(make_sdesc_sw64(smem0, 512));
             const uint32_t q_lo0 = sdesc_lo(make_sdesc_sw64(qb, 512));
             auto issue_qk = [&](int t, uint32_t sb, int ncols) {
                 const uint32_t idesc = make_idesc_bf16(128, ncols, 0, 0);
-                const uint32_t q_lo = q_lo0 + ((t * 128 * kHalfBytes) >> 4), k_lo = sdesc_lo(make_sdesc_sw64(sb, 512));
+                const uint32_t q_lo = q_lo0 + ((t * 128 * kPartBytes) >> 4), k_lo = sdesc_lo(make_sdesc_sw64(sb, 512));
                 const uint32_t t_d = tmem_base + t * 256;
                 if (elect_one()) {
                     mma_ss_h<false>(t_d, q_lo, k_lo, sd_hi, idesc);
                     mma_ss_h<true>(t_d, q_lo + 2, k_lo + 2, sd_hi, idesc);
-                    mma_ss_h<true>(t_d, q_lo + (kQHalf >> 4), k_lo + (kKHalf >> 4), sd_hi, idesc);
-                    mma_ss_h<true>(t_d, q_lo + (kQHalf >> 4) + 2, k_lo + (kKHalf >> 4) + 2, sd_hi, idesc);
+#pragma unroll
+                    for (int pt = 1; pt < kParts; ++pt) {
+                        mma_ss_h<true>(t_d, q_lo + pt * (kQPart >> 4), k_lo + pt * (kKPart >> 4), sd_hi, idesc);
+                        mma_ss_h<true>(t_d, q_lo + pt * (kQPart >> 4) + 2, k_lo + pt * (kKPart >> 4) + 2, sd_hi, idesc);
+                    }
                     mma_commit(bar_sready(t));
                 }
                 __syncwarp();
@@ -528,7 +691,7 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                         ok = mbar_wait_all(bar_ofree(t), (n_items_t[t] - 1) & 1, cta_abort);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint64_t vd = make_sdesc_sw64_mn(sb + kOffVlo, kKHalf, 512);
+                    const uint64_t vd = make_sdesc_sw64_mn(sb + kOffV, kKPart, 512);
                     const uint32_t v_lo = sdesc_lo(vd), d_hi = sdesc_hi(vd);
                     const uint32_t t_o = tmem_base + t * 256 + kColO, t_p = tmem_base + t * 256;
                     const int nks = ncols >> 4;
@@ -587,6 +750,7 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             // ---- pass A: row maximum over all chunks
             float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
             float mxe = -INFINITY;
+            float psum[2] = {0.f, 0.f};
             for (int c = 0; c < x.nch; ++c) {
                 const int ncols = min(kChunk, x.npad - c * kChunk);
                 ok = mbar_wait_all(bar_sready(wg), n_s & 1, cta_abort);
@@ -654,16 +818,16 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                     uint32_t pk[16];
                     tmem_ld_wait();
                     if (i + 1 < nfull) tmem_ld32(t_s + 32 * (i + 1), rb);
-                    if (row32) softmax_cols32_row(ra, pk, top_c - 4 * i * cs, scale, neg_m);
-                    else if (x.masked) softmax_cols<32, true>(ra, pk, 32 * i, bias_i, a_kc, a_klab, label_i, scale, neg_m);
-                    else softmax_cols<32, false>(ra, pk, 32 * i, bias_i, a_kc, a_klab, label_i, scale, neg_m);
+                    if (row32) softmax_cols32_row<kSum>(ra, pk, top_c - 4 * i * cs, scale, neg_m, psum);
+                    else if (x.masked) softmax_cols<32, true, kSum>(ra, pk, 32 * i, bias_i, a_kc, a_klab, label_i, scale, neg_m, psum);
+                    else softmax_cols<32, false, kSum>(ra, pk, 32 * i, bias_i, a_kc, a_klab, label_i, scale, neg_m, psum);
                     tmem_st16(t_s + 16 * i, pk);
                     if (i + 1 < nfull) {
                         tmem_ld_wait();
                         if (i + 2 < nfull) tmem_ld32(t_s + 32 * (i + 2), ra);
-                        if (row32) softmax_cols32_row(rb, pk, top_c - 4 * (i + 1) * cs, scale, neg_m);
-                        else if (x.masked) softmax_cols<32, true>(rb, pk, 32 * (i + 1), bias_i, a_kc, a_klab, label_i, scale, neg_m);
-                        else softmax_cols<32, false>(rb, pk, 32 * (i + 1), bias_i, a_kc, a_klab, label_i, scale, neg_m);
+                        if (row32) softmax_cols32_row<kSum>(rb, pk, top_c - 4 * (i + 1) * cs, scale, neg_m, psum);
+                        else if (x.masked) softmax_cols<32, true, kSum>(rb, pk, 32 * (i + 1), bias_i, a_kc, a_klab, label_i, scale, neg_m, psum);
+                        else softmax_cols<32, false, kSum>(rb, pk, 32 * (i + 1), bias_i, a_kc, a_klab, label_i, scale, neg_m, psum);
                         tmem_st16(t_s + 16 * (i + 1), pk);
                     }
                 }
@@ -671,8 +835,8 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                     uint32_t rt[16], pk[8];
                     tmem_ld16(t_s + 32 * nfull, rt);
                     tmem_ld_wait();
-                    if (x.masked) softmax_cols<16, true>(rt, pk, 32 * nfull, bias_i, a_kc, a_klab, label_i, scale, neg_m);
-                    else softmax_cols<16, false>(rt, pk, 32 * nfull, bias_i, a_kc, a_klab, label_i, scale, neg_m);
+                    if (x.masked) softmax_cols<16, true, kSum>(rt, pk, 32 * nfull, bias_i, a_kc, a_klab, label_i, scale, neg_m, psum);
+                    else softmax_cols<16, false, kSum>(rt, pk, 32 * nfull, bias_i, a_kc, a_klab, label_i, scale, neg_m, psum);
                     tmem_st8(t_s + 16 * nfull, pk);
                 }
                 tmem_st_wait();
@@ -684,36 +848,44 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             if (!mbar_wait_all(bar_oready(wg), n_o & 1, cta_abort)) break;
             ++n_o;
             tc_fence_after();
-            uint32_t ro[32], ro2[32], rsum;
-            tmem_ld32(t_s + kColO, ro);
-            tmem_ld32(t_s + kColO + 32, ro2);
-            tmem_ld1(t_s + kColO + kD, rsum);
-            tmem_ld_wait();
-            tc_fence_before();
-            mbar_arrive(bar_ofree(wg));
-            if (tok >= 0) {
-                const float sum = __uint_as_float(rsum);
-                const size_t row_off = ((size_t)x.b * HW + (size_t)tok) * g.heads + head;
-                lse[row_off] = (m + log2f(sum)) * kLn2;
-                const float inv = 1.f / sum;
-                uint4* dst = reinterpret_cast<uint4*>(o + row_off * kD);
-#pragma unroll
-                for (int c4 = 0; c4 < 4; ++c4) {
-                    uint4 val;
-                    val.x = pack_bf16(__uint_as_float(ro[c4 * 8 + 0]) * inv, __uint_as_float(ro[c4 * 8 + 1]) * inv);
-                    val.y = pack_bf16(__uint_as_float(ro[c4 * 8 + 2]) * inv, __uint_as_float(ro[c4 * 8 + 3]) * inv);
-                    val.z = pack_bf16(__uint_as_float(ro[c4 * 8 + 4]) * inv, __uint_as_float(ro[c4 * 8 + 5]) * inv);
-                    val.w = pack_bf16(__uint_as_float(ro[c4 * 8 + 6]) * inv, __uint_as_float(ro[c4 * 8 + 7]) * inv);
-                    dst[c4] = val;
+            if (!kSum) {
+                uint32_t ro[32], ro2[32], rsum;
+                tmem_ld32(t_s + kColO, ro);
+                tmem_ld32(t_s + kColO + 32, ro2);
+                tmem_ld1(t_s + kColO + D, rsum);
+                tmem_ld_wait();
+                tc_fence_before();
+                mbar_arrive(bar_ofree(wg));
+                if (tok >= 0) {
+                    const float sum = __uint_as_float(rsum);
+                    const size_t row_off = ((size_t)x.b * HW + (size_t)tok) * g.heads + head;
+                    lse[row_off] = (m + log2f(sum)) * kLn2;
+                    const float inv = 1.f / sum;
+                    uint4* dst = reinterpret_cast<uint4*>(o + row_off * D);
+                    store_o32(dst, ro, inv);
+                    store_o32(dst + 4, ro2, inv);
                 }
+            } else {
+                // the accumulator's 128 columns in two rounds of 64, to keep the registers in hand
+                const float sum = psum[0] + psum[1];
+                const float inv = 1.f / sum;
+                const size_t row_off = ((size_t)x.b * HW + (size_t)(tok >= 0 ? tok : 0)) * g.heads + head;
+                uint4* dst = reinterpret_cast<uint4*>(o + row_off * D);
+                if (tok >= 0) lse[row_off] = (m + log2f(sum)) * kLn2;
 #pragma unroll
-                for (int c4 = 0; c4 < 4; ++c4) {
-                    uint4 val;
-                    val.x = pack_bf16(__uint_as_float(ro2[c4 * 8 + 0]) * inv, __uint_as_float(ro2[c4 * 8 + 1]) * inv);
-                    val.y = pack_bf16(__uint_as_float(ro2[c4 * 8 + 2]) * inv, __uint_as_float(ro2[c4 * 8 + 3]) * inv);
-                    val.z = pack_bf16(__uint_as_float(ro2[c4 * 8 + 4]) * inv, __uint_as_float(ro2[c4 * 8 + 5]) * inv);
-                    val.w = pack_bf16(__uint_as_float(ro2[c4 * 8 + 6]) * inv, __uint_as_float(ro2[c4 * 8 + 7]) * inv);
-                    dst[4 + c4] = val;
+                for (int hq = 0; hq < D / 64; ++hq) {
+                    uint32_t ro[32], ro2[32];
+                    tmem_ld32(t_s + kColO + 64 * hq, ro);
+                    tmem_ld32(t_s + kColO + 64 * hq + 32, ro2);
+                    tmem_ld_wait();
+                    if (hq == D / 64 - 1) {
+                        tc_fence_before();
+                        mbar_arrive(bar_ofree(wg));
+                    }
+                    if (tok >= 0) {
+                        store_o32(dst + 8 * hq, ro, inv);
+                        store_o32(dst + 8 * hq + 4, ro2, inv);
+                    }
                 }
             }
         }
@@ -786,7 +958,7 @@ cudaError_t launch_bias_prep64(const Geo& g, const float* bias, float* prep, cud
     return cudaGetLastError();
 }
 
-bool fwd_tc64_supported(const Geo& g) { return g.d == 64 && g.w <= 32 && g.nmax <= 1024 && g.heads <= 148; }
+bool fwd_tc64_supported(const Geo& g) { return (g.d == 64 || g.d == 128) && g.w <= 32 && g.nmax <= 1024 && g.heads <= 148; }
 
 size_t fwd_tc64_workspace_bytes(const Geo& g) { return (size_t)g.heads * kBiasFloats * sizeof(float); }
 
@@ -802,12 +974,25 @@ cudaError_t launch_fwd_tc64(const Geo& g, const void* q, const void* k, const vo
     long long cph = sm_count / g.heads;
     if (cph < 1) cph = 1;
     if (cph > items) cph = items;
-    e = cudaFuncSetAttribute(swin_fwd_tc64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    const unsigned grid = (unsigned)(cph * g.heads);
+    FwdMaps64 maps;
+    std::memset(&maps, 0, sizeof maps);
+    static const bool tma_off = [] { const char* e_ = std::getenv("TERRA_NO_TMA"); return e_ && e_[0] == '1'; }();
+    bool tma = !tma_off && (g.w == 16 || g.w == 32) && g.H % g.w == 0 && g.W % g.w == 0 && g.sw % 8 == 0 &&
+               (long long)g.B * g.H * g.W < 0x7fffffffLL;
+    for (int i = 0; i < 3 && tma; ++i) {
+        const int box = 32 >> i;
+        tma = make_row_map(&maps.q.m[i], g, q, g.ts, box) && make_row_map(&maps.k.m[i], g, k, g.ts, box) &&
+              make_row_map(&maps.v.m[i], g, v, g.ts, box);
+    }
+    auto kern = g.d == 64 ? (tma ? swin_fwd_tc64_kernel<64, true> : swin_fwd_tc64_kernel<64, false>)
+                          : (tma ? swin_fwd_tc64_kernel<128, true> : swin_fwd_tc64_kernel<128, false>);
+    const int smem_bytes = g.d == 64 ? Lay<64>::kSmemBytes : Lay<128>::kSmemBytes;
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
     if (e != cudaSuccess) return e;
     prof_begin("swin_fwd_tc64_kernel", stream);
-    swin_fwd_tc64_kernel<<<(unsigned)(cph * g.heads), kThreads, kSmemBytes, stream>>>(
-        g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, prep, (__nv_bfloat16*)o, lse,
-        items, (int)cph, max_pairs);
+    kern<<<grid, kThreads, smem_bytes, stream>>>(g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, prep,
+                                                 (__nv_bfloat16*)o, lse, items, (int)cph, max_pairs, maps);
     count_launch(stream);
     return cudaGetLastError();
 }

@@ -20,6 +20,10 @@ SHAPES = [
     ("d128_w32_ragged", 1, 70, 45, 1, 128, 32, 20, 30, 0, 0),       # 13-wide last column, 6-high last row
     ("d128_w5", 1, 23, 31, 2, 128, 5, 2, 3, 0, 1),
     ("d128_w16_noshift", 1, 40, 48, 2, 128, 16, 0, 0, 0, 1),
+    # complete windows and a longitude shift that is a multiple of 8: rows arrive by tiled bulk copies
+    ("d128_w16_bulk", 1, 32, 48, 2, 128, 16, 8, 8, 0, 1),
+    ("d128_w32_bulk_shift24", 1, 64, 64, 1, 128, 32, 8, 24, 0, 0),  # seam after 8 of a row's 32 tokens, masks on both axes
+    ("d128_w32_bulk_noshift", 2, 32, 64, 2, 128, 32, 0, 0, 0, 1),
 ]
 
 

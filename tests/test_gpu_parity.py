@@ -29,6 +29,8 @@ EDGE = [
     # 16-wide windows whose rows are runs of consecutive tokens: the forward fetches them with tiled TMA copies
     ("tma_rows_wrap_lat", 2, 30, 56, 3, 32, 16, 8, 8, 0, 1),     # last column 8 wide, last row 14 high, latitude wrap + mask
     ("tma_nonperiodic", 1, 46, 64, 2, 32, 16, 8, 16, 0, 0),      # masks on both axes
+    ("bulk64_w32", 1, 64, 96, 2, 64, 32, 16, 8, 0, 1),           # head dim 64, complete windows: rows by tiled bulk copies
+    ("bulk64_w16", 2, 32, 48, 2, 64, 16, 8, 8, 0, 0),
     ("tma_noshift", 1, 32, 40, 2, 32, 16, 0, 0, 0, 1),
 ]
 
@@ -195,6 +197,7 @@ LARGE = [
     ("x8_d64_w32", 1, 70, 80, 2, 64, 32, 16, 16, 0, 0, 8.0),
     ("x32_d64_w32", 1, 70, 80, 2, 64, 32, 16, 16, 0, 0, 32.0),
     ("x8_d64_w20", 1, 45, 50, 2, 64, 20, 10, 10, 0, 1, 8.0),
+    ("x8_d128_w32", 1, 64, 64, 1, 128, 32, 16, 16, 0, 0, 8.0),
 ]
 
 
