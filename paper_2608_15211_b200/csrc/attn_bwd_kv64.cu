@@ -19,6 +19,10 @@
 #include "swin_common.cuh"
 #include "swin_kernels.h"
 #include "tc_common.cuh"
+#include "tma_rows.cuh"
+
+#include <cstdlib>
+#include <cstring>
 
 namespace terra {
 
@@ -36,28 +40,36 @@ constexpr int kWorkThreads = 256;
 constexpr int kRegsLaunch = 168, kRegsWork = 208, kRegsOther = 80;
 static_assert(2 * (kRegsWork - kRegsLaunch) <= (kRegsLaunch - kRegsOther), "register hand-over does not balance");
 
-constexpr int kD = 64;
-constexpr int kHalfBytes = 64;
+constexpr int kPartBytes = 64;                        // one 32-column part of a row
 constexpr int kTile = 128;                            // keys per item, queries per chunk
-constexpr int kHalf = kTile * kHalfBytes;             // 8192: one 32-column half of 128 rows
-constexpr int kKvStages = 2, kSlots = 3;
-// key stage: K lo | K hi | V lo | V hi, then per key row: 4 * bias code, label, token
-constexpr int kOffKlo = 0, kOffKhi = kHalf, kOffVlo = 2 * kHalf, kOffVhi = 3 * kHalf;
-constexpr int kKvRows = 4 * kHalf;                    // 32768
-constexpr int kOffKCode = kKvRows, kOffKLab = kKvRows + 512, kOffKTok = kKvRows + 1024;
-constexpr int kKvStageBytes = kKvRows + 2048;
-// query slot: Q lo | Q hi | dO lo | dO hi, then per query column: 4 * bias code, label, lse, delta
-constexpr int kOffQlo = 0, kOffQhi = kHalf, kOffGlo = 2 * kHalf, kOffGhi = 3 * kHalf;
-constexpr int kOffQCode = 4 * kHalf, kOffQLab = kOffQCode + 512, kOffQLse = kOffQCode + 1024, kOffQDelta = kOffQCode + 1536;
-constexpr int kSlotBytes = 4 * kHalf + 2048;          // 34816
-constexpr int kOffSlots = kKvStages * kKvStageBytes;  // 69632
+constexpr int kPart = kTile * kPartBytes;             // 8192: the region of one 32-column part of 128 rows
 constexpr int kBiasFloats = 6048;
-constexpr int kOffBias = kOffSlots + kSlots * kSlotBytes;
-constexpr int kOffBars = ((kOffBias + kBiasFloats * 4 + 1023) / 1024) * 1024;
-constexpr int kSmemBytes = kOffBars + 1024;
-static_assert(kKvStageBytes % 1024 == 0 && kSlotBytes % 1024 == 0, "tiles keep the swizzle alignment");
-static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
-constexpr int kColS = 0, kColDP = 128, kColDV = 256, kColDK = 320;
+constexpr int kColS = 0, kColDP = 128, kColDV = 256;  // dK follows dV
+
+// Shared-memory plan per head dim D (64 or 128): a row is kept as D / 32 parts of 32 columns, each part a region in
+// the 64-byte-swizzled operand layout.  Head dim 64: two key stages, three query slots; head dim 128: one and two.
+template <int D>
+struct Lay {
+    static constexpr int kParts = D / 32;
+    static constexpr int kKvStages = D == 64 ? 2 : 1, kSlots = D == 64 ? 3 : 2;
+    static constexpr int kRows = 2 * kParts * kPart;  // two tensors' rows
+    // key stage: K parts | V parts, then per key row: 4 * bias code, label, token
+    static constexpr int kOffK = 0, kOffV = kParts * kPart;
+    static constexpr int kOffKCode = kRows, kOffKLab = kRows + 512, kOffKTok = kRows + 1024;
+    static constexpr int kKvStageBytes = kRows + 2048;
+    // query slot: Q parts | dO parts, then per query column: 4 * bias code, label, lse, delta
+    static constexpr int kOffQ = 0, kOffG = kParts * kPart;
+    static constexpr int kOffQCode = kRows, kOffQLab = kRows + 512, kOffQLse = kRows + 1024, kOffQDelta = kRows + 1536;
+    static constexpr int kSlotBytes = kRows + 2048;
+    static constexpr int kOffSlots = kKvStages * kKvStageBytes;
+    static constexpr int kOffBias = kOffSlots + kSlots * kSlotBytes;
+    static constexpr int kOffBars = ((kOffBias + kBiasFloats * 4 + 1023) / 1024) * 1024;
+    static constexpr int kSmemBytes = kOffBars + 1024;
+    static constexpr int kColDK = kColDV + D;
+    static_assert(kKvStageBytes % 1024 == 0 && kSlotBytes % 1024 == 0, "tiles keep the swizzle alignment");
+    static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
+    static_assert(kColDK + D <= 512, "tensor memory columns");
+};
 
 __device__ __forceinline__ int code_stride(int w) { return w + 32; }
 
@@ -124,9 +136,11 @@ __device__ __forceinline__ int lds_i32(uint32_t addr) {
 // token); a query column without a token has lse = +inf, so its P is 0.
 // ROW32: the window is 32 tokens wide, so the group's 16 queries sit in one window row and their bias codes are
 // consecutive: `code4` = 4 * code of column c, no per-query code table is read.
+// `sl_a` = shared address of the slot's per-query tables (code, label, lse, delta: 512 bytes each).
 template <bool MASKED, bool ROW32 = false>
 __device__ __forceinline__ void cols16(const uint32_t (&rs)[16], const uint32_t (&rp)[16], int c, uint32_t bias_row, int klabel,
                                        uint32_t sl_a, float scale, uint32_t (&pk_p)[8], uint32_t (&pk_ds)[8], int code4 = 0) {
+    constexpr int kOffQCode = 0, kOffQLab = 512, kOffQLse = 1024, kOffQDelta = 1536;
     // all table loads first (they are issued in program order), then the gathers that depend on them, then the math
     int co[16], ql[16];
     float l2[16], dl[16], bv[16];
@@ -168,12 +182,39 @@ __device__ __forceinline__ void cols16(const uint32_t (&rs)[16], const uint32_t 
     }
 }
 
+// 32 accumulator columns of one row, scaled, as 64 bytes of bf16
+__device__ __forceinline__ void store_scaled32(uint4* dst, const uint32_t (&r)[32], float f) {
+#pragma unroll
+    for (int c4 = 0; c4 < 4; ++c4) {
+        uint4 a;
+        a.x = pack_bf16(__uint_as_float(r[c4 * 8 + 0]) * f, __uint_as_float(r[c4 * 8 + 1]) * f);
+        a.y = pack_bf16(__uint_as_float(r[c4 * 8 + 2]) * f, __uint_as_float(r[c4 * 8 + 3]) * f);
+        a.z = pack_bf16(__uint_as_float(r[c4 * 8 + 4]) * f, __uint_as_float(r[c4 * 8 + 5]) * f);
+        a.w = pack_bf16(__uint_as_float(r[c4 * 8 + 6]) * f, __uint_as_float(r[c4 * 8 + 7]) * f);
+        dst[c4] = a;
+    }
+}
+
+struct KvMaps64 {
+    RowMaps3 q, k, v, g;      // g: the output gradient dO
+};
+
+// TMA: complete windows of side 16 or 32 and a longitude shift that is a multiple of 8: one loader warp fetches every
+// window row with tiled bulk copies (per-query lse and delta by 4-byte cp.async copies tied to the same barrier);
+// otherwise three loader warps gather the rows with 16-byte cp.async copies.
+template <int D, bool TMA>
 __global__ void __launch_bounds__(kThreads, 1)
 swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                      const __nv_bfloat16* __restrict__ v, const __nv_bfloat16* __restrict__ d_o,
                      const float* __restrict__ bias_prep, const float* __restrict__ lse, const float* __restrict__ delta,
                      __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv, long long n_items, int ctas_per_head,
-                     int max_tiles) {
+                     int max_tiles, const __grid_constant__ KvMaps64 maps) {
+    using L = Lay<D>;
+    constexpr int kParts = L::kParts, kKvStages = L::kKvStages, kSlots = L::kSlots;
+    constexpr int kOffK = L::kOffK, kOffV = L::kOffV, kOffKCode = L::kOffKCode, kOffKLab = L::kOffKLab, kOffKTok = L::kOffKTok;
+    constexpr int kKvStageBytes = L::kKvStageBytes, kOffQ = L::kOffQ, kOffG = L::kOffG, kOffQCode = L::kOffQCode;
+    constexpr int kOffQLab = L::kOffQLab, kOffQLse = L::kOffQLse, kOffQDelta = L::kOffQDelta, kSlotBytes = L::kSlotBytes;
+    constexpr int kOffSlots = L::kOffSlots, kOffBias = L::kOffBias, kOffBars = L::kOffBars, kColDK = L::kColDK;
     extern __shared__ __align__(1024) unsigned char smem[];
     const uint32_t smem0 = smem_u32(smem);
     const uint32_t bar0 = smem0 + kOffBars;
@@ -198,11 +239,11 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
 
     if (tid == 0) {
         for (int s = 0; s < kKvStages; ++s) {
-            mbar_init(bar_kvfull(s), kLoaderThreads);
+            mbar_init(bar_kvfull(s), TMA ? 32 : kLoaderThreads);
             mbar_init(bar_kvempty(s), 1 + kWorkThreads);   // the issuer's commit + every elementwise thread
         }
         for (int s = 0; s < kSlots; ++s) {
-            mbar_init(bar_qfull(s), kLoaderThreads);
+            mbar_init(bar_qfull(s), TMA ? 32 : kLoaderThreads);
             mbar_init(bar_qempty(s), 1);
         }
         for (int h = 0; h < 2; ++h) {
@@ -232,14 +273,88 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
 
     if (warp >= kMmaWarp) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kRegsOther));
-    if (warp >= kLoaderWarp0) {
+    if (TMA && warp >= kLoaderWarp0) {
+        // ------------------------------------------------------------------ loader warp (TMA); the other two have no work
+        if (warp == kLoaderWarp0) {
+            const int wrows = kTile / g.w;                    // window rows per 128 slots
+            const int per_tensor = wrows * kParts;
+            int kuse = 0;
+            long long ru = 0;
+            bool ok = true;
+            ItemCursor cur = cursor_init(cta_in_head, ctas_per_head, max_tiles, g.Mw, g.Mh);
+            for (long long it = cta_in_head; ok && it < n_items; it += ctas_per_head, cursor_advance(cur, max_tiles, g.Mw, g.Mh)) {
+                const Item x = make_item(g, cur);
+                if (!x.has) continue;
+                const int ks = kuse % kKvStages;
+                ok = mbar_wait_all(bar_kvempty(ks), ((kuse / kKvStages) & 1) ^ 1, cta_abort);
+                if (!ok) break;
+                const size_t sample_off = (size_t)x.b * HW;
+                const int ew = x.r.ew;                        // = w: the windows are complete
+                int v0 = x.r.wc * g.w + g.sw;
+                if (v0 >= g.W) v0 -= g.W;
+                // ---- the key tile
+                {
+                    unsigned char* st = smem + ks * kKvStageBytes;
+                    const int slot0 = x.kt * kTile;
+                    for (int row = lane; row < kTile; row += 32) {
+                        const int slot = slot0 + row;
+                        int code, label;
+                        const int a = slot / ew;
+                        const int tok = offset_token(g, x.r, a, slot - a * ew, code, label);
+                        reinterpret_cast<int*>(st + kOffKCode)[row] = 4 * code;
+                        reinterpret_cast<int*>(st + kOffKLab)[row] = label;
+                        reinterpret_cast<int*>(st + kOffKTok)[row] = tok;
+                    }
+                    const uint32_t sb = smem0 + ks * kKvStageBytes;
+                    for (int i = lane; i < 2 * per_tensor; i += 32) {
+                        const int tsr = i >= per_tensor ? 1 : 0, rem = i - tsr * per_tensor;
+                        const int ar = rem / kParts, part = rem - ar * kParts;
+                        bulk_copy_window_row(tsr ? maps.v : maps.k, sb + (tsr ? kOffV : kOffK) + part * kPart + ar * g.w * kPartBytes, g,
+                                             x.b, x.r.wr, v0, x.kt * wrows + ar, head * D + part * 32, bar_kvfull(ks));
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_expect_tx(bar_kvfull(ks), (uint32_t)(kTile * D * 2 * 2));
+                    else mbar_arrive(bar_kvfull(ks));
+                }
+                // ---- the window's queries, chunk by chunk
+                for (int c = 0; c < x.nch; ++c, ++ru) {
+                    const int s = (int)(ru % kSlots);
+                    ok = mbar_wait_all(bar_qempty(s), (uint32_t)((ru / kSlots) & 1) ^ 1u, cta_abort);
+                    if (!ok) break;
+                    unsigned char* sl = smem + kOffSlots + s * kSlotBytes;
+                    const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes;
+                    for (int row = lane; row < kTile; row += 32) {
+                        const int slot = c * kTile + row;
+                        int code, label;
+                        const int a = slot / ew;
+                        const int tok = offset_token(g, x.r, a, slot - a * ew, code, label);
+                        const size_t li = (sample_off + (size_t)tok) * g.heads + head;
+                        cp_async4(sb + kOffQLse + 4 * row, lse + li);
+                        cp_async4(sb + kOffQDelta + 4 * row, delta + li);
+                        reinterpret_cast<int*>(sl + kOffQCode)[row] = 4 * code;
+                        reinterpret_cast<int*>(sl + kOffQLab)[row] = label;
+                    }
+                    for (int i = lane; i < 2 * per_tensor; i += 32) {
+                        const int tsr = i >= per_tensor ? 1 : 0, rem = i - tsr * per_tensor;
+                        const int ar = rem / kParts, part = rem - ar * kParts;
+                        bulk_copy_window_row(tsr ? maps.g : maps.q, sb + (tsr ? kOffG : kOffQ) + part * kPart + ar * g.w * kPartBytes, g,
+                                             x.b, x.r.wr, v0, c * wrows + ar, head * D + part * 32, bar_qfull(s));
+                    }
+                    if (lane == 0) mbar_expect_tx(bar_qfull(s), (uint32_t)(kTile * D * 2 * 2));
+                    // the lane's arrival: when its lse / delta copies have landed (its table entries were written before)
+                    cp_async_mbar_arrive_noinc(bar_qfull(s));
+                }
+                ++kuse;
+            }
+        }
+    } else if (warp >= kLoaderWarp0) {
         // ------------------------------------------------------------------ loaders
-        // Two lanes per row (lane parity = the row's lo / hi half, four 16-byte copies each).  A group of copies is
+        // D / 32 lanes per row (one 32-column part of the row each, four 16-byte copies).  A group of copies is
         // published when the next one has been issued; if a ring has no free place the pending group is published first.
         const int lt = (warp - kLoaderWarp0) * 32 + lane;
-        const int hf = lt & 1;
-        const int lrow = lt >> 1;
-        constexpr int kRowsPerIter = kLoaderThreads / 2;      // 48
+        const int hf = lt % kParts;
+        const int lrow = lt / kParts;
+        constexpr int kRowsPerIter = kLoaderThreads / kParts;
         int kuse = 0;
         long long ru = 0;
         uint32_t pending_bar = 0;
@@ -275,7 +390,7 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             // ---- the key tile: K, V rows (rows without a token as zeros) and the key tables
             {
                 unsigned char* st = smem + ks * kKvStageBytes;
-                const uint32_t sb = smem0 + ks * kKvStageBytes + hf * kHalf;
+                const uint32_t sb = smem0 + ks * kKvStageBytes + hf * kPart;
                 const int slot0 = x.kt * kTile;
                 for (int row = lt; row < kTile; row += kLoaderThreads) {
                     const int slot = slot0 + row;
@@ -296,15 +411,15 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                     if (slot0 + row < x.r.n) {
                         int code, label;
                         const int tok = offset_token(g, x.r, a_r, b_r, code, label);
-                        const size_t off = (sample_off + (size_t)tok) * g.ts + head * kD + hf * 32;
+                        const size_t off = (sample_off + (size_t)tok) * g.ts + head * D + hf * 32;
                         sk = k + off; sv = v + off;
                         bytes = 16;
                     }
 #pragma unroll
                     for (int c4 = 0; c4 < 4; ++c4) {
                         const uint32_t so = tile_off<32>(row, c4);
-                        cp_async16(sb + kOffKlo + so, bytes ? sk + c4 * 8 : sk, bytes);
-                        cp_async16(sb + kOffVlo + so, bytes ? sv + c4 * 8 : sv, bytes);
+                        cp_async16(sb + kOffK + so, bytes ? sk + c4 * 8 : sk, bytes);
+                        cp_async16(sb + kOffV + so, bytes ? sv + c4 * 8 : sv, bytes);
                     }
                 }
                 issued(bar_kvfull(ks));
@@ -315,7 +430,7 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                 ok = acquire(bar_qempty(s), (uint32_t)((ru / kSlots) & 1) ^ 1u);
                 if (!ok) break;
                 unsigned char* sl = smem + kOffSlots + s * kSlotBytes;
-                const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes + hf * kHalf;
+                const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes + hf * kPart;
                 const int ncols = min(kTile, x.npad - c * kTile);
                 for (int row = lt; row < kTile; row += kLoaderThreads) {
                     const int slot = c * kTile + row;
@@ -343,15 +458,15 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                     if (c * kTile + row < x.r.n) {
                         int code, label;
                         const int tok = offset_token(g, x.r, a_r, b_r, code, label);
-                        sq = q + (sample_off + (size_t)tok) * g.ts + head * kD + hf * 32;
-                        sg = d_o + ((sample_off + (size_t)tok) * g.heads + head) * kD + hf * 32;
+                        sq = q + (sample_off + (size_t)tok) * g.ts + head * D + hf * 32;
+                        sg = d_o + ((sample_off + (size_t)tok) * g.heads + head) * D + hf * 32;
                         bytes = 16;
                     }
 #pragma unroll
                     for (int c4 = 0; c4 < 4; ++c4) {
                         const uint32_t so = tile_off<32>(row, c4);
-                        cp_async16(sb + kOffQlo + so, bytes ? sq + c4 * 8 : sq, bytes);
-                        cp_async16(sb + kOffGlo + so, bytes ? sg + c4 * 8 : sg, bytes);
+                        cp_async16(sb + kOffQ + so, bytes ? sq + c4 * 8 : sq, bytes);
+                        cp_async16(sb + kOffG + so, bytes ? sg + c4 * 8 : sg, bytes);
                     }
                 }
                 issued(bar_qfull(s));
@@ -365,7 +480,7 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
         }
     } else {
         // ------------------------------------------------------------------ MMA issuer
-        const uint32_t idesc_acc = make_idesc_bf16(128, kD, 0, 1);       // A from TMEM, B = 16 rows x 64 (MN-major)
+        const uint32_t idesc_acc = make_idesc_bf16(128, D, 0, 1);        // A from TMEM, B = 16 rows x D (MN-major)
         const uint32_t sd_hi = sdesc_hi(make_sdesc_sw64(smem0, 512));    // common high word of the K-major descriptors
         int kuse = 0;
         int n_ds[2] = {0, 0};
@@ -388,24 +503,30 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                 return true;
             };
             // S^T = K Q^T, dP^T = V dO^T for the 64 queries of half h of the chunk in ring slot `sb`
-            // (descriptor low words = start address in 16-byte units: + 2 per 32-byte K step, + kHalf / 16 for the hi half)
-            const uint32_t k_lo = sdesc_lo(make_sdesc_sw64(kb + kOffKlo, 512)), v_lo = sdesc_lo(make_sdesc_sw64(kb + kOffVlo, 512));
+            // (descriptor low words = start address in 16-byte units: + 2 per 32-byte K step, + kPart / 16 per 32-column part)
+            const uint32_t k_lo = sdesc_lo(make_sdesc_sw64(kb + kOffK, 512)), v_lo = sdesc_lo(make_sdesc_sw64(kb + kOffV, 512));
             auto issue_sdp = [&](int h, uint32_t sb, int nc) {
                 const uint32_t idesc = make_idesc_bf16(128, nc, 0, 0);
-                const uint32_t q_lo = sdesc_lo(make_sdesc_sw64(sb + kOffQlo + h * 64 * kHalfBytes, 512));
-                const uint32_t g_lo = sdesc_lo(make_sdesc_sw64(sb + kOffGlo + h * 64 * kHalfBytes, 512));
+                const uint32_t q_lo = sdesc_lo(make_sdesc_sw64(sb + kOffQ + h * 64 * kPartBytes, 512));
+                const uint32_t g_lo = sdesc_lo(make_sdesc_sw64(sb + kOffG + h * 64 * kPartBytes, 512));
                 const uint32_t t_s = tmem_base + kColS + 64 * h, t_dp = tmem_base + kColDP + 64 * h;
-                constexpr uint32_t kHi = kHalf >> 4;
+                constexpr uint32_t kNext = kPart >> 4;
                 tc_fence_after();
                 if (elect_one()) {
                     mma_ss_h<false>(t_s, k_lo, q_lo, sd_hi, idesc);
                     mma_ss_h<true>(t_s, k_lo + 2, q_lo + 2, sd_hi, idesc);
-                    mma_ss_h<true>(t_s, k_lo + kHi, q_lo + kHi, sd_hi, idesc);
-                    mma_ss_h<true>(t_s, k_lo + kHi + 2, q_lo + kHi + 2, sd_hi, idesc);
+#pragma unroll
+                    for (int pt = 1; pt < kParts; ++pt) {
+                        mma_ss_h<true>(t_s, k_lo + pt * kNext, q_lo + pt * kNext, sd_hi, idesc);
+                        mma_ss_h<true>(t_s, k_lo + pt * kNext + 2, q_lo + pt * kNext + 2, sd_hi, idesc);
+                    }
                     mma_ss_h<false>(t_dp, v_lo, g_lo, sd_hi, idesc);
                     mma_ss_h<true>(t_dp, v_lo + 2, g_lo + 2, sd_hi, idesc);
-                    mma_ss_h<true>(t_dp, v_lo + kHi, g_lo + kHi, sd_hi, idesc);
-                    mma_ss_h<true>(t_dp, v_lo + kHi + 2, g_lo + kHi + 2, sd_hi, idesc);
+#pragma unroll
+                    for (int pt = 1; pt < kParts; ++pt) {
+                        mma_ss_h<true>(t_dp, v_lo + pt * kNext, g_lo + pt * kNext, sd_hi, idesc);
+                        mma_ss_h<true>(t_dp, v_lo + pt * kNext + 2, g_lo + pt * kNext + 2, sd_hi, idesc);
+                    }
                     mma_commit(bar_sdp(h));
                 }
                 __syncwarp();
@@ -432,8 +553,8 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                     if (!ok) break;
                     tc_fence_after();
                     // dV += P^T dO, dK += dS^T Q over the half chunk's query columns
-                    const uint64_t gd = make_sdesc_sw64_mn(sb + kOffGlo + h * 64 * kHalfBytes, kHalf, 512);
-                    const uint64_t qd = make_sdesc_sw64_mn(sb + kOffQlo + h * 64 * kHalfBytes, kHalf, 512);
+                    const uint64_t gd = make_sdesc_sw64_mn(sb + kOffG + h * 64 * kPartBytes, kPart, 512);
+                    const uint64_t qd = make_sdesc_sw64_mn(sb + kOffQ + h * 64 * kPartBytes, kPart, 512);
                     const uint32_t g_lo = sdesc_lo(gd), q_lo = sdesc_lo(qd), d_hi = sdesc_hi(gd);
                     const uint32_t t_p = tmem_base + kColS + 64 * h, t_ds = tmem_base + kColDP + 64 * h;
                     const int nks = nc >> 4;
@@ -495,7 +616,7 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             const bool row32 = x.r.ew == 32;
             for (int c = 0; c < x.nch && ok; ++c, ++ru) {
                 const int s = (int)(ru % kSlots);
-                const uint32_t sl_a = smem0 + kOffSlots + s * kSlotBytes;
+                const uint32_t sl_a = smem0 + kOffSlots + s * kSlotBytes + kOffQCode;      // the slot's per-query tables
                 const int ncols = min(kTile, x.npad - c * kTile);
                 if (ncols <= 64 * hcol) continue;          // this group's half of the chunk does not exist
                 ok = mbar_wait_all(bar_sdp(hcol), n_half & 1, cta_abort);
@@ -544,33 +665,22 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             // ---- read-out: dV rows by warps 0-3, dK rows by warps 4-7
             if (!mbar_wait_all(bar_acc, kuse & 1, cta_abort)) break;
             tc_fence_after();
-            uint32_t r0[32], r1[32];
-            tmem_ld32(tmem_base + lane_addr + (hcol == 0 ? kColDV : kColDK), r0);
-            tmem_ld32(tmem_base + lane_addr + (hcol == 0 ? kColDV : kColDK) + 32, r1);
-            tmem_ld_wait();
-            tc_fence_before();
-            mbar_arrive(bar_accfree);
-            if (ktok >= 0) {
-                const float f = hcol == 0 ? 1.f : out_scale;
-                __nv_bfloat16* out = hcol == 0 ? dv : dk;
-                uint4* dst = reinterpret_cast<uint4*>(out + ((size_t)x.b * HW + (size_t)ktok) * g.ts + head * kD);
+            const float f = hcol == 0 ? 1.f : out_scale;
+            __nv_bfloat16* out = hcol == 0 ? dv : dk;
+            uint4* dst = reinterpret_cast<uint4*>(out + ((size_t)x.b * HW + (size_t)(ktok >= 0 ? ktok : 0)) * g.ts + head * D);
 #pragma unroll
-                for (int c4 = 0; c4 < 4; ++c4) {
-                    uint4 a;
-                    a.x = pack_bf16(__uint_as_float(r0[c4 * 8 + 0]) * f, __uint_as_float(r0[c4 * 8 + 1]) * f);
-                    a.y = pack_bf16(__uint_as_float(r0[c4 * 8 + 2]) * f, __uint_as_float(r0[c4 * 8 + 3]) * f);
-                    a.z = pack_bf16(__uint_as_float(r0[c4 * 8 + 4]) * f, __uint_as_float(r0[c4 * 8 + 5]) * f);
-                    a.w = pack_bf16(__uint_as_float(r0[c4 * 8 + 6]) * f, __uint_as_float(r0[c4 * 8 + 7]) * f);
-                    dst[c4] = a;
+            for (int hq = 0; hq < D / 64; ++hq) {
+                uint32_t r0[32], r1[32];
+                tmem_ld32(tmem_base + lane_addr + (hcol == 0 ? kColDV : kColDK) + 64 * hq, r0);
+                tmem_ld32(tmem_base + lane_addr + (hcol == 0 ? kColDV : kColDK) + 64 * hq + 32, r1);
+                tmem_ld_wait();
+                if (hq == D / 64 - 1) {
+                    tc_fence_before();
+                    mbar_arrive(bar_accfree);
                 }
-#pragma unroll
-                for (int c4 = 0; c4 < 4; ++c4) {
-                    uint4 a;
-                    a.x = pack_bf16(__uint_as_float(r1[c4 * 8 + 0]) * f, __uint_as_float(r1[c4 * 8 + 1]) * f);
-                    a.y = pack_bf16(__uint_as_float(r1[c4 * 8 + 2]) * f, __uint_as_float(r1[c4 * 8 + 3]) * f);
-                    a.z = pack_bf16(__uint_as_float(r1[c4 * 8 + 4]) * f, __uint_as_float(r1[c4 * 8 + 5]) * f);
-                    a.w = pack_bf16(__uint_as_float(r1[c4 * 8 + 6]) * f, __uint_as_float(r1[c4 * 8 + 7]) * f);
-                    dst[4 + c4] = a;
+                if (ktok >= 0) {
+                    store_scaled32(dst + 8 * hq, r0, f);
+                    store_scaled32(dst + 8 * hq + 4, r1, f);
                 }
             }
             ++kuse;
@@ -596,7 +706,14 @@ cudaError_t read_bwd_kv64_status(int* timed_out) {
     return e;
 }
 
-bool bwd_kv64_supported(const Geo& g) { return g.d == 64 && g.w <= 32 && g.nmax <= 1024 && g.heads <= 148; }
+namespace {
+bool no_tma_env() {
+    static const bool off = [] { const char* e_ = std::getenv("TERRA_NO_TMA"); return e_ && e_[0] == '1'; }();
+    return off;
+}
+}  // namespace
+
+bool bwd_kv64_supported(const Geo& g) { return (g.d == 64 || g.d == 128) && g.w <= 32 && g.nmax <= 1024 && g.heads <= 148; }
 
 // `prep` = the prepared bias tables of the head-dim-64 forward kernel (kBiasFloats per head), filled by the caller
 cudaError_t launch_bwd_kv64(const Geo& g, const void* q, const void* k, const void* v, const void* d_o, const float* prep,
@@ -606,12 +723,19 @@ cudaError_t launch_bwd_kv64(const Geo& g, const void* q, const void* k, const vo
     long long cph = sm_count / g.heads;
     if (cph < 1) cph = 1;
     if (cph > items) cph = items;
-    cudaError_t e = cudaFuncSetAttribute(swin_bwd_kv64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    KvMaps64 maps;
+    std::memset(&maps, 0, sizeof maps);
+    const bool tma = !no_tma_env() && bulk_rows_shape(g) && make_row_maps3(&maps.q, g, q, g.ts) && make_row_maps3(&maps.k, g, k, g.ts) &&
+                     make_row_maps3(&maps.v, g, v, g.ts) && make_row_maps3(&maps.g, g, d_o, g.heads * g.d);
+    auto kern = g.d == 64 ? (tma ? swin_bwd_kv64_kernel<64, true> : swin_bwd_kv64_kernel<64, false>)
+                          : (tma ? swin_bwd_kv64_kernel<128, true> : swin_bwd_kv64_kernel<128, false>);
+    const int smem_bytes = g.d == 64 ? Lay<64>::kSmemBytes : Lay<128>::kSmemBytes;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
     if (e != cudaSuccess) return e;
     prof_begin("swin_bwd_kv64_kernel", stream);
-    swin_bwd_kv64_kernel<<<(unsigned)(cph * g.heads), kThreads, kSmemBytes, stream>>>(
+    kern<<<(unsigned)(cph * g.heads), kThreads, smem_bytes, stream>>>(
         g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)d_o, prep, lse, delta,
-        (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, items, (int)cph, max_tiles);
+        (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, items, (int)cph, max_tiles, maps);
     count_launch(stream);
     return cudaGetLastError();
 }

@@ -540,14 +540,16 @@ cudaError_t TERRA_ELEM_FN(launch_bwd_mma)(const Geo& g, const void* q, const voi
                            bool query_side_only) {
     cudaError_t e = cudaMemsetAsync(dbias, 0, sizeof(float) * (size_t)(2 * g.w - 1) * (2 * g.w - 1) * g.heads, stream);
     if (e != cudaSuccess) return e;
+    if (query_side_only) {    // dK, dV come from another kernel
+        if (g.d == 128) return launch_one<128, false>(g, q, k, v, d_o, bias, lse, delta, dq, nullptr, dbias, sm_count, stream);
+        return g.d == 32 ? launch_one<32, false>(g, q, k, v, d_o, bias, lse, delta, dq, nullptr, dbias, sm_count, stream)
+                         : launch_one<64, false>(g, q, k, v, d_o, bias, lse, delta, dq, nullptr, dbias, sm_count, stream);
+    }
     if (g.d == 128) {
         e = launch_one<128, true>(g, q, k, v, d_o, bias, lse, delta, dk, dv, nullptr, sm_count, stream);
         if (e != cudaSuccess) return e;
         return launch_one<128, false>(g, q, k, v, d_o, bias, lse, delta, dq, nullptr, dbias, sm_count, stream);
     }
-    if (query_side_only)      // dK, dV come from another kernel
-        return g.d == 32 ? launch_one<32, false>(g, q, k, v, d_o, bias, lse, delta, dq, nullptr, dbias, sm_count, stream)
-                         : launch_one<64, false>(g, q, k, v, d_o, bias, lse, delta, dq, nullptr, dbias, sm_count, stream);
     if (g.d == 32) {
         e = launch_one<32, true>(g, q, k, v, d_o, bias, lse, delta, dk, dv, nullptr, sm_count, stream);
         if (e != cudaSuccess) return e;

@@ -26,6 +26,7 @@
 #include "swin_common.cuh"
 #include "swin_kernels.h"
 #include "tc_common.cuh"
+#include "tma_rows.cuh"
 
 namespace terra {
 
@@ -846,6 +847,12 @@ bool make_row_map(void* map, const Geo& g, const void* base, int token_stride, i
     const cuuint32_t estr[2] = {1u, 1u};
     return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool make_row_maps3(RowMaps3* maps, const Geo& g, const void* base, int token_stride) {
+    for (int i = 0; i < 3; ++i)
+        if (!make_row_map(&maps->m[i], g, base, token_stride, 32 >> i)) return false;
+    return true;
 }
 
 size_t fwd_tc_workspace_bytes(const Geo& g) { return (size_t)g.heads * kFwdBiasFloats * sizeof(float); }

@@ -20,13 +20,13 @@
 // in place by bf16 P (64 columns); the O accumulator (64 + 16 columns) at +128.
 // Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, all roles leave their loops, TMEM is
 // released and the host reads the device status word.  Every role follows every ring item by item.
-#include <cuda.h>
 #include <cstdlib>
 #include <cstring>
 
 #include "swin_common.cuh"
 #include "swin_kernels.h"
 #include "tc_common.cuh"
+#include "tma_rows.cuh"
 
 namespace terra {
 
@@ -259,11 +259,6 @@ __device__ __forceinline__ void max_cols(const uint32_t (&r)[N], float (&mx)[4])
     }
 }
 
-// tensor maps over the token stream of one tensor ([tokens, heads * d], 64-byte-swizzled boxes of 32 columns) with
-// boxes of 32, 16 and 8 tokens
-struct RowMaps3 {
-    CUtensorMap m[3];
-};
 struct FwdMaps64 {
     RowMaps3 q, k, v;
 };
@@ -361,19 +356,7 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             int xb = 0, xwr = 0;
             // the copies of window row `a`, part `part` of a row: w consecutive slots from `dst` on
             auto copy_row = [&](const RowMaps3& m3, uint32_t dst, int a, int part, uint32_t bar) {
-                int u = xwr * g.w + a + g.sh;
-                if (u >= g.H) u -= g.H;
-                const int y0 = (xb * g.H + u) * g.W, xc = head * D + part * 32;
-                const int n1 = min(g.w, g.W - v0);            // tokens up to the seam; the rest starts at column 0
-                int y = y0 + v0, n = n1;
-#pragma unroll
-                for (int seg = 0; seg < 2; ++seg) {
-                    if (n >= 32) { tma_load_2d(dst, &m3.m[0], xc, y, bar); dst += 32 * kPartBytes; y += 32; n -= 32; }
-                    if (n >= 16) { tma_load_2d(dst, &m3.m[1], xc, y, bar); dst += 16 * kPartBytes; y += 16; n -= 16; }
-                    if (n >= 8) { tma_load_2d(dst, &m3.m[2], xc, y, bar); dst += 8 * kPartBytes; }
-                    y = y0;
-                    n = g.w - n1;
-                }
+                bulk_copy_window_row(m3, dst, g, xb, xwr, v0, a, head * D + part * 32, bar);
             };
             int kuse = 0;
             long long ru = 0;
@@ -978,13 +961,8 @@ cudaError_t launch_fwd_tc64(const Geo& g, const void* q, const void* k, const vo
     FwdMaps64 maps;
     std::memset(&maps, 0, sizeof maps);
     static const bool tma_off = [] { const char* e_ = std::getenv("TERRA_NO_TMA"); return e_ && e_[0] == '1'; }();
-    bool tma = !tma_off && (g.w == 16 || g.w == 32) && g.H % g.w == 0 && g.W % g.w == 0 && g.sw % 8 == 0 &&
-               (long long)g.B * g.H * g.W < 0x7fffffffLL;
-    for (int i = 0; i < 3 && tma; ++i) {
-        const int box = 32 >> i;
-        tma = make_row_map(&maps.q.m[i], g, q, g.ts, box) && make_row_map(&maps.k.m[i], g, k, g.ts, box) &&
-              make_row_map(&maps.v.m[i], g, v, g.ts, box);
-    }
+    const bool tma = !tma_off && bulk_rows_shape(g) && make_row_maps3(&maps.q, g, q, g.ts) && make_row_maps3(&maps.k, g, k, g.ts) &&
+                     make_row_maps3(&maps.v, g, v, g.ts);
     auto kern = g.d == 64 ? (tma ? swin_fwd_tc64_kernel<64, true> : swin_fwd_tc64_kernel<64, false>)
                           : (tma ? swin_fwd_tc64_kernel<128, true> : swin_fwd_tc64_kernel<128, false>);
     const int smem_bytes = g.d == 64 ? Lay<64>::kSmemBytes : Lay<128>::kSmemBytes;

@@ -126,6 +126,16 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t tx)
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(tx) : "memory");
 }
 
+// announces `tx` bytes of asynchronous copies to the barrier's current phase, without arriving
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t tx) {
+    asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(tx) : "memory");
+}
+// this thread's arrival on `bar` (one of the arrivals the barrier was initialised for) happens when the cp.async
+// copies it has issued so far are complete; the thread does not wait
+__device__ __forceinline__ void cp_async_mbar_arrive_noinc(uint32_t bar) {
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];\n" ::"r"(bar) : "memory");
+}
+
 // ---- tcgen05: TMEM allocation -----------------------------------------------------------------------
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_dst), "r"(ncols) : "memory");

@@ -1,0 +1,48 @@
+// Window rows by tiled bulk copies (TMA), shared by the large-window tcgen05 kernels.
+//
+// On a grid of complete windows whose longitude shift is a multiple of 8, the tokens of one window row are one run of
+// consecutive tokens of the tensor, or two where the rolled row crosses the longitude seam, each a multiple of 8 long.
+// A tensor is described as [tokens, heads * d] with boxes of 32 columns (one 64-byte-swizzled part of a row) by 32,
+// 16 or 8 tokens; a run is covered by at most one box of each size.
+#pragma once
+#include <cuda.h>
+
+#include "swin_common.cuh"
+#include "tc_common.cuh"
+
+namespace terra {
+
+struct RowMaps3 {
+    CUtensorMap m[3];     // boxes of 32, 16, 8 tokens
+};
+
+// host: the three maps of one tensor (`token_stride` in elements); false if the driver's encoder is not available
+bool make_row_maps3(RowMaps3* maps, const Geo& g, const void* base, int token_stride);
+
+// host: the geometry the bulk-copy loaders are written for
+inline bool bulk_rows_shape(const Geo& g) {
+    return (g.w == 16 || g.w == 32) && g.H % g.w == 0 && g.W % g.w == 0 && g.sw % 8 == 0 &&
+           (long long)g.B * g.H * g.W < 0x7fffffffLL;
+}
+
+// device: the copies of window row `a` of window row-index `wr` in sample `b`: w slots of 64 bytes from `dst` on
+// (a multiple of 512 bytes into a swizzled region), columns [xc, xc + 32) of every token; `v0` = the window's first
+// token column after the roll.  The bytes are counted on `bar`.
+__device__ __forceinline__ void bulk_copy_window_row(const RowMaps3& m3, uint32_t dst, const Geo& g, int b, int wr, int v0, int a,
+                                                     int xc, uint32_t bar) {
+    int u = wr * g.w + a + g.sh;
+    if (u >= g.H) u -= g.H;
+    const int y0 = (b * g.H + u) * g.W;
+    const int n1 = min(g.w, g.W - v0);            // tokens up to the seam; the rest starts at column 0
+    int y = y0 + v0, n = n1;
+#pragma unroll
+    for (int seg = 0; seg < 2; ++seg) {
+        if (n >= 32) { tc::tma_load_2d(dst, &m3.m[0], xc, y, bar); dst += 32 * 64; y += 32; n -= 32; }
+        if (n >= 16) { tc::tma_load_2d(dst, &m3.m[1], xc, y, bar); dst += 16 * 64; y += 16; n -= 16; }
+        if (n >= 8) { tc::tma_load_2d(dst, &m3.m[2], xc, y, bar); dst += 8 * 64; }
+        y = y0;
+        n = g.w - n1;
+    }
+}
+
+}  // namespace terra
