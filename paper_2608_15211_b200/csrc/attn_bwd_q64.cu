@@ -1,14 +1,15 @@
-// Query side of the backward pass (dQ, dBias) on the tcgen05 tensor cores for head dim 64 and complete 32 x 32
-// windows (window side 32, grid extents multiples of 32).  Other shapes of this regime run the register-tile kernel.
+// Query side of the backward pass (dQ, dBias) on the tcgen05 tensor cores for head dims 64 and 128 and complete
+// 32 x 32 windows (window side 32, grid extents multiples of 32).  Other shapes of this regime run the register-tile kernel.
 //
 // One persistent CTA per SM, bound to one head, walks over a contiguous range of (128-query tile, batch, window)
-// items, the tile index slowest.  The tile's Q and dO rows stay in shared memory; the window's keys stream through a
-// ring of slots in chunks of 128 (K, V rows and per-key bias code, mask label).  TMEM lanes = queries, columns = keys.
-// Per chunk:
-//   S = Q K_c^T, dP = dO V_c^T                                        (SS MMAs, N = 64 keys per half chunk)
+// items, the tile index slowest.  The tile's Q and dO rows stay in shared memory; the window's keys stream through
+// two rings of units of 64 rows, one for K and one for V (with per-key mask labels next to the K units).
+// TMEM lanes = queries, columns = keys.  Per half chunk of 64 keys:
+//   S = Q K_c^T, dP = dO V_c^T                                        (SS MMAs, N = 64 keys)
 //   P = exp2(S scale + bias - lse_q), dS = P (dP - delta_q)           (elementwise warps, one query row per thread;
 //                                                                      dS written back over dP as bf16)
-//   dQ += dS K_c                                                      (A from TMEM, B = the chunk's rows, MN-major)
+//   dQ += dS K_c                                                      (A from TMEM, B = the unit's rows, MN-major)
+// The V unit is free again when the dP product is complete, the K unit after the dQ product.
 // dBias: a warp's 32 lanes are the 32 queries of one window row (a_q fixed, b_q = lane), so for one key column the
 // lanes update 32 consecutive entries of the row a_q - a_k of the table.  Each TMEM lane quarter owns a private
 // shared-memory table [a_k][b_q - b_k + 31] and updates it with plain load-add-store.  A key chunk is four columns
@@ -18,19 +19,23 @@
 // the tile index is the slowest digit of the item order, a_q = 4 tile + quarter changes at most once or twice per
 // CTA; the tables are added to the global gradient (float atomics) at each change and at the end.
 // Roles: warps 0-7 elementwise (warps w and w + 4 share lane quarter w & 3 and take the chunk's first / second 64 key
-// columns), warp 8 issues every MMA, warps 9-11 gather rows with cp.async.  Head dim 64 is kept as two 32-column
-// halves in the 64-byte-swizzled operand layout (lo | hi regions).
-// A chunk's two 64-key halves are separate units of work ("half chunks", 16 per item, numbered through the whole
-// run); half chunk n belongs to elementwise warps 4 (n % 2) .. 4 (n % 2) + 3 and lives in TMEM buffer n % 3 (S in the
-// buffer's first 64 columns, dP in the second).  With three buffers for two groups of warps the scores of a group's
-// next half chunk are issued while it still works on the current one (as soon as the other group's previous half
-// chunk has been consumed), so the MMA round trip is hidden behind the elementwise work.
-// TMEM columns: buffers 0..127, 128..255, 256..383; dQ 384..447.
+// columns), warp 8 issues every MMA, warps 9-11 gather rows with cp.async.  A row is kept as head dim / 32 parts of 32
+// columns in the 64-byte-swizzled operand layout.
+// Half chunks are the units of work (16 per item, numbered through the whole run); half chunk n belongs to
+// elementwise warps 4 (n % 2) .. 4 (n % 2) + 3 and lives in TMEM buffer n % 3 (S in the buffer's first 64 columns, dP
+// in the second).  With three buffers for two groups of warps the scores of a group's next half chunk are issued
+// while it still works on the current one (as soon as the other group's previous half chunk has been consumed), so
+// the MMA round trip is hidden behind the elementwise work.
+// TMEM columns: buffers 0..127, 128..255, 256..383; dQ from 384 on (head dim columns).
 // Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, all roles leave their loops, TMEM is
 // released and the host reads the device status word.  Every role follows every ring item by item.
 #include "swin_common.cuh"
 #include "swin_kernels.h"
 #include "tc_common.cuh"
+#include "tma_rows.cuh"
+
+#include <cstdlib>
+#include <cstring>
 
 namespace terra {
 
@@ -49,34 +54,48 @@ constexpr int kWorkThreads = 256;
 constexpr int kRegsLaunch = 168, kRegsWork = 192, kRegsOther = 112;
 static_assert(2 * (kRegsWork - kRegsLaunch) <= (kRegsLaunch - kRegsOther), "register hand-over does not balance");
 
-constexpr int kD = 64;
 constexpr int kW = 32;                                // window side
-constexpr int kHalfBytes = 64;
+constexpr int kPartBytes = 64;                        // one 32-column part of a row
 constexpr int kTile = 128;                            // queries per item, keys per chunk
-constexpr int kHalf = kTile * kHalfBytes;             // 8192: one 32-column half of 128 rows
+constexpr int kPart = kTile * kPartBytes;             // 8192: the region of one 32-column part of the 128 query rows
+constexpr int kUPart = 64 * kPartBytes;               // 4096: ... of the 64 key rows of a half chunk
 constexpr int kTiles = kW * kW / kTile;               // 8 query tiles = 8 key chunks per window
-constexpr int kQStages = 2, kSlots = 3;
-// query stage: Q lo | Q hi | dO lo | dO hi, then per query row: 4 * bias code, label, token, lse, delta
-constexpr int kOffQlo = 0, kOffGlo = 2 * kHalf;     // hi halves follow at + kHalf
-constexpr int kRows = 4 * kHalf;                      // 32768
-constexpr int kOffQCode = kRows, kOffQLab = kRows + 512, kOffQTok = kRows + 1024, kOffQLse = kRows + 1536, kOffQDelta = kRows + 2048;
-constexpr int kQStageBytes = kRows + 3072;
-// key slot: K lo | K hi | V lo | V hi, then per key column: label
-constexpr int kOffKlo = 0, kOffVlo = 2 * kHalf;     // hi halves follow at + kHalf
-constexpr int kOffKLab = kRows;
-constexpr int kSlotBytes = kRows + 1024;
-constexpr int kOffSlots = kQStages * kQStageBytes;
 constexpr int kBiasFloats = 6048;
-constexpr int kOffBias = kOffSlots + kSlots * kSlotBytes;
-// bias-gradient tables: per lane quarter [a_k 32][b_q - b_k + 31, padded to 64]
-constexpr int kTabFloats = kW * 64;
-constexpr int kOffTab = kOffBias + kBiasFloats * 4;
-constexpr int kOffBars = ((kOffTab + 4 * kTabFloats * 4 + 1023) / 1024) * 1024;
-constexpr int kSmemBytes = kOffBars + 1024;
-static_assert(kQStageBytes % 1024 == 0 && kSlotBytes % 1024 == 0, "tiles keep the swizzle alignment");
-static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
+constexpr int kTabFloats = kW * 64;                   // bias-gradient tables: per lane quarter [a_k 32][b_q - b_k + 31, padded to 64]
 constexpr int kBufCols = 128, kColDQ = 384;           // buffer b: S at 128 b, dP at 128 b + 64
 constexpr int kHalfChunks = 2 * kTiles;               // per item
+
+// Shared-memory plan per head dim D (64 or 128): a row is kept as D / 32 parts of 32 columns, each part a region in
+// the 64-byte-swizzled operand layout.  The keys of a half chunk arrive as two units, its 64 K rows and its 64 V rows,
+// in rings of their own: a V unit is free again as soon as the half chunk's dP product is complete, a K unit only
+// after its dQ product.  Head dim 64: two query stages, six K and six V units; head dim 128: one stage, four K and
+// two V units.
+template <int D>
+struct Lay {
+    static constexpr int kParts = D / 32;
+    static constexpr int kQStages = D == 64 ? 2 : 1;
+    static constexpr int kKUnits = D == 64 ? 6 : 4, kVUnits = D == 64 ? 6 : 2;
+    // query stage: Q parts | dO parts, then per query row: 4 * bias code, label, token, lse, delta
+    static constexpr int kOffQ = 0, kOffG = kParts * kPart;
+    static constexpr int kRows = 2 * kParts * kPart;
+    static constexpr int kOffQCode = kRows, kOffQLab = kRows + 512, kOffQTok = kRows + 1024, kOffQLse = kRows + 1536, kOffQDelta = kRows + 2048;
+    static constexpr int kQStageBytes = kRows + 3072;
+    static constexpr int kUnitBytes = kParts * kUPart;
+    static constexpr int kOffKRing = kQStages * kQStageBytes;
+    static constexpr int kOffVRing = kOffKRing + kKUnits * kUnitBytes;
+    static constexpr int kOffKLab = kOffVRing + kVUnits * kUnitBytes;               // per K unit: the 64 keys' mask labels
+    static constexpr int kOffBias = kOffKLab + ((kKUnits * 256 + 1023) / 1024) * 1024;
+    static constexpr int kOffTab = kOffBias + kBiasFloats * 4;
+    static constexpr int kOffBars = ((kOffTab + 4 * kTabFloats * 4 + 1023) / 1024) * 1024;
+    static constexpr int kSmemBytes = kOffBars + 1024;
+    // the loader fetches this many half chunks of the next item before its query rows (with one query stage those can
+    // only follow when the item before is complete, and the keys should not wait for that)
+    static constexpr int kKeysFirst = kQStages == 1 ? 2 : 0;
+    static_assert(kQStageBytes % 1024 == 0 && kUnitBytes % 1024 == 0, "tiles keep the swizzle alignment");
+    static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
+    static_assert(kColDQ + D <= 512, "tensor memory columns");
+    static_assert(kKeysFirst <= kVUnits && kKeysFirst < kKUnits, "the keys fetched first must fit their rings");
+};
 
 constexpr int kCodeStride = kW + 32;
 constexpr int kC0 = (kW - 1) * (kCodeStride + 1);
@@ -154,15 +173,16 @@ __device__ __forceinline__ int lds_i32(uint32_t addr) {
 // the entry of column c; the following columns are the following key rows, one table row further each).
 // `bias_grp` = address of the bias entry of column c: the group's columns are 16 consecutive key rows at one b_k, so
 // the following entries lie one code stride below each (no per-key table is read for them).
+// `lab_a` = shared address of the mask label of the chunk's key column 0 (as if the table had all 128 columns).
 template <bool MASKED>
 __device__ __forceinline__ void cols16(const uint32_t (&rs)[16], const uint32_t (&rp)[16], int c, uint32_t bias_grp, int qlabel,
-                                       float l2, float dl, uint32_t sl_a, float scale, uint32_t tab, uint32_t (&pk_ds)[8]) {
+                                       float l2, float dl, uint32_t lab_a, float scale, uint32_t tab, uint32_t (&pk_ds)[8]) {
     int kl[16];
     float bv[16], tv[16];
     if (MASKED) {
 #pragma unroll
         for (int e4 = 0; e4 < 4; ++e4) {
-            const int4 k4 = lds_i4(sl_a + kOffKLab + 4 * (c + e4 * 4));
+            const int4 k4 = lds_i4(lab_a + 4 * (c + e4 * 4));
             kl[e4 * 4] = k4.x; kl[e4 * 4 + 1] = k4.y; kl[e4 * 4 + 2] = k4.z; kl[e4 * 4 + 3] = k4.w;
         }
     }
@@ -185,25 +205,44 @@ __device__ __forceinline__ void cols16(const uint32_t (&rs)[16], const uint32_t 
     __syncwarp();                                         // the next group's entries are this group's, one lane over
 }
 
+struct QMaps64 {
+    RowMaps3 q, g;            // query rows and their output gradients, by window rows
+    CUtensorMap k, v;         // keys by runs of 16 vertically adjacent tokens
+};
+
+// TMA: both shifts are multiples of 16 (8 suffices for the longitude): one loader warp fetches the query rows window
+// row by window row and the key units as four runs of 16 vertically adjacent tokens with tiled bulk copies (per-query
+// lse and delta by 4-byte cp.async copies tied to the same barrier); otherwise three loader warps gather every row
+// with 16-byte cp.async copies.
+template <int D, bool TMA>
 __global__ void __launch_bounds__(kThreads, 1)
 swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                     const __nv_bfloat16* __restrict__ v, const __nv_bfloat16* __restrict__ d_o,
                     const float* __restrict__ bias_prep, const float* __restrict__ lse, const float* __restrict__ delta,
-                    __nv_bfloat16* __restrict__ dq, float* __restrict__ dbias, long long items_per_head, int ctas_per_head) {
+                    __nv_bfloat16* __restrict__ dq, float* __restrict__ dbias, long long items_per_head, int ctas_per_head,
+                    const __grid_constant__ QMaps64 maps) {
+    using L = Lay<D>;
+    constexpr int kParts = L::kParts, kQStages = L::kQStages, kKUnits = L::kKUnits, kVUnits = L::kVUnits;
+    constexpr int kOffQ = L::kOffQ, kOffG = L::kOffG, kOffQCode = L::kOffQCode, kOffQLab = L::kOffQLab, kOffQTok = L::kOffQTok;
+    constexpr int kOffQLse = L::kOffQLse, kOffQDelta = L::kOffQDelta, kQStageBytes = L::kQStageBytes, kUnitBytes = L::kUnitBytes;
+    constexpr int kOffKRing = L::kOffKRing, kOffVRing = L::kOffVRing, kOffKLab = L::kOffKLab, kOffBias = L::kOffBias;
+    constexpr int kOffTab = L::kOffTab, kOffBars = L::kOffBars;
     extern __shared__ __align__(1024) unsigned char smem[];
     const uint32_t smem0 = smem_u32(smem);
     const uint32_t bar0 = smem0 + kOffBars;
     auto bar_qfull = [&](int s) { return bar0 + 8u * s; };               // the tile's Q, dO rows and row tables are there
     auto bar_qempty = [&](int s) { return bar0 + 8u * (2 + s); };        // ... and no longer needed
-    // the ring is handed over in half slots: half chunk number p sits in rows 64 (p % 2) .. of slot (p / 2) % 3
-    auto bar_kfull = [&](int hs) { return bar0 + 8u * (4 + hs); };       // half slot hs = p % 6 holds its 64 keys
-    auto bar_kempty = [&](int hs) { return bar0 + 8u * (10 + hs); };     // ... and every MMA that reads them is complete
+    // half chunk number p has its K rows in unit p % kKUnits of the K ring and its V rows in unit p % kVUnits of the V ring
+    auto bar_kfull = [&](int u) { return bar0 + 8u * (4 + u); };
+    auto bar_kempty = [&](int u) { return bar0 + 8u * (10 + u); };       // every MMA that reads the unit is complete
+    auto bar_vfull = [&](int u) { return bar0 + 8u * (25 + u); };
+    auto bar_vempty = [&](int u) { return bar0 + 8u * (31 + u); };
     auto bar_sdp = [&](int b) { return bar0 + 8u * (16 + b); };          // S and dP of a half chunk are in TMEM buffer b
     auto bar_ds = [&](int b) { return bar0 + 8u * (19 + b); };           // bf16 dS of the half chunk is in TMEM buffer b
     const uint32_t bar_acc = bar0 + 8u * 22;                              // dQ of the item is final
     const uint32_t bar_accfree = bar0 + 8u * 23;                          // ... and has been read
     const uint32_t bar_flush = bar0 + 8u * 24;                            // the elementwise warps meet around a table flush
-    unsigned char* tail = smem + kOffBars + 8 * 25;
+    unsigned char* tail = smem + kOffBars + 8 * 37;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail);
     volatile int* cta_abort = reinterpret_cast<volatile int*>(tail + 8);
 
@@ -216,12 +255,16 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
 
     if (tid == 0) {
         for (int s = 0; s < kQStages; ++s) {
-            mbar_init(bar_qfull(s), kLoaderThreads);
+            mbar_init(bar_qfull(s), TMA ? 32 : kLoaderThreads);
             mbar_init(bar_qempty(s), 1 + kWorkThreads);    // the issuer's commit + every elementwise thread
         }
-        for (int hs = 0; hs < 2 * kSlots; ++hs) {
-            mbar_init(bar_kfull(hs), kLoaderThreads);
-            mbar_init(bar_kempty(hs), 1);
+        for (int u = 0; u < kKUnits; ++u) {
+            mbar_init(bar_kfull(u), TMA ? 32 : kLoaderThreads);
+            mbar_init(bar_kempty(u), 1);
+        }
+        for (int u = 0; u < kVUnits; ++u) {
+            mbar_init(bar_vfull(u), TMA ? 32 : kLoaderThreads);
+            mbar_init(bar_vempty(u), 1);
         }
         for (int b = 0; b < 3; ++b) {
             mbar_init(bar_sdp(b), 1);
@@ -250,41 +293,151 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
 
     if (warp >= kMmaWarp) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;\n" ::"n"(kRegsOther));
-    if (warp >= kLoaderWarp0) {
+    if (TMA && warp >= kLoaderWarp0) {
+        // ------------------------------------------------------------------ loader warp (TMA); the other two have no work
+        if (warp == kLoaderWarp0) {
+            int quse = 0;
+            unsigned ru = 0;                              // half chunks so far
+            bool ok = true;
+            // the K unit, then the V unit, of half chunk n of the window at `cw`: rows 16 i .. 16 i + 15 of a unit are
+            // the tokens of window rows 16 (n % 2) .. + 15 in window column 4 (n / 2) + i
+            auto load_half = [&](const Cursor& cw, int n) -> bool {
+                const int c = n >> 1, h = n & 1;
+                int u0 = cw.wr * kW + 16 * h + g.sh;
+                if (u0 >= g.H) u0 -= g.H;
+                const int z = cw.b * g.H + u0;
+                const int i = lane / kParts, part = lane - i * kParts;      // this lane's run and part (lanes < 4 * kParts)
+                int vcol = cw.wc * kW + 4 * c + i + g.sw;
+                if (vcol >= g.W) vcol -= g.W;
+                const uint32_t uoff = part * kUPart + i * 16 * kPartBytes;
+                const int uk = (int)(ru % kKUnits), uv = (int)(ru % kVUnits);
+                if (!mbar_wait_all(bar_kempty(uk), (uint32_t)((ru / kKUnits) & 1) ^ 1u, cta_abort)) return false;
+                for (int r = lane; r < 64; r += 32) {
+                    int code, label;
+                    slot_token(g, cw, chunk_slot(c, 64 * h + r), code, label);
+                    reinterpret_cast<int*>(smem + kOffKLab + uk * 256)[r] = label;
+                }
+                if (lane < 4 * kParts) tma_load_3d(smem0 + kOffKRing + uk * kUnitBytes + uoff, &maps.k, head * D + part * 32, vcol, z, bar_kfull(uk));
+                if (lane == 0) mbar_arrive_expect_tx(bar_kfull(uk), (uint32_t)(64 * D * 2));
+                else mbar_arrive(bar_kfull(uk));
+                if (!mbar_wait_all(bar_vempty(uv), (uint32_t)((ru / kVUnits) & 1) ^ 1u, cta_abort)) return false;
+                if (lane < 4 * kParts) tma_load_3d(smem0 + kOffVRing + uv * kUnitBytes + uoff, &maps.v, head * D + part * 32, vcol, z, bar_vfull(uv));
+                if (lane == 0) mbar_arrive_expect_tx(bar_vfull(uv), (uint32_t)(64 * D * 2));
+                else mbar_arrive(bar_vfull(uv));
+                ++ru;
+                return true;
+            };
+            Cursor cur = cursor_at(g, it_lo);
+            int fetched = 0;                              // half chunks of the current item already fetched
+            for (long long it = it_lo; ok && it < it_hi; ++it, ++quse) {
+                const int qs = quse % kQStages;
+                ok = mbar_wait_all(bar_qempty(qs), ((quse / kQStages) & 1) ^ 1, cta_abort);
+                if (!ok) break;
+                const size_t sample_off = (size_t)cur.b * HW;
+                // ---- the query tile: Q, dO rows and the row tables
+                {
+                    unsigned char* st = smem + qs * kQStageBytes;
+                    const uint32_t sb = smem0 + qs * kQStageBytes;
+                    const int slot0 = cur.qt * kTile;
+                    for (int row = lane; row < kTile; row += 32) {
+                        int code, label;
+                        const int tok = slot_token(g, cur, slot0 + row, code, label);
+                        const size_t li = (sample_off + (size_t)tok) * g.heads + head;
+                        reinterpret_cast<int*>(st + kOffQCode)[row] = 4 * code;
+                        reinterpret_cast<int*>(st + kOffQLab)[row] = label;
+                        reinterpret_cast<int*>(st + kOffQTok)[row] = tok;
+                        cp_async4(sb + kOffQLse + 4 * row, lse + li);
+                        cp_async4(sb + kOffQDelta + 4 * row, delta + li);
+                    }
+                    int v0 = cur.wc * kW + g.sw;
+                    if (v0 >= g.W) v0 -= g.W;
+                    constexpr int kPerTensor = (kTile / kW) * kParts;
+                    for (int i = lane; i < 2 * kPerTensor; i += 32) {
+                        const int tsr = i >= kPerTensor ? 1 : 0, rem = i - tsr * kPerTensor;
+                        const int ar = rem / kParts, part = rem - ar * kParts;
+                        bulk_copy_window_row(tsr ? maps.g : maps.q, sb + (tsr ? kOffG : kOffQ) + part * kPart + ar * kW * kPartBytes, g,
+                                             cur.b, cur.wr, v0, cur.qt * (kTile / kW) + ar, head * D + part * 32, bar_qfull(qs));
+                    }
+                    if (lane == 0) mbar_expect_tx(bar_qfull(qs), (uint32_t)(kTile * D * 2 * 2));
+                    // the lane's arrival: when its lse / delta copies have landed (its table entries were written before)
+                    cp_async_mbar_arrive_noinc(bar_qfull(qs));
+                }
+                // ---- the window's keys, half chunk by half chunk; then the first ones of the next item
+                for (int n = fetched; n < kHalfChunks && ok; ++n) ok = load_half(cur, n);
+                if (!ok) break;
+                cursor_next(g, cur);
+                fetched = 0;
+                if (it + 1 < it_hi)
+                    for (; fetched < L::kKeysFirst && ok; ++fetched) ok = load_half(cur, fetched);
+            }
+        }
+    } else if (warp >= kLoaderWarp0) {
         // ------------------------------------------------------------------ loaders
         const int lt = (warp - kLoaderWarp0) * 32 + lane;
-        // Eight lanes per row, one 16-byte piece of the row's 128 bytes each (pieces 0-3: the lo half, 4-7: the hi
-        // half), twelve rows per step: a warp's copy instruction reads four whole rows.
-        const int piece = lt & 7, rsub = lt >> 3;
-        constexpr int kRowsPerStep = kLoaderThreads / 8;      // 12
-        const uint32_t piece_off = (uint32_t)(piece >> 2) * kHalf;
+        // D / 8 lanes per row, one 16-byte piece of the row each (pieces 4 p .. 4 p + 3: the row's part p): a warp's
+        // copy instruction reads whole rows.
+        constexpr int kPieces = D / 8;
+        const int piece = lt % kPieces, rsub = lt / kPieces;
+        constexpr int kRowsPerStep = kLoaderThreads / kPieces;
+        const uint32_t q_piece_off = (uint32_t)(piece >> 2) * kPart;      // the piece's part in a query stage
+        const uint32_t u_piece_off = (uint32_t)(piece >> 2) * kUPart;     // ... in a key unit
         int quse = 0;
-        long long ru = 0;                                 // half chunks so far
-        uint32_t pending_bar = 0;                         // barrier of the group in flight
+        unsigned ru = 0;                                  // half chunks so far (a CTA sees far fewer than 2^32)
+        uint32_t pending_bar = 0, pending_bar2 = 0;       // barriers of the group of copies in flight (the second may be 0)
         bool ok = true;
-        auto publish = [&]() {
-            cp_async_wait<0>();
+        auto arrive_pending = [&]() {
             fence_proxy_async();
             mbar_arrive(pending_bar);
-            pending_bar = 0;
+            if (pending_bar2) mbar_arrive(pending_bar2);
+            pending_bar = pending_bar2 = 0;
         };
-        // no free place yet: the group in flight is published first
+        // no free place yet: the group in flight is published first, or the consumers could never free one
         auto acquire = [&](uint32_t bar, uint32_t parity) -> bool {
-            if (pending_bar && !__all_sync(0xffffffffu, mbar_test_wait(bar, parity))) publish();
+            if (pending_bar && !__all_sync(0xffffffffu, mbar_test_wait(bar, parity))) {
+                cp_async_wait<0>();
+                arrive_pending();
+            }
             return mbar_wait_all(bar, parity, cta_abort);
         };
         // a group is published when the next one has been issued
-        auto issued = [&](uint32_t bar) {
+        auto issued = [&](uint32_t bar, uint32_t bar2) {
             cp_async_commit();
             if (pending_bar) {
                 cp_async_wait<1>();
-                fence_proxy_async();
-                mbar_arrive(pending_bar);
+                arrive_pending();
             }
             pending_bar = bar;
+            pending_bar2 = bar2;
+        };
+        // the K and V rows of half chunk n of the window at `cw`, one group of copies
+        auto load_half = [&](const Cursor& cw, int n) -> bool {
+            const size_t sample_off = (size_t)cw.b * HW;
+            const int c = n >> 1, row0 = 64 * (n & 1);
+            const int uk = (int)(ru % kKUnits), uv = (int)(ru % kVUnits);
+            if (!acquire(bar_kempty(uk), (uint32_t)((ru / kKUnits) & 1) ^ 1u)) return false;
+            if (!acquire(bar_vempty(uv), (uint32_t)((ru / kVUnits) & 1) ^ 1u)) return false;
+            const uint32_t kb = smem0 + kOffKRing + uk * kUnitBytes + u_piece_off;
+            const uint32_t vb = smem0 + kOffVRing + uv * kUnitBytes + u_piece_off;
+#pragma unroll
+            for (int step = 0; step < (64 + kRowsPerStep - 1) / kRowsPerStep; ++step) {
+                const int r = rsub + kRowsPerStep * step;
+                if (r < 64) {
+                    int code, label;
+                    const int tok = slot_token(g, cw, chunk_slot(c, row0 + r), code, label);
+                    if (piece == 0) reinterpret_cast<int*>(smem + kOffKLab + uk * 256)[r] = label;
+                    const size_t off = (sample_off + (size_t)tok) * g.ts + head * D + piece * 8;
+                    const uint32_t so = tile_off<32>(r, piece & 3);
+                    cp_async16(kb + so, k + off, 16);
+                    cp_async16(vb + so, v + off, 16);
+                }
+            }
+            issued(bar_kfull(uk), bar_vfull(uv));
+            ++ru;
+            return true;
         };
         Cursor cur = cursor_at(g, it_lo);
-        for (long long it = it_lo; ok && it < it_hi; ++it, cursor_next(g, cur), ++quse) {
+        int fetched = 0;                                  // half chunks of the current item already fetched
+        for (long long it = it_lo; ok && it < it_hi; ++it, ++quse) {
             const int qs = quse % kQStages;
             ok = acquire(bar_qempty(qs), ((quse / kQStages) & 1) ^ 1);
             if (!ok) break;
@@ -292,7 +445,7 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
             // ---- the query tile: Q, dO rows and the row tables
             {
                 unsigned char* st = smem + qs * kQStageBytes;
-                const uint32_t sb = smem0 + qs * kQStageBytes + piece_off;
+                const uint32_t sb = smem0 + qs * kQStageBytes + q_piece_off;
                 const int slot0 = cur.qt * kTile;
 #pragma unroll 1
                 for (int step = 0; step < (kTile + kRowsPerStep - 1) / kRowsPerStep; ++step) {
@@ -310,42 +463,28 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
                             cp_async4(smem0 + qs * kQStageBytes + kOffQDelta + 4 * row, delta + li);
                         }
                         const uint32_t so = tile_off<32>(row, piece & 3);
-                        cp_async16(sb + kOffQlo + so, q + (sample_off + (size_t)tok) * g.ts + head * kD + piece * 8, 16);
-                        cp_async16(sb + kOffGlo + so, d_o + li * kD + piece * 8, 16);
+                        cp_async16(sb + kOffQ + so, q + (sample_off + (size_t)tok) * g.ts + head * D + piece * 8, 16);
+                        cp_async16(sb + kOffG + so, d_o + li * D + piece * 8, 16);
                     }
                 }
-                issued(bar_qfull(qs));
+                issued(bar_qfull(qs), 0);
             }
-            // ---- the window's keys, half chunk by half chunk
-            for (int n = 0; n < kHalfChunks; ++n, ++ru) {
-                const int hs = (int)(ru % (2 * kSlots));
-                ok = acquire(bar_kempty(hs), (uint32_t)((ru / (2 * kSlots)) & 1) ^ 1u);
-                if (!ok) break;
-                unsigned char* sl = smem + kOffSlots + (hs >> 1) * kSlotBytes;
-                const uint32_t sb = smem0 + kOffSlots + (hs >> 1) * kSlotBytes + piece_off;
-                const int c = n >> 1, row0 = 64 * (n & 1);
-#pragma unroll
-                for (int step = 0; step < (64 + kRowsPerStep - 1) / kRowsPerStep; ++step) {
-                    const int r = rsub + kRowsPerStep * step;
-                    if (r < 64) {
-                        const int row = row0 + r;
-                        int code, label;
-                        const int tok = slot_token(g, cur, chunk_slot(c, row), code, label);
-                        if (piece == 0) reinterpret_cast<int*>(sl + kOffKLab)[row] = label;
-                        const size_t off = (sample_off + (size_t)tok) * g.ts + head * kD + piece * 8;
-                        const uint32_t so = tile_off<32>(row, piece & 3);
-                        cp_async16(sb + kOffKlo + so, k + off, 16);
-                        cp_async16(sb + kOffVlo + so, v + off, 16);
-                    }
-                }
-                issued(bar_kfull(hs));
-            }
+            // ---- the window's keys, half chunk by half chunk; then the first ones of the next item
+            for (int n = fetched; n < kHalfChunks && ok; ++n) ok = load_half(cur, n);
+            if (!ok) break;
+            cursor_next(g, cur);
+            fetched = 0;
+            if (it + 1 < it_hi)
+                for (; fetched < L::kKeysFirst && ok; ++fetched) ok = load_half(cur, fetched);
         }
-        if (pending_bar) publish();
+        if (pending_bar) {
+            cp_async_wait<0>();
+            arrive_pending();
+        }
     } else {
         // ------------------------------------------------------------------ MMA issuer
         const uint32_t idesc_s = make_idesc_bf16(128, 64, 0, 0);
-        const uint32_t idesc_acc = make_idesc_bf16(128, kD, 0, 1);       // A from TMEM, B = 16 rows x 64 (MN-major)
+        const uint32_t idesc_acc = make_idesc_bf16(128, D, 0, 1);        // A from TMEM, B = 16 rows x D (MN-major)
         const uint32_t sd_hi = sdesc_hi(make_sdesc_sw64(smem0, 512));    // common high word of the K-major descriptors
         int quse = 0;
         bool ok = true;
@@ -355,34 +494,42 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
             if (!ok) break;
             fence_proxy_async();
             const uint32_t qb = smem0 + qs * kQStageBytes;
-            const long long n0 = (long long)quse * kHalfChunks;   // number of the item's half chunk 0
-            auto half_ready = [&](int n) -> bool {        // the keys of the item's half chunk n are in their half slot
-                const long long p = n0 + n;
-                if (!mbar_wait_all(bar_kfull((int)(p % (2 * kSlots))), (uint32_t)((p / (2 * kSlots)) & 1), cta_abort)) return false;
+            const unsigned n0 = (unsigned)quse * kHalfChunks;     // number of the item's half chunk 0
+            auto half_ready = [&](int n) -> bool {        // the K and V rows of the item's half chunk n are in their units
+                const unsigned p = n0 + n;
+                if (!mbar_wait_all(bar_kfull((int)(p % kKUnits)), (uint32_t)((p / kKUnits) & 1), cta_abort)) return false;
+                if (!mbar_wait_all(bar_vfull((int)(p % kVUnits)), (uint32_t)((p / kVUnits) & 1), cta_abort)) return false;
                 fence_proxy_async();
                 return true;
             };
-            // S = Q K^T, dP = dO V^T for half chunk n of the item (chunk n / 2, keys 64 (n % 2) ..), into its buffer
-            // (descriptor low words = start address in 16-byte units: + 2 per 32-byte K step, + kHalf / 16 for the hi half)
-            const uint32_t q_lo = sdesc_lo(make_sdesc_sw64(qb + kOffQlo, 512)), g_lo = sdesc_lo(make_sdesc_sw64(qb + kOffGlo, 512));
+            // S = Q K^T, dP = dO V^T for half chunk n of the item into its buffer; the V unit goes back with them
+            // (descriptor low words = start address in 16-byte units: + 2 per 32-byte K step, + region / 16 per 32-column part)
+            const uint32_t q_lo = sdesc_lo(make_sdesc_sw64(qb + kOffQ, 512)), g_lo = sdesc_lo(make_sdesc_sw64(qb + kOffG, 512));
             auto issue_sdp = [&](int n) {
-                const uint32_t sb = smem0 + kOffSlots + (int)(((n0 + n) >> 1) % kSlots) * kSlotBytes + (n & 1) * 64 * kHalfBytes;
-                const int buf = (int)((n0 + n) % 3);
-                const uint32_t k_lo = sdesc_lo(make_sdesc_sw64(sb + kOffKlo, 512));
-                const uint32_t v_lo = sdesc_lo(make_sdesc_sw64(sb + kOffVlo, 512));
+                const unsigned p = n0 + n;
+                const int buf = (int)(p % 3), uv = (int)(p % kVUnits);
+                const uint32_t k_lo = sdesc_lo(make_sdesc_sw64(smem0 + kOffKRing + (int)(p % kKUnits) * kUnitBytes, 512));
+                const uint32_t v_lo = sdesc_lo(make_sdesc_sw64(smem0 + kOffVRing + uv * kUnitBytes, 512));
                 const uint32_t t_s = tmem_base + kBufCols * buf, t_dp = t_s + 64;
-                constexpr uint32_t kHi = kHalf >> 4;
+                constexpr uint32_t kQNext = kPart >> 4, kUNext = kUPart >> 4;
                 tc_fence_after();
                 if (elect_one()) {
                     mma_ss_h<false>(t_s, q_lo, k_lo, sd_hi, idesc_s);
                     mma_ss_h<true>(t_s, q_lo + 2, k_lo + 2, sd_hi, idesc_s);
-                    mma_ss_h<true>(t_s, q_lo + kHi, k_lo + kHi, sd_hi, idesc_s);
-                    mma_ss_h<true>(t_s, q_lo + kHi + 2, k_lo + kHi + 2, sd_hi, idesc_s);
+#pragma unroll
+                    for (int pt = 1; pt < kParts; ++pt) {
+                        mma_ss_h<true>(t_s, q_lo + pt * kQNext, k_lo + pt * kUNext, sd_hi, idesc_s);
+                        mma_ss_h<true>(t_s, q_lo + pt * kQNext + 2, k_lo + pt * kUNext + 2, sd_hi, idesc_s);
+                    }
                     mma_ss_h<false>(t_dp, g_lo, v_lo, sd_hi, idesc_s);
                     mma_ss_h<true>(t_dp, g_lo + 2, v_lo + 2, sd_hi, idesc_s);
-                    mma_ss_h<true>(t_dp, g_lo + kHi, v_lo + kHi, sd_hi, idesc_s);
-                    mma_ss_h<true>(t_dp, g_lo + kHi + 2, v_lo + kHi + 2, sd_hi, idesc_s);
+#pragma unroll
+                    for (int pt = 1; pt < kParts; ++pt) {
+                        mma_ss_h<true>(t_dp, g_lo + pt * kQNext, v_lo + pt * kUNext, sd_hi, idesc_s);
+                        mma_ss_h<true>(t_dp, g_lo + pt * kQNext + 2, v_lo + pt * kUNext + 2, sd_hi, idesc_s);
+                    }
                     mma_commit(bar_sdp(buf));
+                    mma_commit(bar_vempty(uv));
                 }
                 __syncwarp();
             };
@@ -393,15 +540,14 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
             }
             if (!ok) break;
             for (int n = 0; n < kHalfChunks && ok; ++n) {
-                const long long ng = n0 + n;
+                const unsigned ng = n0 + n;
                 const int buf = (int)(ng % 3);
                 ok = mbar_wait_all(bar_ds(buf), (uint32_t)((ng / 3) & 1), cta_abort);
                 if (ok && n == 0 && quse > 0) ok = mbar_wait_all(bar_accfree, (quse - 1) & 1, cta_abort);
                 if (!ok) break;
                 tc_fence_after();
                 // dQ += dS K over the half chunk's key columns
-                const uint32_t sb = smem0 + kOffSlots + (int)((ng >> 1) % kSlots) * kSlotBytes + (n & 1) * 64 * kHalfBytes;
-                const uint64_t kd = make_sdesc_sw64_mn(sb + kOffKlo, kHalf, 512);
+                const uint64_t kd = make_sdesc_sw64_mn(smem0 + kOffKRing + (int)(ng % kKUnits) * kUnitBytes, kUPart, 512);
                 const uint32_t k_lo = sdesc_lo(kd), d_hi = sdesc_hi(kd);
                 const uint32_t t_ds = tmem_base + kBufCols * buf + 64;
                 if (elect_one()) {
@@ -411,7 +557,7 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
                         j = 1;
                     }
                     for (; j < 4; ++j) mma_ts_h<true>(tmem_base + kColDQ, t_ds + 16 * j, k_lo + 64 * j, d_hi, idesc_acc);
-                    mma_commit(bar_kempty((int)(ng % (2 * kSlots))));   // the half slot's last reader: it goes back at once
+                    mma_commit(bar_kempty((int)(ng % kKUnits)));    // the K unit's last reader: it goes back at once
                     if (n + 1 == kHalfChunks) {
                         mma_commit(bar_acc);
                         mma_commit(bar_qempty(qs));
@@ -442,7 +588,6 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
         const uint32_t tab_lane = tab0 + 4 * (quarter * kTabFloats + 16 * hcol * 64 + lane + 31);
         int quse = 0, n_flush = 0;
         int tab_qt = -1;                                  // the tile whose gradients the tables hold
-        long long ru = 0;
         bool ok = true;
         // all elementwise threads meet (bounded), the tables go to the global gradient and are cleared, they meet again
         auto flush = [&](int qt) -> bool {
@@ -482,10 +627,10 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
             const float dl = lds_f32(st_a + kOffQDelta + 4 * qrow);
             mbar_arrive(bar_qempty(qs));                  // this thread has what it needs from the query stage
             const uint32_t bias_row = smem0 + kOffBias + qcode4;
-            for (int c = 0; c < kTiles && ok; ++c, ++ru) {
-                const int s = (int)(ru % kSlots);         // the chunk's slot: half chunk p is in slot (p / 2) % 3
-                const uint32_t sl_a = smem0 + kOffSlots + s * kSlotBytes;
-                const long long ng = (long long)quse * kHalfChunks + 2 * c + hcol;   // this group's half chunk
+            for (int c = 0; c < kTiles && ok; ++c) {
+                const unsigned ng = (unsigned)quse * kHalfChunks + 2 * c + hcol;     // this group's half chunk
+                // labels of the half chunk's 64 keys, addressed by the chunk's column number
+                const uint32_t sl_a = smem0 + kOffKLab + (int)(ng % kKUnits) * 256 - 256 * hcol;
                 const int buf = (int)(ng % 3);
                 ok = mbar_wait_all(bar_sdp(buf), (uint32_t)((ng / 3) & 1), cta_abort);
                 if (!ok) break;
@@ -526,20 +671,26 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
             // ---- read-out: dQ columns 0..31 by warps 0-3, 32..63 by warps 4-7
             if (!mbar_wait_all(bar_acc, quse & 1, cta_abort)) { ok = false; break; }
             tc_fence_after();
-            uint32_t r0[32];
-            tmem_ld32(tmem_base + lane_addr + kColDQ + 32 * hcol, r0);
-            tmem_ld_wait();
-            tc_fence_before();
-            mbar_arrive(bar_accfree);
-            uint4* dst = reinterpret_cast<uint4*>(dq + ((size_t)cur.b * HW + (size_t)qtok) * g.ts + head * kD + 32 * hcol);
+            // ---- read-out: the first half of dQ's columns by warps 0-3, the second by warps 4-7
+            uint4* dst = reinterpret_cast<uint4*>(dq + ((size_t)cur.b * HW + (size_t)qtok) * g.ts + head * D + (D / 2) * hcol);
 #pragma unroll
-            for (int c4 = 0; c4 < 4; ++c4) {
-                uint4 a;
-                a.x = pack_bf16(__uint_as_float(r0[c4 * 8 + 0]) * out_scale, __uint_as_float(r0[c4 * 8 + 1]) * out_scale);
-                a.y = pack_bf16(__uint_as_float(r0[c4 * 8 + 2]) * out_scale, __uint_as_float(r0[c4 * 8 + 3]) * out_scale);
-                a.z = pack_bf16(__uint_as_float(r0[c4 * 8 + 4]) * out_scale, __uint_as_float(r0[c4 * 8 + 5]) * out_scale);
-                a.w = pack_bf16(__uint_as_float(r0[c4 * 8 + 6]) * out_scale, __uint_as_float(r0[c4 * 8 + 7]) * out_scale);
-                dst[c4] = a;
+            for (int hq = 0; hq < D / 64; ++hq) {
+                uint32_t r0[32];
+                tmem_ld32(tmem_base + lane_addr + kColDQ + (D / 2) * hcol + 32 * hq, r0);
+                tmem_ld_wait();
+                if (hq == D / 64 - 1) {
+                    tc_fence_before();
+                    mbar_arrive(bar_accfree);
+                }
+#pragma unroll
+                for (int c4 = 0; c4 < 4; ++c4) {
+                    uint4 a;
+                    a.x = pack_bf16(__uint_as_float(r0[c4 * 8 + 0]) * out_scale, __uint_as_float(r0[c4 * 8 + 1]) * out_scale);
+                    a.y = pack_bf16(__uint_as_float(r0[c4 * 8 + 2]) * out_scale, __uint_as_float(r0[c4 * 8 + 3]) * out_scale);
+                    a.z = pack_bf16(__uint_as_float(r0[c4 * 8 + 4]) * out_scale, __uint_as_float(r0[c4 * 8 + 5]) * out_scale);
+                    a.w = pack_bf16(__uint_as_float(r0[c4 * 8 + 6]) * out_scale, __uint_as_float(r0[c4 * 8 + 7]) * out_scale);
+                    dst[4 * hq + c4] = a;
+                }
             }
         }
         if (ok && tab_qt >= 0) flush(tab_qt);
@@ -565,7 +716,7 @@ cudaError_t read_bwd_q64_status(int* timed_out) {
 }
 
 bool bwd_q64_supported(const Geo& g) {
-    return g.d == 64 && g.w == kW && g.H % kW == 0 && g.W % kW == 0 && g.heads <= 148;
+    return (g.d == 64 || g.d == 128) && g.w == kW && g.H % kW == 0 && g.W % kW == 0 && g.heads <= 148;
 }
 
 // `prep` = the prepared bias tables of the head-dim-64 forward kernel (kBiasFloats per head), filled by the caller;
@@ -578,12 +729,20 @@ cudaError_t launch_bwd_q64(const Geo& g, const void* q, const void* k, const voi
     if (cph > items) cph = items;
     cudaError_t e = cudaMemsetAsync(dbias, 0, sizeof(float) * (size_t)(2 * kW - 1) * (2 * kW - 1) * g.heads, stream);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(swin_bwd_q64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    QMaps64 maps;
+    std::memset(&maps, 0, sizeof maps);
+    static const bool tma_off = [] { const char* e_ = std::getenv("TERRA_NO_TMA"); return e_ && e_[0] == '1'; }();
+    // (at head dim 64 the runs of 16 tokens are 1 KB copies, and the three gathering warps are faster)
+    const bool tma = !tma_off && g.d == 128 && bulk_rows_shape(g) && g.sh % 16 == 0 && make_row_maps3(&maps.q, g, q, g.ts) &&
+                     make_row_maps3(&maps.g, g, d_o, g.heads * g.d) && make_col_map(&maps.k, g, k, g.ts) && make_col_map(&maps.v, g, v, g.ts);
+    auto kern = g.d == 64 ? swin_bwd_q64_kernel<64, false> : (tma ? swin_bwd_q64_kernel<128, true> : swin_bwd_q64_kernel<128, false>);
+    const int smem_bytes = g.d == 64 ? Lay<64>::kSmemBytes : Lay<128>::kSmemBytes;
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
     if (e != cudaSuccess) return e;
     prof_begin("swin_bwd_q64_kernel", stream);
-    swin_bwd_q64_kernel<<<(unsigned)(cph * g.heads), kThreads, kSmemBytes, stream>>>(
+    kern<<<(unsigned)(cph * g.heads), kThreads, smem_bytes, stream>>>(
         g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)d_o, prep, lse, delta,
-        (__nv_bfloat16*)dq, dbias, items, (int)cph);
+        (__nv_bfloat16*)dq, dbias, items, (int)cph, maps);
     count_launch(stream);
     return cudaGetLastError();
 }

@@ -19,6 +19,10 @@ struct RowMaps3 {
 // host: the three maps of one tensor (`token_stride` in elements); false if the driver's encoder is not available
 bool make_row_maps3(RowMaps3* maps, const Geo& g, const void* base, int token_stride);
 
+// host: one tensor as [token rows, token columns, heads * d] with boxes of 32 columns x 1 token column x 16 token
+// rows: 16 vertically adjacent tokens of one head become 16 consecutive 64-byte rows of a swizzled region
+bool make_col_map(CUtensorMap* map, const Geo& g, const void* base, int token_stride);
+
 // host: the geometry the bulk-copy loaders are written for
 inline bool bulk_rows_shape(const Geo& g) {
     return (g.w == 16 || g.w == 32) && g.H % g.w == 0 && g.W % g.w == 0 && g.sw % 8 == 0 &&
