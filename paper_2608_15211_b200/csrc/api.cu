@@ -112,7 +112,10 @@ static bool force_register_path() {
 
 // the tcgen05 kernels are written for bf16 operands; fp16 runs on the register-tile kernels
 static bool use_fwd_tc(const Geo& g) { return fwd_tc_supported(g) && !g.f16; }
-static bool use_fwd_tc64(const Geo& g) { return fwd_tc64_supported(g) && !force_register_path() && !g.f16; }
+// head dim 128 with windows of fewer than 256 tokens (the 8 x 8 windows of the paper's small and medium models): a
+// 128-row tile would be mostly empty and the path is bound by HBM, the register-tile kernels are about twice as fast
+static bool small_window_128(const Geo& g) { return g.d == 128 && g.nmax < 256; }
+static bool use_fwd_tc64(const Geo& g) { return fwd_tc64_supported(g) && !force_register_path() && !g.f16 && !small_window_128(g); }
 
 static size_t fwd_bytes(const Geo& g) {
     if (force_register_path() || g.f16) return 0;
@@ -123,7 +126,7 @@ static size_t fwd_bytes(const Geo& g) {
 
 static bool use_bwd_tc(const Geo& g) { return bwd_tc_supported(g) && !force_register_path() && !g.f16; }
 
-static bool use_bwd_kv64(const Geo& g) { return bwd_kv64_supported(g) && !force_register_path() && !g.f16; }
+static bool use_bwd_kv64(const Geo& g) { return bwd_kv64_supported(g) && !force_register_path() && !g.f16 && !small_window_128(g); }
 
 static size_t delta_bytes(const Geo& g) {
     if (use_bwd_tc(g)) return align_up(bwd_tc_workspace_bytes(g), 256);

@@ -305,7 +305,7 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             mbar_init(bar_qempty(s), 1 + 256);        // the issuer's commit + every softmax thread
         }
         for (int s = 0; s < kSlots; ++s) {
-            mbar_init(bar_kvfull(s), TMA ? 32 : kLoaderThreads);
+            mbar_init(bar_kvfull(s), kLoaderThreads);     // TMA: the bulk-copy warp's lanes + the 64 threads that gather V rows
             mbar_init(bar_kvempty(s), 1);
         }
         for (int t = 0; t < 2; ++t) {
@@ -420,55 +420,74 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                                 klab[row] = label;
                             }
                         }
+                        // K rows (the V rows of pass B are gathered by the other two loader warps: the bulk-copy
+                        // engine takes a fixed time per 64-byte row, and the two ways of loading run side by side)
                         const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes;
-                        const int per_tensor = wrows * kParts, combos = per_tensor * (pass + 1);
-                        for (int i = lane; i < combos; i += 32) {
-                            const int tsr = i >= per_tensor ? 1 : 0, rem = i - tsr * per_tensor;
-                            const int ar = rem / kParts, part = rem - ar * kParts;
-                            copy_row(tsr ? maps.v : maps.k, sb + (tsr ? kOffV : kOffK) + part * kKPart + ar * g.w * kPartBytes,
-                                     c * wrows + ar, part, bar_kvfull(s));
+                        for (int i = lane; i < wrows * kParts; i += 32) {
+                            const int ar = i / kParts, part = i - ar * kParts;
+                            copy_row(maps.k, sb + kOffK + part * kKPart + ar * g.w * kPartBytes, c * wrows + ar, part, bar_kvfull(s));
                         }
                         __syncwarp();
-                        if (lane == 0) mbar_arrive_expect_tx(bar_kvfull(s), (uint32_t)(kChunk * D * 2 * (pass + 1)));
+                        if (lane == 0) mbar_arrive_expect_tx(bar_kvfull(s), (uint32_t)(kChunk * D * 2));
                         else mbar_arrive(bar_kvfull(s));
                     }
                 }
                 ++kuse;
             }
+        } else {
+            // ---- warps 10, 11: the V rows of pass B with 16-byte cp.async copies; a thread's arrival on the chunk's
+            // barrier is tied to the completion of its copies, so it never waits for data
+            const int vt = (warp - kLoaderWarp0 - 1) * 32 + lane;      // 0 .. 63
+            const int part = vt % kParts, row0 = vt / kParts;
+            constexpr int kRowStep = 64 / kParts;
+            long long ru = 0;
+            bool ok = true;
+            ItemCursor cur = cursor_init(cta_in_head, ctas_per_head, max_pairs, g.Mw, g.Mh);
+            for (long long it = cta_in_head; ok && it < n_items; it += ctas_per_head, cursor_advance(cur, max_pairs, g.Mw, g.Mh)) {
+                const Item x = make_item(g, cur);
+                if (x.ntiles == 0) continue;
+                const size_t sample_off = (size_t)x.b * HW;
+                const int ew = x.r.ew;
+                for (int pass = 0; pass < 2 && ok; ++pass) {
+                    for (int c = 0; c < x.nch; ++c, ++ru) {
+                        const int s = (int)(ru % kSlots);
+                        ok = mbar_wait_all(bar_kvempty(s), (uint32_t)((ru / kSlots) & 1) ^ 1u, cta_abort);
+                        if (!ok) break;
+                        if (pass == 0) {
+                            mbar_arrive(bar_kvfull(s));
+                            continue;
+                        }
+                        const uint32_t vb = smem0 + kOffSlots + s * kSlotBytes + kOffV + part * kKPart;
+                        for (int row = row0; row < kChunk; row += kRowStep) {
+                            const int slot = c * kChunk + row, a = slot / ew;
+                            int code, label;
+                            const int tok = offset_token(g, x.r, a, slot - a * ew, code, label);
+                            const __nv_bfloat16* src = v + (sample_off + (size_t)tok) * g.ts + head * D + part * 32;
+#pragma unroll
+                            for (int c4 = 0; c4 < 4; ++c4) cp_async16(vb + tile_off<32>(row, c4), src + c4 * 8, 16);
+                        }
+                        cp_async_mbar_arrive_noinc(bar_kvfull(s));
+                    }
+                }
+            }
         }
     } else if (warp >= kLoaderWarp0) {
         // ------------------------------------------------------------------ loaders
         // D / 32 lanes per row: each takes one 32-column part of the row and issues its four 16-byte copies with one
-        // address computation.  A chunk is published (its barrier arrived on) only when the next
-        // one has been issued, so that two chunks are in flight; if the ring has no free slot the pending chunk is
-        // published first, or the consumers could never free one.
+        // address computation.  A thread never waits for data: its arrival on a stage's or slot's barrier is tied to
+        // the completion of the copies it has issued, so as many chunks are in flight as the ring has free slots.
         const int lt = (warp - kLoaderWarp0) * 32 + lane;
         const int hf = lt % kParts;                       // which 32-column part of the row this thread copies
         const int lrow = lt / kParts;
         constexpr int kRowsPerIter = kLoaderThreads / kParts;
         int kuse = 0;
         long long ru = 0;                                 // ring uses so far
-        uint32_t pending_bar = 0;                         // barrier of the group of copies issued last (0: none)
         bool ok = true;
-        // waits for `bar` (a slot's or stage's release); publishes the pending copies first if that is not immediate
-        auto acquire = [&](uint32_t bar, uint32_t parity) -> bool {
-            if (pending_bar && !__all_sync(0xffffffffu, mbar_test_wait(bar, parity))) {
-                cp_async_wait<0>();
-                fence_proxy_async();
-                mbar_arrive(pending_bar);
-                pending_bar = 0;
-            }
-            return mbar_wait_all(bar, parity, cta_abort);
-        };
-        // the copies just issued become the pending group; the group before them is complete and is published
+        auto acquire = [&](uint32_t bar, uint32_t parity) -> bool { return mbar_wait_all(bar, parity, cta_abort); };
+        // the thread's table entries are visible to the CTA before its arrival, which follows its copies
         auto issued = [&](uint32_t bar) {
-            cp_async_commit();
-            if (pending_bar) {
-                cp_async_wait<1>();
-                fence_proxy_async();
-                mbar_arrive(pending_bar);
-            }
-            pending_bar = bar;
+            __threadfence_block();
+            cp_async_mbar_arrive_noinc(bar);
         };
         ItemCursor cur = cursor_init(cta_in_head, ctas_per_head, max_pairs, g.Mw, g.Mh);
         for (long long it = cta_in_head; ok && it < n_items; it += ctas_per_head, cursor_advance(cur, max_pairs, g.Mw, g.Mh)) {
@@ -561,11 +580,6 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                 }
             }
             ++kuse;
-        }
-        if (pending_bar) {
-            cp_async_wait<0>();
-            fence_proxy_async();
-            mbar_arrive(pending_bar);
         }
     } else {
         // ------------------------------------------------------------------ MMA issuer
