@@ -1,23 +1,24 @@
-// Forward shifted-window attention on the tcgen05 tensor cores for head dim 64 and windows of up to 1024 tokens
-// (window side <= 32): the large-window regime, where a score row no longer fits tensor memory.
+// Forward shifted-window attention on the tcgen05 tensor cores for head dims 64 and 128 and windows of up to 1024
+// tokens (window side <= 32): the large-window regime, where a score row no longer fits tensor memory.
 //
 // One persistent CTA per SM, bound to one head, walks over (batch, window, pair of 128-row query tiles) items.
-// The window's keys are streamed in chunks of 128 through a ring of shared-memory slots, twice:
-//   pass A   S = Q K_c^T per chunk, the softmax threads only take the row maximum: for complete windows without mask
-//            labels the upper bound max_j(raw) * scale + max(bias) of the small-window kernel; for windows that mix
-//            mask labels or hold slots without a token, and for heads whose bias table spreads over more than 64
-//            octaves, the exact maximum over the keys the row may see (the chunk's key tables are then staged in
-//            pass A as well, and its ring slot is released only when the softmax threads have read them);
-//   pass B   S = Q K_c^T again, P = exp2(S * scale + bias - m) written back over S as bf16, O += P [V_c | 1]
-//            (16 columns of ones behind V: the accumulator's columns 64..79 carry the row sums of P).
-// Recomputing S costs tensor-pipe time, of which there is plenty next to the exp work, and spares the running
-// rescale of O of an online softmax.
+// The window's keys are streamed once, in chunks of 128, through a ring of shared-memory slots.  Per chunk:
+//   S = Q K_c^T                                                        (SS MMAs into the tile's columns)
+//   online softmax: the softmax threads take the chunk's maximum (for complete windows without mask labels the bound
+//   max_j(raw) * scale + max(bias); for windows that mix mask labels or hold slots without a token, and for heads
+//   whose bias table spreads over more than 64 octaves, the exact maximum over the keys the row may see), raise the
+//   row's reference m when the chunk exceeds it by more than 8 octaves (then O and the row sum are scaled down in
+//   tensor memory), and write P = exp2(S * scale + bias - m) back over S as bf16;
+//   O += P [V_c | 1]                                                   (A from TMEM; at head dim 64, 16 columns of
+//   ones behind V make the accumulator's columns 64..79 carry the row sums; at head dim 128 tensor memory has no
+//   columns left for them and the softmax threads add the row sums themselves).
 // Roles: warps 0-3 / 4-7 softmax warpgroups (one thread per query row of the pair's first / second tile),
-// warp 8 issues every tcgen05.mma (whole warp runs the loop, one elected lane issues), warps 9-11 gather rows
-// with cp.async, undoing the roll.  Head dim 64 is kept as two 32-column halves in the 64-byte-swizzled operand
-// layout of the small-window kernels (lo | hi regions), so that the same descriptors serve.
+// warp 8 issues every tcgen05.mma (whole warp runs the loop, one elected lane issues), warps 9-11 load rows, undoing
+// the roll: on grids of complete windows warp 9 fetches Q and K rows with tiled bulk copies and warps 10-11 gather V
+// rows with cp.async; otherwise all three gather with cp.async.  A row is kept as head dim / 32 parts of 32 columns in
+// the 64-byte-swizzled operand layout of the small-window kernels, so that the same descriptors serve.
 // TMEM: columns [256 t, 256 t + 256) belong to query tile t of the pair: S chunk (fp32, 128 columns), overwritten
-// in place by bf16 P (64 columns); the O accumulator (64 + 16 columns) at +128.
+// in place by bf16 P (64 columns); the O accumulator at +128.
 // Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, all roles leave their loops, TMEM is
 // released and the host reads the device status word.  Every role follows every ring item by item.
 #include <cstdlib>
@@ -286,7 +287,6 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
     auto bar_kvfull = [&](int s) { return bar0 + 8u * (4 + s); };        // a key chunk is in ring slot s
     auto bar_kvempty = [&](int s) { return bar0 + 8u * (7 + s); };       // ... and every MMA that reads it is complete
     auto bar_sready = [&](int t) { return bar0 + 8u * (10 + t); };       // S of a chunk is in tile t's columns
-    auto bar_sfree = [&](int t) { return bar0 + 8u * (12 + t); };        // pass A: the softmax threads have read it
     auto bar_pready = [&](int t) { return bar0 + 8u * (14 + t); };       // pass B: P of the chunk is in TMEM
     auto bar_oready = [&](int t) { return bar0 + 8u * (16 + t); };       // O of the item is final
     auto bar_ofree = [&](int t) { return bar0 + 8u * (18 + t); };        // ... and has been read
@@ -310,7 +310,6 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
         }
         for (int t = 0; t < 2; ++t) {
             mbar_init(bar_sready(t), 1);
-            mbar_init(bar_sfree(t), 128);
             mbar_init(bar_pready(t), 128);
             mbar_init(bar_oready(t), 1);
             mbar_init(bar_ofree(t), 128);
@@ -398,14 +397,13 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                     if (lane == 0) mbar_arrive_expect_tx(bar_qfull(qs), (uint32_t)(x.ntiles * 128 * D * 2));
                     else mbar_arrive(bar_qfull(qs));
                 }
-                // ---- the key chunks: pass A needs K only (and the key tables if the row maxima are taken exactly), pass B K and V
-                const int first_meta_pass = exact_max(x) ? 0 : 1;
-                for (int pass = 0; pass < 2 && ok; ++pass) {
+                // ---- the key chunks (K rows and the key tables)
+                {
                     for (int c = 0; c < x.nch; ++c, ++ru) {
                         const int s = (int)(ru % kSlots);
                         ok = mbar_wait_all(bar_kvempty(s), (uint32_t)((ru / kSlots) & 1) ^ 1u, cta_abort);
                         if (!ok) break;
-                        if (pass >= first_meta_pass) {
+                        {
                             int* kcs = reinterpret_cast<int*>(smem + kOffKeyMeta + s * 1024);
                             int* klab = kcs + 128;
                             for (int row = lane; row < kChunk; row += 32) {
@@ -420,7 +418,7 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                                 klab[row] = label;
                             }
                         }
-                        // K rows (the V rows of pass B are gathered by the other two loader warps: the bulk-copy
+                        // K rows (the V rows are gathered by the other two loader warps: the bulk-copy
                         // engine takes a fixed time per 64-byte row, and the two ways of loading run side by side)
                         const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes;
                         for (int i = lane; i < wrows * kParts; i += 32) {
@@ -435,7 +433,7 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                 ++kuse;
             }
         } else {
-            // ---- warps 10, 11: the V rows of pass B with 16-byte cp.async copies; a thread's arrival on the chunk's
+            // ---- warps 10, 11: the V rows with 16-byte cp.async copies; a thread's arrival on the chunk's
             // barrier is tied to the completion of its copies, so it never waits for data
             const int vt = (warp - kLoaderWarp0 - 1) * 32 + lane;      // 0 .. 63
             const int part = vt % kParts, row0 = vt / kParts;
@@ -448,15 +446,11 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                 if (x.ntiles == 0) continue;
                 const size_t sample_off = (size_t)x.b * HW;
                 const int ew = x.r.ew;
-                for (int pass = 0; pass < 2 && ok; ++pass) {
+                {
                     for (int c = 0; c < x.nch; ++c, ++ru) {
                         const int s = (int)(ru % kSlots);
                         ok = mbar_wait_all(bar_kvempty(s), (uint32_t)((ru / kSlots) & 1) ^ 1u, cta_abort);
                         if (!ok) break;
-                        if (pass == 0) {
-                            mbar_arrive(bar_kvfull(s));
-                            continue;
-                        }
                         const uint32_t vb = smem0 + kOffSlots + s * kSlotBytes + kOffV + part * kKPart;
                         for (int row = row0; row < kChunk; row += kRowStep) {
                             const int slot = c * kChunk + row, a = slot / ew;
@@ -532,16 +526,15 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                 }
                 issued(bar_qfull(qs));
             }
-            // ---- the key chunks: pass A needs K only (and the key tables if the row maxima are taken exactly), pass B K and V
-            const int first_meta_pass = exact_max(x) ? 0 : 1;
-            for (int pass = 0; pass < 2 && ok; ++pass) {
+            // ---- the key chunks: K and V rows and the key tables
+            {
                 for (int c = 0; c < x.nch; ++c, ++ru) {
                     const int s = (int)(ru % kSlots);
                     ok = acquire(bar_kvempty(s), (uint32_t)((ru / kSlots) & 1) ^ 1u);
                     if (!ok) break;
                     const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes + hf * kKPart;
                     const int ncols = min(kChunk, x.npad - c * kChunk);
-                    if (pass >= first_meta_pass) {
+                    {
                         int* kcs = reinterpret_cast<int*>(smem + kOffKeyMeta + s * 1024);
                         int* klab = kcs + 128;
                         for (int row = lt; row < kChunk; row += kLoaderThreads) {
@@ -573,7 +566,7 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                         for (int c4 = 0; c4 < 4; ++c4) {
                             const uint32_t so = tile_off<32>(row, c4);
                             cp_async16(sb + kOffK + so, bytes ? sk + c4 * 8 : sk, bytes);
-                            if (pass == 1) cp_async16(sb + kOffV + so, bytes ? sv + c4 * 8 : sv, bytes);
+                            cp_async16(sb + kOffV + so, bytes ? sv + c4 * 8 : sv, bytes);
                         }
                     }
                     issued(bar_kvfull(s));
@@ -586,7 +579,7 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
         const uint32_t idesc_pv = make_idesc_bf16(128, kNO, 0, 1);
         int kuse = 0;
         long long ru = 0;
-        int n_s[2] = {0, 0}, n_free[2] = {0, 0}, n_p[2] = {0, 0}, n_items_t[2] = {0, 0};
+        int n_p[2] = {0, 0}, n_items_t[2] = {0, 0};
         bool ok = true;
         ItemCursor cur = cursor_init(cta_in_head, ctas_per_head, max_pairs, g.Mw, g.Mh);
         for (long long it = cta_in_head; ok && it < n_items; it += ctas_per_head, cursor_advance(cur, max_pairs, g.Mw, g.Mh)) {
@@ -618,56 +611,16 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                 }
                 __syncwarp();
             };
-            // tile t's S columns are free for a new QK product: after pass-A chunks once the softmax threads have read
-            // the chunk before (every S of pass A is read and released); after pass-B chunks by the order of the MMAs
-            // (the P that replaced S was consumed by its PV product, issued earlier from this thread)
-            auto s_free = [&](int t) -> bool {
-                while (n_free[t] < n_s[t]) {
-                    if (!mbar_wait_all(bar_sfree(t), n_free[t] & 1, cta_abort)) return false;
-                    ++n_free[t];
-                }
-                tc_fence_after();
-                return true;
-            };
+            // tile t's S columns are free for the next chunk's QK product by the order of the MMAs: the P that replaced S
+            // was consumed by its PV product, issued earlier from this thread
             auto chunk_ready = [&](long long use) -> bool {
                 if (!mbar_wait_all(bar_kvfull((int)(use % kSlots)), (uint32_t)((use / kSlots) & 1), cta_abort)) return false;
                 fence_proxy_async();
                 return true;
             };
-            // ---- pass A: S of every chunk, for the row maxima
-            // Exact row maxima: the softmax threads also read the chunk's key tables from the ring slot, so the slot is
-            // released (plain arrival) only after they have given the chunk's S columns back, one chunk later.
-            const bool exact = exact_max(x);
-            int held = -1;                                       // exact: slot of the chunk before, not released yet
-            for (int c = 0; c < x.nch && ok; ++c, ++ru) {
-                const int s = (int)(ru % kSlots);
-                ok = chunk_ready(ru);
-                if (!ok) break;
-                const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes;
-                const int ncols = min(kChunk, x.npad - c * kChunk);
-                for (int t = 0; t < x.ntiles && ok; ++t) {
-                    ok = s_free(t);
-                    if (!ok) break;
-                    issue_qk(t, sb, ncols);
-                    ++n_s[t];
-                }
-                if (!ok) break;
-                if (elect_one()) {
-                    if (!exact) mma_commit(bar_kvempty(s));      // the slot is free once the MMAs issued so far are complete
-                    else if (held >= 0) mbar_arrive(bar_kvempty(held));   // every tile's softmax threads are done with it
-                }
-                __syncwarp();
-                held = exact ? s : -1;
-            }
-            if (!ok) break;
-            // ---- pass B: per tile, PV of chunk c is followed at once by QK of chunk c + 1, so that a tile's softmax
-            // threads wait for one PV and one QK product only, whatever the other tile is doing
+            // ---- per tile, PV of chunk c is followed at once by QK of chunk c + 1, so that a tile's softmax threads wait
+            // for one PV and one QK product only, whatever the other tile is doing
             ok = chunk_ready(ru);
-            for (int t = 0; t < x.ntiles && ok; ++t) ok = s_free(t);
-            if (ok && held >= 0) {
-                if (elect_one()) mbar_arrive(bar_kvempty(held));
-                __syncwarp();
-            }
             for (int t = 0; t < x.ntiles && ok; ++t)
                 issue_qk(t, smem0 + kOffSlots + (int)(ru % kSlots) * kSlotBytes, min(kChunk, x.npad));
             for (int c = 0; c < x.nch && ok; ++c, ++ru) {
@@ -736,7 +689,7 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             mbar_arrive(bar_qempty(qs));                  // this thread has what it needs from the stage
             ++kuse;
             const long long ru0 = ru;
-            ru += 2 * x.nch;
+            ru += x.nch;
             if (wg >= x.ntiles) continue;                 // the pair's second tile does not exist in this window
             const uint32_t bias_i = smem0 + kOffBias + 4 * meta_code(rmeta);
             const int label_i = meta_label(rmeta);
@@ -744,70 +697,88 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             const bool row32 = g.w == 32 && x.r.ew == 32 && !x.masked;       // then every key slot holds a token, too
             const bool exact = exact_max(x);
             bool ok = true;
-            // ---- pass A: row maximum over all chunks
-            float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-            float mxe = -INFINITY;
+            // Online softmax, chunk by chunk: P is formed against a reference m that is at least the row's maximum so
+            // far minus 8 octaves; only when a chunk's maximum exceeds the reference by more than that is the reference
+            // raised and the accumulated O (with the row sum) scaled down by 2^(old - new).  Without mask labels the
+            // chunk maximum is the bound max_j(raw) * scale + max(bias); for windows that mix mask labels or hold slots
+            // without a token, and for heads whose bias table spreads over more than 64 octaves, it is the exact
+            // maximum over the keys the row may see.  A row that has seen no key yet forms its P against 0: exactly 0.
+            float m = -INFINITY;
             float psum[2] = {0.f, 0.f};
             for (int c = 0; c < x.nch; ++c) {
                 const int ncols = min(kChunk, x.npad - c * kChunk);
-                ok = mbar_wait_all(bar_sready(wg), n_s & 1, cta_abort);
-                if (!ok) break;
-                ++n_s;
-                tc_fence_after();
-                uint32_t ra[32], rb[32];
-                int cc = 0;
-                if (exact) {
-                    const uint32_t a_kc = smem0 + kOffKeyMeta + (int)((ru0 + c) % kSlots) * 1024, a_klab = a_kc + 512;
-                    for (; cc + 32 <= ncols; cc += 32) {
-                        tmem_ld32(t_s + cc, ra);
-                        tmem_ld_wait();
-                        mxe = score_max_cols<32>(ra, cc, bias_i, a_kc, a_klab, label_i, scale, mxe);
-                    }
-                    if (cc < ncols) {
-                        uint32_t rt[16];
-                        tmem_ld16(t_s + cc, rt);
-                        tmem_ld_wait();
-                        mxe = score_max_cols<16>(rt, cc, bias_i, a_kc, a_klab, label_i, scale, mxe);
-                        cc = ncols;
-                    }
-                }
-                for (; cc + 64 <= ncols; cc += 64) {
-                    tmem_ld32(t_s + cc, ra);
-                    tmem_ld32(t_s + cc + 32, rb);
-                    tmem_ld_wait();
-                    max_cols<32>(ra, mx4);
-                    max_cols<32>(rb, mx4);
-                }
-                if (cc + 32 <= ncols) {
-                    tmem_ld32(t_s + cc, ra);
-                    tmem_ld_wait();
-                    max_cols<32>(ra, mx4);
-                    cc += 32;
-                }
-                if (cc < ncols) {
-                    uint32_t rt[16];
-                    tmem_ld16(t_s + cc, rt);
-                    tmem_ld_wait();
-                    max_cols<16>(rt, mx4);
-                }
-                tc_fence_before();
-                mbar_arrive(bar_sfree(wg));
-            }
-            if (!ok) break;
-            // a row without a token sees no key: its P is formed against 0 and is exactly 0
-            const float m = exact ? (mxe == -INFINITY ? 0.f : mxe) : fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale + bmax;
-            const float neg_m = -m;
-            // ---- pass B: P chunk by chunk
-            for (int c = 0; c < x.nch; ++c) {
-                const int ncols = min(kChunk, x.npad - c * kChunk);
-                const int s = (int)((ru0 + x.nch + c) % kSlots);
+                const int s = (int)((ru0 + c) % kSlots);
                 const uint32_t a_kc = smem0 + kOffKeyMeta + s * 1024, a_klab = a_kc + 512;
                 ok = mbar_wait_all(bar_sready(wg), n_s & 1, cta_abort);
                 if (!ok) break;
                 ++n_s;
                 tc_fence_after();
-                const int nfull = ncols >> 5;
                 uint32_t ra[32], rb[32];
+                // ---- the chunk's maximum
+                float mc;
+                {
+                    int cc = 0;
+                    if (exact) {
+                        float mxe = -INFINITY;
+                        for (; cc + 32 <= ncols; cc += 32) {
+                            tmem_ld32(t_s + cc, ra);
+                            tmem_ld_wait();
+                            mxe = score_max_cols<32>(ra, cc, bias_i, a_kc, a_klab, label_i, scale, mxe);
+                        }
+                        if (cc < ncols) {
+                            uint32_t rt[16];
+                            tmem_ld16(t_s + cc, rt);
+                            tmem_ld_wait();
+                            mxe = score_max_cols<16>(rt, cc, bias_i, a_kc, a_klab, label_i, scale, mxe);
+                        }
+                        mc = mxe;
+                    } else {
+                        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                        for (; cc + 64 <= ncols; cc += 64) {
+                            tmem_ld32(t_s + cc, ra);
+                            tmem_ld32(t_s + cc + 32, rb);
+                            tmem_ld_wait();
+                            max_cols<32>(ra, mx4);
+                            max_cols<32>(rb, mx4);
+                        }
+                        if (cc + 32 <= ncols) {
+                            tmem_ld32(t_s + cc, ra);
+                            tmem_ld_wait();
+                            max_cols<32>(ra, mx4);
+                            cc += 32;
+                        }
+                        if (cc < ncols) {
+                            uint32_t rt[16];
+                            tmem_ld16(t_s + cc, rt);
+                            tmem_ld_wait();
+                            max_cols<16>(rt, mx4);
+                        }
+                        mc = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale + bmax;
+                    }
+                }
+                // ---- raise the reference if the chunk exceeds it by more than 8 octaves (always from -inf)
+                const bool raise = mc > m + 8.f || (m == -INFINITY && mc > -INFINITY);
+                const bool rescale = raise && m > -INFINITY;          // O holds contributions formed against the old reference
+                if (c > 0 && __any_sync(0xffffffffu, rescale)) {
+                    // the PV products issued so far are complete (this chunk's S was committed after them) and the next
+                    // one waits for this thread's arrival below: O is this thread's to modify
+                    const float f = rescale ? fast_exp2(m - mc) : 1.f;
+#pragma unroll 1
+                    for (int oc = 0; oc < kNO; oc += 16) {
+                        uint32_t ro[16];
+                        tmem_ld16(t_s + kColO + oc, ro);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) ro[e] = __float_as_uint(__uint_as_float(ro[e]) * f);
+                        tmem_st16(t_s + kColO + oc, ro);
+                    }
+                    psum[0] *= f;
+                    psum[1] *= f;
+                }
+                if (raise) m = mc;
+                const float neg_m = m == -INFINITY ? 0.f : -m;
+                // ---- P
+                const int nfull = ncols >> 5;
                 if (nfull > 0) tmem_ld32(t_s, ra);
                 // full-width 32-wide window without mask labels: 32-column group i of chunk c is key row 4 c + i
                 const uint32_t top_c = bias_i + 4 * (c0 - 4 * c * cs);
