@@ -64,8 +64,8 @@ struct Lay {
     static constexpr int kOffK = 0, kOffV = kParts * kKPart, kOffOnes = 2 * kParts * kKPart;
     static constexpr int kSlotBytes = (2 * kParts + (kOnes ? 1 : 0)) * kKPart;
     static constexpr int kOffSlots = kQStages * kQStageBytes;
-    static constexpr int kOffKeyMeta = kOffSlots + kSlots * kSlotBytes;            // per slot: kc[128], klab[128]
-    static constexpr int kOffRowMeta = kOffKeyMeta + kSlots * 1024;                // per Q stage: rowmeta[256], rowtok[256]
+    static constexpr int kOffKeyMeta = kOffSlots + kSlots * kSlotBytes;            // per chunk number % 4: kc[128], klab[128]
+    static constexpr int kOffRowMeta = kOffKeyMeta + 4 * 1024;                     // per Q stage: rowmeta[256], rowtok[256]
     static constexpr int kOffBias = kOffRowMeta + kQStages * 2048;
     static constexpr int kOffBars = ((kOffBias + kBiasFloats * 4 + 1023) / 1024) * 1024;
     static constexpr int kSmemBytes = kOffBars + 1024;
@@ -284,13 +284,17 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
     const uint32_t bar0 = smem0 + kOffBars;
     auto bar_qfull = [&](int s) { return bar0 + 8u * s; };               // Q rows and row tables of an item are there
     auto bar_qempty = [&](int s) { return bar0 + 8u * (2 + s); };        // ... and no longer needed
-    auto bar_kvfull = [&](int s) { return bar0 + 8u * (4 + s); };        // a key chunk is in ring slot s
-    auto bar_kvempty = [&](int s) { return bar0 + 8u * (7 + s); };       // ... and every MMA that reads it is complete
+    // a ring slot's K rows and V rows are handed over separately: the K rows go back when the chunk's QK products are
+    // complete, long before its PV products, so that the K rows of the chunk after next are on their way early
+    auto bar_kfull = [&](int s) { return bar0 + 8u * (4 + s); };         // the K rows (and key tables) of a chunk are in slot s
+    auto bar_kempty = [&](int s) { return bar0 + 8u * (7 + s); };        // ... and every MMA that reads them is complete
+    auto bar_vfull = [&](int s) { return bar0 + 8u * (20 + s); };        // the same for the V rows
+    auto bar_vempty = [&](int s) { return bar0 + 8u * (23 + s); };
     auto bar_sready = [&](int t) { return bar0 + 8u * (10 + t); };       // S of a chunk is in tile t's columns
     auto bar_pready = [&](int t) { return bar0 + 8u * (14 + t); };       // pass B: P of the chunk is in TMEM
     auto bar_oready = [&](int t) { return bar0 + 8u * (16 + t); };       // O of the item is final
     auto bar_ofree = [&](int t) { return bar0 + 8u * (18 + t); };        // ... and has been read
-    unsigned char* tail = smem + kOffBars + 8 * 20;
+    unsigned char* tail = smem + kOffBars + 8 * 26;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail);
     volatile int* cta_abort = reinterpret_cast<volatile int*>(tail + 8);
 
@@ -305,8 +309,10 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             mbar_init(bar_qempty(s), 1 + 256);        // the issuer's commit + every softmax thread
         }
         for (int s = 0; s < kSlots; ++s) {
-            mbar_init(bar_kvfull(s), kLoaderThreads);     // TMA: the bulk-copy warp's lanes + the 64 threads that gather V rows
-            mbar_init(bar_kvempty(s), 1);
+            mbar_init(bar_kfull(s), TMA ? 32 : kLoaderThreads);       // TMA: the bulk-copy warp's lanes
+            mbar_init(bar_vfull(s), TMA ? 64 : kLoaderThreads);       // TMA: the 64 threads that gather V rows
+            mbar_init(bar_kempty(s), 1);
+            mbar_init(bar_vempty(s), 1);
         }
         for (int t = 0; t < 2; ++t) {
             mbar_init(bar_sready(t), 1);
@@ -401,10 +407,10 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                 {
                     for (int c = 0; c < x.nch; ++c, ++ru) {
                         const int s = (int)(ru % kSlots);
-                        ok = mbar_wait_all(bar_kvempty(s), (uint32_t)((ru / kSlots) & 1) ^ 1u, cta_abort);
+                        ok = mbar_wait_all(bar_kempty(s), (uint32_t)((ru / kSlots) & 1) ^ 1u, cta_abort);
                         if (!ok) break;
                         {
-                            int* kcs = reinterpret_cast<int*>(smem + kOffKeyMeta + s * 1024);
+                            int* kcs = reinterpret_cast<int*>(smem + kOffKeyMeta + (int)(ru & 3) * 1024);
                             int* klab = kcs + 128;
                             for (int row = lane; row < kChunk; row += 32) {
                                 const int slot = c * kChunk + row;
@@ -423,11 +429,11 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                         const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes;
                         for (int i = lane; i < wrows * kParts; i += 32) {
                             const int ar = i / kParts, part = i - ar * kParts;
-                            copy_row(maps.k, sb + kOffK + part * kKPart + ar * g.w * kPartBytes, c * wrows + ar, part, bar_kvfull(s));
+                            copy_row(maps.k, sb + kOffK + part * kKPart + ar * g.w * kPartBytes, c * wrows + ar, part, bar_kfull(s));
                         }
                         __syncwarp();
-                        if (lane == 0) mbar_arrive_expect_tx(bar_kvfull(s), (uint32_t)(kChunk * D * 2));
-                        else mbar_arrive(bar_kvfull(s));
+                        if (lane == 0) mbar_arrive_expect_tx(bar_kfull(s), (uint32_t)(kChunk * D * 2));
+                        else mbar_arrive(bar_kfull(s));
                     }
                 }
                 ++kuse;
@@ -449,7 +455,7 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                 {
                     for (int c = 0; c < x.nch; ++c, ++ru) {
                         const int s = (int)(ru % kSlots);
-                        ok = mbar_wait_all(bar_kvempty(s), (uint32_t)((ru / kSlots) & 1) ^ 1u, cta_abort);
+                        ok = mbar_wait_all(bar_vempty(s), (uint32_t)((ru / kSlots) & 1) ^ 1u, cta_abort);
                         if (!ok) break;
                         const uint32_t vb = smem0 + kOffSlots + s * kSlotBytes + kOffV + part * kKPart;
                         for (int row = row0; row < kChunk; row += kRowStep) {
@@ -460,7 +466,7 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
 #pragma unroll
                             for (int c4 = 0; c4 < 4; ++c4) cp_async16(vb + tile_off<32>(row, c4), src + c4 * 8, 16);
                         }
-                        cp_async_mbar_arrive_noinc(bar_kvfull(s));
+                        cp_async_mbar_arrive_noinc(bar_vfull(s));
                     }
                 }
             }
@@ -530,12 +536,12 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             {
                 for (int c = 0; c < x.nch; ++c, ++ru) {
                     const int s = (int)(ru % kSlots);
-                    ok = acquire(bar_kvempty(s), (uint32_t)((ru / kSlots) & 1) ^ 1u);
+                    ok = acquire(bar_kempty(s), (uint32_t)((ru / kSlots) & 1) ^ 1u) && acquire(bar_vempty(s), (uint32_t)((ru / kSlots) & 1) ^ 1u);
                     if (!ok) break;
                     const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes + hf * kKPart;
                     const int ncols = min(kChunk, x.npad - c * kChunk);
                     {
-                        int* kcs = reinterpret_cast<int*>(smem + kOffKeyMeta + s * 1024);
+                        int* kcs = reinterpret_cast<int*>(smem + kOffKeyMeta + (int)(ru & 3) * 1024);
                         int* klab = kcs + 128;
                         for (int row = lt; row < kChunk; row += kLoaderThreads) {
                             const int slot = c * kChunk + row;
@@ -569,7 +575,8 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                             cp_async16(sb + kOffV + so, bytes ? sv + c4 * 8 : sv, bytes);
                         }
                     }
-                    issued(bar_kvfull(s));
+                    issued(bar_kfull(s));
+                    cp_async_mbar_arrive_noinc(bar_vfull(s));
                 }
             }
             ++kuse;
@@ -613,25 +620,43 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             };
             // tile t's S columns are free for the next chunk's QK product by the order of the MMAs: the P that replaced S
             // was consumed by its PV product, issued earlier from this thread
-            auto chunk_ready = [&](long long use) -> bool {
-                if (!mbar_wait_all(bar_kvfull((int)(use % kSlots)), (uint32_t)((use / kSlots) & 1), cta_abort)) return false;
+            auto k_ready = [&](long long use) -> bool {
+                if (!mbar_wait_all(bar_kfull((int)(use % kSlots)), (uint32_t)((use / kSlots) & 1), cta_abort)) return false;
                 fence_proxy_async();
                 return true;
             };
+            auto v_ready = [&](long long use) -> bool {
+                if (!mbar_wait_all(bar_vfull((int)(use % kSlots)), (uint32_t)((use / kSlots) & 1), cta_abort)) return false;
+                fence_proxy_async();
+                return true;
+            };
+            // after the QK products of the item's last chunk have been issued: the commit frees the Q stage when they
+            // are complete, so that the next item's query rows load while this item's last chunk is worked on
+            auto last_qk_issued = [&]() {
+                if (elect_one()) mma_commit(bar_qempty(qs));
+                __syncwarp();
+            };
             // ---- per tile, PV of chunk c is followed at once by QK of chunk c + 1, so that a tile's softmax threads wait
             // for one PV and one QK product only, whatever the other tile is doing
-            ok = chunk_ready(ru);
+            ok = k_ready(ru);
             for (int t = 0; t < x.ntiles && ok; ++t)
                 issue_qk(t, smem0 + kOffSlots + (int)(ru % kSlots) * kSlotBytes, min(kChunk, x.npad));
+            if (ok) {
+                if (elect_one()) mma_commit(bar_kempty((int)(ru % kSlots)));
+                __syncwarp();
+                if (x.nch == 1) last_qk_issued();
+            }
             for (int c = 0; c < x.nch && ok; ++c, ++ru) {
                 const int s = (int)(ru % kSlots);
                 const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes;
                 const int ncols = min(kChunk, x.npad - c * kChunk);
                 const bool has_next = c + 1 < x.nch;
                 if (has_next) {
-                    ok = chunk_ready(ru + 1);
+                    ok = k_ready(ru + 1);
                     if (!ok) break;
                 }
+                ok = v_ready(ru);
+                if (!ok) break;
                 const uint32_t sb_n = smem0 + kOffSlots + (int)((ru + 1) % kSlots) * kSlotBytes;
                 const int ncols_n = min(kChunk, x.npad - (c + 1) * kChunk);
                 for (int t = 0; t < x.ntiles && ok; ++t) {
@@ -659,12 +684,14 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                     else issue_qk(t, sb_n, ncols_n);
                 }
                 if (!ok) break;
-                if (elect_one()) mma_commit(bar_kvempty(s));
+                if (elect_one()) {
+                    mma_commit(bar_vempty(s));
+                    if (has_next) mma_commit(bar_kempty((int)((ru + 1) % kSlots)));
+                }
                 __syncwarp();
+                if (has_next && c + 2 == x.nch) last_qk_issued();
             }
             if (!ok) break;
-            if (elect_one()) mma_commit(bar_qempty(qs));
-            __syncwarp();
             ++kuse;
         }
     }
@@ -707,8 +734,7 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             float psum[2] = {0.f, 0.f};
             for (int c = 0; c < x.nch; ++c) {
                 const int ncols = min(kChunk, x.npad - c * kChunk);
-                const int s = (int)((ru0 + c) % kSlots);
-                const uint32_t a_kc = smem0 + kOffKeyMeta + s * 1024, a_klab = a_kc + 512;
+                const uint32_t a_kc = smem0 + kOffKeyMeta + (int)((ru0 + c) & 3) * 1024, a_klab = a_kc + 512;
                 ok = mbar_wait_all(bar_sready(wg), n_s & 1, cta_abort);
                 if (!ok) break;
                 ++n_s;
