@@ -201,7 +201,8 @@ struct KvMaps64 {
 
 // TMA: complete windows of side 16 or 32 and a longitude shift that is a multiple of 8: one loader warp fetches every
 // window row with tiled bulk copies (per-query lse and delta by 4-byte cp.async copies tied to the same barrier);
-// otherwise three loader warps gather the rows with 16-byte cp.async copies.
+// otherwise three loader warps gather the rows with 16-byte cp.async copies.  (Gathering the dO rows with the two
+// idle warps next to the bulk copies, as the forward kernel does with V, was measured and is slightly slower here.)
 template <int D, bool TMA>
 __global__ void __launch_bounds__(kThreads, 1)
 swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
@@ -349,33 +350,20 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
         }
     } else if (warp >= kLoaderWarp0) {
         // ------------------------------------------------------------------ loaders
-        // D / 32 lanes per row (one 32-column part of the row each, four 16-byte copies).  A group of copies is
-        // published when the next one has been issued; if a ring has no free place the pending group is published first.
+        // D / 32 lanes per row (one 32-column part of the row each, four 16-byte copies).  A thread never waits for
+        // data: its arrival on a stage's or slot's barrier is tied to the completion of the copies it has issued.
         const int lt = (warp - kLoaderWarp0) * 32 + lane;
         const int hf = lt % kParts;
         const int lrow = lt / kParts;
         constexpr int kRowsPerIter = kLoaderThreads / kParts;
         int kuse = 0;
         long long ru = 0;
-        uint32_t pending_bar = 0;
         bool ok = true;
-        auto acquire = [&](uint32_t bar, uint32_t parity) -> bool {
-            if (pending_bar && !__all_sync(0xffffffffu, mbar_test_wait(bar, parity))) {
-                cp_async_wait<0>();
-                fence_proxy_async();
-                mbar_arrive(pending_bar);
-                pending_bar = 0;
-            }
-            return mbar_wait_all(bar, parity, cta_abort);
-        };
+        auto acquire = [&](uint32_t bar, uint32_t parity) -> bool { return mbar_wait_all(bar, parity, cta_abort); };
+        // the thread's table entries are visible to the CTA before its arrival, which follows its copies
         auto issued = [&](uint32_t bar) {
-            cp_async_commit();
-            if (pending_bar) {
-                cp_async_wait<1>();
-                fence_proxy_async();
-                mbar_arrive(pending_bar);
-            }
-            pending_bar = bar;
+            __threadfence_block();
+            cp_async_mbar_arrive_noinc(bar);
         };
         ItemCursor cur = cursor_init(cta_in_head, ctas_per_head, max_tiles, g.Mw, g.Mh);
         for (long long it = cta_in_head; ok && it < n_items; it += ctas_per_head, cursor_advance(cur, max_tiles, g.Mw, g.Mh)) {
@@ -472,11 +460,6 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                 issued(bar_qfull(s));
             }
             ++kuse;
-        }
-        if (pending_bar) {
-            cp_async_wait<0>();
-            fence_proxy_async();
-            mbar_arrive(pending_bar);
         }
     } else {
         // ------------------------------------------------------------------ MMA issuer

@@ -207,13 +207,13 @@ __device__ __forceinline__ void cols16(const uint32_t (&rs)[16], const uint32_t 
 
 struct QMaps64 {
     RowMaps3 q, g;            // query rows and their output gradients, by window rows
-    CUtensorMap k, v;         // keys by runs of 16 vertically adjacent tokens
+    CUtensorMap k;            // K rows by runs of 16 vertically adjacent tokens
 };
 
 // TMA: both shifts are multiples of 16 (8 suffices for the longitude): one loader warp fetches the query rows window
-// row by window row and the key units as four runs of 16 vertically adjacent tokens with tiled bulk copies (per-query
-// lse and delta by 4-byte cp.async copies tied to the same barrier); otherwise three loader warps gather every row
-// with 16-byte cp.async copies.
+// row by window row and the K units as four runs of 16 vertically adjacent tokens with tiled bulk copies (per-query
+// lse and delta by 4-byte cp.async copies tied to the same barrier), the other two gather the V units with 16-byte
+// cp.async copies; otherwise all three gather every row.
 template <int D, bool TMA>
 __global__ void __launch_bounds__(kThreads, 1)
 swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
@@ -263,7 +263,7 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
             mbar_init(bar_kempty(u), 1);
         }
         for (int u = 0; u < kVUnits; ++u) {
-            mbar_init(bar_vfull(u), TMA ? 32 : kLoaderThreads);
+            mbar_init(bar_vfull(u), TMA ? 64 : kLoaderThreads);       // TMA: the 64 threads that gather V rows
             mbar_init(bar_vempty(u), 1);
         }
         for (int b = 0; b < 3; ++b) {
@@ -299,8 +299,9 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
             int quse = 0;
             unsigned ru = 0;                              // half chunks so far
             bool ok = true;
-            // the K unit, then the V unit, of half chunk n of the window at `cw`: rows 16 i .. 16 i + 15 of a unit are
-            // the tokens of window rows 16 (n % 2) .. + 15 in window column 4 (n / 2) + i
+            // the K unit of half chunk n of the window at `cw`: rows 16 i .. 16 i + 15 of a unit are the tokens of window
+            // rows 16 (n % 2) .. + 15 in window column 4 (n / 2) + i.  (The V units are gathered by the other two loader
+            // warps: the bulk-copy engine takes a fixed time per 64-byte row, and the two ways of loading run side by side.)
             auto load_half = [&](const Cursor& cw, int n) -> bool {
                 const int c = n >> 1, h = n & 1;
                 int u0 = cw.wr * kW + 16 * h + g.sh;
@@ -310,7 +311,7 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
                 int vcol = cw.wc * kW + 4 * c + i + g.sw;
                 if (vcol >= g.W) vcol -= g.W;
                 const uint32_t uoff = part * kUPart + i * 16 * kPartBytes;
-                const int uk = (int)(ru % kKUnits), uv = (int)(ru % kVUnits);
+                const int uk = (int)(ru % kKUnits);
                 if (!mbar_wait_all(bar_kempty(uk), (uint32_t)((ru / kKUnits) & 1) ^ 1u, cta_abort)) return false;
                 for (int r = lane; r < 64; r += 32) {
                     int code, label;
@@ -320,10 +321,6 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
                 if (lane < 4 * kParts) tma_load_3d(smem0 + kOffKRing + uk * kUnitBytes + uoff, &maps.k, head * D + part * 32, vcol, z, bar_kfull(uk));
                 if (lane == 0) mbar_arrive_expect_tx(bar_kfull(uk), (uint32_t)(64 * D * 2));
                 else mbar_arrive(bar_kfull(uk));
-                if (!mbar_wait_all(bar_vempty(uv), (uint32_t)((ru / kVUnits) & 1) ^ 1u, cta_abort)) return false;
-                if (lane < 4 * kParts) tma_load_3d(smem0 + kOffVRing + uv * kUnitBytes + uoff, &maps.v, head * D + part * 32, vcol, z, bar_vfull(uv));
-                if (lane == 0) mbar_arrive_expect_tx(bar_vfull(uv), (uint32_t)(64 * D * 2));
-                else mbar_arrive(bar_vfull(uv));
                 ++ru;
                 return true;
             };
@@ -370,6 +367,29 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
                 if (it + 1 < it_hi)
                     for (; fetched < L::kKeysFirst && ok; ++fetched) ok = load_half(cur, fetched);
             }
+        } else {
+            // ---- warps 10, 11: the V units, one row of 64 per thread, with 16-byte cp.async copies; a thread's arrival
+            // on the unit's barrier is tied to the completion of its copies, so it never waits for data
+            const int r = (warp - kLoaderWarp0 - 1) * 32 + lane;       // 0 .. 63
+            unsigned ru = 0;
+            bool ok = true;
+            Cursor cur = cursor_at(g, it_lo);
+            for (long long it = it_lo; ok && it < it_hi; ++it, cursor_next(g, cur)) {
+                const size_t sample_off = (size_t)cur.b * HW;
+                for (int n = 0; n < kHalfChunks; ++n, ++ru) {
+                    const int uv = (int)(ru % kVUnits);
+                    ok = mbar_wait_all(bar_vempty(uv), (uint32_t)((ru / kVUnits) & 1) ^ 1u, cta_abort);
+                    if (!ok) break;
+                    int code, label;
+                    const int tok = slot_token(g, cur, chunk_slot(n >> 1, 64 * (n & 1) + r), code, label);
+                    const __nv_bfloat16* src = v + (sample_off + (size_t)tok) * g.ts + head * D;
+                    const uint32_t vb = smem0 + kOffVRing + uv * kUnitBytes;
+#pragma unroll
+                    for (int piece = 0; piece < D / 8; ++piece)
+                        cp_async16(vb + (piece >> 2) * kUPart + tile_off<32>(r, piece & 3), src + piece * 8, 16);
+                    cp_async_mbar_arrive_noinc(bar_vfull(uv));
+                }
+            }
         }
     } else if (warp >= kLoaderWarp0) {
         // ------------------------------------------------------------------ loaders
@@ -383,31 +403,14 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
         const uint32_t u_piece_off = (uint32_t)(piece >> 2) * kUPart;     // ... in a key unit
         int quse = 0;
         unsigned ru = 0;                                  // half chunks so far (a CTA sees far fewer than 2^32)
-        uint32_t pending_bar = 0, pending_bar2 = 0;       // barriers of the group of copies in flight (the second may be 0)
         bool ok = true;
-        auto arrive_pending = [&]() {
-            fence_proxy_async();
-            mbar_arrive(pending_bar);
-            if (pending_bar2) mbar_arrive(pending_bar2);
-            pending_bar = pending_bar2 = 0;
-        };
-        // no free place yet: the group in flight is published first, or the consumers could never free one
-        auto acquire = [&](uint32_t bar, uint32_t parity) -> bool {
-            if (pending_bar && !__all_sync(0xffffffffu, mbar_test_wait(bar, parity))) {
-                cp_async_wait<0>();
-                arrive_pending();
-            }
-            return mbar_wait_all(bar, parity, cta_abort);
-        };
-        // a group is published when the next one has been issued
+        // A thread never waits for data: its arrival on a barrier is tied to the completion of the copies it has issued.
+        auto acquire = [&](uint32_t bar, uint32_t parity) -> bool { return mbar_wait_all(bar, parity, cta_abort); };
+        // (the thread's table entries are visible to the CTA before its arrivals, which follow its copies)
         auto issued = [&](uint32_t bar, uint32_t bar2) {
-            cp_async_commit();
-            if (pending_bar) {
-                cp_async_wait<1>();
-                arrive_pending();
-            }
-            pending_bar = bar;
-            pending_bar2 = bar2;
+            __threadfence_block();
+            cp_async_mbar_arrive_noinc(bar);
+            if (bar2) cp_async_mbar_arrive_noinc(bar2);
         };
         // the K and V rows of half chunk n of the window at `cw`, one group of copies
         auto load_half = [&](const Cursor& cw, int n) -> bool {
@@ -476,10 +479,6 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
             fetched = 0;
             if (it + 1 < it_hi)
                 for (; fetched < L::kKeysFirst && ok; ++fetched) ok = load_half(cur, fetched);
-        }
-        if (pending_bar) {
-            cp_async_wait<0>();
-            arrive_pending();
         }
     } else {
         // ------------------------------------------------------------------ MMA issuer
@@ -734,7 +733,7 @@ cudaError_t launch_bwd_q64(const Geo& g, const void* q, const void* k, const voi
     static const bool tma_off = [] { const char* e_ = std::getenv("TERRA_NO_TMA"); return e_ && e_[0] == '1'; }();
     // (at head dim 64 the runs of 16 tokens are 1 KB copies, and the three gathering warps are faster)
     const bool tma = !tma_off && g.d == 128 && bulk_rows_shape(g) && g.sh % 16 == 0 && make_row_maps3(&maps.q, g, q, g.ts) &&
-                     make_row_maps3(&maps.g, g, d_o, g.heads * g.d) && make_col_map(&maps.k, g, k, g.ts) && make_col_map(&maps.v, g, v, g.ts);
+                     make_row_maps3(&maps.g, g, d_o, g.heads * g.d) && make_col_map(&maps.k, g, k, g.ts);
     auto kern = g.d == 64 ? swin_bwd_q64_kernel<64, false> : (tma ? swin_bwd_q64_kernel<128, true> : swin_bwd_q64_kernel<128, false>);
     const int smem_bytes = g.d == 64 ? Lay<64>::kSmemBytes : Lay<128>::kSmemBytes;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
