@@ -64,6 +64,9 @@ CONFIGS = {
     # The window-assignment study's largest window (Section VII-E: small model, w = 128; the 2041 x 4320 field at
     # patch 4 and sampling factor 2 padded to a 2 x 5 grid of 128 x 128 windows, i.e. 256 x 640 tokens)
     "tv_small_w128": SwinConfig("tv_small_w128", 1, 256, 640, 8, 128, 128, 64, 64, index=9),
+    # A 3 x 5-window slice of the large model's block (same heads, head dim, window, shift): 2.3 GB on the device
+    # with gradients, the size a full-counter profiler capture of the head-dim-128 tcgen05 kernels is taken on
+    "tv_large_slice": SwinConfig("tv_large_slice", 1, 96, 160, 64, 128, 32, 16, 16, index=10),
 }
 
 TENSOR_INDEX = {"q": 0, "k": 1, "v": 2, "do": 3, "bias": 4}

@@ -24,6 +24,8 @@ SHAPES = [
     ("d128_w16_bulk", 1, 32, 48, 2, 128, 16, 8, 8, 0, 1),
     ("d128_w32_bulk_shift24", 1, 64, 64, 1, 128, 32, 8, 24, 0, 0),  # seam after 8 of a row's 32 tokens, masks on both axes
     ("d128_w32_bulk_noshift", 2, 32, 64, 2, 128, 32, 0, 0, 0, 1),
+    # complete windows whose shifts are not multiples of 8: every row is gathered with 16-byte copies
+    ("d128_w32_gather", 1, 64, 64, 1, 128, 32, 12, 12, 0, 1),
 ]
 
 

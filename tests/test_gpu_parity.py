@@ -31,6 +31,7 @@ EDGE = [
     ("tma_nonperiodic", 1, 46, 64, 2, 32, 16, 8, 16, 0, 0),      # masks on both axes
     ("bulk64_w32", 1, 64, 96, 2, 64, 32, 16, 8, 0, 1),           # head dim 64, complete windows: rows by tiled bulk copies
     ("bulk64_w16", 2, 32, 48, 2, 64, 16, 8, 8, 0, 0),
+    ("gather64_w32", 1, 64, 64, 2, 64, 32, 12, 20, 0, 0),        # complete windows, shifts not multiples of 8: rows gathered
     ("tma_noshift", 1, 32, 40, 2, 32, 16, 0, 0, 0, 1),
 ]
 
