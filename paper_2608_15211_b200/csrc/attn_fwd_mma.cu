@@ -39,8 +39,8 @@ __device__ __forceinline__ void load_rows(unsigned char* s_tile, const __nv_bflo
 // bias table no longer fit shared memory, so the tables cover the CTA's 64 query rows plus the key block in flight
 // (two stages) and the bias is read from the caller's table in global memory.
 template <int D, bool BIG>
-__global__ void __launch_bounds__(NTHREADS)
-swin_fwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
+__device__ __forceinline__ void
+swin_fwd_mma_body(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                     const __nv_bfloat16* __restrict__ v, const float* __restrict__ bias,
                     __nv_bfloat16* __restrict__ o, float* __restrict__ lse, int qtiles) {
     constexpr int KS = D / 16;       // k-steps of Q K^T
@@ -68,8 +68,10 @@ swin_fwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
     int* s_meta = s_tok + ntab;
     float* s_bias = reinterpret_cast<float*>(s_meta + ntab);
     unsigned char* s_q = smem + (((size_t)ntab * 8 + (BIG ? 0 : (size_t)nbias * 4) + 127) / 128) * 128;
-    unsigned char* s_k = s_q + TILE_BYTES;           // two stages
-    unsigned char* s_v = s_k + 2 * TILE_BYTES;       // two stages
+    // K and V: two stages each; one where no window has more than one key block (then more CTAs fit an SM)
+    const int nstages = (BIG || npad_max > BN) ? 2 : 1;
+    unsigned char* s_k = s_q + TILE_BYTES;
+    unsigned char* s_v = s_k + nstages * TILE_BYTES;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int gq = lane >> 2, tq = lane & 3;
@@ -259,11 +261,30 @@ swin_fwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
     }
 }
 
+template <int D, bool BIG>
+__global__ void __launch_bounds__(NTHREADS)
+swin_fwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
+                    const __nv_bfloat16* __restrict__ v, const float* __restrict__ bias,
+                    __nv_bfloat16* __restrict__ o, float* __restrict__ lse, int qtiles) {
+    swin_fwd_mma_body<D, BIG>(g, q, k, v, bias, o, lse, qtiles);
+}
+
+// Head dim 128 with windows of at most 64 tokens (the paper's 8 x 8 windows): one key block per window, so a CTA needs
+// three tiles of shared memory instead of five, and with 168 registers per thread three CTAs share an SM; the path is
+// bound by HBM and lives on the loads the resident CTAs keep in flight.
+__global__ void __launch_bounds__(NTHREADS, 3)
+swin_fwd_mma_d128_small_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
+                               const __nv_bfloat16* __restrict__ v, const float* __restrict__ bias,
+                               __nv_bfloat16* __restrict__ o, float* __restrict__ lse, int qtiles) {
+    swin_fwd_mma_body<128, false>(g, q, k, v, bias, o, lse, qtiles);
+}
+
 size_t fwd_smem_bytes(const Geo& g) {
     int npad_max = ((g.nmax + BN - 1) / BN) * BN;
     int nbias = (2 * g.w - 1) * (2 * g.w - 1);
     size_t head = g.w > 32 ? (size_t)3 * BN * 8 : (((size_t)npad_max * 8 + (size_t)nbias * 4 + 127) / 128) * 128;
-    return head + 5 * (size_t)BN * g.d * 2;
+    const int nstages = (g.w > 32 || npad_max > BN) ? 2 : 1;
+    return head + (size_t)(1 + 2 * nstages) * BN * g.d * 2;
 }
 
 }  // namespace
@@ -274,7 +295,8 @@ cudaError_t TERRA_ELEM_FN(launch_fwd_mma)(const Geo& g, const void* q, const voi
     const long long items = (long long)g.B * g.Mh * g.Mw * g.heads * qtiles;
     const size_t smem = fwd_smem_bytes(g);
     auto kern = g.w > 32 ? ((g.d == 32) ? swin_fwd_mma_kernel<32, true> : (g.d == 64) ? swin_fwd_mma_kernel<64, true> : swin_fwd_mma_kernel<128, true>)
-                         : ((g.d == 32) ? swin_fwd_mma_kernel<32, false> : (g.d == 64) ? swin_fwd_mma_kernel<64, false> : swin_fwd_mma_kernel<128, false>);
+                         : ((g.d == 32) ? swin_fwd_mma_kernel<32, false> : (g.d == 64) ? swin_fwd_mma_kernel<64, false>
+                            : (g.nmax <= BN ? swin_fwd_mma_d128_small_kernel : swin_fwd_mma_kernel<128, false>));
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     prof_begin("swin_fwd_mma_kernel", stream);
