@@ -124,6 +124,15 @@ static size_t fwd_bytes(const Geo& g) {
     return 0;
 }
 
+// TERRA_SPLIT_SMALL=1: a debugging switch that keeps small windows at head dim 128 on the two-kernel register-tile backward
+static bool force_split_small() {
+    static const bool on = [] {
+        const char* v = std::getenv("TERRA_SPLIT_SMALL");
+        return v && v[0] == '1';
+    }();
+    return on;
+}
+
 static bool use_bwd_tc(const Geo& g) { return bwd_tc_supported(g) && !force_register_path() && !g.f16; }
 
 static bool use_bwd_kv64(const Geo& g) { return bwd_kv64_supported(g) && !force_register_path() && !g.f16 && !small_window_128(g); }
@@ -243,6 +252,12 @@ static int bwd_call(const Geo& g, const void* q, const void* k, const void* v,
     if (use_bwd_tc(g)) {
         cudaError_t et = launch_bwd_tc(g, q, k, v, bias_table, o, lse, d_o, dq, dk, dv, dbias, workspace, sms, st);
         return et == cudaSuccess ? TERRA_OK : cuda_fail(et, "terra_swin_attn_bwd");
+    }
+    if (bwd_small_supported(g) && !force_split_small()) {
+        // windows of at most 64 tokens at head dim 128: one kernel reads every tensor once
+        cudaError_t es = g.f16 ? launch_bwd_small_f16(g, q, k, v, o, d_o, bias_table, lse, dq, dk, dv, dbias, sms, st)
+                               : launch_bwd_small(g, q, k, v, o, d_o, bias_table, lse, dq, dk, dv, dbias, sms, st);
+        return es == cudaSuccess ? TERRA_OK : cuda_fail(es, "terra_swin_attn_bwd");
     }
     float* delta = reinterpret_cast<float*>(workspace);
     if (g.f16) {

@@ -441,6 +441,253 @@ swin_bwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
     }
 }
 
+// out (16 x D per warp, the warp's 16 key rows) += coef^T x block, where coef is a 64 x 64 tile in shared memory
+// ([query][key], 128-byte rows in the swizzled layout of a 64-column tile) and block the 64 x D rows of the queries
+template <int D>
+__device__ __forceinline__ void coef_t_times_block(float (&out)[D / 8][4], const unsigned char* coef, const unsigned char* blk,
+                                                   int warp, int lane) {
+#pragma unroll
+    for (int ks = 0; ks < BN / 16; ++ks) {
+        // A fragment (16 keys x 16 queries) = transpose of coef[16 ks .. + 15][16 warp .. + 15]
+        uint32_t pf[4];
+        const int mat = lane >> 3;
+        ldmatrix_x4_trans(pf, smem_u32(coef + tile_off<64>(ks * 16 + (mat >> 1) * 8 + (lane & 7), 2 * warp + (mat & 1))));
+#pragma unroll
+        for (int dp = 0; dp < D / 16; ++dp) {
+            uint32_t bf[4];
+            int r = ks * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+            ldmatrix_x4_trans(bf, smem_u32(blk + tile_off<D>(r, 2 * dp + (lane >> 4))));
+            mma_elem(out[2 * dp], pf, bf[0], bf[1]);
+            mma_elem(out[2 * dp + 1], pf, bf[2], bf[3]);
+        }
+    }
+}
+
+// The whole backward of windows of at most 64 tokens in one kernel (the paper's 8 x 8 windows): a CTA holds the
+// window's Q, K, V, dO and O rows of one head, so every tensor is read once and dQ, dK, dV are written once (the
+// split into a key side and a query side reads the inputs twice, and a third time for delta).
+//   delta = rowsum(dO * O)                                 (per query row, from the two tiles)
+//   query-major, a warp owns 16 query rows:  S = Q K^T, dP = dO V^T, P = exp2(S scale + bias - lse), dS = P (dP - delta),
+//   the bias gradient (as in the query-side kernel above), dQ = dS K; P and dS go to shared memory as 64 x 64 tiles
+//   key-major, a warp owns 16 key rows:      dV = P^T dO, dK = dS^T Q  (A fragments by transposing loads of those tiles)
+// Persistent CTAs bound to one head walk over (batch, window).  Shared memory: the four operand tiles, one more that
+// holds O first and P | dS afterwards, the slot tables, the summed-dS image and the staging tile of the bias gradient.
+template <int D>
+__global__ void __launch_bounds__(NTHREADS, 2)
+swin_bwd_small_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
+                      const __nv_bfloat16* __restrict__ v, const __nv_bfloat16* __restrict__ o,
+                      const __nv_bfloat16* __restrict__ d_o, const float* __restrict__ bias, const float* __restrict__ lse,
+                      __nv_bfloat16* __restrict__ dq, __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv,
+                      float* __restrict__ dbias, int ctas_per_head, int acc_stride) {
+    constexpr int KS = D / 16;
+    constexpr int DT = D / 8;
+    constexpr int TILE_BYTES = BN * D * 2;
+    constexpr int X_BYTES = TILE_BYTES > 16384 ? TILE_BYTES : 16384;      // O, then P (8 KB) | dS (8 KB)
+    extern __shared__ __align__(128) unsigned char smem[];
+
+    const int nbias = (2 * g.w - 1) * (2 * g.w - 1);
+    int* s_tok = reinterpret_cast<int*>(smem);
+    int* s_meta = s_tok + BN;
+    float* s_lse = reinterpret_cast<float*>(s_meta + BN);
+    float* s_delta = s_lse + BN;
+    float* s_bias = s_delta + BN;
+    float* s_dbias = s_bias + nbias;
+    unsigned char* s_q = smem + (((size_t)BN * 16 + (size_t)nbias * 8 + 127) / 128) * 128;
+    unsigned char* s_k = s_q + TILE_BYTES;
+    unsigned char* s_v = s_k + TILE_BYTES;
+    unsigned char* s_g = s_v + TILE_BYTES;            // dO
+    unsigned char* s_x = s_g + TILE_BYTES;
+    unsigned char* s_p = s_x;                         // P as a 64 x 64 tile
+    unsigned char* s_ds = s_x + 8192;                 // dS as a 64 x 64 tile
+    float* s_acc = reinterpret_cast<float*>(s_x + X_BYTES);              // 64 x acc_stride image of summed dS
+    float* s_stage = s_acc + BM * acc_stride;                            // 4 warps x 16 x kStageStride
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int gq = lane >> 2, tq = lane & 3;
+    const int head = blockIdx.x % g.heads;
+    const int M = g.Mh * g.Mw;
+    const int c0 = (g.w - 1) * 2 * g.w;
+    const long long n_items = (long long)g.B * M;
+    const int dense = g.heads * D;                    // token stride of o and dO
+
+    for (int i = tid; i < nbias; i += NTHREADS) {
+        s_bias[i] = bias[(size_t)i * g.heads + head] * kLog2e;
+        s_dbias[i] = 0.f;
+    }
+    for (int i = tid; i < BM * acc_stride; i += NTHREADS) s_acc[i] = 0.f;
+
+    for (long long item = blockIdx.x / g.heads; item < n_items; item += ctas_per_head) {
+        const int win = (int)(item % M);
+        const int b = (int)(item / M);
+        const WindowRef r = window_ref(g, win);
+        const size_t sample_off = (size_t)b * g.H * g.W;
+
+        __syncthreads();   // the previous item's readers of the tables and tiles are done
+        if (tid < BN) {
+            int meta = 0xff << 16, tok = -1;
+            float l2 = INFINITY;                    // padded queries: P = exp2(x - inf) = 0
+            if (tid < r.n) {
+                tok = slot_token(g, r, tid, meta);
+                l2 = lse[(sample_off + (size_t)tok) * g.heads + head] * kLog2e;
+            }
+            s_tok[tid] = tok;
+            s_meta[tid] = meta;
+            s_lse[tid] = l2;
+        }
+        __syncthreads();
+        load_rows<D>(s_q, q, s_tok, 0, sample_off, g.ts, head, tid);
+        load_rows<D>(s_k, k, s_tok, 0, sample_off, g.ts, head, tid);
+        load_rows<D>(s_v, v, s_tok, 0, sample_off, g.ts, head, tid);
+        load_rows<D>(s_g, d_o, s_tok, 0, sample_off, dense, head, tid);
+        load_rows<D>(s_x, o, s_tok, 0, sample_off, dense, head, tid);
+        cp_async_commit();
+        cp_async_wait<0>();
+        __syncthreads();
+
+        // ---- delta of the warp's 16 query rows: two lanes per row, half a row each
+        {
+            const int row = warp * 16 + (lane >> 1);
+            float acc = 0.f;
+#pragma unroll
+            for (int c = 0; c < DT / 2; ++c) {
+                const int chunk = (lane & 1) * (DT / 2) + c;
+                const uint4 a = *reinterpret_cast<const uint4*>(s_x + tile_off<D>(row, chunk));
+                const uint4 bb = *reinterpret_cast<const uint4*>(s_g + tile_off<D>(row, chunk));
+                const uint32_t* pa = reinterpret_cast<const uint32_t*>(&a);
+                const uint32_t* pb = reinterpret_cast<const uint32_t*>(&bb);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float2 x = elem2_to_float2(pa[e]), y = elem2_to_float2(pb[e]);
+                    acc += x.x * y.x + x.y * y.y;
+                }
+            }
+            acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+            if ((lane & 1) == 0) s_delta[row] = acc;
+        }
+        __syncthreads();   // O has been read by every warp: its tile becomes P | dS
+
+        // ---- query-major part
+        const int row_tab[2] = {warp * 16 + gq, warp * 16 + gq + 8};
+        const int meta_r[2] = {s_meta[row_tab[0]], s_meta[row_tab[1]]};
+        const float lse_r[2] = {s_lse[row_tab[0]], s_lse[row_tab[1]]};
+        const float del_r[2] = {s_delta[row_tab[0]], s_delta[row_tab[1]]};
+        float acc1[DT][4];
+        {
+            static_assert(!kFragsInRegs<D>, "the own-row fragments are read from shared memory at each use");
+            uint32_t f0[1][4];
+            float acc_s[BN / 8][4], acc_dp[BN / 8][4];
+            rows_times_block_t<D>(acc_s, f0, s_q, s_k, warp, lane);
+            rows_times_block_t<D>(acc_dp, f0, s_g, s_v, warp, lane);
+#pragma unroll
+            for (int nt = 0; nt < BN / 8; ++nt) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int col = nt * 8 + 2 * tq + (e & 1);
+                    const int mc = s_meta[col];
+                    const int mr = meta_r[e >> 1];
+                    const bool ok = meta_label(mr) == meta_label(mc);
+                    const int bidx = meta_code(mr) - meta_code(mc) + c0;
+                    float p = fast_exp2(acc_s[nt][e] * g.scale_log2e + s_bias[bidx] - lse_r[e >> 1]);
+                    p = ok ? p : 0.f;
+                    acc_s[nt][e] = p;
+                    acc_dp[nt][e] = p * (acc_dp[nt][e] - del_r[e >> 1]);
+                }
+            }
+            // bias gradient
+            if (r.ew == g.w) {
+                // full-width window: this thread owns these cells of the image (binned into the table at the end)
+                float2* cell0 = reinterpret_cast<float2*>(s_acc + (warp * 16 + gq) * acc_stride + 2 * tq);
+                float2 cur[BN / 8][2];
+#pragma unroll
+                for (int nt = 0; nt < BN / 8; ++nt) {
+                    cur[nt][0] = cell0[nt * 4];
+                    cur[nt][1] = cell0[nt * 4 + 4 * acc_stride];
+                }
+#pragma unroll
+                for (int nt = 0; nt < BN / 8; ++nt) {
+                    cur[nt][0].x += acc_dp[nt][0]; cur[nt][0].y += acc_dp[nt][1];
+                    cur[nt][1].x += acc_dp[nt][2]; cur[nt][1].y += acc_dp[nt][3];
+                }
+#pragma unroll
+                for (int nt = 0; nt < BN / 8; ++nt) {
+                    cell0[nt * 4] = cur[nt][0];
+                    cell0[nt * 4 + 4 * acc_stride] = cur[nt][1];
+                }
+            } else {
+                // narrow edge window: through the staging tile, one shared-memory atomic per pair, 32 different table
+                // entries per instruction
+                float* stage = s_stage + warp * 16 * kStageStride;
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+#pragma unroll
+                    for (int nt = 4 * half; nt < 4 * half + 4; ++nt) {
+                        const int col = (nt - 4 * half) * 8 + 2 * tq;
+                        *reinterpret_cast<float2*>(stage + gq * kStageStride + col) = make_float2(acc_dp[nt][0], acc_dp[nt][1]);
+                        *reinterpret_cast<float2*>(stage + (gq + 8) * kStageStride + col) = make_float2(acc_dp[nt][2], acc_dp[nt][3]);
+                    }
+                    __syncwarp();
+                    const int code_c = meta_code(s_meta[half * 32 + lane]);
+                    for (int rr = 0; rr < 16; ++rr) {
+                        const int code_r = meta_code(s_meta[warp * 16 + rr]) + c0;
+                        const float v0 = stage[rr * kStageStride + lane];
+                        if (v0 != 0.f) atomicAdd(&s_dbias[code_r - code_c], v0);
+                    }
+                    __syncwarp();
+                }
+            }
+            // P and dS as 64 x 64 tiles for the key-major part
+            stage_rows<64>(s_p, acc_s, 1.f, warp, gq, tq);
+            stage_rows<64>(s_ds, acc_dp, 1.f, warp, gq, tq);
+            // dQ = dS K
+#pragma unroll
+            for (int i = 0; i < DT; ++i)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) acc1[i][e] = 0.f;
+            coef_times_block<D>(acc1, acc_dp, s_k, lane);
+        }
+        __syncthreads();   // P, dS are complete; K and V have been read by every warp
+        const float scale = g.scale_log2e * kLn2;
+        stage_rows<D>(s_v, acc1, scale, warp, gq, tq);           // dQ into the V tile
+
+        // ---- key-major part
+#pragma unroll
+        for (int i = 0; i < DT; ++i)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc1[i][e] = 0.f;
+        coef_t_times_block<D>(acc1, s_p, s_g, warp, lane);       // dV = P^T dO
+        stage_rows<D>(s_k, acc1, 1.f, warp, gq, tq);             // dV into the K tile
+#pragma unroll
+        for (int i = 0; i < DT; ++i)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc1[i][e] = 0.f;
+        coef_t_times_block<D>(acc1, s_ds, s_q, warp, lane);      // dK = dS^T Q
+        __syncthreads();   // Q has been read by every warp
+        stage_rows<D>(s_q, acc1, scale, warp, gq, tq);           // dK into the Q tile
+        __syncthreads();
+        scatter_rows<D>(s_v, dq, s_tok, 0, r.n, sample_off, g.ts, head, tid);
+        scatter_rows<D>(s_k, dv, s_tok, 0, r.n, sample_off, g.ts, head, tid);
+        scatter_rows<D>(s_q, dk, s_tok, 0, r.n, sample_off, g.ts, head, tid);
+    }
+
+    __syncthreads();
+    // bin the image: cell (row, col) of a full-width window belongs to table row code(row) - code(col) + c0
+    const int n_full = g.nmax;
+    for (int cell = tid; cell < BM * n_full; cell += NTHREADS) {
+        const int row = cell / n_full, col = cell - row * n_full;
+        if (row >= n_full) continue;
+        const float val = s_acc[row * acc_stride + col];
+        if (val == 0.f) continue;
+        const int code_r = (row / g.w) * (2 * g.w - 1) + row % g.w;
+        const int code_c = (col / g.w) * (2 * g.w - 1) + col % g.w;
+        atomicAdd(&s_dbias[code_r - code_c + c0], val);
+    }
+    __syncthreads();
+    for (int i = tid; i < nbias; i += NTHREADS) {
+        float val = s_dbias[i];
+        if (val != 0.f) atomicAdd(&dbias[(size_t)i * g.heads + head], val);
+    }
+}
+
 // delta[b, token, head] = sum_c dO[b, token, head, c] * O[b, token, head, c]
 template <int D>
 __global__ void __launch_bounds__(256)
@@ -516,7 +763,42 @@ cudaError_t launch_one(const Geo& g, const void* q, const void* k, const void* v
                     : launch_one_sized<D, KV, false>(g, q, k, v, d_o, bias, lse, delta, out1, out2, dbias, sm_count, stream);
 }
 
+size_t bwd_small_smem_bytes(const Geo& g) {
+    const int nbias = (2 * g.w - 1) * (2 * g.w - 1);
+    const size_t head = (((size_t)BN * 16 + (size_t)nbias * 8 + 127) / 128) * 128;
+    const size_t tile = (size_t)BN * g.d * 2;
+    return head + 4 * tile + (tile > 16384 ? tile : 16384) + ((size_t)BM * (BN + 8) + (size_t)BM * kStageStride) * sizeof(float);
+}
+
 }  // namespace
+
+// windows of at most 64 tokens at head dim 128: the one-kernel backward
+bool TERRA_ELEM_FN(bwd_small_supported)(const Geo& g) { return g.d == 128 && g.nmax <= BN && g.w <= 32; }
+
+cudaError_t TERRA_ELEM_FN(launch_bwd_small)(const Geo& g, const void* q, const void* k, const void* v, const void* o, const void* d_o,
+                                            const float* bias, const float* lse, void* dq, void* dk, void* dv, float* dbias,
+                                            int sm_count, cudaStream_t stream) {
+    cudaError_t e = cudaMemsetAsync(dbias, 0, sizeof(float) * (size_t)(2 * g.w - 1) * (2 * g.w - 1) * g.heads, stream);
+    if (e != cudaSuccess) return e;
+    auto kern = swin_bwd_small_kernel<128>;
+    const size_t smem = bwd_small_smem_bytes(g);
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    int occ = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, NTHREADS, smem);
+    if (e != cudaSuccess) return e;
+    if (occ < 1) occ = 1;
+    const long long items = (long long)g.B * g.Mh * g.Mw;
+    long long cph = ((long long)sm_count * occ) / g.heads;
+    if (cph < 1) cph = 1;
+    if (cph > items) cph = items;
+    prof_begin("swin_bwd_small_kernel", stream);
+    kern<<<(unsigned)(cph * g.heads), NTHREADS, smem, stream>>>(
+        g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)o,
+        (const __nv_bfloat16*)d_o, bias, lse, (__nv_bfloat16*)dq, (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, dbias, (int)cph, BN + 8);
+    count_launch(stream);
+    return cudaGetLastError();
+}
 
 cudaError_t TERRA_ELEM_FN(launch_bwd_delta)(const Geo& g, const void* o, const void* d_o, float* delta, cudaStream_t stream) {
     const long long rows = (long long)g.B * g.H * g.W * g.heads;

@@ -21,6 +21,10 @@ cudaError_t launch_fwd_mma(const Geo& g, const void* q, const void* k, const voi
 // the register-tile kernels for fp16 activations and gradients (same arguments)
 cudaError_t launch_fwd_mma_f16(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
                                void* o, float* lse, cudaStream_t stream);
+bool bwd_small_supported_f16(const Geo& g);
+cudaError_t launch_bwd_small_f16(const Geo& g, const void* q, const void* k, const void* v, const void* o, const void* d_o,
+                                 const float* bias, const float* lse, void* dq, void* dk, void* dv, float* dbias,
+                                 int sm_count, cudaStream_t stream);
 cudaError_t launch_bwd_delta_f16(const Geo& g, const void* o, const void* d_o, float* delta, cudaStream_t stream);
 cudaError_t launch_bwd_mma_f16(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
                                const float* lse, const float* delta, const void* d_o,
@@ -75,6 +79,11 @@ cudaError_t launch_bwd_tc(const Geo& g, const void* q, const void* k, const void
 cudaError_t read_bwd_tc_status(int* timed_out);
 
 // delta[b, token, head] = sum_c dO * O   (fp32, same indexing as lse)
+// the whole backward in one kernel for windows of at most 64 tokens at head dim 128 (no delta kernel, no workspace)
+bool bwd_small_supported(const Geo& g);
+cudaError_t launch_bwd_small(const Geo& g, const void* q, const void* k, const void* v, const void* o, const void* d_o,
+                             const float* bias, const float* lse, void* dq, void* dk, void* dv, float* dbias,
+                             int sm_count, cudaStream_t stream);
 cudaError_t launch_bwd_delta(const Geo& g, const void* o, const void* d_o, float* delta, cudaStream_t stream);
 
 // dK, dV (key-tile CTAs) and dQ, dBias (query-tile CTAs)
