@@ -162,12 +162,15 @@ int terra_swin_attn_bwd_packed(const terra_swin_desc* desc, const void* qkv, con
  *
  * Arguments, layouts and error codes are those of terra_swin_attn_fwd.  Results: the same within the
  * library's tolerance; bit-equal to terra_swin_attn_fwd for head_dim 32 with window <= 16, where both run the
- * same tensor-core kernel.  For every other shape this entry point runs the register-tile forward kernel
- * (`swin_fwd_mma_kernel`, which needs no scratch) while terra_swin_attn_fwd may pick a faster chunked
- * tensor-core kernel that does need a workspace: equal within tolerance, not bit for bit, and slower.
+ * same kernel (the tensor-core kernel for windows of more than 64 tokens, the register-tile kernel for smaller
+ * ones), and for every shape whose windows hold at most 64 tokens.  For every other shape this entry point runs
+ * the register-tile forward kernel (`swin_fwd_mma_kernel`, which needs no scratch) while terra_swin_attn_fwd
+ * may pick a faster chunked tensor-core kernel that does need a workspace: equal within tolerance, not bit for
+ * bit, and slower.
  * Extra rules:
  *   - heads > TERRA_NOALLOC_MAX_HEADS is refused with TERRA_ERR_NOALLOC_LIMIT when the shape uses the
- *     scratch (head_dim 32, window <= 16); other shapes need no scratch and are not limited;
+ *     scratch (head_dim 32, window <= 16, windows of more than 64 tokens); other shapes need no scratch and are
+ *     not limited;
  *   - the first call on each device looks the array's device address up (the device must be current);
  *     make that first call before any stream capture begins;
  *   - all calls on a device share the one array and every call rewrites the part it uses, so nothing has to

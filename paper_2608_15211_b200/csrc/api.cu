@@ -110,16 +110,21 @@ static bool force_register_path() {
     return on;
 }
 
+// Windows of at most 64 tokens (the 8 x 8 windows of configs 1, 2 and of the paper's small and medium models) half
+// fill a 128-row tcgen05 tile and are bound by HBM and launch overheads: the register-tile forward and the one-kernel
+// register-tile backward are faster there at every head dim (config 2: 0.117 ms against 0.188 ms per step).
+static bool small_windows(const Geo& g) { return g.nmax <= 64; }
+
 // the tcgen05 kernels are written for bf16 operands; fp16 runs on the register-tile kernels
-static bool use_fwd_tc(const Geo& g) { return fwd_tc_supported(g) && !g.f16; }
+static bool use_fwd_tc(const Geo& g) { return fwd_tc_supported(g) && !g.f16 && !small_windows(g); }
 // head dim 128 with windows of fewer than 256 tokens (the 8 x 8 windows of the paper's small and medium models): a
 // 128-row tile would be mostly empty and the path is bound by HBM, the register-tile kernels are about twice as fast
-static bool small_window_128(const Geo& g) { return g.d == 128 && g.nmax < 256; }
+static bool small_window_128(const Geo& g) { return (g.d == 128 && g.nmax < 256) || small_windows(g); }
 static bool use_fwd_tc64(const Geo& g) { return fwd_tc64_supported(g) && !force_register_path() && !g.f16 && !small_window_128(g); }
 
 static size_t fwd_bytes(const Geo& g) {
     if (force_register_path() || g.f16) return 0;
-    if (fwd_tc_supported(g)) return align_up(fwd_tc_workspace_bytes(g), 256);
+    if (use_fwd_tc(g)) return align_up(fwd_tc_workspace_bytes(g), 256);
     if (use_fwd_tc64(g)) return align_up(fwd_tc64_workspace_bytes(g), 256);
     return 0;
 }
@@ -133,7 +138,7 @@ static bool force_split_small() {
     return on;
 }
 
-static bool use_bwd_tc(const Geo& g) { return bwd_tc_supported(g) && !force_register_path() && !g.f16; }
+static bool use_bwd_tc(const Geo& g) { return bwd_tc_supported(g) && !force_register_path() && !g.f16 && !small_windows(g); }
 
 static bool use_bwd_kv64(const Geo& g) { return bwd_kv64_supported(g) && !force_register_path() && !g.f16 && !small_window_128(g); }
 

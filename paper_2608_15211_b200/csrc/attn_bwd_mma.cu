@@ -463,7 +463,7 @@ __device__ __forceinline__ void coef_t_times_block(float (&out)[D / 8][4], const
     }
 }
 
-// The whole backward of windows of at most 64 tokens in one kernel (the paper's 8 x 8 windows): a CTA holds the
+// The whole backward of windows of at most 64 tokens in one kernel (the paper's 8 x 8 windows), any head dim: a CTA holds the
 // window's Q, K, V, dO and O rows of one head, so every tensor is read once and dQ, dK, dV are written once (the
 // split into a key side and a query side reads the inputs twice, and a third time for delta).
 //   delta = rowsum(dO * O)                                 (per query row, from the two tiles)
@@ -573,11 +573,19 @@ swin_bwd_small_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
         const float del_r[2] = {s_delta[row_tab[0]], s_delta[row_tab[1]]};
         float acc1[DT][4];
         {
-            static_assert(!kFragsInRegs<D>, "the own-row fragments are read from shared memory at each use");
-            uint32_t f0[1][4];
+            // fragments of the warp's own Q and dO rows (head dim 128: read from shared memory at each use instead)
+            uint32_t f1[kFragsInRegs<D> ? KS : 1][4], f2[kFragsInRegs<D> ? KS : 1][4];
+            if constexpr (kFragsInRegs<D>) {
+#pragma unroll
+                for (int ks = 0; ks < KS; ++ks) {
+                    const int row = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+                    ldmatrix_x4(f1[ks], smem_u32(s_q + tile_off<D>(row, 2 * ks + (lane >> 4))));
+                    ldmatrix_x4(f2[ks], smem_u32(s_g + tile_off<D>(row, 2 * ks + (lane >> 4))));
+                }
+            }
             float acc_s[BN / 8][4], acc_dp[BN / 8][4];
-            rows_times_block_t<D>(acc_s, f0, s_q, s_k, warp, lane);
-            rows_times_block_t<D>(acc_dp, f0, s_g, s_v, warp, lane);
+            rows_times_block_t<D>(acc_s, f1, s_q, s_k, warp, lane);
+            rows_times_block_t<D>(acc_dp, f2, s_g, s_v, warp, lane);
 #pragma unroll
             for (int nt = 0; nt < BN / 8; ++nt) {
 #pragma unroll
@@ -772,15 +780,15 @@ size_t bwd_small_smem_bytes(const Geo& g) {
 
 }  // namespace
 
-// windows of at most 64 tokens at head dim 128: the one-kernel backward
-bool TERRA_ELEM_FN(bwd_small_supported)(const Geo& g) { return g.d == 128 && g.nmax <= BN && g.w <= 32; }
+// windows of at most 64 tokens: the one-kernel backward
+bool TERRA_ELEM_FN(bwd_small_supported)(const Geo& g) { return g.nmax <= BN && g.w <= 32; }
 
 cudaError_t TERRA_ELEM_FN(launch_bwd_small)(const Geo& g, const void* q, const void* k, const void* v, const void* o, const void* d_o,
                                             const float* bias, const float* lse, void* dq, void* dk, void* dv, float* dbias,
                                             int sm_count, cudaStream_t stream) {
     cudaError_t e = cudaMemsetAsync(dbias, 0, sizeof(float) * (size_t)(2 * g.w - 1) * (2 * g.w - 1) * g.heads, stream);
     if (e != cudaSuccess) return e;
-    auto kern = swin_bwd_small_kernel<128>;
+    auto kern = g.d == 32 ? swin_bwd_small_kernel<32> : g.d == 64 ? swin_bwd_small_kernel<64> : swin_bwd_small_kernel<128>;
     const size_t smem = bwd_small_smem_bytes(g);
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;

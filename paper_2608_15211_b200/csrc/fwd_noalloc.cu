@@ -62,7 +62,7 @@ extern "C" int terra_swin_attn_fwd_noalloc(const terra_swin_desc* desc, const vo
     cudaError_t e;
     if (g.f16) {
         e = launch_fwd_mma_f16(g, q, k, v, bias_table, o, lse, (cudaStream_t)stream);   // fp16: register-tile kernel, no scratch
-    } else if (fwd_tc_supported(g)) {
+    } else if (fwd_tc_supported(g) && g.nmax > 64) {        // (windows of at most 64 tokens: the register-tile kernel, as in the regular forward)
         // the one shape-dependent limit of this entry point: the fixed scratch holds this many heads
         if (g.heads > kNoAllocMaxHeads) return TERRA_ERR_NOALLOC_LIMIT;
         float* scratch = nullptr;

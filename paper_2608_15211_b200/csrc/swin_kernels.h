@@ -79,7 +79,7 @@ cudaError_t launch_bwd_tc(const Geo& g, const void* q, const void* k, const void
 cudaError_t read_bwd_tc_status(int* timed_out);
 
 // delta[b, token, head] = sum_c dO * O   (fp32, same indexing as lse)
-// the whole backward in one kernel for windows of at most 64 tokens at head dim 128 (no delta kernel, no workspace)
+// the whole backward in one kernel for windows of at most 64 tokens (no delta kernel, no workspace)
 bool bwd_small_supported(const Geo& g);
 cudaError_t launch_bwd_small(const Geo& g, const void* q, const void* k, const void* v, const void* o, const void* d_o,
                              const float* bias, const float* lse, void* dq, void* dk, void* dv, float* dbias,

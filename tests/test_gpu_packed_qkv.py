@@ -47,8 +47,8 @@ def test_packed_calls_match_the_oracle_and_the_unpacked_calls(cfg):
                            ("dv", gpu_rows(dqkv[:, :, :, 2].contiguous(), cfg, tok), rv),
                            ("dbias", dbias.cpu().double().numpy(), rb)):
         gate(name, got, ref, strict=False)
-    if cfg.head_dim == 32 and cfg.window <= 16:
-        assert torch.equal(dbias, dbias2)            # fixed summation order on this path
+    if cfg.head_dim == 32 and 8 < cfg.window <= 16:
+        assert torch.equal(dbias, dbias2)            # fixed summation order on the tcgen05 path (windows of more than 64 tokens)
 
 
 def test_packed_full_size_config3_runs_at_the_same_speed():

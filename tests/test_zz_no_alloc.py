@@ -68,7 +68,7 @@ def test_noalloc_forward_on_a_shape_without_scratch_and_its_limit():
     (o, lse), (o_ref, lse_ref) = _both_paths(cfg, 3)
     gate("o", o.float().cpu().numpy(), o_ref.float().cpu().numpy())
     gate("lse", lse.cpu().numpy(), lse_ref.cpu().numpy())
-    big = small_config("na4", 1, 8, 8, 65, 32, 4, 2, 2)               # one head more than the fixed scratch holds
+    big = small_config("na4", 1, 16, 16, 65, 32, 16, 8, 8)            # one head more than the fixed scratch holds
     x = {k: v.cuda() for k, v in make_inputs(big).items()}
     d = terra.make_desc(big)
     o = torch.empty_like(x["q"])
