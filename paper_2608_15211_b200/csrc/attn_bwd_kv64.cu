@@ -1,19 +1,23 @@
-// Key side of the backward pass (dK, dV) on the tcgen05 tensor cores for head dim 64 and windows of up to 1024
-// tokens (window side <= 32).  The query side (dQ, dBias) of this regime runs the register-tile kernel.
+// Key side of the backward pass (dK, dV) on the tcgen05 tensor cores for head dims 64 and 128 and windows of up to
+// 1024 tokens (window side <= 32).  The query side (dQ, dBias) of this regime runs its own tcgen05 kernel on grids of
+// complete 32 x 32 windows and the register-tile kernel otherwise.
 //
 // One persistent CTA per SM, bound to one head, walks over (batch, window, 128-key tile) items.  The tile's K and V
 // rows stay in shared memory; the window's queries stream through a ring of slots in chunks of 128 (Q, dO rows and
 // per-query lse, delta, bias code, mask label).  Orientation as in the small-window backward kernel: TMEM lanes =
-// keys, columns = queries.  Per chunk:
-//   S^T = K Q_c^T, dP^T = V dO_c^T                                   (SS MMAs, N = the chunk's queries)
+// keys, columns = queries.  Per half chunk of 64 queries:
+//   S^T = K Q_c^T, dP^T = V dO_c^T                                   (SS MMAs, N = the half chunk's queries)
 //   P^T = exp2(S^T scale + bias - lse_q), dS^T = P^T (dP^T - delta_q)   (elementwise warps, one key row per thread,
 //                                                                      written back over S^T / dP^T as bf16)
 //   dV += P^T dO_c, dK += dS^T Q_c                                   (A from TMEM, B = the chunk's rows, MN-major)
 // P is recomputed from the saved log-sum-exp, so the chunks are independent.
 // Roles: warps 0-7 elementwise (warps w and w + 4 share TMEM lane quarter w & 3 and take the chunk's first / second
-// 64 query columns), warp 8 issues every MMA, warps 9-11 gather rows with cp.async.  Head dim 64 is kept as two
-// 32-column halves in the 64-byte-swizzled operand layout (lo | hi regions), as in the forward kernel of this regime.
-// TMEM columns: S^T 0..127, dP^T 128..255, dV 256..319, dK 320..383.
+// 64 query columns), warp 8 issues every MMA, warps 9-11 load rows (bulk copies from warp 9 on grids of complete
+// windows, else cp.async gathers from all three).  A row is kept as head dim / 32 parts of 32 columns in the
+// 64-byte-swizzled operand layout, as in the forward kernel of this regime.
+// Half chunks rotate through TMEM buffers (S^T 64 columns | dP^T 64 columns): three at head dim 64, so that the scores of
+// a group's next half chunk are issued while it still works on the current one, two at head dim 128, where the
+// accumulators dV and dK (head dim columns each, behind the buffers) take the rest of the 512 columns.
 // Every mbarrier wait is bounded; on expiry the CTA raises an abort flag, all roles leave their loops, TMEM is
 // released and the host reads the device status word.  Every role follows every ring item by item.
 #include "swin_common.cuh"
@@ -44,7 +48,7 @@ constexpr int kPartBytes = 64;                        // one 32-column part of a
 constexpr int kTile = 128;                            // keys per item, queries per chunk
 constexpr int kPart = kTile * kPartBytes;             // 8192: the region of one 32-column part of 128 rows
 constexpr int kBiasFloats = 6048;
-constexpr int kColS = 0, kColDP = 128, kColDV = 256;  // dK follows dV
+constexpr int kBufCols = 128;                         // TMEM buffer b: S^T of a half chunk at 128 b, dP^T at 128 b + 64
 
 // Shared-memory plan per head dim D (64 or 128): a row is kept as D / 32 parts of 32 columns, each part a region in
 // the 64-byte-swizzled operand layout.  Head dim 64: two key stages, three query slots; head dim 128: one and two.
@@ -65,7 +69,10 @@ struct Lay {
     static constexpr int kOffBias = kOffSlots + kSlots * kSlotBytes;
     static constexpr int kOffBars = ((kOffBias + kBiasFloats * 4 + 1023) / 1024) * 1024;
     static constexpr int kSmemBytes = kOffBars + 1024;
-    static constexpr int kColDK = kColDV + D;
+    // Half chunks (64 queries) rotate through kBufs TMEM buffers; with three (head dim 64) the scores of a group's next
+    // half chunk are issued while it still works on the current one.  At head dim 128 the accumulators leave room for two.
+    static constexpr int kBufs = D == 64 ? 3 : 2;
+    static constexpr int kColDV = kBufs * kBufCols, kColDK = kColDV + D;
     static_assert(kKvStageBytes % 1024 == 0 && kSlotBytes % 1024 == 0, "tiles keep the swizzle alignment");
     static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
     static_assert(kColDK + D <= 512, "tensor memory columns");
@@ -215,7 +222,8 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
     constexpr int kOffK = L::kOffK, kOffV = L::kOffV, kOffKCode = L::kOffKCode, kOffKLab = L::kOffKLab, kOffKTok = L::kOffKTok;
     constexpr int kKvStageBytes = L::kKvStageBytes, kOffQ = L::kOffQ, kOffG = L::kOffG, kOffQCode = L::kOffQCode;
     constexpr int kOffQLab = L::kOffQLab, kOffQLse = L::kOffQLse, kOffQDelta = L::kOffQDelta, kSlotBytes = L::kSlotBytes;
-    constexpr int kOffSlots = L::kOffSlots, kOffBias = L::kOffBias, kOffBars = L::kOffBars, kColDK = L::kColDK;
+    constexpr int kOffSlots = L::kOffSlots, kOffBias = L::kOffBias, kOffBars = L::kOffBars, kColDV = L::kColDV, kColDK = L::kColDK;
+    constexpr int kBufs = L::kBufs;
     extern __shared__ __align__(1024) unsigned char smem[];
     const uint32_t smem0 = smem_u32(smem);
     const uint32_t bar0 = smem0 + kOffBars;
@@ -223,13 +231,14 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
     auto bar_kvempty = [&](int s) { return bar0 + 8u * (2 + s); };       // ... and no longer needed
     auto bar_qfull = [&](int s) { return bar0 + 8u * (4 + s); };         // a query chunk is in ring slot s
     auto bar_qempty = [&](int s) { return bar0 + 8u * (7 + s); };        // ... and every MMA that reads it is complete
-    // a chunk's two 64-query halves are separate buffers (columns 64 h of S^T and dP^T) with their own hand-overs:
-    // half h belongs to elementwise warps 4 h .. 4 h + 3, and the MMAs of one half run while the other is worked on
-    auto bar_sdp = [&](int h) { return bar0 + 8u * (10 + h); };          // S^T and dP^T of a half chunk are in TMEM
-    auto bar_ds = [&](int h) { return bar0 + 8u * (12 + h); };           // bf16 P^T and dS^T of the half chunk are in TMEM
-    const uint32_t bar_acc = bar0 + 8u * 14;                              // dV, dK of the item are final
-    const uint32_t bar_accfree = bar0 + 8u * 15;                          // ... and have been read
-    unsigned char* tail = smem + kOffBars + 8 * 16;
+    // A chunk's 64-query halves are separate units of work, numbered through the whole run (only halves that exist
+    // count); half number p belongs to elementwise warps 4 h .. 4 h + 3 (h = which half of its chunk) and lives in TMEM
+    // buffer p % kBufs, with the buffer's own hand-overs.
+    auto bar_sdp = [&](int b) { return bar0 + 8u * (10 + b); };          // S^T and dP^T of a half chunk are in TMEM buffer b
+    auto bar_ds = [&](int b) { return bar0 + 8u * (13 + b); };           // bf16 P^T and dS^T of the half chunk are in buffer b
+    const uint32_t bar_acc = bar0 + 8u * 16;                              // dV, dK of the item are final
+    const uint32_t bar_accfree = bar0 + 8u * 17;                          // ... and have been read
+    unsigned char* tail = smem + kOffBars + 8 * 18;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail);
     volatile int* cta_abort = reinterpret_cast<volatile int*>(tail + 8);
 
@@ -247,9 +256,9 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             mbar_init(bar_qfull(s), TMA ? 32 : kLoaderThreads);
             mbar_init(bar_qempty(s), 1);
         }
-        for (int h = 0; h < 2; ++h) {
-            mbar_init(bar_sdp(h), 1);
-            mbar_init(bar_ds(h), kWorkThreads / 2);
+        for (int b = 0; b < kBufs; ++b) {
+            mbar_init(bar_sdp(b), 1);
+            mbar_init(bar_ds(b), kWorkThreads / 2);
         }
         mbar_init(bar_acc, 1);
         mbar_init(bar_accfree, kWorkThreads);
@@ -466,7 +475,7 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
         const uint32_t idesc_acc = make_idesc_bf16(128, D, 0, 1);        // A from TMEM, B = 16 rows x D (MN-major)
         const uint32_t sd_hi = sdesc_hi(make_sdesc_sw64(smem0, 512));    // common high word of the K-major descriptors
         int kuse = 0;
-        int n_ds[2] = {0, 0};
+        unsigned p0 = 0;                                  // half chunks before the current item
         long long ru = 0;
         bool ok = true;
         ItemCursor cur = cursor_init(cta_in_head, ctas_per_head, max_tiles, g.Mw, g.Mh);
@@ -488,11 +497,11 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             // S^T = K Q^T, dP^T = V dO^T for the 64 queries of half h of the chunk in ring slot `sb`
             // (descriptor low words = start address in 16-byte units: + 2 per 32-byte K step, + kPart / 16 per 32-column part)
             const uint32_t k_lo = sdesc_lo(make_sdesc_sw64(kb + kOffK, 512)), v_lo = sdesc_lo(make_sdesc_sw64(kb + kOffV, 512));
-            auto issue_sdp = [&](int h, uint32_t sb, int nc) {
+            auto issue_sdp = [&](int h, uint32_t sb, int nc, int buf) {
                 const uint32_t idesc = make_idesc_bf16(128, nc, 0, 0);
                 const uint32_t q_lo = sdesc_lo(make_sdesc_sw64(sb + kOffQ + h * 64 * kPartBytes, 512));
                 const uint32_t g_lo = sdesc_lo(make_sdesc_sw64(sb + kOffG + h * 64 * kPartBytes, 512));
-                const uint32_t t_s = tmem_base + kColS + 64 * h, t_dp = tmem_base + kColDP + 64 * h;
+                const uint32_t t_s = tmem_base + kBufCols * buf, t_dp = t_s + 64;
                 constexpr uint32_t kNext = kPart >> 4;
                 tc_fence_after();
                 if (elect_one()) {
@@ -510,64 +519,77 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                         mma_ss_h<true>(t_dp, v_lo + pt * kNext, g_lo + pt * kNext, sd_hi, idesc);
                         mma_ss_h<true>(t_dp, v_lo + pt * kNext + 2, g_lo + pt * kNext + 2, sd_hi, idesc);
                     }
-                    mma_commit(bar_sdp(h));
+                    mma_commit(bar_sdp(buf));
                 }
                 __syncwarp();
             };
-            ok = chunk_ready(ru);
-            if (!ok) break;
-            for (int h = 0; h < 2; ++h)
-                if (half_cols(0, h) > 0) issue_sdp(h, smem0 + kOffSlots + (int)(ru % kSlots) * kSlotBytes, half_cols(0, h));
-            for (int c = 0; c < x.nch && ok; ++c, ++ru) {
-                const int s = (int)(ru % kSlots);
+            // the item's half chunks in order: half i is half i % 2 of chunk i / 2 (only the last chunk can lack its second half)
+            const int nh = 2 * x.nch - (half_cols(x.nch - 1, 1) > 0 ? 0 : 1);
+            int ready_chunks = 0;                         // chunks of the item known to be in their ring slots
+            // the chunk of half i is in its ring slot
+            auto ensure_chunk = [&](int i) -> bool {
+                while (ready_chunks <= (i >> 1)) {
+                    if (!chunk_ready(ru + ready_chunks)) return false;
+                    ++ready_chunks;
+                }
+                return true;
+            };
+            // scores of half i into its buffer
+            auto issue_half = [&](int i) {
+                const int c = i >> 1, h = i & 1;
+                issue_sdp(h, smem0 + kOffSlots + (int)((ru + c) % kSlots) * kSlotBytes, half_cols(c, h), (int)((p0 + i) % kBufs));
+            };
+            for (int i = 0; i < kBufs && i < nh && ok; ++i) {
+                ok = ensure_chunk(i);
+                if (ok) issue_half(i);
+            }
+            for (int i = 0; i < nh && ok; ++i) {
+                const int c = i >> 1, h = i & 1;
+                const unsigned p = p0 + i;
+                const int buf = (int)(p % kBufs);
+                const int s = (int)((ru + c) % kSlots);
                 const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes;
-                const bool has_next = c + 1 < x.nch;
-                if (has_next) {
-                    ok = chunk_ready(ru + 1);
-                    if (!ok) break;
-                }
-                const uint32_t sb_n = smem0 + kOffSlots + (int)((ru + 1) % kSlots) * kSlotBytes;
-                for (int h = 0; h < 2 && ok; ++h) {
-                    const int nc = half_cols(c, h);
-                    if (nc == 0) continue;
-                    ok = mbar_wait_all(bar_ds(h), n_ds[h] & 1, cta_abort);
-                    ++n_ds[h];
-                    if (ok && c == 0 && h == 0 && kuse > 0) ok = mbar_wait_all(bar_accfree, (kuse - 1) & 1, cta_abort);
-                    if (!ok) break;
-                    tc_fence_after();
-                    // dV += P^T dO, dK += dS^T Q over the half chunk's query columns
-                    const uint64_t gd = make_sdesc_sw64_mn(sb + kOffG + h * 64 * kPartBytes, kPart, 512);
-                    const uint64_t qd = make_sdesc_sw64_mn(sb + kOffQ + h * 64 * kPartBytes, kPart, 512);
-                    const uint32_t g_lo = sdesc_lo(gd), q_lo = sdesc_lo(qd), d_hi = sdesc_hi(gd);
-                    const uint32_t t_p = tmem_base + kColS + 64 * h, t_ds = tmem_base + kColDP + 64 * h;
-                    const int nks = nc >> 4;
-                    if (elect_one()) {
-                        int j = 0;
-                        if (c == 0 && h == 0) {
-                            mma_ts_h<false>(tmem_base + kColDV, t_p, g_lo, d_hi, idesc_acc);
-                            mma_ts_h<false>(tmem_base + kColDK, t_ds, q_lo, d_hi, idesc_acc);
-                            j = 1;
-                        }
-                        for (; j < nks; ++j) {
-                            mma_ts_h<true>(tmem_base + kColDV, t_p + 16 * j, g_lo + 64 * j, d_hi, idesc_acc);
-                            mma_ts_h<true>(tmem_base + kColDK, t_ds + 16 * j, q_lo + 64 * j, d_hi, idesc_acc);
-                        }
-                    }
-                    __syncwarp();
-                    // the half's buffers are free again (the products that read them were issued just above): the
-                    // next chunk's scores for this half follow at once, while the other half is being worked on
-                    if (has_next && half_cols(c + 1, h) > 0) issue_sdp(h, sb_n, half_cols(c + 1, h));
-                }
+                const int nc = half_cols(c, h);
+                ok = mbar_wait_all(bar_ds(buf), (p / kBufs) & 1, cta_abort);
+                if (ok && i == 0 && kuse > 0) ok = mbar_wait_all(bar_accfree, (kuse - 1) & 1, cta_abort);
                 if (!ok) break;
+                tc_fence_after();
+                // dV += P^T dO, dK += dS^T Q over the half chunk's query columns
+                const uint64_t gd = make_sdesc_sw64_mn(sb + kOffG + h * 64 * kPartBytes, kPart, 512);
+                const uint64_t qd = make_sdesc_sw64_mn(sb + kOffQ + h * 64 * kPartBytes, kPart, 512);
+                const uint32_t g_lo = sdesc_lo(gd), q_lo = sdesc_lo(qd), d_hi = sdesc_hi(gd);
+                const uint32_t t_p = tmem_base + kBufCols * buf, t_ds = t_p + 64;
+                const int nks = nc >> 4;
+                const bool chunk_done = h == 1 || half_cols(c, 1) == 0;      // the chunk's last half
                 if (elect_one()) {
-                    mma_commit(bar_qempty(s));
-                    if (!has_next) {
+                    int j = 0;
+                    if (i == 0) {
+                        mma_ts_h<false>(tmem_base + kColDV, t_p, g_lo, d_hi, idesc_acc);
+                        mma_ts_h<false>(tmem_base + kColDK, t_ds, q_lo, d_hi, idesc_acc);
+                        j = 1;
+                    }
+                    for (; j < nks; ++j) {
+                        mma_ts_h<true>(tmem_base + kColDV, t_p + 16 * j, g_lo + 64 * j, d_hi, idesc_acc);
+                        mma_ts_h<true>(tmem_base + kColDK, t_ds + 16 * j, q_lo + 64 * j, d_hi, idesc_acc);
+                    }
+                    if (chunk_done) mma_commit(bar_qempty(s));       // the slot's last readers were issued just above
+                    if (i + 1 == nh) {
                         mma_commit(bar_acc);
                         mma_commit(bar_kvempty(ks));
                     }
                 }
                 __syncwarp();
+                // the buffer is free again (the products that read it were issued just above): the scores of the half
+                // chunk kBufs further on follow at once
+                // (its chunk is waited for only now: where the rows are late, the current half should not wait for them)
+                if (i + kBufs < nh) {
+                    ok = ensure_chunk(i + kBufs);
+                    if (ok) issue_half(i + kBufs);
+                }
             }
+            if (!ok) break;
+            ru += x.nch;
+            p0 += (unsigned)nh;
             ++kuse;
         }
     }
@@ -580,7 +602,8 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
         const uint32_t lane_addr = ((uint32_t)(32 * quarter)) << 16;
         const float scale = g.scale_log2e;
         const float out_scale = g.scale_log2e * kLn2;     // dK carries the score scale
-        int kuse = 0, n_half = 0;                       // items; half chunks this group has worked on
+        int kuse = 0;
+        unsigned p0 = 0;                                  // half chunks before the current item
         long long ru = 0;
         bool ok = true;
         ItemCursor cur = cursor_init(cta_in_head, ctas_per_head, max_tiles, g.Mw, g.Mh);
@@ -602,11 +625,13 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                 const uint32_t sl_a = smem0 + kOffSlots + s * kSlotBytes + kOffQCode;      // the slot's per-query tables
                 const int ncols = min(kTile, x.npad - c * kTile);
                 if (ncols <= 64 * hcol) continue;          // this group's half of the chunk does not exist
-                ok = mbar_wait_all(bar_sdp(hcol), n_half & 1, cta_abort);
+                const unsigned p = p0 + 2 * c + hcol;      // the half chunk's number; its buffer holds S^T at column 0, dP^T at 64
+                const int buf = (int)(p % kBufs);
+                ok = mbar_wait_all(bar_sdp(buf), (p / kBufs) & 1, cta_abort);
                 if (!ok) break;
-                ++n_half;
                 tc_fence_after();
-                const uint32_t t_s = tmem_base + lane_addr + kColS, t_dp = tmem_base + lane_addr + kColDP;
+                // (addressed by the chunk's column number: the group's columns start at 64 hcol)
+                const uint32_t t_s = tmem_base + lane_addr + kBufCols * buf - 64 * hcol, t_dp = t_s + 64;
                 const int col_end = min(ncols, 64 * hcol + 64);
                 // 4 * bias code of query column `col` of this chunk in a 32-wide window: slot = 128 c + col = 32 a + b
                 auto code4_of = [&](int col) { return 4 * ((4 * c + (col >> 5)) * cs + (col & 31)); };
@@ -642,9 +667,10 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                 }
                 tmem_st_wait();
                 tc_fence_before();
-                mbar_arrive(bar_ds(hcol));
+                mbar_arrive(bar_ds(buf));
             }
             if (!ok) break;
+            p0 += (unsigned)(2 * x.nch - (min(kTile, x.npad - (x.nch - 1) * kTile) > 64 ? 0 : 1));
             // ---- read-out: dV rows by warps 0-3, dK rows by warps 4-7
             if (!mbar_wait_all(bar_acc, kuse & 1, cta_abort)) break;
             tc_fence_after();
