@@ -305,3 +305,28 @@ def test_side_stream_and_interleaved_shapes_give_the_same_bits():
                 assert torch.allclose(a, b, rtol=1e-4, atol=1e-5 * float(b.abs().max()))
             else:
                 assert torch.equal(a, b), (n, nm)
+
+
+LATE_MAXIMA = [
+    # name,     B, H,  W,  heads, d,  w,  sh, sw, ph, pw
+    ("late128", 1, 64, 64, 1, 128, 32, 0, 0, 0, 1),
+    ("late64", 1, 64, 96, 2, 64, 32, 16, 8, 0, 1),
+    ("late64_ragged", 1, 70, 80, 2, 64, 32, 16, 16, 0, 0),
+    ("late128_w16", 1, 32, 48, 2, 128, 16, 8, 8, 0, 1),
+]
+
+
+@pytest.mark.parametrize("case", LATE_MAXIMA, ids=[c[0] for c in LATE_MAXIMA])
+def test_forward_when_the_keys_streamed_last_dominate(case):
+    """The large-window forward streams the keys once and keeps a running reference for the row maximum: here the keys
+    in the lower half of every window are 24 times larger, so the chunks streamed last raise the row maxima by many
+    octaves and the accumulated output has to be scaled down on the way (log-sum-exp up to 150 nats)."""
+    cfg = small_config(*case)
+    x = make_inputs(cfg)
+    rows = torch.arange(cfg.H).view(1, cfg.H, 1, 1, 1)
+    k = x["k"].float()
+    x["k"] = torch.where(((rows - cfg.shift_h) % cfg.window) >= cfg.window // 2, k * 24.0, k).to(torch.bfloat16)
+    x["bias"] = x["bias"] * 25.0
+    xg = _to_gpu(x)
+    d, o, lse = _run_fwd(cfg, xg)
+    _check_forward(cfg, x, o, lse, None)
