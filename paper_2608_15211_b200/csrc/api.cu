@@ -115,15 +115,15 @@ static bool force_register_path() {
 // register-tile backward are faster there at every head dim (config 2: 0.117 ms against 0.188 ms per step).
 static bool small_windows(const Geo& g) { return g.nmax <= 64; }
 
-// the tcgen05 kernels are written for bf16 operands; fp16 runs on the register-tile kernels
-static bool use_fwd_tc(const Geo& g) { return fwd_tc_supported(g) && !g.f16 && !small_windows(g); }
+// (every kernel exists for bf16 and for fp16 activations: `f16` only selects the build of the kernel)
+static bool use_fwd_tc(const Geo& g) { return fwd_tc_supported(g) && !small_windows(g); }
 // head dim 128 with windows of fewer than 256 tokens (the 8 x 8 windows of the paper's small and medium models): a
 // 128-row tile would be mostly empty and the path is bound by HBM, the register-tile kernels are about twice as fast
 static bool small_window_128(const Geo& g) { return (g.d == 128 && g.nmax < 256) || small_windows(g); }
-static bool use_fwd_tc64(const Geo& g) { return fwd_tc64_supported(g) && !force_register_path() && !g.f16 && !small_window_128(g); }
+static bool use_fwd_tc64(const Geo& g) { return fwd_tc64_supported(g) && !force_register_path() && !small_window_128(g); }
 
 static size_t fwd_bytes(const Geo& g) {
-    if (force_register_path() || g.f16) return 0;
+    if (force_register_path()) return 0;
     if (use_fwd_tc(g)) return align_up(fwd_tc_workspace_bytes(g), 256);
     if (use_fwd_tc64(g)) return align_up(fwd_tc64_workspace_bytes(g), 256);
     return 0;
@@ -138,9 +138,9 @@ static bool force_split_small() {
     return on;
 }
 
-static bool use_bwd_tc(const Geo& g) { return bwd_tc_supported(g) && !force_register_path() && !g.f16 && !small_windows(g); }
+static bool use_bwd_tc(const Geo& g) { return bwd_tc_supported(g) && !force_register_path() && !small_windows(g); }
 
-static bool use_bwd_kv64(const Geo& g) { return bwd_kv64_supported(g) && !force_register_path() && !g.f16 && !small_window_128(g); }
+static bool use_bwd_kv64(const Geo& g) { return bwd_kv64_supported(g) && !force_register_path() && !small_window_128(g); }
 
 static size_t delta_bytes(const Geo& g) {
     if (use_bwd_tc(g)) return align_up(bwd_tc_workspace_bytes(g), 256);
@@ -205,14 +205,15 @@ static int fwd_call(const Geo& g, const void* q, const void* k, const void* v,
     rc = device_props(&sms);
     if (rc) return rc;
     cudaError_t e;
-    if (g.f16)
-        e = launch_fwd_mma_f16(g, q, k, v, bias_table, o, lse, (cudaStream_t)stream);
-    else if (need > 0 && use_fwd_tc64(g) && !use_fwd_tc(g))
-        e = launch_fwd_tc64(g, q, k, v, bias_table, o, lse, workspace, sms, (cudaStream_t)stream);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (need > 0 && use_fwd_tc64(g) && !use_fwd_tc(g))
+        e = g.f16 ? launch_fwd_tc64_f16(g, q, k, v, bias_table, o, lse, workspace, sms, st)
+                  : launch_fwd_tc64(g, q, k, v, bias_table, o, lse, workspace, sms, st);
     else if (need > 0)
-        e = launch_fwd_tc(g, q, k, v, bias_table, o, lse, workspace, sms, (cudaStream_t)stream);
+        e = g.f16 ? launch_fwd_tc_f16(g, q, k, v, bias_table, o, lse, workspace, sms, st)
+                  : launch_fwd_tc(g, q, k, v, bias_table, o, lse, workspace, sms, st);
     else
-        e = launch_fwd_mma(g, q, k, v, bias_table, o, lse, (cudaStream_t)stream);
+        e = g.f16 ? launch_fwd_mma_f16(g, q, k, v, bias_table, o, lse, st) : launch_fwd_mma(g, q, k, v, bias_table, o, lse, st);
     return e == cudaSuccess ? TERRA_OK : cuda_fail(e, "terra_swin_attn_fwd");
 }
 
@@ -255,7 +256,8 @@ static int bwd_call(const Geo& g, const void* q, const void* k, const void* v,
     if (rc) return rc;
     cudaStream_t st = (cudaStream_t)stream;
     if (use_bwd_tc(g)) {
-        cudaError_t et = launch_bwd_tc(g, q, k, v, bias_table, o, lse, d_o, dq, dk, dv, dbias, workspace, sms, st);
+        cudaError_t et = g.f16 ? launch_bwd_tc_f16(g, q, k, v, bias_table, o, lse, d_o, dq, dk, dv, dbias, workspace, sms, st)
+                               : launch_bwd_tc(g, q, k, v, bias_table, o, lse, d_o, dq, dk, dv, dbias, workspace, sms, st);
         return et == cudaSuccess ? TERRA_OK : cuda_fail(et, "terra_swin_attn_bwd");
     }
     if (bwd_small_supported(g) && !force_split_small()) {
@@ -265,27 +267,32 @@ static int bwd_call(const Geo& g, const void* q, const void* k, const void* v,
         return es == cudaSuccess ? TERRA_OK : cuda_fail(es, "terra_swin_attn_bwd");
     }
     float* delta = reinterpret_cast<float*>(workspace);
-    if (g.f16) {
-        cudaError_t ef = launch_bwd_delta_f16(g, o, d_o, delta, st);
-        if (ef == cudaSuccess) ef = launch_bwd_mma_f16(g, q, k, v, bias_table, lse, delta, d_o, dq, dk, dv, dbias, sms, st);
-        return ef == cudaSuccess ? TERRA_OK : cuda_fail(ef, "terra_swin_attn_bwd");
-    }
-    cudaError_t e = launch_bwd_delta(g, o, d_o, delta, st);
+    cudaError_t e = g.f16 ? launch_bwd_delta_f16(g, o, d_o, delta, st) : launch_bwd_delta(g, o, d_o, delta, st);
     if (e != cudaSuccess) return cuda_fail(e, "terra_swin_attn_bwd (delta)");
+    // the register-tile backward, both sides or the query side only
+    auto bwd_mma = [&](bool query_side_only) {
+        return g.f16 ? launch_bwd_mma_f16(g, q, k, v, bias_table, lse, delta, d_o, dq, dk, dv, dbias, sms, st, query_side_only)
+                     : launch_bwd_mma(g, q, k, v, bias_table, lse, delta, d_o, dq, dk, dv, dbias, sms, st, query_side_only);
+    };
     if (use_bwd_kv64(g)) {
         // key side (dK, dV) on tcgen05
         float* prep = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(workspace) +
                                                align_up(sizeof(float) * (size_t)g.B * g.H * g.W * g.heads, 256));
         e = launch_bias_prep64(g, bias_table, prep, st);
-        if (e == cudaSuccess) e = launch_bwd_kv64(g, q, k, v, d_o, prep, lse, delta, dk, dv, sms, st);
+        if (e == cudaSuccess)
+            e = g.f16 ? launch_bwd_kv64_f16(g, q, k, v, d_o, prep, lse, delta, dk, dv, sms, st)
+                      : launch_bwd_kv64(g, q, k, v, d_o, prep, lse, delta, dk, dv, sms, st);
         if (e == cudaSuccess) {
             // query side (dQ, dBias): tcgen05 for complete 32 x 32 windows, else the register-tile kernel
-            if (bwd_q64_supported(g)) e = launch_bwd_q64(g, q, k, v, d_o, prep, lse, delta, dq, dbias, sms, st);
-            else e = launch_bwd_mma(g, q, k, v, bias_table, lse, delta, d_o, dq, dk, dv, dbias, sms, st, true);
+            if (bwd_q64_supported(g))
+                e = g.f16 ? launch_bwd_q64_f16(g, q, k, v, d_o, prep, lse, delta, dq, dbias, sms, st)
+                          : launch_bwd_q64(g, q, k, v, d_o, prep, lse, delta, dq, dbias, sms, st);
+            else
+                e = bwd_mma(true);
         }
         return e == cudaSuccess ? TERRA_OK : cuda_fail(e, "terra_swin_attn_bwd");
     }
-    e = launch_bwd_mma(g, q, k, v, bias_table, lse, delta, d_o, dq, dk, dv, dbias, sms, st);
+    e = bwd_mma(false);
     return e == cudaSuccess ? TERRA_OK : cuda_fail(e, "terra_swin_attn_bwd");
 }
 
@@ -339,7 +346,16 @@ int terra_swin_check(void* stream) {
     int timed_out_q = 0;
     e = read_bwd_q64_status(&timed_out_q);
     if (e != cudaSuccess) return cuda_fail(e, "terra_swin_check");
-    return (timed_out || timed_out_bwd || timed_out_64 || timed_out_kv || timed_out_q) ? TERRA_ERR_DEVICE_TIMEOUT : TERRA_OK;
+    // the fp16 builds of the same kernels keep status words of their own
+    int t16[5] = {0, 0, 0, 0, 0};
+    e = read_tc_status_f16(&t16[0], (cudaStream_t)stream);
+    if (e == cudaSuccess) e = read_bwd_tc_status_f16(&t16[1]);
+    if (e == cudaSuccess) e = read_fwd_tc64_status_f16(&t16[2]);
+    if (e == cudaSuccess) e = read_bwd_kv64_status_f16(&t16[3]);
+    if (e == cudaSuccess) e = read_bwd_q64_status_f16(&t16[4]);
+    if (e != cudaSuccess) return cuda_fail(e, "terra_swin_check");
+    const bool any16 = t16[0] || t16[1] || t16[2] || t16[3] || t16[4];
+    return (timed_out || timed_out_bwd || timed_out_64 || timed_out_kv || timed_out_q || any16) ? TERRA_ERR_DEVICE_TIMEOUT : TERRA_OK;
 }
 
 int terra_profile_enable(int on) {

@@ -28,6 +28,14 @@
 #include "swin_kernels.h"
 #include "tc_common.cuh"
 
+// fp16 build of this file (through the _f16 wrapper file): the kernel, its launcher and its status word get names of
+// their own; the element-independent helpers are compiled in the bf16 build only
+#ifdef TERRA_ELEM_F16
+#define g_bwd_tc_timeout g_bwd_tc_timeout_f16
+#define launch_bwd_tc launch_bwd_tc_f16
+#define read_bwd_tc_status read_bwd_tc_status_f16
+#endif
+
 namespace terra {
 
 __device__ int g_bwd_tc_timeout = 0;   // set when a bounded wait expired in any CTA of the kernel below
@@ -273,8 +281,8 @@ __device__ __forceinline__ void cols16(const uint32_t (&rs)[16], const uint32_t 
     }
 #pragma unroll
     for (int e2 = 0; e2 < 8; ++e2) {
-        pk_p[e2] = pack_bf16(p[2 * e2], p[2 * e2 + 1]);
-        pk_ds[e2] = pack_bf16(ds[2 * e2], ds[2 * e2 + 1]);
+        pk_p[e2] = pack_elem(p[2 * e2], p[2 * e2 + 1]);
+        pk_ds[e2] = pack_elem(ds[2 * e2], ds[2 * e2 + 1]);
     }
 }
 
@@ -308,8 +316,8 @@ __device__ __forceinline__ void math16_row(const uint32_t (&rs)[16], const uint3
     }
 #pragma unroll
     for (int e2 = 0; e2 < 8; ++e2) {
-        pk_p[e2] = pack_bf16(p[2 * e2], p[2 * e2 + 1]);
-        pk_ds[e2] = pack_bf16(ds[2 * e2], ds[2 * e2 + 1]);
+        pk_p[e2] = pack_elem(p[2 * e2], p[2 * e2 + 1]);
+        pk_ds[e2] = pack_elem(ds[2 * e2], ds[2 * e2 + 1]);
     }
 }
 
@@ -394,11 +402,11 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                 tmem_ld16(taddr + 16 * half, r);
                 tmem_ld_wait();
                 sts_u4(rows_a + tile_off<kD>(lane, 2 * half),
-                       pack_bf16(__uint_as_float(r[0]) * f, __uint_as_float(r[1]) * f), pack_bf16(__uint_as_float(r[2]) * f, __uint_as_float(r[3]) * f),
-                       pack_bf16(__uint_as_float(r[4]) * f, __uint_as_float(r[5]) * f), pack_bf16(__uint_as_float(r[6]) * f, __uint_as_float(r[7]) * f));
+                       pack_elem(__uint_as_float(r[0]) * f, __uint_as_float(r[1]) * f), pack_elem(__uint_as_float(r[2]) * f, __uint_as_float(r[3]) * f),
+                       pack_elem(__uint_as_float(r[4]) * f, __uint_as_float(r[5]) * f), pack_elem(__uint_as_float(r[6]) * f, __uint_as_float(r[7]) * f));
                 sts_u4(rows_a + tile_off<kD>(lane, 2 * half + 1),
-                       pack_bf16(__uint_as_float(r[8]) * f, __uint_as_float(r[9]) * f), pack_bf16(__uint_as_float(r[10]) * f, __uint_as_float(r[11]) * f),
-                       pack_bf16(__uint_as_float(r[12]) * f, __uint_as_float(r[13]) * f), pack_bf16(__uint_as_float(r[14]) * f, __uint_as_float(r[15]) * f));
+                       pack_elem(__uint_as_float(r[8]) * f, __uint_as_float(r[9]) * f), pack_elem(__uint_as_float(r[10]) * f, __uint_as_float(r[11]) * f),
+                       pack_elem(__uint_as_float(r[12]) * f, __uint_as_float(r[13]) * f), pack_elem(__uint_as_float(r[14]) * f, __uint_as_float(r[15]) * f));
             }
         };
         // the warp's 32 staged rows -> global memory, four lanes per row; `tok` = this lane's row's grid token (-1: none)
@@ -567,8 +575,8 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
         // The CTA's blocks form one sequence across tiles and items: block J uses S / dP buffer J & 1, and its
         // S^T / dP^T are issued two blocks ahead (from the previous item's last blocks where needed, as soon as
         // the item's stage is loaded), so the elementwise warps find them ready.
-        const uint32_t idesc_acc = make_idesc_bf16(128, kD, 0, 1);   // A from TMEM, B = 16 rows x 32 (MN-major)
-        const uint32_t idesc_dq = make_idesc_bf16(128, kD, 1, 1);    // A = dS^T tile read transposed, B = 16 K rows x 32
+        const uint32_t idesc_acc = make_idesc_elem(128, kD, 0, 1);   // A from TMEM, B = 16 rows x 32 (MN-major)
+        const uint32_t idesc_dq = make_idesc_elem(128, kD, 1, 1);    // A = dS^T tile read transposed, B = 16 K rows x 32
         // shared-memory descriptors: one common high word, low words = start address (16-byte units)
         const uint32_t d_hi = sdesc_hi(make_sdesc_sw64(smem0, 512));
         const uint32_t d_q = sdesc_lo(make_sdesc_sw64(smem0 + kOffQ, 512)), d_k = sdesc_lo(make_sdesc_sw64(smem0 + kOffK, 512));
@@ -584,7 +592,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
             const int ncols = min(CB, npad_i - b * CB);
             const uint32_t so = (uint32_t)((stage * kStageBytes) >> 4);
             const uint32_t ro = so + (uint32_t)((t * 128 * kRowBytes) >> 4), co = so + (uint32_t)((b * CB * kRowBytes) >> 4);
-            const uint32_t idesc = make_idesc_bf16(128, ncols, 0, 0);
+            const uint32_t idesc = make_idesc_elem(128, ncols, 0, 0);
             const uint32_t t_s = tmem_base + buf * kColBuf, t_dp = t_s + CB;
             if (elect_one()) {
                 mma_ss_h<false>(t_s, d_k + ro, d_q + co, d_hi, idesc);
@@ -894,6 +902,7 @@ cudaError_t read_bwd_tc_status(int* timed_out) {
 
 constexpr int kMaxGrid = 160;   // CTAs whose bias-gradient tables fit the workspace
 
+#ifndef TERRA_ELEM_F16
 bool bwd_tc_supported(const Geo& g) { return g.d == 32 && g.nmax <= kMaxSlots && g.w <= 16 && g.heads <= 148; }
 
 // workspace: delta [B*H*W*heads] fp32, the prepared bias tables [heads * kFwdBiasFloats] fp32, one
@@ -902,6 +911,7 @@ size_t bwd_tc_workspace_bytes(const Geo& g) {
     const size_t delta = (((size_t)g.B * g.H * g.W * g.heads * sizeof(float)) + 255) / 256 * 256;
     return delta + (size_t)g.heads * kFwdBiasFloats * sizeof(float) + (size_t)kMaxGrid * kDBiasFloats * sizeof(float);
 }
+#endif  // !TERRA_ELEM_F16
 
 cudaError_t launch_bwd_tc(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
                           const void* o, const float* lse, const void* d_o, void* dq, void* dk, void* dv, float* dbias,
@@ -909,7 +919,7 @@ cudaError_t launch_bwd_tc(const Geo& g, const void* q, const void* k, const void
     float* delta = reinterpret_cast<float*>(workspace);
     const size_t delta_bytes = (((size_t)g.B * g.H * g.W * g.heads * sizeof(float)) + 255) / 256 * 256;
     float* prep = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(workspace) + delta_bytes);
-    cudaError_t e = launch_bwd_delta(g, o, d_o, delta, stream);
+    cudaError_t e = TERRA_ELEM_FN(launch_bwd_delta)(g, o, d_o, delta, stream);
     if (e != cudaSuccess) return e;
     e = launch_bias_prep(g, bias, prep, stream);
     if (e != cudaSuccess) return e;

@@ -28,6 +28,14 @@
 #include <cstdlib>
 #include <cstring>
 
+// fp16 build of this file (through the _f16 wrapper file): the kernel, its launcher and its status word get names of
+// their own; the element-independent helpers are compiled in the bf16 build only
+#ifdef TERRA_ELEM_F16
+#define g_bwd_kv64_timeout g_bwd_kv64_timeout_f16
+#define launch_bwd_kv64 launch_bwd_kv64_f16
+#define read_bwd_kv64_status read_bwd_kv64_status_f16
+#endif
+
 namespace terra {
 
 __device__ int g_bwd_kv64_timeout = 0;   // set when a bounded wait expired in any CTA of the kernel below
@@ -184,8 +192,8 @@ __device__ __forceinline__ void cols16(const uint32_t (&rs)[16], const uint32_t 
     }
 #pragma unroll
     for (int e2 = 0; e2 < 8; ++e2) {
-        pk_p[e2] = pack_bf16(p[2 * e2], p[2 * e2 + 1]);
-        pk_ds[e2] = pack_bf16(ds[2 * e2], ds[2 * e2 + 1]);
+        pk_p[e2] = pack_elem(p[2 * e2], p[2 * e2 + 1]);
+        pk_ds[e2] = pack_elem(ds[2 * e2], ds[2 * e2 + 1]);
     }
 }
 
@@ -194,10 +202,10 @@ __device__ __forceinline__ void store_scaled32(uint4* dst, const uint32_t (&r)[3
 #pragma unroll
     for (int c4 = 0; c4 < 4; ++c4) {
         uint4 a;
-        a.x = pack_bf16(__uint_as_float(r[c4 * 8 + 0]) * f, __uint_as_float(r[c4 * 8 + 1]) * f);
-        a.y = pack_bf16(__uint_as_float(r[c4 * 8 + 2]) * f, __uint_as_float(r[c4 * 8 + 3]) * f);
-        a.z = pack_bf16(__uint_as_float(r[c4 * 8 + 4]) * f, __uint_as_float(r[c4 * 8 + 5]) * f);
-        a.w = pack_bf16(__uint_as_float(r[c4 * 8 + 6]) * f, __uint_as_float(r[c4 * 8 + 7]) * f);
+        a.x = pack_elem(__uint_as_float(r[c4 * 8 + 0]) * f, __uint_as_float(r[c4 * 8 + 1]) * f);
+        a.y = pack_elem(__uint_as_float(r[c4 * 8 + 2]) * f, __uint_as_float(r[c4 * 8 + 3]) * f);
+        a.z = pack_elem(__uint_as_float(r[c4 * 8 + 4]) * f, __uint_as_float(r[c4 * 8 + 5]) * f);
+        a.w = pack_elem(__uint_as_float(r[c4 * 8 + 6]) * f, __uint_as_float(r[c4 * 8 + 7]) * f);
         dst[c4] = a;
     }
 }
@@ -472,7 +480,7 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
         }
     } else {
         // ------------------------------------------------------------------ MMA issuer
-        const uint32_t idesc_acc = make_idesc_bf16(128, D, 0, 1);        // A from TMEM, B = 16 rows x D (MN-major)
+        const uint32_t idesc_acc = make_idesc_elem(128, D, 0, 1);        // A from TMEM, B = 16 rows x D (MN-major)
         const uint32_t sd_hi = sdesc_hi(make_sdesc_sw64(smem0, 512));    // common high word of the K-major descriptors
         int kuse = 0;
         unsigned p0 = 0;                                  // half chunks before the current item
@@ -498,7 +506,7 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             // (descriptor low words = start address in 16-byte units: + 2 per 32-byte K step, + kPart / 16 per 32-column part)
             const uint32_t k_lo = sdesc_lo(make_sdesc_sw64(kb + kOffK, 512)), v_lo = sdesc_lo(make_sdesc_sw64(kb + kOffV, 512));
             auto issue_sdp = [&](int h, uint32_t sb, int nc, int buf) {
-                const uint32_t idesc = make_idesc_bf16(128, nc, 0, 0);
+                const uint32_t idesc = make_idesc_elem(128, nc, 0, 0);
                 const uint32_t q_lo = sdesc_lo(make_sdesc_sw64(sb + kOffQ + h * 64 * kPartBytes, 512));
                 const uint32_t g_lo = sdesc_lo(make_sdesc_sw64(sb + kOffG + h * 64 * kPartBytes, 512));
                 const uint32_t t_s = tmem_base + kBufCols * buf, t_dp = t_s + 64;
@@ -722,7 +730,9 @@ bool no_tma_env() {
 }
 }  // namespace
 
+#ifndef TERRA_ELEM_F16
 bool bwd_kv64_supported(const Geo& g) { return (g.d == 64 || g.d == 128) && g.w <= 32 && g.nmax <= 1024 && g.heads <= 148; }
+#endif  // !TERRA_ELEM_F16
 
 // `prep` = the prepared bias tables of the head-dim-64 forward kernel (kBiasFloats per head), filled by the caller
 cudaError_t launch_bwd_kv64(const Geo& g, const void* q, const void* k, const void* v, const void* d_o, const float* prep,

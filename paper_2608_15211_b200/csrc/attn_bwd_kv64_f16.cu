@@ -1,0 +1,3 @@
+// The key side of the large-window tcgen05 backward for fp16 activations: the same source, compiled with the fp16 element operations.
+#define TERRA_ELEM_F16 1
+#include "attn_bwd_kv64.cu"

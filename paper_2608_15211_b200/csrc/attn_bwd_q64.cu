@@ -37,6 +37,14 @@
 #include <cstdlib>
 #include <cstring>
 
+// fp16 build of this file (through the _f16 wrapper file): the kernel, its launcher and its status word get names of
+// their own; the element-independent helpers are compiled in the bf16 build only
+#ifdef TERRA_ELEM_F16
+#define g_bwd_q64_timeout g_bwd_q64_timeout_f16
+#define launch_bwd_q64 launch_bwd_q64_f16
+#define read_bwd_q64_status read_bwd_q64_status_f16
+#endif
+
 namespace terra {
 
 __device__ int g_bwd_q64_timeout = 0;   // set when a bounded wait expired in any CTA of the kernel below
@@ -201,7 +209,7 @@ __device__ __forceinline__ void cols16(const uint32_t (&rs)[16], const uint32_t 
 #pragma unroll
     for (int e = 0; e < 16; ++e) sts_f32(tab + 256 * e, tv[e] + ds[e]);
 #pragma unroll
-    for (int e2 = 0; e2 < 8; ++e2) pk_ds[e2] = pack_bf16(ds[2 * e2], ds[2 * e2 + 1]);
+    for (int e2 = 0; e2 < 8; ++e2) pk_ds[e2] = pack_elem(ds[2 * e2], ds[2 * e2 + 1]);
     __syncwarp();                                         // the next group's entries are this group's, one lane over
 }
 
@@ -482,8 +490,8 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
         }
     } else {
         // ------------------------------------------------------------------ MMA issuer
-        const uint32_t idesc_s = make_idesc_bf16(128, 64, 0, 0);
-        const uint32_t idesc_acc = make_idesc_bf16(128, D, 0, 1);        // A from TMEM, B = 16 rows x D (MN-major)
+        const uint32_t idesc_s = make_idesc_elem(128, 64, 0, 0);
+        const uint32_t idesc_acc = make_idesc_elem(128, D, 0, 1);        // A from TMEM, B = 16 rows x D (MN-major)
         const uint32_t sd_hi = sdesc_hi(make_sdesc_sw64(smem0, 512));    // common high word of the K-major descriptors
         int quse = 0;
         bool ok = true;
@@ -684,10 +692,10 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
 #pragma unroll
                 for (int c4 = 0; c4 < 4; ++c4) {
                     uint4 a;
-                    a.x = pack_bf16(__uint_as_float(r0[c4 * 8 + 0]) * out_scale, __uint_as_float(r0[c4 * 8 + 1]) * out_scale);
-                    a.y = pack_bf16(__uint_as_float(r0[c4 * 8 + 2]) * out_scale, __uint_as_float(r0[c4 * 8 + 3]) * out_scale);
-                    a.z = pack_bf16(__uint_as_float(r0[c4 * 8 + 4]) * out_scale, __uint_as_float(r0[c4 * 8 + 5]) * out_scale);
-                    a.w = pack_bf16(__uint_as_float(r0[c4 * 8 + 6]) * out_scale, __uint_as_float(r0[c4 * 8 + 7]) * out_scale);
+                    a.x = pack_elem(__uint_as_float(r0[c4 * 8 + 0]) * out_scale, __uint_as_float(r0[c4 * 8 + 1]) * out_scale);
+                    a.y = pack_elem(__uint_as_float(r0[c4 * 8 + 2]) * out_scale, __uint_as_float(r0[c4 * 8 + 3]) * out_scale);
+                    a.z = pack_elem(__uint_as_float(r0[c4 * 8 + 4]) * out_scale, __uint_as_float(r0[c4 * 8 + 5]) * out_scale);
+                    a.w = pack_elem(__uint_as_float(r0[c4 * 8 + 6]) * out_scale, __uint_as_float(r0[c4 * 8 + 7]) * out_scale);
                     dst[4 * hq + c4] = a;
                 }
             }
@@ -714,9 +722,11 @@ cudaError_t read_bwd_q64_status(int* timed_out) {
     return e;
 }
 
+#ifndef TERRA_ELEM_F16
 bool bwd_q64_supported(const Geo& g) {
     return (g.d == 64 || g.d == 128) && g.w == kW && g.H % kW == 0 && g.W % kW == 0 && g.heads <= 148;
 }
+#endif  // !TERRA_ELEM_F16
 
 // `prep` = the prepared bias tables of the head-dim-64 forward kernel (kBiasFloats per head), filled by the caller;
 // dbias is overwritten

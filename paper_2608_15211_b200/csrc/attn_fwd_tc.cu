@@ -28,6 +28,14 @@
 #include "tc_common.cuh"
 #include "tma_rows.cuh"
 
+// fp16 build of this file (through attn_fwd_tc_f16.cu): the kernel, its launcher and its status word get names of
+// their own; the element-independent helpers below are compiled in the bf16 build only
+#ifdef TERRA_ELEM_F16
+#define g_tc_timeout g_tc_timeout_f16
+#define launch_fwd_tc launch_fwd_tc_f16
+#define read_tc_status read_tc_status_f16
+#endif
+
 namespace terra {
 
 __device__ int g_tc_timeout = 0;   // set when a bounded wait expired in any CTA
@@ -170,8 +178,8 @@ __device__ __forceinline__ float softmax_cols(const uint32_t (&r)[N], uint32_t (
                 p[e + 1] = fast_exp2(xv[e + 1]);
             }
         }
-        pk[e4 * 2] = pack_bf16(p[0], p[1]);
-        pk[e4 * 2 + 1] = pack_bf16(p[2], p[3]);
+        pk[e4 * 2] = pack_elem(p[0], p[1]);
+        pk[e4 * 2 + 1] = pack_elem(p[2], p[3]);
     }
     return 0.f;       // the row sum comes from the ones columns of the P V product
 }
@@ -217,7 +225,7 @@ __device__ __forceinline__ void softmax_cols16_row(const uint32_t* r, uint32_t* 
         float x0, x1;
         fma2(x0, x1, __uint_as_float(r[2 * e2]), __uint_as_float(r[2 * e2 + 1]), scale, bv[2 * e2], bv[2 * e2 + 1]);
         add2(x0, x1, x0, x1, neg_m);
-        pk[e2] = pack_bf16(fast_exp2(x0), fast_exp2(x1));
+        pk[e2] = pack_elem(fast_exp2(x0), fast_exp2(x1));
     }
 }
 
@@ -399,7 +407,7 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
     }
     for (int i = tid; i < kMaxSlots * 4; i += kThreads) {          // (row, 16-byte chunk): chunks 0, 1 = ones, 2, 3 = zeros
         const int row = i >> 2, chunk = i & 3;
-        const uint32_t val = chunk < 2 ? 0x3F803F80u : 0u;
+        const uint32_t val = chunk < 2 ? kElemOnesPair : 0u;
         *reinterpret_cast<uint4*>(smem + kOffOnes + tile_off<kD>(row, chunk)) = make_uint4(val, val, val, val);
     }
     fence_proxy_async();
@@ -564,13 +572,13 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
         // The whole warp runs the loop and waits (a warp whose 32 lanes wait together is parked and woken as a
         // whole); one elected lane issues the MMAs and commits.
         {
-            const uint32_t idesc_pv = make_idesc_bf16(128, kNO, 0, 1);   // B = [V | ones]: 32 + 16 columns
+            const uint32_t idesc_pv = make_idesc_elem(128, kNO, 0, 1);   // B = [V | ones]: 32 + 16 columns
             int kuse = 0, use_t[2] = {0, 0}, freed_t[2] = {0, 0};   // uses begun / s_free phases consumed
             bool ok = true;
             auto issue_qk = [&](const Item& x, int s, int t) {
                 const uint32_t qa = smem0 + s * kStageBytes + kOffQ + t * 128 * kRowBytes;
                 const uint32_t ka = smem0 + s * kStageBytes + kOffK;
-                const uint32_t idesc = make_idesc_bf16(128, x.npad, 0, 0);
+                const uint32_t idesc = make_idesc_elem(128, x.npad, 0, 0);
                 if (elect_one()) {
 #pragma unroll
                     for (int ks = 0; ks < kD / 16; ++ks)
@@ -739,10 +747,10 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
 #pragma unroll
                 for (int c4 = 0; c4 < 4; ++c4) {
                     uint4 val;
-                    val.x = pack_bf16(__uint_as_float(ro[c4 * 8 + 0]) * inv, __uint_as_float(ro[c4 * 8 + 1]) * inv);
-                    val.y = pack_bf16(__uint_as_float(ro[c4 * 8 + 2]) * inv, __uint_as_float(ro[c4 * 8 + 3]) * inv);
-                    val.z = pack_bf16(__uint_as_float(ro[c4 * 8 + 4]) * inv, __uint_as_float(ro[c4 * 8 + 5]) * inv);
-                    val.w = pack_bf16(__uint_as_float(ro[c4 * 8 + 6]) * inv, __uint_as_float(ro[c4 * 8 + 7]) * inv);
+                    val.x = pack_elem(__uint_as_float(ro[c4 * 8 + 0]) * inv, __uint_as_float(ro[c4 * 8 + 1]) * inv);
+                    val.y = pack_elem(__uint_as_float(ro[c4 * 8 + 2]) * inv, __uint_as_float(ro[c4 * 8 + 3]) * inv);
+                    val.z = pack_elem(__uint_as_float(ro[c4 * 8 + 4]) * inv, __uint_as_float(ro[c4 * 8 + 5]) * inv);
+                    val.w = pack_elem(__uint_as_float(ro[c4 * 8 + 6]) * inv, __uint_as_float(ro[c4 * 8 + 7]) * inv);
                     dst[c4] = val;
                 }
             }
@@ -800,6 +808,7 @@ swin_fwd_bias_prep_kernel(const float* __restrict__ bias, float* __restrict__ pr
 
 }  // namespace
 
+#ifndef TERRA_ELEM_F16
 bool fwd_tc_supported(const Geo& g) { return g.d == 32 && g.nmax <= kMaxSlots && g.w <= 16; }
 
 // The TMA variants fetch a window row with one tiled copy: every window row must be one run of consecutive tokens
@@ -867,6 +876,7 @@ bool make_row_maps3(RowMaps3* maps, const Geo& g, const void* base, int token_st
 }
 
 size_t fwd_tc_workspace_bytes(const Geo& g) { return (size_t)g.heads * kFwdBiasFloats * sizeof(float); }
+#endif  // !TERRA_ELEM_F16
 
 cudaError_t launch_fwd_tc(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
                           void* o, float* lse, void* workspace, int sm_count, cudaStream_t stream) {
@@ -893,6 +903,7 @@ cudaError_t launch_fwd_tc(const Geo& g, const void* q, const void* k, const void
     return cudaGetLastError();
 }
 
+#ifndef TERRA_ELEM_F16
 // Self-test of the failure report: one CTA waits, with a short cycle limit, on a barrier that nothing ever
 // arrives on; the wait gives up, the kernel raises the device status word and returns normally.
 __global__ void bounded_wait_selftest_kernel(long long limit_cycles) {
@@ -921,6 +932,8 @@ cudaError_t launch_bias_prep(const Geo& g, const float* bias, float* prep, cudaS
     count_launch(stream);
     return cudaGetLastError();
 }
+
+#endif  // !TERRA_ELEM_F16
 
 cudaError_t read_tc_status(int* timed_out, cudaStream_t stream) {
     cudaError_t e = cudaStreamSynchronize(stream);

@@ -29,6 +29,14 @@
 #include "tc_common.cuh"
 #include "tma_rows.cuh"
 
+// fp16 build of this file (through the _f16 wrapper file): the kernel, its launcher and its status word get names of
+// their own; the element-independent helpers are compiled in the bf16 build only
+#ifdef TERRA_ELEM_F16
+#define g_fwd_tc64_timeout g_fwd_tc64_timeout_f16
+#define launch_fwd_tc64 launch_fwd_tc64_f16
+#define read_fwd_tc64_status read_fwd_tc64_status_f16
+#endif
+
 namespace terra {
 
 __device__ int g_fwd_tc64_timeout = 0;   // set when a bounded wait expired in any CTA of the kernel below
@@ -150,8 +158,8 @@ __device__ __forceinline__ void softmax_cols(const uint32_t (&r)[N], uint32_t (&
             if (MASKED && kl[e] != label_i) xv = -INFINITY;
             p[e] = fast_exp2(xv);
         }
-        pk[e4 * 2] = pack_bf16(p[0], p[1]);
-        pk[e4 * 2 + 1] = pack_bf16(p[2], p[3]);
+        pk[e4 * 2] = pack_elem(p[0], p[1]);
+        pk[e4 * 2 + 1] = pack_elem(p[2], p[3]);
         if (SUM) {
             sum[0] += p[0] + p[2];
             sum[1] += p[1] + p[3];
@@ -209,7 +217,7 @@ __device__ __forceinline__ void softmax_cols32_row(const uint32_t (&r)[32], uint
     for (int e2 = 0; e2 < 16; ++e2) {
         const float p0 = fast_exp2(fmaf(__uint_as_float(r[2 * e2]), scale, bv[2 * e2]) + neg_m);
         const float p1 = fast_exp2(fmaf(__uint_as_float(r[2 * e2 + 1]), scale, bv[2 * e2 + 1]) + neg_m);
-        pk[e2] = pack_bf16(p0, p1);
+        pk[e2] = pack_elem(p0, p1);
         if (SUM) {
             sum[0] += p0;
             sum[1] += p1;
@@ -242,10 +250,10 @@ __device__ __forceinline__ void store_o32(uint4* dst, const uint32_t (&ro)[32], 
 #pragma unroll
     for (int c4 = 0; c4 < 4; ++c4) {
         uint4 val;
-        val.x = pack_bf16(__uint_as_float(ro[c4 * 8 + 0]) * inv, __uint_as_float(ro[c4 * 8 + 1]) * inv);
-        val.y = pack_bf16(__uint_as_float(ro[c4 * 8 + 2]) * inv, __uint_as_float(ro[c4 * 8 + 3]) * inv);
-        val.z = pack_bf16(__uint_as_float(ro[c4 * 8 + 4]) * inv, __uint_as_float(ro[c4 * 8 + 5]) * inv);
-        val.w = pack_bf16(__uint_as_float(ro[c4 * 8 + 6]) * inv, __uint_as_float(ro[c4 * 8 + 7]) * inv);
+        val.x = pack_elem(__uint_as_float(ro[c4 * 8 + 0]) * inv, __uint_as_float(ro[c4 * 8 + 1]) * inv);
+        val.y = pack_elem(__uint_as_float(ro[c4 * 8 + 2]) * inv, __uint_as_float(ro[c4 * 8 + 3]) * inv);
+        val.z = pack_elem(__uint_as_float(ro[c4 * 8 + 4]) * inv, __uint_as_float(ro[c4 * 8 + 5]) * inv);
+        val.w = pack_elem(__uint_as_float(ro[c4 * 8 + 6]) * inv, __uint_as_float(ro[c4 * 8 + 7]) * inv);
         dst[c4] = val;
     }
 }
@@ -329,7 +337,7 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
     if (L::kOnes) {
         for (int i = tid; i < kSlots * kChunk * 4; i += kThreads) {
             const int s = i / (kChunk * 4), rem = i - s * (kChunk * 4), row = rem >> 2, chunk = rem & 3;
-            const uint32_t val = chunk < 2 ? 0x3F803F80u : 0u;
+            const uint32_t val = chunk < 2 ? kElemOnesPair : 0u;
             *reinterpret_cast<uint4*>(smem + kOffSlots + s * kSlotBytes + L::kOffOnes + tile_off<32>(row, chunk)) = make_uint4(val, val, val, val);
         }
     }
@@ -583,7 +591,7 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
         }
     } else {
         // ------------------------------------------------------------------ MMA issuer
-        const uint32_t idesc_pv = make_idesc_bf16(128, kNO, 0, 1);
+        const uint32_t idesc_pv = make_idesc_elem(128, kNO, 0, 1);
         int kuse = 0;
         long long ru = 0;
         int n_p[2] = {0, 0}, n_items_t[2] = {0, 0};
@@ -603,7 +611,7 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             const uint32_t sd_hi = sdesc_hi(make_sdesc_sw64(smem0, 512));
             const uint32_t q_lo0 = sdesc_lo(make_sdesc_sw64(qb, 512));
             auto issue_qk = [&](int t, uint32_t sb, int ncols) {
-                const uint32_t idesc = make_idesc_bf16(128, ncols, 0, 0);
+                const uint32_t idesc = make_idesc_elem(128, ncols, 0, 0);
                 const uint32_t q_lo = q_lo0 + ((t * 128 * kPartBytes) >> 4), k_lo = sdesc_lo(make_sdesc_sw64(sb, 512));
                 const uint32_t t_d = tmem_base + t * 256;
                 if (elect_one()) {
@@ -945,6 +953,7 @@ cudaError_t read_fwd_tc64_status(int* timed_out) {
     return e;
 }
 
+#ifndef TERRA_ELEM_F16
 // prepared bias tables (kBiasFloats = 6048 floats per head) for the kernels of the head-dim-64 regime
 cudaError_t launch_bias_prep64(const Geo& g, const float* bias, float* prep, cudaStream_t stream) {
     swin_fwd_bias_prep64_kernel<<<g.heads, 256, 0, stream>>>(bias, prep, g.w, g.heads);
@@ -955,6 +964,7 @@ cudaError_t launch_bias_prep64(const Geo& g, const float* bias, float* prep, cud
 bool fwd_tc64_supported(const Geo& g) { return (g.d == 64 || g.d == 128) && g.w <= 32 && g.nmax <= 1024 && g.heads <= 148; }
 
 size_t fwd_tc64_workspace_bytes(const Geo& g) { return (size_t)g.heads * kBiasFloats * sizeof(float); }
+#endif  // !TERRA_ELEM_F16
 
 cudaError_t launch_fwd_tc64(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
                             void* o, float* lse, void* workspace, int sm_count, cudaStream_t stream) {

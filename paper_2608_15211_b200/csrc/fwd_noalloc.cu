@@ -60,17 +60,18 @@ extern "C" int terra_swin_attn_fwd_noalloc(const terra_swin_desc* desc, const vo
     rc = current_device_sm_count(&sms);
     if (rc) return rc;
     cudaError_t e;
-    if (g.f16) {
-        e = launch_fwd_mma_f16(g, q, k, v, bias_table, o, lse, (cudaStream_t)stream);   // fp16: register-tile kernel, no scratch
-    } else if (fwd_tc_supported(g) && g.nmax > 64) {        // (windows of at most 64 tokens: the register-tile kernel, as in the regular forward)
+    if (fwd_tc_supported(g) && g.nmax > 64) {        // (windows of at most 64 tokens: the register-tile kernel, as in the regular forward)
         // the one shape-dependent limit of this entry point: the fixed scratch holds this many heads
         if (g.heads > kNoAllocMaxHeads) return TERRA_ERR_NOALLOC_LIMIT;
         float* scratch = nullptr;
         rc = scratch_for_current_device(&scratch);
         if (rc) return rc;
-        e = launch_fwd_tc(g, q, k, v, bias_table, o, lse, scratch, sms, (cudaStream_t)stream);
+        e = g.f16 ? launch_fwd_tc_f16(g, q, k, v, bias_table, o, lse, scratch, sms, (cudaStream_t)stream)
+                  : launch_fwd_tc(g, q, k, v, bias_table, o, lse, scratch, sms, (cudaStream_t)stream);
     } else {
-        e = launch_fwd_mma(g, q, k, v, bias_table, o, lse, (cudaStream_t)stream);   // this kernel needs no scratch
+        // this kernel needs no scratch
+        e = g.f16 ? launch_fwd_mma_f16(g, q, k, v, bias_table, o, lse, (cudaStream_t)stream)
+                  : launch_fwd_mma(g, q, k, v, bias_table, o, lse, (cudaStream_t)stream);
     }
     return e == cudaSuccess ? TERRA_OK : report_cuda_failure(e, "terra_swin_attn_fwd_noalloc");
 }

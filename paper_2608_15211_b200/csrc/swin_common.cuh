@@ -156,17 +156,20 @@ __device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
     __half2 v = __floats2half2_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
 }
-// The register-tile kernel files are compiled twice, for bf16 and (with TERRA_ELEM_F16 defined by a one-line wrapper
-// file) for fp16 activations: same code, the element type enters through these three operations and the name suffix.
+// The kernel files are compiled twice, for bf16 and (with TERRA_ELEM_F16 defined by a one-line wrapper file) for fp16
+// activations: same code, the element type enters through these operations, the tcgen05 instruction descriptor's
+// operand formats (make_idesc_elem) and the name suffix.
 #ifdef TERRA_ELEM_F16
 #define TERRA_ELEM_FN(name) name##_f16
 #define mma_elem mma_f16
 #define pack_elem pack_f16
+#define kElemOnesPair 0x3C003C00u         /* two fp16 ones */
 __device__ __forceinline__ float2 elem2_to_float2(uint32_t v) { return __half22float2(*reinterpret_cast<const __half2*>(&v)); }
 #else
 #define TERRA_ELEM_FN(name) name
 #define mma_elem mma_bf16
 #define pack_elem pack_bf16
+#define kElemOnesPair 0x3F803F80u         /* two bf16 ones */
 __device__ __forceinline__ float2 elem2_to_float2(uint32_t v) { return __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&v)); }
 #endif
 __device__ __forceinline__ float fast_exp2(float x) {

@@ -25,6 +25,23 @@ bool bwd_small_supported_f16(const Geo& g);
 cudaError_t launch_bwd_small_f16(const Geo& g, const void* q, const void* k, const void* v, const void* o, const void* d_o,
                                  const float* bias, const float* lse, void* dq, void* dk, void* dv, float* dbias,
                                  int sm_count, cudaStream_t stream);
+// the tcgen05 kernels compiled for fp16 activations (same shapes, workspaces and helpers as the bf16 ones)
+cudaError_t launch_fwd_tc_f16(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
+                              void* o, float* lse, void* workspace, int sm_count, cudaStream_t stream);
+cudaError_t read_tc_status_f16(int* timed_out, cudaStream_t stream);
+cudaError_t launch_bwd_tc_f16(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
+                              const void* o, const float* lse, const void* d_o, void* dq, void* dk, void* dv, float* dbias,
+                              void* workspace, int sm_count, cudaStream_t stream);
+cudaError_t read_bwd_tc_status_f16(int* timed_out);
+cudaError_t launch_fwd_tc64_f16(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
+                                void* o, float* lse, void* workspace, int sm_count, cudaStream_t stream);
+cudaError_t read_fwd_tc64_status_f16(int* timed_out);
+cudaError_t launch_bwd_kv64_f16(const Geo& g, const void* q, const void* k, const void* v, const void* d_o, const float* prep,
+                                const float* lse, const float* delta, void* dk, void* dv, int sm_count, cudaStream_t stream);
+cudaError_t read_bwd_kv64_status_f16(int* timed_out);
+cudaError_t launch_bwd_q64_f16(const Geo& g, const void* q, const void* k, const void* v, const void* d_o, const float* prep,
+                               const float* lse, const float* delta, void* dq, float* dbias, int sm_count, cudaStream_t stream);
+cudaError_t read_bwd_q64_status_f16(int* timed_out);
 cudaError_t launch_bwd_delta_f16(const Geo& g, const void* o, const void* d_o, float* delta, cudaStream_t stream);
 cudaError_t launch_bwd_mma_f16(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
                                const float* lse, const float* delta, const void* d_o,

@@ -162,6 +162,15 @@ __host__ __device__ constexpr uint32_t make_idesc_bf16(int M, int N, int a_mn, i
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
            ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
+// the same for fp16 operands (operand format fields 0)
+__host__ __device__ constexpr uint32_t make_idesc_f16(int M, int N, int a_mn, int b_mn) {
+    return (1u << 4) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+#ifdef TERRA_ELEM_F16
+#define make_idesc_elem make_idesc_f16
+#else
+#define make_idesc_elem make_idesc_bf16
+#endif
 // Shared-memory matrix descriptor for rows of 64 bytes under the 64-byte swizzle: 8-row groups are
 // `sbo_bytes` apart; the leading-dimension field is unused for a single swizzle atom along the row.
 __device__ __forceinline__ uint64_t make_sdesc_sw64(uint32_t smem_addr, uint32_t sbo_bytes) {

@@ -18,6 +18,10 @@ SHAPES = [
     ("f16_d64_w20_ragged", 1, 45, 50, 2, 64, 20, 10, 10, 0, 1),
     ("f16_d128_w8", 1, 30, 44, 2, 128, 8, 4, 4, 0, 1),
     ("f16_d128_w32", 1, 40, 70, 1, 128, 32, 16, 16, 0, 0),
+    # grids of complete windows: the bulk-copy loaders and the tcgen05 query side of the fp16 builds
+    ("f16_d128_w32_complete", 1, 64, 64, 1, 128, 32, 16, 16, 0, 1),
+    ("f16_d32_w16_complete", 2, 32, 64, 3, 32, 16, 8, 0, 0, 1),
+    ("f16_d64_w16_complete", 1, 32, 48, 2, 64, 16, 8, 8, 0, 0),
 ]
 
 
