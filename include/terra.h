@@ -48,9 +48,9 @@ typedef enum {
 } terra_status;
 
 /*
- * Element type of the activations and their gradients.  bf16 is the type the tensor-core kernels of this library
- * are written for; fp16 is what the paper trains in (Section VII-A: FP16 mixed precision) and runs on the
- * register-tile kernels for every shape.  Scores, softmax, accumulation, lse, bias_table and dbias are fp32 either
+ * Element type of the activations and their gradients: bf16, or fp16, which is what the paper trains in (Section
+ * VII-A: FP16 mixed precision).  Every kernel of the library exists in a build for either type and the same kernel is
+ * chosen for a shape whatever the type.  Scores, softmax, accumulation, lse, bias_table and dbias are fp32 either
  * way.  A descriptor zero-initialised beyond `scale` selects bf16.
  */
 #define TERRA_DTYPE_BF16 0
