@@ -1,51 +1,80 @@
-"""Seeded random shapes (head dim, window side, grid extents complete or ragged, shifts, periodic flags): forward and
-backward through the C ABI against the oracle.  The shapes cross every dispatch boundary of the library (windows of at
-most 64 tokens, the small-window and the chunked tcgen05 kernels, bulk-copy and gathering loaders, register tiles)."""
+"""Seeded random small shapes through the C ABI against the oracle: window sides 1..16 at head dim 32 (the
+tcgen05 kernels: every tile / block / mask / truncation combination the shapes happen to hit), larger
+windows or head dim 64 (the chunked tcgen05 kernels and the register-tile kernels), and grids with hundreds to thousands of (window, head) items
+(several items per CTA in mixed order of one-tile and two-tile windows)."""
 import random
 
 import pytest
+import torch
 
 import oracle
-import paper_2608_15211_b200 as terra
 from paper_2608_15211_b200.workloads import make_inputs, small_config
 from tests._parity import gate, gpu_rows
+from tests.test_gpu_parity import _run_bwd, _run_fwd, _to_gpu
 
 pytestmark = pytest.mark.gpu
 
 
-def _random_config(rng, i):
-    d = rng.choice([32, 64, 128, 128])
-    w = rng.choice([4, 7, 8, 8, 12, 16, 16, 20, 32, 32])
-    if rng.random() < 0.5:                                   # a grid of complete windows
-        H, W = w * rng.randint(1, 3), w * rng.randint(1, 3)
-    else:
-        H, W = rng.randint(max(2, w // 2), 2 * w + 5), rng.randint(max(2, w // 2), 2 * w + 9)
-    if H * W > 6000:
-        H = max(2, 6000 // W)
-    heads, B = rng.randint(1, 3), rng.randint(1, 2)
-    sh = rng.choice([0, w // 2, rng.randint(0, w - 1), 8 * rng.randint(0, 3)]) % max(1, min(w, H))
-    sw = rng.choice([0, w // 2, rng.randint(0, w - 1), 8 * rng.randint(0, 3)]) % max(1, min(w, W))
-    return small_config(f"random{i}", B, H, W, heads, d, w, sh, sw, rng.randint(0, 1), rng.randint(0, 1))
+def _shapes():
+    rng = random.Random(20260815)
+    out = []
+    for i in range(14):                      # head dim 32, window side <= 16
+        w = rng.choice([1, 3, 4, 5, 7, 8, 8, 9, 11, 12, 13, 14, 14, 15, 16, 16, 16])
+        H, W = rng.randint(1, 6 * w + 7), rng.randint(1, 6 * w + 9)
+        out.append((f"r{i}_w{w}", rng.choice([1, 1, 2, 3]), H, W, rng.choice([1, 2, 3, 5]), 32, w,
+                    rng.randint(0, H + 2), rng.randint(0, W + 2), rng.randint(0, 1), rng.randint(0, 1)))
+    for i in range(6):                       # head dim 64 and / or windows larger than 16
+        d = rng.choice([64, 64, 32])
+        w = rng.choice([32, 32, 24, 20, 17])
+        H, W = rng.randint(w // 2, 2 * w + 9), rng.randint(w // 2, 3 * w + 5)
+        out.append((f"g{i}_d{d}_w{w}", rng.choice([1, 2]), H, W, rng.choice([1, 2, 3]), d, w,
+                    rng.randint(0, H), rng.randint(0, W), rng.randint(0, 1), rng.randint(0, 1)))
+    rng = random.Random(20260816)
+    for i in range(8):                       # many items per CTA: the persistent kernels' rings turn several times
+        w = rng.choice([3, 5, 6, 8, 9, 12, 13, 14, 16])
+        H, W = rng.randint(6 * w, 14 * w + 7), rng.randint(6 * w, 14 * w + 9)
+        out.append((f"m{i}_w{w}", rng.choice([1, 2, 3]), H, W, rng.choice([3, 5, 6, 7]), 32, w,
+                    rng.randint(0, H + 2), rng.randint(0, W + 2), rng.randint(0, 1), rng.randint(0, 1)))
+    # found by fuzzing: 540 items on 148 CTAs, two of which meet three one-tile windows (6 wide) and then a
+    # two-tile one, i.e. the second query tile's first use comes after a whole turn of the forward kernel's stage ring
+    out.append(("ring_turn_then_second_tile", 2, 111, 71, 5, 32, 13, 45, 48, 0, 0))
+    # head dim 64 on the chunked tcgen05 forward: 1, 3, 5 and 8 query tiles per window (a pair's second tile missing
+    # for the odd counts), truncated and masked 32-wide windows, sides below 32, several items per CTA
+    out += [("d64_w32_full", 1, 64, 96, 2, 64, 32, 16, 16, 0, 1),
+            ("d64_w32_rows9", 2, 41, 64, 3, 64, 32, 5, 7, 0, 0),         # last window row 9 high: 288 tokens, 3 tiles
+            ("d64_w24", 1, 60, 72, 2, 64, 24, 12, 12, 0, 1),             # 576 tokens: 5 tiles
+            ("d64_w17", 2, 40, 50, 3, 64, 17, 8, 9, 1, 0),               # 289 tokens: 3 tiles, ragged chunks
+            ("d64_w8_many", 2, 64, 96, 5, 64, 8, 4, 4, 0, 1),            # one-tile windows, 960 items
+            ("d64_w32_narrow", 1, 70, 45, 2, 64, 32, 20, 30, 0, 0)]      # 13-wide last column, 6-high last row
+    # complete 32 x 32 windows at head dim 64: the tcgen05 query side of the backward pass (dQ, dBias).  One item per
+    # CTA; both masks and two samples; CTAs whose item range crosses a query-tile boundary (their bias-gradient tables
+    # are flushed in mid-run); one or two items per CTA with 29 CTAs per head
+    out += [("d64_w32_one_window", 1, 32, 32, 1, 64, 32, 0, 0, 1, 1),
+            ("d64_w32_masks_b2", 2, 64, 96, 3, 64, 32, 5, 9, 0, 0),
+            ("d64_w32_heads12", 1, 96, 160, 12, 64, 32, 16, 16, 0, 1),
+            ("d64_w32_heads5", 1, 64, 64, 5, 64, 32, 40, 3, 0, 1)]
+    return out
 
 
-@pytest.mark.parametrize("seed", [11, 12, 13])
-def test_random_shapes_forward_backward(seed):
-    rng = random.Random(seed)
-    for i in range(30):
-        cfg = _random_config(rng, i)
-        x = make_inputs(cfg)
-        x["bias"] = x["bias"] * 25.0
-        xg = {k: v.cuda() for k, v in x.items()}
-        d = terra.make_desc(cfg)
-        o, lse = terra.terra_swin_attn_fwd(d, xg["q"], xg["k"], xg["v"], xg["bias"])
-        dq, dk, dv, dbias = terra.terra_swin_attn_bwd(d, xg["q"], xg["k"], xg["v"], xg["bias"], o, lse, xg["do"])
-        terra.terra_swin_check()
-        table = x["bias"].double().numpy()
-        ro, rl = oracle.attn_fwd(cfg, x["q"], x["k"], x["v"], table)
-        rq, rk, rv, rb = oracle.attn_bwd(cfg, x["q"], x["k"], x["v"], x["do"], table)
-        tok = oracle.selection_tokens(cfg, None)
-        shape = f"B={cfg.B} H={cfg.H} W={cfg.W} heads={cfg.heads} d={cfg.head_dim} w={cfg.window}"
-        for name, got, ref in (("o", gpu_rows(o, cfg, tok), ro), ("lse", gpu_rows(lse, cfg, tok), rl),
-                               ("dq", gpu_rows(dq, cfg, tok), rq), ("dk", gpu_rows(dk, cfg, tok), rk),
-                               ("dv", gpu_rows(dv, cfg, tok), rv), ("dbias", dbias.cpu().double().numpy(), rb)):
-            gate(f"{shape} {name}", got, ref, strict=False)
+SHAPES = _shapes()
+
+
+@pytest.mark.parametrize("case", SHAPES, ids=[c[0] for c in SHAPES])
+def test_random_shape_forward_backward(case):
+    cfg = small_config(*case)
+    x = make_inputs(cfg)
+    x["bias"] = x["bias"] * 25.0          # make the bias matter (std 0.5)
+    xg = _to_gpu(x)
+    d, o, lse = _run_fwd(cfg, xg)
+    dq, dk, dv, dbias = _run_bwd(cfg, d, xg, o, lse)
+    torch.cuda.synchronize()
+    bias64 = x["bias"].double().numpy()
+    ro, rl = oracle.attn_fwd(cfg, x["q"], x["k"], x["v"], bias64)
+    rq, rk, rv, rb = oracle.attn_bwd(cfg, x["q"], x["k"], x["v"], x["do"], bias64)
+    tok = oracle.selection_tokens(cfg, None)
+    # the two gates of the tolerance statement; the tighter diagnostic gate is kept for the fixed cases, where a
+    # single element a hair above it on a 150-token window would not be a finding
+    for name, got, ref in (("o", gpu_rows(o, cfg, tok), ro), ("lse", gpu_rows(lse, cfg, tok), rl),
+                           ("dq", gpu_rows(dq, cfg, tok), rq), ("dk", gpu_rows(dk, cfg, tok), rk),
+                           ("dv", gpu_rows(dv, cfg, tok), rv), ("dbias", dbias.cpu().double().numpy(), rb)):
+        gate(name, got, ref, strict=False)
