@@ -525,14 +525,15 @@ swin_bwd_small_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
         __syncthreads();   // the previous item's readers of the tables and tiles are done
         if (tid < BN) {
             int meta = 0xff << 16, tok = -1;
-            float l2 = INFINITY;                    // padded queries: P = exp2(x - inf) = 0
             if (tid < r.n) {
                 tok = slot_token(g, r, tid, meta);
-                l2 = lse[(sample_off + (size_t)tok) * g.heads + head] * kLog2e;
+                // the row's log-sum-exp travels with the tiles (no load that the copies below would have to wait for)
+                cp_async4(smem_u32(&s_lse[tid]), lse + (sample_off + (size_t)tok) * g.heads + head);
+            } else {
+                s_lse[tid] = INFINITY;              // padded queries: P = exp2(x - inf) = 0
             }
             s_tok[tid] = tok;
             s_meta[tid] = meta;
-            s_lse[tid] = l2;
         }
         __syncthreads();
         load_rows<D>(s_q, q, s_tok, 0, sample_off, g.ts, head, tid);
@@ -569,7 +570,7 @@ swin_bwd_small_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
         // ---- query-major part
         const int row_tab[2] = {warp * 16 + gq, warp * 16 + gq + 8};
         const int meta_r[2] = {s_meta[row_tab[0]], s_meta[row_tab[1]]};
-        const float lse_r[2] = {s_lse[row_tab[0]], s_lse[row_tab[1]]};
+        const float lse_r[2] = {s_lse[row_tab[0]] * kLog2e, s_lse[row_tab[1]] * kLog2e};
         const float del_r[2] = {s_delta[row_tab[0]], s_delta[row_tab[1]]};
         float acc1[DT][4];
         {
