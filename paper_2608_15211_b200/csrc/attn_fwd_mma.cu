@@ -269,14 +269,190 @@ swin_fwd_mma_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
     swin_fwd_mma_body<D, BIG>(g, q, k, v, bias, o, lse, qtiles);
 }
 
-// Head dim 128 with windows of at most 64 tokens (the paper's 8 x 8 windows): one key block per window, so a CTA needs
-// three tiles of shared memory instead of five, and with 168 registers per thread three CTAs share an SM; the path is
-// bound by HBM and lives on the loads the resident CTAs keep in flight.
-__global__ void __launch_bounds__(NTHREADS, 3)
-swin_fwd_mma_d128_small_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
-                               const __nv_bfloat16* __restrict__ v, const float* __restrict__ bias,
-                               __nv_bfloat16* __restrict__ o, float* __restrict__ lse, int qtiles) {
-    swin_fwd_mma_body<128, false>(g, q, k, v, bias, o, lse, qtiles);
+// Windows of at most 64 tokens (the paper's 8 x 8 windows), every head dim: persistent CTAs bound to one head walk over
+// (batch, window); a window is one 64-row tile of Q, K and V.  The tiles are double-buffered: while a window is
+// computed and its output rows are written, the next window's rows are already on their way, so a CTA always has
+// loads in flight (these shapes are bound by HBM).  No online softmax: the whole score row is in registers.
+template <int D>
+__global__ void __launch_bounds__(NTHREADS, 2)
+swin_fwd_small_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
+                      const __nv_bfloat16* __restrict__ v, const float* __restrict__ bias,
+                      __nv_bfloat16* __restrict__ o, float* __restrict__ lse, int ctas_per_head) {
+    constexpr int KS = D / 16;
+    constexpr int DT = D / 8;
+    constexpr int TILE_BYTES = BN * D * 2;
+    constexpr int BUF_BYTES = 3 * TILE_BYTES;
+    extern __shared__ __align__(128) unsigned char smem[];
+
+    const int nbias = (2 * g.w - 1) * (2 * g.w - 1);
+    int* s_tok = reinterpret_cast<int*>(smem);                // [2][64]
+    int* s_meta = s_tok + 2 * BN;                             // [2][64]
+    float* s_bias = reinterpret_cast<float*>(s_meta + 2 * BN);
+    unsigned char* s_tiles = smem + (((size_t)BN * 16 + (size_t)nbias * 4 + 127) / 128) * 128;   // [2][Q | K | V]
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int gq = lane >> 2, tq = lane & 3;
+    const int head = blockIdx.x % g.heads;
+    const int M = g.Mh * g.Mw;
+    const int c0 = (g.w - 1) * 2 * g.w;
+    const long long n_items = (long long)g.B * M;
+    const long long first = blockIdx.x / g.heads;
+
+    for (int i = tid; i < nbias; i += NTHREADS) s_bias[i] = bias[(size_t)i * g.heads + head] * kLog2e;
+
+    // slot tables of item `item` into buffer `b`
+    auto fill_tables = [&](long long item, int b) {
+        if (tid < BN) {
+            const WindowRef r = window_ref(g, (int)(item % M));
+            int meta = 0xff << 16, tok = -1;
+            if (tid < r.n) tok = slot_token(g, r, tid, meta);
+            s_tok[b * BN + tid] = tok;
+            s_meta[b * BN + tid] = meta;
+        }
+    };
+    // the copies of item `item` into buffer `b` (its tables must be visible), one group
+    auto issue_loads = [&](long long item, int b) {
+        const size_t sample_off = (size_t)(item / M) * g.H * g.W;
+        unsigned char* t = s_tiles + b * BUF_BYTES;
+        load_rows<D>(t, q, s_tok + b * BN, 0, sample_off, g.ts, head, tid);
+        load_rows<D>(t + TILE_BYTES, k, s_tok + b * BN, 0, sample_off, g.ts, head, tid);
+        load_rows<D>(t + 2 * TILE_BYTES, v, s_tok + b * BN, 0, sample_off, g.ts, head, tid);
+        cp_async_commit();
+    };
+    if (first < n_items) {
+        fill_tables(first, 0);
+        __syncthreads();
+        issue_loads(first, 0);
+    }
+    int buf = 0;
+    for (long long item = first; item < n_items; item += ctas_per_head, buf ^= 1) {
+        const long long next = item + ctas_per_head;
+        // the other buffer was last read by the scatter of the item before this one, which ended with a barrier
+        if (next < n_items) fill_tables(next, buf ^ 1);
+        __syncthreads();
+        if (next < n_items) {
+            issue_loads(next, buf ^ 1);
+            cp_async_wait<1>();
+        } else {
+            cp_async_wait<0>();
+        }
+        __syncthreads();
+        const WindowRef r = window_ref(g, (int)(item % M));
+        const size_t sample_off = (size_t)(item / M) * g.H * g.W;
+        unsigned char* s_q = s_tiles + buf * BUF_BYTES;
+        const unsigned char* s_k = s_q + TILE_BYTES;
+        const unsigned char* s_v = s_q + 2 * TILE_BYTES;
+        const int* tokb = s_tok + buf * BN;
+        const int* metab = s_meta + buf * BN;
+
+        // S = Q K^T for the warp's 16 query rows
+        float acc_s[BN / 8][4];
+#pragma unroll
+        for (int i = 0; i < BN / 8; ++i)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc_s[i][e] = 0.f;
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+            uint32_t qf[4];
+            const int row = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+            ldmatrix_x4(qf, smem_u32(s_q + tile_off<D>(row, 2 * ks + (lane >> 4))));
+#pragma unroll
+            for (int np = 0; np < BN / 16; ++np) {
+                uint32_t bf[4];
+                const int key = np * 16 + (lane & 7) + (lane >> 4) * 8;
+                ldmatrix_x4(bf, smem_u32(s_k + tile_off<D>(key, 2 * ks + ((lane >> 3) & 1))));
+                mma_elem(acc_s[2 * np], qf, bf[0], bf[1]);
+                mma_elem(acc_s[2 * np + 1], qf, bf[2], bf[3]);
+            }
+        }
+        // scale + relative-position bias + shift mask, in the log2 domain; row maxima
+        const int meta_r[2] = {metab[warp * 16 + gq], metab[warp * 16 + gq + 8]};
+        float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+        for (int nt = 0; nt < BN / 8; ++nt) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int mj = metab[nt * 8 + 2 * tq + (e & 1)];
+                const int mi = meta_r[e >> 1];
+                const bool ok = meta_label(mi) == meta_label(mj);
+                float sc = acc_s[nt][e] * g.scale_log2e + s_bias[meta_code(mi) - meta_code(mj) + c0];
+                sc = ok ? sc : -INFINITY;
+                acc_s[nt][e] = sc;
+                mx[e >> 1] = fmaxf(mx[e >> 1], sc);
+            }
+        }
+        float m_use[2], l_row[2] = {0.f, 0.f};
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 1));
+            mx[h] = fmaxf(mx[h], __shfl_xor_sync(0xffffffffu, mx[h], 2));
+            m_use[h] = (mx[h] == -INFINITY) ? 0.f : mx[h];     // a row without a token sees no key
+        }
+#pragma unroll
+        for (int nt = 0; nt < BN / 8; ++nt) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float p = fast_exp2(acc_s[nt][e] - m_use[e >> 1]);
+                acc_s[nt][e] = p;
+                l_row[e >> 1] += p;
+            }
+        }
+        // O = P V
+        float acc_o[DT][4];
+#pragma unroll
+        for (int i = 0; i < DT; ++i)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc_o[i][e] = 0.f;
+#pragma unroll
+        for (int ks = 0; ks < BN / 16; ++ks) {
+            uint32_t pf[4];
+            pf[0] = pack_elem(acc_s[2 * ks][0], acc_s[2 * ks][1]);
+            pf[1] = pack_elem(acc_s[2 * ks][2], acc_s[2 * ks][3]);
+            pf[2] = pack_elem(acc_s[2 * ks + 1][0], acc_s[2 * ks + 1][1]);
+            pf[3] = pack_elem(acc_s[2 * ks + 1][2], acc_s[2 * ks + 1][3]);
+#pragma unroll
+            for (int dp = 0; dp < DT / 2; ++dp) {
+                uint32_t bf[4];
+                const int key = ks * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+                ldmatrix_x4_trans(bf, smem_u32(s_v + tile_off<D>(key, 2 * dp + (lane >> 4))));
+                mma_elem(acc_o[2 * dp], pf, bf[0], bf[1]);
+                mma_elem(acc_o[2 * dp + 1], pf, bf[2], bf[3]);
+            }
+        }
+        float inv[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            float l = l_row[h];
+            l += __shfl_xor_sync(0xffffffffu, l, 1);
+            l += __shfl_xor_sync(0xffffffffu, l, 2);
+            l_row[h] = l;
+            inv[h] = 1.f / l;
+        }
+        __syncthreads();   // every warp has read its Q fragments: the Q tile becomes the output tile
+#pragma unroll
+        for (int i = 0; i < DT; ++i) {
+            const int lr = warp * 16 + gq;
+            *reinterpret_cast<uint32_t*>(s_q + tile_off<D>(lr, i) + tq * 4) = pack_elem(acc_o[i][0] * inv[0], acc_o[i][1] * inv[0]);
+            *reinterpret_cast<uint32_t*>(s_q + tile_off<D>(lr + 8, i) + tq * 4) = pack_elem(acc_o[i][2] * inv[1], acc_o[i][3] * inv[1]);
+        }
+        if (tq == 0) {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int slot = warp * 16 + gq + 8 * h;
+                if (slot < r.n) lse[(sample_off + (size_t)tokb[slot]) * g.heads + head] = (mx[h] + log2f(l_row[h])) * kLn2;
+            }
+        }
+        __syncthreads();
+        constexpr int CPR = D / 8;
+        for (int idx = tid; idx < BM * CPR; idx += NTHREADS) {
+            const int row = idx / CPR, chunk = idx - row * CPR;
+            if (row < r.n) {
+                const uint4 val = *reinterpret_cast<const uint4*>(s_q + tile_off<D>(row, chunk));
+                *reinterpret_cast<uint4*>(o + ((sample_off + (size_t)tokb[row]) * g.heads + head) * D + chunk * 8) = val;
+            }
+        }
+        __syncthreads();   // the buffer's tiles and tables are free for the item after next
+    }
 }
 
 size_t fwd_smem_bytes(const Geo& g) {
@@ -291,12 +467,34 @@ size_t fwd_smem_bytes(const Geo& g) {
 
 cudaError_t TERRA_ELEM_FN(launch_fwd_mma)(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
                            void* o, float* lse, cudaStream_t stream) {
+    if (g.nmax <= BN && g.w <= 32) {
+        // windows of at most 64 tokens: the persistent double-buffered kernel
+        auto kern = g.d == 32 ? swin_fwd_small_kernel<32> : g.d == 64 ? swin_fwd_small_kernel<64> : swin_fwd_small_kernel<128>;
+        const int nbias = (2 * g.w - 1) * (2 * g.w - 1);
+        const size_t smem = (((size_t)BN * 16 + (size_t)nbias * 4 + 127) / 128) * 128 + 6 * (size_t)BN * g.d * 2;
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        int occ = 0, dev = 0, sms = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, NTHREADS, smem);
+        if (e == cudaSuccess) e = cudaGetDevice(&dev);
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        if (occ < 1) occ = 1;
+        const long long items = (long long)g.B * g.Mh * g.Mw;
+        long long cph = ((long long)sms * occ) / g.heads;
+        if (cph < 1) cph = 1;
+        if (cph > items) cph = items;
+        prof_begin("swin_fwd_small_kernel", stream);
+        kern<<<(unsigned)(cph * g.heads), NTHREADS, smem, stream>>>(g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k,
+                                                                   (const __nv_bfloat16*)v, bias, (__nv_bfloat16*)o, lse, (int)cph);
+        count_launch(stream);
+        return cudaGetLastError();
+    }
     const int qtiles = (g.nmax + BM - 1) / BM;
     const long long items = (long long)g.B * g.Mh * g.Mw * g.heads * qtiles;
     const size_t smem = fwd_smem_bytes(g);
     auto kern = g.w > 32 ? ((g.d == 32) ? swin_fwd_mma_kernel<32, true> : (g.d == 64) ? swin_fwd_mma_kernel<64, true> : swin_fwd_mma_kernel<128, true>)
-                         : ((g.d == 32) ? swin_fwd_mma_kernel<32, false> : (g.d == 64) ? swin_fwd_mma_kernel<64, false>
-                            : (g.nmax <= BN ? swin_fwd_mma_d128_small_kernel : swin_fwd_mma_kernel<128, false>));
+                         : ((g.d == 32) ? swin_fwd_mma_kernel<32, false> : (g.d == 64) ? swin_fwd_mma_kernel<64, false> : swin_fwd_mma_kernel<128, false>);
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     prof_begin("swin_fwd_mma_kernel", stream);
