@@ -433,6 +433,7 @@ def main():
         pairs = wk["score_elements"]
         d = cfg.head_dim
         kernel_flop = {"swin_fwd_tc_kernel": 4 * d * pairs, "swin_fwd_tc64_kernel": 4 * d * pairs, "swin_fwd_mma_kernel": 4 * d * pairs,
+                       "swin_fwd_small_kernel": 4 * d * pairs,
                        "swin_bwd_fused_kernel": 8 * d * pairs, "swin_bwd_small_kernel": 8 * d * pairs,
                        "swin_bwd_mma_kernel<key tiles>": 4 * d * pairs, "swin_bwd_mma_kernel<query tiles>": 4 * d * pairs,
                        "swin_bwd_kv64_kernel": 4 * d * pairs, "swin_bwd_q64_kernel": 4 * d * pairs,
