@@ -215,13 +215,13 @@ __device__ __forceinline__ void softmax_cols32_row(const uint32_t (&r)[32], uint
     bv[31] = lds_f32_at<0>(bb);
 #pragma unroll
     for (int e2 = 0; e2 < 16; ++e2) {
-        const float p0 = fast_exp2(fmaf(__uint_as_float(r[2 * e2]), scale, bv[2 * e2]) + neg_m);
-        const float p1 = fast_exp2(fmaf(__uint_as_float(r[2 * e2 + 1]), scale, bv[2 * e2 + 1]) + neg_m);
+        // two-wide fp32 operations: one instruction per pair of columns
+        float x0, x1;
+        fma2(x0, x1, __uint_as_float(r[2 * e2]), __uint_as_float(r[2 * e2 + 1]), scale, bv[2 * e2], bv[2 * e2 + 1]);
+        add2(x0, x1, x0, x1, neg_m);
+        const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
         pk[e2] = pack_elem(p0, p1);
-        if (SUM) {
-            sum[0] += p0;
-            sum[1] += p1;
-        }
+        if (SUM) add2vv(sum[0], sum[1], sum[0], sum[1], p0, p1);
     }
 }
 

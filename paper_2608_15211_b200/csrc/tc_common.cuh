@@ -302,6 +302,13 @@ __device__ __forceinline__ void add2(float& x0, float& x1, float a0, float a1, f
         "add.rn.f32x2 rd, ra, rb;\n\t"
         "mov.b64 {%0, %1}, rd;\n\t}\n" : "=f"(x0), "=f"(x1) : "f"(a0), "f"(a1), "f"(b));
 }
+// (x0, x1) = (a0, a1) + (b0, b1)
+__device__ __forceinline__ void add2vv(float& x0, float& x1, float a0, float a1, float b0, float b1) {
+    asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+        "add.rn.f32x2 rd, ra, rb;\n\t"
+        "mov.b64 {%0, %1}, rd;\n\t}\n" : "=f"(x0), "=f"(x1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+}
 // (x0, x1) = (a0, a1) - (b0, b1)
 __device__ __forceinline__ void sub2(float& x0, float& x1, float a0, float a1, float b0, float b1) {
     asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
