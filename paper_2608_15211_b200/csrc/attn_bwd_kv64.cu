@@ -179,13 +179,19 @@ __device__ __forceinline__ void cols16(const uint32_t (&rs)[16], const uint32_t 
     }
 #pragma unroll
     for (int e = 0; e < 16; ++e) bv[e] = ROW32 ? lds_f32(bias_row + code4 + 4 * e) : lds_f32(bias_row + co[e]);
+    // two-wide fp32 operations: one instruction per pair of columns
     float p[16], ds[16];
 #pragma unroll
-    for (int e = 0; e < 16; ++e) {
-        float xv = fmaf(-l2[e], kLog2e, fmaf(__uint_as_float(rs[e]), scale, bv[e]));
-        if (MASKED && ql[e] != klabel) xv = -INFINITY;
-        p[e] = fast_exp2(xv);
-        ds[e] = p[e] * (__uint_as_float(rp[e]) - dl[e]);
+    for (int e = 0; e < 16; e += 2) {
+        float x0, x1, t0, t1;
+        fma2(x0, x1, __uint_as_float(rs[e]), __uint_as_float(rs[e + 1]), scale, bv[e], bv[e + 1]);
+        fma2(x0, x1, l2[e], l2[e + 1], -kLog2e, x0, x1);
+        if (MASKED && ql[e] != klabel) x0 = -INFINITY;
+        if (MASKED && ql[e + 1] != klabel) x1 = -INFINITY;
+        p[e] = fast_exp2(x0);
+        p[e + 1] = fast_exp2(x1);
+        sub2(t0, t1, __uint_as_float(rp[e]), __uint_as_float(rp[e + 1]), dl[e], dl[e + 1]);
+        mul2(ds[e], ds[e + 1], p[e], p[e + 1], t0, t1);
     }
 #pragma unroll
     for (int e2 = 0; e2 < 8; ++e2) {

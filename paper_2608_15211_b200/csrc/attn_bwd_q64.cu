@@ -193,13 +193,18 @@ __device__ __forceinline__ void cols16(const uint32_t (&rs)[16], const uint32_t 
     }
 #pragma unroll
     for (int e = 0; e < 16; ++e) bv[e] = lds_f32(bias_grp - 4 * kCodeStride * e);
+    // two-wide fp32 operations: one instruction per pair of columns
     float ds[16];
 #pragma unroll
-    for (int e = 0; e < 16; ++e) {
-        float xv = fmaf(__uint_as_float(rs[e]), scale, bv[e]) - l2;
-        if (MASKED && kl[e] != qlabel) xv = -INFINITY;
-        const float p = fast_exp2(xv);
-        ds[e] = p * (__uint_as_float(rp[e]) - dl);
+    for (int e = 0; e < 16; e += 2) {
+        float x0, x1, t0, t1;
+        fma2(x0, x1, __uint_as_float(rs[e]), __uint_as_float(rs[e + 1]), scale, bv[e], bv[e + 1]);
+        add2(x0, x1, x0, x1, -l2);
+        if (MASKED && kl[e] != qlabel) x0 = -INFINITY;
+        if (MASKED && kl[e + 1] != qlabel) x1 = -INFINITY;
+        const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+        add2(t0, t1, __uint_as_float(rp[e]), __uint_as_float(rp[e + 1]), -dl);
+        mul2(ds[e], ds[e + 1], p0, p1, t0, t1);
     }
 #pragma unroll
     for (int e = 0; e < 16; ++e) tv[e] = lds_f32(tab + 256 * e);
