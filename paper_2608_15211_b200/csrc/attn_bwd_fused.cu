@@ -271,11 +271,19 @@ __device__ __forceinline__ void cols16(const uint32_t (&rs)[16], const uint32_t 
     }
     float p[16];
 #pragma unroll
+    for (int e = 0; e < 16; e += 2) {
+        float x0, x1, t0, t1;
+        fma2(x0, x1, __uint_as_float(rs[e]), __uint_as_float(rs[e + 1]), scale, bv[e], bv[e + 1]);
+        sub2(x0, x1, x0, x1, l2[e], l2[e + 1]);
+        if (MASKED && kl[e] != rc.label) x0 = -INFINITY;
+        if (MASKED && kl[e + 1] != rc.label) x1 = -INFINITY;
+        p[e] = fast_exp2(x0);
+        p[e + 1] = fast_exp2(x1);
+        sub2(t0, t1, __uint_as_float(rp[e]), __uint_as_float(rp[e + 1]), dl[e], dl[e + 1]);
+        mul2(ds[e], ds[e + 1], p[e], p[e + 1], t0, t1);
+    }
+#pragma unroll
     for (int e = 0; e < 16; ++e) {
-        float xv = fmaf(__uint_as_float(rs[e]), scale, bv[e]) - l2[e];
-        if (MASKED && kl[e] != rc.label) xv = -INFINITY;
-        p[e] = fast_exp2(xv);
-        ds[e] = p[e] * (__uint_as_float(rp[e]) - dl[e]);
         addr[e] = rc.dbias_row + co[e];
         if (RAGGED && (!rc.valid || l2[e] == INFINITY)) addr[e] = rc.scratch;
     }
@@ -307,12 +315,17 @@ __device__ __forceinline__ void load16_row(int c, int code0x4, const RowCtx& rc,
 }
 __device__ __forceinline__ void math16_row(const uint32_t (&rs)[16], const uint32_t (&rp)[16], const float (&bv)[16], const float (&l2)[16],
                                            const float (&dl)[16], float scale, uint32_t (&pk_p)[8], uint32_t (&pk_ds)[8], float (&ds)[16]) {
+    // two-wide fp32 operations: one instruction per pair of columns
     float p[16];
 #pragma unroll
-    for (int e = 0; e < 16; ++e) {
-        const float xv = fmaf(__uint_as_float(rs[e]), scale, bv[e]) - l2[e];
-        p[e] = fast_exp2(xv);
-        ds[e] = p[e] * (__uint_as_float(rp[e]) - dl[e]);
+    for (int e = 0; e < 16; e += 2) {
+        float x0, x1, t0, t1;
+        fma2(x0, x1, __uint_as_float(rs[e]), __uint_as_float(rs[e + 1]), scale, bv[e], bv[e + 1]);
+        sub2(x0, x1, x0, x1, l2[e], l2[e + 1]);
+        p[e] = fast_exp2(x0);
+        p[e + 1] = fast_exp2(x1);
+        sub2(t0, t1, __uint_as_float(rp[e]), __uint_as_float(rp[e + 1]), dl[e], dl[e + 1]);
+        mul2(ds[e], ds[e + 1], p[e], p[e + 1], t0, t1);
     }
 #pragma unroll
     for (int e2 = 0; e2 < 8; ++e2) {
