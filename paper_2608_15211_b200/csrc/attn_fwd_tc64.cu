@@ -150,13 +150,18 @@ __device__ __forceinline__ void softmax_cols(const uint32_t (&r)[N], uint32_t (&
             const int4 kl4 = lds_i4(a_klab + 4 * (c + e4 * 4));
             kl[0] = kl4.x; kl[1] = kl4.y; kl[2] = kl4.z; kl[3] = kl4.w;
         }
-        float p[4];
+        float p[4], bv[4];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const float bv = lds_f32(bias_i + kc[e]);
-            float xv = fmaf(__uint_as_float(r[e4 * 4 + e]), scale, bv) + neg_m;
-            if (MASKED && kl[e] != label_i) xv = -INFINITY;
-            p[e] = fast_exp2(xv);
+        for (int e = 0; e < 4; ++e) bv[e] = lds_f32(bias_i + kc[e]);
+#pragma unroll
+        for (int e = 0; e < 4; e += 2) {
+            float x0, x1;
+            fma2(x0, x1, __uint_as_float(r[e4 * 4 + e]), __uint_as_float(r[e4 * 4 + e + 1]), scale, bv[e], bv[e + 1]);
+            add2(x0, x1, x0, x1, neg_m);
+            if (MASKED && kl[e] != label_i) x0 = -INFINITY;
+            if (MASKED && kl[e + 1] != label_i) x1 = -INFINITY;
+            p[e] = fast_exp2(x0);
+            p[e + 1] = fast_exp2(x1);
         }
         pk[e4 * 2] = pack_elem(p[0], p[1]);
         pk[e4 * 2 + 1] = pack_elem(p[2], p[3]);
