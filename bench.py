@@ -209,6 +209,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-packed", action="store_true", help="skip the packed-QKV leg")
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp16"],
+                    help="element type of the activations and gradients (the benchmark's metric is quoted on bf16)")
     ap.add_argument("--rows", type=int, default=0,
                     help="profiling aid: keep the configuration but use this many token rows (a smaller case of the "
                          "same kernels for ncu captures); the JSON names the changed grid")
@@ -249,9 +251,10 @@ def main():
     peaks, peak_kind = load_peaks()
 
     # inputs resident in HBM (seeded device generators)
-    q, k, v, d_o = (make_activation(cfg, t, dev) for t in ("q", "k", "v", "do"))
+    act_dtype = torch.float16 if args.dtype == "fp16" else torch.bfloat16
+    q, k, v, d_o = (make_activation(cfg, t, dev).to(act_dtype) for t in ("q", "k", "v", "do"))
     bias = make_bias_table(cfg, dev)
-    desc = terra.make_desc(cfg)
+    desc = terra.make_desc(cfg, dtype=act_dtype)
     nt, nw, _ = terra.terra_route_sizes(desc)
     route = {n: torch.empty(nt, dtype=torch.int32, device=dev) for n in ("perm", "inv_perm", "pos", "label")}
     route["win_offsets"] = torch.empty(nw + 1, dtype=torch.int32, device=dev)
@@ -450,7 +453,7 @@ def main():
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "vs_baseline": None, "dtype": args.dtype, "data": "synthetic",
             "config": workload_config(cfg, "inputs exceed L2 (4 bf16 tensors of %.0f MB each)" % (wk["tensor_bytes"] / 1e6)),
             "tokens_per_s": world * cfg.tokens / (ms_step * 1e-3),
             "pct_of_bf16_peak": {"of_measured_burst": 100 * value / world / peaks["bf16_tflops"],
