@@ -1,5 +1,6 @@
-// Forward shifted-window attention on the tcgen05 tensor cores for head dims 64 and 128 and windows of up to 1024
-// tokens (window side <= 32): the large-window regime, where a score row no longer fits tensor memory.
+// Forward shifted-window attention on the tcgen05 tensor cores for head dims 64 and 128 in the large-window regime,
+// where a score row no longer fits tensor memory: windows of up to 1024 tokens (window side <= 32) on any grid, and
+// complete windows of side 64 and 128 (4096 and 16 384 tokens) whose rows the bulk-copy loader can fetch.
 //
 // One persistent CTA per SM, bound to one head, walks over (batch, window, pair of 128-row query tiles) items.
 // The window's keys are streamed once, in chunks of 128, through a ring of shared-memory slots.  Per chunk:
@@ -181,11 +182,8 @@ __device__ __forceinline__ float lds_f32_at(uint32_t addr) {
 // 32 key columns that are one window row of a full-width 32-wide window without mask labels: their bias entries are
 // consecutive (descending with the key), so each address is one base plus an immediate offset: no per-key offsets to
 // load, no address arithmetic.  `top` = shared address of the entry of the row's first key.
-template <bool SUM>
-__device__ __forceinline__ void softmax_cols32_row(const uint32_t (&r)[32], uint32_t (&pk)[16], uint32_t top, float scale, float neg_m,
-                                                   float (&sum)[2]) {
+__device__ __forceinline__ void load_bias_row32(float (&bv)[32], uint32_t top) {
     const uint32_t bb = top - 124;
-    float bv[32];
     bv[0] = lds_f32_at<124>(bb);
     bv[1] = lds_f32_at<120>(bb);
     bv[2] = lds_f32_at<116>(bb);
@@ -218,12 +216,25 @@ __device__ __forceinline__ void softmax_cols32_row(const uint32_t (&r)[32], uint
     bv[29] = lds_f32_at<8>(bb);
     bv[30] = lds_f32_at<4>(bb);
     bv[31] = lds_f32_at<0>(bb);
+}
+// MASKED: keys whose mask label (32 ints at shared address `a_klab`) differs from the row's give P = 0
+template <bool SUM, bool MASKED = false>
+__device__ __forceinline__ void softmax_cols32_row(const uint32_t (&r)[32], uint32_t (&pk)[16], uint32_t top, float scale, float neg_m,
+                                                   float (&sum)[2], uint32_t a_klab = 0, int label_i = 0) {
+    float bv[32];
+    load_bias_row32(bv, top);
 #pragma unroll
     for (int e2 = 0; e2 < 16; ++e2) {
         // two-wide fp32 operations: one instruction per pair of columns
         float x0, x1;
         fma2(x0, x1, __uint_as_float(r[2 * e2]), __uint_as_float(r[2 * e2 + 1]), scale, bv[2 * e2], bv[2 * e2 + 1]);
         add2(x0, x1, x0, x1, neg_m);
+        if (MASKED) {
+            int kl0, kl1;
+            asm volatile("ld.shared.v2.s32 {%0,%1}, [%2];\n" : "=r"(kl0), "=r"(kl1) : "r"(a_klab + 8 * e2));
+            if (kl0 != label_i) x0 = -INFINITY;
+            if (kl1 != label_i) x1 = -INFINITY;
+        }
         const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
         pk[e2] = pack_elem(p0, p1);
         if (SUM) add2vv(sum[0], sum[1], sum[0], sum[1], p0, p1);
@@ -244,6 +255,24 @@ __device__ __forceinline__ float score_max_cols(const uint32_t* r, int c, uint32
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             const float xv = fmaf(__uint_as_float(r[e4 * 4 + e]), scale, lds_f32(bias_i + kc[e]));
+            mx = fmaxf(mx, kl[e] == label_i ? xv : -INFINITY);
+        }
+    }
+    return mx;
+}
+
+// the same for 32 key columns whose bias entries are consecutive (see softmax_cols32_row)
+__device__ __forceinline__ float score_max_cols32_row(const uint32_t (&r)[32], uint32_t top, uint32_t a_klab, int label_i, float scale,
+                                                      float mx) {
+    float bv[32];
+    load_bias_row32(bv, top);
+#pragma unroll
+    for (int e4 = 0; e4 < 8; ++e4) {
+        const int4 kl4 = lds_i4(a_klab + 16 * e4);
+        const int kl[4] = {kl4.x, kl4.y, kl4.z, kl4.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float xv = fmaf(__uint_as_float(r[e4 * 4 + e]), scale, bv[e4 * 4 + e]);
             mx = fmaxf(mx, kl[e] == label_i ? xv : -INFINITY);
         }
     }
@@ -280,13 +309,23 @@ struct FwdMaps64 {
 // TMA: the grid consists of complete windows of side 16 or 32 and the longitude shift is a multiple of 8: a window row
 // is then one run of tokens (two where it wraps around the longitude seam), and one loader warp fetches every row with
 // tiled bulk copies; otherwise three loader warps gather the rows with 16-byte cp.async copies.
-template <int D, bool TMA>
+//
+// MODE 0: gathered rows.  MODE 1: bulk-copied Q and K rows, window side 16 or 32, the head's whole bias table in
+// shared memory.  MODE 2: bulk-copied rows, window side 64 or 128 (complete windows of 4096 or 16384 tokens): the bias
+// table no longer fits, and the bulk-copy warp stages, per chunk and query tile, the table rows the tile's rows need.
+// A chunk's 128 keys are kr = 128 / w window rows and a tile's 128 queries qr = kr window rows, so the row offsets
+// between them span 2 kr - 1 table rows; in the prepared layout (2 w floats per table row) those are one contiguous
+// block, and within a 32-key group the entries a query row needs are consecutive, as in the 32-wide case.
+template <int D, int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
 swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                      const __nv_bfloat16* __restrict__ v, const float* __restrict__ bias_prep,
                      __nv_bfloat16* __restrict__ o, float* __restrict__ lse, long long n_items, int ctas_per_head,
                      int max_pairs, const __grid_constant__ FwdMaps64 maps) {
     using L = Lay<D>;
+    constexpr bool TMA = MODE >= 1, ROWS = MODE == 2;
+    constexpr int kStageBytes = 4096, kStageTile = 1536;      // MODE 2: ring of four bias stages, two tiles each
+    static_assert(4 * kStageBytes <= (kBiasFloats - 1) * 4, "bias stages lie below the table's last float");
     constexpr int kParts = L::kParts, kQStages = L::kQStages, kSlots = L::kSlots, kQStageBytes = L::kQStageBytes;
     constexpr int kOffK = L::kOffK, kOffV = L::kOffV, kSlotBytes = L::kSlotBytes, kOffSlots = L::kOffSlots;
     constexpr int kOffKeyMeta = L::kOffKeyMeta, kOffRowMeta = L::kOffRowMeta, kOffBias = L::kOffBias, kOffBars = L::kOffBars;
@@ -337,8 +376,14 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
         fence_barrier_init();
     }
     // the head's prepared bias table; the ones block of every ring slot (first 16 bf16 of a row = 1)
-    for (int i = tid; i < kBiasFloats; i += kThreads)
-        reinterpret_cast<float*>(smem + kOffBias)[i] = bias_prep[(size_t)head * kBiasFloats + i];
+    const int lw = 31 - __clz(g.w);                         // MODE 2: w = 1 << lw
+    const int rows_floats = (2 * g.w - 1) * 2 * g.w + 4;    // MODE 2: floats of one head's prepared table
+    if (ROWS) {
+        if (tid == 0) reinterpret_cast<float*>(smem + kOffBias)[kBiasFloats - 1] = bias_prep[(size_t)(head + 1) * rows_floats - 1];
+    } else {
+        for (int i = tid; i < kBiasFloats; i += kThreads)
+            reinterpret_cast<float*>(smem + kOffBias)[i] = bias_prep[(size_t)head * kBiasFloats + i];
+    }
     if (L::kOnes) {
         for (int i = tid; i < kSlots * kChunk * 4; i += kThreads) {
             const int s = i / (kChunk * 4), rem = i - s * (kChunk * 4), row = rem >> 2, chunk = rem & 3;
@@ -437,6 +482,14 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                                 klab[row] = label;
                             }
                         }
+                        if (ROWS && lane < x.ntiles) {
+                            // the 2 kr - 1 table rows that tile `lane` of the pair needs against this chunk
+                            const int kr = kChunk >> lw;
+                            const int r0 = (((x.pair * kQRows + lane * 128) >> lw) - c * kr - (kr - 1)) + g.w - 1;
+                            bulk_load(smem0 + kOffBias + (int)(ru & 3) * kStageBytes + lane * kStageTile,
+                                      bias_prep + (size_t)head * rows_floats + (size_t)r0 * 2 * g.w, (uint32_t)((2 * kr - 1) * 8 * g.w),
+                                      bar_kfull(s));
+                        }
                         // K rows (the V rows are gathered by the other two loader warps: the bulk-copy
                         // engine takes a fixed time per 64-byte row, and the two ways of loading run side by side)
                         const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes;
@@ -445,7 +498,8 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                             copy_row(maps.k, sb + kOffK + part * kKPart + ar * g.w * kPartBytes, c * wrows + ar, part, bar_kfull(s));
                         }
                         __syncwarp();
-                        if (lane == 0) mbar_arrive_expect_tx(bar_kfull(s), (uint32_t)(kChunk * D * 2));
+                        if (lane == 0)
+                            mbar_arrive_expect_tx(bar_kfull(s), (uint32_t)(kChunk * D * 2 + (ROWS ? x.ntiles * (2 * (kChunk >> lw) - 1) * 8 * g.w : 0)));
                         else mbar_arrive(bar_kfull(s));
                     }
                 }
@@ -737,6 +791,14 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             const bool row32 = g.w == 32 && x.r.ew == 32 && !x.masked;       // then every key slot holds a token, too
             const bool exact = exact_max(x);
             bool ok = true;
+            // MODE 2: this row's window row within its tile, and the byte offset of its entry for key column 0 of a table row
+            const int slot_q = x.pair * kQRows + wg * 128 + row;
+            const int aq_l = (slot_q >> lw) - ((x.pair * kQRows + wg * 128) >> lw), kr = kChunk >> lw;
+            const int colq = 4 * ((slot_q & (g.w - 1)) + g.w - 1);
+            // shared address of the entry of this row for the first key of 32-column group i, in a stage at `stage`
+            auto row_top = [&](uint32_t stage, int i) -> uint32_t {
+                return stage + wg * kStageTile + (aq_l - ((32 * i) >> lw) + kr - 1) * 8 * g.w + colq - 4 * ((32 * i) & (g.w - 1));
+            };
             // Online softmax, chunk by chunk: P is formed against a reference m that is at least the row's maximum so
             // far minus 8 octaves; only when a chunk's maximum exceeds the reference by more than that is the reference
             // raised and the accumulated O (with the row sum) scaled down by 2^(old - new).  Without mask labels the
@@ -748,6 +810,7 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             for (int c = 0; c < x.nch; ++c) {
                 const int ncols = min(kChunk, x.npad - c * kChunk);
                 const uint32_t a_kc = smem0 + kOffKeyMeta + (int)((ru0 + c) & 3) * 1024, a_klab = a_kc + 512;
+                const uint32_t stage = smem0 + kOffBias + (int)((ru0 + c) & 3) * kStageBytes;
                 ok = mbar_wait_all(bar_sready(wg), n_s & 1, cta_abort);
                 if (!ok) break;
                 ++n_s;
@@ -762,7 +825,8 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                         for (; cc + 32 <= ncols; cc += 32) {
                             tmem_ld32(t_s + cc, ra);
                             tmem_ld_wait();
-                            mxe = score_max_cols<32>(ra, cc, bias_i, a_kc, a_klab, label_i, scale, mxe);
+                            if (ROWS) mxe = score_max_cols32_row(ra, row_top(stage, cc >> 5), a_klab + 4 * cc, label_i, scale, mxe);
+                            else mxe = score_max_cols<32>(ra, cc, bias_i, a_kc, a_klab, label_i, scale, mxe);
                         }
                         if (cc < ncols) {
                             uint32_t rt[16];
@@ -825,14 +889,20 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                     uint32_t pk[16];
                     tmem_ld_wait();
                     if (i + 1 < nfull) tmem_ld32(t_s + 32 * (i + 1), rb);
-                    if (row32) softmax_cols32_row<kSum>(ra, pk, top_c - 4 * i * cs, scale, neg_m, psum);
+                    if (ROWS) {
+                        if (x.masked) softmax_cols32_row<kSum, true>(ra, pk, row_top(stage, i), scale, neg_m, psum, a_klab + 128 * i, label_i);
+                        else softmax_cols32_row<kSum>(ra, pk, row_top(stage, i), scale, neg_m, psum);
+                    } else if (row32) softmax_cols32_row<kSum>(ra, pk, top_c - 4 * i * cs, scale, neg_m, psum);
                     else if (x.masked) softmax_cols<32, true, kSum>(ra, pk, 32 * i, bias_i, a_kc, a_klab, label_i, scale, neg_m, psum);
                     else softmax_cols<32, false, kSum>(ra, pk, 32 * i, bias_i, a_kc, a_klab, label_i, scale, neg_m, psum);
                     tmem_st16(t_s + 16 * i, pk);
                     if (i + 1 < nfull) {
                         tmem_ld_wait();
                         if (i + 2 < nfull) tmem_ld32(t_s + 32 * (i + 2), ra);
-                        if (row32) softmax_cols32_row<kSum>(rb, pk, top_c - 4 * (i + 1) * cs, scale, neg_m, psum);
+                        if (ROWS) {
+                            if (x.masked) softmax_cols32_row<kSum, true>(rb, pk, row_top(stage, i + 1), scale, neg_m, psum, a_klab + 128 * (i + 1), label_i);
+                            else softmax_cols32_row<kSum>(rb, pk, row_top(stage, i + 1), scale, neg_m, psum);
+                        } else if (row32) softmax_cols32_row<kSum>(rb, pk, top_c - 4 * (i + 1) * cs, scale, neg_m, psum);
                         else if (x.masked) softmax_cols<32, true, kSum>(rb, pk, 32 * (i + 1), bias_i, a_kc, a_klab, label_i, scale, neg_m, psum);
                         else softmax_cols<32, false, kSum>(rb, pk, 32 * (i + 1), bias_i, a_kc, a_klab, label_i, scale, neg_m, psum);
                         tmem_st16(t_s + 16 * (i + 1), pk);
@@ -911,16 +981,19 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
 //   table[(da + w - 1) * cs + (db + w - 1)] = T[(da + w - 1) * (2w - 1) + (db + w - 1), head] * log2(e)   (cs = w + 32),
 //   table[2 c0 + 1 .. 3 c0 + 1] = -inf (where key slots without a token point), the head's largest entry in the last float
 //   (+inf instead if the head's entries spread over more than 64 octaves).
+// Window sides 64 and 128 (`rows`): per head (2w - 1) table rows of 2w floats (the last one padding) and four more
+// floats, the last of which is the head's largest entry as above.
 __global__ void __launch_bounds__(256)
-swin_fwd_bias_prep64_kernel(const float* __restrict__ bias, float* __restrict__ prep, int w, int heads) {
+swin_fwd_bias_prep64_kernel(const float* __restrict__ bias, float* __restrict__ prep, int w, int heads, int rows) {
     const int head = blockIdx.x;
-    const int cs = w + 32, nw = 2 * w - 1;
+    const int cs = rows ? 2 * w : w + 32, nw = 2 * w - 1;
     const int c0 = (w - 1) * (cs + 1);
-    float* dst = prep + (size_t)head * kBiasFloats;
+    const int total = rows ? nw * cs + 4 : kBiasFloats;
+    float* dst = prep + (size_t)head * total;
     float mx = -INFINITY, mn = INFINITY;
-    for (int e = threadIdx.x; e < kBiasFloats - 1; e += blockDim.x) {
+    for (int e = threadIdx.x; e < total - 1; e += blockDim.x) {
         float val = 0.f;
-        if (e > 2 * c0) {
+        if (!rows && e > 2 * c0) {
             val = -INFINITY;
         } else {
             const int ra = e / cs, rb = e - ra * cs;
@@ -944,7 +1017,7 @@ swin_fwd_bias_prep64_kernel(const float* __restrict__ bias, float* __restrict__ 
         for (int i = 1; i < 8; ++i) { mx = fmaxf(mx, red[i]); mn = fminf(mn, red_mn[i]); }
         // a table that spreads over more than 64 octaves makes the bound max(raw) * scale + max(bias) on the row
         // maximum too loose for the exponent range: +inf here tells the forward kernel to take exact row maxima
-        dst[kBiasFloats - 1] = (mx - mn <= 64.f) ? mx : INFINITY;
+        dst[total - 1] = (mx - mn <= 64.f) ? mx : INFINITY;
     }
 }
 
@@ -961,20 +1034,29 @@ cudaError_t read_fwd_tc64_status(int* timed_out) {
 #ifndef TERRA_ELEM_F16
 // prepared bias tables (kBiasFloats = 6048 floats per head) for the kernels of the head-dim-64 regime
 cudaError_t launch_bias_prep64(const Geo& g, const float* bias, float* prep, cudaStream_t stream) {
-    swin_fwd_bias_prep64_kernel<<<g.heads, 256, 0, stream>>>(bias, prep, g.w, g.heads);
+    swin_fwd_bias_prep64_kernel<<<g.heads, 256, 0, stream>>>(bias, prep, g.w, g.heads, 0);
     count_launch(stream);
     return cudaGetLastError();
 }
 
-bool fwd_tc64_supported(const Geo& g) { return (g.d == 64 || g.d == 128) && g.w <= 32 && g.nmax <= 1024 && g.heads <= 148; }
+// window sides up to 32 on any grid; sides 64 and 128 on grids of complete windows that the bulk-copy loaders serve
+bool fwd_tc64_supported(const Geo& g) {
+    if (!(g.d == 64 || g.d == 128) || g.heads > 148) return false;
+    if (g.w <= 32) return g.nmax <= 1024;
+    return (g.w == 64 || g.w == 128) && bulk_rows_shape(g);
+}
 
-size_t fwd_tc64_workspace_bytes(const Geo& g) { return (size_t)g.heads * kBiasFloats * sizeof(float); }
+size_t fwd_tc64_workspace_bytes(const Geo& g) {
+    const size_t per_head = g.w <= 32 ? (size_t)kBiasFloats : (size_t)(2 * g.w - 1) * 2 * g.w + 4;
+    return (size_t)g.heads * per_head * sizeof(float);
+}
 #endif  // !TERRA_ELEM_F16
 
 cudaError_t launch_fwd_tc64(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
                             void* o, float* lse, void* workspace, int sm_count, cudaStream_t stream) {
     float* prep = reinterpret_cast<float*>(workspace);
-    swin_fwd_bias_prep64_kernel<<<g.heads, 256, 0, stream>>>(bias, prep, g.w, g.heads);
+    const bool rows = g.w > 32;
+    swin_fwd_bias_prep64_kernel<<<g.heads, 256, 0, stream>>>(bias, prep, g.w, g.heads, rows ? 1 : 0);
     count_launch(stream);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
@@ -987,10 +1069,11 @@ cudaError_t launch_fwd_tc64(const Geo& g, const void* q, const void* k, const vo
     FwdMaps64 maps;
     std::memset(&maps, 0, sizeof maps);
     static const bool tma_off = [] { const char* e_ = std::getenv("TERRA_NO_TMA"); return e_ && e_[0] == '1'; }();
-    const bool tma = !tma_off && bulk_rows_shape(g) && make_row_maps3(&maps.q, g, q, g.ts) && make_row_maps3(&maps.k, g, k, g.ts) &&
+    const bool tma = (!tma_off || rows) && bulk_rows_shape(g) && make_row_maps3(&maps.q, g, q, g.ts) && make_row_maps3(&maps.k, g, k, g.ts) &&
                      make_row_maps3(&maps.v, g, v, g.ts);
-    auto kern = g.d == 64 ? (tma ? swin_fwd_tc64_kernel<64, true> : swin_fwd_tc64_kernel<64, false>)
-                          : (tma ? swin_fwd_tc64_kernel<128, true> : swin_fwd_tc64_kernel<128, false>);
+    if (rows && !tma) return cudaErrorNotSupported;       // windows of side 64 and 128 have no gathering loader
+    auto kern = g.d == 64 ? (rows ? swin_fwd_tc64_kernel<64, 2> : tma ? swin_fwd_tc64_kernel<64, 1> : swin_fwd_tc64_kernel<64, 0>)
+                          : (rows ? swin_fwd_tc64_kernel<128, 2> : tma ? swin_fwd_tc64_kernel<128, 1> : swin_fwd_tc64_kernel<128, 0>);
     const int smem_bytes = g.d == 64 ? Lay<64>::kSmemBytes : Lay<128>::kSmemBytes;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
     if (e != cudaSuccess) return e;

@@ -3,7 +3,7 @@
 // On a grid of complete windows whose longitude shift is a multiple of 8, the tokens of one window row are one run of
 // consecutive tokens of the tensor, or two where the rolled row crosses the longitude seam, each a multiple of 8 long.
 // A tensor is described as [tokens, heads * d] with boxes of 32 columns (one 64-byte-swizzled part of a row) by 32,
-// 16 or 8 tokens; a run is covered by at most one box of each size.
+// 16 or 8 tokens; a run is covered by boxes of 32 and at most one box of each smaller size.
 #pragma once
 #include <cuda.h>
 
@@ -25,7 +25,7 @@ bool make_col_map(CUtensorMap* map, const Geo& g, const void* base, int token_st
 
 // host: the geometry the bulk-copy loaders are written for
 inline bool bulk_rows_shape(const Geo& g) {
-    return (g.w == 16 || g.w == 32) && g.H % g.w == 0 && g.W % g.w == 0 && g.sw % 8 == 0 &&
+    return (g.w == 16 || g.w == 32 || g.w == 64 || g.w == 128) && g.H % g.w == 0 && g.W % g.w == 0 && g.sw % 8 == 0 &&
            (long long)g.B * g.H * g.W < 0x7fffffffLL;
 }
 
@@ -41,7 +41,7 @@ __device__ __forceinline__ void bulk_copy_window_row(const RowMaps3& m3, uint32_
     int y = y0 + v0, n = n1;
 #pragma unroll
     for (int seg = 0; seg < 2; ++seg) {
-        if (n >= 32) { tc::tma_load_2d(dst, &m3.m[0], xc, y, bar); dst += 32 * 64; y += 32; n -= 32; }
+        while (n >= 32) { tc::tma_load_2d(dst, &m3.m[0], xc, y, bar); dst += 32 * 64; y += 32; n -= 32; }
         if (n >= 16) { tc::tma_load_2d(dst, &m3.m[1], xc, y, bar); dst += 16 * 64; y += 16; n -= 16; }
         if (n >= 8) { tc::tma_load_2d(dst, &m3.m[2], xc, y, bar); dst += 8 * 64; }
         y = y0;

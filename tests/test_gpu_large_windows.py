@@ -14,6 +14,11 @@ SHAPES = [
     ("w40_d32", 2, 50, 90, 2, 32, 40, 20, 20, 0, 1),                 # a side that is no multiple of 32
     ("w128_d32", 1, 130, 140, 1, 32, 128, 64, 64, 0, 1),             # one complete 128 x 128 window and three truncated ones
     ("w128_d128_one_window", 1, 128, 128, 1, 128, 128, 0, 0, 1, 1),  # 16 384 tokens, head dim 128
+    # complete windows with a longitude shift that is a multiple of 8: the forward kernel that stages bias-table rows
+    ("w64_d64_complete", 1, 128, 192, 2, 64, 64, 32, 40, 0, 1),      # latitude mask, rows that wrap around the seam
+    ("w64_d128_complete", 2, 64, 128, 2, 128, 64, 16, 8, 0, 0),      # masks on both axes
+    ("w128_d64_complete", 1, 128, 128, 2, 64, 128, 40, 16, 0, 0),
+    ("w128_d128_masked", 1, 128, 256, 1, 128, 128, 64, 72, 0, 1),    # two windows, latitude mask, seam
 ]
 
 
