@@ -221,7 +221,13 @@ struct KvMaps64 {
 // window row with tiled bulk copies (per-query lse and delta by 4-byte cp.async copies tied to the same barrier);
 // otherwise three loader warps gather the rows with 16-byte cp.async copies.  (Gathering the dO rows with the two
 // idle warps next to the bulk copies, as the forward kernel does with V, was measured and is slightly slower here.)
-template <int D, bool TMA>
+//
+// MODE 0: gathered rows.  MODE 1: bulk-copied rows, window side 16 or 32, the head's whole bias table in shared memory.
+// MODE 2: bulk-copied rows, complete windows of side 64 or 128: the table does not fit, and the loader warp stages,
+// with every query chunk, the 2 kr - 1 table rows (kr = 128 / w window rows per 128 slots) that the chunk's queries
+// need against the item's key tile; in the prepared layout (2 w floats per table row) they are one contiguous block,
+// and the 16 queries of a column group read consecutive entries, as in the 32-wide case.
+template <int D, int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
 swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                      const __nv_bfloat16* __restrict__ v, const __nv_bfloat16* __restrict__ d_o,
@@ -229,6 +235,8 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                      __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv, long long n_items, int ctas_per_head,
                      int max_tiles, const __grid_constant__ KvMaps64 maps) {
     using L = Lay<D>;
+    constexpr bool TMA = MODE >= 1, ROWS = MODE == 2;
+    constexpr int kStageBytes = 1536;                 // MODE 2: the staged table rows of one query slot
     constexpr int kParts = L::kParts, kKvStages = L::kKvStages, kSlots = L::kSlots;
     constexpr int kOffK = L::kOffK, kOffV = L::kOffV, kOffKCode = L::kOffKCode, kOffKLab = L::kOffKLab, kOffKTok = L::kOffKTok;
     constexpr int kKvStageBytes = L::kKvStageBytes, kOffQ = L::kOffQ, kOffG = L::kOffG, kOffQCode = L::kOffQCode;
@@ -276,8 +284,10 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
         *cta_abort = 0;
         fence_barrier_init();
     }
-    for (int i = tid; i < kBiasFloats; i += kThreads)
-        reinterpret_cast<float*>(smem + kOffBias)[i] = bias_prep[(size_t)head * kBiasFloats + i];
+    if (!ROWS) {
+        for (int i = tid; i < kBiasFloats; i += kThreads)
+            reinterpret_cast<float*>(smem + kOffBias)[i] = bias_prep[(size_t)head * kBiasFloats + i];
+    }
     fence_proxy_async();
     if (warp == kMmaWarp) {
         tmem_alloc(smem_u32(tmem_slot), 512);
@@ -360,6 +370,14 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                         const int ar = rem / kParts, part = rem - ar * kParts;
                         bulk_copy_window_row(tsr ? maps.g : maps.q, sb + (tsr ? kOffG : kOffQ) + part * kPart + ar * g.w * kPartBytes, g,
                                              x.b, x.r.wr, v0, c * wrows + ar, head * D + part * 32, bar_qfull(s));
+                    }
+                    if (ROWS && lane == 0) {
+                        const int lw = 31 - __clz(g.w), kr = kTile >> lw;
+                        const int r0 = (c - x.kt) * kr - (kr - 1) + g.w - 1;
+                        bulk_load(smem0 + kOffBias + s * kStageBytes,
+                                  bias_prep + (size_t)head * ((2 * g.w - 1) * 2 * g.w + 4) + (size_t)r0 * 2 * g.w,
+                                  (uint32_t)((2 * kr - 1) * 8 * g.w), bar_qfull(s));
+                        mbar_expect_tx(bar_qfull(s), (uint32_t)((2 * kr - 1) * 8 * g.w));
                     }
                     if (lane == 0) mbar_expect_tx(bar_qfull(s), (uint32_t)(kTile * D * 2 * 2));
                     // the lane's arrival: when its lse / delta copies have landed (its table entries were written before)
@@ -629,8 +647,14 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             const int ktok = lds_i32(st_a + kOffKTok + 4 * krow);
             mbar_arrive(bar_kvempty(ks));                 // this thread has what it needs from the key stage
             // bias index = code_query - code_key + c0; a key row without a token reads the table's -inf zone
-            const uint32_t bias_row = smem0 + kOffBias + (ktok >= 0 ? 4 * c0 - kcode4 : 4 * (2 * c0 + 1));
-            const bool row32 = x.r.ew == 32;
+            uint32_t bias_row = smem0 + kOffBias + (ktok >= 0 ? 4 * c0 - kcode4 : 4 * (2 * c0 + 1));
+            const bool row32 = ROWS || x.r.ew == 32;
+            const int lw = 31 - __clz(g.w);
+            if (ROWS) {
+                // relative to a slot's stage: this key's window row within the tile and its column
+                const int kslot = x.kt * kTile + krow, kr = kTile >> lw;
+                bias_row = smem0 + kOffBias + (kr - 1 - ((kslot >> lw) - ((x.kt * kTile) >> lw))) * 8 * g.w + 4 * (g.w - 1 - (kslot & (g.w - 1)));
+            }
             for (int c = 0; c < x.nch && ok; ++c, ++ru) {
                 const int s = (int)(ru % kSlots);
                 const uint32_t sl_a = smem0 + kOffSlots + s * kSlotBytes + kOffQCode;      // the slot's per-query tables
@@ -645,7 +669,10 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                 const uint32_t t_s = tmem_base + lane_addr + kBufCols * buf - 64 * hcol, t_dp = t_s + 64;
                 const int col_end = min(ncols, 64 * hcol + 64);
                 // 4 * bias code of query column `col` of this chunk in a 32-wide window: slot = 128 c + col = 32 a + b
-                auto code4_of = [&](int col) { return 4 * ((4 * c + (col >> 5)) * cs + (col & 31)); };
+                // (MODE 2: the offset into the slot's staged table rows)
+                auto code4_of = [&](int col) {
+                    return ROWS ? s * kStageBytes + (col >> lw) * 8 * g.w + 4 * (col & (g.w - 1)) : 4 * ((4 * c + (col >> 5)) * cs + (col & 31));
+                };
                 // groups of 16 columns; the next group's S^T / dP^T travel from TMEM while this one is worked on
                 uint32_t rs[16], rp[16], rs2[16], rp2[16], pk_p[8], pk_ds[8];
                 if (64 * hcol < col_end) {
@@ -658,7 +685,8 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                         tmem_ld16(t_s + cc + 16, rs2);
                         tmem_ld16(t_dp + cc + 16, rp2);
                     }
-                    if (x.masked) cols16<true>(rs, rp, cc, bias_row, klabel, sl_a, scale, pk_p, pk_ds);
+                    if (ROWS && x.masked) cols16<true, true>(rs, rp, cc, bias_row, klabel, sl_a, scale, pk_p, pk_ds, code4_of(cc));
+                    else if (x.masked) cols16<true>(rs, rp, cc, bias_row, klabel, sl_a, scale, pk_p, pk_ds);
                     else if (row32) cols16<false, true>(rs, rp, cc, bias_row, klabel, sl_a, scale, pk_p, pk_ds, code4_of(cc));
                     else cols16<false>(rs, rp, cc, bias_row, klabel, sl_a, scale, pk_p, pk_ds);
                     tmem_st8(t_s + cc, pk_p);              // 16 queries -> 8 packed columns at the group's own place
@@ -669,7 +697,8 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                             tmem_ld16(t_s + cc + 32, rs);
                             tmem_ld16(t_dp + cc + 32, rp);
                         }
-                        if (x.masked) cols16<true>(rs2, rp2, cc + 16, bias_row, klabel, sl_a, scale, pk_p, pk_ds);
+                        if (ROWS && x.masked) cols16<true, true>(rs2, rp2, cc + 16, bias_row, klabel, sl_a, scale, pk_p, pk_ds, code4_of(cc + 16));
+                        else if (x.masked) cols16<true>(rs2, rp2, cc + 16, bias_row, klabel, sl_a, scale, pk_p, pk_ds);
                         else if (row32) cols16<false, true>(rs2, rp2, cc + 16, bias_row, klabel, sl_a, scale, pk_p, pk_ds, code4_of(cc + 16));
                         else cols16<false>(rs2, rp2, cc + 16, bias_row, klabel, sl_a, scale, pk_p, pk_ds);
                         tmem_st8(t_s + cc + 16, pk_p);
@@ -734,10 +763,16 @@ bool no_tma_env() {
 }  // namespace
 
 #ifndef TERRA_ELEM_F16
-bool bwd_kv64_supported(const Geo& g) { return (g.d == 64 || g.d == 128) && g.w <= 32 && g.nmax <= 1024 && g.heads <= 148; }
+// window sides up to 32 on any grid; sides 64 and 128 on grids of complete windows that the bulk-copy loader serves
+bool bwd_kv64_supported(const Geo& g) {
+    if (!(g.d == 64 || g.d == 128) || g.heads > 148) return false;
+    if (g.w <= 32) return g.nmax <= 1024;
+    return (g.w == 64 || g.w == 128) && bulk_rows_shape(g);
+}
 #endif  // !TERRA_ELEM_F16
 
-// `prep` = the prepared bias tables of the head-dim-64 forward kernel (kBiasFloats per head), filled by the caller
+// `prep` = the prepared bias tables of the head-dim-64 forward kernel (kBiasFloats per head; for window sides 64 and
+// 128 its layout of whole table rows), filled by the caller
 cudaError_t launch_bwd_kv64(const Geo& g, const void* q, const void* k, const void* v, const void* d_o, const float* prep,
                             const float* lse, const float* delta, void* dk, void* dv, int sm_count, cudaStream_t stream) {
     const int max_tiles = (g.nmax + 127) >> 7;
@@ -747,10 +782,12 @@ cudaError_t launch_bwd_kv64(const Geo& g, const void* q, const void* k, const vo
     if (cph > items) cph = items;
     KvMaps64 maps;
     std::memset(&maps, 0, sizeof maps);
-    const bool tma = !no_tma_env() && bulk_rows_shape(g) && make_row_maps3(&maps.q, g, q, g.ts) && make_row_maps3(&maps.k, g, k, g.ts) &&
+    const bool rows = g.w > 32;
+    const bool tma = (!no_tma_env() || rows) && bulk_rows_shape(g) && make_row_maps3(&maps.q, g, q, g.ts) && make_row_maps3(&maps.k, g, k, g.ts) &&
                      make_row_maps3(&maps.v, g, v, g.ts) && make_row_maps3(&maps.g, g, d_o, g.heads * g.d);
-    auto kern = g.d == 64 ? (tma ? swin_bwd_kv64_kernel<64, true> : swin_bwd_kv64_kernel<64, false>)
-                          : (tma ? swin_bwd_kv64_kernel<128, true> : swin_bwd_kv64_kernel<128, false>);
+    if (rows && !tma) return cudaErrorNotSupported;       // windows of side 64 and 128 have no gathering loader
+    auto kern = g.d == 64 ? (rows ? swin_bwd_kv64_kernel<64, 2> : tma ? swin_bwd_kv64_kernel<64, 1> : swin_bwd_kv64_kernel<64, 0>)
+                          : (rows ? swin_bwd_kv64_kernel<128, 2> : tma ? swin_bwd_kv64_kernel<128, 1> : swin_bwd_kv64_kernel<128, 0>);
     const int smem_bytes = g.d == 64 ? Lay<64>::kSmemBytes : Lay<128>::kSmemBytes;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
     if (e != cudaSuccess) return e;

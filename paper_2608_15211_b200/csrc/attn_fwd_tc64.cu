@@ -1032,9 +1032,10 @@ cudaError_t read_fwd_tc64_status(int* timed_out) {
 }
 
 #ifndef TERRA_ELEM_F16
-// prepared bias tables (kBiasFloats = 6048 floats per head) for the kernels of the head-dim-64 regime
+// prepared bias tables for the kernels of the large-window regime: kBiasFloats = 6048 floats per head for window
+// sides up to 32, whole table rows for sides 64 and 128 (see the kernel above)
 cudaError_t launch_bias_prep64(const Geo& g, const float* bias, float* prep, cudaStream_t stream) {
-    swin_fwd_bias_prep64_kernel<<<g.heads, 256, 0, stream>>>(bias, prep, g.w, g.heads, 0);
+    swin_fwd_bias_prep64_kernel<<<g.heads, 256, 0, stream>>>(bias, prep, g.w, g.heads, g.w > 32 ? 1 : 0);
     count_launch(stream);
     return cudaGetLastError();
 }
