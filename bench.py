@@ -440,6 +440,7 @@ def main():
                        "swin_bwd_fused_kernel": 8 * d * pairs, "swin_bwd_small_kernel": 8 * d * pairs,
                        "swin_bwd_mma_kernel<key tiles>": 4 * d * pairs, "swin_bwd_mma_kernel<query tiles>": 4 * d * pairs,
                        "swin_bwd_kv64_kernel": 4 * d * pairs, "swin_bwd_q64_kernel": 4 * d * pairs,
+                       "swin_bwd_kv64_kernel<query side>": 4 * d * pairs,
                        "swin_bwd_delta_kernel": 0}
         kernels = []
         for kname, vals in kernel_ms.items():

@@ -146,7 +146,8 @@ static size_t delta_bytes(const Geo& g) {
     if (use_bwd_tc(g)) return align_up(bwd_tc_workspace_bytes(g), 256);
     const size_t delta = align_up(sizeof(float) * (size_t)g.B * g.H * g.W * g.heads, 256);
     // the tcgen05 key-side kernel of the head-dim-64 regime also wants the prepared bias tables
-    return use_bwd_kv64(g) ? delta + align_up(fwd_tc64_workspace_bytes(g), 256) : delta;
+    // (windows of side 64 and 128: twice, the second copy reflected for the query-side use of that kernel)
+    return use_bwd_kv64(g) ? delta + (g.w > 32 ? 2 : 1) * align_up(fwd_tc64_workspace_bytes(g), 256) : delta;
 }
 
 // Descriptor check + geometry, and the SM count of the current device, for entry points that live in
@@ -283,8 +284,15 @@ static int bwd_call(const Geo& g, const void* q, const void* k, const void* v,
             e = g.f16 ? launch_bwd_kv64_f16(g, q, k, v, d_o, prep, lse, delta, dk, dv, sms, st)
                       : launch_bwd_kv64(g, q, k, v, d_o, prep, lse, delta, dk, dv, sms, st);
         if (e == cudaSuccess) {
-            // query side (dQ, dBias): tcgen05 for complete 32 x 32 windows, else the register-tile kernel
-            if (bwd_q64_supported(g))
+            // query side (dQ, dBias): tcgen05 for complete 32 x 32 windows and for complete windows of side 64 and 128
+            // (the key-side kernel with the tensors' roles exchanged), else the register-tile kernel
+            if (g.w > 32) {
+                float* prep_r = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(prep) + align_up(fwd_tc64_workspace_bytes(g), 256));
+                e = launch_bias_prep64(g, bias_table, prep_r, st, true);
+                if (e == cudaSuccess)
+                    e = g.f16 ? launch_bwd_kv64_qside_f16(g, q, k, v, d_o, prep_r, lse, delta, dq, dbias, sms, st)
+                              : launch_bwd_kv64_qside(g, q, k, v, d_o, prep_r, lse, delta, dq, dbias, sms, st);
+            } else if (bwd_q64_supported(g))
                 e = g.f16 ? launch_bwd_q64_f16(g, q, k, v, d_o, prep, lse, delta, dq, dbias, sms, st)
                           : launch_bwd_q64(g, q, k, v, d_o, prep, lse, delta, dq, dbias, sms, st);
             else

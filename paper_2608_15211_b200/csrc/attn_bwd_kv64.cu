@@ -33,6 +33,7 @@
 #ifdef TERRA_ELEM_F16
 #define g_bwd_kv64_timeout g_bwd_kv64_timeout_f16
 #define launch_bwd_kv64 launch_bwd_kv64_f16
+#define launch_bwd_kv64_qside launch_bwd_kv64_qside_f16
 #define read_bwd_kv64_status read_bwd_kv64_status_f16
 #endif
 
@@ -200,6 +201,40 @@ __device__ __forceinline__ void cols16(const uint32_t (&rs)[16], const uint32_t 
     }
 }
 
+// Query-side use of the kernel (rows = queries, columns = keys): 16 key columns [c, c + 16) of one query row.
+// `neg_l2` = -lse * log2(e) and `dl` = delta of the row; `bias_a` = shared address of the row's bias entry for column
+// c (the following keys' entries follow); the key columns' mask labels are the slot's label table.  dS leaves as
+// packed bf16 for the dQ product and in fp32 for the bias gradient.
+template <bool MASKED>
+__device__ __forceinline__ void cols16_qside(const uint32_t (&rs)[16], const uint32_t (&rp)[16], int c, uint32_t bias_a, int rlabel,
+                                             uint32_t sl_a, float scale, float neg_l2, float dl, uint32_t (&pk_ds)[8], float (&ds)[16]) {
+    constexpr int kOffQLab = 512;
+    int cl[16];
+    float bv[16];
+    if (MASKED) {
+#pragma unroll
+        for (int e4 = 0; e4 < 4; ++e4) {
+            const int4 q4 = lds_i4(sl_a + kOffQLab + 4 * (c + e4 * 4));
+            cl[e4 * 4] = q4.x; cl[e4 * 4 + 1] = q4.y; cl[e4 * 4 + 2] = q4.z; cl[e4 * 4 + 3] = q4.w;
+        }
+    }
+#pragma unroll
+    for (int e = 0; e < 16; ++e) bv[e] = lds_f32(bias_a + 4 * e);
+#pragma unroll
+    for (int e = 0; e < 16; e += 2) {
+        float x0, x1, t0, t1;
+        fma2(x0, x1, __uint_as_float(rs[e]), __uint_as_float(rs[e + 1]), scale, bv[e], bv[e + 1]);
+        add2(x0, x1, x0, x1, neg_l2);
+        if (MASKED && cl[e] != rlabel) x0 = -INFINITY;
+        if (MASKED && cl[e + 1] != rlabel) x1 = -INFINITY;
+        const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+        add2(t0, t1, __uint_as_float(rp[e]), __uint_as_float(rp[e + 1]), -dl);
+        mul2(ds[e], ds[e + 1], p0, p1, t0, t1);
+    }
+#pragma unroll
+    for (int e2 = 0; e2 < 8; ++e2) pk_ds[e2] = pack_elem(ds[2 * e2], ds[2 * e2 + 1]);
+}
+
 // 32 accumulator columns of one row, scaled, as 64 bytes of bf16
 __device__ __forceinline__ void store_scaled32(uint4* dst, const uint32_t (&r)[32], float f) {
 #pragma unroll
@@ -227,15 +262,24 @@ struct KvMaps64 {
 // with every query chunk, the 2 kr - 1 table rows (kr = 128 / w window rows per 128 slots) that the chunk's queries
 // need against the item's key tile; in the prepared layout (2 w floats per table row) they are one contiguous block,
 // and the 16 queries of a column group read consecutive entries, as in the 32-wide case.
+// MODE 3: MODE 2 put to use for the query side (dQ, dBias) of such windows.  The host hands over the tensors with the
+// roles exchanged (Q and dO as the "key tile", K and V as the streamed "queries") and the bias table reflected through
+// its centre, so that rows are queries and columns keys: S = Q K_c^T, dP = dO V_c^T, dS as above with the row's own
+// lse and delta, and the accumulator that is dK in the key-side use is dQ = dS K_c; the other one is not computed.
+// dBias: the 32 lanes of a warp are 32 consecutive queries of one window row and a half chunk's 64 columns are 64
+// consecutive keys of one window row, so the entries (b_q - b_k) run along the diagonals of the warp's 32 x 64 block.
+// A lane carries the partial sum of the diagonal through its current column, hands it to the next lane when the
+// column advances (one shuffle and one add per element), lane 31 adds the diagonal that leaves the block to the
+// global gradient, and after the last column every lane adds what it holds: 95 float atomics per warp and half chunk.
 template <int D, int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
 swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                      const __nv_bfloat16* __restrict__ v, const __nv_bfloat16* __restrict__ d_o,
                      const float* __restrict__ bias_prep, const float* __restrict__ lse, const float* __restrict__ delta,
-                     __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv, long long n_items, int ctas_per_head,
-                     int max_tiles, const __grid_constant__ KvMaps64 maps) {
+                     __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv, float* __restrict__ dbias, long long n_items,
+                     int ctas_per_head, int max_tiles, const __grid_constant__ KvMaps64 maps) {
     using L = Lay<D>;
-    constexpr bool TMA = MODE >= 1, ROWS = MODE == 2;
+    constexpr bool TMA = MODE >= 1, ROWS = MODE >= 2, QS = MODE == 3;
     constexpr int kStageBytes = 1536;                 // MODE 2: the staged table rows of one query slot
     constexpr int kParts = L::kParts, kKvStages = L::kKvStages, kSlots = L::kSlots;
     constexpr int kOffK = L::kOffK, kOffV = L::kOffV, kOffKCode = L::kOffKCode, kOffKLab = L::kOffKLab, kOffKTok = L::kOffKTok;
@@ -360,8 +404,10 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                         const int a = slot / ew;
                         const int tok = offset_token(g, x.r, a, slot - a * ew, code, label);
                         const size_t li = (sample_off + (size_t)tok) * g.heads + head;
-                        cp_async4(sb + kOffQLse + 4 * row, lse + li);
-                        cp_async4(sb + kOffQDelta + 4 * row, delta + li);
+                        if (!QS) {
+                            cp_async4(sb + kOffQLse + 4 * row, lse + li);
+                            cp_async4(sb + kOffQDelta + 4 * row, delta + li);
+                        }
                         reinterpret_cast<int*>(sl + kOffQCode)[row] = 4 * code;
                         reinterpret_cast<int*>(sl + kOffQLab)[row] = label;
                     }
@@ -381,7 +427,8 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                     }
                     if (lane == 0) mbar_expect_tx(bar_qfull(s), (uint32_t)(kTile * D * 2 * 2));
                     // the lane's arrival: when its lse / delta copies have landed (its table entries were written before)
-                    cp_async_mbar_arrive_noinc(bar_qfull(s));
+                    if (QS) mbar_arrive(bar_qfull(s));
+                    else cp_async_mbar_arrive_noinc(bar_qfull(s));
                 }
                 ++kuse;
             }
@@ -593,12 +640,12 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                 if (elect_one()) {
                     int j = 0;
                     if (i == 0) {
-                        mma_ts_h<false>(tmem_base + kColDV, t_p, g_lo, d_hi, idesc_acc);
+                        if (!QS) mma_ts_h<false>(tmem_base + kColDV, t_p, g_lo, d_hi, idesc_acc);
                         mma_ts_h<false>(tmem_base + kColDK, t_ds, q_lo, d_hi, idesc_acc);
                         j = 1;
                     }
                     for (; j < nks; ++j) {
-                        mma_ts_h<true>(tmem_base + kColDV, t_p + 16 * j, g_lo + 64 * j, d_hi, idesc_acc);
+                        if (!QS) mma_ts_h<true>(tmem_base + kColDV, t_p + 16 * j, g_lo + 64 * j, d_hi, idesc_acc);
                         mma_ts_h<true>(tmem_base + kColDK, t_ds + 16 * j, q_lo + 64 * j, d_hi, idesc_acc);
                     }
                     if (chunk_done) mma_commit(bar_qempty(s));       // the slot's last readers were issued just above
@@ -646,6 +693,13 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             const int klabel = lds_i32(st_a + kOffKLab + 4 * krow);
             const int ktok = lds_i32(st_a + kOffKTok + 4 * krow);
             mbar_arrive(bar_kvempty(ks));                 // this thread has what it needs from the key stage
+            // MODE 3: the row is a query; its lse and delta
+            float neg_l2 = 0.f, row_dl = 0.f;
+            if (QS) {
+                const size_t li = ((size_t)x.b * HW + (size_t)ktok) * g.heads + head;
+                neg_l2 = -lse[li] * kLog2e;
+                row_dl = delta[li];
+            }
             // bias index = code_query - code_key + c0; a key row without a token reads the table's -inf zone
             uint32_t bias_row = smem0 + kOffBias + (ktok >= 0 ? 4 * c0 - kcode4 : 4 * (2 * c0 + 1));
             const bool row32 = ROWS || x.r.ew == 32;
@@ -675,6 +729,39 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                 };
                 // groups of 16 columns; the next group's S^T / dP^T travel from TMEM while this one is worked on
                 uint32_t rs[16], rp[16], rs2[16], rp2[16], pk_p[8], pk_ds[8];
+                if (QS) {
+                    // this warp's rows: 32 queries b_q = bq0 + lane of window row a_q; the half chunk's columns: 64 keys
+                    // b_k = bk0 + j of window row a_k.  `dst`: the lane's entry of the gradient for the current column.
+                    const int nw = 2 * g.w - 1;
+                    const int qslot = x.kt * kTile + krow, kslot = c * kTile + 64 * hcol;
+                    const int da = (qslot >> lw) - (kslot >> lw) + g.w - 1, db = (qslot & (g.w - 1)) - (kslot & (g.w - 1)) + g.w - 1;
+                    float* dst = dbias + ((size_t)da * nw + db) * g.heads + head;
+                    float acc = 0.f;
+                    float ds[16];
+                    tmem_ld16(t_s + 64 * hcol, rs);
+                    tmem_ld16(t_dp + 64 * hcol, rp);
+#pragma unroll 1
+                    for (int cc = 64 * hcol; cc < 64 * hcol + 64; cc += 16) {
+                        tmem_ld_wait();
+                        if (x.masked) cols16_qside<true>(rs, rp, cc, bias_row + code4_of(cc), klabel, sl_a, scale, neg_l2, row_dl, pk_ds, ds);
+                        else cols16_qside<false>(rs, rp, cc, bias_row + code4_of(cc), klabel, sl_a, scale, neg_l2, row_dl, pk_ds, ds);
+                        if (cc + 16 < 64 * hcol + 64) {
+                            tmem_ld16(t_s + cc + 16, rs);
+                            tmem_ld16(t_dp + cc + 16, rp);
+                        }
+                        tmem_st8(t_dp + cc, pk_ds);
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) {
+                            // the diagonal that lane 31 carried through the previous column ends there
+                            if (lane == 31 && (cc + e) != 64 * hcol) atomicAdd(dst, acc);
+                            if (cc + e != 64 * hcol) dst -= g.heads;
+                            acc = __shfl_up_sync(0xffffffffu, acc, 1);
+                            if (lane == 0) acc = 0.f;
+                            acc += ds[e];
+                        }
+                    }
+                    atomicAdd(dst, acc);
+                } else {
                 if (64 * hcol < col_end) {
                     tmem_ld16(t_s + 64 * hcol, rs);
                     tmem_ld16(t_dp + 64 * hcol, rp);
@@ -705,6 +792,7 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                         tmem_st8(t_dp + cc + 16, pk_ds);
                     }
                 }
+                }
                 tmem_st_wait();
                 tc_fence_before();
                 mbar_arrive(bar_ds(buf));
@@ -714,9 +802,24 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             // ---- read-out: dV rows by warps 0-3, dK rows by warps 4-7
             if (!mbar_wait_all(bar_acc, kuse & 1, cta_abort)) break;
             tc_fence_after();
-            const float f = hcol == 0 ? 1.f : out_scale;
-            __nv_bfloat16* out = hcol == 0 ? dv : dk;
+            const float f = (QS || hcol != 0) ? out_scale : 1.f;
+            __nv_bfloat16* out = (QS || hcol != 0) ? dk : dv;
             uint4* dst = reinterpret_cast<uint4*>(out + ((size_t)x.b * HW + (size_t)(ktok >= 0 ? ktok : 0)) * g.ts + head * D);
+            if (QS) {
+                // one accumulator (dQ): each group of warps reads half of its columns
+#pragma unroll
+                for (int hq = 0; hq < D / 64; ++hq) {
+                    uint32_t r0[32];
+                    const int col = hcol * (D / 2) + 32 * hq;
+                    tmem_ld32(tmem_base + lane_addr + kColDK + col, r0);
+                    tmem_ld_wait();
+                    if (hq == D / 64 - 1) {
+                        tc_fence_before();
+                        mbar_arrive(bar_accfree);
+                    }
+                    store_scaled32(dst + col / 8, r0, f);
+                }
+            } else {
 #pragma unroll
             for (int hq = 0; hq < D / 64; ++hq) {
                 uint32_t r0[32], r1[32];
@@ -731,6 +834,7 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                     store_scaled32(dst + 8 * hq, r0, f);
                     store_scaled32(dst + 8 * hq + 4, r1, f);
                 }
+            }
             }
             ++kuse;
         }
@@ -773,8 +877,30 @@ bool bwd_kv64_supported(const Geo& g) {
 
 // `prep` = the prepared bias tables of the head-dim-64 forward kernel (kBiasFloats per head; for window sides 64 and
 // 128 its layout of whole table rows), filled by the caller
+static cudaError_t launch_kv64(const Geo& g, const void* q, const void* k, const void* v, const void* d_o, const float* prep,
+                               const float* lse, const float* delta, void* dk, void* dv, float* dbias, bool qside, int sm_count,
+                               cudaStream_t stream);
+
 cudaError_t launch_bwd_kv64(const Geo& g, const void* q, const void* k, const void* v, const void* d_o, const float* prep,
                             const float* lse, const float* delta, void* dk, void* dv, int sm_count, cudaStream_t stream) {
+    return launch_kv64(g, q, k, v, d_o, prep, lse, delta, dk, dv, nullptr, false, sm_count, stream);
+}
+
+// The query side (dQ, dBias) of complete windows of side 64 and 128 with the same kernel: the tensors change roles and
+// `prep_reflected` is the bias table reflected through its centre (launch_bias_prep64 with reflect = true); dbias is
+// overwritten.
+cudaError_t launch_bwd_kv64_qside(const Geo& g, const void* q, const void* k, const void* v, const void* d_o,
+                                  const float* prep_reflected, const float* lse, const float* delta, void* dq, float* dbias,
+                                  int sm_count, cudaStream_t stream) {
+    if (g.w <= 32) return cudaErrorNotSupported;
+    cudaError_t e = cudaMemsetAsync(dbias, 0, sizeof(float) * (size_t)(2 * g.w - 1) * (2 * g.w - 1) * g.heads, stream);
+    if (e != cudaSuccess) return e;
+    return launch_kv64(g, q, k, v, d_o, prep_reflected, lse, delta, dq, nullptr, dbias, true, sm_count, stream);
+}
+
+static cudaError_t launch_kv64(const Geo& g, const void* q, const void* k, const void* v, const void* d_o, const float* prep,
+                               const float* lse, const float* delta, void* dk, void* dv, float* dbias, bool qside, int sm_count,
+                               cudaStream_t stream) {
     const int max_tiles = (g.nmax + 127) >> 7;
     const long long items = (long long)g.B * g.Mh * g.Mw * max_tiles;
     long long cph = sm_count / g.heads;
@@ -783,18 +909,22 @@ cudaError_t launch_bwd_kv64(const Geo& g, const void* q, const void* k, const vo
     KvMaps64 maps;
     std::memset(&maps, 0, sizeof maps);
     const bool rows = g.w > 32;
-    const bool tma = (!no_tma_env() || rows) && bulk_rows_shape(g) && make_row_maps3(&maps.q, g, q, g.ts) && make_row_maps3(&maps.k, g, k, g.ts) &&
-                     make_row_maps3(&maps.v, g, v, g.ts) && make_row_maps3(&maps.g, g, d_o, g.heads * g.d);
-    if (rows && !tma) return cudaErrorNotSupported;       // windows of side 64 and 128 have no gathering loader
-    auto kern = g.d == 64 ? (rows ? swin_bwd_kv64_kernel<64, 2> : tma ? swin_bwd_kv64_kernel<64, 1> : swin_bwd_kv64_kernel<64, 0>)
-                          : (rows ? swin_bwd_kv64_kernel<128, 2> : tma ? swin_bwd_kv64_kernel<128, 1> : swin_bwd_kv64_kernel<128, 0>);
+    // the kernel's tile rows ("k", "v") and streamed rows ("q", "g"); the query side exchanges the roles
+    const bool tma = (!no_tma_env() || rows) && bulk_rows_shape(g) &&
+                     (qside ? make_row_maps3(&maps.k, g, q, g.ts) && make_row_maps3(&maps.v, g, d_o, g.heads * g.d) &&
+                                  make_row_maps3(&maps.q, g, k, g.ts) && make_row_maps3(&maps.g, g, v, g.ts)
+                            : make_row_maps3(&maps.q, g, q, g.ts) && make_row_maps3(&maps.k, g, k, g.ts) &&
+                                  make_row_maps3(&maps.v, g, v, g.ts) && make_row_maps3(&maps.g, g, d_o, g.heads * g.d));
+    if ((rows || qside) && !tma) return cudaErrorNotSupported;       // windows of side 64 and 128 have no gathering loader
+    auto kern = g.d == 64 ? (qside ? swin_bwd_kv64_kernel<64, 3> : rows ? swin_bwd_kv64_kernel<64, 2> : tma ? swin_bwd_kv64_kernel<64, 1> : swin_bwd_kv64_kernel<64, 0>)
+                          : (qside ? swin_bwd_kv64_kernel<128, 3> : rows ? swin_bwd_kv64_kernel<128, 2> : tma ? swin_bwd_kv64_kernel<128, 1> : swin_bwd_kv64_kernel<128, 0>);
     const int smem_bytes = g.d == 64 ? Lay<64>::kSmemBytes : Lay<128>::kSmemBytes;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
     if (e != cudaSuccess) return e;
-    prof_begin("swin_bwd_kv64_kernel", stream);
+    prof_begin(qside ? "swin_bwd_kv64_kernel<query side>" : "swin_bwd_kv64_kernel", stream);
     kern<<<(unsigned)(cph * g.heads), kThreads, smem_bytes, stream>>>(
         g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)d_o, prep, lse, delta,
-        (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, items, (int)cph, max_tiles, maps);
+        (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, dbias, items, (int)cph, max_tiles, maps);
     count_launch(stream);
     return cudaGetLastError();
 }

@@ -982,7 +982,8 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
 //   table[2 c0 + 1 .. 3 c0 + 1] = -inf (where key slots without a token point), the head's largest entry in the last float
 //   (+inf instead if the head's entries spread over more than 64 octaves).
 // Window sides 64 and 128 (`rows`): per head (2w - 1) table rows of 2w floats (the last one padding) and four more
-// floats, the last of which is the head's largest entry as above.
+// floats, the last of which is the head's largest entry as above; `rows` = 2: the table reflected through its centre
+// (entry (r, c) holds T[2w - 2 - r][2w - 2 - c]), for the query-side use of the key-major backward kernel.
 __global__ void __launch_bounds__(256)
 swin_fwd_bias_prep64_kernel(const float* __restrict__ bias, float* __restrict__ prep, int w, int heads, int rows) {
     const int head = blockIdx.x;
@@ -998,7 +999,8 @@ swin_fwd_bias_prep64_kernel(const float* __restrict__ bias, float* __restrict__ 
         } else {
             const int ra = e / cs, rb = e - ra * cs;
             if (rb < nw && ra < nw) {
-                val = bias[(size_t)(ra * nw + rb) * heads + head] * kLog2e;
+                const int sa = rows == 2 ? nw - 1 - ra : ra, sb = rows == 2 ? nw - 1 - rb : rb;
+                val = bias[(size_t)(sa * nw + sb) * heads + head] * kLog2e;
                 mx = fmaxf(mx, val);
                 mn = fminf(mn, val);
             }
@@ -1034,8 +1036,9 @@ cudaError_t read_fwd_tc64_status(int* timed_out) {
 #ifndef TERRA_ELEM_F16
 // prepared bias tables for the kernels of the large-window regime: kBiasFloats = 6048 floats per head for window
 // sides up to 32, whole table rows for sides 64 and 128 (see the kernel above)
-cudaError_t launch_bias_prep64(const Geo& g, const float* bias, float* prep, cudaStream_t stream) {
-    swin_fwd_bias_prep64_kernel<<<g.heads, 256, 0, stream>>>(bias, prep, g.w, g.heads, g.w > 32 ? 1 : 0);
+cudaError_t launch_bias_prep64(const Geo& g, const float* bias, float* prep, cudaStream_t stream, bool reflect) {
+    if (reflect && g.w <= 32) return cudaErrorNotSupported;
+    swin_fwd_bias_prep64_kernel<<<g.heads, 256, 0, stream>>>(bias, prep, g.w, g.heads, g.w > 32 ? (reflect ? 2 : 1) : 0);
     count_launch(stream);
     return cudaGetLastError();
 }

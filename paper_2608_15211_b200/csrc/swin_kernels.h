@@ -39,6 +39,9 @@ cudaError_t read_fwd_tc64_status_f16(int* timed_out);
 cudaError_t launch_bwd_kv64_f16(const Geo& g, const void* q, const void* k, const void* v, const void* d_o, const float* prep,
                                 const float* lse, const float* delta, void* dk, void* dv, int sm_count, cudaStream_t stream);
 cudaError_t read_bwd_kv64_status_f16(int* timed_out);
+cudaError_t launch_bwd_kv64_qside_f16(const Geo& g, const void* q, const void* k, const void* v, const void* d_o,
+                                      const float* prep_reflected, const float* lse, const float* delta, void* dq, float* dbias,
+                                      int sm_count, cudaStream_t stream);
 cudaError_t launch_bwd_q64_f16(const Geo& g, const void* q, const void* k, const void* v, const void* d_o, const float* prep,
                                const float* lse, const float* delta, void* dq, float* dbias, int sm_count, cudaStream_t stream);
 cudaError_t read_bwd_q64_status_f16(int* timed_out);
@@ -68,7 +71,8 @@ size_t fwd_tc64_workspace_bytes(const Geo& g);
 cudaError_t launch_fwd_tc64(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
                             void* o, float* lse, void* workspace, int sm_count, cudaStream_t stream);
 cudaError_t read_fwd_tc64_status(int* timed_out);     // after the stream has been synchronised
-cudaError_t launch_bias_prep64(const Geo& g, const float* bias, float* prep, cudaStream_t stream);
+// (window sides 64 and 128: whole table rows; `reflect`: the table reflected through its centre)
+cudaError_t launch_bias_prep64(const Geo& g, const float* bias, float* prep, cudaStream_t stream, bool reflect = false);
 
 // tcgen05 key side (dK, dV) of the backward pass for head dim 64 and windows of up to 1024 tokens; `prep` = the
 // tables of launch_bias_prep64, `delta` as for the register-tile kernels
@@ -76,6 +80,11 @@ bool bwd_kv64_supported(const Geo& g);
 cudaError_t launch_bwd_kv64(const Geo& g, const void* q, const void* k, const void* v, const void* d_o, const float* prep,
                             const float* lse, const float* delta, void* dk, void* dv, int sm_count, cudaStream_t stream);
 cudaError_t read_bwd_kv64_status(int* timed_out);
+// the query side (dQ, dBias) of complete windows of side 64 and 128 with the same kernel; `prep_reflected` = the
+// tables of launch_bias_prep64 with reflect = true; dbias is overwritten
+cudaError_t launch_bwd_kv64_qside(const Geo& g, const void* q, const void* k, const void* v, const void* d_o,
+                                  const float* prep_reflected, const float* lse, const float* delta, void* dq, float* dbias,
+                                  int sm_count, cudaStream_t stream);
 
 // tcgen05 query side (dQ, dBias) of the same regime for complete 32 x 32 windows (window side 32, grid extents
 // multiples of 32); dbias is overwritten
