@@ -268,9 +268,9 @@ struct KvMaps64 {
 // lse and delta, and the accumulator that is dK in the key-side use is dQ = dS K_c; the other one is not computed.
 // dBias: the 32 lanes of a warp are 32 consecutive queries of one window row and a half chunk's 64 columns are 64
 // consecutive keys of one window row, so the entries (b_q - b_k) run along the diagonals of the warp's 32 x 64 block.
-// A lane carries the partial sum of the diagonal through its current column, hands it to the next lane when the
-// column advances (one shuffle and one add per element), lane 31 adds the diagonal that leaves the block to the
-// global gradient, and after the last column every lane adds what it holds: 95 float atomics per warp and half chunk.
+// The block has 95 diagonals; each is summed in one of three accumulators of one lane: a column's 32 values reach
+// their diagonals' lanes with one rotation of the warp (one shuffle per element, no chain between columns), and after
+// the half chunk the lanes add their accumulators to the global gradient: 95 float atomics per warp and half chunk.
 template <int D, int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
 swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
@@ -732,35 +732,45 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                 if (QS) {
                     // this warp's rows: 32 queries b_q = bq0 + lane of window row a_q; the half chunk's columns: 64 keys
                     // b_k = bk0 + j of window row a_k.  `dst`: the lane's entry of the gradient for the current column.
+                    // Diagonal D = lane - j (j = column within the half chunk, -63 <= D <= 31) is kept by lane (D + 63) % 32
+                    // in accumulator (D + 63) / 32: column j's values move up by r = 31 - j % 32 lanes (around the warp),
+                    // the lanes below r receive values of the next higher accumulator.
                     const int nw = 2 * g.w - 1;
-                    const int qslot = x.kt * kTile + krow, kslot = c * kTile + 64 * hcol;
-                    const int da = (qslot >> lw) - (kslot >> lw) + g.w - 1, db = (qslot & (g.w - 1)) - (kslot & (g.w - 1)) + g.w - 1;
-                    float* dst = dbias + ((size_t)da * nw + db) * g.heads + head;
-                    float acc = 0.f;
+                    const int qslot0 = x.kt * kTile + 32 * quarter, kslot = c * kTile + 64 * hcol;
+                    const int da = (qslot0 >> lw) - (kslot >> lw) + g.w - 1, db0 = (qslot0 & (g.w - 1)) - (kslot & (g.w - 1)) + g.w - 1;
+                    float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f;
                     float ds[16];
+                    auto diag16 = [&](int j0, float& lo, float& hi) {
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) {
+                            const int r = 31 - ((j0 + e) & 31);
+                            const float val = __shfl_sync(0xffffffffu, ds[e], (lane - r) & 31);
+                            const bool up = lane < r;
+                            hi += up ? val : 0.f;
+                            lo += up ? 0.f : val;
+                        }
+                    };
                     tmem_ld16(t_s + 64 * hcol, rs);
                     tmem_ld16(t_dp + 64 * hcol, rp);
-#pragma unroll 1
-                    for (int cc = 64 * hcol; cc < 64 * hcol + 64; cc += 16) {
+#pragma unroll
+                    for (int gi = 0; gi < 4; ++gi) {
+                        const int cc = 64 * hcol + 16 * gi;
                         tmem_ld_wait();
                         if (x.masked) cols16_qside<true>(rs, rp, cc, bias_row + code4_of(cc), klabel, sl_a, scale, neg_l2, row_dl, pk_ds, ds);
                         else cols16_qside<false>(rs, rp, cc, bias_row + code4_of(cc), klabel, sl_a, scale, neg_l2, row_dl, pk_ds, ds);
-                        if (cc + 16 < 64 * hcol + 64) {
+                        if (gi < 3) {
                             tmem_ld16(t_s + cc + 16, rs);
                             tmem_ld16(t_dp + cc + 16, rp);
                         }
                         tmem_st8(t_dp + cc, pk_ds);
-#pragma unroll
-                        for (int e = 0; e < 16; ++e) {
-                            // the diagonal that lane 31 carried through the previous column ends there
-                            if (lane == 31 && (cc + e) != 64 * hcol) atomicAdd(dst, acc);
-                            if (cc + e != 64 * hcol) dst -= g.heads;
-                            acc = __shfl_up_sync(0xffffffffu, acc, 1);
-                            if (lane == 0) acc = 0.f;
-                            acc += ds[e];
-                        }
+                        if (gi < 2) diag16(16 * gi, acc1, acc2);          // columns 0..31: diagonals -31..31
+                        else diag16(16 * gi, acc0, acc1);                 // columns 32..63: diagonals -63..-1
                     }
-                    atomicAdd(dst, acc);
+                    // accumulator a of this lane is diagonal 32 a + lane - 63: entry db0 + that of table row da
+                    float* dst = dbias + ((size_t)da * nw + (db0 + lane - 63)) * g.heads + head;
+                    atomicAdd(dst, acc0);
+                    atomicAdd(dst + 32 * g.heads, acc1);
+                    if (lane < 31) atomicAdd(dst + 64 * g.heads, acc2);
                 } else {
                 if (64 * hcol < col_end) {
                     tmem_ld16(t_s + 64 * hcol, rs);
