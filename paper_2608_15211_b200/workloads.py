@@ -67,6 +67,9 @@ CONFIGS = {
     # A 3 x 5-window slice of the large model's block (same heads, head dim, window, shift): 2.3 GB on the device
     # with gradients, the size a full-counter profiler capture of the head-dim-128 tcgen05 kernels is taken on
     "tv_large_slice": SwinConfig("tv_large_slice", 1, 96, 160, 64, 128, 32, 16, 16, index=10),
+    # One row of three 128 x 128 windows of the window-assignment study's block (same heads, head dim, window, shift):
+    # 0.9 GB on the device with gradients, for profiler captures of the tcgen05 kernels at window side 128
+    "tv_small_w128_slice": SwinConfig("tv_small_w128_slice", 1, 128, 384, 8, 128, 128, 64, 64, index=11),
 }
 
 TENSOR_INDEX = {"q": 0, "k": 1, "v": 2, "do": 3, "bias": 4}
