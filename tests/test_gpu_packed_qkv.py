@@ -18,6 +18,7 @@ CASES = [
     small_config("packed_d64", 1, 45, 50, 2, 64, 20, 10, 10, 0, 1),    # register-tile kernels
     small_config("packed_d64_w32", 1, 64, 64, 2, 64, 32, 16, 16, 0, 1),  # chunked tcgen05 kernels, complete windows
     small_config("packed_noshift", 1, 32, 32, 2, 32, 16, 0, 0, 0, 1),  # the unshifted W-MSA sibling of the block
+    small_config("packed_d64_w64", 1, 64, 128, 2, 64, 64, 32, 24, 0, 1),  # chunked tcgen05 kernels with staged bias rows
 ]
 
 
