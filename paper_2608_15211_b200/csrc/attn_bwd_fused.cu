@@ -24,6 +24,8 @@
 // CTAs are bound to one head (grid = heads x CTAs per head): the head's bias table is staged once per CTA
 // and the bias-gradient tables belong to one head; they are summed in a fixed order (reproducible dBias).
 // Every mbarrier wait is bounded; on expiry the CTA raises an abort flag and all roles leave their loops.
+#include <cstdlib>
+
 #include "swin_common.cuh"
 #include "swin_kernels.h"
 #include "tc_common.cuh"
@@ -96,6 +98,8 @@ constexpr int kColDK = 288;
 constexpr int kColDQ = 384;         // dQ of query pair p at 384 + 32 p
 
 __device__ __forceinline__ int code_stride(int w) { return w + 32; }
+// floats in front of a warp's bias-gradient table in the 16-slots-per-row layout of window sides 9 .. 15
+__host__ __device__ __forceinline__ int dbias_margin(int w) { return (16 - w) * (w + 32) + 8; }
 
 // Key rows of a tile are interleaved over the elementwise warps: lane l of warp W = 4 t + quarter holds slot
 // 32 ((W + c l) mod M) + l, M = 4 * (tiles in use).  c = 1, except c = 5 for two-tile windows whose side does not
@@ -112,11 +116,14 @@ struct Item {
     bool ragged;   // some row of a key tile, or some column below npad, has no token
 };
 
-__device__ __forceinline__ Item make_item(const Geo& g, const ItemCursor& c) {
+// pad16: the window's slots are laid out 16 to a window row (slot = 16 a + b; the slots with b >= the window's width
+// hold no token), so that every group of 16 query columns is one window row whatever the window side
+__device__ __forceinline__ Item make_item(const Geo& g, const ItemCursor& c, bool pad16 = false) {
     Item x;
     x.win = c.wr * g.Mw + c.wc;
     x.b = c.b;
     x.r = window_ref_rc(g, c.wr, c.wc);
+    if (pad16) x.r.n = x.r.eh * 16;
     x.npad = (x.r.n + 15) & ~15;
     x.ntiles = (x.r.n + 127) >> 7;
     x.nblk = (x.npad + CB - 1) / CB;
@@ -124,7 +131,7 @@ __device__ __forceinline__ Item make_item(const Geo& g, const ItemCursor& c) {
     const bool mh = !g.ph && g.sh > 0 && r0 < g.H - g.sh && r0 + x.r.eh > g.H - g.sh;
     const bool mw = !g.pw && g.sw > 0 && c0 < g.W - g.sw && c0 + x.r.ew > g.W - g.sw;
     x.masked = mh || mw;
-    x.ragged = x.npad != x.r.n || x.r.n != x.ntiles * 128;
+    x.ragged = pad16 || x.npad != x.r.n || x.r.n != x.ntiles * 128;
     return x;
 }
 
@@ -209,6 +216,67 @@ __device__ __forceinline__ void rmw8_consecutive_f32(uint32_t a, const float* v)
         "st.shared.f32 [%0], t0;\n\tst.shared.f32 [%0+4], t1;\n\tst.shared.f32 [%0+8], t2;\n\tst.shared.f32 [%0+12], t3;\n\t"
         "st.shared.f32 [%0+16], t4;\n\tst.shared.f32 [%0+20], t5;\n\tst.shared.f32 [%0+24], t6;\n\tst.shared.f32 [%0+28], t7;\n\t}\n"
         ::"r"(a), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]) : "memory");
+    __syncwarp();
+}
+// The same for the first N < 8 of 8 consecutive entries (the others belong to pairs without a token).
+template <int N>
+__device__ __forceinline__ void rmw_consecutive_f32(uint32_t a, const float* v) {
+    if (N == 1) {
+        asm volatile(
+            "{\n\t.reg .f32 t0;\n\t"
+            "ld.shared.f32 t0, [%0];\n\t"
+            "add.f32 t0, t0, %1;\n\t"
+            "st.shared.f32 [%0], t0;\n\t}\n"
+            ::"r"(a), "f"(v[0]) : "memory");
+    }
+    if (N == 2) {
+        asm volatile(
+            "{\n\t.reg .f32 t0, t1;\n\t"
+            "ld.shared.f32 t0, [%0];\n\tld.shared.f32 t1, [%0+4];\n\t"
+            "add.f32 t0, t0, %1;\n\tadd.f32 t1, t1, %2;\n\t"
+            "st.shared.f32 [%0], t0;\n\tst.shared.f32 [%0+4], t1;\n\t}\n"
+            ::"r"(a), "f"(v[0]), "f"(v[1]) : "memory");
+    }
+    if (N == 3) {
+        asm volatile(
+            "{\n\t.reg .f32 t0, t1, t2;\n\t"
+            "ld.shared.f32 t0, [%0];\n\tld.shared.f32 t1, [%0+4];\n\tld.shared.f32 t2, [%0+8];\n\t"
+            "add.f32 t0, t0, %1;\n\tadd.f32 t1, t1, %2;\n\tadd.f32 t2, t2, %3;\n\t"
+            "st.shared.f32 [%0], t0;\n\tst.shared.f32 [%0+4], t1;\n\tst.shared.f32 [%0+8], t2;\n\t}\n"
+            ::"r"(a), "f"(v[0]), "f"(v[1]), "f"(v[2]) : "memory");
+    }
+    if (N == 4) {
+        asm volatile(
+            "{\n\t.reg .f32 t0, t1, t2, t3;\n\t"
+            "ld.shared.f32 t0, [%0];\n\tld.shared.f32 t1, [%0+4];\n\tld.shared.f32 t2, [%0+8];\n\tld.shared.f32 t3, [%0+12];\n\t"
+            "add.f32 t0, t0, %1;\n\tadd.f32 t1, t1, %2;\n\tadd.f32 t2, t2, %3;\n\tadd.f32 t3, t3, %4;\n\t"
+            "st.shared.f32 [%0], t0;\n\tst.shared.f32 [%0+4], t1;\n\tst.shared.f32 [%0+8], t2;\n\tst.shared.f32 [%0+12], t3;\n\t}\n"
+            ::"r"(a), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]) : "memory");
+    }
+    if (N == 5) {
+        asm volatile(
+            "{\n\t.reg .f32 t0, t1, t2, t3, t4;\n\t"
+            "ld.shared.f32 t0, [%0];\n\tld.shared.f32 t1, [%0+4];\n\tld.shared.f32 t2, [%0+8];\n\tld.shared.f32 t3, [%0+12];\n\tld.shared.f32 t4, [%0+16];\n\t"
+            "add.f32 t0, t0, %1;\n\tadd.f32 t1, t1, %2;\n\tadd.f32 t2, t2, %3;\n\tadd.f32 t3, t3, %4;\n\tadd.f32 t4, t4, %5;\n\t"
+            "st.shared.f32 [%0], t0;\n\tst.shared.f32 [%0+4], t1;\n\tst.shared.f32 [%0+8], t2;\n\tst.shared.f32 [%0+12], t3;\n\tst.shared.f32 [%0+16], t4;\n\t}\n"
+            ::"r"(a), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]) : "memory");
+    }
+    if (N == 6) {
+        asm volatile(
+            "{\n\t.reg .f32 t0, t1, t2, t3, t4, t5;\n\t"
+            "ld.shared.f32 t0, [%0];\n\tld.shared.f32 t1, [%0+4];\n\tld.shared.f32 t2, [%0+8];\n\tld.shared.f32 t3, [%0+12];\n\tld.shared.f32 t4, [%0+16];\n\tld.shared.f32 t5, [%0+20];\n\t"
+            "add.f32 t0, t0, %1;\n\tadd.f32 t1, t1, %2;\n\tadd.f32 t2, t2, %3;\n\tadd.f32 t3, t3, %4;\n\tadd.f32 t4, t4, %5;\n\tadd.f32 t5, t5, %6;\n\t"
+            "st.shared.f32 [%0], t0;\n\tst.shared.f32 [%0+4], t1;\n\tst.shared.f32 [%0+8], t2;\n\tst.shared.f32 [%0+12], t3;\n\tst.shared.f32 [%0+16], t4;\n\tst.shared.f32 [%0+20], t5;\n\t}\n"
+            ::"r"(a), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]) : "memory");
+    }
+    if (N == 7) {
+        asm volatile(
+            "{\n\t.reg .f32 t0, t1, t2, t3, t4, t5, t6;\n\t"
+            "ld.shared.f32 t0, [%0];\n\tld.shared.f32 t1, [%0+4];\n\tld.shared.f32 t2, [%0+8];\n\tld.shared.f32 t3, [%0+12];\n\tld.shared.f32 t4, [%0+16];\n\tld.shared.f32 t5, [%0+20];\n\tld.shared.f32 t6, [%0+24];\n\t"
+            "add.f32 t0, t0, %1;\n\tadd.f32 t1, t1, %2;\n\tadd.f32 t2, t2, %3;\n\tadd.f32 t3, t3, %4;\n\tadd.f32 t4, t4, %5;\n\tadd.f32 t5, t5, %6;\n\tadd.f32 t6, t6, %7;\n\t"
+            "st.shared.f32 [%0], t0;\n\tst.shared.f32 [%0+4], t1;\n\tst.shared.f32 [%0+8], t2;\n\tst.shared.f32 [%0+12], t3;\n\tst.shared.f32 [%0+16], t4;\n\tst.shared.f32 [%0+20], t5;\n\tst.shared.f32 [%0+24], t6;\n\t}\n"
+            ::"r"(a), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]) : "memory");
+    }
     __syncwarp();
 }
 template <int OFF>
@@ -313,12 +381,18 @@ __device__ __forceinline__ void load16_row(int c, int code0x4, const RowCtx& rc,
         dl[e4 * 4] = b.x; dl[e4 * 4 + 1] = b.y; dl[e4 * 4 + 2] = b.z; dl[e4 * 4 + 3] = b.w;
     }
 }
+// BW < 16: only the first BW of the 16 query columns hold a token; the others have P = dS = 0 and cost nothing.
+template <int BW = 16>
 __device__ __forceinline__ void math16_row(const uint32_t (&rs)[16], const uint32_t (&rp)[16], const float (&bv)[16], const float (&l2)[16],
                                            const float (&dl)[16], float scale, uint32_t (&pk_p)[8], uint32_t (&pk_ds)[8], float (&ds)[16]) {
     // two-wide fp32 operations: one instruction per pair of columns
     float p[16];
 #pragma unroll
     for (int e = 0; e < 16; e += 2) {
+        if (e >= BW) {
+            p[e] = p[e + 1] = ds[e] = ds[e + 1] = 0.f;
+            continue;
+        }
         float x0, x1, t0, t1;
         fma2(x0, x1, __uint_as_float(rs[e]), __uint_as_float(rs[e + 1]), scale, bv[e], bv[e + 1]);
         sub2(x0, x1, x0, x1, l2[e], l2[e + 1]);
@@ -334,12 +408,55 @@ __device__ __forceinline__ void math16_row(const uint32_t (&rs)[16], const uint3
     }
 }
 
+// One block of a two-tile window of width BW (9 .. 15) in the layout of 16 slots per window row: this warp's steps h
+// and h + 2 (one window row of queries each; the window's last block may lack the second), as in the 16-wide case.
+// A query column beyond the width has lse = +inf in the slot table, so an odd width's last pair needs no special case.
+template <int BW>
+__device__ __forceinline__ void pad_block16(uint32_t t_s, uint32_t t_dp, int h, int ca, int cb2, int cs, bool has_b, const RowCtx& rc,
+                                            uint32_t st_a, float scale, uint32_t (&pk_dsa)[8], uint32_t (&pk_dsb)[8]) {
+    uint32_t sa[16], pa[16], pk_p[8];
+    float ds[16], bv[16], l2[16], dl[16];
+    tmem_ld16(t_s + 16 * h, sa);
+    tmem_ld16(t_dp + 16 * h, pa);
+    tmem_ld_wait();
+    const int code_a = 4 * cs * (ca >> 4), code_b = 4 * cs * (cb2 >> 4);
+    load16_row(ca, code_a, rc, st_a, bv, l2, dl);
+    math16_row<BW>(sa, pa, bv, l2, dl, scale, pk_p, pk_dsa, ds);
+    uint32_t a0 = rc.dbias_row + code_a;
+    tmem_st8(t_s + 16 * h, pk_p);
+    tmem_st8(t_dp + 16 * h, pk_dsa);
+    if (has_b) {
+        tmem_ld16(t_s + 16 * (h + 2), sa);
+        tmem_ld16(t_dp + 16 * (h + 2), pa);
+        load16_row(cb2, code_b, rc, st_a, bv, l2, dl);       // the second step's table values, in flight during the updates
+    }
+    rmw8_consecutive_f32(a0, &ds[0]);
+    rmw_consecutive_f32<BW - 8>(a0 + 32, &ds[8]);
+    if (has_b) {
+        tmem_ld_wait();
+        math16_row<BW>(sa, pa, bv, l2, dl, scale, pk_p, pk_dsb, ds);
+        a0 = rc.dbias_row + code_b;
+        tmem_st8(t_s + 16 * (h + 2), pk_p);
+        tmem_st8(t_dp + 16 * (h + 2), pk_dsb);
+        rmw8_consecutive_f32(a0, &ds[0]);
+        rmw_consecutive_f32<BW - 8>(a0 + 32, &ds[8]);
+    }
+}
+
+// PADW = the window side, 9 .. 15, of a launch that lays the slots out 16 to a window row (see make_item; 0 otherwise):
+// full-width two-tile windows without mask labels then take the immediate-offset table addressing and the grouped bias-gradient updates of the 16-wide case.
+// Every slot, with or without a token, carries the bias code 16-wide geometry gives it (a (w + 32) + b with b up to 15,
+// a up to 15), so that the update addresses of a warp's 32 key rows stay distinct; a pair without a token adds 0.  Such
+// codes reach up to 16 - w table rows and 7 entries in front of the table and 7 entries behind it: each warp's
+// bias-gradient table starts `dbias_margin(w)` floats into its block (the tables of these sides leave that room).
+template <int PADW>
 __global__ void __launch_bounds__(kThreads, 1)
 swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                       const __nv_bfloat16* __restrict__ v, const __nv_bfloat16* __restrict__ d_o,
                       const float* __restrict__ bias_prep, const float* __restrict__ lse, const float* __restrict__ delta,
                       __nv_bfloat16* __restrict__ dq, __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv,
                       float* __restrict__ dbias_parts, long long n_items, int ctas_per_head) {
+    constexpr bool PAD = PADW != 0;
     extern __shared__ __align__(1024) unsigned char smem[];
     const uint32_t smem0 = smem_u32(smem);
     const uint32_t bar0 = smem0 + kOffBars;
@@ -440,7 +557,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
             int npad, ntiles;
             size_t sample_off;
             {
-                const Item x = make_item(g, cur_it);
+                const Item x = make_item(g, cur_it, PAD);
                 npad = x.npad; ntiles = x.ntiles; sample_off = (size_t)x.b * HW;
             }
             const int s = kuse % kStages;
@@ -451,7 +568,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                 ok = mbar_wait_all_relaxed(bar_acc(set), (n_tile >> 1) & 1, cta_abort);
                 if (!ok) break;
                 tc_fence_after();
-                const int slot = 32 * ((4 * t + quarter + key_interleave(g.w, ntiles) * lane) & (4 * ntiles - 1)) + lane;      // interleaved key order
+                const int slot = 32 * ((4 * t + quarter + key_interleave(PAD ? 16 : g.w, ntiles) * lane) & (4 * ntiles - 1)) + lane;      // interleaved key order
                 const int tok = lds_i32(st_a + kOffTok + 4 * slot);
                 const uint32_t rows_a = st_a + (uint32_t)((t * 128 + 32 * quarter) * kRowBytes);
                 stage_row(tq + kColDV + 64 * set, rows_a + kOffV, 1.f);
@@ -498,7 +615,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                 pending_s = -1;
             }
             if (!mbar_wait_all_relaxed(bar_empty(s), ((kuse / kStages) & 1) ^ 1, cta_abort)) break;
-            const Item x = make_item(g, cur_it);
+            const Item x = make_item(g, cur_it, PAD);
             unsigned char* st = smem + s * kStageBytes;
             const uint32_t st_a = smem0 + s * kStageBytes;
             const size_t sample_off = (size_t)x.b * HW;
@@ -507,7 +624,8 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
             float l2v[kSlotIters], dlv[kSlotIters];
             // Slots advance by a fixed step, so their window offsets (a, b) = (slot / width, slot mod width) are
             // carried along instead of divided out each time (a division is a long chain through the reciprocal unit).
-            const int ew = x.r.ew;
+            const int ew = PAD ? 16 : x.r.ew;               // slots per window row
+            const int bw = x.r.ew;                          // PAD: offsets b >= bw hold no token
             const int q_s = kLoaderThreads / ew, r_s = kLoaderThreads - q_s * ew;              // slot loop: step of kLoaderThreads
             const int q_r = (kLoaderThreads / 4) / ew, r_r = (kLoaderThreads / 4) - q_r * ew;  // row loop: step of kLoaderThreads / 4
             int a_s = lt / ew, b_s = lt - a_s * ew;
@@ -519,11 +637,13 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                 dlv[i] = 0.f;
                 if (slot >= kMaxSlots) continue;
                 int code = 0, label = 0xff, tok = -1;
-                if (slot < x.r.n) {
+                if (slot < x.r.n && (!PAD || b_s < bw)) {
                     tok = offset_token_tc(g, x.r, a_s, b_s, code, label);
                     const size_t li = (sample_off + (size_t)tok) * g.heads + head;
                     l2v[i] = __ldg(lse + li);
                     dlv[i] = __ldg(delta + li);
+                } else if (PAD) {
+                    code = a_s * cs + b_s;               // the slot's place in 16-wide geometry (see the kernel's header)
                 }
                 reinterpret_cast<int*>(st + kOffColOff)[slot] = 4 * code;
                 reinterpret_cast<int*>(st + kOffLab)[slot] = label;
@@ -537,14 +657,14 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
             const int hc = head * kD + chunk * 8;
             const int nrows = x.ntiles * 128;
             const int M = 4 * x.ntiles;
-            const int kc = key_interleave(g.w, x.ntiles);
+            const int kc = key_interleave(PAD ? 16 : g.w, x.ntiles);
             int a_r = (lt >> 2) / ew, b_r = (lt >> 2) - a_r * ew;
             for (int row = lt >> 2; row < nrows; row += kLoaderThreads / 4, a_r += q_r, b_r += r_r) {
                 if (b_r >= ew) { b_r -= ew; ++a_r; }
                 const int kl = row & 31, kw = ((row >> 5) - kc * kl) & (M - 1), krow = 128 * (kw >> 2) + 32 * (kw & 3) + kl;
                 const __nv_bfloat16 *sq = q, *sk = k, *sv = v, *sg = d_o;
                 int bytes = 0;
-                if (row < x.r.n) {
+                if (row < x.r.n && (!PAD || b_r < bw)) {
                     int code, label;
                     const int tok = offset_token_tc(g, x.r, a_r, b_r, code, label);
                     const size_t t_abs = sample_off + (size_t)tok;
@@ -619,7 +739,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
         ItemCursor nx_it = cursor_init(cta_in_head, ctas_per_head, 1, g.Mw, g.Mh);     // runs one item ahead
         int npad = 0, ntiles = 0, nblk = 1;
         if (cta_in_head < n_items) {
-            const Item x = make_item(g, nx_it);
+            const Item x = make_item(g, nx_it, PAD);
             npad = x.npad; ntiles = x.ntiles; nblk = x.nblk;
             cursor_advance(nx_it, 1, g.Mw, g.Mh);
         }
@@ -629,7 +749,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
             // the item after this one
             int nb_n = 0, npad_n = 0, nblk_n = 1, ntiles_n = 0;
             if (it + ctas_per_head < n_items) {
-                const Item xn = make_item(g, nx_it);
+                const Item xn = make_item(g, nx_it, PAD);
                 cursor_advance(nx_it, 1, g.Mw, g.Mh);
                 nb_n = xn.ntiles * xn.nblk; npad_n = xn.npad; nblk_n = xn.nblk; ntiles_n = xn.ntiles;
             }
@@ -744,14 +864,14 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
         int J = 0;                       // number of this block in the CTA's sequence; its S / dP buffer is J & 1
         ItemCursor cur_it = cursor_init(cta_in_head, ctas_per_head, 1, g.Mw, g.Mh);
         for (long long it = cta_in_head; ok && it < n_items; it += ctas_per_head, ++kuse, cursor_advance(cur_it, 1, g.Mw, g.Mh)) {
-            const Item x = make_item(g, cur_it);
+            const Item x = make_item(g, cur_it, PAD);
             const int s = kuse % kStages;
             const uint32_t st_a = smem0 + s * kStageBytes;
             if (!mbar_wait_all(bar_full(s), (kuse / kStages) & 1, cta_abort)) break;
             for (int t = 0; t < x.ntiles && ok; ++t) {
                 const int krow = 32 * quarter + lane;            // key row inside the tile
                 const int M = 4 * x.ntiles;
-                const int slot = 32 * ((4 * t + quarter + key_interleave(g.w, x.ntiles) * lane) & (M - 1)) + lane;     // interleaved key order
+                const int slot = 32 * ((4 * t + quarter + key_interleave(PAD ? 16 : g.w, x.ntiles) * lane) & (M - 1)) + lane;     // interleaved key order
                 // Bias-gradient updates.  In a full-width window (width = w) the bias code of a slot is the slot
                 // number plus 32 per window row, so code mod 32 = slot mod 32 = lane: the 32 updates of one warp
                 // instruction (32 keys, one query) fall into 32 different banks and entries.  If w also divides 32
@@ -765,11 +885,12 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                 // window of side 9 .. 16 (checked exhaustively on the host over all heights; the parity tests cover
                 // sides 12 and 14).  Other windows are updated one query at a time.
                 int rmw_mode = 1;
-                if (x.r.ew == g.w && g.w >= 4) {
+                if (!PAD && x.r.ew == g.w && g.w >= 4) {
                     if ((32 % g.w) == 0) rmw_mode = (M == 8 && g.w >= 8) ? 8 : 4;
                     else if (M == 8) rmw_mode = 4;
                 }
-                const bool row16 = g.w == 16 && x.r.n == 256 && !x.masked;    // full 16 x 16 window: update groups of 8 apply as well
+                // full 16 x 16 window: update groups of 8 apply as well; PAD: every two-tile window without mask labels
+                const bool row16 = PAD ? (M == 8 && !x.masked && x.r.ew == PADW) : (g.w == 16 && x.r.n == 256 && !x.masked);
                 const int coloff_i = lds_i32(st_a + kOffColOff + 4 * slot);
                 const int tok = lds_i32(st_a + kOffTok + 4 * slot);
                 RowCtx rc;
@@ -777,7 +898,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                 rc.valid = tok >= 0;
                 // bias index = code_query - code_key + c0; a key row without a token reads the table's -inf zone
                 rc.bias_row = smem0 + kOffBias + (rc.valid ? 4 * c0 - coloff_i : 4 * (2 * c0 + 1));
-                rc.dbias_row = smem0 + kOffDBias + 4 * (warp * kDBiasFloats + c0) - coloff_i;
+                rc.dbias_row = smem0 + kOffDBias + 4 * (warp * kDBiasFloats + c0 + (PAD ? dbias_margin(g.w) : 0)) - coloff_i;
                 rc.scratch = smem0 + kOffDBias + 4 * (warp * kDBiasFloats + kDBiasEntries + lane);
                 for (int b = 0; b < x.nblk; ++b) {
                     const int buf = J & 1;
@@ -793,7 +914,9 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                     uint32_t sa[16], pa[16], pk_p[8], pk_dsa[8], pk_dsb[8], addr[16];
                     float ds[16];
                     const int ca = b * CB + 16 * h, cb2 = ca + 32;
-                    if (row16) {
+                    if (row16 && PAD) {
+                        if (has_a) pad_block16<PAD ? PADW : 15>(t_s, t_dp, h, ca, cb2, cs, has_b, rc, st_a, scale, pk_dsa, pk_dsb);
+                    } else if (row16) {
                         // full 16 x 16 window (four steps per block, no mask): one window row per step
                         tmem_ld16(t_s + 16 * h, sa);
                         tmem_ld16(t_dp + 16 * h, pa);
@@ -883,7 +1006,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
             float acc = 0.f;
 #pragma unroll
             for (int wq = 0; wq < 8; ++wq) acc += tbl[wq * kDBiasFloats + e];
-            dbias_parts[(size_t)blockIdx.x * kDBiasFloats + e] = acc;
+            dbias_parts[(size_t)blockIdx.x * kDBiasFloats + e] = acc;       // (PAD: the table starts dbias_margin(w) floats in)
         }
     }
     if (tid == 0 && *cta_abort) atomicExch(&g_bwd_tc_timeout, 1);
@@ -892,12 +1015,13 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
 // dbias[(da, db), head] = sum over the head's CTAs of their tables (entry (da + w - 1) * cs + (db + w - 1)).
 // Fixed summation order over warps and CTAs: the bias gradient is reproducible run to run.
 __global__ void __launch_bounds__(256)
-swin_bwd_dbias_finalize_kernel(const float* __restrict__ parts, float* __restrict__ dbias, int w, int heads, int ctas_per_head) {
+swin_bwd_dbias_finalize_kernel(const float* __restrict__ parts, float* __restrict__ dbias, int w, int heads, int ctas_per_head,
+                               int margin) {
     const int nw = 2 * w - 1, cs = w + 32;
     const int i = blockIdx.x * blockDim.x + threadIdx.x;       // (table row, head)
     if (i >= nw * nw * heads) return;
     const int head = i % heads, r = i / heads;
-    const int e = (r / nw) * cs + (r % nw);
+    const int e = margin + (r / nw) * cs + (r % nw);
     float acc = 0.f;
     for (int c = 0; c < ctas_per_head; ++c) acc += parts[(size_t)(c * heads + head) * kDBiasFloats + e];
     dbias[i] = acc;
@@ -942,17 +1066,32 @@ cudaError_t launch_bwd_tc(const Geo& g, const void* q, const void* k, const void
     if (cph < 1) cph = 1;
     if (cph > items) cph = items;
     const unsigned grid = (unsigned)(cph * g.heads);
-    e = cudaFuncSetAttribute(swin_bwd_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    // window sides 9 .. 15: the layout of 16 slots per window row (TERRA_NO_PAD16=1: a debugging switch that keeps the packed layout)
+    static const bool pad_off = [] { const char* e_ = std::getenv("TERRA_NO_PAD16"); return e_ && e_[0] == '1'; }();
+    const bool pad = g.w > 8 && g.w < 16 && !pad_off;
+    auto kern = swin_bwd_fused_kernel<0>;
+    if (pad) {
+        switch (g.w) {
+            case 9: kern = swin_bwd_fused_kernel<9>; break;
+            case 10: kern = swin_bwd_fused_kernel<10>; break;
+            case 11: kern = swin_bwd_fused_kernel<11>; break;
+            case 12: kern = swin_bwd_fused_kernel<12>; break;
+            case 13: kern = swin_bwd_fused_kernel<13>; break;
+            case 14: kern = swin_bwd_fused_kernel<14>; break;
+            default: kern = swin_bwd_fused_kernel<15>; break;
+        }
+    }
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
     prof_begin("swin_bwd_fused_kernel", stream);
-    swin_bwd_fused_kernel<<<grid, kThreads, kSmemBytes, stream>>>(
+    kern<<<grid, kThreads, kSmemBytes, stream>>>(
         g, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, (const __nv_bfloat16*)d_o, prep, lse, delta,
         (__nv_bfloat16*)dq, (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, parts, items, (int)cph);
     count_launch(stream);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     const int nrows = (2 * g.w - 1) * (2 * g.w - 1) * g.heads;
-    swin_bwd_dbias_finalize_kernel<<<(nrows + 255) / 256, 256, 0, stream>>>(parts, dbias, g.w, g.heads, (int)cph);
+    swin_bwd_dbias_finalize_kernel<<<(nrows + 255) / 256, 256, 0, stream>>>(parts, dbias, g.w, g.heads, (int)cph, pad ? dbias_margin(g.w) : 0);
     count_launch(stream);
     return cudaGetLastError();
 }

@@ -100,12 +100,15 @@ struct Item {
     bool masked;   // the window mixes shift-mask labels
 };
 
-__device__ __forceinline__ Item make_item(const Geo& g, const ItemCursor& c) {
+// pad16: the window's slots are laid out 16 to a window row (slot = 16 a + b; the slots with b >= the window's width
+// hold no token), so that every group of 16 key columns is one window row whatever the window side
+__device__ __forceinline__ Item make_item(const Geo& g, const ItemCursor& c, bool pad16 = false) {
     Item x;
     x.head = c.head;
     x.win = c.wr * g.Mw + c.wc;
     x.b = c.b;
     x.r = window_ref_rc(g, c.wr, c.wc);
+    if (pad16) x.r.n = x.r.eh * 16;
     x.npad = (x.r.n + 15) & ~15;
     x.ntiles = (x.r.n + 127) >> 7;
     // rolled rows >= H - sh (columns >= W - sw) hold the tokens that wrapped across a non-periodic edge
@@ -213,19 +216,33 @@ __device__ __forceinline__ float lds_f32_at(uint32_t addr) {
 // 16 key columns that are one window row of a full 16 x 16 window without mask labels: their bias entries are
 // consecutive (descending with the key), so each address is one base plus an immediate offset.  `top` = shared
 // address of the entry of the row's first key.
+// BW < 16: only the row's first BW keys hold a token; the others get P = 0 and cost nothing.
+template <int BW = 16>
 __device__ __forceinline__ void softmax_cols16_row(const uint32_t* r, uint32_t* pk, uint32_t top, float scale, float neg_m) {
     const uint32_t bb = top - 60;
     float bv[16];
     bv[0] = lds_f32_at<60>(bb);  bv[1] = lds_f32_at<56>(bb);  bv[2] = lds_f32_at<52>(bb);  bv[3] = lds_f32_at<48>(bb);
     bv[4] = lds_f32_at<44>(bb);  bv[5] = lds_f32_at<40>(bb);  bv[6] = lds_f32_at<36>(bb);  bv[7] = lds_f32_at<32>(bb);
-    bv[8] = lds_f32_at<28>(bb);  bv[9] = lds_f32_at<24>(bb);  bv[10] = lds_f32_at<20>(bb); bv[11] = lds_f32_at<16>(bb);
-    bv[12] = lds_f32_at<12>(bb); bv[13] = lds_f32_at<8>(bb);  bv[14] = lds_f32_at<4>(bb);  bv[15] = lds_f32_at<0>(bb);
+    if (BW > 8) bv[8] = lds_f32_at<28>(bb);
+    if (BW > 9) bv[9] = lds_f32_at<24>(bb);
+    if (BW > 10) bv[10] = lds_f32_at<20>(bb);
+    if (BW > 11) bv[11] = lds_f32_at<16>(bb);
+    if (BW > 12) bv[12] = lds_f32_at<12>(bb);
+    if (BW > 13) bv[13] = lds_f32_at<8>(bb);
+    if (BW > 14) bv[14] = lds_f32_at<4>(bb);
+    if (BW > 15) bv[15] = lds_f32_at<0>(bb);
 #pragma unroll
     for (int e2 = 0; e2 < 8; ++e2) {
-        float x0, x1;
-        fma2(x0, x1, __uint_as_float(r[2 * e2]), __uint_as_float(r[2 * e2 + 1]), scale, bv[2 * e2], bv[2 * e2 + 1]);
-        add2(x0, x1, x0, x1, neg_m);
-        pk[e2] = pack_elem(fast_exp2(x0), fast_exp2(x1));
+        if (2 * e2 + 1 < BW) {
+            float x0, x1;
+            fma2(x0, x1, __uint_as_float(r[2 * e2]), __uint_as_float(r[2 * e2 + 1]), scale, bv[2 * e2], bv[2 * e2 + 1]);
+            add2(x0, x1, x0, x1, neg_m);
+            pk[e2] = pack_elem(fast_exp2(x0), fast_exp2(x1));
+        } else if (2 * e2 < BW) {
+            pk[e2] = pack_elem(fast_exp2(fmaf(__uint_as_float(r[2 * e2]), scale, bv[2 * e2]) + neg_m), 0.f);
+        } else {
+            pk[e2] = 0u;
+        }
     }
 }
 
@@ -236,6 +253,15 @@ __device__ __forceinline__ void max_cols(const uint32_t (&r)[N], float (&mx)[4])
 #pragma unroll
         for (int a = 0; a < 4; ++a)
             mx[a] = max3(mx[a], __uint_as_float(r[e + 2 * a]), __uint_as_float(r[e + 2 * a + 1]));
+    }
+}
+// the same over the first BW of every 16 columns only (the others are key slots without a token)
+template <int N, int BW>
+__device__ __forceinline__ void max_cols_width(const uint32_t (&r)[N], float (&mx)[4]) {
+#pragma unroll
+    for (int e = 0; e < N; e += 2) {
+        if ((e & 15) + 1 < BW) mx[(e >> 1) & 3] = max3(mx[(e >> 1) & 3], __uint_as_float(r[e]), __uint_as_float(r[e + 1]));
+        else if ((e & 15) < BW) mx[(e >> 1) & 3] = fmaxf(mx[(e >> 1) & 3], __uint_as_float(r[e]));
     }
 }
 // the same over the first `nv` of N columns only (the others are key slots without a token: zero rows, raw score 0)
@@ -249,10 +275,13 @@ __device__ __forceinline__ void max_cols_limit(const uint32_t (&r)[N], int nv, f
 // flight while the current one is processed.  Returns m (log2 domain); the row sum goes to sum_out.
 // ROW16: full 16 x 16 window without mask labels (npad = 256); `top0` = shared address of the bias entry of key 0
 // for this query, `row_step` = bytes between the entries of keys one window row apart.
-template <bool MASKED, bool ROW16 = false>
+// BW < 16 (with ROW16): of every 16 columns only the first BW are keys with a token; the others are left out of the
+// maximum and get P = 0.
+template <bool MASKED, bool ROW16 = false, int BW = 16>
 __device__ __forceinline__ float softmax_row(uint32_t t_s, int npad, int nvalid, uint32_t bias_i, uint32_t a_kc, uint32_t a_klab,
                                              int label_i, float scale, float bmax, float& sum_out, uint32_t bar_half,
                                              uint32_t top0 = 0, uint32_t row_step = 0) {
+    constexpr bool COLMASK = BW < 16;
     const int nfull = npad >> 5;
     const bool tail = (npad & 16) != 0;
     uint32_t ra[32], rb[32];
@@ -285,15 +314,23 @@ __device__ __forceinline__ float softmax_row(uint32_t t_s, int npad, int nvalid,
             tmem_ld32(t_s + 32 * (i + 2), rc);
             tmem_ld32(t_s + 32 * (i + 3), rd);
             tmem_ld_wait();
-            max_cols<32>(ra, mx4);
-            max_cols<32>(rb, mx4);
-            max_cols<32>(rc, mx4);
-            max_cols<32>(rd, mx4);
+            if (COLMASK) {
+                max_cols_width<32, BW>(ra, mx4);
+                max_cols_width<32, BW>(rb, mx4);
+                max_cols_width<32, BW>(rc, mx4);
+                max_cols_width<32, BW>(rd, mx4);
+            } else {
+                max_cols<32>(ra, mx4);
+                max_cols<32>(rb, mx4);
+                max_cols<32>(rc, mx4);
+                max_cols<32>(rd, mx4);
+            }
         }
         for (; i < nplain; ++i) {
             tmem_ld32(t_s + 32 * i, ra);
             tmem_ld_wait();
-            max_cols<32>(ra, mx4);
+            if (COLMASK) max_cols_width<32, BW>(ra, mx4);
+            else max_cols<32>(ra, mx4);
         }
         if (i < nfull) {                       // last full group, with a ragged end
             tmem_ld32(t_s + 32 * i, ra);
@@ -305,6 +342,7 @@ __device__ __forceinline__ float softmax_row(uint32_t t_s, int npad, int nvalid,
             tmem_ld16(t_s + 32 * nfull, rt);
             tmem_ld_wait();
             if (limit) max_cols_limit<16>(rt, nvalid - 32 * nfull, mx4);
+            else if (COLMASK) max_cols_width<16, BW>(rt, mx4);
             else max_cols<16>(rt, mx4);
         }
         const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
@@ -319,8 +357,8 @@ __device__ __forceinline__ float softmax_row(uint32_t t_s, int npad, int nvalid,
         tmem_ld_wait();
         if (i + 1 < nfull) tmem_ld32(t_s + 32 * (i + 1), rb);
         if (ROW16) {
-            softmax_cols16_row(&ra[0], &pk[0], top0 - (2 * i) * row_step, scale, neg_m);
-            softmax_cols16_row(&ra[16], &pk[8], top0 - (2 * i + 1) * row_step, scale, neg_m);
+            softmax_cols16_row<BW>(&ra[0], &pk[0], top0 - (2 * i) * row_step, scale, neg_m);
+            softmax_cols16_row<BW>(&ra[16], &pk[8], top0 - (2 * i + 1) * row_step, scale, neg_m);
         } else {
             sum += softmax_cols<32, MASKED>(ra, pk, 32 * i, bias_i, a_kc, a_klab, label_i, scale, neg_m);
         }
@@ -329,8 +367,8 @@ __device__ __forceinline__ float softmax_row(uint32_t t_s, int npad, int nvalid,
             tmem_ld_wait();
             if (i + 2 < nfull) tmem_ld32(t_s + 32 * (i + 2), ra);
             if (ROW16) {
-                softmax_cols16_row(&rb[0], &pk[0], top0 - (2 * i + 2) * row_step, scale, neg_m);
-                softmax_cols16_row(&rb[16], &pk[8], top0 - (2 * i + 3) * row_step, scale, neg_m);
+                softmax_cols16_row<BW>(&rb[0], &pk[0], top0 - (2 * i + 2) * row_step, scale, neg_m);
+                softmax_cols16_row<BW>(&rb[16], &pk[8], top0 - (2 * i + 3) * row_step, scale, neg_m);
             } else {
                 sum += softmax_cols<32, MASKED>(rb, pk, 32 * (i + 1), bias_i, a_kc, a_klab, label_i, scale, neg_m);
             }
@@ -366,12 +404,16 @@ struct FwdMaps {
 // TMA = the window rows are fetched by tiled tensor copies (one per window row and tensor, issued by the lanes of
 // ONE producer warp, the head's bias table by one bulk copy) instead of 16-byte cp.async copies from three loader
 // warps.  For grids of 16-wide windows whose every window row is one run of consecutive tokens in memory.
-template <bool W16, bool TMA>
+// PADW = the window side, 9 .. 15, of a launch that lays the slots out 16 to a window row (see make_item): full-width
+// windows without mask labels then take the immediate-offset addressing of the 16-wide case, with the columns beyond the
+// window's width (a compile-time number) left out at no cost; 0 otherwise.  Never together with W16 or TMA.
+template <bool W16, bool TMA, int PADW = 0>
 __global__ void __launch_bounds__(kThreads, 1)
 swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                    const __nv_bfloat16* __restrict__ v, const float* __restrict__ bias_prep,
                    __nv_bfloat16* __restrict__ o, float* __restrict__ lse, long long n_items,
                    const __grid_constant__ FwdMaps maps) {
+    constexpr bool PAD = PADW != 0;
     extern __shared__ __align__(1024) unsigned char smem[];
     const uint32_t smem0 = smem_u32(smem);
     const uint32_t bar0 = smem0 + kStages * kStageBytes;
@@ -435,7 +477,7 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
             for (long long it = blockIdx.x; it < n_items; it += gridDim.x, ++kuse, cursor_advance(cur_it, g.heads, g.Mw, g.Mh)) {
                 const int s = kuse % kStages;
                 if (!mbar_wait_all(bar_empty(s), ((kuse / kStages) & 1) ^ 1, cta_abort)) break;
-                const Item x = make_item(g, cur_it);
+                const Item x = make_item(g, cur_it, PAD);
                 unsigned char* st = smem + s * kStageBytes;
                 const uint32_t st_a = smem0 + s * kStageBytes;
                 const int ew = x.r.ew;                       // 16, or 8 in the last window column
@@ -502,7 +544,7 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
                 pending_s = -1;
             }
             if (!mbar_wait_all_relaxed(bar_empty(s), ((kuse / kStages) & 1) ^ 1, cta_abort)) break;
-            const Item x = make_item(g, cur_it);
+            const Item x = make_item(g, cur_it, PAD);
             unsigned char* st = smem + s * kStageBytes;
             const uint32_t st_a = smem0 + s * kStageBytes;
             int* s_kc = reinterpret_cast<int*>(st + kOffKc);
@@ -513,14 +555,15 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
 
             // Slots advance by a fixed step, so their window offsets (a, b) = (slot / width, slot mod width) are
             // carried along instead of divided out each time (a division is a long chain through the reciprocal unit).
-            const int ew = x.r.ew;
+            const int ew = PAD ? 16 : x.r.ew;               // slots per window row
+            const int bw = x.r.ew;                          // PAD: offsets b >= bw hold no token
             const int q_s = kLoaderThreads / ew, r_s = kLoaderThreads - q_s * ew;              // slot loop: step of kLoaderThreads
             const int q_r = (kLoaderThreads / 4) / ew, r_r = (kLoaderThreads / 4) - q_r * ew;  // row loop: step of kLoaderThreads / 4
             int a_s = lt / ew, b_s = lt - a_s * ew;
             for (int slot = lt; slot < kMaxSlots; slot += kLoaderThreads) {
                 // a slot without a token: as a key its bias index lands in the table's -inf zone
                 int code = 0, label = 0xff, tok = -1, kc = 4 * (2 * c0 + 1);
-                if (slot < x.r.n) {
+                if (slot < x.r.n && (!PAD || b_s < bw)) {
                     tok = offset_token_tc(g, x.r, a_s, b_s, code, label);
                     kc = 4 * (c0 - code);
                 }
@@ -537,7 +580,7 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
             for (int row = lt >> 2; row < x.npad; row += kLoaderThreads / 4) {
                 const __nv_bfloat16 *sq = q, *sk = k, *sv = v;
                 int bytes = 0;   // rows past the window's end are written as zeros
-                if (row < x.r.n) {
+                if (row < x.r.n && (!PAD || b_r < bw)) {
                     int code, label;
                     const int tok = offset_token_tc(g, x.r, a_r, b_r, code, label);
                     const size_t off = (sample_off + (size_t)tok) * g.ts + x.head * kD + chunk * 8;
@@ -610,7 +653,7 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
             ItemCursor nx_it = cursor_init(blockIdx.x, gridDim.x, g.heads, g.Mw, g.Mh);     // runs one item ahead
             Item cur;
             if (it < n_items) {
-                cur = make_item(g, nx_it);
+                cur = make_item(g, nx_it, PAD);
                 cursor_advance(nx_it, g.heads, g.Mw, g.Mh);
                 ok = mbar_wait_all(bar_full(0), 0, cta_abort);
                 if (ok) {
@@ -626,7 +669,7 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
                 Item nx;
                 const int sn = (kuse + 1) % kStages;
                 if (has_next) {
-                    nx = make_item(g, nx_it);
+                    nx = make_item(g, nx_it, PAD);
                     cursor_advance(nx_it, g.heads, g.Mw, g.Mh);
                 }
                 bool next_ready = false;
@@ -690,7 +733,7 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
         int kuse = 0, use = 0;
         ItemCursor cur_it = cursor_init(blockIdx.x, gridDim.x, g.heads, g.Mw, g.Mh);
         for (long long it = blockIdx.x; it < n_items; it += gridDim.x, ++kuse, cursor_advance(cur_it, g.heads, g.Mw, g.Mh)) {
-            const Item x = make_item(g, cur_it);
+            const Item x = make_item(g, cur_it, PAD);
             const int s = kuse % kStages;
             const uint32_t st_a = smem0 + s * kStageBytes;
             // Every warpgroup follows the stage ring item by item, also the second one through items that have no
@@ -712,7 +755,14 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
             tc_fence_after();
             float m, sum;
             const bool wide = bmax == INFINITY;      // the head's bias table spreads too far for the bound on the row maximum
-            if (W16) {
+            if (PAD) {
+                // full-width windows without mask labels: the row path, compiled for this width; the others: by the tables
+                if (x.masked || wide || x.r.ew != PADW)
+                    m = softmax_row<true>(t_s, x.npad, x.r.n, bias_i, st_a + kOffKc, st_a + kOffKlab, label_i, scale, bmax, sum, bar_phalf(wg));
+                else
+                    m = softmax_row<false, true, PAD ? PADW : 16>(t_s, x.npad, x.r.n, bias_i, st_a + kOffKc, st_a + kOffKlab, label_i, scale, bmax,
+                                                                  sum, bar_phalf(wg), bias_i + 4 * c0, 4 * cs);
+            } else if (W16) {
                 if (x.masked || x.r.n != 256 || wide)
                     m = softmax_row<true>(t_s, x.npad, x.r.n, bias_i, st_a + kOffKc, st_a + kOffKlab, label_i, scale, bmax, sum, bar_phalf(wg));
                 else
@@ -892,7 +942,21 @@ cudaError_t launch_fwd_tc(const Geo& g, const void* q, const void* k, const void
     const bool tma = !tma_off && tma_row_shape(g) && make_row_map(&maps.q16, g, q, g.ts, 16) && make_row_map(&maps.k16, g, k, g.ts, 16) &&
                      make_row_map(&maps.v16, g, v, g.ts, 16) && make_row_map(&maps.q8, g, q, g.ts, 8) && make_row_map(&maps.k8, g, k, g.ts, 8) &&
                      make_row_map(&maps.v8, g, v, g.ts, 8);
+    // window sides 9 .. 15: the layout of 16 slots per window row (TERRA_NO_PAD16=1: a debugging switch that keeps the packed layout)
+    static const bool pad_off = [] { const char* e_ = std::getenv("TERRA_NO_PAD16"); return e_ && e_[0] == '1'; }();
+    const bool pad = g.w > 8 && g.w < 16 && !pad_off;
     auto kern = tma ? swin_fwd_tc_kernel<true, true> : (g.w == 16 ? swin_fwd_tc_kernel<true, false> : swin_fwd_tc_kernel<false, false>);
+    if (pad) {
+        switch (g.w) {
+            case 9: kern = swin_fwd_tc_kernel<false, false, 9>; break;
+            case 10: kern = swin_fwd_tc_kernel<false, false, 10>; break;
+            case 11: kern = swin_fwd_tc_kernel<false, false, 11>; break;
+            case 12: kern = swin_fwd_tc_kernel<false, false, 12>; break;
+            case 13: kern = swin_fwd_tc_kernel<false, false, 13>; break;
+            case 14: kern = swin_fwd_tc_kernel<false, false, 14>; break;
+            default: kern = swin_fwd_tc_kernel<false, false, 15>; break;
+        }
+    }
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
     const unsigned grid = (unsigned)(items < sm_count ? items : sm_count);
