@@ -57,3 +57,30 @@ def test_grouped_updates_never_meet_and_full_width_rows_are_bank_conflict_free(w
         # every slot of every tile is held by exactly one (warp, lane)
         held = sorted(32 * ((W + c * lane) % M) + lane for W in range(M) for lane in range(32))
         assert held == list(range(128 * ntiles))
+
+
+@pytest.mark.parametrize("w", range(9, 16))
+def test_sixteen_slots_per_window_row_layout_of_sides_9_to_15(w):
+    """Sides 9 .. 15 with 16 slots per window row: every one of the 256 slots, with or without a token, carries the
+    code a (w + 32) + b of 16-wide geometry; key order c = 1; groups of 8 queries for two-tile windows.  The 32 x 8
+    entries of a group are pairwise distinct, and with the kernel's margin in front of the table every entry that any
+    (key slot, query column) pair can address lies inside the warp's 1472-float block."""
+    cs, c0 = w + 32, (w - 1) * (w + 33)
+    margin = (16 - w) * (w + 32) + 8                      # the kernel's dbias_margin(w)
+    entries_of_table = 1472
+
+    def code(slot):
+        return (slot // 16) * cs + slot % 16
+
+    for eh in range(9, w + 1):                            # two tiles: 16 eh > 128
+        n = 16 * eh
+        for W in range(8):
+            slots = [32 * ((W + lane) % 8) + lane for lane in range(32)]
+            for q0 in range(0, n, 8):
+                entries = [code(q) - code(ks) for ks in slots for q in range(q0, q0 + 8)]
+                assert len(entries) == len(set(entries)), (w, eh, W, q0)
+                lo, hi = min(entries) + c0 + margin, max(entries) + c0 + margin
+                assert 0 <= lo and hi < entries_of_table, (w, eh, lo, hi)
+    # the entries of pairs that hold tokens are those of the packed layout: (a_q - a_k + w - 1) cs + (b_q - b_k + w - 1)
+    for aq, bq, ak, bk in ((0, 0, w - 1, w - 1), (w - 1, w - 1, 0, 0), (3, w - 1, 5, 0)):
+        assert code(16 * aq + bq) - code(16 * ak + bk) + c0 == (aq - ak + w - 1) * cs + (bq - bk + w - 1)
