@@ -23,6 +23,7 @@ SHAPES = [
     ("f16_d32_w16_complete", 2, 32, 64, 3, 32, 16, 8, 0, 0, 1),
     ("f16_d64_w16_complete", 1, 32, 48, 2, 64, 16, 8, 8, 0, 0),
     ("f16_d128_w64_complete", 1, 64, 128, 2, 128, 64, 16, 40, 0, 0),  # staged bias rows; query side by exchanged roles
+    ("f16_d32_w12", 1, 40, 62, 2, 32, 12, 6, 6, 0, 1),                # 16 slots per window row, full-width and truncated windows
 ]
 
 
