@@ -97,9 +97,11 @@ constexpr int kColDV = 256;         // accumulator set s: dV at 256 + 64 s, dK a
 constexpr int kColDK = 288;
 constexpr int kColDQ = 384;         // dQ of query pair p at 384 + 32 p
 
-__device__ __forceinline__ int code_stride(int w) { return w + 32; }
+// (48, the stride of side 16, in the layout of 16 slots per window row: code = slot + 32 a again, so a warp's 32 key
+// rows update 32 different banks)
+__device__ __forceinline__ int code_stride(int w, bool pad16 = false) { return pad16 ? 48 : w + 32; }
 // floats in front of a warp's bias-gradient table in the 16-slots-per-row layout of window sides 9 .. 15
-__host__ __device__ __forceinline__ int dbias_margin(int w) { return (16 - w) * (w + 32) + 8; }
+__host__ __device__ __forceinline__ int dbias_margin(int w) { return (16 - w) * 48 + 8; }
 
 // Key rows of a tile are interleaved over the elementwise warps: lane l of warp W = 4 t + quarter holds slot
 // 32 ((W + c l) mod M) + l, M = 4 * (tiles in use).  c = 1, except c = 5 for two-tile windows whose side does not
@@ -136,13 +138,13 @@ __device__ __forceinline__ Item make_item(const Geo& g, const ItemCursor& c, boo
 }
 
 // window offset (a, b) -> grid token, bias code and shift-mask label
-__device__ __forceinline__ int offset_token_tc(const Geo& g, const WindowRef& r, int a, int b, int& code, int& label) {
+__device__ __forceinline__ int offset_token_tc(const Geo& g, const WindowRef& r, int a, int b, int cs, int& code, int& label) {
     int u = r.wr * g.w + a + g.sh;
     if (u >= g.H) u -= g.H;
     int v = r.wc * g.w + b + g.sw;
     if (v >= g.W) v -= g.W;
     label = ((!g.ph && u < g.sh) ? 2 : 0) + ((!g.pw && v < g.sw) ? 1 : 0);
-    code = a * code_stride(g.w) + b;
+    code = a * cs + b;
     return u * g.W + v;
 }
 
@@ -445,8 +447,8 @@ __device__ __forceinline__ void pad_block16(uint32_t t_s, uint32_t t_dp, int h, 
 
 // PADW = the window side, 9 .. 15, of a launch that lays the slots out 16 to a window row (see make_item; 0 otherwise):
 // full-width two-tile windows without mask labels then take the immediate-offset table addressing and the grouped bias-gradient updates of the 16-wide case.
-// Every slot, with or without a token, carries the bias code 16-wide geometry gives it (a (w + 32) + b with b up to 15,
-// a up to 15), so that the update addresses of a warp's 32 key rows stay distinct; a pair without a token adds 0.  Such
+// Every slot, with or without a token, carries the bias code 16-wide geometry gives it (48 a + b with a, b up to 15,
+// the code stride of side 16), so that the update addresses of a warp's 32 key rows stay distinct; a pair without a token adds 0.  Such
 // codes reach up to 16 - w table rows and 7 entries in front of the table and 7 entries behind it: each warp's
 // bias-gradient table starts `dbias_margin(w)` floats into its block (the tables of these sides leave that room).
 template <int PADW>
@@ -511,7 +513,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    const int cs = code_stride(g.w);
+    const int cs = code_stride(g.w, PAD);
     const int c0 = (g.w - 1) * (cs + 1);
     const size_t HW = (size_t)g.H * g.W;
 
@@ -638,7 +640,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                 if (slot >= kMaxSlots) continue;
                 int code = 0, label = 0xff, tok = -1;
                 if (slot < x.r.n && (!PAD || b_s < bw)) {
-                    tok = offset_token_tc(g, x.r, a_s, b_s, code, label);
+                    tok = offset_token_tc(g, x.r, a_s, b_s, cs, code, label);
                     const size_t li = (sample_off + (size_t)tok) * g.heads + head;
                     l2v[i] = __ldg(lse + li);
                     dlv[i] = __ldg(delta + li);
@@ -666,7 +668,7 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
                 int bytes = 0;
                 if (row < x.r.n && (!PAD || b_r < bw)) {
                     int code, label;
-                    const int tok = offset_token_tc(g, x.r, a_r, b_r, code, label);
+                    const int tok = offset_token_tc(g, x.r, a_r, b_r, cs, code, label);
                     const size_t t_abs = sample_off + (size_t)tok;
                     const size_t off = t_abs * g.ts + hc;
                     sq = q + off; sk = k + off; sv = v + off;
@@ -1016,8 +1018,8 @@ swin_bwd_fused_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __
 // Fixed summation order over warps and CTAs: the bias gradient is reproducible run to run.
 __global__ void __launch_bounds__(256)
 swin_bwd_dbias_finalize_kernel(const float* __restrict__ parts, float* __restrict__ dbias, int w, int heads, int ctas_per_head,
-                               int margin) {
-    const int nw = 2 * w - 1, cs = w + 32;
+                               int margin, int cs) {
+    const int nw = 2 * w - 1;
     const int i = blockIdx.x * blockDim.x + threadIdx.x;       // (table row, head)
     if (i >= nw * nw * heads) return;
     const int head = i % heads, r = i / heads;
@@ -1066,9 +1068,7 @@ cudaError_t launch_bwd_tc(const Geo& g, const void* q, const void* k, const void
     if (cph < 1) cph = 1;
     if (cph > items) cph = items;
     const unsigned grid = (unsigned)(cph * g.heads);
-    // window sides 9 .. 15: the layout of 16 slots per window row (TERRA_NO_PAD16=1: a debugging switch that keeps the packed layout)
-    static const bool pad_off = [] { const char* e_ = std::getenv("TERRA_NO_PAD16"); return e_ && e_[0] == '1'; }();
-    const bool pad = g.w > 8 && g.w < 16 && !pad_off;
+    const bool pad = pad16_layout(g);       // window sides 9 .. 15: 16 slots per window row
     auto kern = swin_bwd_fused_kernel<0>;
     if (pad) {
         switch (g.w) {
@@ -1091,7 +1091,8 @@ cudaError_t launch_bwd_tc(const Geo& g, const void* q, const void* k, const void
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     const int nrows = (2 * g.w - 1) * (2 * g.w - 1) * g.heads;
-    swin_bwd_dbias_finalize_kernel<<<(nrows + 255) / 256, 256, 0, stream>>>(parts, dbias, g.w, g.heads, (int)cph, pad ? dbias_margin(g.w) : 0);
+    swin_bwd_dbias_finalize_kernel<<<(nrows + 255) / 256, 256, 0, stream>>>(parts, dbias, g.w, g.heads, (int)cph, pad ? dbias_margin(g.w) : 0,
+                                                                            pad ? 48 : g.w + 32);
     count_launch(stream);
     return cudaGetLastError();
 }

@@ -90,7 +90,9 @@ __device__ __forceinline__ int p_col(int chunk32) { return chunk32 < 4 ? 16 * ch
 
 // Bias codes use a row stride of w + 32 instead of 2w - 1: the 32 rows of a warp (consecutive slots of a
 // full-width window) then read 32 different shared-memory banks.
-__device__ __forceinline__ int code_stride(int w) { return w + 32; }
+// (In the layout of 16 slots per window row the stride is that of side 16, 48: a warp's 32 consecutive slots are two
+// window rows, 48 = 16 mod 32 codes apart, and again read 32 different banks.)
+__device__ __forceinline__ int code_stride(int w, bool pad16 = false) { return pad16 ? 48 : w + 32; }
 
 struct Item {
     int b, win, head;
@@ -120,13 +122,13 @@ __device__ __forceinline__ Item make_item(const Geo& g, const ItemCursor& c, boo
 }
 
 // window offset (a, b) -> grid token, bias code a * (w + 32) + b and shift-mask label
-__device__ __forceinline__ int offset_token_tc(const Geo& g, const WindowRef& r, int a, int b, int& code, int& label) {
+__device__ __forceinline__ int offset_token_tc(const Geo& g, const WindowRef& r, int a, int b, int cs, int& code, int& label) {
     int u = r.wr * g.w + a + g.sh;
     if (u >= g.H) u -= g.H;
     int v = r.wc * g.w + b + g.sw;
     if (v >= g.W) v -= g.W;
     label = ((!g.ph && u < g.sh) ? 2 : 0) + ((!g.pw && v < g.sw) ? 1 : 0);
-    code = a * code_stride(g.w) + b;
+    code = a * cs + b;
     return u * g.W + v;
 }
 
@@ -462,7 +464,7 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    const int cs = code_stride(g.w);
+    const int cs = code_stride(g.w, PAD);
     const int c0 = (g.w - 1) * (cs + 1);     // code of the last in-window offset; bias index = code_q - code_k + c0
     const size_t HW = (size_t)g.H * g.W;
 
@@ -508,7 +510,7 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
                         const int slot = 8 * lane + i;
                         int code = 0, label = 0xff, tok = -1, kc = 4 * (2 * c0 + 1);
                         if (slot < x.r.n) {
-                            tok = offset_token_tc(g, x.r, a_s, b_s, code, label);
+                            tok = offset_token_tc(g, x.r, a_s, b_s, cs, code, label);
                             kc = 4 * (c0 - code);
                         }
                         reinterpret_cast<int*>(st + kOffKc)[slot] = kc;
@@ -564,7 +566,7 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
                 // a slot without a token: as a key its bias index lands in the table's -inf zone
                 int code = 0, label = 0xff, tok = -1, kc = 4 * (2 * c0 + 1);
                 if (slot < x.r.n && (!PAD || b_s < bw)) {
-                    tok = offset_token_tc(g, x.r, a_s, b_s, code, label);
+                    tok = offset_token_tc(g, x.r, a_s, b_s, cs, code, label);
                     kc = 4 * (c0 - code);
                 }
                 s_kc[slot] = kc;
@@ -582,7 +584,7 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
                 int bytes = 0;   // rows past the window's end are written as zeros
                 if (row < x.r.n && (!PAD || b_r < bw)) {
                     int code, label;
-                    const int tok = offset_token_tc(g, x.r, a_r, b_r, code, label);
+                    const int tok = offset_token_tc(g, x.r, a_r, b_r, cs, code, label);
                     const size_t off = (sample_off + (size_t)tok) * g.ts + x.head * kD + chunk * 8;
                     sq = q + off; sk = k + off; sv = v + off;
                     bytes = 16;
@@ -822,9 +824,9 @@ swin_fwd_tc_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_
 //   token point), and the head's largest entry in the last float (+inf instead if the head's entries spread over
 //   more than 64 octaves: the forward kernel then takes exact row maxima).
 __global__ void __launch_bounds__(256)
-swin_fwd_bias_prep_kernel(const float* __restrict__ bias, float* __restrict__ prep, int w, int heads) {
+swin_fwd_bias_prep_kernel(const float* __restrict__ bias, float* __restrict__ prep, int w, int heads, int cs) {
     const int head = blockIdx.x;
-    const int cs = w + 32, nw = 2 * w - 1;
+    const int nw = 2 * w - 1;
     const int c0 = (w - 1) * (cs + 1);
     float* dst = prep + (size_t)head * kFwdBiasFloats;
     float mx = -INFINITY, mn = INFINITY;
@@ -859,6 +861,13 @@ swin_fwd_bias_prep_kernel(const float* __restrict__ bias, float* __restrict__ pr
 }  // namespace
 
 #ifndef TERRA_ELEM_F16
+// window sides 9 .. 15 run in the layout of 16 slots per window row (TERRA_NO_PAD16=1: a debugging switch that keeps
+// the packed layout)
+bool pad16_layout(const Geo& g) {
+    static const bool pad_off = [] { const char* e_ = std::getenv("TERRA_NO_PAD16"); return e_ && e_[0] == '1'; }();
+    return g.d == 32 && g.w > 8 && g.w < 16 && !pad_off;
+}
+
 bool fwd_tc_supported(const Geo& g) { return g.d == 32 && g.nmax <= kMaxSlots && g.w <= 16; }
 
 // The TMA variants fetch a window row with one tiled copy: every window row must be one run of consecutive tokens
@@ -932,7 +941,8 @@ cudaError_t launch_fwd_tc(const Geo& g, const void* q, const void* k, const void
                           void* o, float* lse, void* workspace, int sm_count, cudaStream_t stream) {
     const long long items = (long long)g.B * g.Mh * g.Mw * g.heads;
     float* prep = reinterpret_cast<float*>(workspace);
-    swin_fwd_bias_prep_kernel<<<g.heads, 256, 0, stream>>>(bias, prep, g.w, g.heads);
+    const bool pad = pad16_layout(g);
+    swin_fwd_bias_prep_kernel<<<g.heads, 256, 0, stream>>>(bias, prep, g.w, g.heads, pad ? 48 : g.w + 32);
     count_launch(stream);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
@@ -942,9 +952,6 @@ cudaError_t launch_fwd_tc(const Geo& g, const void* q, const void* k, const void
     const bool tma = !tma_off && tma_row_shape(g) && make_row_map(&maps.q16, g, q, g.ts, 16) && make_row_map(&maps.k16, g, k, g.ts, 16) &&
                      make_row_map(&maps.v16, g, v, g.ts, 16) && make_row_map(&maps.q8, g, q, g.ts, 8) && make_row_map(&maps.k8, g, k, g.ts, 8) &&
                      make_row_map(&maps.v8, g, v, g.ts, 8);
-    // window sides 9 .. 15: the layout of 16 slots per window row (TERRA_NO_PAD16=1: a debugging switch that keeps the packed layout)
-    static const bool pad_off = [] { const char* e_ = std::getenv("TERRA_NO_PAD16"); return e_ && e_[0] == '1'; }();
-    const bool pad = g.w > 8 && g.w < 16 && !pad_off;
     auto kern = tma ? swin_fwd_tc_kernel<true, true> : (g.w == 16 ? swin_fwd_tc_kernel<true, false> : swin_fwd_tc_kernel<false, false>);
     if (pad) {
         switch (g.w) {
@@ -992,7 +999,7 @@ cudaError_t launch_bounded_wait_selftest(long long limit_cycles, cudaStream_t st
 
 // prepared bias tables for every head (also used by the backward kernels)
 cudaError_t launch_bias_prep(const Geo& g, const float* bias, float* prep, cudaStream_t stream) {
-    swin_fwd_bias_prep_kernel<<<g.heads, 256, 0, stream>>>(bias, prep, g.w, g.heads);
+    swin_fwd_bias_prep_kernel<<<g.heads, 256, 0, stream>>>(bias, prep, g.w, g.heads, pad16_layout(g) ? 48 : g.w + 32);
     count_launch(stream);
     return cudaGetLastError();
 }

@@ -54,6 +54,7 @@ cudaError_t launch_bwd_mma_f16(const Geo& g, const void* q, const void* k, const
 // tcgen05 forward path (head dim 32, window side <= 16)
 constexpr int kFwdBiasFloats = 2304;   // prepared bias table per head (padded rows, -inf zone, maximum in the last float)
 bool fwd_tc_supported(const Geo& g);
+bool pad16_layout(const Geo& g);       // window sides 9 .. 15: slots laid out 16 to a window row, bias codes with stride 48
 size_t fwd_tc_workspace_bytes(const Geo& g);
 cudaError_t launch_fwd_tc(const Geo& g, const void* q, const void* k, const void* v, const float* bias,
                           void* o, float* lse, void* workspace, int sm_count, cudaStream_t stream);

@@ -62,11 +62,11 @@ def test_grouped_updates_never_meet_and_full_width_rows_are_bank_conflict_free(w
 @pytest.mark.parametrize("w", range(9, 16))
 def test_sixteen_slots_per_window_row_layout_of_sides_9_to_15(w):
     """Sides 9 .. 15 with 16 slots per window row: every one of the 256 slots, with or without a token, carries the
-    code a (w + 32) + b of 16-wide geometry; key order c = 1; groups of 8 queries for two-tile windows.  The 32 x 8
+    code 48 a + b of 16-wide geometry (stride 48 whatever the side); key order c = 1; groups of 8 queries for two-tile windows.  The 32 x 8
     entries of a group are pairwise distinct, and with the kernel's margin in front of the table every entry that any
     (key slot, query column) pair can address lies inside the warp's 1472-float block."""
-    cs, c0 = w + 32, (w - 1) * (w + 33)
-    margin = (16 - w) * (w + 32) + 8                      # the kernel's dbias_margin(w)
+    cs, c0 = 48, (w - 1) * 49
+    margin = (16 - w) * 48 + 8                            # the kernel's dbias_margin(w)
     entries_of_table = 1472
 
     def code(slot):
@@ -81,6 +81,8 @@ def test_sixteen_slots_per_window_row_layout_of_sides_9_to_15(w):
                 assert len(entries) == len(set(entries)), (w, eh, W, q0)
                 lo, hi = min(entries) + c0 + margin, max(entries) + c0 + margin
                 assert 0 <= lo and hi < entries_of_table, (w, eh, lo, hi)
+                for q in range(q0, q0 + 8):               # one query: the warp's 32 key rows update 32 different banks
+                    assert len({(code(q) - code(ks)) % 32 for ks in slots}) == 32
     # the entries of pairs that hold tokens are those of the packed layout: (a_q - a_k + w - 1) cs + (b_q - b_k + w - 1)
     for aq, bq, ak, bk in ((0, 0, w - 1, w - 1), (w - 1, w - 1, 0, 0), (3, w - 1, 5, 0)):
         assert code(16 * aq + bq) - code(16 * ak + bk) + c0 == (aq - ak + w - 1) * cs + (bq - bk + w - 1)
