@@ -56,24 +56,33 @@ static_assert(2 * (kRegsWork - kRegsLaunch) <= (kRegsLaunch - kRegsOther), "regi
 constexpr int kPartBytes = 64;                        // one 32-column part of a row
 constexpr int kTile = 128;                            // keys per item, queries per chunk
 constexpr int kPart = kTile * kPartBytes;             // 8192: the region of one 32-column part of 128 rows
+constexpr int kHalf = 64;                             // queries per half chunk
 constexpr int kBiasFloats = 6048;
 constexpr int kBufCols = 128;                         // TMEM buffer b: S^T of a half chunk at 128 b, dP^T at 128 b + 64
 
 // Shared-memory plan per head dim D (64 or 128): a row is kept as D / 32 parts of 32 columns, each part a region in
-// the 64-byte-swizzled operand layout.  Head dim 64: two key stages, three query slots; head dim 128: one and two.
+// the 64-byte-swizzled operand layout.  The queries stream through a ring of slots.  Head dim 64: two key stages, three
+// slots of a whole chunk (128 rows, 32 KB); head dim 128: one key stage and four slots of a half chunk (64 rows, 32 KB:
+// with two 64 KB slots one copy was in flight at a time and the issuing warp waited for rows more than half of the
+// time; several smaller copies in flight hide the copy latency better.  At head dim 64 the same split was slower).
 template <int D>
 struct Lay {
     static constexpr int kParts = D / 32;
-    static constexpr int kKvStages = D == 64 ? 2 : 1, kSlots = D == 64 ? 3 : 2;
+    static constexpr int kKvStages = D == 64 ? 2 : 1, kSlots = D == 64 ? 3 : 4;
+    static constexpr int kHPS = D == 64 ? 2 : 1;      // half chunks per ring slot
+    static constexpr int kSlotQ = kHalf * kHPS;       // query rows per ring slot
+    static constexpr int kSPart = kSlotQ * kPartBytes;            // the region of one 32-column part of a slot's rows
     static constexpr int kRows = 2 * kParts * kPart;  // two tensors' rows
     // key stage: K parts | V parts, then per key row: 4 * bias code, label, token
     static constexpr int kOffK = 0, kOffV = kParts * kPart;
     static constexpr int kOffKCode = kRows, kOffKLab = kRows + 512, kOffKTok = kRows + 1024;
     static constexpr int kKvStageBytes = kRows + 2048;
     // query slot: Q parts | dO parts, then per query column: 4 * bias code, label, lse, delta
-    static constexpr int kOffQ = 0, kOffG = kParts * kPart;
-    static constexpr int kOffQCode = kRows, kOffQLab = kRows + 512, kOffQLse = kRows + 1024, kOffQDelta = kRows + 1536;
-    static constexpr int kSlotBytes = kRows + 2048;
+    static constexpr int kSlotRows = 2 * kParts * kSPart;
+    static constexpr int kTab = 4 * kSlotQ;           // bytes of one per-query table
+    static constexpr int kOffQ = 0, kOffG = kParts * kSPart;
+    static constexpr int kOffQCode = kSlotRows, kOffQLab = kSlotRows + kTab, kOffQLse = kSlotRows + 2 * kTab, kOffQDelta = kSlotRows + 3 * kTab;
+    static constexpr int kSlotBytes = kSlotRows + 4 * kTab;
     static constexpr int kOffSlots = kKvStages * kKvStageBytes;
     static constexpr int kOffBias = kOffSlots + kSlots * kSlotBytes;
     static constexpr int kOffBars = ((kOffBias + kBiasFloats * 4 + 1023) / 1024) * 1024;
@@ -83,6 +92,7 @@ struct Lay {
     static constexpr int kBufs = D == 64 ? 3 : 2;
     static constexpr int kColDV = kBufs * kBufCols, kColDK = kColDV + D;
     static_assert(kKvStageBytes % 1024 == 0 && kSlotBytes % 1024 == 0, "tiles keep the swizzle alignment");
+    static_assert(kSlots * 1536 <= kBiasFloats * 4, "the staged table rows of every slot fit the bias table's place");
     static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
     static_assert(kColDK + D <= 512, "tensor memory columns");
 };
@@ -149,11 +159,11 @@ __device__ __forceinline__ int lds_i32(uint32_t addr) {
 // token); a query column without a token has lse = +inf, so its P is 0.
 // ROW32: the window is 32 tokens wide, so the group's 16 queries sit in one window row and their bias codes are
 // consecutive: `code4` = 4 * code of column c, no per-query code table is read.
-// `sl_a` = shared address of the slot's per-query tables (code, label, lse, delta: 512 bytes each).
-template <bool MASKED, bool ROW32 = false>
+// `sl_a` = shared address of the slot's per-query tables (code, label, lse, delta: TAB bytes each); c counts within the slot.
+template <bool MASKED, bool ROW32, int TAB>
 __device__ __forceinline__ void cols16(const uint32_t (&rs)[16], const uint32_t (&rp)[16], int c, uint32_t bias_row, int klabel,
                                        uint32_t sl_a, float scale, uint32_t (&pk_p)[8], uint32_t (&pk_ds)[8], int code4 = 0) {
-    constexpr int kOffQCode = 0, kOffQLab = 512, kOffQLse = 1024, kOffQDelta = 1536;
+    constexpr int kOffQCode = 0, kOffQLab = TAB, kOffQLse = 2 * TAB, kOffQDelta = 3 * TAB;
     // all table loads first (they are issued in program order), then the gathers that depend on them, then the math
     int co[16], ql[16];
     float l2[16], dl[16], bv[16];
@@ -205,10 +215,10 @@ __device__ __forceinline__ void cols16(const uint32_t (&rs)[16], const uint32_t 
 // `neg_l2` = -lse * log2(e) and `dl` = delta of the row; `bias_a` = shared address of the row's bias entry for column
 // c (the following keys' entries follow); the key columns' mask labels are the slot's label table.  dS leaves as
 // packed bf16 for the dQ product and in fp32 for the bias gradient.
-template <bool MASKED>
+template <bool MASKED, int TAB>
 __device__ __forceinline__ void cols16_qside(const uint32_t (&rs)[16], const uint32_t (&rp)[16], int c, uint32_t bias_a, int rlabel,
                                              uint32_t sl_a, float scale, float neg_l2, float dl, uint32_t (&pk_ds)[8], float (&ds)[16]) {
-    constexpr int kOffQLab = 512;
+    constexpr int kOffQLab = TAB;
     int cl[16];
     float bv[16];
     if (MASKED) {
@@ -281,6 +291,7 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
     using L = Lay<D>;
     constexpr bool TMA = MODE >= 1, ROWS = MODE >= 2, QS = MODE == 3;
     constexpr int kStageBytes = 1536;                 // MODE 2: the staged table rows of one query slot
+    constexpr int kHPS = L::kHPS, kSlotQ = L::kSlotQ, kSPart = L::kSPart, kTab = L::kTab;
     constexpr int kParts = L::kParts, kKvStages = L::kKvStages, kSlots = L::kSlots;
     constexpr int kOffK = L::kOffK, kOffV = L::kOffV, kOffKCode = L::kOffKCode, kOffKLab = L::kOffKLab, kOffKTok = L::kOffKTok;
     constexpr int kKvStageBytes = L::kKvStageBytes, kOffQ = L::kOffQ, kOffG = L::kOffG, kOffQCode = L::kOffQCode;
@@ -292,16 +303,16 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
     const uint32_t bar0 = smem0 + kOffBars;
     auto bar_kvfull = [&](int s) { return bar0 + 8u * s; };              // the tile's K, V rows and key tables are there
     auto bar_kvempty = [&](int s) { return bar0 + 8u * (2 + s); };       // ... and no longer needed
-    auto bar_qfull = [&](int s) { return bar0 + 8u * (4 + s); };         // a query chunk is in ring slot s
-    auto bar_qempty = [&](int s) { return bar0 + 8u * (7 + s); };        // ... and every MMA that reads it is complete
+    auto bar_qfull = [&](int s) { return bar0 + 8u * (4 + s); };         // a half chunk of queries is in ring slot s
+    auto bar_qempty = [&](int s) { return bar0 + 8u * (10 + s); };       // ... and every MMA that reads it is complete
     // A chunk's 64-query halves are separate units of work, numbered through the whole run (only halves that exist
     // count); half number p belongs to elementwise warps 4 h .. 4 h + 3 (h = which half of its chunk) and lives in TMEM
     // buffer p % kBufs, with the buffer's own hand-overs.
-    auto bar_sdp = [&](int b) { return bar0 + 8u * (10 + b); };          // S^T and dP^T of a half chunk are in TMEM buffer b
-    auto bar_ds = [&](int b) { return bar0 + 8u * (13 + b); };           // bf16 P^T and dS^T of the half chunk are in buffer b
-    const uint32_t bar_acc = bar0 + 8u * 16;                              // dV, dK of the item are final
-    const uint32_t bar_accfree = bar0 + 8u * 17;                          // ... and have been read
-    unsigned char* tail = smem + kOffBars + 8 * 18;
+    auto bar_sdp = [&](int b) { return bar0 + 8u * (16 + b); };          // S^T and dP^T of a half chunk are in TMEM buffer b
+    auto bar_ds = [&](int b) { return bar0 + 8u * (19 + b); };           // bf16 P^T and dS^T of the half chunk are in buffer b
+    const uint32_t bar_acc = bar0 + 8u * 22;                              // dV, dK of the item are final
+    const uint32_t bar_accfree = bar0 + 8u * 23;                          // ... and have been read
+    unsigned char* tail = smem + kOffBars + 8 * 24;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail);
     volatile int* cta_abort = reinterpret_cast<volatile int*>(tail + 8);
 
@@ -351,10 +362,10 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
     if (TMA && warp >= kLoaderWarp0) {
         // ------------------------------------------------------------------ loader warp (TMA); the other two have no work
         if (warp == kLoaderWarp0) {
-            const int wrows = kTile / g.w;                    // window rows per 128 slots
+            const int wrows = max(1, kTile / g.w);            // window rows per 128 slots
             const int per_tensor = wrows * kParts;
             int kuse = 0;
-            long long ru = 0;
+            unsigned ru = 0;                                  // half chunks so far (every role counts them the same way)
             bool ok = true;
             ItemCursor cur = cursor_init(cta_in_head, ctas_per_head, max_tiles, g.Mw, g.Mh);
             for (long long it = cta_in_head; ok && it < n_items; it += ctas_per_head, cursor_advance(cur, max_tiles, g.Mw, g.Mh)) {
@@ -391,15 +402,18 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                     if (lane == 0) mbar_arrive_expect_tx(bar_kvfull(ks), (uint32_t)(kTile * D * 2 * 2));
                     else mbar_arrive(bar_kvfull(ks));
                 }
-                // ---- the window's queries, chunk by chunk
-                for (int c = 0; c < x.nch; ++c, ++ru) {
+                // ---- the window's queries, slot by slot (the windows are complete: every slot is full)
+                const int nu = x.npad / kSlotQ;
+                const int n_run = min(g.w, kSlotQ), runs = kSlotQ / n_run;        // runs of one window row per slot
+                for (int i = 0; i < nu; ++i, ++ru) {
                     const int s = (int)(ru % kSlots);
                     ok = mbar_wait_all(bar_qempty(s), (uint32_t)((ru / kSlots) & 1) ^ 1u, cta_abort);
                     if (!ok) break;
                     unsigned char* sl = smem + kOffSlots + s * kSlotBytes;
                     const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes;
-                    for (int row = lane; row < kTile; row += 32) {
-                        const int slot = c * kTile + row;
+                    const int slot0 = i * kSlotQ;
+                    for (int row = lane; row < kSlotQ; row += 32) {
+                        const int slot = slot0 + row;
                         int code, label;
                         const int a = slot / ew;
                         const int tok = offset_token(g, x.r, a, slot - a * ew, code, label);
@@ -411,21 +425,23 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                         reinterpret_cast<int*>(sl + kOffQCode)[row] = 4 * code;
                         reinterpret_cast<int*>(sl + kOffQLab)[row] = label;
                     }
-                    for (int i = lane; i < 2 * per_tensor; i += 32) {
-                        const int tsr = i >= per_tensor ? 1 : 0, rem = i - tsr * per_tensor;
-                        const int ar = rem / kParts, part = rem - ar * kParts;
-                        bulk_copy_window_row(tsr ? maps.g : maps.q, sb + (tsr ? kOffG : kOffQ) + part * kPart + ar * g.w * kPartBytes, g,
-                                             x.b, x.r.wr, v0, c * wrows + ar, head * D + part * 32, bar_qfull(s));
+                    for (int j = lane; j < 2 * runs * kParts; j += 32) {
+                        const int tsr = j >= runs * kParts ? 1 : 0, rem = j - tsr * runs * kParts;
+                        const int rr = rem / kParts, part = rem - rr * kParts;
+                        const int rslot = slot0 + rr * n_run, a = rslot / g.w;
+                        bulk_copy_window_run(tsr ? maps.g : maps.q, sb + (tsr ? kOffG : kOffQ) + part * kSPart + rr * n_run * kPartBytes, g,
+                                             x.b, x.r.wr, v0, a, rslot - a * g.w, n_run, head * D + part * 32, bar_qfull(s));
                     }
                     if (ROWS && lane == 0) {
-                        const int lw = 31 - __clz(g.w), kr = kTile >> lw;
-                        const int r0 = (c - x.kt) * kr - (kr - 1) + g.w - 1;
+                        // the table rows that this slot's ur window rows need against the key tile's kr window rows
+                        const int lw = 31 - __clz(g.w), kr = kTile >> lw, ur = max(1, kSlotQ >> lw);
+                        const int r0 = (slot0 >> lw) - x.kt * kr - (kr - 1) + g.w - 1;
                         bulk_load(smem0 + kOffBias + s * kStageBytes,
                                   bias_prep + (size_t)head * ((2 * g.w - 1) * 2 * g.w + 4) + (size_t)r0 * 2 * g.w,
-                                  (uint32_t)((2 * kr - 1) * 8 * g.w), bar_qfull(s));
-                        mbar_expect_tx(bar_qfull(s), (uint32_t)((2 * kr - 1) * 8 * g.w));
+                                  (uint32_t)((ur + kr - 1) * 8 * g.w), bar_qfull(s));
+                        mbar_expect_tx(bar_qfull(s), (uint32_t)((ur + kr - 1) * 8 * g.w));
                     }
-                    if (lane == 0) mbar_expect_tx(bar_qfull(s), (uint32_t)(kTile * D * 2 * 2));
+                    if (lane == 0) mbar_expect_tx(bar_qfull(s), (uint32_t)(kSlotQ * D * 2 * 2));
                     // the lane's arrival: when its lse / delta copies have landed (its table entries were written before)
                     if (QS) mbar_arrive(bar_qfull(s));
                     else cp_async_mbar_arrive_noinc(bar_qfull(s));
@@ -442,7 +458,7 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
         const int lrow = lt / kParts;
         constexpr int kRowsPerIter = kLoaderThreads / kParts;
         int kuse = 0;
-        long long ru = 0;
+        unsigned ru = 0;                                      // half chunks so far
         bool ok = true;
         auto acquire = [&](uint32_t bar, uint32_t parity) -> bool { return mbar_wait_all(bar, parity, cta_abort); };
         // the thread's table entries are visible to the CTA before its arrival, which follows its copies
@@ -497,16 +513,18 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                 }
                 issued(bar_kvfull(ks));
             }
-            // ---- the window's queries, chunk by chunk
-            for (int c = 0; c < x.nch; ++c, ++ru) {
+            // ---- the window's queries, slot by slot (the last one may be partly filled)
+            const int nu = (x.npad + kSlotQ - 1) / kSlotQ;
+            for (int i = 0; i < nu; ++i, ++ru) {
                 const int s = (int)(ru % kSlots);
                 ok = acquire(bar_qempty(s), (uint32_t)((ru / kSlots) & 1) ^ 1u);
                 if (!ok) break;
                 unsigned char* sl = smem + kOffSlots + s * kSlotBytes;
-                const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes + hf * kPart;
-                const int ncols = min(kTile, x.npad - c * kTile);
-                for (int row = lt; row < kTile; row += kLoaderThreads) {
-                    const int slot = c * kTile + row;
+                const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes + hf * kSPart;
+                const int slot0 = i * kSlotQ;
+                const int ncols = min(kSlotQ, x.npad - slot0);
+                for (int row = lt; row < kSlotQ; row += kLoaderThreads) {
+                    const int slot = slot0 + row;
                     int code = 0, label = 0xff;
                     if (slot < x.r.n) {
                         // lse and delta travel with the rows (no load the loader would have to wait for)
@@ -522,13 +540,13 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                     reinterpret_cast<int*>(sl + kOffQCode)[row] = 4 * code;
                     reinterpret_cast<int*>(sl + kOffQLab)[row] = label;
                 }
-                const int slot_first = c * kTile + lrow;
+                const int slot_first = slot0 + lrow;
                 int a_r = slot_first / ew, b_r = slot_first - a_r * ew;
                 for (int row = lrow; row < ncols; row += kRowsPerIter, a_r += q_r, b_r += r_r) {
                     if (b_r >= ew) { b_r -= ew; ++a_r; }
                     const __nv_bfloat16 *sq = q, *sg = d_o;
                     int bytes = 0;
-                    if (c * kTile + row < x.r.n) {
+                    if (slot0 + row < x.r.n) {
                         int code, label;
                         const int tok = offset_token(g, x.r, a_r, b_r, code, label);
                         sq = q + (sample_off + (size_t)tok) * g.ts + head * D + hf * 32;
@@ -552,7 +570,7 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
         const uint32_t sd_hi = sdesc_hi(make_sdesc_sw64(smem0, 512));    // common high word of the K-major descriptors
         int kuse = 0;
         unsigned p0 = 0;                                  // half chunks before the current item
-        long long ru = 0;
+        unsigned u0 = 0;                                  // ring slots used before the current item; use u is in slot u % kSlots
         bool ok = true;
         ItemCursor cur = cursor_init(cta_in_head, ctas_per_head, max_tiles, g.Mw, g.Mh);
         for (long long it = cta_in_head; ok && it < n_items; it += ctas_per_head, cursor_advance(cur, max_tiles, g.Mw, g.Mh)) {
@@ -565,35 +583,36 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             const uint32_t kb = smem0 + ks * kKvStageBytes;
             // queries of half h of chunk c (a multiple of 16; 0: the half does not exist)
             auto half_cols = [&](int c, int h) { return max(0, min(64, x.npad - c * kTile - 64 * h)); };
-            auto chunk_ready = [&](long long use) -> bool {
+            auto half_ready = [&](unsigned use) -> bool {
                 if (!mbar_wait_all(bar_qfull((int)(use % kSlots)), (uint32_t)((use / kSlots) & 1), cta_abort)) return false;
                 fence_proxy_async();
                 return true;
             };
-            // S^T = K Q^T, dP^T = V dO^T for the 64 queries of half h of the chunk in ring slot `sb`
-            // (descriptor low words = start address in 16-byte units: + 2 per 32-byte K step, + kPart / 16 per 32-column part)
+            // S^T = K Q^T, dP^T = V dO^T for the queries of the half chunk in ring slot `sb`
+            // (descriptor low words = start address in 16-byte units: + 2 per 32-byte K step, + region / 16 per 32-column part)
             const uint32_t k_lo = sdesc_lo(make_sdesc_sw64(kb + kOffK, 512)), v_lo = sdesc_lo(make_sdesc_sw64(kb + kOffV, 512));
-            auto issue_sdp = [&](int h, uint32_t sb, int nc, int buf) {
+            // (`sb` = the address of the half chunk's first row in its slot)
+            auto issue_sdp = [&](uint32_t sb, int nc, int buf) {
                 const uint32_t idesc = make_idesc_elem(128, nc, 0, 0);
-                const uint32_t q_lo = sdesc_lo(make_sdesc_sw64(sb + kOffQ + h * 64 * kPartBytes, 512));
-                const uint32_t g_lo = sdesc_lo(make_sdesc_sw64(sb + kOffG + h * 64 * kPartBytes, 512));
+                const uint32_t q_lo = sdesc_lo(make_sdesc_sw64(sb + kOffQ, 512));
+                const uint32_t g_lo = sdesc_lo(make_sdesc_sw64(sb + kOffG, 512));
                 const uint32_t t_s = tmem_base + kBufCols * buf, t_dp = t_s + 64;
-                constexpr uint32_t kNext = kPart >> 4;
+                constexpr uint32_t kNext = kPart >> 4, kNextH = kSPart >> 4;
                 tc_fence_after();
                 if (elect_one()) {
                     mma_ss_h<false>(t_s, k_lo, q_lo, sd_hi, idesc);
                     mma_ss_h<true>(t_s, k_lo + 2, q_lo + 2, sd_hi, idesc);
 #pragma unroll
                     for (int pt = 1; pt < kParts; ++pt) {
-                        mma_ss_h<true>(t_s, k_lo + pt * kNext, q_lo + pt * kNext, sd_hi, idesc);
-                        mma_ss_h<true>(t_s, k_lo + pt * kNext + 2, q_lo + pt * kNext + 2, sd_hi, idesc);
+                        mma_ss_h<true>(t_s, k_lo + pt * kNext, q_lo + pt * kNextH, sd_hi, idesc);
+                        mma_ss_h<true>(t_s, k_lo + pt * kNext + 2, q_lo + pt * kNextH + 2, sd_hi, idesc);
                     }
                     mma_ss_h<false>(t_dp, v_lo, g_lo, sd_hi, idesc);
                     mma_ss_h<true>(t_dp, v_lo + 2, g_lo + 2, sd_hi, idesc);
 #pragma unroll
                     for (int pt = 1; pt < kParts; ++pt) {
-                        mma_ss_h<true>(t_dp, v_lo + pt * kNext, g_lo + pt * kNext, sd_hi, idesc);
-                        mma_ss_h<true>(t_dp, v_lo + pt * kNext + 2, g_lo + pt * kNext + 2, sd_hi, idesc);
+                        mma_ss_h<true>(t_dp, v_lo + pt * kNext, g_lo + pt * kNextH, sd_hi, idesc);
+                        mma_ss_h<true>(t_dp, v_lo + pt * kNext + 2, g_lo + pt * kNextH + 2, sd_hi, idesc);
                     }
                     mma_commit(bar_sdp(buf));
                 }
@@ -601,42 +620,42 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
             };
             // the item's half chunks in order: half i is half i % 2 of chunk i / 2 (only the last chunk can lack its second half)
             const int nh = 2 * x.nch - (half_cols(x.nch - 1, 1) > 0 ? 0 : 1);
-            int ready_chunks = 0;                         // chunks of the item known to be in their ring slots
-            // the chunk of half i is in its ring slot
-            auto ensure_chunk = [&](int i) -> bool {
-                while (ready_chunks <= (i >> 1)) {
-                    if (!chunk_ready(ru + ready_chunks)) return false;
-                    ++ready_chunks;
+            int ready_units = 0;                          // ring slots of the item known to be filled
+            // the rows of half i are in their ring slot
+            auto ensure_half = [&](int i) -> bool {
+                while (ready_units <= i / kHPS) {
+                    if (!half_ready(u0 + (unsigned)ready_units)) return false;
+                    ++ready_units;
                 }
                 return true;
             };
-            // scores of half i into its buffer
-            auto issue_half = [&](int i) {
-                const int c = i >> 1, h = i & 1;
-                issue_sdp(h, smem0 + kOffSlots + (int)((ru + c) % kSlots) * kSlotBytes, half_cols(c, h), (int)((p0 + i) % kBufs));
+            // the address of half i's first row in its slot
+            auto half_rows = [&](int i) -> uint32_t {
+                return smem0 + kOffSlots + (int)((u0 + (unsigned)(i / kHPS)) % kSlots) * kSlotBytes + (i % kHPS) * kHalf * kPartBytes;
             };
+            // scores of half i into its buffer
+            auto issue_half = [&](int i) { issue_sdp(half_rows(i), half_cols(i >> 1, i & 1), (int)((p0 + i) % kBufs)); };
             for (int i = 0; i < kBufs && i < nh && ok; ++i) {
-                ok = ensure_chunk(i);
+                ok = ensure_half(i);
                 if (ok) issue_half(i);
             }
             for (int i = 0; i < nh && ok; ++i) {
                 const int c = i >> 1, h = i & 1;
                 const unsigned p = p0 + i;
                 const int buf = (int)(p % kBufs);
-                const int s = (int)((ru + c) % kSlots);
-                const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes;
+                const int s = (int)((u0 + (unsigned)(i / kHPS)) % kSlots);
+                const uint32_t sb = half_rows(i);
                 const int nc = half_cols(c, h);
                 ok = mbar_wait_all(bar_ds(buf), (p / kBufs) & 1, cta_abort);
                 if (ok && i == 0 && kuse > 0) ok = mbar_wait_all(bar_accfree, (kuse - 1) & 1, cta_abort);
                 if (!ok) break;
                 tc_fence_after();
                 // dV += P^T dO, dK += dS^T Q over the half chunk's query columns
-                const uint64_t gd = make_sdesc_sw64_mn(sb + kOffG + h * 64 * kPartBytes, kPart, 512);
-                const uint64_t qd = make_sdesc_sw64_mn(sb + kOffQ + h * 64 * kPartBytes, kPart, 512);
+                const uint64_t gd = make_sdesc_sw64_mn(sb + kOffG, kSPart, 512);
+                const uint64_t qd = make_sdesc_sw64_mn(sb + kOffQ, kSPart, 512);
                 const uint32_t g_lo = sdesc_lo(gd), q_lo = sdesc_lo(qd), d_hi = sdesc_hi(gd);
                 const uint32_t t_p = tmem_base + kBufCols * buf, t_ds = t_p + 64;
                 const int nks = nc >> 4;
-                const bool chunk_done = h == 1 || half_cols(c, 1) == 0;      // the chunk's last half
                 if (elect_one()) {
                     int j = 0;
                     if (i == 0) {
@@ -648,7 +667,8 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                         if (!QS) mma_ts_h<true>(tmem_base + kColDV, t_p + 16 * j, g_lo + 64 * j, d_hi, idesc_acc);
                         mma_ts_h<true>(tmem_base + kColDK, t_ds + 16 * j, q_lo + 64 * j, d_hi, idesc_acc);
                     }
-                    if (chunk_done) mma_commit(bar_qempty(s));       // the slot's last readers were issued just above
+                    // the slot's last readers were issued just above
+                    if (kHPS == 1 || h == 1 || half_cols(c, 1) == 0) mma_commit(bar_qempty(s));
                     if (i + 1 == nh) {
                         mma_commit(bar_acc);
                         mma_commit(bar_kvempty(ks));
@@ -657,15 +677,15 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                 __syncwarp();
                 // the buffer is free again (the products that read it were issued just above): the scores of the half
                 // chunk kBufs further on follow at once
-                // (its chunk is waited for only now: where the rows are late, the current half should not wait for them)
+                // (its rows are waited for only now: where they are late, the current half should not wait for them)
                 if (i + kBufs < nh) {
-                    ok = ensure_chunk(i + kBufs);
+                    ok = ensure_half(i + kBufs);
                     if (ok) issue_half(i + kBufs);
                 }
             }
             if (!ok) break;
-            ru += x.nch;
             p0 += (unsigned)nh;
+            u0 += (unsigned)((nh + kHPS - 1) / kHPS);
             ++kuse;
         }
     }
@@ -680,7 +700,7 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
         const float out_scale = g.scale_log2e * kLn2;     // dK carries the score scale
         int kuse = 0;
         unsigned p0 = 0;                                  // half chunks before the current item
-        long long ru = 0;
+        unsigned u0 = 0;                                  // ring slots used before the current item
         bool ok = true;
         ItemCursor cur = cursor_init(cta_in_head, ctas_per_head, max_tiles, g.Mw, g.Mh);
         for (long long it = cta_in_head; ok && it < n_items; it += ctas_per_head, cursor_advance(cur, max_tiles, g.Mw, g.Mh)) {
@@ -709,23 +729,25 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                 const int kslot = x.kt * kTile + krow, kr = kTile >> lw;
                 bias_row = smem0 + kOffBias + (kr - 1 - ((kslot >> lw) - ((x.kt * kTile) >> lw))) * 8 * g.w + 4 * (g.w - 1 - (kslot & (g.w - 1)));
             }
-            for (int c = 0; c < x.nch && ok; ++c, ++ru) {
-                const int s = (int)(ru % kSlots);
-                const uint32_t sl_a = smem0 + kOffSlots + s * kSlotBytes + kOffQCode;      // the slot's per-query tables
+            for (int c = 0; c < x.nch && ok; ++c) {
                 const int ncols = min(kTile, x.npad - c * kTile);
                 if (ncols <= 64 * hcol) continue;          // this group's half of the chunk does not exist
                 const unsigned p = p0 + 2 * c + hcol;      // the half chunk's number; its buffer holds S^T at column 0, dP^T at 64
                 const int buf = (int)(p % kBufs);
+                const int s = (int)((u0 + (unsigned)((2 * c + hcol) / kHPS)) % kSlots);     // ... and its rows and tables are in this ring slot
+                const int sc0 = ((2 * c + hcol) % kHPS) * kHalf;                            // its first column within the slot
+                const uint32_t sl_a = smem0 + kOffSlots + s * kSlotBytes + kOffQCode + 4 * sc0;      // the half chunk's part of the slot's per-query tables
                 ok = mbar_wait_all(bar_sdp(buf), (p / kBufs) & 1, cta_abort);
                 if (!ok) break;
                 tc_fence_after();
-                // (addressed by the chunk's column number: the group's columns start at 64 hcol)
-                const uint32_t t_s = tmem_base + lane_addr + kBufCols * buf - 64 * hcol, t_dp = t_s + 64;
-                const int col_end = min(ncols, 64 * hcol + 64);
-                // 4 * bias code of query column `col` of this chunk in a 32-wide window: slot = 128 c + col = 32 a + b
-                // (MODE 2: the offset into the slot's staged table rows)
+                // (columns count within the half chunk)
+                const uint32_t t_s = tmem_base + lane_addr + kBufCols * buf, t_dp = t_s + 64;
+                const int col_end = min(ncols - 64 * hcol, 64);
+                // 4 * bias code of query column `col` of this half chunk in a 32-wide window: slot = 128 c + 64 hcol + col = 32 a + b
+                // (MODE 2: the offset into the slot's staged table rows; the half chunk lies in one window row)
                 auto code4_of = [&](int col) {
-                    return ROWS ? s * kStageBytes + (col >> lw) * 8 * g.w + 4 * (col & (g.w - 1)) : 4 * ((4 * c + (col >> 5)) * cs + (col & 31));
+                    return ROWS ? s * kStageBytes + (((sc0 + col) >> lw) * 2 * g.w + ((64 * hcol + col) & (g.w - 1))) * 4
+                                : 4 * ((4 * c + 2 * hcol + (col >> 5)) * cs + (col & 31));
                 };
                 // groups of 16 columns; the next group's S^T / dP^T travel from TMEM while this one is worked on
                 uint32_t rs[16], rp[16], rs2[16], rp2[16], pk_p[8], pk_ds[8];
@@ -750,14 +772,14 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                             lo += up ? 0.f : val;
                         }
                     };
-                    tmem_ld16(t_s + 64 * hcol, rs);
-                    tmem_ld16(t_dp + 64 * hcol, rp);
+                    tmem_ld16(t_s, rs);
+                    tmem_ld16(t_dp, rp);
 #pragma unroll
                     for (int gi = 0; gi < 4; ++gi) {
-                        const int cc = 64 * hcol + 16 * gi;
+                        const int cc = 16 * gi;
                         tmem_ld_wait();
-                        if (x.masked) cols16_qside<true>(rs, rp, cc, bias_row + code4_of(cc), klabel, sl_a, scale, neg_l2, row_dl, pk_ds, ds);
-                        else cols16_qside<false>(rs, rp, cc, bias_row + code4_of(cc), klabel, sl_a, scale, neg_l2, row_dl, pk_ds, ds);
+                        if (x.masked) cols16_qside<true, kTab>(rs, rp, cc, bias_row + code4_of(cc), klabel, sl_a, scale, neg_l2, row_dl, pk_ds, ds);
+                        else cols16_qside<false, kTab>(rs, rp, cc, bias_row + code4_of(cc), klabel, sl_a, scale, neg_l2, row_dl, pk_ds, ds);
                         if (gi < 3) {
                             tmem_ld16(t_s + cc + 16, rs);
                             tmem_ld16(t_dp + cc + 16, rp);
@@ -772,20 +794,20 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                     atomicAdd(dst + 32 * g.heads, acc1);
                     if (lane < 31) atomicAdd(dst + 64 * g.heads, acc2);
                 } else {
-                if (64 * hcol < col_end) {
-                    tmem_ld16(t_s + 64 * hcol, rs);
-                    tmem_ld16(t_dp + 64 * hcol, rp);
+                if (0 < col_end) {
+                    tmem_ld16(t_s, rs);
+                    tmem_ld16(t_dp, rp);
                 }
-                for (int cc = 64 * hcol; cc < col_end; cc += 32) {
+                for (int cc = 0; cc < col_end; cc += 32) {
                     tmem_ld_wait();
                     if (cc + 16 < col_end) {
                         tmem_ld16(t_s + cc + 16, rs2);
                         tmem_ld16(t_dp + cc + 16, rp2);
                     }
-                    if (ROWS && x.masked) cols16<true, true>(rs, rp, cc, bias_row, klabel, sl_a, scale, pk_p, pk_ds, code4_of(cc));
-                    else if (x.masked) cols16<true>(rs, rp, cc, bias_row, klabel, sl_a, scale, pk_p, pk_ds);
-                    else if (row32) cols16<false, true>(rs, rp, cc, bias_row, klabel, sl_a, scale, pk_p, pk_ds, code4_of(cc));
-                    else cols16<false>(rs, rp, cc, bias_row, klabel, sl_a, scale, pk_p, pk_ds);
+                    if (ROWS && x.masked) cols16<true, true, kTab>(rs, rp, cc, bias_row, klabel, sl_a, scale, pk_p, pk_ds, code4_of(cc));
+                    else if (x.masked) cols16<true, false, kTab>(rs, rp, cc, bias_row, klabel, sl_a, scale, pk_p, pk_ds);
+                    else if (row32) cols16<false, true, kTab>(rs, rp, cc, bias_row, klabel, sl_a, scale, pk_p, pk_ds, code4_of(cc));
+                    else cols16<false, false, kTab>(rs, rp, cc, bias_row, klabel, sl_a, scale, pk_p, pk_ds);
                     tmem_st8(t_s + cc, pk_p);              // 16 queries -> 8 packed columns at the group's own place
                     tmem_st8(t_dp + cc, pk_ds);
                     if (cc + 16 < col_end) {
@@ -794,10 +816,10 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                             tmem_ld16(t_s + cc + 32, rs);
                             tmem_ld16(t_dp + cc + 32, rp);
                         }
-                        if (ROWS && x.masked) cols16<true, true>(rs2, rp2, cc + 16, bias_row, klabel, sl_a, scale, pk_p, pk_ds, code4_of(cc + 16));
-                        else if (x.masked) cols16<true>(rs2, rp2, cc + 16, bias_row, klabel, sl_a, scale, pk_p, pk_ds);
-                        else if (row32) cols16<false, true>(rs2, rp2, cc + 16, bias_row, klabel, sl_a, scale, pk_p, pk_ds, code4_of(cc + 16));
-                        else cols16<false>(rs2, rp2, cc + 16, bias_row, klabel, sl_a, scale, pk_p, pk_ds);
+                        if (ROWS && x.masked) cols16<true, true, kTab>(rs2, rp2, cc + 16, bias_row, klabel, sl_a, scale, pk_p, pk_ds, code4_of(cc + 16));
+                        else if (x.masked) cols16<true, false, kTab>(rs2, rp2, cc + 16, bias_row, klabel, sl_a, scale, pk_p, pk_ds);
+                        else if (row32) cols16<false, true, kTab>(rs2, rp2, cc + 16, bias_row, klabel, sl_a, scale, pk_p, pk_ds, code4_of(cc + 16));
+                        else cols16<false, false, kTab>(rs2, rp2, cc + 16, bias_row, klabel, sl_a, scale, pk_p, pk_ds);
                         tmem_st8(t_s + cc + 16, pk_p);
                         tmem_st8(t_dp + cc + 16, pk_ds);
                     }
@@ -808,7 +830,11 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                 mbar_arrive(bar_ds(buf));
             }
             if (!ok) break;
-            p0 += (unsigned)(2 * x.nch - (min(kTile, x.npad - (x.nch - 1) * kTile) > 64 ? 0 : 1));
+            {
+                const int nh = 2 * x.nch - (min(kTile, x.npad - (x.nch - 1) * kTile) > 64 ? 0 : 1);
+                p0 += (unsigned)nh;
+                u0 += (unsigned)((nh + kHPS - 1) / kHPS);
+            }
             // ---- read-out: dV rows by warps 0-3, dK rows by warps 4-7
             if (!mbar_wait_all(bar_acc, kuse & 1, cta_abort)) break;
             tc_fence_after();

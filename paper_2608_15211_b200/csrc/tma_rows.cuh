@@ -29,24 +29,32 @@ inline bool bulk_rows_shape(const Geo& g) {
            (long long)g.B * g.H * g.W < 0x7fffffffLL;
 }
 
-// device: the copies of window row `a` of window row-index `wr` in sample `b`: w slots of 64 bytes from `dst` on
-// (a multiple of 512 bytes into a swizzled region), columns [xc, xc + 32) of every token; `v0` = the window's first
-// token column after the roll.  The bytes are counted on `bar`.
-__device__ __forceinline__ void bulk_copy_window_row(const RowMaps3& m3, uint32_t dst, const Geo& g, int b, int wr, int v0, int a,
-                                                     int xc, uint32_t bar) {
+// device: the copies of `n_run` slots (a multiple of 8) of window row `a`, from window column `b0` (a multiple of 8) on,
+// of window row-index `wr` in sample `b`: 64 bytes per slot from `dst` on (a multiple of 512 bytes into a swizzled
+// region), columns [xc, xc + 32) of every token; `v0` = the window's first token column after the roll.  The bytes
+// are counted on `bar`.
+__device__ __forceinline__ void bulk_copy_window_run(const RowMaps3& m3, uint32_t dst, const Geo& g, int b, int wr, int v0, int a,
+                                                     int b0, int n_run, int xc, uint32_t bar) {
     int u = wr * g.w + a + g.sh;
     if (u >= g.H) u -= g.H;
     const int y0 = (b * g.H + u) * g.W;
-    const int n1 = min(g.w, g.W - v0);            // tokens up to the seam; the rest starts at column 0
-    int y = y0 + v0, n = n1;
+    int vs = v0 + b0;
+    if (vs >= g.W) vs -= g.W;
+    const int n1 = min(n_run, g.W - vs);          // tokens up to the seam; the rest starts at column 0
+    int y = y0 + vs, n = n1;
 #pragma unroll
     for (int seg = 0; seg < 2; ++seg) {
         while (n >= 32) { tc::tma_load_2d(dst, &m3.m[0], xc, y, bar); dst += 32 * 64; y += 32; n -= 32; }
         if (n >= 16) { tc::tma_load_2d(dst, &m3.m[1], xc, y, bar); dst += 16 * 64; y += 16; n -= 16; }
         if (n >= 8) { tc::tma_load_2d(dst, &m3.m[2], xc, y, bar); dst += 8 * 64; }
         y = y0;
-        n = g.w - n1;
+        n = n_run - n1;
     }
+}
+// the whole window row
+__device__ __forceinline__ void bulk_copy_window_row(const RowMaps3& m3, uint32_t dst, const Geo& g, int b, int wr, int v0, int a,
+                                                     int xc, uint32_t bar) {
+    bulk_copy_window_run(m3, dst, g, b, wr, v0, a, 0, g.w, xc, bar);
 }
 
 }  // namespace terra
