@@ -931,6 +931,12 @@ bool make_col_map(CUtensorMap* map, const Geo& g, const void* base, int token_st
 bool make_row_maps3(RowMaps3* maps, const Geo& g, const void* base, int token_stride) {
     for (int i = 0; i < 3; ++i)
         if (!make_row_map(&maps->m[i], g, base, token_stride, 32 >> i)) return false;
+    // the large boxes serve window sides 64 and 128 only; a box may not be longer than the token axis
+    for (int i = 3; i < 5; ++i) {
+        const long long tokens = (long long)g.B * g.H * g.W;
+        const int box = (g.w >= 64 && tokens >= (8 << i)) ? (8 << i) : 32;           // m[3]: 64 tokens, m[4]: 128 tokens
+        if (!make_row_map(&maps->m[i], g, base, token_stride, box)) return false;
+    }
     return true;
 }
 

@@ -2,8 +2,9 @@
 //
 // On a grid of complete windows whose longitude shift is a multiple of 8, the tokens of one window row are one run of
 // consecutive tokens of the tensor, or two where the rolled row crosses the longitude seam, each a multiple of 8 long.
-// A tensor is described as [tokens, heads * d] with boxes of 32 columns (one 64-byte-swizzled part of a row) by 32,
-// 16 or 8 tokens; a run is covered by boxes of 32 and at most one box of each smaller size.
+// A tensor is described as [tokens, heads * d] with boxes of 32 columns (one 64-byte-swizzled part of a row) by 128,
+// 64, 32, 16 or 8 tokens; a run is covered by the largest boxes that fit (the copy engine's time per box grows far
+// slower than the box: 2 KB boxes reach a third of the bytes per clock of 8 KB boxes).
 #pragma once
 #include <cuda.h>
 
@@ -13,7 +14,7 @@
 namespace terra {
 
 struct RowMaps3 {
-    CUtensorMap m[3];     // boxes of 32, 16, 8 tokens
+    CUtensorMap m[5];     // boxes of 32, 16, 8 tokens; 64 and 128 tokens (window sides 64 and 128 only)
 };
 
 // host: the three maps of one tensor (`token_stride` in elements); false if the driver's encoder is not available
@@ -44,6 +45,10 @@ __device__ __forceinline__ void bulk_copy_window_run(const RowMaps3& m3, uint32_
     int y = y0 + vs, n = n1;
 #pragma unroll
     for (int seg = 0; seg < 2; ++seg) {
+        if (g.w >= 64) {
+            while (n >= 128) { tc::tma_load_2d(dst, &m3.m[4], xc, y, bar); dst += 128 * 64; y += 128; n -= 128; }
+            if (n >= 64) { tc::tma_load_2d(dst, &m3.m[3], xc, y, bar); dst += 64 * 64; y += 64; n -= 64; }
+        }
         while (n >= 32) { tc::tma_load_2d(dst, &m3.m[0], xc, y, bar); dst += 32 * 64; y += 32; n -= 32; }
         if (n >= 16) { tc::tma_load_2d(dst, &m3.m[1], xc, y, bar); dst += 16 * 64; y += 16; n -= 16; }
         if (n >= 8) { tc::tma_load_2d(dst, &m3.m[2], xc, y, bar); dst += 8 * 64; }
