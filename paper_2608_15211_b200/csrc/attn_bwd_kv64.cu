@@ -363,7 +363,6 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
         // ------------------------------------------------------------------ loader warp (TMA); the other two have no work
         if (warp == kLoaderWarp0) {
             const int wrows = max(1, kTile / g.w);            // window rows per 128 slots
-            const int per_tensor = wrows * kParts;
             int kuse = 0;
             unsigned ru = 0;                                  // half chunks so far (every role counts them the same way)
             bool ok = true;
@@ -392,11 +391,21 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                         reinterpret_cast<int*>(st + kOffKTok)[row] = tok;
                     }
                     const uint32_t sb = smem0 + ks * kKvStageBytes;
-                    for (int i = lane; i < 2 * per_tensor; i += 32) {
-                        const int tsr = i >= per_tensor ? 1 : 0, rem = i - tsr * per_tensor;
-                        const int ar = rem / kParts, part = rem - ar * kParts;
-                        bulk_copy_window_row(tsr ? maps.v : maps.k, sb + (tsr ? kOffV : kOffK) + part * kPart + ar * g.w * kPartBytes, g,
-                                             x.b, x.r.wr, v0, x.kt * wrows + ar, head * D + part * 32, bar_kvfull(ks));
+                    if (!ROWS && g.w == 32) {
+                        // one lane per tensor and part: the tile's four window rows, in groups where the copies allow it
+                        for (int i = lane; i < 2 * kParts; i += 32) {
+                            const int tsr = i >= kParts ? 1 : 0, part = i - tsr * kParts;
+                            bulk_copy_window_rows(tsr ? maps.v : maps.k, sb + (tsr ? kOffV : kOffK) + part * kPart, g, x.b, x.r.wr, v0,
+                                                  x.kt * wrows, wrows, head * D + part * 32, bar_kvfull(ks));
+                        }
+                    } else {
+                        const int per_tensor = wrows * kParts;
+                        for (int i = lane; i < 2 * per_tensor; i += 32) {
+                            const int tsr = i >= per_tensor ? 1 : 0, rem = i - tsr * per_tensor;
+                            const int ar = rem / kParts, part = rem - ar * kParts;
+                            bulk_copy_window_row(tsr ? maps.v : maps.k, sb + (tsr ? kOffV : kOffK) + part * kPart + ar * g.w * kPartBytes, g,
+                                                 x.b, x.r.wr, v0, x.kt * wrows + ar, head * D + part * 32, bar_kvfull(ks));
+                        }
                     }
                     __syncwarp();
                     if (lane == 0) mbar_arrive_expect_tx(bar_kvfull(ks), (uint32_t)(kTile * D * 2 * 2));
@@ -425,12 +434,21 @@ swin_bwd_kv64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                         reinterpret_cast<int*>(sl + kOffQCode)[row] = 4 * code;
                         reinterpret_cast<int*>(sl + kOffQLab)[row] = label;
                     }
-                    for (int j = lane; j < 2 * runs * kParts; j += 32) {
-                        const int tsr = j >= runs * kParts ? 1 : 0, rem = j - tsr * runs * kParts;
-                        const int rr = rem / kParts, part = rem - rr * kParts;
-                        const int rslot = slot0 + rr * n_run, a = rslot / g.w;
-                        bulk_copy_window_run(tsr ? maps.g : maps.q, sb + (tsr ? kOffG : kOffQ) + part * kSPart + rr * n_run * kPartBytes, g,
-                                             x.b, x.r.wr, v0, a, rslot - a * g.w, n_run, head * D + part * 32, bar_qfull(s));
+                    if (!ROWS && g.w == 32) {
+                        // whole window rows: one lane per tensor and part, groups of window rows where the copies allow it
+                        for (int j = lane; j < 2 * kParts; j += 32) {
+                            const int tsr = j >= kParts ? 1 : 0, part = j - tsr * kParts;
+                            bulk_copy_window_rows(tsr ? maps.g : maps.q, sb + (tsr ? kOffG : kOffQ) + part * kSPart, g, x.b, x.r.wr, v0,
+                                                  slot0 / 32, runs, head * D + part * 32, bar_qfull(s));
+                        }
+                    } else {
+                        for (int j = lane; j < 2 * runs * kParts; j += 32) {
+                            const int tsr = j >= runs * kParts ? 1 : 0, rem = j - tsr * runs * kParts;
+                            const int rr = rem / kParts, part = rem - rr * kParts;
+                            const int rslot = slot0 + rr * n_run, a = rslot / g.w;
+                            bulk_copy_window_run(tsr ? maps.g : maps.q, sb + (tsr ? kOffG : kOffQ) + part * kSPart + rr * n_run * kPartBytes, g,
+                                                 x.b, x.r.wr, v0, a, rslot - a * g.w, n_run, head * D + part * 32, bar_qfull(s));
+                        }
                     }
                     if (ROWS && lane == 0) {
                         // the table rows that this slot's ur window rows need against the key tile's kr window rows

@@ -358,12 +358,11 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
                     }
                     int v0 = cur.wc * kW + g.sw;
                     if (v0 >= g.W) v0 -= g.W;
-                    constexpr int kPerTensor = (kTile / kW) * kParts;
-                    for (int i = lane; i < 2 * kPerTensor; i += 32) {
-                        const int tsr = i >= kPerTensor ? 1 : 0, rem = i - tsr * kPerTensor;
-                        const int ar = rem / kParts, part = rem - ar * kParts;
-                        bulk_copy_window_row(tsr ? maps.g : maps.q, sb + (tsr ? kOffG : kOffQ) + part * kPart + ar * kW * kPartBytes, g,
-                                             cur.b, cur.wr, v0, cur.qt * (kTile / kW) + ar, head * D + part * 32, bar_qfull(qs));
+                    // (one lane per tensor and part: the tile's four window rows, as one copy where the grid allows it)
+                    for (int i = lane; i < 2 * kParts; i += 32) {
+                        const int tsr = i >= kParts ? 1 : 0, part = i - tsr * kParts;
+                        bulk_copy_window_rows(tsr ? maps.g : maps.q, sb + (tsr ? kOffG : kOffQ) + part * kPart, g, cur.b, cur.wr, v0,
+                                              cur.qt * (kTile / kW), kTile / kW, head * D + part * 32, bar_qfull(qs));
                     }
                     if (lane == 0) mbar_expect_tx(bar_qfull(qs), (uint32_t)(kTile * D * 2 * 2));
                     // the lane's arrival: when its lse / delta copies have landed (its table entries were written before)

@@ -931,9 +931,23 @@ bool make_col_map(CUtensorMap* map, const Geo& g, const void* base, int token_st
 bool make_row_maps3(RowMaps3* maps, const Geo& g, const void* base, int token_stride) {
     for (int i = 0; i < 3; ++i)
         if (!make_row_map(&maps->m[i], g, base, token_stride, 32 >> i)) return false;
-    // the large boxes serve window sides 64 and 128 only; a box may not be longer than the token axis
+    // window sides 64 and 128: boxes of 64 and 128 tokens (a box may not be longer than the token axis); window side 32
+    // on grids of complete windows: boxes of 2 and 4 token rows x 32 token columns of the tensor as a 3-D array
     for (int i = 3; i < 5; ++i) {
         const long long tokens = (long long)g.B * g.H * g.W;
+        if (g.w == 32 && g.H % 32 == 0 && g.W % 32 == 0) {
+            EncodeTiledFn enc = encode_tiled_fn();
+            if (!enc) return false;
+            const cuuint64_t dims[3] = {(cuuint64_t)g.heads * g.d, (cuuint64_t)g.W, (cuuint64_t)g.B * g.H};
+            const cuuint64_t strides[2] = {(cuuint64_t)token_stride * 2, (cuuint64_t)g.W * token_stride * 2};
+            const cuuint32_t box[3] = {32u, 32u, i == 3 ? 2u : 4u};
+            const cuuint32_t estr[3] = {1u, 1u, 1u};
+            if (enc(&maps->m[i], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+                return false;
+            continue;
+        }
         const int box = (g.w >= 64 && tokens >= (8 << i)) ? (8 << i) : 32;           // m[3]: 64 tokens, m[4]: 128 tokens
         if (!make_row_map(&maps->m[i], g, base, token_stride, box)) return false;
     }

@@ -14,7 +14,10 @@
 namespace terra {
 
 struct RowMaps3 {
-    CUtensorMap m[5];     // boxes of 32, 16, 8 tokens; 64 and 128 tokens (window sides 64 and 128 only)
+    // boxes of 32, 16, 8 tokens; then, at window sides 64 and 128, boxes of 64 and 128 tokens, and at window side 32 the
+    // tensor as [token rows, token columns, heads * d] with boxes of 2 and 4 token rows x 32 token columns (2 and 4
+    // window rows of a window in one copy)
+    CUtensorMap m[5];
 };
 
 // host: the three maps of one tensor (`token_stride` in elements); false if the driver's encoder is not available
@@ -57,6 +60,29 @@ __device__ __forceinline__ void bulk_copy_window_run(const RowMaps3& m3, uint32_
     }
 }
 // the whole window row
+__device__ __forceinline__ void bulk_copy_window_row(const RowMaps3& m3, uint32_t dst, const Geo& g, int b, int wr, int v0, int a,
+                                                     int xc, uint32_t bar);
+// `nrows` consecutive window rows a0, a0 + 1, .. into consecutive slots.  In a 32-wide window whose rows do not cross
+// the longitude seam, groups of 4 or 2 window rows that do not cross the latitude wrap travel as one copy each.
+__device__ __forceinline__ void bulk_copy_window_rows(const RowMaps3& m3, uint32_t dst, const Geo& g, int b, int wr, int v0, int a0,
+                                                      int nrows, int xc, uint32_t bar) {
+    const bool groups = g.w == 32 && v0 + 32 <= g.W;
+    int a = a0;
+    while (nrows > 0) {
+        int u = wr * g.w + a + g.sh;
+        if (u >= g.H) u -= g.H;
+        if (groups && nrows >= 4 && u + 4 <= g.H) {
+            tc::tma_load_3d(dst, &m3.m[4], xc, v0, b * g.H + u, bar);
+            dst += 4 * 32 * 64; a += 4; nrows -= 4;
+        } else if (groups && nrows >= 2 && u + 2 <= g.H) {
+            tc::tma_load_3d(dst, &m3.m[3], xc, v0, b * g.H + u, bar);
+            dst += 2 * 32 * 64; a += 2; nrows -= 2;
+        } else {
+            bulk_copy_window_row(m3, dst, g, b, wr, v0, a, xc, bar);
+            dst += g.w * 64; ++a; --nrows;
+        }
+    }
+}
 __device__ __forceinline__ void bulk_copy_window_row(const RowMaps3& m3, uint32_t dst, const Geo& g, int b, int wr, int v0, int a,
                                                      int xc, uint32_t bar) {
     bulk_copy_window_run(m3, dst, g, b, wr, v0, a, 0, g.w, xc, bar);
