@@ -218,6 +218,8 @@ __device__ __forceinline__ void cols16(const uint32_t (&rs)[16], const uint32_t 
 struct QMaps64 {
     RowMaps3 q, g;            // query rows and their output gradients, by window rows
     CUtensorMap k;            // K rows by runs of 16 vertically adjacent tokens
+    CUtensorMap k4;           // ... four such runs (4 adjacent token columns) in one copy, if the encoder took the axis order
+    int k4_ok;
 };
 
 // TMA: both shifts are multiples of 16 (8 suffices for the longitude): one loader warp fetches the query rows window
@@ -328,7 +330,15 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
                     slot_token(g, cw, chunk_slot(c, 64 * h + r), code, label);
                     reinterpret_cast<int*>(smem + kOffKLab + uk * 256)[r] = label;
                 }
-                if (lane < 4 * kParts) tma_load_3d(smem0 + kOffKRing + uk * kUnitBytes + uoff, &maps.k, head * D + part * 32, vcol, z, bar_kfull(uk));
+                int vcol0 = cw.wc * kW + 4 * c + g.sw;
+                if (vcol0 >= g.W) vcol0 -= g.W;
+                if (maps.k4_ok && vcol0 + 4 <= g.W) {
+                    // the unit's four token columns do not cross the longitude seam: one copy per part
+                    if (lane < kParts)
+                        tma_load_3d(smem0 + kOffKRing + uk * kUnitBytes + lane * kUPart, &maps.k4, head * D + lane * 32, z, vcol0, bar_kfull(uk));
+                } else if (lane < 4 * kParts) {
+                    tma_load_3d(smem0 + kOffKRing + uk * kUnitBytes + uoff, &maps.k, head * D + part * 32, vcol, z, bar_kfull(uk));
+                }
                 if (lane == 0) mbar_arrive_expect_tx(bar_kfull(uk), (uint32_t)(64 * D * 2));
                 else mbar_arrive(bar_kfull(uk));
                 ++ru;
@@ -745,6 +755,8 @@ cudaError_t launch_bwd_q64(const Geo& g, const void* q, const void* k, const voi
     // (at head dim 64 the runs of 16 tokens are 1 KB copies, and the three gathering warps are faster)
     const bool tma = !tma_off && g.d == 128 && bulk_rows_shape(g) && g.sh % 16 == 0 && make_row_maps3(&maps.q, g, q, g.ts) &&
                      make_row_maps3(&maps.g, g, d_o, g.heads * g.d) && make_col_map(&maps.k, g, k, g.ts);
+    static const bool k4_off = [] { const char* e_ = std::getenv("TERRA_NO_K4"); return e_ && e_[0] == '1'; }();
+    maps.k4_ok = (tma && !k4_off && make_col_map4(&maps.k4, g, k, g.ts)) ? 1 : 0;
     auto kern = g.d == 64 ? swin_bwd_q64_kernel<64, false> : (tma ? swin_bwd_q64_kernel<128, true> : swin_bwd_q64_kernel<128, false>);
     const int smem_bytes = g.d == 64 ? Lay<64>::kSmemBytes : Lay<128>::kSmemBytes;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);

@@ -928,6 +928,17 @@ bool make_col_map(CUtensorMap* map, const Geo& g, const void* base, int token_st
                CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+bool make_col_map4(CUtensorMap* map, const Geo& g, const void* base, int token_stride) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc || g.W < 4 || g.H < 16) return false;
+    const cuuint64_t dims[3] = {(cuuint64_t)g.heads * g.d, (cuuint64_t)g.B * g.H, (cuuint64_t)g.W};
+    const cuuint64_t strides[2] = {(cuuint64_t)g.W * token_stride * 2, (cuuint64_t)token_stride * 2};
+    const cuuint32_t box[3] = {32u, 16u, 4u};
+    const cuuint32_t estr[3] = {1u, 1u, 1u};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 bool make_row_maps3(RowMaps3* maps, const Geo& g, const void* base, int token_stride) {
     for (int i = 0; i < 3; ++i)
         if (!make_row_map(&maps->m[i], g, base, token_stride, 32 >> i)) return false;

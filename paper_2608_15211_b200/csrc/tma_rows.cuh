@@ -26,6 +26,10 @@ bool make_row_maps3(RowMaps3* maps, const Geo& g, const void* base, int token_st
 // host: one tensor as [token rows, token columns, heads * d] with boxes of 32 columns x 1 token column x 16 token
 // rows: 16 vertically adjacent tokens of one head become 16 consecutive 64-byte rows of a swizzled region
 bool make_col_map(CUtensorMap* map, const Geo& g, const void* base, int token_stride);
+// host: the same tensor with the token-row axis BEFORE the token-column axis ([token columns, token rows, heads * d]) and
+// boxes of 32 columns x 16 token rows x 4 token columns: four runs of 16 vertically adjacent tokens in one copy.
+// false if the encoder refuses the axis order (the callers then keep to make_col_map's boxes).
+bool make_col_map4(CUtensorMap* map, const Geo& g, const void* base, int token_stride);
 
 // host: the geometry the bulk-copy loaders are written for
 inline bool bulk_rows_shape(const Geo& g) {
