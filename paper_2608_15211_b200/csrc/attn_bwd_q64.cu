@@ -218,7 +218,7 @@ __device__ __forceinline__ void cols16(const uint32_t (&rs)[16], const uint32_t 
 struct QMaps64 {
     RowMaps3 q, g;            // query rows and their output gradients, by window rows
     CUtensorMap k;            // K rows by runs of 16 vertically adjacent tokens
-    CUtensorMap k4;           // ... four such runs (4 adjacent token columns) in one copy, if the encoder took the axis order
+    CUtensorMap k4, v4;       // ... four such runs (4 adjacent token columns) of K / V in one copy, if the encoder took the axis order
     int k4_ok;
 };
 
@@ -399,10 +399,21 @@ swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv
                     const int uv = (int)(ru % kVUnits);
                     ok = mbar_wait_all(bar_vempty(uv), (uint32_t)((ru / kVUnits) & 1) ^ 1u, cta_abort);
                     if (!ok) break;
+                    const uint32_t vb = smem0 + kOffVRing + uv * kUnitBytes;
+                    int vcol0 = cur.wc * kW + 4 * (n >> 1) + g.sw;
+                    if (vcol0 >= g.W) vcol0 -= g.W;
+                    if (maps.k4_ok && vcol0 + 4 <= g.W) {
+                        // the unit's four token columns do not cross the longitude seam: one bulk copy per part
+                        int u0 = cur.wr * kW + 16 * (n & 1) + g.sh;
+                        if (u0 >= g.H) u0 -= g.H;
+                        if (r < kParts) tma_load_3d(vb + r * kUPart, &maps.v4, head * D + r * 32, cur.b * g.H + u0, vcol0, bar_vfull(uv));
+                        if (r == 0) mbar_arrive_expect_tx(bar_vfull(uv), (uint32_t)(64 * D * 2));
+                        else mbar_arrive(bar_vfull(uv));
+                        continue;
+                    }
                     int code, label;
                     const int tok = slot_token(g, cur, chunk_slot(n >> 1, 64 * (n & 1) + r), code, label);
                     const __nv_bfloat16* src = v + (sample_off + (size_t)tok) * g.ts + head * D;
-                    const uint32_t vb = smem0 + kOffVRing + uv * kUnitBytes;
 #pragma unroll
                     for (int piece = 0; piece < D / 8; ++piece)
                         cp_async16(vb + (piece >> 2) * kUPart + tile_off<32>(r, piece & 3), src + piece * 8, 16);
@@ -756,7 +767,7 @@ cudaError_t launch_bwd_q64(const Geo& g, const void* q, const void* k, const voi
     const bool tma = !tma_off && g.d == 128 && bulk_rows_shape(g) && g.sh % 16 == 0 && make_row_maps3(&maps.q, g, q, g.ts) &&
                      make_row_maps3(&maps.g, g, d_o, g.heads * g.d) && make_col_map(&maps.k, g, k, g.ts);
     static const bool k4_off = [] { const char* e_ = std::getenv("TERRA_NO_K4"); return e_ && e_[0] == '1'; }();
-    maps.k4_ok = (tma && !k4_off && make_col_map4(&maps.k4, g, k, g.ts)) ? 1 : 0;
+    maps.k4_ok = (tma && !k4_off && make_col_map4(&maps.k4, g, k, g.ts) && make_col_map4(&maps.v4, g, v, g.ts)) ? 1 : 0;
     auto kern = g.d == 64 ? swin_bwd_q64_kernel<64, false> : (tma ? swin_bwd_q64_kernel<128, true> : swin_bwd_q64_kernel<128, false>);
     const int smem_bytes = g.d == 64 ? Lay<64>::kSmemBytes : Lay<128>::kSmemBytes;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
