@@ -362,7 +362,8 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
         }
         for (int s = 0; s < kSlots; ++s) {
             mbar_init(bar_kfull(s), TMA ? 32 : kLoaderThreads);       // TMA: the bulk-copy warp's lanes
-            mbar_init(bar_vfull(s), ROWS ? 32 : TMA ? 64 : kLoaderThreads);       // TMA: the 64 threads that gather V rows (MODE 2: one warp's lanes)
+            // TMA: the 64 threads that gather V rows; MODE 2 and 32-wide windows: the lanes of the warp that bulk-copies them
+            mbar_init(bar_vfull(s), (ROWS || (TMA && g.w == 32)) ? 32 : TMA ? 64 : kLoaderThreads);
             mbar_init(bar_kempty(s), 1);
             mbar_init(bar_vempty(s), 1);
         }
@@ -505,8 +506,8 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                 }
                 ++kuse;
             }
-        } else if (ROWS) {
-            // ---- MODE 2, warp 10: the V rows by bulk copies as well (a window row is one or two boxes of 64 or 128 tokens,
+        } else if (ROWS || g.w == 32) {
+            // ---- MODE 2 and 32-wide windows, warp 10: the V rows by bulk copies as well (a window row is one or two boxes of 64 or 128 tokens,
             // which the copy engine moves at several times the rate of 32-token boxes); warp 11 has no work
             if (warp == kLoaderWarp0 + 1) {
                 const int wrows = kChunk / g.w;
@@ -523,11 +524,10 @@ swin_fwd_tc64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __n
                         ok = mbar_wait_all(bar_vempty(s), (uint32_t)((ru / kSlots) & 1) ^ 1u, cta_abort);
                         if (!ok) break;
                         const uint32_t sb = smem0 + kOffSlots + s * kSlotBytes;
-                        for (int i = lane; i < wrows * kParts; i += 32) {
-                            const int ar = i / kParts, part = i - ar * kParts;
-                            bulk_copy_window_row(maps.v, sb + kOffV + part * kKPart + ar * g.w * kPartBytes, g, x.b, x.r.wr, v0, c * wrows + ar,
-                                                 head * D + part * 32, bar_vfull(s));
-                        }
+                        // (one lane per part: the chunk's window rows, in groups of 4 where a 32-wide window allows it)
+                        if (lane < kParts)
+                            bulk_copy_window_rows(maps.v, sb + kOffV + lane * kKPart, g, x.b, x.r.wr, v0, c * wrows, wrows, head * D + lane * 32,
+                                                  bar_vfull(s));
                         __syncwarp();
                         if (lane == 0) mbar_arrive_expect_tx(bar_vfull(s), (uint32_t)(kChunk * D * 2));
                         else mbar_arrive(bar_vfull(s));
