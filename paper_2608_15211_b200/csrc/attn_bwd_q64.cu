@@ -222,10 +222,12 @@ struct QMaps64 {
     int k4_ok;
 };
 
-// TMA: both shifts are multiples of 16 (8 suffices for the longitude): one loader warp fetches the query rows window
-// row by window row and the K units as four runs of 16 vertically adjacent tokens with tiled bulk copies (per-query
-// lse and delta by 4-byte cp.async copies tied to the same barrier), the other two gather the V units with 16-byte
-// cp.async copies; otherwise all three gather every row.
+// TMA: both shifts are multiples of 16 (8 suffices for the longitude): one loader warp fetches the query rows (four
+// window rows per copy where the grid allows it) and the K units with tiled bulk copies (per-query lse and delta by
+// 4-byte cp.async copies tied to the same barrier), the other two fetch the V units.  A unit is four runs of 16
+// vertically adjacent tokens: one 4 KB copy per 32-column part where its four token columns do not cross the longitude
+// seam (a tensor map with the token-row axis before the token-column axis), else four 1 KB copies (K) or 16-byte
+// cp.async copies (V).  Otherwise all three warps gather every row.
 template <int D, bool TMA>
 __global__ void __launch_bounds__(kThreads, 1)
 swin_bwd_q64_kernel(const Geo g, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,

@@ -15,8 +15,9 @@
 //   columns left for them and the softmax threads add the row sums themselves).
 // Roles: warps 0-3 / 4-7 softmax warpgroups (one thread per query row of the pair's first / second tile),
 // warp 8 issues every tcgen05.mma (whole warp runs the loop, one elected lane issues), warps 9-11 load rows, undoing
-// the roll: on grids of complete windows warp 9 fetches Q and K rows with tiled bulk copies and warps 10-11 gather V
-// rows with cp.async; otherwise all three gather with cp.async.  A row is kept as head dim / 32 parts of 32 columns in
+// the roll: on grids of complete windows warp 9 fetches Q and K rows with tiled bulk copies, and the V rows come from
+// warp 10 by bulk copies of large boxes (window sides 32, 64, 128: four window rows, or one, per copy) or are gathered
+// by warps 10-11 with cp.async (window side 16); otherwise all three gather with cp.async.  A row is kept as head dim / 32 parts of 32 columns in
 // the 64-byte-swizzled operand layout of the small-window kernels, so that the same descriptors serve.
 // TMEM: columns [256 t, 256 t + 256) belong to query tile t of the pair: S chunk (fp32, 128 columns), overwritten
 // in place by bf16 P (64 columns); the O accumulator at +128.
