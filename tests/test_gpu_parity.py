@@ -32,6 +32,10 @@ EDGE = [
     ("bulk64_w32", 1, 64, 96, 2, 64, 32, 16, 8, 0, 1),           # head dim 64, complete windows: rows by tiled bulk copies
     ("bulk64_w16", 2, 32, 48, 2, 64, 16, 8, 8, 0, 0),
     ("gather64_w32", 1, 64, 64, 2, 64, 32, 12, 20, 0, 0),        # complete windows, shifts not multiples of 8: rows gathered
+    # 32-wide complete windows whose latitude shift is no multiple of 4: groups of window rows that would cross the
+    # latitude wrap fall back to one bulk copy per window row; the last window column crosses the longitude seam
+    ("bulk64_w32_odd_shift", 1, 64, 64, 2, 64, 32, 5, 24, 0, 1),
+    ("bulk128_w32_odd_shift", 1, 64, 96, 1, 128, 32, 13, 8, 1, 1),
     ("tma_noshift", 1, 32, 40, 2, 32, 16, 0, 0, 0, 1),
 ]
 
